@@ -1,0 +1,386 @@
+#!/usr/bin/env python
+"""Benchmark of the HORA rollout-allocation hot path on B200.
+
+One step = one pass of the whole path over one synthetic batch:
+    hora_gains -> hora_allocate -> hora_group_advantage      on workload cfg4 (N = 2^20 prompts, G0 = 8,
+                                                              ld = 256, B = 24 N, per-prompt real priors, GRPO)
+    hora_token_broadcast                                      of the first 262144 rollout advantages of that
+                                                              batch over response lengths ~ U{32..2048}
+                                                              (the cfg3 token layout, ~2.7e8 tokens)
+`value` is prompts per second over the whole step with every input resident in HBM; `e2e` is the same
+metric with the step's inputs copied from pinned host memory and its results copied back inside the
+timed region.  With --gpus N every rank runs its own independent batch (the paper allocates in
+independent shards), no data-path collective, weak scaling.
+
+`--impl reference` times the CPU oracle (a deliberately plain program) on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "hora_alloc_advantage_prompts_per_s"
+UNIT = "prompts/s"
+WORKLOAD = "cfg4"
+BCAST_ROLLOUTS = 262144
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised
+# under profiles/; None = no capture of the kernel as it stands.
+TRAFFIC_BYTES = {"gains_kernel": None}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.005):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+            nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def shard_seed(rank: int) -> int:
+    """Every rank draws its own independent batch; rank 0 uses the workload's published seed."""
+    return 3 + rank
+
+
+# --------------------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2605_07114_b200 import hora, workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    hora.load()
+
+    w = wl.make(WORKLOAD, args.prompts, seed=shard_seed(rank))
+    N, ld, G0, B = w.N, w.ld, w.G0, w.B
+    h_alpha = torch.from_numpy(w.alpha).pin_memory()
+    h_beta = torch.from_numpy(w.beta).pin_memory()
+    h_c = torch.from_numpy(w.c).pin_memory()
+    alpha, beta, c = h_alpha.to(dev), h_beta.to(dev), h_c.to(dev)
+    cap_scalar = ld
+    al = hora.Allocator(N, ld, G0, exact_int=False, device=dev)
+
+    # one untimed pass fixes the group layout, from which the synthetic rewards are drawn
+    al.run(alpha, beta, 1.0, 1.0, c, None, cap_scalar, B)
+    info = al.read_info()
+    if info.status != 0:
+        raise RuntimeError(f"allocation failed: {hora.status_string(info.status)}")
+    off_h = al.group_offsets.cpu().numpy()
+    total = int(off_h[-1])
+    h_rewards = torch.from_numpy(w.rewards(off_h)).pin_memory()
+    rewards = h_rewards.to(dev)
+    adv = torch.empty(total, dtype=torch.float32, device=dev)
+    R = min(BCAST_ROLLOUTS, total)
+    tok_h = w.token_offsets(R)
+    T = int(tok_h[-1])
+    tok = torch.from_numpy(tok_h).to(dev)
+    token_adv = torch.empty(T, dtype=torch.float32, device=dev)
+    h_delta = torch.empty(N, dtype=torch.int32).pin_memory()
+    h_G = torch.empty(N, dtype=torch.int32).pin_memory()
+    h_adv = torch.empty(total, dtype=torch.float32).pin_memory()
+    eps = float(w.eps)
+
+    def step(events=None):
+        if events is not None:
+            events[0].record()
+        hora.hora_gains(alpha, beta, 1.0, 1.0, c, G0, None, cap_scalar, N, ld, al.gains)
+        if events is not None:
+            events[1].record()
+        hora.hora_allocate(alpha, beta, 1.0, 1.0, c, G0, None, cap_scalar, N, ld, al.gains, B, al.flags, al.delta,
+                           al.G, al.group_offsets, al.info, al.workspace)
+        if events is not None:
+            events[2].record()
+        hora.hora_group_advantage(rewards, al.group_offsets, N, w.adv_mode, eps, w.ddof, adv)
+        if events is not None:
+            events[3].record()
+        hora.hora_token_broadcast(adv, tok, R, T, token_adv)
+        if events is not None:
+            events[4].record()
+
+    def step_e2e():
+        alpha.copy_(h_alpha, non_blocking=True)
+        beta.copy_(h_beta, non_blocking=True)
+        c.copy_(h_c, non_blocking=True)
+        rewards.copy_(h_rewards, non_blocking=True)
+        step()
+        h_delta.copy_(al.delta, non_blocking=True)
+        h_G.copy_(al.G, non_blocking=True)
+        h_adv.copy_(adv, non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
+        step()
+    barrier()
+
+    # ---- timed region: device-resident inputs ----
+    stage_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    launches0 = hora.hora_launch_count()
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    barrier()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for k in range(args.steps):
+        step(stage_ev[k])
+    t1.record()
+    barrier()
+    clocks = sampler.stop()
+    launches = hora.hora_launch_count() - launches0
+    ms_total = max_over_ranks(t0.elapsed_time(t1))
+    ms_step = ms_total / args.steps
+    stages = np.array([[ev[i].elapsed_time(ev[i + 1]) for i in range(4)] for ev in stage_ev])
+    st_mean = stages.mean(axis=0)
+    st_min = stages.min(axis=0)
+
+    info = al.read_info()
+    if info.status != 0 or info.sum_G != total:
+        raise RuntimeError("allocation changed during the timed loop")
+
+    # ---- end to end: pinned host inputs in, results out, every step ----
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        step_e2e()
+    barrier()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        step_e2e()
+    e1.record()
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+    h2d = h_alpha.numel() * 8 + h_beta.numel() * 8 + h_c.numel() * 4 + h_rewards.numel() * 4
+    d2h = h_delta.numel() * 4 + h_G.numel() * 4 + h_adv.numel() * 4
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    cand = N * ld
+    bytes_gains = cand * 8 + N * 20
+    bytes_alloc = cand * 8 + N * (20 + 4 + 4 + 8)
+    bytes_adv = total * 8 + (N + 1) * 8
+    bytes_bc = T * 4 + R * 12
+    algo = [bytes_gains, bytes_alloc, bytes_adv, bytes_bc]
+    names = ["hora_gains", "hora_allocate", "hora_group_advantage", "hora_token_broadcast"]
+    stage_report = {}
+    for nm, by, ms, mn in zip(names, algo, st_mean, st_min):
+        gbs = by / (ms * 1e-3) / 1e9
+        stage_report[nm] = {"ms": round(float(ms), 4), "ms_min": round(float(mn), 4), "algorithmic_bytes": int(by),
+                            "gbs": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peak, 4)}
+    pipe_bytes = sum(algo[:3])
+    pipe_ms = float(st_mean[:3].sum())
+    g_ms = float(st_mean[0])                           # hora_gains is exactly one launch (gains_kernel)
+    achieved = bytes_gains / (g_ms * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": N * world / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{WORKLOAD}: N={N} prompts per GPU, G0={G0}, ld={ld}, B={B}, per-prompt real priors, "
+                               f"GRPO; then token broadcast of {R} rollouts to {T} tokens (lengths U{{32..2048}})",
+                   "l2": "inputs larger than L2 (the gains matrix alone is %.2f GB)" % (cand * 8 / 1e9),
+                   "shard": "one independent batch per GPU, no collective"},
+        "clocks": clocks,
+        "e2e": {"value": N * world / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "gains_kernel (the one launch of hora_gains)",
+                     "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": round(achieved / peak, 4), "traffic": TRAFFIC_BYTES.get("gains_kernel"),
+                     "algorithmic_bytes_per_launch": int(bytes_gains), "ms_per_launch": round(g_ms, 4)},
+        "pipeline": {"calls": "hora_gains+hora_allocate+hora_group_advantage", "ms": round(pipe_ms, 4),
+                     "algorithmic_bytes": int(pipe_bytes), "gbs": round(pipe_bytes / (pipe_ms * 1e-3) / 1e9, 1),
+                     "frac_of_hbm_peak": round(pipe_bytes / (pipe_ms * 1e-3) / 1e9 / peak, 4),
+                     "prompts_per_s": N / (pipe_ms * 1e-3), "candidate_gains_per_s": cand / (pipe_ms * 1e-3)},
+        "tokens_per_s": T / (float(st_mean[3]) * 1e-3),
+        "stages": stage_report,
+        "allocation": {"lambda": info.lambda_, "n_above": info.n_above, "n_tied": info.n_tied,
+                       "objective": info.objective},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(w, args.cpu_sample)
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------- oracle timing
+def oracle_step(w, n):
+    """The oracle, as it stands, on the first n prompts of the workload (budget scaled with n).
+    Returns the seconds spent inside oracle calls (input generation excluded)."""
+    from oracle import hora_oracle as orc
+    sl = slice(0, n)
+    alpha, beta, c, cap = w.alpha[sl], w.beta[sl], w.c[sl], w.cap[sl]
+    B = (w.B // w.N) * n
+    t0 = time.perf_counter()
+    orc.gains(alpha, beta, w.alpha0, w.beta0, c, w.G0, cap, w.ld)
+    d, G, lam, obj = orc.greedy_real(alpha, beta, w.alpha0, w.beta0, c, w.G0, cap, B)
+    t1 = time.perf_counter()
+    off = np.zeros(n + 1, np.int64)
+    np.cumsum(G.astype(np.int64), out=off[1:])
+    sub = type(w)(**{**w.__dict__, "N": n, "p": w.p[sl], "c": c, "cap": cap, "alpha": alpha, "beta": beta, "B": B})
+    rewards = sub.rewards(off)
+    R = max(1, min(len(rewards), BCAST_ROLLOUTS * n // w.N))
+    tok = sub.token_offsets(R)
+    t2 = time.perf_counter()
+    adv = orc.group_advantage(rewards, off, w.adv_mode, float(np.float32(w.eps)), w.ddof)
+    orc.token_broadcast(adv[:R], tok)
+    t3 = time.perf_counter()
+    return (t1 - t0) + (t3 - t2)
+
+
+def cpu_baseline(w, n):
+    n = min(n, w.N)
+    secs = oracle_step(w, n)
+    return {"value": n / secs, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(secs, 2),
+            "sample": f"first {n} of {w.N} prompts of {WORKLOAD} (budget and token count scaled by the same factor), "
+                      "one pass: long-double gain rows, heap greedy, group advantages, token repeat"}
+
+
+def reference_sample_size(steps: int, warmup: int, N: int) -> int:
+    """Prompts per oracle step so that the whole run stays near 100 s of CPU work."""
+    budget_prompts = 5.0e6
+    n = int(budget_prompts / max(1, steps + warmup))
+    n = 1 << (max(n, 1).bit_length() - 1)
+    return max(1024, min(1 << 19, n, N))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2605_07114_b200 import workloads as wl
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    w = wl.make(WORKLOAD, args.prompts, seed=shard_seed(0))
+    steps, warm = args.steps, args.warmup
+    n = reference_sample_size(steps, warm, w.N)
+    for _ in range(warm):
+        oracle_step(w, n)
+    secs = [oracle_step(w, n) for _ in range(steps)]
+    ms = 1e3 * sum(secs) / steps
+    val = n / (ms * 1e-3)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f80", "data": "synthetic",
+        "config": {"workload": f"{WORKLOAD}: each step is the first {n} of {w.N} prompts (budget and tokens scaled), "
+                               "CPU oracle, one host thread"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"first {n} prompts of {WORKLOAD} per step"},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--prompts", type=int, default=None, help="override N (default: the workload's 2^20)")
+    ap.add_argument("--cpu-sample", type=int, default=1 << 19)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,174 @@
+/*
+ * hora.h — C ABI of the HORA rollout-allocation hot path for NVIDIA B200 (sm_100a).
+ *
+ * HORA ("Hit-Utility Optimal Rollout Allocation for Group-Based RLVR") splits the rollouts of a
+ * training batch in two phases.  Phase A draws G0 rollouts for each of N prompts and counts the
+ * correct ones, c_i.  With a Beta(alpha_i, beta_i) prior the posterior of the prompt's success
+ * rate is Beta(a_i, b_i), a_i = alpha_i + c_i, b_i = beta_i + G0 - c_i (Eq. posterior).  Phase B
+ * hands out B further rollouts so as to maximise sum_i U_i(Delta_i), where U_i(Delta) is the posterior
+ * probability that at least one of Delta more rollouts is correct (Eq. hit-utility, Eq.
+ * allocation-problem).  The marginal gains g_i(Delta) = U_i(Delta) - U_i(Delta-1) decrease in Delta, so the
+ * optimum is the set of the B largest gains over all (prompt, Delta) candidates (Proposition 1).
+ * Advantages are then computed over the variable-size groups G_i = G0 + Delta_i and replicated over
+ * the tokens of each rollout.
+ *
+ * This library covers exactly that path, four calls, in execution order:
+ *   hora_gains -> hora_allocate -> [rollouts and rewards happen elsewhere] ->
+ *   hora_group_advantage -> hora_token_broadcast
+ *
+ * Conventions for every call
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer on the current CUDA device.
+ *   - The caller owns every buffer.  The library allocates nothing; hora_allocate works in a
+ *     caller-provided workspace whose size hora_allocate_workspace_bytes returns.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls enqueue
+ *     work and return; they never synchronise the device.
+ *   - The return value reports what the host can see at enqueue time (bad sizes, null pointers,
+ *     a too-small workspace, a failed launch).  Errors that depend on device DATA (a non-finite
+ *     prior, B larger than the total cap, ...) are written to a status word in device memory; the
+ *     caller reads it after synchronising.  Nothing traps, spins or aborts.
+ *   - Results are deterministic: the same inputs give bitwise identical outputs on every run.
+ *   - Calls on different streams may run concurrently as long as they do not share output
+ *     buffers or workspaces.
+ */
+#ifndef HORA_H
+#define HORA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum hora_status {
+    HORA_OK = 0,
+    HORA_ERR_INVALID_ARG = 1,    /* host-visible: null pointer, negative size, ld < 1, unknown mode ... */
+    HORA_ERR_INVALID_VALUE = 2,  /* device data: prior not finite or <= 0, c outside [0,G0], cap outside [0,ld],
+                                    a gain row that is not finite/non-negative/non-increasing, offsets that decrease */
+    HORA_ERR_INFEASIBLE = 3,     /* B > sum_i cap_i */
+    HORA_ERR_NOT_INTEGER = 4,    /* HORA_FLAG_EXACT_INT given but some alpha_i or beta_i is not a positive integer */
+    HORA_ERR_EXACT_RANGE = 5,    /* exact path: parameters too large for 128-bit integers or too many tie types */
+    HORA_ERR_WORKSPACE = 6,      /* workspace missing, misaligned (needs 256 B) or too small */
+    HORA_ERR_CUDA = 7            /* a CUDA runtime call or kernel launch failed */
+} hora_status_t;
+
+enum {
+    HORA_FLAG_EXACT_INT = 1u,      /* priors are integer-valued: decide ties by exact rational equality */
+    HORA_FLAG_SKIP_OBJECTIVE = 2u  /* do not compute hora_alloc_info.objective (left 0) */
+};
+
+enum { HORA_ADV_GRPO = 0, HORA_ADV_RLOO = 1 };
+
+/* Summary of one allocation; lives in DEVICE memory (64 bytes, 8-byte aligned). */
+typedef struct hora_alloc_info {
+    int32_t status;        /* hora_status_t of the data-dependent checks */
+    int32_t reserved;
+    double  lambda;        /* gain of the B-th best candidate (the selection threshold); 0 when B == 0 */
+    int64_t n_above;       /* candidates strictly better than lambda (all taken) */
+    int64_t n_tied;        /* candidates equal to lambda */
+    int64_t n_tied_taken;  /* B - n_above: how many of the tied ones were taken, lowest prompt index first */
+    double  objective;     /* sum_i U_i(Delta_i) */
+    int64_t sum_G;         /* sum_i G_i = N*G0 + B */
+    int64_t sum_cap;       /* sum_i cap_i */
+} hora_alloc_info;
+
+/*
+ * hora_gains — marginal hit-utility rows (Eq. marginal and the recurrence stated after it).
+ *
+ *   gains[i*ld + (Delta-1)] = g_i(Delta) = M_i(Delta-1)
+ *                            = a_i/(a_i+b_i+Delta-1) * prod_{j<Delta-1} (b_i+j)/(a_i+b_i+j)     for 1 <= Delta <= cap_i
+ *                            = 0.0                                                              for cap_i < Delta <= ld
+ *
+ * computed in fp64 as a prefix product (one warp per row, warp scan); every entry is within
+ * 4*ld ulp of the exact value.  Rows are strictly decreasing up to cap_i.
+ *
+ *   alpha, beta   [N] fp64 per-prompt prior, or both NULL to use the shared prior (alpha0, beta0)
+ *   c             [N] int32 Phase-A success counts, 0 <= c_i <= G0
+ *   cap           [N] int32 per-prompt cap, 0 <= cap_i <= ld, or NULL to use cap_scalar for all
+ *   gains         [N*ld] fp64 out, row-major, 8-byte aligned (16-byte aligned enables vector stores)
+ *   status_dev    optional int32 in device memory: receives HORA_ERR_INVALID_VALUE if any row's inputs
+ *                 are invalid (that row is written as zeros); it is never cleared by this call
+ * Returns HORA_ERR_INVALID_ARG for N < 0, ld < 1, G0 < 0, missing pointers.  N == 0 is a no-op.
+ */
+hora_status_t hora_gains(const double *alpha, const double *beta, double alpha0, double beta0,
+                         const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar,
+                         int64_t N, int32_t ld, double *gains, int32_t *status_dev, void *stream);
+
+/*
+ * hora_allocate — budgeted optimal allocation (Eq. allocation-problem; Algorithm 1 Phase B; Proposition 1).
+ *
+ * Computes the result of B greedy steps "give one more rollout to the prompt with the largest
+ * current marginal gain" without running them one by one: because every row of gains decreases,
+ * that result is the set of the B largest candidates g_i(Delta), Delta <= cap_i.  The call finds the
+ * B-th largest value lambda by a multi-level radix selection on the 64-bit patterns of the gains
+ * (one full read of the matrix, then per-row segment refinement), counts per row the candidates
+ * above lambda, and gives the remaining B - n_above rollouts to the tied candidates in order of
+ * increasing prompt index (then increasing Delta).  Outputs:
+ *
+ *   delta[i]          = Delta_i, 0 <= Delta_i <= cap_i, sum = B                    int32 [N]
+ *   G[i]              = G0 + Delta_i                                              int32 [N]
+ *   group_offsets[i]  = sum_{j<i} G[j] (CSR offsets of the pooled groups)         int64 [N+1], may be NULL
+ *   info_dev          = summary (see hora_alloc_info)                             device, may be NULL
+ *
+ * Ties.  Without HORA_FLAG_EXACT_INT a tie is equality of the fp64 gains as hora_gains computes
+ * them.  With HORA_FLAG_EXACT_INT (every alpha_i, beta_i a positive integer) candidates within a
+ * relative band of 2^-30 around the fp64 threshold are re-ranked on exact integers
+ * (g = a*(b)_a / (b+Delta-1)_{a+1} compared by 256-bit cross multiplication), so a tie is an exact
+ * rational equality and the result equals exact greedy with lowest-index tie-breaking.
+ *
+ *   alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld   as for hora_gains
+ *   gains            [N*ld] the matrix hora_gains wrote for the same inputs, or NULL to have it built
+ *                    inside the workspace (the workspace must then be sized with gains_is_null = 1)
+ *   B                number of Phase-B rollouts, 0 <= B <= sum_i cap_i
+ *   workspace        device scratch, 256-byte aligned, at least hora_allocate_workspace_bytes(...);
+ *                    contents are undefined on entry and on exit
+ * Data-dependent failures (INVALID_VALUE, INFEASIBLE, NOT_INTEGER, EXACT_RANGE) set info_dev->status and
+ * leave delta, G and group_offsets all zero.
+ */
+size_t hora_allocate_workspace_bytes(int64_t N, int32_t ld, int32_t gains_is_null, uint32_t flags);
+
+hora_status_t hora_allocate(const double *alpha, const double *beta, double alpha0, double beta0,
+                            const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar,
+                            int64_t N, int32_t ld, const double *gains, int64_t B, uint32_t flags,
+                            int32_t *delta, int32_t *G, int64_t *group_offsets, hora_alloc_info *info_dev,
+                            void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * hora_group_advantage — group-relative advantages over ragged groups (Sec. 3.1 for GRPO; the RLOO
+ * compatibility paragraph of Sec. 4 for the leave-one-out form).
+ *
+ * Group g holds rewards[group_offsets[g] .. group_offsets[g+1]).  With S the group's sum and n its size:
+ *   HORA_ADV_GRPO:  adv_j = (r_j - S/n) / (sqrt(sum_k (r_k - S/n)^2 / (n - ddof)) + eps); 0 when that
+ *                   denominator is 0 (a zero-variance group gives no signal) or n - ddof <= 0
+ *   HORA_ADV_RLOO:  adv_j = r_j - (S - r_j)/(n - 1); 0 when n == 1
+ * Sums are accumulated in fp64 and rounded to fp32 once.  Empty groups are allowed.
+ *
+ *   rewards [total] fp32, group_offsets [N+1] int64 non-decreasing with group_offsets[0] == 0,
+ *   adv [total] fp32 out, ddof in {0,1}, eps >= 0, status_dev optional (INVALID_VALUE on decreasing offsets).
+ */
+hora_status_t hora_group_advantage(const float *rewards, const int64_t *group_offsets, int64_t N,
+                                   int32_t mode, float eps, int32_t ddof, float *adv,
+                                   int32_t *status_dev, void *stream);
+
+/*
+ * hora_token_broadcast — per-token advantages (Eq. grpo-objective: the advantage of a rollout does not
+ * depend on the token position).
+ *
+ *   token_adv[t] = adv[r]   for token_offsets[r] <= t < token_offsets[r+1],   r = 0..R-1
+ *
+ *   adv [R] fp32, token_offsets [R+1] int64 non-decreasing with token_offsets[0] == 0,
+ *   T = token_offsets[R] (the caller knows it: it sized token_adv), token_adv [T] fp32 out.
+ * Zero-length rollouts are allowed.  Tokens at or beyond token_offsets[R] are not written.
+ */
+hora_status_t hora_token_broadcast(const float *adv, const int64_t *token_offsets, int64_t R, int64_t T,
+                                   float *token_adv, void *stream);
+
+const char *hora_status_string(hora_status_t status);   /* host: static string */
+int         hora_version(void);                         /* host: major*10000 + minor*100 + patch */
+uint64_t    hora_launch_count(void);                    /* host: kernels this library has launched so far in this
+                                                           process (memsets not counted); for benchmarks' bookkeeping */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HORA_H */

@@ -1,0 +1,770 @@
+// hora_allocate: the B largest marginal gains over all (prompt, Delta) candidates, i.e. the result of
+// Algorithm 1's Phase-B greedy loop (Proposition 1), found by selection instead of B sequential steps.
+//
+// Keys.  A gain is a non-negative finite double, so its bit pattern orders like the value.  The 64-bit
+// key is resolved 13 bits at a time (shifts 51, 38, 25, 12, then the last 12 bits):
+//
+//   level 0   one coalesced read of the whole matrix (a warp per row), histogram of the top 13 bits
+//             in shared memory, merged into a global histogram; the last CTA to finish locates the
+//             digit that holds the B-th largest key.
+//   level 1   a thread per row: because a row is non-increasing, its keys with the selected top digit
+//             form ONE contiguous segment, found by binary search; only that segment is read again
+//             and its next digit histogrammed.  The segment [p_hi, p_lo) is kept per row.
+//   level 2-4 a thread per row narrows its segment by the digit just selected and histograms the next.
+//   sum       narrows by the last digit: p_hi = #keys > lambda, p_lo - p_hi = #keys == lambda; block sums
+//             and their scan give n_above, n_tied and the exclusive prefixes over prompts.
+//   out       Delta_i = p_hi + (tied candidates of row i that fall within the first R = B - n_above tied
+//             candidates in prompt order); G_i, CSR offsets, objective.
+//
+// No kernel waits on another CTA: every "last CTA" step uses an atomic ticket after a fence.
+//
+// Exact mode (integer priors).  After the fp64 selection, candidates within a relative band of 2^-30
+// around lambda (far wider than the fp64 evaluation error, far narrower than the gap between two
+// entries of one row) are the only ones whose exact rank is in doubt.  Each row has at most one.
+// Their types (a, b, Delta) are collected in a small hash table with instance counts, ranked exactly
+// by 256-bit cross multiplication of num/den = a (b)_a / (b+Delta-1)_{a+1}  (or the equivalent
+// a (b)_{Delta-1} / (a+b)_Delta when that has fewer factors), and the threshold class is found by
+// walking the ranked types.  Rows are relabelled above / tied / below and the same sum/out steps run.
+#include "hora_common.cuh"
+
+namespace hora {
+
+constexpr int kLevels = 5;
+constexpr int kBins = 8192;
+constexpr int kSelThreads = 256;
+constexpr int kRowsPerBlock = 1024;          // rows per CTA in the sum / out kernels (4 per thread)
+constexpr int kTypeSlots = 4096;             // hash slots for exact tie types
+constexpr int kMaxTypes = 1024;              // distinct types the exact ranking accepts
+constexpr unsigned long long kKeyInf = 0x7FF0000000000000ull;
+
+__host__ __device__ __forceinline__ int level_shift(int level) { return level == 4 ? 0 : 51 - 13 * level; }
+__host__ __device__ __forceinline__ int level_bins(int level) { return level == 4 ? 4096 : 8192; }
+
+struct AllocHeader {
+    int32_t status;
+    int32_t pad0;
+    unsigned int ticket[16];
+    unsigned long long sum_cap;
+    unsigned long long prefix_key;     // key bits resolved so far (the threshold once all levels ran)
+    long long need;                    // rank of the threshold inside the current bin (1-based)
+    int32_t sel_digit[8];
+    unsigned long long n_above, n_tied;
+    long long R;                       // tied candidates to take
+    double lambda;
+    double objective;
+    unsigned long long band_above;     // exact mode: candidates above the band
+    unsigned int n_types;
+    unsigned int pad1;
+};
+
+struct Workspace {
+    AllocHeader *hdr;
+    unsigned long long *hist;          // [kLevels][kBins]
+    int2 *rowstate;                    // [N] (p_hi, p_lo)
+    long long *bsum_hi, *bsum_t;       // [NB] block sums, overwritten by exclusive prefixes
+    double *objpart;                   // [NB]
+    unsigned long long *tkeys, *tcounts;   // [kTypeSlots]
+    int32_t *tlabel;                   // [kTypeSlots]
+    int32_t *rowslot;                  // [N]
+    double *gains;                     // [N*ld] when the caller passed none
+    size_t bytes;
+};
+
+static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+static Workspace carve(void *base, int64_t N, int32_t ld, bool need_gains, bool exact) {
+    Workspace w{};
+    size_t o = 0;
+    char *p = static_cast<char *>(base);
+    const int64_t NB = (N + kRowsPerBlock - 1) / kRowsPerBlock;
+    auto take = [&](size_t n) { char *q = p ? p + o : nullptr; o = align256(o + n); return q; };
+    w.hdr = reinterpret_cast<AllocHeader *>(take(sizeof(AllocHeader)));
+    w.hist = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kLevels * kBins));
+    w.rowstate = reinterpret_cast<int2 *>(take(sizeof(int2) * (size_t)N));
+    w.bsum_hi = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
+    w.bsum_t = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
+    w.objpart = reinterpret_cast<double *>(take(sizeof(double) * (size_t)NB));
+    if (exact) {
+        w.tkeys = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kTypeSlots));
+        w.tcounts = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kTypeSlots));
+        w.tlabel = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * kTypeSlots));
+        w.rowslot = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (size_t)N));
+    }
+    if (need_gains) w.gains = reinterpret_cast<double *>(take(sizeof(double) * (size_t)N * (size_t)ld));
+    w.bytes = o;
+    return w;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// "Last CTA" ticket: returns true in exactly one CTA, after every other CTA's global writes are visible.
+__device__ __forceinline__ bool last_block(unsigned int *ticket) {
+    __shared__ bool s_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (s_last) __threadfence();
+    return s_last;
+}
+
+// Block-wide exclusive sum over kSelThreads values (long long), also returns the total.
+__device__ __forceinline__ long long block_exclusive_sum(long long v, long long *total, long long *s_warp) {
+    const int lane = lane_id(), warp = threadIdx.x >> 5;
+    long long inc = v;
+#pragma unroll
+    for (int d = 1; d < kWarp; d <<= 1) {
+        const long long t = __shfl_up_sync(kFull, inc, d);
+        if (lane >= d) inc += t;
+    }
+    __syncthreads();
+    if (lane == kWarp - 1) s_warp[warp] = inc;
+    __syncthreads();
+    long long base = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < kSelThreads / kWarp; ++w) {
+        const long long x = s_warp[w];
+        if (w < warp) base += x;
+        tot += x;
+    }
+    *total = tot;
+    return base + inc - v;
+}
+
+// Run by ONE CTA: find the digit d with  count(digit > d) < need <= count(digit >= d)  in hist[0..bins).
+__device__ void find_digit(AllocHeader *hdr, const unsigned long long *hist, int level, long long *s_warp) {
+    const int bins = level_bins(level);
+    const int per = bins / kSelThreads;
+    const long long need = hdr->need;
+    const int top = bins - 1 - (int)threadIdx.x * per;      // this thread scans bins top, top-1, ..., top-per+1
+    long long local = 0;
+    for (int j = 0; j < per; ++j) local += (long long)__ldcg(hist + top - j);
+    long long total;
+    const long long above = block_exclusive_sum(local, &total, s_warp);
+    if (need >= 1 && above < need && need <= above + local) {
+        long long run = above;
+        for (int j = 0; j < per; ++j) {
+            const long long cnt = (long long)__ldcg(hist + top - j);
+            if (run + cnt >= need) {
+                hdr->sel_digit[level] = top - j;
+                hdr->need = need - run;
+                hdr->prefix_key |= (unsigned long long)(top - j) << level_shift(level);
+                break;
+            }
+            run += cnt;
+        }
+    }
+}
+
+__device__ __forceinline__ void flush_hist(const unsigned int *s_hist, unsigned long long *hist, int bins) {
+    for (int b = threadIdx.x; b < bins; b += kSelThreads) {
+        const unsigned int v = s_hist[b];
+        if (v) atomicAdd(hist + b, (unsigned long long)v);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Level 0: the one full read.  A warp per row, a lane takes E consecutive keys (the row is sorted, so a
+// lane's keys fall into few bins and are merged before they touch shared memory).  Also validates the
+// inputs and sums the caps.
+template <int E, bool VEC2>
+__global__ void __launch_bounds__(kSelThreads)
+select_level0(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
+              const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
+              int64_t N, int32_t ld, const double *__restrict__ gains, int64_t B, AllocHeader *hdr,
+              unsigned long long *hist) {
+    __shared__ unsigned int s_hist[kBins];
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
+    __syncthreads();
+    const int lane = lane_id();
+    const int64_t warp0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5);
+    const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
+    long long capsum = 0;
+    bool bad = false;
+    for (int64_t row = warp0; row < N; row += stride) {
+        const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row);
+        bad |= !p.ok;
+        if (lane == 0) capsum += p.cap;
+        const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+        unsigned long long prev_last = ~0ull;                  // last key of the previous lane / chunk
+        for (int32_t k0 = 0; k0 < p.cap; k0 += kWarp * E) {
+            const int32_t k = k0 + lane * E;
+            unsigned long long key[E];
+            if (VEC2) {
+#pragma unroll
+                for (int m = 0; m < E; m += 2) {
+                    ulonglong2 v = make_ulonglong2(0ull, 0ull);
+                    if (k + m < p.cap) v = __ldg(reinterpret_cast<const ulonglong2 *>(keys + k + m));
+                    key[m] = v.x;
+                    key[m + 1] = v.y;
+                }
+            } else {
+#pragma unroll
+                for (int m = 0; m < E; ++m) key[m] = (k + m < p.cap) ? __ldg(keys + k + m) : 0ull;
+            }
+            unsigned long long before = __shfl_up_sync(kFull, key[E - 1], 1);
+            if (lane == 0) before = prev_last;
+            prev_last = __shfl_sync(kFull, key[E - 1], kWarp - 1);
+            int run_bin = -1;
+            unsigned int run_len = 0;
+#pragma unroll
+            for (int m = 0; m < E; ++m) {
+                if (k + m < p.cap) {
+                    bad |= (key[m] >= kKeyInf) | (key[m] > before);
+                    before = key[m];
+                    const int bin = (int)(key[m] >> 51) & (kBins - 1);
+                    if (bin == run_bin) {
+                        ++run_len;
+                    } else {
+                        if (run_len) atomicAdd(&s_hist[run_bin], run_len);
+                        run_bin = bin;
+                        run_len = 1;
+                    }
+                }
+            }
+            if (run_len) atomicAdd(&s_hist[run_bin], run_len);
+        }
+    }
+    if (bad) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);
+    __syncthreads();
+    flush_hist(s_hist, hist, kBins);
+    long long tot;
+    block_exclusive_sum(capsum, &tot, s_warp);
+    if (threadIdx.x == 0 && tot) atomicAdd(&hdr->sum_cap, (unsigned long long)tot);
+    if (last_block(&hdr->ticket[0])) {
+        const unsigned long long sum_cap = *(volatile unsigned long long *)&hdr->sum_cap;
+        if (threadIdx.x == 0) {
+            if ((unsigned long long)B > sum_cap) raise_status(&hdr->status, HORA_ERR_INFEASIBLE);
+            hdr->need = B;
+        }
+        __syncthreads();
+        find_digit(hdr, hist, 0, s_warp);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Levels 1..4: a thread per row (grid-stride).  Level 1 finds the row's segment by binary search; later
+// levels narrow the stored segment by the digit selected one level up.  The keys that remain are
+// histogrammed on the current level's digit.
+__global__ void __launch_bounds__(kSelThreads)
+select_refine(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
+              const double *__restrict__ gains, int level, AllocHeader *hdr, unsigned long long *hist_all,
+              int2 *__restrict__ rowstate) {
+    __shared__ unsigned int s_hist[kBins];
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    if (*(volatile int32_t *)&hdr->status != 0) return;
+    const int bins = level_bins(level);
+    for (int b = threadIdx.x; b < bins; b += kSelThreads) s_hist[b] = 0;
+    __syncthreads();
+    const int shift_prev = level_shift(level - 1), shift_cur = level_shift(level);
+    const unsigned long long d_prev = (unsigned long long)hdr->sel_digit[level - 1];
+    const unsigned long long mask_prev = kBins - 1, mask_cur = (unsigned long long)bins - 1;
+    const int64_t stride = (int64_t)gridDim.x * kSelThreads;
+    for (int64_t row = (int64_t)blockIdx.x * kSelThreads + threadIdx.x; row < N; row += stride) {
+        const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+        int32_t p_hi, p_end;
+        if (level == 1) {
+            int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
+            capi = capi < 0 ? 0 : (capi > ld ? ld : capi);
+            int32_t lo = 0, hi = capi;                 // first index whose top digit is <= d_prev
+            while (lo < hi) {
+                const int32_t mid = (lo + hi) >> 1;
+                if ((__ldg(keys + mid) >> shift_prev) > d_prev) lo = mid + 1; else hi = mid;
+            }
+            p_hi = lo;
+            p_end = capi;
+        } else {
+            const int2 st = rowstate[row];
+            p_hi = st.x;
+            p_end = st.y;
+        }
+        int32_t p = p_hi, new_hi = p_hi;
+        while (p < p_end) {
+            const unsigned long long key = __ldg(keys + p);
+            const unsigned long long dp = (key >> shift_prev) & mask_prev;
+            if (dp > d_prev) {
+                new_hi = p + 1;
+            } else if (dp == d_prev) {
+                atomicAdd(&s_hist[(key >> shift_cur) & mask_cur], 1u);
+            } else {
+                break;
+            }
+            ++p;
+        }
+        rowstate[row] = make_int2(new_hi, p);
+    }
+    __syncthreads();
+    flush_hist(s_hist, hist_all + (size_t)level * kBins, bins);
+    if (last_block(&hdr->ticket[level])) find_digit(hdr, hist_all + (size_t)level * kBins, level, s_warp);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Exact arithmetic helpers (unsigned 128-bit as two words; overflow is reported, never wrapped).
+struct U128 { unsigned long long lo, hi; };
+
+__device__ __forceinline__ bool mul_small(U128 &x, unsigned long long m) {   // returns false on overflow
+    const unsigned long long lo = x.lo * m, carry = __umul64hi(x.lo, m);
+    const unsigned long long hi = x.hi * m;
+    const bool ovf = (__umul64hi(x.hi, m) != 0) || (hi + carry < hi);
+    x.lo = lo;
+    x.hi = hi + carry;
+    return !ovf;
+}
+
+// 128 x 128 -> 256 bit product, little-endian words
+__device__ void mul_wide(const U128 &p, const U128 &q, unsigned long long r[4]) {
+    const unsigned long long a0 = p.lo, a1 = p.hi, b0 = q.lo, b1 = q.hi;
+    r[0] = a0 * b0;
+    const unsigned long long t1 = __umul64hi(a0, b0);
+    const unsigned long long l01 = a0 * b1, h01 = __umul64hi(a0, b1);
+    const unsigned long long l10 = a1 * b0, h10 = __umul64hi(a1, b0);
+    const unsigned long long s = t1 + l01;
+    unsigned long long c1 = s < t1;
+    const unsigned long long s2 = s + l10;
+    c1 += s2 < s;
+    r[1] = s2;
+    const unsigned long long l11 = a1 * b1, h11 = __umul64hi(a1, b1);
+    const unsigned long long q2 = h01 + h10;
+    unsigned long long c2 = q2 < h01;
+    const unsigned long long q3 = q2 + l11;
+    c2 += q3 < q2;
+    const unsigned long long q4 = q3 + c1;
+    c2 += q4 < q3;
+    r[2] = q4;
+    r[3] = h11 + c2;
+}
+
+// sign of x*y - u*v with full 256-bit products
+__device__ int cmp_products(const U128 &x, const U128 &y, const U128 &u, const U128 &v) {
+    unsigned long long L[4], Rr[4];
+    mul_wide(x, y, L);
+    mul_wide(u, v, Rr);
+    for (int i = 3; i >= 0; --i) {
+        if (L[i] != Rr[i]) return L[i] > Rr[i] ? 1 : -1;
+    }
+    return 0;
+}
+
+// Exact gain of type (a, b, Delta) as num/den (not reduced).  Returns false if 128 bits do not suffice.
+__device__ bool exact_gain(unsigned long long a, unsigned long long b, unsigned long long Delta, U128 &num, U128 &den) {
+    num.lo = a; num.hi = 0;
+    den.lo = 1; den.hi = 0;
+    bool ok = true;
+    if (a + 1 <= Delta) {               // a (b)_a / (b+Delta-1)_{a+1}
+        for (unsigned long long k = 0; k < a && ok; ++k) ok = mul_small(num, b + k);
+        for (unsigned long long k = 0; k <= a && ok; ++k) ok = mul_small(den, b + Delta - 1 + k);
+    } else {                            // a (b)_{Delta-1} / (a+b)_{Delta}
+        for (unsigned long long j = 0; j + 1 < Delta && ok; ++j) ok = mul_small(num, b + j);
+        for (unsigned long long j = 0; j < Delta && ok; ++j) ok = mul_small(den, a + b + j);
+    }
+    return ok;
+}
+
+__device__ __forceinline__ unsigned long long pack_type(unsigned long long a, unsigned long long b, unsigned long long D) {
+    return (a << 43) | (b << 22) | D;   // a, b < 2^21, D < 2^22
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Exact mode, step 1: per row, find the (at most one) candidate inside the band around the fp64
+// threshold, register its type, and store the provisional state (everything above the band is taken).
+__global__ void __launch_bounds__(kSelThreads)
+exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
+              const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
+              int64_t N, int32_t ld, const double *__restrict__ gains, AllocHeader *hdr, int2 *__restrict__ rowstate,
+              int32_t *__restrict__ rowslot, unsigned long long *tkeys, unsigned long long *tcounts) {
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    if (*(volatile int32_t *)&hdr->status != 0) return;
+    const double lam = __longlong_as_double((long long)hdr->prefix_key);
+    const double delta_rel = 9.313225746154785e-10;   // 2^-30
+    const unsigned long long k_hi = (unsigned long long)__double_as_longlong(lam * (1.0 + delta_rel));
+    const unsigned long long k_lo = (unsigned long long)__double_as_longlong(lam * (1.0 - delta_rel));
+    const int lane = lane_id();
+    const int64_t stride = (int64_t)gridDim.x * kSelThreads;
+    long long above = 0;
+    int32_t err = 0;
+    for (int64_t base = (int64_t)blockIdx.x * kSelThreads; base < N; base += stride) {
+        const int64_t row = base + threadIdx.x;
+        unsigned long long tkey = 0;
+        int32_t q = 0;
+        if (row < N) {
+            const double al = alpha ? __ldg(alpha + row) : alpha0, be = beta ? __ldg(beta + row) : beta0;
+            const int32_t ci = __ldg(c + row);
+            const int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
+            if (!(al >= 1.0 && be >= 1.0 && al == floor(al) && be == floor(be))) err = HORA_ERR_NOT_INTEGER;
+            else if (al + be + (double)G0 + (double)ld >= 1048576.0) err = err ? err : HORA_ERR_EXACT_RANGE;
+            const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+            const int2 st = rowstate[row];
+            q = st.x;                                         // #keys > lambda
+            if (q > 0 && __ldg(keys + q - 1) <= k_hi) {
+                --q;
+                if (q > 0 && __ldg(keys + q - 1) <= k_hi) err = err ? err : HORA_ERR_EXACT_RANGE;
+            }
+            const bool has = (q < capi) && (__ldg(keys + q) >= k_lo);
+            if (has && q + 1 < capi && __ldg(keys + q + 1) >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
+            if (has && !err)
+                tkey = pack_type((unsigned long long)al + ci, (unsigned long long)be + (G0 - ci), (unsigned long long)q + 1);
+            above += q;
+        }
+        // one table update per distinct type per warp
+        const unsigned int peers = __match_any_sync(kFull, tkey);
+        int32_t slot = -1;
+        if (tkey != 0) {
+            const int leader = __ffs(peers) - 1;
+            if (lane == leader) {
+                unsigned int h = (unsigned int)((tkey * 0x9E3779B97F4A7C15ull) >> 52) & (kTypeSlots - 1);
+                for (int probe = 0; probe < kTypeSlots; ++probe) {
+                    const unsigned long long old = atomicCAS(tkeys + h, 0ull, tkey);
+                    if (old == 0ull || old == tkey) {
+                        if (old == 0ull) atomicAdd(&hdr->n_types, 1u);
+                        slot = (int32_t)h;
+                        break;
+                    }
+                    h = (h + 1) & (kTypeSlots - 1);
+                }
+                if (slot >= 0) atomicAdd(tcounts + slot, (unsigned long long)__popc(peers));
+                else err = err ? err : HORA_ERR_EXACT_RANGE;
+            }
+            slot = __shfl_sync(peers, slot, leader);
+        }
+        if (row < N) {
+            rowslot[row] = slot;
+            rowstate[row] = make_int2(q, q);
+        }
+    }
+    if (err) raise_status(&hdr->status, err);
+    long long tot;
+    block_exclusive_sum(above, &tot, s_warp);
+    if (threadIdx.x == 0 && tot) atomicAdd(&hdr->band_above, (unsigned long long)tot);
+}
+
+// Exact mode, step 2 (one CTA): rank the collected types exactly and label them.
+//   label 2: strictly better than the threshold class (taken)   1: threshold class   0: worse
+__global__ void __launch_bounds__(1024)
+exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ tkeys,
+           const unsigned long long *__restrict__ tcounts, int32_t *__restrict__ tlabel) {
+    __shared__ U128 s_num[kMaxTypes], s_den[kMaxTypes];
+    __shared__ unsigned long long s_cnt[kMaxTypes];
+    __shared__ int s_slot[kMaxTypes];
+    __shared__ int s_n;
+    __shared__ int s_err;
+    if (hdr->status != 0) return;
+    if (threadIdx.x == 0) { s_n = 0; s_err = 0; }
+    __syncthreads();
+    for (int h = threadIdx.x; h < kTypeSlots; h += blockDim.x) {
+        tlabel[h] = 0;
+        const unsigned long long key = tkeys[h];
+        if (key != 0ull) {
+            const int j = atomicAdd(&s_n, 1);
+            if (j < kMaxTypes) {
+                U128 nu, de;
+                if (!exact_gain(key >> 43, (key >> 22) & 0x1FFFFFull, key & 0x3FFFFFull, nu, de)) s_err = 1;
+                s_num[j] = nu;
+                s_den[j] = de;
+                s_cnt[j] = tcounts[h];
+                s_slot[j] = h;
+            }
+        }
+    }
+    __syncthreads();
+    const int n = s_n;
+    if (n > kMaxTypes || s_err) {
+        if (threadIdx.x == 0) raise_status(&hdr->status, HORA_ERR_EXACT_RANGE);
+        return;
+    }
+    const long long Rp = B - (long long)hdr->band_above;     // rollouts to hand out inside the band
+    for (int t = threadIdx.x; t < n; t += blockDim.x) {
+        long long above = 0, equal = 0;
+        for (int u = 0; u < n; ++u) {
+            const int s = cmp_products(s_num[u], s_den[t], s_num[t], s_den[u]);   // sign(val_u - val_t)
+            if (s > 0) above += (long long)s_cnt[u];
+            else if (s == 0) equal += (long long)s_cnt[u];
+        }
+        int label = 0;
+        if (above + equal < Rp) label = 2;
+        else if (above < Rp) label = 1;
+        tlabel[s_slot[t]] = label;
+        if (label == 1) {          // every member of the threshold class writes the same values
+            hdr->R = Rp - above;
+            hdr->lambda = ((double)s_num[t].hi * 18446744073709551616.0 + (double)s_num[t].lo) /
+                          ((double)s_den[t].hi * 18446744073709551616.0 + (double)s_den[t].lo);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Block sums of (p_hi, tied) in prompt order, and their exclusive scan by the last CTA.
+//   mode 0: rowstate is final    mode 1: narrow by the last digit first    mode 2: apply the exact labels first
+__global__ void __launch_bounds__(kSelThreads)
+select_sum(int64_t N, int32_t ld, const double *__restrict__ gains, int mode, int64_t B, AllocHeader *hdr,
+           int2 *__restrict__ rowstate, const int32_t *__restrict__ rowslot, const int32_t *__restrict__ tlabel,
+           long long *bsum_hi, long long *bsum_t, int64_t NB) {
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    const bool failed = *(volatile int32_t *)&hdr->status != 0;
+    long long hi_sum = 0, t_sum = 0;
+    if (!failed) {
+        const unsigned long long d_last = (unsigned long long)hdr->sel_digit[kLevels - 1];
+        const int64_t row0 = (int64_t)blockIdx.x * kRowsPerBlock;
+#pragma unroll
+        for (int q = 0; q < kRowsPerBlock / kSelThreads; ++q) {
+            const int64_t row = row0 + q * kSelThreads + threadIdx.x;
+            if (row >= N) break;
+            int2 st = rowstate[row];
+            if (mode == 1) {
+                const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+                int32_t p = st.x, new_hi = st.x;
+                while (p < st.y) {
+                    const unsigned long long dp = __ldg(keys + p) & 4095ull;
+                    if (dp > d_last) new_hi = p + 1;
+                    else if (dp < d_last) break;
+                    ++p;
+                }
+                st = make_int2(new_hi, p);
+                rowstate[row] = st;
+            } else if (mode == 2) {
+                const int32_t slot = rowslot[row];
+                const int label = slot >= 0 ? tlabel[slot] : 0;
+                st = make_int2(st.x + (label == 2), st.x + (label == 2) + (label == 1));
+                rowstate[row] = st;
+            }
+            hi_sum += st.x;
+            t_sum += st.y - st.x;
+        }
+    }
+    long long tot_hi, tot_t;
+    block_exclusive_sum(hi_sum, &tot_hi, s_warp);
+    block_exclusive_sum(t_sum, &tot_t, s_warp);
+    if (threadIdx.x == 0) { bsum_hi[blockIdx.x] = tot_hi; bsum_t[blockIdx.x] = tot_t; }
+    if (last_block(&hdr->ticket[8 + mode])) {
+        // exclusive scan of NB block sums, kSelThreads at a time, in index order
+        long long run_hi = 0, run_t = 0;
+        for (int64_t b0 = 0; b0 < NB; b0 += kSelThreads) {
+            const int64_t b = b0 + threadIdx.x;
+            const long long vh = b < NB ? __ldcg(bsum_hi + b) : 0, vt = b < NB ? __ldcg(bsum_t + b) : 0;
+            long long th, tt;
+            const long long eh = block_exclusive_sum(vh, &th, s_warp);
+            const long long et = block_exclusive_sum(vt, &tt, s_warp);
+            if (b < NB) { bsum_hi[b] = run_hi + eh; bsum_t[b] = run_t + et; }
+            run_hi += th;
+            run_t += tt;
+        }
+        if (threadIdx.x == 0 && !failed) {
+            hdr->n_above = (unsigned long long)run_hi;
+            hdr->n_tied = (unsigned long long)run_t;
+            hdr->R = B - run_hi;
+            if (mode != 2) hdr->lambda = B > 0 ? __longlong_as_double((long long)hdr->prefix_key) : 0.0;
+        }
+    }
+}
+
+// U(Delta) = 1 - prod_{j<Delta} (b+j)/(a+b+j)  (Eq. appendix-hit-closed-form written as a product)
+__device__ __forceinline__ double hit_utility(double a, double b, int32_t Delta) {
+    double q = 1.0, num = 1.0, den = 1.0;
+    const double ab = a + b;
+    for (int32_t j = 0; j < Delta; ++j) {
+        num *= b + (double)j;
+        den *= ab + (double)j;
+        if ((j & 7) == 7) { q *= num / den; num = 1.0; den = 1.0; }
+    }
+    q *= num / den;
+    return 1.0 - q;
+}
+
+// Outputs.  A CTA owns kRowsPerBlock consecutive prompts, a thread four consecutive ones.
+__global__ void __launch_bounds__(kSelThreads)
+select_out(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
+           const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N,
+           int32_t ld, int64_t B, uint32_t flags, AllocHeader *hdr, const int2 *__restrict__ rowstate,
+           const long long *__restrict__ bpre_hi, const long long *__restrict__ bpre_t, double *objpart, int64_t NB,
+           int32_t *__restrict__ delta, int32_t *__restrict__ G, int64_t *__restrict__ offsets,
+           hora_alloc_info *info) {
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    __shared__ double s_obj[kSelThreads / kWarp];
+    const int32_t status = *(volatile int32_t *)&hdr->status;
+    const bool failed = status != 0;
+    constexpr int kPer = kRowsPerBlock / kSelThreads;
+    const int64_t row0 = (int64_t)blockIdx.x * kRowsPerBlock + (int64_t)threadIdx.x * kPer;
+    int32_t hi[kPer], tied[kPer];
+    long long hi_sum = 0, t_sum = 0;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+        hi[q] = 0;
+        tied[q] = 0;
+        if (!failed && row0 + q < N) {
+            const int2 st = rowstate[row0 + q];
+            hi[q] = st.x;
+            tied[q] = st.y - st.x;
+        }
+        hi_sum += hi[q];
+        t_sum += tied[q];
+    }
+    long long th, tt;
+    long long pre_hi = block_exclusive_sum(hi_sum, &th, s_warp);
+    long long pre_t = block_exclusive_sum(t_sum, &tt, s_warp);
+    double obj = 0.0;
+    if (!failed) {
+        pre_hi += bpre_hi[blockIdx.x];
+        pre_t += bpre_t[blockIdx.x];
+    }
+    const long long R = failed ? 0 : hdr->R;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+        const int64_t row = row0 + q;
+        if (row < N) {
+            long long take = R - pre_t;
+            take = take < 0 ? 0 : (take > tied[q] ? tied[q] : take);
+            const int32_t d = failed ? 0 : hi[q] + (int32_t)take;
+            delta[row] = d;
+            G[row] = failed ? 0 : G0 + d;
+            if (offsets) offsets[row] = failed ? 0 : row * (int64_t)G0 + pre_hi + (pre_t < R ? pre_t : R);
+            if (!failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE) && d > 0) {
+                const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row);
+                obj += hit_utility(p.a, p.b, d);
+            }
+            pre_hi += hi[q];
+            pre_t += tied[q];
+        }
+    }
+    if (offsets && blockIdx.x == gridDim.x - 1 && threadIdx.x == kSelThreads - 1)
+        offsets[N] = failed ? 0 : N * (int64_t)G0 + B;
+    // objective: fixed-order tree (lanes by butterfly, then warps and blocks in index order)
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) obj += __shfl_xor_sync(kFull, obj, d);
+    if (lane_id() == 0) s_obj[threadIdx.x >> 5] = obj;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double s = 0.0;
+        for (int w = 0; w < kSelThreads / kWarp; ++w) s += s_obj[w];
+        objpart[blockIdx.x] = s;
+    }
+    if (last_block(&hdr->ticket[12])) {
+        double part = 0.0;
+        for (int64_t b = threadIdx.x; b < NB; b += kSelThreads) part += __ldcg(objpart + b);
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) part += __shfl_xor_sync(kFull, part, d);
+        __syncthreads();
+        if (lane_id() == 0) s_obj[threadIdx.x >> 5] = part;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double s = 0.0;
+            for (int w = 0; w < kSelThreads / kWarp; ++w) s += s_obj[w];
+            hdr->objective = s;
+            if (info) {
+                info->status = status;
+                info->reserved = 0;
+                info->lambda = failed ? 0.0 : hdr->lambda;
+                info->n_above = failed ? 0 : (int64_t)hdr->n_above;
+                info->n_tied = failed ? 0 : (int64_t)hdr->n_tied;
+                info->n_tied_taken = failed ? 0 : hdr->R;
+                info->objective = failed ? 0.0 : s;
+                info->sum_G = failed ? 0 : N * (int64_t)G0 + B;
+                info->sum_cap = (int64_t)hdr->sum_cap;
+            }
+        }
+    }
+}
+
+// N == 0: nothing to select; still produce a well-defined summary.
+__global__ void write_empty(int64_t B, int64_t *offsets, hora_alloc_info *info) {
+    if (offsets) offsets[0] = 0;
+    if (info) {
+        info->status = B > 0 ? HORA_ERR_INFEASIBLE : HORA_OK;
+        info->reserved = 0;
+        info->lambda = 0.0;
+        info->n_above = info->n_tied = info->n_tied_taken = 0;
+        info->objective = 0.0;
+        info->sum_G = 0;
+        info->sum_cap = 0;
+    }
+}
+
+template <int E>
+static void launch_level0(bool vec2, int grid, cudaStream_t s, const double *alpha, const double *beta, double alpha0,
+                          double beta0, const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N,
+                          int32_t ld, const double *gains, int64_t B, AllocHeader *hdr, unsigned long long *hist) {
+    if (vec2)
+        select_level0<E, true><<<grid, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
+                                                            gains, B, hdr, hist);
+    else
+        select_level0<E, false><<<grid, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
+                                                             gains, B, hdr, hist);
+}
+
+}  // namespace hora
+
+extern "C" size_t hora_allocate_workspace_bytes(int64_t N, int32_t ld, int32_t gains_is_null, uint32_t flags) {
+    if (N < 0 || ld < 1) return 0;
+    return hora::carve(nullptr, N, ld, gains_is_null != 0, (flags & HORA_FLAG_EXACT_INT) != 0).bytes;
+}
+
+extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, double alpha0, double beta0,
+                                       const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N,
+                                       int32_t ld, const double *gains, int64_t B, uint32_t flags, int32_t *delta,
+                                       int32_t *G, int64_t *group_offsets, hora_alloc_info *info_dev, void *workspace,
+                                       size_t workspace_bytes, void *stream) {
+    using namespace hora;
+    if (N < 0 || ld < 1 || G0 < 0 || B < 0) return HORA_ERR_INVALID_ARG;
+    if ((alpha == nullptr) != (beta == nullptr)) return HORA_ERR_INVALID_ARG;
+    if (alpha == nullptr && !(alpha0 > 0.0 && beta0 > 0.0 && alpha0 < 1.0e300 && beta0 < 1.0e300))
+        return HORA_ERR_INVALID_ARG;
+    if (cap == nullptr && (cap_scalar < 0 || cap_scalar > ld)) return HORA_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE)) return HORA_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (N == 0) {
+        write_empty<<<1, 1, 0, s>>>(B, group_offsets, info_dev);
+        count_launches(1);
+        return cuda_ok(cudaGetLastError());
+    }
+    if (c == nullptr || delta == nullptr || G == nullptr) return HORA_ERR_INVALID_ARG;
+    if (gains != nullptr && (reinterpret_cast<uintptr_t>(gains) & 7u)) return HORA_ERR_INVALID_ARG;
+    const bool exact = (flags & HORA_FLAG_EXACT_INT) != 0;
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HORA_ERR_WORKSPACE;
+    const Workspace w = carve(workspace, N, ld, gains == nullptr, exact);
+    if (workspace_bytes < w.bytes) return HORA_ERR_WORKSPACE;
+    const int64_t NB = (N + kRowsPerBlock - 1) / kRowsPerBlock;
+
+    // header and histograms are contiguous at the start of the workspace
+    const size_t zero_bytes = reinterpret_cast<char *>(w.rowstate) - reinterpret_cast<char *>(w.hdr);
+    if (cudaMemsetAsync(w.hdr, 0, zero_bytes, s) != cudaSuccess) return HORA_ERR_CUDA;
+    if (exact) {
+        const size_t tb = reinterpret_cast<char *>(w.rowslot) - reinterpret_cast<char *>(w.tkeys);
+        if (cudaMemsetAsync(w.tkeys, 0, tb, s) != cudaSuccess) return HORA_ERR_CUDA;
+    }
+    if (gains == nullptr) {
+        const hora_status_t st = launch_gains(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, w.gains,
+                                              &w.hdr->status, s);
+        if (st != HORA_OK) return st;
+        gains = w.gains;
+    }
+    const bool vec2 = (ld % 2 == 0) && ((reinterpret_cast<uintptr_t>(gains) & 15u) == 0);
+    const int rows_per_cta = kSelThreads / kWarp;
+    const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 6);
+    if (ld > 128)
+        launch_level0<8>(vec2, grid0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist);
+    else if (ld > 64)
+        launch_level0<4>(vec2, grid0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist);
+    else
+        launch_level0<2>(vec2, grid0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist);
+    const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 4);
+    if (B > 0) {
+        for (int level = 1; level < kLevels; ++level)
+            select_refine<<<grid_rows, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, level, w.hdr, w.hist, w.rowstate);
+        select_sum<<<(int)NB, kSelThreads, 0, s>>>(N, ld, gains, 1, B, w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi,
+                                                   w.bsum_t, NB);
+        if (exact) {
+            exact_collect<<<grid_rows, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
+                                                            gains, w.hdr, w.rowstate, w.rowslot, w.tkeys, w.tcounts);
+            exact_rank<<<1, 1024, 0, s>>>(B, w.hdr, w.tkeys, w.tcounts, w.tlabel);
+            select_sum<<<(int)NB, kSelThreads, 0, s>>>(N, ld, gains, 2, B, w.hdr, w.rowstate, w.rowslot, w.tlabel,
+                                                       w.bsum_hi, w.bsum_t, NB);
+        }
+    } else {
+        if (cudaMemsetAsync(w.rowstate, 0, sizeof(int2) * (size_t)N, s) != cudaSuccess) return HORA_ERR_CUDA;
+        select_sum<<<(int)NB, kSelThreads, 0, s>>>(N, ld, gains, 0, B, w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi,
+                                                   w.bsum_t, NB);
+    }
+    select_out<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, flags, w.hdr,
+                                               w.rowstate, w.bsum_hi, w.bsum_t, w.objpart, NB, delta, G, group_offsets,
+                                               info_dev);
+    count_launches(B > 0 ? (exact ? 10 : 7) : 3);
+    return cuda_ok(cudaGetLastError());
+}

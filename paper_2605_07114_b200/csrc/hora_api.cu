@@ -1,0 +1,27 @@
+// Host-only entry points of the HORA library.
+#include <atomic>
+
+#include "hora_common.cuh"
+
+namespace hora {
+static std::atomic<unsigned long long> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+}  // namespace hora
+
+extern "C" const char *hora_status_string(hora_status_t status) {
+    switch (status) {
+        case HORA_OK: return "ok";
+        case HORA_ERR_INVALID_ARG: return "invalid argument";
+        case HORA_ERR_INVALID_VALUE: return "invalid value in device data";
+        case HORA_ERR_INFEASIBLE: return "budget exceeds the total cap";
+        case HORA_ERR_NOT_INTEGER: return "exact mode needs integer-valued priors";
+        case HORA_ERR_EXACT_RANGE: return "exact mode: parameters out of range";
+        case HORA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case HORA_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+extern "C" int hora_version(void) { return 100; }
+
+extern "C" uint64_t hora_launch_count(void) { return hora::g_launches.load(std::memory_order_relaxed); }

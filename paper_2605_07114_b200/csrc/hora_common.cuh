@@ -1,0 +1,64 @@
+// Shared device/host helpers of the HORA CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hora.h"
+
+namespace hora {
+
+constexpr int kWarp = 32;
+constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kSmCount = 148;              // B200: grids are sized in multiples of this
+
+// First data-dependent error wins; later kernels of the same call see it and stand down.
+__device__ __forceinline__ void raise_status(int32_t *status, int32_t code) {
+    if (status != nullptr) atomicCAS(status, 0, code);
+}
+
+__device__ __forceinline__ int lane_id() { return threadIdx.x & (kWarp - 1); }
+
+__device__ __forceinline__ double shfl_up_f64(double v, int d) { return __shfl_up_sync(kFull, v, d); }
+__device__ __forceinline__ double shfl_idx_f64(double v, int l) { return __shfl_sync(kFull, v, l); }
+
+// Posterior parameters of one prompt (Eq. posterior) with the validity checks every kernel repeats.
+struct Posterior {
+    double a, b;
+    int32_t cap;
+    bool ok;
+};
+
+__device__ __forceinline__ Posterior load_posterior(const double *alpha, const double *beta, double alpha0,
+                                                    double beta0, const int32_t *c, int32_t G0,
+                                                    const int32_t *cap, int32_t cap_scalar, int32_t ld, int64_t i) {
+    Posterior p;
+    const double al = alpha ? __ldg(alpha + i) : alpha0;
+    const double be = beta ? __ldg(beta + i) : beta0;
+    const int32_t ci = __ldg(c + i);
+    p.cap = cap ? __ldg(cap + i) : cap_scalar;
+    p.ok = (al > 0.0) && (be > 0.0) && (al < 1.0e300) && (be < 1.0e300) && (ci >= 0) && (ci <= G0) &&
+           (p.cap >= 0) && (p.cap <= ld);
+    p.a = al + (double)ci;
+    p.b = be + (double)(G0 - ci);
+    if (!p.ok) p.cap = 0;
+    return p;
+}
+
+inline hora_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? HORA_OK : HORA_ERR_CUDA; }
+
+inline int clamp_grid(int64_t want, int per_sm) {
+    const int64_t cap = (int64_t)kSmCount * per_sm;
+    if (want < 1) want = 1;
+    return (int)(want < cap ? want : cap);
+}
+
+// Host-side count of kernels this library has launched in this process (see hora_launch_count).
+void count_launches(int n);
+
+// Launchers shared between translation units.
+hora_status_t launch_gains(const double *alpha, const double *beta, double alpha0, double beta0,
+                           const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N,
+                           int32_t ld, double *gains, int32_t *status_dev, cudaStream_t stream);
+
+}  // namespace hora

@@ -1,0 +1,114 @@
+// hora_gains: fp64 marginal-gain rows by a warp-level prefix product (Eq. marginal and its recurrence).
+//
+// With k = Delta-1 the row is an inclusive prefix product of factors phi_k = num_k / den_k,
+//     num_0 = a,  num_k = b + k - 1 (k >= 1),   den_k = a + b + k,
+// so g[0] = a/(a+b) and g[k+1] = g[k] (b+k)/(a+b+k+1), which is the paper's recurrence.
+// One warp owns one row.  A lane takes E consecutive factors, multiplies numerators forwards and
+// denominators backwards, and needs ONE reciprocal for its E entries (1/(d_0..d_m) = (d_{m+1}..d_{E-1}) / (d_0..d_{E-1})).
+// The lanes' E-factor products are combined by a multiplicative warp scan; rows longer than 32*E
+// carry the running product from chunk to chunk.  The value of an entry depends on (a, b, k, E) only,
+// never on the row index, so equal posteriors give bitwise equal rows.
+#include "hora_common.cuh"
+
+namespace hora {
+
+constexpr int kGainsWarps = 8;
+
+template <int E, bool VEC2>
+__global__ void __launch_bounds__(kGainsWarps *kWarp)
+gains_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
+             const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
+             int64_t N, int32_t ld, double *__restrict__ gains, int32_t *status_dev) {
+    const int lane = lane_id();
+    const int64_t warp0 = (int64_t)blockIdx.x * kGainsWarps + (threadIdx.x >> 5);
+    const int64_t stride = (int64_t)gridDim.x * kGainsWarps;
+    for (int64_t row = warp0; row < N; row += stride) {
+        const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row);
+        if (!p.ok && lane == 0) raise_status(status_dev, HORA_ERR_INVALID_VALUE);
+        const double a = p.ok ? p.a : 1.0, b = p.ok ? p.b : 1.0;
+        const double ab = a + b;
+        double *out = gains + row * (int64_t)ld;
+        double carry = 1.0;
+        for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E) {
+            const int32_t k = k0 + lane * E;
+            double P[E + 1], S[E + 1];
+            P[0] = 1.0;
+#pragma unroll
+            for (int m = 0; m < E; ++m) {
+                const int32_t km = k + m;
+                const double num = (km == 0) ? a : b + (double)(km - 1);
+                P[m + 1] = P[m] * num;
+            }
+            S[E] = 1.0;
+#pragma unroll
+            for (int m = E - 1; m >= 0; --m) S[m] = S[m + 1] * (ab + (double)(k + m));
+            const double r = 1.0 / S[0];
+            double inc = P[E] * r;                       // this lane's E-factor product
+#pragma unroll
+            for (int d = 1; d < kWarp; d <<= 1) {
+                const double t = shfl_up_f64(inc, d);
+                if (lane >= d) inc *= t;
+            }
+            double excl = shfl_up_f64(inc, 1);
+            if (lane == 0) excl = 1.0;
+            const double total = shfl_idx_f64(inc, kWarp - 1);
+            const double base = carry * excl * r;
+            carry *= total;
+            double g[E];
+#pragma unroll
+            for (int m = 0; m < E; ++m) g[m] = (k + m < p.cap) ? (base * P[m + 1]) * S[m + 1] : 0.0;
+            if (VEC2) {
+#pragma unroll
+                for (int m = 0; m < E; m += 2)
+                    if (k + m < ld) *reinterpret_cast<double2 *>(out + k + m) = make_double2(g[m], g[m + 1]);
+            } else {
+#pragma unroll
+                for (int m = 0; m < E; ++m)
+                    if (k + m < ld) out[k + m] = g[m];
+            }
+        }
+    }
+}
+
+template <int E>
+static hora_status_t launch_e(const double *alpha, const double *beta, double alpha0, double beta0, const int32_t *c,
+                              int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N, int32_t ld, double *gains,
+                              int32_t *status_dev, cudaStream_t stream) {
+    const int grid = clamp_grid((N + kGainsWarps - 1) / kGainsWarps, 8);
+    const bool vec2 = (ld % 2 == 0) && ((reinterpret_cast<uintptr_t>(gains) & 15u) == 0);
+    if (vec2)
+        gains_kernel<E, true><<<grid, kGainsWarps * kWarp, 0, stream>>>(alpha, beta, alpha0, beta0, c, G0, cap,
+                                                                        cap_scalar, N, ld, gains, status_dev);
+    else
+        gains_kernel<E, false><<<grid, kGainsWarps * kWarp, 0, stream>>>(alpha, beta, alpha0, beta0, c, G0, cap,
+                                                                         cap_scalar, N, ld, gains, status_dev);
+    count_launches(1);
+    return cuda_ok(cudaGetLastError());
+}
+
+hora_status_t launch_gains(const double *alpha, const double *beta, double alpha0, double beta0, const int32_t *c,
+                           int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N, int32_t ld, double *gains,
+                           int32_t *status_dev, cudaStream_t stream) {
+    if (ld > 128)
+        return launch_e<8>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
+    if (ld > 64)
+        return launch_e<4>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
+    return launch_e<2>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
+}
+
+}  // namespace hora
+
+extern "C" hora_status_t hora_gains(const double *alpha, const double *beta, double alpha0, double beta0,
+                                    const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N,
+                                    int32_t ld, double *gains, int32_t *status_dev, void *stream) {
+    if (N < 0 || ld < 1 || G0 < 0) return HORA_ERR_INVALID_ARG;
+    if ((alpha == nullptr) != (beta == nullptr)) return HORA_ERR_INVALID_ARG;
+    if (alpha == nullptr && !(alpha0 > 0.0 && beta0 > 0.0 && alpha0 < 1.0e300 && beta0 < 1.0e300))
+        return HORA_ERR_INVALID_ARG;
+    if (cap == nullptr && (cap_scalar < 0 || cap_scalar > ld)) return HORA_ERR_INVALID_ARG;
+    if (N == 0) return HORA_OK;
+    if (c == nullptr || gains == nullptr) return HORA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(gains) & 7u) return HORA_ERR_INVALID_ARG;
+    return hora::launch_gains(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev,
+                              static_cast<cudaStream_t>(stream));
+}

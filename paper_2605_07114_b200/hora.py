@@ -1,0 +1,191 @@
+"""Thin ctypes binding over ``libhora.so`` — same names and arguments as ``include/hora.h``.
+
+Argument marshalling only: tensors are passed as device pointers, the stream is torch's current
+stream, and every step of the path runs in the library's CUDA kernels.  There is no CPU
+fallback: if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libhora.so")
+
+OK, ERR_INVALID_ARG, ERR_INVALID_VALUE, ERR_INFEASIBLE, ERR_NOT_INTEGER, ERR_EXACT_RANGE, ERR_WORKSPACE, ERR_CUDA = range(8)
+FLAG_EXACT_INT = 1
+FLAG_SKIP_OBJECTIVE = 2
+ADV_GRPO, ADV_RLOO = 0, 1
+
+EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora_group_advantage",
+           "hora_token_broadcast", "hora_status_string", "hora_version", "hora_launch_count")
+
+
+class HoraError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+        self.code = code
+
+
+class hora_alloc_info(C.Structure):
+    _fields_ = [("status", C.c_int32), ("reserved", C.c_int32), ("lambda_", C.c_double),
+                ("n_above", C.c_int64), ("n_tied", C.c_int64), ("n_tied_taken", C.c_int64),
+                ("objective", C.c_double), ("sum_G", C.c_int64), ("sum_cap", C.c_int64)]
+
+
+INFO_BYTES = C.sizeof(hora_alloc_info)
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Load the CUDA library built in-tree.  Raises if it is not there: nothing else can do its work."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(f"{LIB_PATH} not found: build it with `python -m paper_2605_07114_b200.build`")
+    L = C.CDLL(LIB_PATH)
+    p, i32, i64, f64, u32 = C.c_void_p, C.c_int32, C.c_int64, C.c_double, C.c_uint32
+    L.hora_gains.argtypes = [p, p, f64, f64, p, i32, p, i32, i64, i32, p, p, p]
+    L.hora_gains.restype = C.c_int
+    L.hora_allocate_workspace_bytes.argtypes = [i64, i32, i32, u32]
+    L.hora_allocate_workspace_bytes.restype = C.c_size_t
+    L.hora_allocate.argtypes = [p, p, f64, f64, p, i32, p, i32, i64, i32, p, i64, u32, p, p, p, p, p, C.c_size_t, p]
+    L.hora_allocate.restype = C.c_int
+    L.hora_group_advantage.argtypes = [p, p, i64, i32, C.c_float, i32, p, p, p]
+    L.hora_group_advantage.restype = C.c_int
+    L.hora_token_broadcast.argtypes = [p, p, i64, i64, p, p]
+    L.hora_token_broadcast.restype = C.c_int
+    L.hora_status_string.argtypes = [C.c_int]
+    L.hora_status_string.restype = C.c_char_p
+    L.hora_version.restype = C.c_int
+    L.hora_launch_count.restype = C.c_uint64
+    _lib = L
+    return L
+
+
+def status_string(code: int) -> str:
+    return load().hora_status_string(int(code)).decode()
+
+
+hora_status_string = status_string
+
+
+def hora_version() -> int:
+    return load().hora_version()
+
+
+def hora_launch_count() -> int:
+    return int(load().hora_launch_count())
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, name="tensor"):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc: int, where: str):
+    if rc != OK:
+        raise HoraError(rc, where)
+
+
+def hora_gains(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev=None):
+    rc = load().hora_gains(_ptr(alpha, torch.float64, "alpha"), _ptr(beta, torch.float64, "beta"), alpha0, beta0,
+                           _ptr(c, torch.int32, "c"), G0, _ptr(cap, torch.int32, "cap"), cap_scalar, N, ld,
+                           _ptr(gains, torch.float64, "gains"), _ptr(status_dev, torch.int32, "status_dev"), _stream())
+    _check(rc, "hora_gains")
+
+
+def hora_allocate_workspace_bytes(N, ld, gains_is_null, flags) -> int:
+    return int(load().hora_allocate_workspace_bytes(N, ld, int(bool(gains_is_null)), flags))
+
+
+def hora_allocate(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, flags, delta, G,
+                  group_offsets, info_dev, workspace):
+    rc = load().hora_allocate(_ptr(alpha, torch.float64, "alpha"), _ptr(beta, torch.float64, "beta"), alpha0, beta0,
+                              _ptr(c, torch.int32, "c"), G0, _ptr(cap, torch.int32, "cap"), cap_scalar, N, ld,
+                              _ptr(gains, torch.float64, "gains"), B, flags, _ptr(delta, torch.int32, "delta"),
+                              _ptr(G, torch.int32, "G"), _ptr(group_offsets, torch.int64, "group_offsets"),
+                              _ptr(info_dev, torch.uint8, "info_dev"), _ptr(workspace, torch.uint8, "workspace"),
+                              0 if workspace is None else workspace.numel(), _stream())
+    _check(rc, "hora_allocate")
+
+
+def hora_group_advantage(rewards, group_offsets, N, mode, eps, ddof, adv, status_dev=None):
+    rc = load().hora_group_advantage(_ptr(rewards, torch.float32, "rewards"),
+                                     _ptr(group_offsets, torch.int64, "group_offsets"), N, mode, eps, ddof,
+                                     _ptr(adv, torch.float32, "adv"), _ptr(status_dev, torch.int32, "status_dev"),
+                                     _stream())
+    _check(rc, "hora_group_advantage")
+
+
+def hora_token_broadcast(adv, token_offsets, R, T, token_adv):
+    rc = load().hora_token_broadcast(_ptr(adv, torch.float32, "adv"), _ptr(token_offsets, torch.int64, "token_offsets"),
+                                     R, T, _ptr(token_adv, torch.float32, "token_adv"), _stream())
+    _check(rc, "hora_token_broadcast")
+
+
+# ------------------------------------------------------------------------------------------------
+# Convenience layer: buffer ownership for callers who hold torch tensors.  No arithmetic here.
+@dataclass
+class AllocInfo:
+    status: int
+    lambda_: float
+    n_above: int
+    n_tied: int
+    n_tied_taken: int
+    objective: float
+    sum_G: int
+    sum_cap: int
+
+
+def read_info(info_dev: torch.Tensor) -> AllocInfo:
+    """Copy the 64-byte summary to the host (synchronises the current stream)."""
+    raw = bytes(info_dev.cpu().numpy().tobytes())
+    s = hora_alloc_info.from_buffer_copy(raw)
+    return AllocInfo(s.status, s.lambda_, s.n_above, s.n_tied, s.n_tied_taken, s.objective, s.sum_G, s.sum_cap)
+
+
+class Allocator:
+    """Owns the device buffers of one allocation problem shape (N, ld) and runs gains -> allocate."""
+
+    def __init__(self, N: int, ld: int, G0: int, *, exact_int: bool = False, skip_objective: bool = False,
+                 materialise: bool = True, device="cuda"):
+        self.N, self.ld, self.G0 = N, ld, G0
+        self.flags = (FLAG_EXACT_INT if exact_int else 0) | (FLAG_SKIP_OBJECTIVE if skip_objective else 0)
+        self.materialise = materialise
+        dev = torch.device(device)
+        self.gains = torch.empty((N, ld), dtype=torch.float64, device=dev) if materialise else None
+        wb = hora_allocate_workspace_bytes(N, ld, not materialise, self.flags)
+        self.workspace = torch.empty(max(wb, 256), dtype=torch.uint8, device=dev)
+        if self.workspace.data_ptr() % 256:
+            raise RuntimeError("device allocation is not 256-byte aligned")
+        self.delta = torch.empty(N, dtype=torch.int32, device=dev)
+        self.G = torch.empty(N, dtype=torch.int32, device=dev)
+        self.group_offsets = torch.empty(N + 1, dtype=torch.int64, device=dev)
+        self.info = torch.zeros(INFO_BYTES, dtype=torch.uint8, device=dev)
+
+    def run(self, alpha, beta, alpha0, beta0, c, cap, cap_scalar, B):
+        if self.materialise:
+            hora_gains(alpha, beta, alpha0, beta0, c, self.G0, cap, cap_scalar, self.N, self.ld, self.gains)
+        hora_allocate(alpha, beta, alpha0, beta0, c, self.G0, cap, cap_scalar, self.N, self.ld, self.gains, B,
+                      self.flags, self.delta, self.G, self.group_offsets, self.info, self.workspace)
+        return self.delta, self.G, self.group_offsets
+
+    def read_info(self) -> AllocInfo:
+        return read_info(self.info)

@@ -1,0 +1,325 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element, on the
+same seeded inputs.  Integer, index and byte results must be bit-exact; fp64 gains within 4*ld ulp of the
+long-double oracle; real-prior allocations may differ only inside the 1e-12 band around the threshold;
+fp32 advantages within 1e-5 absolute; broadcast output bitwise."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+from oracle import hora_oracle as orc  # noqa: E402
+from paper_2605_07114_b200 import workloads as wl  # noqa: E402
+
+U = 2.0 ** -53
+
+
+def _util():
+    import gpu_util
+    return gpu_util
+
+
+# ------------------------------------------------------------------------------------------ gains
+def gains_tol(ld):
+    return 4 * max(ld, 16) * U
+
+
+@pytest.mark.parametrize("ld", [1, 2, 3, 31, 60, 64, 65, 124, 129, 248, 256, 300, 700])
+@pytest.mark.parametrize("integer_prior", [False, True])
+def test_gains_match_oracle(ld, integer_prior):
+    gu = _util()
+    rng = np.random.default_rng(ld * 2 + integer_prior)
+    N, G0 = 333, 8
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    cap[:3] = [ld, 0, min(1, ld)]
+    if integer_prior:
+        alpha = beta = None
+        a0, b0 = 1.0, 1.0
+    else:
+        alpha = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
+        beta = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
+        alpha[0], beta[0] = 0.05, 0.05
+        alpha[1], beta[1] = 20.0, 20.0
+        a0 = b0 = 1.0
+    got, status = gu.gpu_gains(alpha, beta, a0, b0, c, G0, cap, ld)
+    exp = orc.gains(alpha, beta, a0, b0, c, G0, cap, ld)
+    assert status == 0
+    mask = np.arange(ld)[None, :] < cap[:, None]
+    assert (got[~mask] == 0.0).all()                                # padding is exactly zero
+    rel = np.abs(got[mask] - exp[mask]) / exp[mask]
+    assert rel.max(initial=0.0) <= gains_tol(ld), rel.max()
+    # rows strictly decrease (Eq. appendix-monotone) in the computed values too
+    d = np.diff(got, axis=1)
+    assert (d[mask[:, 1:]] < 0).all()
+
+
+def test_gains_scalar_cap_and_equal_posteriors_give_equal_bits():
+    gu = _util()
+    N, G0, ld = 1000, 4, 124
+    c = (np.arange(N) % (G0 + 1)).astype(np.int32)
+    got, status = gu.gpu_gains(None, None, 1.0, 1.0, c, G0, None, ld, cap_scalar=100)
+    assert status == 0
+    assert (got[:, 100:] == 0).all() and (got[:, :100] > 0).all()
+    for k in range(G0 + 1):
+        rows = got[c == k]
+        assert (rows.view(np.uint64) == rows[0].view(np.uint64)).all()
+
+
+def test_gains_flags_invalid_rows():
+    gu = _util()
+    N, G0, ld = 64, 4, 32
+    c = np.full(N, 2, np.int32)
+    cap = np.full(N, ld, np.int32)
+    alpha = np.ones(N)
+    beta = np.ones(N)
+    alpha[5] = -1.0
+    beta[6] = np.nan
+    c[7] = G0 + 1
+    cap[8] = ld + 1
+    alpha[9] = np.inf
+    got, status = gu.gpu_gains(alpha, beta, 1.0, 1.0, c, G0, cap, ld)
+    assert status == 2
+    for i in (5, 6, 7, 8, 9):
+        assert (got[i] == 0).all()
+    assert (got[10] > 0).all()
+
+
+# ------------------------------------------------------------------------------------- allocation
+def run_and_compare(w, materialise=True):
+    gu = _util()
+    d_o, G_o, lam_o, obj_o = gu.oracle_allocate(w)
+    d, G, off, info = gu.gpu_allocate(w.alpha, w.beta, w.alpha0, w.beta0, w.c, w.G0, w.cap, w.ld, w.B,
+                                      exact=w.exact_int, materialise=materialise)
+    gu.assert_allocation_matches(w, d, G, off, info, d_o, lam_o, obj_o)
+    return d, G, off, info
+
+
+@pytest.mark.parametrize("name,N", [("cfg1", None), ("cfg2", None), ("cfg3", None), ("cfg4", 1 << 15), ("cfg5", 1 << 16),
+                                    ("cfg1", 37), ("cfg5", 1000), ("cfg4", 777), ("cfg2", 1)])
+def test_allocation_matches_oracle(name, N):
+    run_and_compare(wl.make(name, N))
+
+
+@pytest.mark.parametrize("name,N", [("cfg1", None), ("cfg2", 2048), ("cfg5", 5000)])
+def test_allocation_without_materialised_gains(name, N):
+    run_and_compare(wl.make(name, N), materialise=False)
+
+
+def test_every_budget_on_the_worked_example():
+    """G0 = 2, c = (0,1,2,0), cap 3: B = 6, 7 hit the cross-class tie 3/20, B = 9, 10 the tie 1/10."""
+    gu = _util()
+    c = np.array([0, 1, 2, 0], np.int32)
+    cap = np.full(4, 3, np.int32)
+    for B in range(0, 13):
+        d_o = orc.greedy_exact(None, None, 1.0, 1.0, c, 2, cap, B)[0]
+        d, G, off, info = gu.gpu_allocate(None, None, 1.0, 1.0, c, 2, cap, 3, B, exact=True)
+        assert info.status == 0
+        np.testing.assert_array_equal(d, d_o)
+        np.testing.assert_array_equal(G, 2 + d_o)
+
+
+@pytest.mark.parametrize("G0", [2, 4, 8])
+def test_budget_sweep_through_cross_class_ties(G0):
+    """Many budgets on a small tie-heavy problem: every threshold, including exact cross-class ties,
+    must reproduce exact greedy with lowest-index tie-breaking."""
+    gu = _util()
+    rng = np.random.default_rng(G0)
+    N, ld = 97, 40
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    total = int(cap.sum())
+    budgets = sorted(set([0, 1, 2, total - 1, total] + list(rng.integers(0, total + 1, 40))))
+    for B in budgets:
+        d_o = orc.greedy_exact(None, None, 1.0, 1.0, c, G0, cap, int(B))[0]
+        d, G, off, info = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, cap, ld, int(B), exact=True)
+        assert info.status == 0, (B, info)
+        np.testing.assert_array_equal(d, d_o, err_msg=f"B={B}")
+
+
+def test_per_prompt_integer_priors_exact():
+    gu = _util()
+    rng = np.random.default_rng(77)
+    N, G0, ld = 500, 4, 30
+    alpha = rng.integers(1, 4, N).astype(np.float64)
+    beta = rng.integers(1, 4, N).astype(np.float64)
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    for B in (1, 100, 2500, int(cap.sum()) // 2):
+        d_o = orc.greedy_exact(alpha, beta, 1.0, 1.0, c, G0, cap, B)[0]
+        d, G, off, info = gu.gpu_allocate(alpha, beta, 1.0, 1.0, c, G0, cap, ld, B, exact=True)
+        assert info.status == 0
+        np.testing.assert_array_equal(d, d_o)
+
+
+def test_single_class_is_pure_index_tie_break():
+    gu = _util()
+    N, G0, ld = 1000, 4, 8
+    c = np.zeros(N, np.int32)
+    cap = np.full(N, ld, np.int32)
+    B = 3 * N + 123
+    d, G, off, info = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, cap, ld, B, exact=True)
+    assert info.status == 0
+    exp = np.full(N, 3, np.int32)
+    exp[:123] = 4
+    np.testing.assert_array_equal(d, exp)
+    assert info.n_tied == N and info.n_tied_taken == 123 and info.n_above == 3 * N
+    # the fp64 path ties on equal bit patterns and must give the same answer here
+    d2, _, _, info2 = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, cap, ld, B, exact=False)
+    np.testing.assert_array_equal(d2, exp)
+
+
+def test_edge_budgets_and_caps():
+    gu = _util()
+    rng = np.random.default_rng(8)
+    N, G0, ld = 301, 8, 17
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    cap = np.zeros(N, np.int32)
+    cap[::3] = rng.integers(0, ld + 1, len(cap[::3]))
+    total = int(cap.sum())
+    for exact in (True, False):
+        d, G, off, info = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, cap, ld, 0, exact=exact)
+        assert info.status == 0 and not d.any() and (G == G0).all() and off[-1] == N * G0 and info.lambda_ == 0.0
+        d, G, off, info = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, cap, ld, total, exact=exact)
+        assert info.status == 0
+        np.testing.assert_array_equal(d, cap)
+        d, G, off, info = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, cap, ld, total + 1, exact=exact)
+        assert info.status == 3 and not d.any() and not G.any() and not off.any()
+    one = np.zeros(N, np.int32)
+    one[200] = 5
+    d, G, off, info = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, one, ld, 4, exact=True)
+    assert info.status == 0 and d[200] == 4 and d.sum() == 4
+
+
+def test_allocation_status_codes():
+    gu = _util()
+    N, G0, ld = 100, 4, 16
+    c = np.full(N, 1, np.int32)
+    cap = np.full(N, ld, np.int32)
+    alpha = np.ones(N)
+    beta = np.ones(N)
+    alpha[3] = 1.5
+    d, G, off, info = gu.gpu_allocate(alpha, beta, 1.0, 1.0, c, G0, cap, ld, 50, exact=True)
+    assert info.status == 4 and not d.any()
+    alpha[3] = 2.0e6
+    d, G, off, info = gu.gpu_allocate(alpha, beta, 1.0, 1.0, c, G0, cap, ld, 50, exact=True)
+    assert info.status == 5 and not d.any()
+    alpha[3] = -1.0
+    d, G, off, info = gu.gpu_allocate(alpha, beta, 1.0, 1.0, c, G0, cap, ld, 50, exact=False)
+    assert info.status == 2 and not d.any()
+
+
+def test_allocation_host_errors():
+    from paper_2605_07114_b200 import hora
+    N, ld = 10, 8
+    c = torch.zeros(N, dtype=torch.int32, device="cuda")
+    delta = torch.zeros(N, dtype=torch.int32, device="cuda")
+    G = torch.zeros(N, dtype=torch.int32, device="cuda")
+    ws = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(hora.HoraError) as e:
+        hora.hora_allocate(None, None, 1.0, 1.0, c, 4, None, ld, N, ld, None, 5, 0, delta, G, None, None, ws)
+    assert e.value.code == hora.ERR_WORKSPACE
+    with pytest.raises(hora.HoraError) as e:
+        hora.hora_allocate(None, None, 1.0, 1.0, c, 4, None, ld, N, ld, None, -5, 0, delta, G, None, None, ws)
+    assert e.value.code == hora.ERR_INVALID_ARG
+
+
+def test_allocation_is_reproducible():
+    gu = _util()
+    w = wl.make("cfg4", 4096)
+    a = gu.gpu_allocate(w.alpha, w.beta, 1.0, 1.0, w.c, w.G0, w.cap, w.ld, w.B, exact=False)
+    b = gu.gpu_allocate(w.alpha, w.beta, 1.0, 1.0, w.c, w.G0, w.cap, w.ld, w.B, exact=False)
+    np.testing.assert_array_equal(a[0], b[0])
+    assert np.float64(a[3].objective).view(np.uint64) == np.float64(b[3].objective).view(np.uint64)
+
+
+# ------------------------------------------------------------------------------------- advantages
+def ragged(rng, n_groups, sizes, values):
+    sizes = rng.choice(sizes, n_groups)
+    off = np.zeros(n_groups + 1, np.int64)
+    np.cumsum(sizes, out=off[1:])
+    return rng.choice(values, int(off[-1])).astype(np.float32), off
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("ddof", [0, 1])
+@pytest.mark.parametrize("eps", [0.0, 1e-6])
+def test_group_advantage_matches_oracle(mode, ddof, eps):
+    gu = _util()
+    rng = np.random.default_rng(mode * 4 + ddof * 2 + (eps > 0))
+    sizes = [0, 1, 2, 3, 8, 9, 31, 32, 33, 64, 100, 264, 288, 289, 500, 3000]
+    for values in ([0.0, 1.0], [0.0, 0.5, 1.0], [1.0], [-3.25, 0.1, 7.0, 1e3]):
+        r, off = ragged(rng, 700, sizes, values)
+        got, status = gu.gpu_advantage(r, off, mode, np.float32(eps), ddof)
+        exp = orc.group_advantage(r, off, mode, float(np.float32(eps)), ddof)
+        assert status == 0
+        tol = 1e-5 * max(1.0, float(np.abs(values).max()))
+        np.testing.assert_allclose(got, exp, rtol=0, atol=tol)
+        if len(values) == 1:
+            assert not got.any()                                  # zero-variance groups give zero advantage
+
+
+def test_group_advantage_on_workload_groups():
+    gu = _util()
+    for name, N in (("cfg1", None), ("cfg2", None), ("cfg5", 20000)):
+        w = wl.make(name, N)
+        d_o = gu.oracle_allocate(w)[0]
+        off = w.group_offsets(d_o)
+        r = w.rewards(off)
+        got, status = gu.gpu_advantage(r, off, w.adv_mode, np.float32(w.eps), w.ddof)
+        exp = orc.group_advantage(r, off, w.adv_mode, float(np.float32(w.eps)), w.ddof)
+        assert status == 0
+        np.testing.assert_allclose(got, exp, rtol=0, atol=1e-5)
+        sums = np.add.reduceat(got.astype(np.float64), off[:-1])
+        assert np.abs(sums).max() < 1e-3                          # advantages of a group sum to zero
+
+
+def test_group_advantage_flags_decreasing_offsets():
+    gu = _util()
+    r = np.ones(10, np.float32)
+    off = np.array([0, 5, 3, 10], np.int64)
+    got, status = gu.gpu_advantage(r, off, 0, np.float32(0), 0)
+    assert status == 2
+
+
+# -------------------------------------------------------------------------------------- broadcast
+@pytest.mark.parametrize("misalign", [0, 1, 3])
+@pytest.mark.parametrize("kind", ["paper", "short", "zeros", "tiny_many", "one_long", "single_token"])
+def test_token_broadcast_bitwise(kind, misalign):
+    gu = _util()
+    rng = np.random.default_rng(len(kind) + misalign)
+    if kind == "paper":
+        lens = rng.integers(32, 2049, 5000)
+    elif kind == "short":
+        lens = rng.integers(0, 9, 40000)
+    elif kind == "zeros":
+        lens = np.where(rng.random(30000) < 0.7, 0, rng.integers(1, 300, 30000))
+    elif kind == "tiny_many":
+        lens = np.concatenate([np.ones(5000, np.int64), np.zeros(4000, np.int64), rng.integers(0, 3, 200000),
+                               rng.integers(1000, 5000, 50)])
+    elif kind == "one_long":
+        lens = np.array([0, 0, 1234567, 0])
+    else:
+        lens = np.array([1])
+    R = len(lens)
+    adv = rng.standard_normal(R).astype(np.float32)
+    off = np.zeros(R + 1, np.int64)
+    np.cumsum(lens, out=off[1:])
+    got = gu.gpu_broadcast(adv, off, misalign=misalign)
+    exp = orc.token_broadcast(adv, off)
+    np.testing.assert_array_equal(got.view(np.uint32), exp.view(np.uint32))
+
+
+def test_token_broadcast_on_cfg3_layout_scaled():
+    gu = _util()
+    w = wl.make("cfg3", 1024)
+    d_o = gu.oracle_allocate(w)[0]
+    off = w.group_offsets(d_o)
+    r = w.rewards(off)
+    adv = orc.group_advantage(r, off, w.adv_mode, float(np.float32(w.eps)), w.ddof)
+    tok = w.token_offsets(len(r))
+    got = gu.gpu_broadcast(adv, tok)
+    np.testing.assert_array_equal(got.view(np.uint32), orc.token_broadcast(adv, tok).view(np.uint32))
