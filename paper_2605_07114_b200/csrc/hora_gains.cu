@@ -19,10 +19,18 @@ constexpr int kTile = 8;                      // consecutive rows a warp takes a
 // (one coalesced load per array) ONE TILE AHEAD, so that latency is hidden behind the arithmetic of the
 // current tile; the values reach the other lanes by shuffles.
 template <int E, bool VEC2>
-__global__ void __launch_bounds__(kGainsWarps *kWarp, 4)
+__global__ void __launch_bounds__(kGainsWarps *kWarp, 3)
 gains_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
              const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
              int64_t N, int32_t ld, double *__restrict__ gains, int32_t *status_dev) {
+    // Staging slab: a lane produces E consecutive entries, but a store instruction should cover one
+    // contiguous 512-byte run of the row (full 32-byte sectors; 16-byte pieces at a 64-byte stride cost
+    // twice the L1-to-L2 traffic).  Pairs go through shared memory with an XOR swizzle on the 16-byte
+    // chunk index that keeps both the lane-major writes and the row-major reads free of bank conflicts.
+    constexpr int P = E / 2;                              // 16-byte chunks per lane
+    constexpr bool kStaged = VEC2 && (P > 1);
+    __shared__ double2 s_stage[kStaged ? kGainsWarps * kWarp * P : 1];
+    double2 *slab = s_stage + (kStaged ? (threadIdx.x >> 5) * kWarp * P : 0);
     const int lane = lane_id();
     const int64_t n_tiles = (N + kTile - 1) / kTile;
     const int64_t tile0 = (int64_t)blockIdx.x * kGainsWarps + (threadIdx.x >> 5);
@@ -80,12 +88,26 @@ gains_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, 
                     pm *= x + (double)(m + 1);
                     const double g1 = (k + m + 1 < capi) ? pm * S[m + 2] : 0.0;
                     if (m + 2 < E) pm *= x + (double)(m + 2);
-                    if (VEC2) {
+                    if (kStaged) {
+                        const int ch = lane * P + (m >> 1);
+                        slab[ch ^ ((ch >> 3) & (P - 1))] = make_double2(g0, g1);
+                    } else if (VEC2) {
                         if (k + m < ld) *reinterpret_cast<double2 *>(out + k + m) = make_double2(g0, g1);
                     } else {
                         if (k + m < ld) out[k + m] = g0;
                         if (k + m + 1 < ld) out[k + m + 1] = g1;
                     }
+                }
+                if (kStaged) {
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < P; ++q) {
+                        const int ch = q * kWarp + lane;
+                        const double2 v = slab[ch ^ ((ch >> 3) & (P - 1))];
+                        const int32_t col = k0 + 2 * ch;
+                        if (col < ld) *reinterpret_cast<double2 *>(out + col) = v;
+                    }
+                    __syncwarp();
                 }
             }
         }
@@ -97,7 +119,7 @@ static hora_status_t launch_e(const double *alpha, const double *beta, double al
                               int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N, int32_t ld, double *gains,
                               int32_t *status_dev, cudaStream_t stream) {
     const int64_t tiles = (N + kTile - 1) / kTile;
-    const int grid = clamp_grid((tiles + kGainsWarps - 1) / kGainsWarps, 4);
+    const int grid = clamp_grid((tiles + kGainsWarps - 1) / kGainsWarps, 3);
     const bool vec2 = (ld % 2 == 0) && ((reinterpret_cast<uintptr_t>(gains) & 15u) == 0);
     if (vec2)
         gains_kernel<E, true><<<grid, kGainsWarps * kWarp, 0, stream>>>(alpha, beta, alpha0, beta0, c, G0, cap,
