@@ -6,10 +6,12 @@
 //
 //   level 0   one coalesced read of the whole matrix (a warp per row), histogram of the top 13 bits
 //             in shared memory, merged into a global histogram; the last CTA to finish locates the
-//             digit that holds the B-th largest key.
-//   level 1   a thread per row: because a row is non-increasing, its keys with the selected top digit
-//             form ONE contiguous segment, found by binary search; only that segment is read again
-//             and its next digit histogrammed.  The segment [p_hi, p_lo) is kept per row.
+//             digit that holds the B-th largest key.  The same pass writes a 2-byte sketch of every
+//             8th key (its top 16 bits), 3 % of the matrix in size.
+//   level 1   a warp per row: because a row is non-increasing, its keys with the selected top digit
+//             form ONE contiguous segment; the sketch brackets it to within 8 keys on each side, so
+//             only that segment is read again (coalesced) and its next digit histogrammed.  The
+//             segment [p_hi, p_lo) is kept per row.
 //   level 2-4 a thread per row narrows its segment by the digit just selected and histograms the next.
 //   sum       narrows by the last digit: p_hi = #keys > lambda, p_lo - p_hi = #keys == lambda; block sums
 //             and their scan give n_above, n_tied and the exclusive prefixes over prompts.
@@ -61,6 +63,8 @@ struct Workspace {
     AllocHeader *hdr;
     unsigned long long *hist;          // [kLevels][kBins]
     int2 *rowstate;                    // [N] (p_hi, p_lo)
+    uint16_t *sketch;                  // [N][sk_ld] top 16 bits of keys 0, 8, 16, ... of each row
+    int32_t sk_ld;
     long long *bsum_hi, *bsum_t;       // [NB] block sums, overwritten by exclusive prefixes
     double *objpart;                   // [NB]
     unsigned long long *tkeys, *tcounts;   // [kTypeSlots]
@@ -81,6 +85,8 @@ static Workspace carve(void *base, int64_t N, int32_t ld, bool need_gains, bool 
     w.hdr = reinterpret_cast<AllocHeader *>(take(sizeof(AllocHeader)));
     w.hist = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kLevels * kBins));
     w.rowstate = reinterpret_cast<int2 *>(take(sizeof(int2) * (size_t)N));
+    w.sk_ld = ((ld + 7) / 8 + 7) & ~7;
+    w.sketch = reinterpret_cast<uint16_t *>(take(sizeof(uint16_t) * (size_t)N * (size_t)w.sk_ld));
     w.bsum_hi = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
     w.bsum_t = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
     w.objpart = reinterpret_cast<double *>(take(sizeof(double) * (size_t)NB));
@@ -163,15 +169,16 @@ __device__ __forceinline__ void flush_hist(const unsigned int *s_hist, unsigned 
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Level 0: the one full read.  A warp per row, a lane takes E consecutive keys (the row is sorted, so a
-// lane's keys fall into few bins and are merged before they touch shared memory).  Also validates the
-// inputs and sums the caps.
+// Level 0: the one full read.  A warp per row, a lane takes E consecutive keys.  The row is sorted, so a
+// lane's keys usually fall into one bin (one shared-memory atomic for all E); otherwise runs of equal
+// bins are merged first.  The pass also checks that the row is finite, non-negative and non-increasing
+// (first key below +inf, every key <= its predecessor, compared as unsigned integers), sums the caps,
+// and writes the sketch: the top 16 bits of keys 0, 8, 16, ... (zero beyond the cap).
 template <int E, bool VEC2>
 __global__ void __launch_bounds__(kSelThreads)
-select_level0(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
-              const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
-              int64_t N, int32_t ld, const double *__restrict__ gains, int64_t B, AllocHeader *hdr,
-              unsigned long long *hist) {
+select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
+              const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist,
+              uint16_t *__restrict__ sketch, int32_t sk_ld) {
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
@@ -182,47 +189,61 @@ select_level0(const double *__restrict__ alpha, const double *__restrict__ beta,
     long long capsum = 0;
     bool bad = false;
     for (int64_t row = warp0; row < N; row += stride) {
-        const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row);
-        bad |= !p.ok;
-        if (lane == 0) capsum += p.cap;
+        int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
+        if (capi < 0 || capi > ld) { bad = true; capi = 0; }
+        if (lane == 0) capsum += capi;
         const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-        unsigned long long prev_last = ~0ull;                  // last key of the previous lane / chunk
-        for (int32_t k0 = 0; k0 < p.cap; k0 += kWarp * E) {
+        uint16_t *sk = sketch + row * (int64_t)sk_ld;
+        unsigned long long prev_last = kKeyInf - 1;            // the first key must be finite
+        for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E) {
             const int32_t k = k0 + lane * E;
+            if (k0 >= capi) {                                  // nothing but padding from here on
+                if ((k & 7) == 0 && k < ld) sk[k >> 3] = 0;
+                continue;
+            }
             unsigned long long key[E];
             if (VEC2) {
 #pragma unroll
                 for (int m = 0; m < E; m += 2) {
                     ulonglong2 v = make_ulonglong2(0ull, 0ull);
-                    if (k + m < p.cap) v = __ldg(reinterpret_cast<const ulonglong2 *>(keys + k + m));
+                    if (k + m < capi) v = __ldg(reinterpret_cast<const ulonglong2 *>(keys + k + m));
                     key[m] = v.x;
-                    key[m + 1] = v.y;
+                    key[m + 1] = (k + m + 1 < capi) ? v.y : 0ull;
                 }
             } else {
 #pragma unroll
-                for (int m = 0; m < E; ++m) key[m] = (k + m < p.cap) ? __ldg(keys + k + m) : 0ull;
+                for (int m = 0; m < E; ++m) key[m] = (k + m < capi) ? __ldg(keys + k + m) : 0ull;
             }
+            // keys past the cap were replaced by 0, which is below every valid key: the order check and the
+            // histogram below can treat a full and a ragged chunk alike, except for the count
             unsigned long long before = __shfl_up_sync(kFull, key[E - 1], 1);
             if (lane == 0) before = prev_last;
             prev_last = __shfl_sync(kFull, key[E - 1], kWarp - 1);
-            int run_bin = -1;
-            unsigned int run_len = 0;
+            bad |= key[0] > before;
 #pragma unroll
-            for (int m = 0; m < E; ++m) {
-                if (k + m < p.cap) {
-                    bad |= (key[m] >= kKeyInf) | (key[m] > before);
-                    before = key[m];
-                    const int bin = (int)(key[m] >> 51) & (kBins - 1);
-                    if (bin == run_bin) {
-                        ++run_len;
-                    } else {
-                        if (run_len) atomicAdd(&s_hist[run_bin], run_len);
-                        run_bin = bin;
-                        run_len = 1;
+            for (int m = 1; m < E; ++m) bad |= key[m] > key[m - 1];
+            if ((k & 7) == 0 && k < ld) sk[k >> 3] = (uint16_t)(key[0] >> 48);
+            const int valid = capi - k < E ? (capi - k > 0 ? capi - k : 0) : E;   // keys of this lane below the cap
+            if (valid == E && (key[0] >> 51) == (key[E - 1] >> 51)) {
+                atomicAdd(&s_hist[(int)(key[0] >> 51)], (unsigned int)E);
+            } else if (valid > 0) {
+                int run_bin = (int)(key[0] >> 51);
+                unsigned int run_len = 1;
+#pragma unroll
+                for (int m = 1; m < E; ++m) {
+                    if (m < valid) {
+                        const int bin = (int)(key[m] >> 51);
+                        if (bin == run_bin) {
+                            ++run_len;
+                        } else {
+                            atomicAdd(&s_hist[run_bin], run_len);
+                            run_bin = bin;
+                            run_len = 1;
+                        }
                     }
                 }
+                atomicAdd(&s_hist[run_bin], run_len);
             }
-            if (run_len) atomicAdd(&s_hist[run_bin], run_len);
         }
     }
     if (bad) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);
@@ -243,13 +264,63 @@ select_level0(const double *__restrict__ alpha, const double *__restrict__ beta,
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Levels 1..4: a thread per row (grid-stride).  Level 1 finds the row's segment by binary search; later
-// levels narrow the stored segment by the digit selected one level up.  The keys that remain are
-// histogrammed on the current level's digit.
+// Level 1: a warp per row.  The sketch says, for every group of 8 keys, which bin its first (largest) key
+// falls in.  With d the digit selected at level 0: groups whose first key is above bin d form a prefix
+// of G1 groups, groups whose first key is in or above bin d a prefix of G2 >= G1 groups.  Every key in
+// bin d therefore sits in groups G1-1 .. G2-1, and so does the boundary between "above" and "in" the
+// bin; only those groups are read (coalesced), counted and histogrammed on the next digit.
 __global__ void __launch_bounds__(kSelThreads)
-select_refine(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
-              const double *__restrict__ gains, int level, AllocHeader *hdr, unsigned long long *hist_all,
-              int2 *__restrict__ rowstate) {
+select_level1(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
+              const double *__restrict__ gains, AllocHeader *hdr, unsigned long long *hist1,
+              const uint16_t *__restrict__ sketch, int32_t sk_ld, int2 *__restrict__ rowstate) {
+    __shared__ unsigned int s_hist[kBins];
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    if (*(volatile int32_t *)&hdr->status != 0) return;
+    for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
+    __syncthreads();
+    const int lane = lane_id();
+    const int d0 = hdr->sel_digit[0];
+    const int64_t warp0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5);
+    const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
+    for (int64_t row = warp0; row < N; row += stride) {
+        int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
+        capi = capi < 0 ? 0 : (capi > ld ? ld : capi);
+        const int n_groups = (capi + 7) >> 3;
+        const uint16_t *sk = sketch + row * (int64_t)sk_ld;
+        int G1 = 0, G2 = 0;
+        for (int g0 = 0; g0 < n_groups; g0 += kWarp) {
+            const int g = g0 + lane;
+            const int dig = g < n_groups ? (int)(__ldg(sk + g) >> 3) : -1;
+            G1 += __popc(__ballot_sync(kFull, dig > d0));
+            G2 += __popc(__ballot_sync(kFull, dig >= d0));
+        }
+        const int32_t lo = G1 > 0 ? (G1 - 1) << 3 : 0;          // first key that may not be above the bin
+        int32_t hi = G2 << 3;                                   // one past the last key that may be in the bin
+        if (hi > capi) hi = capi;
+        const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+        int32_t n_gt = 0, n_eq = 0;
+        for (int32_t j0 = lo; j0 < hi; j0 += kWarp) {
+            const int32_t j = j0 + lane;
+            const unsigned long long key = j < hi ? __ldg(keys + j) : 0ull;
+            const int dig = j < hi ? (int)(key >> 51) : -1;
+            n_gt += __popc(__ballot_sync(kFull, dig > d0));
+            const bool in = dig == d0;
+            n_eq += __popc(__ballot_sync(kFull, in));
+            if (in) atomicAdd(&s_hist[(key >> 38) & (kBins - 1)], 1u);
+        }
+        if (lane == 0) rowstate[row] = make_int2(lo + n_gt, lo + n_gt + n_eq);
+    }
+    __syncthreads();
+    flush_hist(s_hist, hist1, kBins);
+    if (last_block(&hdr->ticket[1])) find_digit(hdr, hist1, 1, s_warp);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Levels 2..4: a thread per row (grid-stride) narrows the stored segment by the digit selected one level
+// up; the keys that remain are histogrammed on the current level's digit.
+__global__ void __launch_bounds__(kSelThreads)
+select_refine(int64_t N, int32_t ld, const double *__restrict__ gains, int level, AllocHeader *hdr,
+              unsigned long long *hist_all, int2 *__restrict__ rowstate) {
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     if (*(volatile int32_t *)&hdr->status != 0) return;
@@ -262,22 +333,9 @@ select_refine(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
     const int64_t stride = (int64_t)gridDim.x * kSelThreads;
     for (int64_t row = (int64_t)blockIdx.x * kSelThreads + threadIdx.x; row < N; row += stride) {
         const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-        int32_t p_hi, p_end;
-        if (level == 1) {
-            int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
-            capi = capi < 0 ? 0 : (capi > ld ? ld : capi);
-            int32_t lo = 0, hi = capi;                 // first index whose top digit is <= d_prev
-            while (lo < hi) {
-                const int32_t mid = (lo + hi) >> 1;
-                if ((__ldg(keys + mid) >> shift_prev) > d_prev) lo = mid + 1; else hi = mid;
-            }
-            p_hi = lo;
-            p_end = capi;
-        } else {
-            const int2 st = rowstate[row];
-            p_hi = st.x;
-            p_end = st.y;
-        }
+        const int2 st = rowstate[row];
+        const int32_t p_hi = st.x, p_end = st.y;
+        if (p_hi >= p_end) continue;                   // nothing of this row is left in the threshold bin
         int32_t p = p_hi, new_hi = p_hi;
         while (p < p_end) {
             const unsigned long long key = __ldg(keys + p);
@@ -291,7 +349,7 @@ select_refine(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
             }
             ++p;
         }
-        rowstate[row] = make_int2(new_hi, p);
+        if (new_hi != p_hi || p != p_end) rowstate[row] = make_int2(new_hi, p);
     }
     __syncthreads();
     flush_hist(s_hist, hist_all + (size_t)level * kBins, bins);
@@ -494,8 +552,11 @@ exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ t
 // ---------------------------------------------------------------------------------------------------
 // Block sums of (p_hi, tied) in prompt order, and their exclusive scan by the last CTA.
 //   mode 0: rowstate is final    mode 1: narrow by the last digit first    mode 2: apply the exact labels first
+// With `validate` the priors and counts of every prompt are checked here (a thread per row, coalesced).
 __global__ void __launch_bounds__(kSelThreads)
-select_sum(int64_t N, int32_t ld, const double *__restrict__ gains, int mode, int64_t B, AllocHeader *hdr,
+select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
+           const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar, int validate,
+           int64_t N, int32_t ld, const double *__restrict__ gains, int mode, int64_t B, AllocHeader *hdr,
            int2 *__restrict__ rowstate, const int32_t *__restrict__ rowslot, const int32_t *__restrict__ tlabel,
            long long *bsum_hi, long long *bsum_t, int64_t NB) {
     __shared__ long long s_warp[kSelThreads / kWarp];
@@ -508,6 +569,8 @@ select_sum(int64_t N, int32_t ld, const double *__restrict__ gains, int mode, in
         for (int q = 0; q < kRowsPerBlock / kSelThreads; ++q) {
             const int64_t row = row0 + q * kSelThreads + threadIdx.x;
             if (row >= N) break;
+            if (validate && !load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row).ok)
+                raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);   // seen by the kernels that follow
             int2 st = rowstate[row];
             if (mode == 1) {
                 const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
@@ -678,15 +741,12 @@ __global__ void write_empty(int64_t B, int64_t *offsets, hora_alloc_info *info) 
 }
 
 template <int E>
-static void launch_level0(bool vec2, int grid, cudaStream_t s, const double *alpha, const double *beta, double alpha0,
-                          double beta0, const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N,
-                          int32_t ld, const double *gains, int64_t B, AllocHeader *hdr, unsigned long long *hist) {
+static void launch_level0(bool vec2, int grid, cudaStream_t s, const int32_t *cap, int32_t cap_scalar, int64_t N,
+                          int32_t ld, const double *gains, int64_t B, const Workspace &w) {
     if (vec2)
-        select_level0<E, true><<<grid, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
-                                                            gains, B, hdr, hist);
+        select_level0<E, true><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist, w.sketch, w.sk_ld);
     else
-        select_level0<E, false><<<grid, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
-                                                             gains, B, hdr, hist);
+        select_level0<E, false><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist, w.sketch, w.sk_ld);
 }
 
 }  // namespace hora
@@ -739,27 +799,32 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     const int rows_per_cta = kSelThreads / kWarp;
     const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 6);
     if (ld > 128)
-        launch_level0<8>(vec2, grid0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist);
+        launch_level0<8>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
     else if (ld > 64)
-        launch_level0<4>(vec2, grid0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist);
+        launch_level0<4>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
     else
-        launch_level0<2>(vec2, grid0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist);
-    const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 4);
+        launch_level0<2>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
+    const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     if (B > 0) {
-        for (int level = 1; level < kLevels; ++level)
-            select_refine<<<grid_rows, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, level, w.hdr, w.hist, w.rowstate);
-        select_sum<<<(int)NB, kSelThreads, 0, s>>>(N, ld, gains, 1, B, w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi,
+        select_level1<<<grid0, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, w.hdr, w.hist + kBins, w.sketch, w.sk_ld,
+                                                    w.rowstate);
+        for (int level = 2; level < kLevels; ++level)
+            select_refine<<<grid_rows, kSelThreads, 0, s>>>(N, ld, gains, level, w.hdr, w.hist, w.rowstate);
+        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 1,
+                                                   N, ld, gains, 1, B, w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi,
                                                    w.bsum_t, NB);
         if (exact) {
             exact_collect<<<grid_rows, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
                                                             gains, w.hdr, w.rowstate, w.rowslot, w.tkeys, w.tcounts);
             exact_rank<<<1, 1024, 0, s>>>(B, w.hdr, w.tkeys, w.tcounts, w.tlabel);
-            select_sum<<<(int)NB, kSelThreads, 0, s>>>(N, ld, gains, 2, B, w.hdr, w.rowstate, w.rowslot, w.tlabel,
+            select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 0,
+                                                       N, ld, gains, 2, B, w.hdr, w.rowstate, w.rowslot, w.tlabel,
                                                        w.bsum_hi, w.bsum_t, NB);
         }
     } else {
         if (cudaMemsetAsync(w.rowstate, 0, sizeof(int2) * (size_t)N, s) != cudaSuccess) return HORA_ERR_CUDA;
-        select_sum<<<(int)NB, kSelThreads, 0, s>>>(N, ld, gains, 0, B, w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi,
+        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 1,
+                                                   N, ld, gains, 0, B, w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi,
                                                    w.bsum_t, NB);
     }
     select_out<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, flags, w.hdr,
