@@ -169,11 +169,56 @@ __device__ __forceinline__ void flush_hist(const unsigned int *s_hist, unsigned 
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Level 0: the one full read.  A warp per row, a lane takes E consecutive keys.  The row is sorted, so a
-// lane's keys usually fall into one bin (one shared-memory atomic for all E); otherwise runs of equal
-// bins are merged first.  The pass also checks that the row is finite, non-negative and non-increasing
-// (first key below +inf, every key <= its predecessor, compared as unsigned integers), sums the caps,
-// and writes the sketch: the top 16 bits of keys 0, 8, 16, ... (zero beyond the cap).
+// Level 0: the one full read.  The matrix is cut into items of 32*E consecutive keys of one row; a warp
+// takes one item at a time and a lane E consecutive keys of it, and the loads of the NEXT item are
+// issued before the current one is processed.  The row is sorted, so a lane's keys usually fall into
+// one bin (one shared-memory atomic for all E); otherwise each key adds itself.  The pass also checks
+// that the row is finite, non-negative and non-increasing (first key below +inf, every key <= its
+// predecessor, compared as unsigned integers), sums the caps, and writes the sketch: the top 16 bits of
+// keys 0, 8, 16, ... (zero beyond the cap).
+template <int E, bool VEC2>
+struct Level0Item {
+    unsigned long long key[E];
+    unsigned long long before;     // lane 0 only: the key just before this item (or the largest finite key)
+    int32_t capi;
+};
+
+template <int E, bool VEC2>
+__device__ __forceinline__ Level0Item<E, VEC2> level0_fetch(const int32_t *__restrict__ cap, int32_t cap_scalar,
+                                                            int64_t n_items, int32_t items_per_row, int32_t ld,
+                                                            const double *__restrict__ gains, int64_t item, int lane,
+                                                            bool *bad) {
+    Level0Item<E, VEC2> it;
+#pragma unroll
+    for (int m = 0; m < E; ++m) it.key[m] = 0ull;
+    it.before = kKeyInf - 1;
+    it.capi = 0;
+    if (item >= n_items) return it;
+    const int64_t row = items_per_row == 1 ? item : item / items_per_row;
+    const int32_t k0 = (int32_t)(item - row * items_per_row) * (kWarp * E);
+    int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
+    if (capi < 0 || capi > ld) { *bad = true; capi = 0; }
+    it.capi = capi;
+    const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+    const int32_t k = k0 + lane * E;
+    if (VEC2) {
+#pragma unroll
+        for (int m = 0; m < E; m += 2) {
+            if (k + m < capi) {
+                const ulonglong2 v = __ldg(reinterpret_cast<const ulonglong2 *>(keys + k + m));
+                it.key[m] = v.x;
+                it.key[m + 1] = (k + m + 1 < capi) ? v.y : 0ull;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int m = 0; m < E; ++m)
+            if (k + m < capi) it.key[m] = __ldg(keys + k + m);
+    }
+    if (lane == 0 && k0 > 0 && k0 < capi) it.before = __ldg(keys + k0 - 1);
+    return it;
+}
+
 template <int E, bool VEC2>
 __global__ void __launch_bounds__(kSelThreads)
 select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
@@ -184,66 +229,35 @@ select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
     __syncthreads();
     const int lane = lane_id();
-    const int64_t warp0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5);
+    const int32_t items_per_row = (ld + kWarp * E - 1) / (kWarp * E);
+    const int64_t n_items = N * items_per_row;
+    const int64_t item0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5);
     const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
     long long capsum = 0;
     bool bad = false;
-    for (int64_t row = warp0; row < N; row += stride) {
-        int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
-        if (capi < 0 || capi > ld) { bad = true; capi = 0; }
-        if (lane == 0) capsum += capi;
-        const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-        uint16_t *sk = sketch + row * (int64_t)sk_ld;
-        unsigned long long prev_last = kKeyInf - 1;            // the first key must be finite
-        for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E) {
-            const int32_t k = k0 + lane * E;
-            if (k0 >= capi) {                                  // nothing but padding from here on
-                if ((k & 7) == 0 && k < ld) sk[k >> 3] = 0;
-                continue;
-            }
-            unsigned long long key[E];
-            if (VEC2) {
+    Level0Item<E, VEC2> nxt = level0_fetch<E, VEC2>(cap, cap_scalar, n_items, items_per_row, ld, gains, item0, lane, &bad);
+    for (int64_t item = item0; item < n_items; item += stride) {
+        const Level0Item<E, VEC2> cur = nxt;
+        nxt = level0_fetch<E, VEC2>(cap, cap_scalar, n_items, items_per_row, ld, gains, item + stride, lane, &bad);
+        const int64_t row = items_per_row == 1 ? item : item / items_per_row;
+        const int32_t k0 = (int32_t)(item - row * items_per_row) * (kWarp * E);
+        const int32_t k = k0 + lane * E;
+        if (lane == 0 && k0 == 0) capsum += cur.capi;
+        // keys past the cap were replaced by 0, which is below every valid key, so a ragged item needs no
+        // special case in the order check
+        unsigned long long before = __shfl_up_sync(kFull, cur.key[E - 1], 1);
+        if (lane == 0) before = cur.before;
+        bad |= cur.key[0] > before;
 #pragma unroll
-                for (int m = 0; m < E; m += 2) {
-                    ulonglong2 v = make_ulonglong2(0ull, 0ull);
-                    if (k + m < capi) v = __ldg(reinterpret_cast<const ulonglong2 *>(keys + k + m));
-                    key[m] = v.x;
-                    key[m + 1] = (k + m + 1 < capi) ? v.y : 0ull;
-                }
-            } else {
+        for (int m = 1; m < E; ++m) bad |= cur.key[m] > cur.key[m - 1];
+        if ((k & 7) == 0 && k < ld) sketch[row * (int64_t)sk_ld + (k >> 3)] = (uint16_t)(cur.key[0] >> 48);
+        const int valid = cur.capi - k;                       // keys of this lane below the cap (may be <= 0 or > E)
+        if (valid >= E && (cur.key[0] >> 51) == (cur.key[E - 1] >> 51)) {
+            atomicAdd(&s_hist[(int)(cur.key[0] >> 51)], (unsigned int)E);
+        } else {
 #pragma unroll
-                for (int m = 0; m < E; ++m) key[m] = (k + m < capi) ? __ldg(keys + k + m) : 0ull;
-            }
-            // keys past the cap were replaced by 0, which is below every valid key: the order check and the
-            // histogram below can treat a full and a ragged chunk alike, except for the count
-            unsigned long long before = __shfl_up_sync(kFull, key[E - 1], 1);
-            if (lane == 0) before = prev_last;
-            prev_last = __shfl_sync(kFull, key[E - 1], kWarp - 1);
-            bad |= key[0] > before;
-#pragma unroll
-            for (int m = 1; m < E; ++m) bad |= key[m] > key[m - 1];
-            if ((k & 7) == 0 && k < ld) sk[k >> 3] = (uint16_t)(key[0] >> 48);
-            const int valid = capi - k < E ? (capi - k > 0 ? capi - k : 0) : E;   // keys of this lane below the cap
-            if (valid == E && (key[0] >> 51) == (key[E - 1] >> 51)) {
-                atomicAdd(&s_hist[(int)(key[0] >> 51)], (unsigned int)E);
-            } else if (valid > 0) {
-                int run_bin = (int)(key[0] >> 51);
-                unsigned int run_len = 1;
-#pragma unroll
-                for (int m = 1; m < E; ++m) {
-                    if (m < valid) {
-                        const int bin = (int)(key[m] >> 51);
-                        if (bin == run_bin) {
-                            ++run_len;
-                        } else {
-                            atomicAdd(&s_hist[run_bin], run_len);
-                            run_bin = bin;
-                            run_len = 1;
-                        }
-                    }
-                }
-                atomicAdd(&s_hist[run_bin], run_len);
-            }
+            for (int m = 0; m < E; ++m)
+                if (m < valid) atomicAdd(&s_hist[(int)(cur.key[m] >> 51)], 1u);
         }
     }
     if (bad) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);
@@ -269,6 +283,8 @@ select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
 // of G1 groups, groups whose first key is in or above bin d a prefix of G2 >= G1 groups.  Every key in
 // bin d therefore sits in groups G1-1 .. G2-1, and so does the boundary between "above" and "in" the
 // bin; only those groups are read (coalesced), counted and histogrammed on the next digit.
+constexpr int kL1Rows = 4;      // rows a warp works on at once: their loads are in flight together
+
 __global__ void __launch_bounds__(kSelThreads)
 select_level1(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
               const double *__restrict__ gains, AllocHeader *hdr, unsigned long long *hist1,
@@ -282,33 +298,80 @@ select_level1(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
     const int d0 = hdr->sel_digit[0];
     const int64_t warp0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5);
     const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
-    for (int64_t row = warp0; row < N; row += stride) {
-        int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
-        capi = capi < 0 ? 0 : (capi > ld ? ld : capi);
-        const int n_groups = (capi + 7) >> 3;
-        const uint16_t *sk = sketch + row * (int64_t)sk_ld;
-        int G1 = 0, G2 = 0;
-        for (int g0 = 0; g0 < n_groups; g0 += kWarp) {
-            const int g = g0 + lane;
-            const int dig = g < n_groups ? (int)(__ldg(sk + g) >> 3) : -1;
-            G1 += __popc(__ballot_sync(kFull, dig > d0));
-            G2 += __popc(__ballot_sync(kFull, dig >= d0));
+    const int64_t n_batches = (N + kL1Rows - 1) / kL1Rows;
+    for (int64_t batch = warp0; batch < n_batches; batch += stride) {
+        int32_t capi[kL1Rows], lo[kL1Rows], hi[kL1Rows];
+        // ---- sketches of all rows of the batch (independent loads), then their brackets ----
+#pragma unroll
+        for (int r = 0; r < kL1Rows; ++r) {
+            const int64_t row = batch * kL1Rows + r;
+            capi[r] = 0;
+            if (row < N) {
+                const int32_t cp = cap ? __ldg(cap + row) : cap_scalar;
+                capi[r] = cp < 0 ? 0 : (cp > ld ? ld : cp);
+            }
         }
-        const int32_t lo = G1 > 0 ? (G1 - 1) << 3 : 0;          // first key that may not be above the bin
-        int32_t hi = G2 << 3;                                   // one past the last key that may be in the bin
-        if (hi > capi) hi = capi;
-        const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-        int32_t n_gt = 0, n_eq = 0;
-        for (int32_t j0 = lo; j0 < hi; j0 += kWarp) {
-            const int32_t j = j0 + lane;
-            const unsigned long long key = j < hi ? __ldg(keys + j) : 0ull;
-            const int dig = j < hi ? (int)(key >> 51) : -1;
-            n_gt += __popc(__ballot_sync(kFull, dig > d0));
-            const bool in = dig == d0;
-            n_eq += __popc(__ballot_sync(kFull, in));
-            if (in) atomicAdd(&s_hist[(key >> 38) & (kBins - 1)], 1u);
+        if (ld <= 8 * kWarp) {                                   // one sketch entry per lane covers the row
+            int dig[kL1Rows];
+#pragma unroll
+            for (int r = 0; r < kL1Rows; ++r) {
+                const int64_t row = batch * kL1Rows + r;
+                const int n_groups = (capi[r] + 7) >> 3;
+                dig[r] = lane < n_groups ? (int)(__ldg(sketch + row * (int64_t)sk_ld + lane) >> 3) : -1;
+            }
+#pragma unroll
+            for (int r = 0; r < kL1Rows; ++r) {
+                const int G1 = __popc(__ballot_sync(kFull, dig[r] > d0));
+                const int G2 = __popc(__ballot_sync(kFull, dig[r] >= d0));
+                lo[r] = G1 > 0 ? (G1 - 1) << 3 : 0;
+                hi[r] = (G2 << 3) > capi[r] ? capi[r] : (G2 << 3);
+            }
+        } else {
+#pragma unroll
+            for (int r = 0; r < kL1Rows; ++r) {
+                const int64_t row = batch * kL1Rows + r;
+                const int n_groups = (capi[r] + 7) >> 3;
+                int G1 = 0, G2 = 0;
+                for (int g0 = 0; g0 < n_groups; g0 += kWarp) {
+                    const int g = g0 + lane;
+                    const int dig = g < n_groups ? (int)(__ldg(sketch + row * (int64_t)sk_ld + g) >> 3) : -1;
+                    G1 += __popc(__ballot_sync(kFull, dig > d0));
+                    G2 += __popc(__ballot_sync(kFull, dig >= d0));
+                }
+                lo[r] = G1 > 0 ? (G1 - 1) << 3 : 0;
+                hi[r] = (G2 << 3) > capi[r] ? capi[r] : (G2 << 3);
+            }
         }
-        if (lane == 0) rowstate[row] = make_int2(lo + n_gt, lo + n_gt + n_eq);
+        // ---- first 64 keys of every bracket (independent loads), then whatever is left ----
+        unsigned long long key0[kL1Rows], key1[kL1Rows];
+#pragma unroll
+        for (int r = 0; r < kL1Rows; ++r) {
+            const int64_t row = batch * kL1Rows + r;
+            const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+            const int32_t j = lo[r] + lane;
+            key0[r] = j < hi[r] ? __ldg(keys + j) : 0ull;
+            key1[r] = j + kWarp < hi[r] ? __ldg(keys + j + kWarp) : 0ull;
+        }
+#pragma unroll
+        for (int r = 0; r < kL1Rows; ++r) {
+            const int64_t row = batch * kL1Rows + r;
+            if (row >= N) break;
+            const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+            int32_t n_gt = 0, n_eq = 0;
+            for (int32_t j0 = lo[r]; j0 < hi[r]; j0 += kWarp) {
+                const int32_t j = j0 + lane;
+                unsigned long long key;
+                if (j0 == lo[r]) key = key0[r];
+                else if (j0 == lo[r] + kWarp) key = key1[r];
+                else key = j < hi[r] ? __ldg(keys + j) : 0ull;
+                const int dig = j < hi[r] ? (int)(key >> 51) : -1;
+                n_gt += __popc(__ballot_sync(kFull, dig > d0));
+                const bool in = dig == d0;
+                n_eq += __popc(__ballot_sync(kFull, in));
+                if (in) atomicAdd(&s_hist[(key >> 38) & (kBins - 1)], 1u);
+            }
+            if (lane == 0) rowstate[row] = make_int2(lo[r] + n_gt, lo[r] + n_gt + n_eq);
+        }
     }
     __syncthreads();
     flush_hist(s_hist, hist1, kBins);
@@ -797,7 +860,8 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     }
     const bool vec2 = (ld % 2 == 0) && ((reinterpret_cast<uintptr_t>(gains) & 15u) == 0);
     const int rows_per_cta = kSelThreads / kWarp;
-    const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 6);
+    const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 3);
+    const int grid1 = clamp_grid((N + rows_per_cta * kL1Rows - 1) / (rows_per_cta * kL1Rows), 6);
     if (ld > 128)
         launch_level0<8>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
     else if (ld > 64)
@@ -806,7 +870,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         launch_level0<2>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
     const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     if (B > 0) {
-        select_level1<<<grid0, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, w.hdr, w.hist + kBins, w.sketch, w.sk_ld,
+        select_level1<<<grid1, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, w.hdr, w.hist + kBins, w.sketch, w.sk_ld,
                                                     w.rowstate);
         for (int level = 2; level < kLevels; ++level)
             select_refine<<<grid_rows, kSelThreads, 0, s>>>(N, ld, gains, level, w.hdr, w.hist, w.rowstate);
