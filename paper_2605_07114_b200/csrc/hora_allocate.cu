@@ -176,24 +176,19 @@ __device__ __forceinline__ void flush_hist(const unsigned int *s_hist, unsigned 
 // that the row is finite, non-negative and non-increasing (first key below +inf, every key <= its
 // predecessor, compared as unsigned integers), sums the caps, and writes the sketch: the top 16 bits of
 // keys 0, 8, 16, ... (zero beyond the cap).
-template <int E, bool VEC2>
+template <int E>
 struct Level0Item {
-    unsigned long long key[E];
+    ulonglong2 v[E / 2];           // this lane's E consecutive keys, in pairs (E is even)
     unsigned long long before;     // lane 0 only: the key just before this item (or the largest finite key)
-    int32_t capi;
+    int32_t capi;                  // the row's cap; -1 marks "no item"
 };
 
 template <int E, bool VEC2>
-__device__ __forceinline__ Level0Item<E, VEC2> level0_fetch(const int32_t *__restrict__ cap, int32_t cap_scalar,
-                                                            int64_t n_items, int32_t items_per_row, int32_t ld,
-                                                            const double *__restrict__ gains, int64_t item, int lane,
-                                                            bool *bad) {
-    Level0Item<E, VEC2> it;
-#pragma unroll
-    for (int m = 0; m < E; ++m) it.key[m] = 0ull;
-    it.before = kKeyInf - 1;
-    it.capi = 0;
-    if (item >= n_items) return it;
+__device__ __forceinline__ void level0_fetch(Level0Item<E> &it, const int32_t *__restrict__ cap, int32_t cap_scalar,
+                                             int64_t n_items, int32_t items_per_row, int32_t ld,
+                                             const double *__restrict__ gains, int64_t item, int lane, bool *bad) {
+    it.capi = -1;
+    if (item >= n_items) return;
     const int64_t row = items_per_row == 1 ? item : item / items_per_row;
     const int32_t k0 = (int32_t)(item - row * items_per_row) * (kWarp * E);
     int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
@@ -201,26 +196,71 @@ __device__ __forceinline__ Level0Item<E, VEC2> level0_fetch(const int32_t *__res
     it.capi = capi;
     const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
     const int32_t k = k0 + lane * E;
-    if (VEC2) {
+    if (VEC2 && k0 + kWarp * E <= capi) {                      // the whole item lies below the cap: plain loads
 #pragma unroll
-        for (int m = 0; m < E; m += 2) {
-            if (k + m < capi) {
-                const ulonglong2 v = __ldg(reinterpret_cast<const ulonglong2 *>(keys + k + m));
-                it.key[m] = v.x;
-                it.key[m + 1] = (k + m + 1 < capi) ? v.y : 0ull;
+        for (int p = 0; p < E / 2; ++p) it.v[p] = __ldg(reinterpret_cast<const ulonglong2 *>(keys + k) + p);
+    } else {                                                   // ragged: keys past the cap read as 0
+#pragma unroll
+        for (int p = 0; p < E / 2; ++p) {
+            it.v[p] = make_ulonglong2(0ull, 0ull);
+            if (VEC2) {
+                if (k + 2 * p < capi) {
+                    it.v[p] = __ldg(reinterpret_cast<const ulonglong2 *>(keys + k) + p);
+                    if (k + 2 * p + 1 >= capi) it.v[p].y = 0ull;
+                }
+            } else {
+                if (k + 2 * p < capi) it.v[p].x = __ldg(keys + k + 2 * p);
+                if (k + 2 * p + 1 < capi) it.v[p].y = __ldg(keys + k + 2 * p + 1);
+            }
+        }
+    }
+    it.before = kKeyInf - 1;
+    if (lane == 0 && k0 > 0 && k0 < capi) it.before = __ldg(keys + k0 - 1);
+}
+
+template <int E>
+__device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t item, int32_t items_per_row,
+                                               int32_t ld, int lane, unsigned int *s_hist,
+                                               uint16_t *__restrict__ sketch, int32_t sk_ld, long long *capsum,
+                                               bool *bad) {
+    const int64_t row = items_per_row == 1 ? item : item / items_per_row;
+    const int32_t k0 = (int32_t)(item - row * items_per_row) * (kWarp * E);
+    const int32_t k = k0 + lane * E;
+    if (lane == 0 && k0 == 0) *capsum += it.capi;
+    // order check; keys past the cap were read as 0, below every valid key, so a ragged item is no special case
+    unsigned long long before = __shfl_up_sync(kFull, it.v[E / 2 - 1].y, 1);
+    if (lane == 0) before = it.before;
+    bool wrong = it.v[0].x > before;
+#pragma unroll
+    for (int p = 0; p < E / 2; ++p) {
+        wrong |= it.v[p].y > it.v[p].x;
+        if (p > 0) wrong |= it.v[p].x > it.v[p - 1].y;
+    }
+    *bad |= wrong;
+    if ((k & 7) == 0 && k < ld) sketch[row * (int64_t)sk_ld + (k >> 3)] = (uint16_t)(it.v[0].x >> 48);
+    const int bin_first = (int)(it.v[0].x >> 51), bin_last = (int)(it.v[E / 2 - 1].y >> 51);
+    if (k0 + kWarp * E <= it.capi) {                           // full item: every lane has E valid keys
+        if (bin_first == bin_last) {
+            atomicAdd(&s_hist[bin_first], (unsigned int)E);
+        } else {
+#pragma unroll
+            for (int p = 0; p < E / 2; ++p) {
+                atomicAdd(&s_hist[(int)(it.v[p].x >> 51)], 1u);
+                atomicAdd(&s_hist[(int)(it.v[p].y >> 51)], 1u);
             }
         }
     } else {
+        const int valid = it.capi - k;                         // may be <= 0 or > E
 #pragma unroll
-        for (int m = 0; m < E; ++m)
-            if (k + m < capi) it.key[m] = __ldg(keys + k + m);
+        for (int p = 0; p < E / 2; ++p) {
+            if (2 * p < valid) atomicAdd(&s_hist[(int)(it.v[p].x >> 51)], 1u);
+            if (2 * p + 1 < valid) atomicAdd(&s_hist[(int)(it.v[p].y >> 51)], 1u);
+        }
     }
-    if (lane == 0 && k0 > 0 && k0 < capi) it.before = __ldg(keys + k0 - 1);
-    return it;
 }
 
 template <int E, bool VEC2>
-__global__ void __launch_bounds__(kSelThreads)
+__global__ void __launch_bounds__(kSelThreads, 4)
 select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
               const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist,
               uint16_t *__restrict__ sketch, int32_t sk_ld) {
@@ -235,30 +275,15 @@ select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
     const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
     long long capsum = 0;
     bool bad = false;
-    Level0Item<E, VEC2> nxt = level0_fetch<E, VEC2>(cap, cap_scalar, n_items, items_per_row, ld, gains, item0, lane, &bad);
-    for (int64_t item = item0; item < n_items; item += stride) {
-        const Level0Item<E, VEC2> cur = nxt;
-        nxt = level0_fetch<E, VEC2>(cap, cap_scalar, n_items, items_per_row, ld, gains, item + stride, lane, &bad);
-        const int64_t row = items_per_row == 1 ? item : item / items_per_row;
-        const int32_t k0 = (int32_t)(item - row * items_per_row) * (kWarp * E);
-        const int32_t k = k0 + lane * E;
-        if (lane == 0 && k0 == 0) capsum += cur.capi;
-        // keys past the cap were replaced by 0, which is below every valid key, so a ragged item needs no
-        // special case in the order check
-        unsigned long long before = __shfl_up_sync(kFull, cur.key[E - 1], 1);
-        if (lane == 0) before = cur.before;
-        bad |= cur.key[0] > before;
-#pragma unroll
-        for (int m = 1; m < E; ++m) bad |= cur.key[m] > cur.key[m - 1];
-        if ((k & 7) == 0 && k < ld) sketch[row * (int64_t)sk_ld + (k >> 3)] = (uint16_t)(cur.key[0] >> 48);
-        const int valid = cur.capi - k;                       // keys of this lane below the cap (may be <= 0 or > E)
-        if (valid >= E && (cur.key[0] >> 51) == (cur.key[E - 1] >> 51)) {
-            atomicAdd(&s_hist[(int)(cur.key[0] >> 51)], (unsigned int)E);
-        } else {
-#pragma unroll
-            for (int m = 0; m < E; ++m)
-                if (m < valid) atomicAdd(&s_hist[(int)(cur.key[m] >> 51)], 1u);
-        }
+    // two items in flight, in two fixed register sets (no copies): A is processed while B's loads land
+    Level0Item<E> A, Bq;
+    level0_fetch<E, VEC2>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item0, lane, &bad);
+    for (int64_t item = item0; item < n_items; item += 2 * stride) {
+        level0_fetch<E, VEC2>(Bq, cap, cap_scalar, n_items, items_per_row, ld, gains, item + stride, lane, &bad);
+        level0_process<E>(A, item, items_per_row, ld, lane, s_hist, sketch, sk_ld, &capsum, &bad);
+        level0_fetch<E, VEC2>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item + 2 * stride, lane, &bad);
+        if (Bq.capi >= 0)
+            level0_process<E>(Bq, item + stride, items_per_row, ld, lane, s_hist, sketch, sk_ld, &capsum, &bad);
     }
     if (bad) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);
     __syncthreads();
@@ -860,7 +885,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     }
     const bool vec2 = (ld % 2 == 0) && ((reinterpret_cast<uintptr_t>(gains) & 15u) == 0);
     const int rows_per_cta = kSelThreads / kWarp;
-    const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 3);
+    const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 4);
     const int grid1 = clamp_grid((N + rows_per_cta * kL1Rows - 1) / (rows_per_cta * kL1Rows), 6);
     if (ld > 128)
         launch_level0<8>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
