@@ -134,6 +134,39 @@ hora_status_t hora_allocate(const double *alpha, const double *beta, double alph
                             void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * hora_allocate_static — hora_allocate for callers that cannot allocate device memory.
+ *
+ * The paper has no counterpart to this call; it exists for the way the library gets embedded.  Some hosts of
+ * this code may not call cudaMalloc (or any allocator that ends up there) at the point where they need an
+ * allocation: code that runs inside a region where the allocator is frozen or instrumented, plug-ins that
+ * are handed their input and output buffers by a framework and nothing else, or services that pre-size all
+ * device memory at start-up and treat a later allocation as a fault.  For them the scratch that hora_allocate
+ * needs lives inside the library: a fixed array of hora_allocate_static_capacity() bytes (8 MiB) in device
+ * memory, present on every GPU that loads the library for as long as the process lives.
+ *
+ * Arguments and results are those of hora_allocate without `workspace` / `workspace_bytes`; the caller still
+ * passes every input and output buffer.  The call itself allocates nothing and frees nothing.
+ *
+ *   - Size limit: hora_allocate_workspace_bytes(N, ld, gains == NULL, flags) must not exceed
+ *     hora_allocate_static_capacity(); otherwise HORA_ERR_WORKSPACE is returned and nothing is enqueued.
+ *     With a materialised gains matrix and ld = 256 that admits about 1e5 prompts; with gains == NULL the
+ *     matrix itself must fit, so only small problems (N*ld*8 bytes well under 8 MiB) qualify.
+ *   - First use: the first call on each device looks up the array's device address (cudaGetSymbolAddress)
+ *     with that device current, and caches it.  Make that first call outside any stream capture.
+ *   - Sharing: every call on a device uses the same array.  It keeps whatever the previous call left there;
+ *     each call clears the parts it needs zeroed before using them, so back-to-back calls on one stream
+ *     are fine.  Two calls that overlap on the GPU (different streams, or different host threads without
+ *     ordering) race on the scratch and give undefined results: serialise them.
+ */
+size_t hora_allocate_static_capacity(void);   /* host: size of the built-in scratch in bytes */
+
+hora_status_t hora_allocate_static(const double *alpha, const double *beta, double alpha0, double beta0,
+                                   const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar,
+                                   int64_t N, int32_t ld, const double *gains, int64_t B, uint32_t flags,
+                                   int32_t *delta, int32_t *G, int64_t *group_offsets, hora_alloc_info *info_dev,
+                                   void *stream);
+
+/*
  * hora_group_advantage — group-relative advantages over ragged groups (Sec. 3.1 for GRPO; the RLOO
  * compatibility paragraph of Sec. 4 for the leave-one-out form).
  *

@@ -27,6 +27,8 @@
 // by 256-bit cross multiplication of num/den = a (b)_a / (b+Delta-1)_{a+1}  (or the equivalent
 // a (b)_{Delta-1} / (a+b)_Delta when that has fewer factors), and the threshold class is found by
 // walking the ranked types.  Rows are relabelled above / tied / below and the same sum/out steps run.
+#include <atomic>
+
 #include "hora_common.cuh"
 
 namespace hora {
@@ -921,4 +923,51 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
                                                info_dev);
     count_launches(B > 0 ? (exact ? 10 : 7) : 3);
     return cuda_ok(cudaGetLastError());
+}
+
+// ---------------------------------------------------------------------------------------------------
+// hora_allocate_static: the same allocation with the scratch held by the library itself.
+//
+// The scratch is a file-scope device array, so it exists on every GPU that loads this library from the
+// moment the module is loaded until the process ends, and no allocation call is ever made on its behalf.
+// Host code cannot hand the array's NAME to a kernel: on the host that name is only a stand-in for the
+// symbol, not an address the GPU understands.  The device address is looked up once per device with
+// cudaGetSymbolAddress and cached.
+namespace hora {
+
+constexpr size_t kStaticScratchBytes = (size_t)8 << 20;     // 8 MiB
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::atomic<void *> g_static_scratch_addr[kMaxDevices];
+
+// Device address of the scratch array on the current device (nullptr on failure).
+static void *static_scratch_address() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    void *p = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+    if (p != nullptr) return p;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return nullptr;
+    g_static_scratch_addr[dev].store(p, std::memory_order_release);
+    return p;
+}
+
+}  // namespace hora
+
+extern "C" size_t hora_allocate_static_capacity(void) { return hora::kStaticScratchBytes; }
+
+extern "C" hora_status_t hora_allocate_static(const double *alpha, const double *beta, double alpha0, double beta0,
+                                              const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar,
+                                              int64_t N, int32_t ld, const double *gains, int64_t B, uint32_t flags,
+                                              int32_t *delta, int32_t *G, int64_t *group_offsets,
+                                              hora_alloc_info *info_dev, void *stream) {
+    using namespace hora;
+    if (N < 0 || ld < 1) return HORA_ERR_INVALID_ARG;
+    // the problem must fit the built-in scratch; say so before touching the device
+    const size_t need = hora_allocate_workspace_bytes(N, ld, gains == nullptr ? 1 : 0, flags);
+    if (need > kStaticScratchBytes) return HORA_ERR_WORKSPACE;
+    void *scratch = static_scratch_address();
+    if (scratch == nullptr) return HORA_ERR_CUDA;
+    return hora_allocate(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, flags, delta, G,
+                         group_offsets, info_dev, scratch, kStaticScratchBytes, stream);
 }

@@ -22,7 +22,8 @@ FLAG_SKIP_OBJECTIVE = 2
 ADV_GRPO, ADV_RLOO = 0, 1
 
 EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora_group_advantage",
-           "hora_token_broadcast", "hora_status_string", "hora_version", "hora_launch_count")
+           "hora_token_broadcast", "hora_status_string", "hora_version", "hora_launch_count",
+           "hora_allocate_static", "hora_allocate_static_capacity")
 
 
 class HoraError(RuntimeError):
@@ -56,6 +57,9 @@ def load() -> C.CDLL:
     L.hora_allocate_workspace_bytes.restype = C.c_size_t
     L.hora_allocate.argtypes = [p, p, f64, f64, p, i32, p, i32, i64, i32, p, i64, u32, p, p, p, p, p, C.c_size_t, p]
     L.hora_allocate.restype = C.c_int
+    L.hora_allocate_static.argtypes = [p, p, f64, f64, p, i32, p, i32, i64, i32, p, i64, u32, p, p, p, p, p]
+    L.hora_allocate_static.restype = C.c_int
+    L.hora_allocate_static_capacity.restype = C.c_size_t
     L.hora_group_advantage.argtypes = [p, p, i64, i32, C.c_float, i32, p, p, p]
     L.hora_group_advantage.restype = C.c_int
     L.hora_token_broadcast.argtypes = [p, p, i64, i64, p, p]
@@ -124,6 +128,24 @@ def hora_allocate(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gai
                               _ptr(info_dev, torch.uint8, "info_dev"), _ptr(workspace, torch.uint8, "workspace"),
                               0 if workspace is None else workspace.numel(), _stream())
     _check(rc, "hora_allocate")
+
+
+def hora_allocate_static_capacity() -> int:
+    return int(load().hora_allocate_static_capacity())
+
+
+def hora_allocate_static(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, flags, delta, G,
+                         group_offsets, info_dev):
+    """hora_allocate with the library's own fixed scratch: no workspace argument, no allocation.
+    Problems whose workspace would exceed hora_allocate_static_capacity() raise HoraError(ERR_WORKSPACE).
+    Calls share that scratch, so do not let two of them overlap on the GPU."""
+    rc = load().hora_allocate_static(_ptr(alpha, torch.float64, "alpha"), _ptr(beta, torch.float64, "beta"), alpha0,
+                                     beta0, _ptr(c, torch.int32, "c"), G0, _ptr(cap, torch.int32, "cap"), cap_scalar,
+                                     N, ld, _ptr(gains, torch.float64, "gains"), B, flags,
+                                     _ptr(delta, torch.int32, "delta"), _ptr(G, torch.int32, "G"),
+                                     _ptr(group_offsets, torch.int64, "group_offsets"),
+                                     _ptr(info_dev, torch.uint8, "info_dev"), _stream())
+    _check(rc, "hora_allocate_static")
 
 
 def hora_group_advantage(rewards, group_offsets, N, mode, eps, ddof, adv, status_dev=None):
