@@ -114,6 +114,22 @@ def shard_seed(rank: int) -> int:
     return 3 + rank
 
 
+def max_over_ranks(x: float, world: int, device=None) -> float:
+    """Slowest rank's time: the job is done when the last shard is."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(prompts_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job prompts per second: every rank processes its own shard of prompts_per_rank prompts."""
+    return prompts_per_rank * world / (ms_per_step * 1e-3)
+
+
 # --------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -192,13 +208,6 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
     warmup = max(args.warmup, 3)
     for _ in range(warmup):
         step()
@@ -219,7 +228,7 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop()
     launches = hora.hora_launch_count() - launches0
-    ms_total = max_over_ranks(t0.elapsed_time(t1))
+    ms_total = max_over_ranks(t0.elapsed_time(t1), world, dev)
     ms_step = ms_total / args.steps
     stages = np.array([[ev[i].elapsed_time(ev[i + 1]) for i in range(4)] for ev in stage_ev])
     st_mean = stages.mean(axis=0)
@@ -241,7 +250,7 @@ def run_ours(args):
         step_e2e()
     e1.record()
     barrier()
-    ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev) / e2e_steps
     h2d = h_alpha.numel() * 8 + h_beta.numel() * 8 + h_c.numel() * 4 + h_rewards.numel() * 4
     d2h = h_delta.numel() * 4 + h_G.numel() * 4 + h_adv.numel() * 4
 
@@ -268,7 +277,7 @@ def run_ours(args):
     g_ms = float(st_mean[0])                           # hora_gains is exactly one launch (gains_kernel)
     achieved = bytes_gains / (g_ms * 1e-3) / 1e9
     out = {
-        "metric": METRIC, "value": N * world / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": job_throughput(N, world, ms_step), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": f"{WORKLOAD}: N={N} prompts per GPU, G0={G0}, ld={ld}, B={B}, per-prompt real priors, "
@@ -276,7 +285,7 @@ def run_ours(args):
                    "l2": "inputs larger than L2 (the gains matrix alone is %.2f GB)" % (cand * 8 / 1e9),
                    "shard": "one independent batch per GPU, no collective"},
         "clocks": clocks,
-        "e2e": {"value": N * world / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+        "e2e": {"value": job_throughput(N, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "gains_kernel (the one launch of hora_gains)",
