@@ -2,19 +2,24 @@
 // Algorithm 1's Phase-B greedy loop (Proposition 1), found by selection instead of B sequential steps.
 //
 // Keys.  A gain is a non-negative finite double, so its bit pattern orders like the value.  The 64-bit
-// key is resolved 13 bits at a time (shifts 51, 38, 25, 12, then the last 12 bits):
+// key of the B-th largest gain is resolved from the top, a digit at a time:
 //
-//   level 0   one coalesced read of the whole matrix (a warp per row), histogram of the top 13 bits
-//             in shared memory, merged into a global histogram; the last CTA to finish locates the
-//             digit that holds the B-th largest key.  The same pass writes a 2-byte sketch of every
-//             8th key (its top 16 bits), 3 % of the matrix in size.
-//   level 1   a warp per row: because a row is non-increasing, its keys with the selected top digit
-//             form ONE contiguous segment; the sketch brackets it to within 8 keys on each side, so
-//             only that segment is read again (coalesced) and its next digit histogrammed.  The
-//             segment [p_hi, p_lo) is kept per row.
-//   level 2-4 a thread per row narrows its segment by the digit just selected and histograms the next.
-//   sum       narrows by the last digit: p_hi = #keys > lambda, p_lo - p_hi = #keys == lambda; block sums
-//             and their scan give n_above, n_tied and the exclusive prefixes over prompts.
+//   estimate  every S-th row (about 8192 rows) is read and histogrammed on the top 13 bits; the scaled rank
+//             says in which two adjacent 13-bit bins the threshold almost surely lies (the "window").
+//   level 0   one coalesced read of the whole matrix (a warp per row-item, two items in flight).  Keys
+//             outside the window are counted per 13-bit bin, keys inside it per 23-bit bin (1024 fine bins
+//             per window bin), all in shared memory, then merged into global histograms.  The last CTA to
+//             finish locates the 13-bit digit of the threshold and, if it is inside the window, its 23-bit
+//             prefix; otherwise the selection simply goes on from 13 bits.  The same pass validates the
+//             rows, sums the caps and writes a 2-byte sketch of every 8th key (its top 16 bits).
+//   level 1   a warp per four rows: a row is non-increasing, so its keys with the resolved prefix form ONE
+//             contiguous segment, which the sketch brackets to within 8 keys on each side; only the
+//             bracket is read (coalesced), the segment [p_hi, p_lo) stored, its next 13 bits histogrammed,
+//             and rows whose segment is not empty are appended to a list.
+//   level 2-4 a thread per listed row narrows its segment by the digit just selected and histograms the
+//             next one (13 bits at a time until all 64 are resolved), then a last narrowing pass.
+//   sum       p_hi = #keys > lambda, p_lo - p_hi = #keys == lambda per row; block sums and their scan give
+//             n_above, n_tied and the exclusive prefixes over prompts; priors are validated here.
 //   out       Delta_i = p_hi + (tied candidates of row i that fall within the first R = B - n_above tied
 //             candidates in prompt order); G_i, CSR offsets, objective.
 //
@@ -33,25 +38,31 @@
 
 namespace hora {
 
-constexpr int kLevels = 5;
-constexpr int kBins = 8192;
+constexpr int kLevels = 5;                   // level 0 (full read) + four digit levels
+constexpr int kBins = 8192;                  // 13-bit digits
+constexpr int kDigitBits = 13;
+constexpr int kWinBins = 2;                  // coarse bins covered by the fine window of level 0
+constexpr int kFineBits = 10;                // extra bits resolved inside the window
+constexpr int kFinePerBin = 1 << kFineBits;
+constexpr int kFineBins = kWinBins * kFinePerBin;
+constexpr int kSampleRows = 8192;            // rows read by the estimate pass
 constexpr int kSelThreads = 256;
 constexpr int kRowsPerBlock = 1024;          // rows per CTA in the sum / out kernels (4 per thread)
 constexpr int kTypeSlots = 4096;             // hash slots for exact tie types
 constexpr int kMaxTypes = 1024;              // distinct types the exact ranking accepts
 constexpr unsigned long long kKeyInf = 0x7FF0000000000000ull;
 
-__host__ __device__ __forceinline__ int level_shift(int level) { return level == 4 ? 0 : 51 - 13 * level; }
-__host__ __device__ __forceinline__ int level_bins(int level) { return level == 4 ? 4096 : 8192; }
-
 struct AllocHeader {
     int32_t status;
-    int32_t pad0;
+    int32_t resolved;                  // key bits resolved so far, from the top
     unsigned int ticket[16];
     unsigned long long sum_cap;
-    unsigned long long prefix_key;     // key bits resolved so far (the threshold once all levels ran)
+    unsigned long long prefix_key;     // the resolved bits in place (the threshold once all 64 are resolved)
     long long need;                    // rank of the threshold inside the current bin (1-based)
-    int32_t sel_digit[8];
+    int32_t lv_shift[8], lv_bits[8], sel_digit[8];   // per level: position, width and value of its digit
+    int32_t win_lo;                    // first 13-bit bin of level 0's fine window
+    unsigned int n_active;             // rows with a non-empty segment after level 1
+    unsigned long long sample_cap;     // sum of the caps of the sampled rows
     unsigned long long n_above, n_tied;
     long long R;                       // tied candidates to take
     double lambda;
@@ -63,10 +74,14 @@ struct AllocHeader {
 
 struct Workspace {
     AllocHeader *hdr;
-    unsigned long long *hist;          // [kLevels][kBins]
+    unsigned long long *hist_est;      // [kBins] estimate pass
+    unsigned long long *hist_coarse;   // [kBins] level 0, 13-bit bins outside the window
+    unsigned long long *hist_fine;     // [kFineBins] level 0, 23-bit bins inside the window
+    unsigned long long *hist_lv;       // [kLevels][kBins] levels 1..4 (slot 0 unused)
     int2 *rowstate;                    // [N] (p_hi, p_lo)
     uint16_t *sketch;                  // [N][sk_ld] top 16 bits of keys 0, 8, 16, ... of each row
     int32_t sk_ld;
+    int32_t *active;                   // [N] rows with a non-empty segment
     long long *bsum_hi, *bsum_t;       // [NB] block sums, overwritten by exclusive prefixes
     double *objpart;                   // [NB]
     unsigned long long *tkeys, *tcounts;   // [kTypeSlots]
@@ -85,10 +100,14 @@ static Workspace carve(void *base, int64_t N, int32_t ld, bool need_gains, bool 
     const int64_t NB = (N + kRowsPerBlock - 1) / kRowsPerBlock;
     auto take = [&](size_t n) { char *q = p ? p + o : nullptr; o = align256(o + n); return q; };
     w.hdr = reinterpret_cast<AllocHeader *>(take(sizeof(AllocHeader)));
-    w.hist = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kLevels * kBins));
-    w.rowstate = reinterpret_cast<int2 *>(take(sizeof(int2) * (size_t)N));
+    w.hist_est = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kBins));
+    w.hist_coarse = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kBins));
+    w.hist_fine = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kFineBins));
+    w.hist_lv = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kLevels * kBins));
+    w.rowstate = reinterpret_cast<int2 *>(take(sizeof(int2) * (size_t)N));          // everything before this is zeroed per call
     w.sk_ld = ((ld + 7) / 8 + 7) & ~7;
     w.sketch = reinterpret_cast<uint16_t *>(take(sizeof(uint16_t) * (size_t)N * (size_t)w.sk_ld));
+    w.active = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (size_t)N));
     w.bsum_hi = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
     w.bsum_t = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
     w.objpart = reinterpret_cast<double *>(take(sizeof(double) * (size_t)NB));
@@ -138,29 +157,37 @@ __device__ __forceinline__ long long block_exclusive_sum(long long v, long long 
     return base + inc - v;
 }
 
-// Run by ONE CTA: find the digit d with  count(digit > d) < need <= count(digit >= d)  in hist[0..bins).
-__device__ void find_digit(AllocHeader *hdr, const unsigned long long *hist, int level, long long *s_warp) {
-    const int bins = level_bins(level);
-    const int per = bins / kSelThreads;
+// Run by ONE CTA: find the digit d with  count(digit > d) < need <= count(digit >= d)  in hist[0..bins),
+// bins a power of two.  The digit sits at bit `shift` of the key.  With `append` it extends the digit
+// already recorded for `level` (the fine part of level 0) instead of starting a new one.
+__device__ void find_digit(AllocHeader *hdr, const unsigned long long *hist, int bins, int bits, int shift, int level,
+                           bool append, long long *s_warp) {
+    const int per = (bins + kSelThreads - 1) / kSelThreads;
     const long long need = hdr->need;
     const int top = bins - 1 - (int)threadIdx.x * per;      // this thread scans bins top, top-1, ..., top-per+1
     long long local = 0;
-    for (int j = 0; j < per; ++j) local += (long long)__ldcg(hist + top - j);
+    for (int j = 0; j < per; ++j)
+        if (top - j >= 0) local += (long long)__ldcg(hist + top - j);
     long long total;
     const long long above = block_exclusive_sum(local, &total, s_warp);
     if (need >= 1 && above < need && need <= above + local) {
         long long run = above;
-        for (int j = 0; j < per; ++j) {
+        for (int j = 0; j < per && top - j >= 0; ++j) {
             const long long cnt = (long long)__ldcg(hist + top - j);
             if (run + cnt >= need) {
-                hdr->sel_digit[level] = top - j;
+                const int digit = top - j;
+                hdr->sel_digit[level] = append ? ((hdr->sel_digit[level] << bits) | digit) : digit;
+                hdr->lv_bits[level] = append ? hdr->lv_bits[level] + bits : bits;
+                hdr->lv_shift[level] = shift;
                 hdr->need = need - run;
-                hdr->prefix_key |= (unsigned long long)(top - j) << level_shift(level);
+                hdr->prefix_key |= (unsigned long long)digit << shift;
+                hdr->resolved += bits;
                 break;
             }
             run += cnt;
         }
     }
+    __syncthreads();
 }
 
 __device__ __forceinline__ void flush_hist(const unsigned int *s_hist, unsigned long long *hist, int bins) {
@@ -170,14 +197,84 @@ __device__ __forceinline__ void flush_hist(const unsigned int *s_hist, unsigned 
     }
 }
 
+// Width and position of the next digit once `resolved` bits are known.
+__device__ __forceinline__ void next_digit(int resolved, int *bits, int *shift) {
+    const int w = 64 - resolved < kDigitBits ? 64 - resolved : kDigitBits;
+    *bits = w;
+    *shift = 64 - resolved - w;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Estimate: a warp per sampled row (every `every`-th row), histogram of the top 13 bits.  The last CTA
+// scales the rank B to the sample and places the two-bin window around the bin it falls in: towards the
+// upper neighbour when the rank falls in the upper half of that bin's count, else towards the lower one.
+__global__ void __launch_bounds__(kSelThreads)
+select_estimate(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld, int64_t every,
+                const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist) {
+    __shared__ unsigned int s_hist[kBins];
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
+    __syncthreads();
+    const int lane = lane_id();
+    const int64_t n_sample = (N + every - 1) / every;
+    const int64_t warp0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5);
+    const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
+    long long capsum = 0;
+    for (int64_t sidx = warp0; sidx < n_sample; sidx += stride) {
+        const int64_t row = sidx * every;
+        int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
+        capi = capi < 0 ? 0 : (capi > ld ? ld : capi);
+        if (lane == 0) capsum += capi;
+        const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+        for (int32_t j = lane; j < capi; j += kWarp) {
+            const unsigned long long key = __ldg(keys + j);
+            atomicAdd(&s_hist[(int)(key >> 51) & (kBins - 1)], 1u);
+        }
+    }
+    __syncthreads();
+    flush_hist(s_hist, hist, kBins);
+    long long tot;
+    block_exclusive_sum(capsum, &tot, s_warp);
+    if (threadIdx.x == 0 && tot) atomicAdd(&hdr->sample_cap, (unsigned long long)tot);
+    if (last_block(&hdr->ticket[15])) {
+        // rank of the threshold within the sample
+        long long need = (long long)((double)B * (double)n_sample / (double)N + 0.5);
+        const long long sample_cap = (long long)*(volatile unsigned long long *)&hdr->sample_cap;
+        if (need < 1) need = 1;
+        if (need > sample_cap) need = sample_cap;
+        const int per = kBins / kSelThreads;
+        const int top = kBins - 1 - (int)threadIdx.x * per;
+        long long local = 0;
+        for (int j = 0; j < per; ++j) local += (long long)__ldcg(hist + top - j);
+        long long total;
+        const long long above = block_exclusive_sum(local, &total, s_warp);
+        if (need >= 1 && above < need && need <= above + local) {
+            long long run = above;
+            for (int j = 0; j < per; ++j) {
+                const long long cnt = (long long)__ldcg(hist + top - j);
+                if (run + cnt >= need) {
+                    const int d = top - j;
+                    const bool upper_half = 2 * (need - run) <= cnt;      // counting from the top of the bin
+                    int lo = upper_half ? d : d - 1;
+                    lo = lo < 0 ? 0 : (lo > kBins - kWinBins ? kBins - kWinBins : lo);
+                    hdr->win_lo = lo;
+                    break;
+                }
+                run += cnt;
+            }
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------------
 // Level 0: the one full read.  The matrix is cut into items of 32*E consecutive keys of one row; a warp
 // takes one item at a time and a lane E consecutive keys of it, and the loads of the NEXT item are
 // issued before the current one is processed.  The row is sorted, so a lane's keys usually fall into
-// one bin (one shared-memory atomic for all E); otherwise each key adds itself.  The pass also checks
-// that the row is finite, non-negative and non-increasing (first key below +inf, every key <= its
-// predecessor, compared as unsigned integers), sums the caps, and writes the sketch: the top 16 bits of
-// keys 0, 8, 16, ... (zero beyond the cap).
+// one 13-bit bin: if that bin is outside the window, one shared-memory atomic counts all E; keys inside
+// the window are counted one by one in the 23-bit bins.  The pass also checks that the row is finite,
+// non-negative and non-increasing (first key below +inf, every key <= its predecessor, compared as
+// unsigned integers), sums the caps, and writes the sketch: the top 16 bits of keys 0, 8, 16, ... (zero
+// beyond the cap).
 template <int E>
 struct Level0Item {
     ulonglong2 v[E / 2];           // this lane's E consecutive keys, in pairs (E is even)
@@ -222,9 +319,9 @@ __device__ __forceinline__ void level0_fetch(Level0Item<E> &it, const int32_t *_
 
 template <int E>
 __device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t item, int32_t items_per_row,
-                                               int32_t ld, int lane, unsigned int *s_hist,
-                                               uint16_t *__restrict__ sketch, int32_t sk_ld, long long *capsum,
-                                               bool *bad) {
+                                               int32_t ld, int lane, unsigned int *s_hist, unsigned int *s_fine,
+                                               int win_lo, uint16_t *__restrict__ sketch, int32_t sk_ld,
+                                               long long *capsum, bool *bad) {
     const int64_t row = items_per_row == 1 ? item : item / items_per_row;
     const int32_t k0 = (int32_t)(item - row * items_per_row) * (kWarp * E);
     const int32_t k = k0 + lane * E;
@@ -240,23 +337,30 @@ __device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t 
     }
     *bad |= wrong;
     if ((k & 7) == 0 && k < ld) sketch[row * (int64_t)sk_ld + (k >> 3)] = (uint16_t)(it.v[0].x >> 48);
+    // one key: a 23-bit bin inside the window, a 13-bit bin outside it
+    auto count_key = [&](unsigned long long key) {
+        const int bin = (int)(key >> 51);
+        const unsigned w = (unsigned)(bin - win_lo);
+        if (w < (unsigned)kWinBins) atomicAdd(&s_fine[w * kFinePerBin + ((unsigned)(key >> (51 - kFineBits)) & (kFinePerBin - 1))], 1u);
+        else atomicAdd(&s_hist[bin], 1u);
+    };
     const int bin_first = (int)(it.v[0].x >> 51), bin_last = (int)(it.v[E / 2 - 1].y >> 51);
     if (k0 + kWarp * E <= it.capi) {                           // full item: every lane has E valid keys
-        if (bin_first == bin_last) {
+        if (bin_first == bin_last && (unsigned)(bin_first - win_lo) >= (unsigned)kWinBins) {
             atomicAdd(&s_hist[bin_first], (unsigned int)E);
         } else {
 #pragma unroll
             for (int p = 0; p < E / 2; ++p) {
-                atomicAdd(&s_hist[(int)(it.v[p].x >> 51)], 1u);
-                atomicAdd(&s_hist[(int)(it.v[p].y >> 51)], 1u);
+                count_key(it.v[p].x);
+                count_key(it.v[p].y);
             }
         }
     } else {
         const int valid = it.capi - k;                         // may be <= 0 or > E
 #pragma unroll
         for (int p = 0; p < E / 2; ++p) {
-            if (2 * p < valid) atomicAdd(&s_hist[(int)(it.v[p].x >> 51)], 1u);
-            if (2 * p + 1 < valid) atomicAdd(&s_hist[(int)(it.v[p].y >> 51)], 1u);
+            if (2 * p < valid) count_key(it.v[p].x);
+            if (2 * p + 1 < valid) count_key(it.v[p].y);
         }
     }
 }
@@ -265,12 +369,15 @@ template <int E, bool VEC2>
 __global__ void __launch_bounds__(kSelThreads, 4)
 select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
               const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist,
-              uint16_t *__restrict__ sketch, int32_t sk_ld) {
+              unsigned long long *hist_fine, uint16_t *__restrict__ sketch, int32_t sk_ld) {
     __shared__ unsigned int s_hist[kBins];
+    __shared__ unsigned int s_fine[kFineBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
+    for (int b = threadIdx.x; b < kFineBins; b += kSelThreads) s_fine[b] = 0;
     __syncthreads();
     const int lane = lane_id();
+    const int win_lo = hdr->win_lo;
     const int32_t items_per_row = (ld + kWarp * E - 1) / (kWarp * E);
     const int64_t n_items = N * items_per_row;
     const int64_t item0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5);
@@ -282,47 +389,71 @@ select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
     level0_fetch<E, VEC2>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item0, lane, &bad);
     for (int64_t item = item0; item < n_items; item += 2 * stride) {
         level0_fetch<E, VEC2>(Bq, cap, cap_scalar, n_items, items_per_row, ld, gains, item + stride, lane, &bad);
-        level0_process<E>(A, item, items_per_row, ld, lane, s_hist, sketch, sk_ld, &capsum, &bad);
+        level0_process<E>(A, item, items_per_row, ld, lane, s_hist, s_fine, win_lo, sketch, sk_ld, &capsum, &bad);
         level0_fetch<E, VEC2>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item + 2 * stride, lane, &bad);
         if (Bq.capi >= 0)
-            level0_process<E>(Bq, item + stride, items_per_row, ld, lane, s_hist, sketch, sk_ld, &capsum, &bad);
+            level0_process<E>(Bq, item + stride, items_per_row, ld, lane, s_hist, s_fine, win_lo, sketch, sk_ld, &capsum,
+                              &bad);
     }
     if (bad) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);
     __syncthreads();
     flush_hist(s_hist, hist, kBins);
+    flush_hist(s_fine, hist_fine, kFineBins);
     long long tot;
     block_exclusive_sum(capsum, &tot, s_warp);
     if (threadIdx.x == 0 && tot) atomicAdd(&hdr->sum_cap, (unsigned long long)tot);
     if (last_block(&hdr->ticket[0])) {
         const unsigned long long sum_cap = *(volatile unsigned long long *)&hdr->sum_cap;
+        // the 13-bit counts of the window bins are the sums of their fine bins
+        for (int wb = 0; wb < kWinBins; ++wb) {
+            long long part = 0;
+            for (int f = threadIdx.x; f < kFinePerBin; f += kSelThreads) part += (long long)__ldcg(hist_fine + wb * kFinePerBin + f);
+            long long sum;
+            block_exclusive_sum(part, &sum, s_warp);
+            if (threadIdx.x == 0) hist[win_lo + wb] = (unsigned long long)sum;
+        }
         if (threadIdx.x == 0) {
             if ((unsigned long long)B > sum_cap) raise_status(&hdr->status, HORA_ERR_INFEASIBLE);
             hdr->need = B;
         }
+        __threadfence();
         __syncthreads();
-        find_digit(hdr, hist, 0, s_warp);
+        find_digit(hdr, hist, kBins, kDigitBits, 51, 0, false, s_warp);
+        const int d0 = hdr->sel_digit[0];
+        const unsigned w = (unsigned)(d0 - win_lo);
+        if (hdr->resolved == kDigitBits && w < (unsigned)kWinBins)        // inside the window: 10 more bits for free
+            find_digit(hdr, hist_fine + w * kFinePerBin, kFinePerBin, kFineBits, 51 - kFineBits, 0, true, s_warp);
     }
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Level 1: a warp per row.  The sketch says, for every group of 8 keys, which bin its first (largest) key
-// falls in.  With d the digit selected at level 0: groups whose first key is above bin d form a prefix
-// of G1 groups, groups whose first key is in or above bin d a prefix of G2 >= G1 groups.  Every key in
-// bin d therefore sits in groups G1-1 .. G2-1, and so does the boundary between "above" and "in" the
-// bin; only those groups are read (coalesced), counted and histogrammed on the next digit.
+// Level 1: a warp per four rows.  r bits of the threshold are known (23 after a window hit, else 13);
+// call P that prefix.  The sketch holds the top 16 bits of the first (largest) key of every group of 8
+// keys.  Compared at min(r, 16) bits: groups whose first key is above P form a prefix of G1 groups,
+// groups whose first key is above or equal a prefix of G2 >= G1 groups.  Every key with prefix P
+// therefore sits in groups G1-1 .. G2-1, and so does the boundary between "above" and "equal"; only
+// those groups are read (coalesced), classified on all r bits, and the keys with prefix P histogrammed
+// on the next digit.  Rows that keep a non-empty segment are appended to the active list.
 constexpr int kL1Rows = 4;      // rows a warp works on at once: their loads are in flight together
 
 __global__ void __launch_bounds__(kSelThreads)
 select_level1(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
               const double *__restrict__ gains, AllocHeader *hdr, unsigned long long *hist1,
-              const uint16_t *__restrict__ sketch, int32_t sk_ld, int2 *__restrict__ rowstate) {
+              const uint16_t *__restrict__ sketch, int32_t sk_ld, int2 *__restrict__ rowstate,
+              int32_t *__restrict__ active) {
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     if (*(volatile int32_t *)&hdr->status != 0) return;
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
     __syncthreads();
     const int lane = lane_id();
-    const int d0 = hdr->sel_digit[0];
+    const int r = hdr->resolved;
+    const unsigned long long P = hdr->prefix_key >> (64 - r);
+    const int sk_shift = r < 16 ? 16 - r : 0;                    // sketch entries compared at min(r, 16) bits
+    const int Psk = (int)((hdr->prefix_key >> 48) >> sk_shift);
+    int bits, shift;
+    next_digit(r, &bits, &shift);
+    const unsigned long long digit_mask = (1ull << bits) - 1ull;
     const int64_t warp0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5);
     const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
     const int64_t n_batches = (N + kL1Rows - 1) / kL1Rows;
@@ -330,102 +461,112 @@ select_level1(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
         int32_t capi[kL1Rows], lo[kL1Rows], hi[kL1Rows];
         // ---- sketches of all rows of the batch (independent loads), then their brackets ----
 #pragma unroll
-        for (int r = 0; r < kL1Rows; ++r) {
-            const int64_t row = batch * kL1Rows + r;
-            capi[r] = 0;
+        for (int q = 0; q < kL1Rows; ++q) {
+            const int64_t row = batch * kL1Rows + q;
+            capi[q] = 0;
             if (row < N) {
                 const int32_t cp = cap ? __ldg(cap + row) : cap_scalar;
-                capi[r] = cp < 0 ? 0 : (cp > ld ? ld : cp);
+                capi[q] = cp < 0 ? 0 : (cp > ld ? ld : cp);
             }
         }
         if (ld <= 8 * kWarp) {                                   // one sketch entry per lane covers the row
             int dig[kL1Rows];
 #pragma unroll
-            for (int r = 0; r < kL1Rows; ++r) {
-                const int64_t row = batch * kL1Rows + r;
-                const int n_groups = (capi[r] + 7) >> 3;
-                dig[r] = lane < n_groups ? (int)(__ldg(sketch + row * (int64_t)sk_ld + lane) >> 3) : -1;
+            for (int q = 0; q < kL1Rows; ++q) {
+                const int64_t row = batch * kL1Rows + q;
+                const int n_groups = (capi[q] + 7) >> 3;
+                dig[q] = lane < n_groups ? (int)(__ldg(sketch + row * (int64_t)sk_ld + lane) >> sk_shift) : -1;
             }
 #pragma unroll
-            for (int r = 0; r < kL1Rows; ++r) {
-                const int G1 = __popc(__ballot_sync(kFull, dig[r] > d0));
-                const int G2 = __popc(__ballot_sync(kFull, dig[r] >= d0));
-                lo[r] = G1 > 0 ? (G1 - 1) << 3 : 0;
-                hi[r] = (G2 << 3) > capi[r] ? capi[r] : (G2 << 3);
+            for (int q = 0; q < kL1Rows; ++q) {
+                const int G1 = __popc(__ballot_sync(kFull, dig[q] > Psk));
+                const int G2 = __popc(__ballot_sync(kFull, dig[q] >= Psk));
+                lo[q] = G1 > 0 ? (G1 - 1) << 3 : 0;
+                hi[q] = (G2 << 3) > capi[q] ? capi[q] : (G2 << 3);
             }
         } else {
 #pragma unroll
-            for (int r = 0; r < kL1Rows; ++r) {
-                const int64_t row = batch * kL1Rows + r;
-                const int n_groups = (capi[r] + 7) >> 3;
+            for (int q = 0; q < kL1Rows; ++q) {
+                const int64_t row = batch * kL1Rows + q;
+                const int n_groups = (capi[q] + 7) >> 3;
                 int G1 = 0, G2 = 0;
                 for (int g0 = 0; g0 < n_groups; g0 += kWarp) {
                     const int g = g0 + lane;
-                    const int dig = g < n_groups ? (int)(__ldg(sketch + row * (int64_t)sk_ld + g) >> 3) : -1;
-                    G1 += __popc(__ballot_sync(kFull, dig > d0));
-                    G2 += __popc(__ballot_sync(kFull, dig >= d0));
+                    const int dig = g < n_groups ? (int)(__ldg(sketch + row * (int64_t)sk_ld + g) >> sk_shift) : -1;
+                    G1 += __popc(__ballot_sync(kFull, dig > Psk));
+                    G2 += __popc(__ballot_sync(kFull, dig >= Psk));
                 }
-                lo[r] = G1 > 0 ? (G1 - 1) << 3 : 0;
-                hi[r] = (G2 << 3) > capi[r] ? capi[r] : (G2 << 3);
+                lo[q] = G1 > 0 ? (G1 - 1) << 3 : 0;
+                hi[q] = (G2 << 3) > capi[q] ? capi[q] : (G2 << 3);
             }
         }
-        // ---- first 64 keys of every bracket (independent loads), then whatever is left ----
-        unsigned long long key0[kL1Rows], key1[kL1Rows];
+        // ---- first 32 keys of every bracket (independent loads), then whatever is left ----
+        unsigned long long key0[kL1Rows];
 #pragma unroll
-        for (int r = 0; r < kL1Rows; ++r) {
-            const int64_t row = batch * kL1Rows + r;
+        for (int q = 0; q < kL1Rows; ++q) {
+            const int64_t row = batch * kL1Rows + q;
             const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-            const int32_t j = lo[r] + lane;
-            key0[r] = j < hi[r] ? __ldg(keys + j) : 0ull;
-            key1[r] = j + kWarp < hi[r] ? __ldg(keys + j + kWarp) : 0ull;
+            const int32_t j = lo[q] + lane;
+            key0[q] = j < hi[q] ? __ldg(keys + j) : 0ull;
         }
 #pragma unroll
-        for (int r = 0; r < kL1Rows; ++r) {
-            const int64_t row = batch * kL1Rows + r;
+        for (int q = 0; q < kL1Rows; ++q) {
+            const int64_t row = batch * kL1Rows + q;
             if (row >= N) break;
             const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
             int32_t n_gt = 0, n_eq = 0;
-            for (int32_t j0 = lo[r]; j0 < hi[r]; j0 += kWarp) {
+            for (int32_t j0 = lo[q]; j0 < hi[q]; j0 += kWarp) {
                 const int32_t j = j0 + lane;
                 unsigned long long key;
-                if (j0 == lo[r]) key = key0[r];
-                else if (j0 == lo[r] + kWarp) key = key1[r];
-                else key = j < hi[r] ? __ldg(keys + j) : 0ull;
-                const int dig = j < hi[r] ? (int)(key >> 51) : -1;
-                n_gt += __popc(__ballot_sync(kFull, dig > d0));
-                const bool in = dig == d0;
+                if (j0 == lo[q]) key = key0[q];
+                else key = j < hi[q] ? __ldg(keys + j) : 0ull;
+                const bool in_range = j < hi[q];
+                const unsigned long long kp = key >> (64 - r);
+                n_gt += __popc(__ballot_sync(kFull, in_range && kp > P));
+                const bool in = in_range && kp == P;
                 n_eq += __popc(__ballot_sync(kFull, in));
-                if (in) atomicAdd(&s_hist[(key >> 38) & (kBins - 1)], 1u);
+                if (in) atomicAdd(&s_hist[(key >> shift) & digit_mask], 1u);
             }
-            if (lane == 0) rowstate[row] = make_int2(lo[r] + n_gt, lo[r] + n_gt + n_eq);
+            if (lane == 0) {
+                rowstate[row] = make_int2(lo[q] + n_gt, lo[q] + n_gt + n_eq);
+                if (n_eq > 0) active[atomicAdd(&hdr->n_active, 1u)] = (int32_t)row;
+            }
         }
     }
     __syncthreads();
-    flush_hist(s_hist, hist1, kBins);
-    if (last_block(&hdr->ticket[1])) find_digit(hdr, hist1, 1, s_warp);
+    flush_hist(s_hist, hist1, 1 << bits);
+    if (last_block(&hdr->ticket[1])) find_digit(hdr, hist1, 1 << bits, bits, shift, 1, false, s_warp);
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Levels 2..4: a thread per row (grid-stride) narrows the stored segment by the digit selected one level
-// up; the keys that remain are histogrammed on the current level's digit.
+// Levels 2..4 and the closing pass (level 5): a thread per ACTIVE row narrows the stored segment by the
+// digit selected one level up; for levels 2..4 the keys that remain are histogrammed on the next digit
+// and the last CTA selects it.  The active list is in no particular order; nothing here depends on it.
 __global__ void __launch_bounds__(kSelThreads)
-select_refine(int64_t N, int32_t ld, const double *__restrict__ gains, int level, AllocHeader *hdr,
-              unsigned long long *hist_all, int2 *__restrict__ rowstate) {
+select_refine(int32_t ld, const double *__restrict__ gains, int level, AllocHeader *hdr,
+              unsigned long long *hist_all, int2 *__restrict__ rowstate, const int32_t *__restrict__ active) {
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     if (*(volatile int32_t *)&hdr->status != 0) return;
-    const int bins = level_bins(level);
-    for (int b = threadIdx.x; b < bins; b += kSelThreads) s_hist[b] = 0;
-    __syncthreads();
-    const int shift_prev = level_shift(level - 1), shift_cur = level_shift(level);
+    const bool closing = level >= kLevels;
+    int bits = 0, shift = 0;
+    if (!closing) next_digit(hdr->resolved, &bits, &shift);
+    const int bins = 1 << bits;
+    if (!closing) {
+        for (int b = threadIdx.x; b < bins; b += kSelThreads) s_hist[b] = 0;
+        __syncthreads();
+    }
+    const int shift_prev = hdr->lv_shift[level - 1];
+    const unsigned long long mask_prev = (1ull << hdr->lv_bits[level - 1]) - 1ull;
     const unsigned long long d_prev = (unsigned long long)hdr->sel_digit[level - 1];
-    const unsigned long long mask_prev = kBins - 1, mask_cur = (unsigned long long)bins - 1;
-    const int64_t stride = (int64_t)gridDim.x * kSelThreads;
-    for (int64_t row = (int64_t)blockIdx.x * kSelThreads + threadIdx.x; row < N; row += stride) {
+    const unsigned long long mask_cur = (unsigned long long)bins - 1ull;
+    const unsigned int n_active = hdr->n_active;
+    const unsigned int stride = gridDim.x * kSelThreads;
+    for (unsigned int idx = blockIdx.x * kSelThreads + threadIdx.x; idx < n_active; idx += stride) {
+        const int64_t row = active[idx];
         const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
         const int2 st = rowstate[row];
         const int32_t p_hi = st.x, p_end = st.y;
-        if (p_hi >= p_end) continue;                   // nothing of this row is left in the threshold bin
         int32_t p = p_hi, new_hi = p_hi;
         while (p < p_end) {
             const unsigned long long key = __ldg(keys + p);
@@ -433,7 +574,7 @@ select_refine(int64_t N, int32_t ld, const double *__restrict__ gains, int level
             if (dp > d_prev) {
                 new_hi = p + 1;
             } else if (dp == d_prev) {
-                atomicAdd(&s_hist[(key >> shift_cur) & mask_cur], 1u);
+                if (!closing) atomicAdd(&s_hist[(key >> shift) & mask_cur], 1u);
             } else {
                 break;
             }
@@ -441,9 +582,11 @@ select_refine(int64_t N, int32_t ld, const double *__restrict__ gains, int level
         }
         if (new_hi != p_hi || p != p_end) rowstate[row] = make_int2(new_hi, p);
     }
+    if (closing) return;
     __syncthreads();
     flush_hist(s_hist, hist_all + (size_t)level * kBins, bins);
-    if (last_block(&hdr->ticket[level])) find_digit(hdr, hist_all + (size_t)level * kBins, level, s_warp);
+    if (last_block(&hdr->ticket[level]))
+        find_digit(hdr, hist_all + (size_t)level * kBins, bins, bits, shift, level, false, s_warp);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -641,19 +784,18 @@ exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ t
 
 // ---------------------------------------------------------------------------------------------------
 // Block sums of (p_hi, tied) in prompt order, and their exclusive scan by the last CTA.
-//   mode 0: rowstate is final    mode 1: narrow by the last digit first    mode 2: apply the exact labels first
+//   mode 0: rowstate is final    mode 2: apply the exact labels first
 // With `validate` the priors and counts of every prompt are checked here (a thread per row, coalesced).
 __global__ void __launch_bounds__(kSelThreads)
 select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
            const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar, int validate,
-           int64_t N, int32_t ld, const double *__restrict__ gains, int mode, int64_t B, AllocHeader *hdr,
+           int64_t N, int32_t ld, int mode, int64_t B, AllocHeader *hdr,
            int2 *__restrict__ rowstate, const int32_t *__restrict__ rowslot, const int32_t *__restrict__ tlabel,
            long long *bsum_hi, long long *bsum_t, int64_t NB) {
     __shared__ long long s_warp[kSelThreads / kWarp];
     const bool failed = *(volatile int32_t *)&hdr->status != 0;
     long long hi_sum = 0, t_sum = 0;
     if (!failed) {
-        const unsigned long long d_last = (unsigned long long)hdr->sel_digit[kLevels - 1];
         const int64_t row0 = (int64_t)blockIdx.x * kRowsPerBlock;
 #pragma unroll
         for (int q = 0; q < kRowsPerBlock / kSelThreads; ++q) {
@@ -662,18 +804,7 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
             if (validate && !load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row).ok)
                 raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);   // seen by the kernels that follow
             int2 st = rowstate[row];
-            if (mode == 1) {
-                const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-                int32_t p = st.x, new_hi = st.x;
-                while (p < st.y) {
-                    const unsigned long long dp = __ldg(keys + p) & 4095ull;
-                    if (dp > d_last) new_hi = p + 1;
-                    else if (dp < d_last) break;
-                    ++p;
-                }
-                st = make_int2(new_hi, p);
-                rowstate[row] = st;
-            } else if (mode == 2) {
+            if (mode == 2) {
                 const int32_t slot = rowslot[row];
                 const int label = slot >= 0 ? tlabel[slot] : 0;
                 st = make_int2(st.x + (label == 2), st.x + (label == 2) + (label == 1));
@@ -834,9 +965,11 @@ template <int E>
 static void launch_level0(bool vec2, int grid, cudaStream_t s, const int32_t *cap, int32_t cap_scalar, int64_t N,
                           int32_t ld, const double *gains, int64_t B, const Workspace &w) {
     if (vec2)
-        select_level0<E, true><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist, w.sketch, w.sk_ld);
+        select_level0<E, true><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_coarse,
+                                                            w.hist_fine, w.sketch, w.sk_ld);
     else
-        select_level0<E, false><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist, w.sketch, w.sk_ld);
+        select_level0<E, false><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_coarse,
+                                                             w.hist_fine, w.sketch, w.sk_ld);
 }
 
 }  // namespace hora
@@ -887,6 +1020,12 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     }
     const bool vec2 = (ld % 2 == 0) && ((reinterpret_cast<uintptr_t>(gains) & 15u) == 0);
     const int rows_per_cta = kSelThreads / kWarp;
+    if (B > 0) {
+        const int64_t every = (N + kSampleRows - 1) / kSampleRows;
+        const int64_t n_sample = (N + every - 1) / every;
+        select_estimate<<<clamp_grid((n_sample + rows_per_cta - 1) / rows_per_cta, 4), kSelThreads, 0, s>>>(
+            cap, cap_scalar, N, ld, every, gains, B, w.hdr, w.hist_est);
+    }
     const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 4);
     const int grid1 = clamp_grid((N + rows_per_cta * kL1Rows - 1) / (rows_per_cta * kL1Rows), 6);
     if (ld > 128)
@@ -897,31 +1036,28 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         launch_level0<2>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
     const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     if (B > 0) {
-        select_level1<<<grid1, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, w.hdr, w.hist + kBins, w.sketch, w.sk_ld,
-                                                    w.rowstate);
-        for (int level = 2; level < kLevels; ++level)
-            select_refine<<<grid_rows, kSelThreads, 0, s>>>(N, ld, gains, level, w.hdr, w.hist, w.rowstate);
-        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 1,
-                                                   N, ld, gains, 1, B, w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi,
-                                                   w.bsum_t, NB);
+        select_level1<<<grid1, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, w.hdr, w.hist_lv + kBins, w.sketch,
+                                                    w.sk_ld, w.rowstate, w.active);
+        for (int level = 2; level <= kLevels; ++level)     // levels 2..4, then the closing pass
+            select_refine<<<2 * kSmCount, kSelThreads, 0, s>>>(ld, gains, level, w.hdr, w.hist_lv, w.rowstate, w.active);
+        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 1, N, ld, 0, B, w.hdr,
+                                                   w.rowstate, nullptr, nullptr, w.bsum_hi, w.bsum_t, NB);
         if (exact) {
             exact_collect<<<grid_rows, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
                                                             gains, w.hdr, w.rowstate, w.rowslot, w.tkeys, w.tcounts);
             exact_rank<<<1, 1024, 0, s>>>(B, w.hdr, w.tkeys, w.tcounts, w.tlabel);
-            select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 0,
-                                                       N, ld, gains, 2, B, w.hdr, w.rowstate, w.rowslot, w.tlabel,
-                                                       w.bsum_hi, w.bsum_t, NB);
+            select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 0, N, ld, 2, B,
+                                                       w.hdr, w.rowstate, w.rowslot, w.tlabel, w.bsum_hi, w.bsum_t, NB);
         }
     } else {
         if (cudaMemsetAsync(w.rowstate, 0, sizeof(int2) * (size_t)N, s) != cudaSuccess) return HORA_ERR_CUDA;
-        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 1,
-                                                   N, ld, gains, 0, B, w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi,
-                                                   w.bsum_t, NB);
+        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 1, N, ld, 0, B, w.hdr,
+                                                   w.rowstate, nullptr, nullptr, w.bsum_hi, w.bsum_t, NB);
     }
     select_out<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, flags, w.hdr,
                                                w.rowstate, w.bsum_hi, w.bsum_t, w.objpart, NB, delta, G, group_offsets,
                                                info_dev);
-    count_launches(B > 0 ? (exact ? 10 : 7) : 3);
+    count_launches(B > 0 ? (exact ? 13 : 10) : 3);
     return cuda_ok(cudaGetLastError());
 }
 
