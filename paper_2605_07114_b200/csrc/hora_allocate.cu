@@ -12,10 +12,10 @@
 //             finish locates the 13-bit digit of the threshold and, if it is inside the window, its 23-bit
 //             prefix; otherwise the selection simply goes on from 13 bits.  The same pass validates the
 //             rows, sums the caps and writes a 2-byte sketch of every 8th key (its top 16 bits).
-//   level 1   a warp per four rows: a row is non-increasing, so its keys with the resolved prefix form ONE
+//   level 1   a thread per row: a row is non-increasing, so its keys with the resolved prefix form ONE
 //             contiguous segment, which the sketch brackets to within 8 keys on each side; only the
-//             bracket is read (coalesced), the segment [p_hi, p_lo) stored, its next 13 bits histogrammed,
-//             and rows whose segment is not empty are appended to a list.
+//             bracket is read, the segment [p_hi, p_lo) stored, its next 13 bits histogrammed, and rows
+//             whose segment is not empty are appended to a list.
 //   level 2-4 a thread per listed row narrows its segment by the digit just selected and histograms the
 //             next one (13 bits at a time until all 64 are resolved), then a last narrowing pass.
 //   sum       p_hi = #keys > lambda, p_lo - p_hi = #keys == lambda per row; block sums and their scan give
@@ -427,15 +427,14 @@ select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Level 1: a warp per four rows.  r bits of the threshold are known (23 after a window hit, else 13);
-// call P that prefix.  The sketch holds the top 16 bits of the first (largest) key of every group of 8
-// keys.  Compared at min(r, 16) bits: groups whose first key is above P form a prefix of G1 groups,
-// groups whose first key is above or equal a prefix of G2 >= G1 groups.  Every key with prefix P
-// therefore sits in groups G1-1 .. G2-1, and so does the boundary between "above" and "equal"; only
-// those groups are read (coalesced), classified on all r bits, and the keys with prefix P histogrammed
-// on the next digit.  Rows that keep a non-empty segment are appended to the active list.
-constexpr int kL1Rows = 4;      // rows a warp works on at once: their loads are in flight together
-
+// Level 1: a thread per row.  r bits of the threshold are known (23 after a window hit, else 13); call
+// P that prefix.  The sketch holds the top 16 bits of the first (largest) key of every group of 8 keys.
+// Compared at min(r, 16) bits: groups whose first key is above P form a prefix of G1 groups, groups whose
+// first key is above or equal a prefix of G2 >= G1 groups.  Every key with prefix P therefore sits in
+// groups G1-1 .. G2-1, and so does the boundary between "above" and "equal"; the thread walks only those
+// keys (a handful after a window hit), classifies them on all r bits and histograms the ones with
+// prefix P on the next digit.  Rows that keep a non-empty segment are appended to the active list.
+// A warp per row was tried first: with a million rows the per-row issue slots, not memory, set its time.
 __global__ void __launch_bounds__(kSelThreads)
 select_level1(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
               const double *__restrict__ gains, AllocHeader *hdr, unsigned long long *hist1,
@@ -450,87 +449,60 @@ select_level1(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
     const int r = hdr->resolved;
     const unsigned long long P = hdr->prefix_key >> (64 - r);
     const int sk_shift = r < 16 ? 16 - r : 0;                    // sketch entries compared at min(r, 16) bits
-    const int Psk = (int)((hdr->prefix_key >> 48) >> sk_shift);
+    const unsigned Psk = (unsigned)((hdr->prefix_key >> 48) >> sk_shift);
     int bits, shift;
     next_digit(r, &bits, &shift);
     const unsigned long long digit_mask = (1ull << bits) - 1ull;
-    const int64_t warp0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5);
-    const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
-    const int64_t n_batches = (N + kL1Rows - 1) / kL1Rows;
-    for (int64_t batch = warp0; batch < n_batches; batch += stride) {
-        int32_t capi[kL1Rows], lo[kL1Rows], hi[kL1Rows];
-        // ---- sketches of all rows of the batch (independent loads), then their brackets ----
+    const int64_t stride = (int64_t)gridDim.x * kSelThreads;
+    for (int64_t base = (int64_t)blockIdx.x * kSelThreads; base < N; base += stride) {
+        const int64_t row = base + threadIdx.x;
+        int32_t n_eq = 0;
+        if (row < N) {
+            int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
+            capi = capi < 0 ? 0 : (capi > ld ? ld : capi);
+            const int n_groups = (capi + 7) >> 3;
+            // the sketch row is 16-byte aligned and padded to a multiple of 8 entries
+            const uint4 *sk4 = reinterpret_cast<const uint4 *>(sketch + row * (int64_t)sk_ld);
+            int G1 = 0, G2 = 0;
+            for (int g0 = 0; g0 < n_groups; g0 += 8) {
+                const uint4 v = __ldg(sk4 + (g0 >> 3));
+                const unsigned w[4] = {v.x, v.y, v.z, v.w};
+                bool below = false;
 #pragma unroll
-        for (int q = 0; q < kL1Rows; ++q) {
-            const int64_t row = batch * kL1Rows + q;
-            capi[q] = 0;
-            if (row < N) {
-                const int32_t cp = cap ? __ldg(cap + row) : cap_scalar;
-                capi[q] = cp < 0 ? 0 : (cp > ld ? ld : cp);
-            }
-        }
-        if (ld <= 8 * kWarp) {                                   // one sketch entry per lane covers the row
-            int dig[kL1Rows];
-#pragma unroll
-            for (int q = 0; q < kL1Rows; ++q) {
-                const int64_t row = batch * kL1Rows + q;
-                const int n_groups = (capi[q] + 7) >> 3;
-                dig[q] = lane < n_groups ? (int)(__ldg(sketch + row * (int64_t)sk_ld + lane) >> sk_shift) : -1;
-            }
-#pragma unroll
-            for (int q = 0; q < kL1Rows; ++q) {
-                const int G1 = __popc(__ballot_sync(kFull, dig[q] > Psk));
-                const int G2 = __popc(__ballot_sync(kFull, dig[q] >= Psk));
-                lo[q] = G1 > 0 ? (G1 - 1) << 3 : 0;
-                hi[q] = (G2 << 3) > capi[q] ? capi[q] : (G2 << 3);
-            }
-        } else {
-#pragma unroll
-            for (int q = 0; q < kL1Rows; ++q) {
-                const int64_t row = batch * kL1Rows + q;
-                const int n_groups = (capi[q] + 7) >> 3;
-                int G1 = 0, G2 = 0;
-                for (int g0 = 0; g0 < n_groups; g0 += kWarp) {
-                    const int g = g0 + lane;
-                    const int dig = g < n_groups ? (int)(__ldg(sketch + row * (int64_t)sk_ld + g) >> sk_shift) : -1;
-                    G1 += __popc(__ballot_sync(kFull, dig > Psk));
-                    G2 += __popc(__ballot_sync(kFull, dig >= Psk));
+                for (int i = 0; i < 4; ++i) {
+                    const unsigned e0 = (w[i] & 0xFFFFu) >> sk_shift, e1 = (w[i] >> 16) >> sk_shift;
+                    const bool v0 = g0 + 2 * i < n_groups, v1 = g0 + 2 * i + 1 < n_groups;
+                    G1 += (v0 && e0 > Psk) + (v1 && e1 > Psk);
+                    G2 += (v0 && e0 >= Psk) + (v1 && e1 >= Psk);
+                    below |= (v1 && e1 < Psk);
                 }
-                lo[q] = G1 > 0 ? (G1 - 1) << 3 : 0;
-                hi[q] = (G2 << 3) > capi[q] ? capi[q] : (G2 << 3);
+                if (below) break;                                // entries only decrease from here on
             }
-        }
-        // ---- first 32 keys of every bracket (independent loads), then whatever is left ----
-        unsigned long long key0[kL1Rows];
-#pragma unroll
-        for (int q = 0; q < kL1Rows; ++q) {
-            const int64_t row = batch * kL1Rows + q;
+            const int32_t lo = G1 > 0 ? (G1 - 1) << 3 : 0;
+            const int32_t hi = (G2 << 3) > capi ? capi : (G2 << 3);
             const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-            const int32_t j = lo[q] + lane;
-            key0[q] = j < hi[q] ? __ldg(keys + j) : 0ull;
-        }
-#pragma unroll
-        for (int q = 0; q < kL1Rows; ++q) {
-            const int64_t row = batch * kL1Rows + q;
-            if (row >= N) break;
-            const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-            int32_t n_gt = 0, n_eq = 0;
-            for (int32_t j0 = lo[q]; j0 < hi[q]; j0 += kWarp) {
-                const int32_t j = j0 + lane;
-                unsigned long long key;
-                if (j0 == lo[q]) key = key0[q];
-                else key = j < hi[q] ? __ldg(keys + j) : 0ull;
-                const bool in_range = j < hi[q];
+            int32_t n_gt = 0;
+            for (int32_t j = lo; j < hi; ++j) {
+                const unsigned long long key = __ldg(keys + j);
                 const unsigned long long kp = key >> (64 - r);
-                n_gt += __popc(__ballot_sync(kFull, in_range && kp > P));
-                const bool in = in_range && kp == P;
-                n_eq += __popc(__ballot_sync(kFull, in));
-                if (in) atomicAdd(&s_hist[(key >> shift) & digit_mask], 1u);
+                if (kp > P) {
+                    ++n_gt;
+                } else if (kp == P) {
+                    ++n_eq;
+                    atomicAdd(&s_hist[(key >> shift) & digit_mask], 1u);
+                } else {
+                    break;                                       // the row is sorted: nothing further can match
+                }
             }
-            if (lane == 0) {
-                rowstate[row] = make_int2(lo[q] + n_gt, lo[q] + n_gt + n_eq);
-                if (n_eq > 0) active[atomicAdd(&hdr->n_active, 1u)] = (int32_t)row;
-            }
+            rowstate[row] = make_int2(lo + n_gt, lo + n_gt + n_eq);
+        }
+        // append the rows that keep a segment: one counter update per warp
+        const unsigned keep = __ballot_sync(kFull, n_eq > 0);
+        if (keep) {
+            unsigned int slot0 = 0;
+            if (lane == 0) slot0 = atomicAdd(&hdr->n_active, (unsigned int)__popc(keep));
+            slot0 = __shfl_sync(kFull, slot0, 0);
+            if (n_eq > 0) active[slot0 + __popc(keep & ((1u << lane) - 1u))] = (int32_t)row;
         }
     }
     __syncthreads();
@@ -1027,7 +999,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
             cap, cap_scalar, N, ld, every, gains, B, w.hdr, w.hist_est);
     }
     const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 4);
-    const int grid1 = clamp_grid((N + rows_per_cta * kL1Rows - 1) / (rows_per_cta * kL1Rows), 6);
+    const int grid1 = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     if (ld > 128)
         launch_level0<8>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
     else if (ld > 64)
