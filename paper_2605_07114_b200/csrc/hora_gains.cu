@@ -14,10 +14,71 @@ namespace hora {
 
 constexpr int kGainsWarps = 8;
 constexpr int kTile = 8;                      // consecutive rows a warp takes at a time
+constexpr int kCtaRows = kGainsWarps * kTile; // rows a CTA stages per step
 
-// A warp takes kTile consecutive rows at a time.  Lane i (< kTile) loads row i's prior, count and cap
-// (one coalesced load per array) ONE TILE AHEAD, so that latency is hidden behind the arithmetic of the
-// current tile; the values reach the other lanes by shuffles.
+// One chunk of 32*E entries of one row, starting at column k0.  FULL: the chunk lies entirely below the
+// row's cap and inside the row, so no entry needs masking.
+template <int E, bool VEC2, bool FULL>
+__device__ __forceinline__ void gains_chunk(double a, double b, double ab, int32_t capi, int32_t ld, int32_t k0,
+                                            int lane, double &carry, double *__restrict__ out, double2 *wr, const double2 *rd) {
+    constexpr int P = E / 2;                              // 16-byte chunks per lane
+    constexpr bool kStaged = VEC2 && (P > 1);
+    const int32_t k = k0 + lane * E;
+    // factors of entries k .. k+E-1: num = a (k = 0) or b + k - 1, then +1 each; den = a + b + k, then +1 each
+    const double x = b + (double)(k - 1), y = ab + (double)k;
+    const double n0 = (k == 0) ? a : x;
+    double S[E + 1];
+    S[E] = 1.0;
+#pragma unroll
+    for (int m = E - 1; m >= 0; --m) S[m] = S[m + 1] * (y + (double)m);
+    double pt = n0;
+#pragma unroll
+    for (int m = 1; m < E; ++m) pt *= x + (double)m;
+    const double r = 1.0 / S[0];
+    double inc = pt * r;                                  // this lane's E-factor product
+#pragma unroll
+    for (int d = 1; d < kWarp; d <<= 1) {
+        const double t = shfl_up_f64(inc, d);
+        if (lane >= d) inc *= t;
+    }
+    double excl = shfl_up_f64(inc, 1);
+    if (lane == 0) excl = 1.0;
+    const double total = shfl_idx_f64(inc, kWarp - 1);
+    double pm = (carry * excl * r) * n0;                  // running numerator product times everything shared
+    carry *= total;
+#pragma unroll
+    for (int m = 0; m < E; m += 2) {                      // E is even: entries are produced and stored in pairs
+        double g0 = pm * S[m + 1];
+        pm *= x + (double)(m + 1);
+        double g1 = pm * S[m + 2];
+        if (m + 2 < E) pm *= x + (double)(m + 2);
+        if (!FULL) {
+            if (k + m >= capi) g0 = 0.0;
+            if (k + m + 1 >= capi) g1 = 0.0;
+        }
+        if (kStaged) {
+            wr[(m >> 1) ^ ((lane >> (P == 4 ? 1 : 2)) & (P - 1))] = make_double2(g0, g1);   // (lane*P + p) >> 3
+        } else if (VEC2) {
+            if (FULL || k + m < ld) *reinterpret_cast<double2 *>(out + k + m) = make_double2(g0, g1);
+        } else {
+            if (FULL || k + m < ld) out[k + m] = g0;
+            if (FULL || k + m + 1 < ld) out[k + m + 1] = g1;
+        }
+    }
+    if (kStaged) {
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < P; ++q) {
+            const double2 v = rd[q * kWarp];
+            const int32_t col = k0 + 2 * (q * kWarp + lane);
+            if (FULL || col < ld) *reinterpret_cast<double2 *>(out + col) = v;
+        }
+        __syncwarp();
+    }
+}
+
+// A CTA stages the posterior parameters of 64 consecutive rows in shared memory (one coalesced load per
+// array, issued one step ahead and parked in registers meanwhile); each warp then takes 8 of those rows.
 template <int E, bool VEC2>
 __global__ void __launch_bounds__(kGainsWarps *kWarp, 3)
 gains_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
@@ -26,89 +87,53 @@ gains_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, 
     // Staging slab: a lane produces E consecutive entries, but a store instruction should cover one
     // contiguous 512-byte run of the row (full 32-byte sectors; 16-byte pieces at a 64-byte stride cost
     // twice the L1-to-L2 traffic).  Pairs go through shared memory with an XOR swizzle on the 16-byte
-    // chunk index that keeps both the lane-major writes and the row-major reads free of bank conflicts.
-    constexpr int P = E / 2;                              // 16-byte chunks per lane
+    // chunk index (chunk ch of the row sits at ch ^ ((ch >> 3) & (P-1))) that keeps both the lane-major
+    // writes and the row-major reads free of bank conflicts.
+    constexpr int P = E / 2;
     constexpr bool kStaged = VEC2 && (P > 1);
     __shared__ double2 s_stage[kStaged ? kGainsWarps * kWarp * P : 1];
-    double2 *slab = s_stage + (kStaged ? (threadIdx.x >> 5) * kWarp * P : 0);
-    const int lane = lane_id();
-    const int64_t n_tiles = (N + kTile - 1) / kTile;
-    const int64_t tile0 = (int64_t)blockIdx.x * kGainsWarps + (threadIdx.x >> 5);
-    const int64_t stride = (int64_t)gridDim.x * kGainsWarps;
-    auto fetch = [&](int64_t tile) {
+    __shared__ double s_a[2][kCtaRows], s_b[2][kCtaRows];
+    __shared__ int32_t s_cap[2][kCtaRows];
+    const int lane = lane_id(), warp = threadIdx.x >> 5;
+    double2 *slab = s_stage + (kStaged ? warp * kWarp * P : 0);
+    // lane-major write: chunks lane*P + p, p = 0..P-1, swizzled within the lane's group of P chunks;
+    // row-major read: chunks q*32 + lane, swizzled by bits 3.. of the chunk index = bits 3.. of the lane
+    double2 *wr = slab + lane * P;
+    const double2 *rd = slab + (lane ^ ((lane >> 3) & (P - 1)));
+    const int64_t n_steps = (N + kCtaRows - 1) / kCtaRows;
+    auto fetch = [&](int64_t step) {
         Posterior p;
         p.a = p.b = 1.0;
         p.cap = 0;
         p.ok = true;
-        const int64_t row = tile * kTile + lane;
-        if (tile < n_tiles && lane < kTile && row < N)
+        const int64_t row = step * kCtaRows + threadIdx.x;
+        if (step < n_steps && threadIdx.x < kCtaRows && row < N)
             p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row);
         return p;
     };
-    Posterior nxt = fetch(tile0);
-    for (int64_t tile = tile0; tile < n_tiles; tile += stride) {
-        const Posterior cur = nxt;
-        nxt = fetch(tile + stride);
-        if (!cur.ok) raise_status(status_dev, HORA_ERR_INVALID_VALUE);
-        const int rows = (int)((N - tile * kTile < kTile) ? N - tile * kTile : kTile);
-        for (int i = 0; i < rows; ++i) {
-            const bool ok = __shfl_sync(kFull, (int)cur.ok, i) != 0;
-            const double a = ok ? shfl_idx_f64(cur.a, i) : 1.0, b = ok ? shfl_idx_f64(cur.b, i) : 1.0;
-            const int32_t capi = __shfl_sync(kFull, cur.cap, i);
+    Posterior nxt = fetch(blockIdx.x);
+    int buf = 0;
+    for (int64_t step = blockIdx.x; step < n_steps; step += gridDim.x, buf ^= 1) {
+        if (threadIdx.x < kCtaRows) {
+            if (!nxt.ok) raise_status(status_dev, HORA_ERR_INVALID_VALUE);
+            s_a[buf][threadIdx.x] = nxt.ok ? nxt.a : 1.0;
+            s_b[buf][threadIdx.x] = nxt.ok ? nxt.b : 1.0;
+            s_cap[buf][threadIdx.x] = nxt.cap;
+        }
+        __syncthreads();                                  // buf was last read two steps ago: safe to have overwritten it
+        nxt = fetch(step + gridDim.x);
+        const int64_t row0 = step * kCtaRows + warp * kTile;
+        for (int i = 0; i < kTile && row0 + i < N; ++i) {
+            const double a = s_a[buf][warp * kTile + i], b = s_b[buf][warp * kTile + i];
+            const int32_t capi = s_cap[buf][warp * kTile + i];
             const double ab = a + b;
-            double *out = gains + (tile * kTile + i) * (int64_t)ld;
+            double *out = gains + (row0 + i) * (int64_t)ld;
             double carry = 1.0;
             for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E) {
-                const int32_t k = k0 + lane * E;
-                // factors of entries k .. k+E-1: num = a (k = 0) or b + k - 1, then +1 each; den = a + b + k, then +1 each
-                const double x = b + (double)(k - 1), y = ab + (double)k;
-                const double n0 = (k == 0) ? a : x;
-                double S[E + 1];
-                S[E] = 1.0;
-#pragma unroll
-                for (int m = E - 1; m >= 0; --m) S[m] = S[m + 1] * (y + (double)m);
-                double pt = n0;
-#pragma unroll
-                for (int m = 1; m < E; ++m) pt *= x + (double)m;
-                const double r = 1.0 / S[0];
-                double inc = pt * r;                     // this lane's E-factor product
-#pragma unroll
-                for (int d = 1; d < kWarp; d <<= 1) {
-                    const double t = shfl_up_f64(inc, d);
-                    if (lane >= d) inc *= t;
-                }
-                double excl = shfl_up_f64(inc, 1);
-                if (lane == 0) excl = 1.0;
-                const double total = shfl_idx_f64(inc, kWarp - 1);
-                double pm = (carry * excl * r) * n0;     // running numerator product times everything shared
-                carry *= total;
-#pragma unroll
-                for (int m = 0; m < E; m += 2) {         // E is even: entries are produced and stored in pairs
-                    const double g0 = (k + m < capi) ? pm * S[m + 1] : 0.0;
-                    pm *= x + (double)(m + 1);
-                    const double g1 = (k + m + 1 < capi) ? pm * S[m + 2] : 0.0;
-                    if (m + 2 < E) pm *= x + (double)(m + 2);
-                    if (kStaged) {
-                        const int ch = lane * P + (m >> 1);
-                        slab[ch ^ ((ch >> 3) & (P - 1))] = make_double2(g0, g1);
-                    } else if (VEC2) {
-                        if (k + m < ld) *reinterpret_cast<double2 *>(out + k + m) = make_double2(g0, g1);
-                    } else {
-                        if (k + m < ld) out[k + m] = g0;
-                        if (k + m + 1 < ld) out[k + m + 1] = g1;
-                    }
-                }
-                if (kStaged) {
-                    __syncwarp();
-#pragma unroll
-                    for (int q = 0; q < P; ++q) {
-                        const int ch = q * kWarp + lane;
-                        const double2 v = slab[ch ^ ((ch >> 3) & (P - 1))];
-                        const int32_t col = k0 + 2 * ch;
-                        if (col < ld) *reinterpret_cast<double2 *>(out + col) = v;
-                    }
-                    __syncwarp();
-                }
+                if (k0 + kWarp * E <= capi)               // capi <= ld: the chunk is inside the row as well
+                    gains_chunk<E, VEC2, true>(a, b, ab, capi, ld, k0, lane, carry, out, wr, rd);
+                else
+                    gains_chunk<E, VEC2, false>(a, b, ab, capi, ld, k0, lane, carry, out, wr, rd);
             }
         }
     }
@@ -118,8 +143,7 @@ template <int E>
 static hora_status_t launch_e(const double *alpha, const double *beta, double alpha0, double beta0, const int32_t *c,
                               int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N, int32_t ld, double *gains,
                               int32_t *status_dev, cudaStream_t stream) {
-    const int64_t tiles = (N + kTile - 1) / kTile;
-    const int grid = clamp_grid((tiles + kGainsWarps - 1) / kGainsWarps, 3);
+    const int grid = clamp_grid((N + kCtaRows - 1) / kCtaRows, 3);
     const bool vec2 = (ld % 2 == 0) && ((reinterpret_cast<uintptr_t>(gains) & 15u) == 0);
     if (vec2)
         gains_kernel<E, true><<<grid, kGainsWarps * kWarp, 0, stream>>>(alpha, beta, alpha0, beta0, c, G0, cap,
