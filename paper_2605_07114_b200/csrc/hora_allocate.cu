@@ -157,35 +157,76 @@ __device__ __forceinline__ long long block_exclusive_sum(long long v, long long 
     return base + inc - v;
 }
 
-// Run by ONE CTA: find the digit d with  count(digit > d) < need <= count(digit >= d)  in hist[0..bins),
-// bins a power of two.  The digit sits at bit `shift` of the key.  With `append` it extends the digit
-// already recorded for `level` (the fine part of level 0) instead of starting a new one.
-__device__ void find_digit(AllocHeader *hdr, const unsigned long long *hist, int bins, int bits, int shift, int level,
-                           bool append, long long *s_warp) {
-    const int per = (bins + kSelThreads - 1) / kSelThreads;
-    const long long need = hdr->need;
-    const int top = bins - 1 - (int)threadIdx.x * per;      // this thread scans bins top, top-1, ..., top-per+1
+// Run by ONE CTA.  Scanning from the top bin down, find the bin where the running count reaches `need`:
+//   count(bins above d) < need <= count(bins above d) + count(d).
+// Returns d (or -1 if need is out of range) to every thread, with the count above d in *above_out and the
+// count of d in *count_out.  Two stages so that no thread walks memory serially: every thread sums a
+// contiguous run of bins (independent loads) and a block scan picks the run that holds the crossing; then
+// the first warp loads that run's bins one per lane (`per` <= 32) and a warp scan pins the bin.
+__device__ int locate_rank(const unsigned long long *hist, int bins, long long need, long long *above_out,
+                           long long *count_out, long long *s_warp) {
+    __shared__ long long s_found[3];                        // top bin of the run, count above the run, found flag
+    const int per = (bins + kSelThreads - 1) / kSelThreads; // <= 32 for bins <= 8192
+    const int top = bins - 1 - (int)threadIdx.x * per;      // this thread's run: bins top, top-1, ..., top-per+1
     long long local = 0;
+#pragma unroll 8
     for (int j = 0; j < per; ++j)
         if (top - j >= 0) local += (long long)__ldcg(hist + top - j);
+    if (threadIdx.x == 0) s_found[2] = 0;
     long long total;
     const long long above = block_exclusive_sum(local, &total, s_warp);
     if (need >= 1 && above < need && need <= above + local) {
-        long long run = above;
-        for (int j = 0; j < per && top - j >= 0; ++j) {
-            const long long cnt = (long long)__ldcg(hist + top - j);
-            if (run + cnt >= need) {
-                const int digit = top - j;
-                hdr->sel_digit[level] = append ? ((hdr->sel_digit[level] << bits) | digit) : digit;
-                hdr->lv_bits[level] = append ? hdr->lv_bits[level] + bits : bits;
-                hdr->lv_shift[level] = shift;
-                hdr->need = need - run;
-                hdr->prefix_key |= (unsigned long long)digit << shift;
-                hdr->resolved += bits;
-                break;
+        s_found[0] = top;
+        s_found[1] = above;
+        s_found[2] = 1;
+    }
+    __syncthreads();
+    int digit = -1;
+    const bool found = s_found[2] != 0;
+    const int run_top = (int)s_found[0];
+    const long long run_above = s_found[1];
+    __syncthreads();                                        // everyone has read the run before it is overwritten
+    if (found) {
+        if (threadIdx.x < kWarp) {
+            const int lane = threadIdx.x;
+            const int bin = run_top - lane;
+            const long long cnt = (lane < per && bin >= 0) ? (long long)__ldcg(hist + bin) : 0;
+            long long inc = cnt;
+#pragma unroll
+            for (int d = 1; d < kWarp; d <<= 1) {
+                const long long t = __shfl_up_sync(kFull, inc, d);
+                if (lane >= d) inc += t;
             }
-            run += cnt;
+            const bool here = run_above + inc - cnt < need && need <= run_above + inc;
+            if (here) {
+                s_found[0] = bin;
+                s_found[1] = run_above + inc - cnt;
+                s_found[2] = cnt;
+            }
         }
+        __syncthreads();
+        digit = (int)s_found[0];
+        *above_out = s_found[1];
+        *count_out = s_found[2];
+    }
+    __syncthreads();
+    return digit;
+}
+
+// Run by ONE CTA: select the next digit of the threshold from hist[0..bins), bins a power of two; the digit
+// sits at bit `shift` of the key.  With `append` it extends the digit already recorded for `level` (the
+// fine part of level 0) instead of starting a new one.
+__device__ void find_digit(AllocHeader *hdr, const unsigned long long *hist, int bins, int bits, int shift, int level,
+                           bool append, long long *s_warp) {
+    long long above = 0, count = 0;
+    const int digit = locate_rank(hist, bins, hdr->need, &above, &count, s_warp);
+    if (digit >= 0 && threadIdx.x == 0) {
+        hdr->sel_digit[level] = append ? ((hdr->sel_digit[level] << bits) | digit) : digit;
+        hdr->lv_bits[level] = append ? hdr->lv_bits[level] + bits : bits;
+        hdr->lv_shift[level] = shift;
+        hdr->need -= above;
+        hdr->prefix_key |= (unsigned long long)digit << shift;
+        hdr->resolved += bits;
     }
     __syncthreads();
 }
@@ -242,26 +283,13 @@ select_estimate(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, 
         const long long sample_cap = (long long)*(volatile unsigned long long *)&hdr->sample_cap;
         if (need < 1) need = 1;
         if (need > sample_cap) need = sample_cap;
-        const int per = kBins / kSelThreads;
-        const int top = kBins - 1 - (int)threadIdx.x * per;
-        long long local = 0;
-        for (int j = 0; j < per; ++j) local += (long long)__ldcg(hist + top - j);
-        long long total;
-        const long long above = block_exclusive_sum(local, &total, s_warp);
-        if (need >= 1 && above < need && need <= above + local) {
-            long long run = above;
-            for (int j = 0; j < per; ++j) {
-                const long long cnt = (long long)__ldcg(hist + top - j);
-                if (run + cnt >= need) {
-                    const int d = top - j;
-                    const bool upper_half = 2 * (need - run) <= cnt;      // counting from the top of the bin
-                    int lo = upper_half ? d : d - 1;
-                    lo = lo < 0 ? 0 : (lo > kBins - kWinBins ? kBins - kWinBins : lo);
-                    hdr->win_lo = lo;
-                    break;
-                }
-                run += cnt;
-            }
+        long long above = 0, count = 0;
+        const int d = locate_rank(hist, kBins, need, &above, &count, s_warp);
+        if (d >= 0 && threadIdx.x == 0) {
+            const bool upper_half = 2 * (need - above) <= count;          // counting from the top of the bin
+            int lo = upper_half ? d : d - 1;
+            lo = lo < 0 ? 0 : (lo > kBins - kWinBins ? kBins - kWinBins : lo);
+            hdr->win_lo = lo;
         }
     }
 }
@@ -464,34 +492,47 @@ select_level1(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
             // the sketch row is 16-byte aligned and padded to a multiple of 8 entries
             const uint4 *sk4 = reinterpret_cast<const uint4 *>(sketch + row * (int64_t)sk_ld);
             int G1 = 0, G2 = 0;
-            for (int g0 = 0; g0 < n_groups; g0 += 8) {
-                const uint4 v = __ldg(sk4 + (g0 >> 3));
-                const unsigned w[4] = {v.x, v.y, v.z, v.w};
-                bool below = false;
+            for (int g0 = 0; g0 < n_groups; g0 += 32) {          // 32 entries (four independent 16-byte loads) at a time
+                uint4 v[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const unsigned e0 = (w[i] & 0xFFFFu) >> sk_shift, e1 = (w[i] >> 16) >> sk_shift;
-                    const bool v0 = g0 + 2 * i < n_groups, v1 = g0 + 2 * i + 1 < n_groups;
-                    G1 += (v0 && e0 > Psk) + (v1 && e1 > Psk);
-                    G2 += (v0 && e0 >= Psk) + (v1 && e1 >= Psk);
-                    below |= (v1 && e1 < Psk);
+                for (int u = 0; u < 4; ++u)
+                    v[u] = (g0 + 8 * u < n_groups) ? __ldg(sk4 + (g0 >> 3) + u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int g = g0 + 8 * u + 2 * i;
+                        const unsigned e0 = (w[i] & 0xFFFFu) >> sk_shift, e1 = (w[i] >> 16) >> sk_shift;
+                        const bool v0 = g < n_groups, v1 = g + 1 < n_groups;
+                        G1 += (v0 && e0 > Psk) + (v1 && e1 > Psk);
+                        G2 += (v0 && e0 >= Psk) + (v1 && e1 >= Psk);
+                    }
                 }
-                if (below) break;                                // entries only decrease from here on
+                if (G2 < g0 + 32) break;                         // entries only decrease: the later ones are below P
             }
             const int32_t lo = G1 > 0 ? (G1 - 1) << 3 : 0;
             const int32_t hi = (G2 << 3) > capi ? capi : (G2 << 3);
             const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
             int32_t n_gt = 0;
-            for (int32_t j = lo; j < hi; ++j) {
-                const unsigned long long key = __ldg(keys + j);
-                const unsigned long long kp = key >> (64 - r);
-                if (kp > P) {
-                    ++n_gt;
-                } else if (kp == P) {
-                    ++n_eq;
-                    atomicAdd(&s_hist[(key >> shift) & digit_mask], 1u);
-                } else {
-                    break;                                       // the row is sorted: nothing further can match
+            bool stop = false;
+            for (int32_t j0 = lo; j0 < hi && !stop; j0 += 8) {   // one group of 8 keys (independent loads) at a time
+                unsigned long long key[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) key[u] = (j0 + u < hi) ? __ldg(keys + j0 + u) : 0ull;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const unsigned long long kp = key[u] >> (64 - r);
+                    if (j0 + u < hi && !stop) {
+                        if (kp > P) {
+                            ++n_gt;
+                        } else if (kp == P) {
+                            ++n_eq;
+                            atomicAdd(&s_hist[(key[u] >> shift) & digit_mask], 1u);
+                        } else {
+                            stop = true;                         // the row is sorted: nothing further can match
+                        }
+                    }
                 }
             }
             rowstate[row] = make_int2(lo + n_gt, lo + n_gt + n_eq);
