@@ -196,6 +196,16 @@ hora_status_t hora_group_advantage(const float *rewards, const int64_t *group_of
 hora_status_t hora_token_broadcast(const float *adv, const int64_t *token_offsets, int64_t R, int64_t T,
                                    float *token_adv, void *stream);
 
+/*
+ * hora_allocate_profile_events — measurement aid, no counterpart in the paper.  With two non-NULL cudaEvent_t
+ * handles (created by the caller with timing enabled), every following hora_allocate / hora_allocate_static
+ * call records `start_event` just before and `stop_event` just after the launch of its full-read selection
+ * pass (the kernel that reads the whole gains matrix) on the call's stream, so that kernel can be timed on
+ * the device without a profiler.  Pass NULLs to switch it off (the default).  Process-wide host setting; set
+ * it from the thread that issues the calls.
+ */
+void hora_allocate_profile_events(void *start_event, void *stop_event);
+
 const char *hora_status_string(hora_status_t status);   /* host: static string */
 int         hora_version(void);                         /* host: major*10000 + minor*100 + patch */
 uint64_t    hora_launch_count(void);                    /* host: kernels this library has launched so far in this

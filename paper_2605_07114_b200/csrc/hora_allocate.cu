@@ -974,6 +974,9 @@ __global__ void write_empty(int64_t B, int64_t *offsets, hora_alloc_info *info) 
     }
 }
 
+// Optional profiling aid (see hora_allocate_profile_events): events recorded around the full-read pass.
+static std::atomic<cudaEvent_t> g_prof_start{nullptr}, g_prof_stop{nullptr};
+
 template <int E>
 static void launch_level0(bool vec2, int grid, cudaStream_t s, const int32_t *cap, int32_t cap_scalar, int64_t N,
                           int32_t ld, const double *gains, int64_t B, const Workspace &w) {
@@ -986,6 +989,11 @@ static void launch_level0(bool vec2, int grid, cudaStream_t s, const int32_t *ca
 }
 
 }  // namespace hora
+
+extern "C" void hora_allocate_profile_events(void *start_event, void *stop_event) {
+    hora::g_prof_start.store(static_cast<cudaEvent_t>(start_event), std::memory_order_relaxed);
+    hora::g_prof_stop.store(static_cast<cudaEvent_t>(stop_event), std::memory_order_relaxed);
+}
 
 extern "C" size_t hora_allocate_workspace_bytes(int64_t N, int32_t ld, int32_t gains_is_null, uint32_t flags) {
     if (N < 0 || ld < 1) return 0;
@@ -1041,12 +1049,16 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     }
     const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 4);
     const int grid1 = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
+    const cudaEvent_t prof_start = g_prof_start.load(std::memory_order_relaxed);
+    const cudaEvent_t prof_stop = g_prof_stop.load(std::memory_order_relaxed);
+    if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_start, s);
     if (ld > 128)
         launch_level0<8>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
     else if (ld > 64)
         launch_level0<4>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
     else
         launch_level0<2>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
+    if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_stop, s);
     const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     if (B > 0) {
         select_level1<<<grid1, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, w.hdr, w.hist_lv + kBins, w.sketch,

@@ -23,7 +23,7 @@ ADV_GRPO, ADV_RLOO = 0, 1
 
 EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora_group_advantage",
            "hora_token_broadcast", "hora_status_string", "hora_version", "hora_launch_count",
-           "hora_allocate_static", "hora_allocate_static_capacity")
+           "hora_allocate_static", "hora_allocate_static_capacity", "hora_allocate_profile_events")
 
 
 class HoraError(RuntimeError):
@@ -60,6 +60,8 @@ def load() -> C.CDLL:
     L.hora_allocate_static.argtypes = [p, p, f64, f64, p, i32, p, i32, i64, i32, p, i64, u32, p, p, p, p, p]
     L.hora_allocate_static.restype = C.c_int
     L.hora_allocate_static_capacity.restype = C.c_size_t
+    L.hora_allocate_profile_events.argtypes = [p, p]
+    L.hora_allocate_profile_events.restype = None
     L.hora_group_advantage.argtypes = [p, p, i64, i32, C.c_float, i32, p, p, p]
     L.hora_group_advantage.restype = C.c_int
     L.hora_token_broadcast.argtypes = [p, p, i64, i64, p, p]
@@ -128,6 +130,13 @@ def hora_allocate(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gai
                               _ptr(info_dev, torch.uint8, "info_dev"), _ptr(workspace, torch.uint8, "workspace"),
                               0 if workspace is None else workspace.numel(), _stream())
     _check(rc, "hora_allocate")
+
+
+def hora_allocate_profile_events(start_event, stop_event):
+    """Record the given events (raw cudaEvent_t handles as ints, or None to switch off) around the full-read
+    selection kernel of every following hora_allocate call."""
+    load().hora_allocate_profile_events(None if start_event is None else C.c_void_p(int(start_event)),
+                                        None if stop_event is None else C.c_void_p(int(stop_event)))
 
 
 def hora_allocate_static_capacity() -> int:
