@@ -347,8 +347,8 @@ __device__ __forceinline__ void level0_fetch(Level0Item<E> &it, const int32_t *_
 
 template <int E>
 __device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t item, int32_t items_per_row,
-                                               int32_t ld, int lane, unsigned int *s_hist, unsigned int *s_fine,
-                                               int win_lo, uint16_t *__restrict__ sketch, int32_t sk_ld,
+                                               int32_t ld, int lane, unsigned int *s_hist, int win_lo,
+                                               uint16_t *__restrict__ sketch, int32_t sk_ld,
                                                long long *capsum, bool *bad) {
     const int64_t row = items_per_row == 1 ? item : item / items_per_row;
     const int32_t k0 = (int32_t)(item - row * items_per_row) * (kWarp * E);
@@ -365,12 +365,14 @@ __device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t 
     }
     *bad |= wrong;
     if ((k & 7) == 0 && k < ld) sketch[row * (int64_t)sk_ld + (k >> 3)] = (uint16_t)(it.v[0].x >> 48);
-    // one key: a 23-bit bin inside the window, a 13-bit bin outside it
+    // one key: a 23-bit bin inside the window, a 13-bit bin outside it.  The two histograms are one array
+    // (fine bins after the coarse ones), so the choice is an index select, not a branch.
     auto count_key = [&](unsigned long long key) {
-        const int bin = (int)(key >> 51);
-        const unsigned w = (unsigned)(bin - win_lo);
-        if (w < (unsigned)kWinBins) atomicAdd(&s_fine[w * kFinePerBin + ((unsigned)(key >> (51 - kFineBits)) & (kFinePerBin - 1))], 1u);
-        else atomicAdd(&s_hist[bin], 1u);
+        const unsigned hi = (unsigned)(key >> 32);
+        const unsigned bin = hi >> 19;
+        const unsigned w = bin - (unsigned)win_lo;
+        const unsigned fine = kBins + w * kFinePerBin + ((hi >> (19 - kFineBits)) & (kFinePerBin - 1));
+        atomicAdd(&s_hist[w < (unsigned)kWinBins ? fine : bin], 1u);
     };
     const int bin_first = (int)(it.v[0].x >> 51), bin_last = (int)(it.v[E / 2 - 1].y >> 51);
     if (k0 + kWarp * E <= it.capi) {                           // full item: every lane has E valid keys
@@ -398,11 +400,9 @@ __global__ void __launch_bounds__(kSelThreads, 4)
 select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
               const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist,
               unsigned long long *hist_fine, uint16_t *__restrict__ sketch, int32_t sk_ld) {
-    __shared__ unsigned int s_hist[kBins];
-    __shared__ unsigned int s_fine[kFineBins];
+    __shared__ unsigned int s_hist[kBins + kFineBins];     // 13-bit bins, then the window's 23-bit bins
     __shared__ long long s_warp[kSelThreads / kWarp];
-    for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
-    for (int b = threadIdx.x; b < kFineBins; b += kSelThreads) s_fine[b] = 0;
+    for (int b = threadIdx.x; b < kBins + kFineBins; b += kSelThreads) s_hist[b] = 0;
     __syncthreads();
     const int lane = lane_id();
     const int win_lo = hdr->win_lo;
@@ -417,16 +417,15 @@ select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
     level0_fetch<E, VEC2>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item0, lane, &bad);
     for (int64_t item = item0; item < n_items; item += 2 * stride) {
         level0_fetch<E, VEC2>(Bq, cap, cap_scalar, n_items, items_per_row, ld, gains, item + stride, lane, &bad);
-        level0_process<E>(A, item, items_per_row, ld, lane, s_hist, s_fine, win_lo, sketch, sk_ld, &capsum, &bad);
+        level0_process<E>(A, item, items_per_row, ld, lane, s_hist, win_lo, sketch, sk_ld, &capsum, &bad);
         level0_fetch<E, VEC2>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item + 2 * stride, lane, &bad);
         if (Bq.capi >= 0)
-            level0_process<E>(Bq, item + stride, items_per_row, ld, lane, s_hist, s_fine, win_lo, sketch, sk_ld, &capsum,
-                              &bad);
+            level0_process<E>(Bq, item + stride, items_per_row, ld, lane, s_hist, win_lo, sketch, sk_ld, &capsum, &bad);
     }
     if (bad) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);
     __syncthreads();
     flush_hist(s_hist, hist, kBins);
-    flush_hist(s_fine, hist_fine, kFineBins);
+    flush_hist(s_hist + kBins, hist_fine, kFineBins);
     long long tot;
     block_exclusive_sum(capsum, &tot, s_warp);
     if (threadIdx.x == 0 && tot) atomicAdd(&hdr->sum_cap, (unsigned long long)tot);
@@ -856,10 +855,12 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
 // U(Delta) = 1 - prod_{j<Delta} (b+j)/(a+b+j)  (Eq. appendix-hit-closed-form written as a product)
 __device__ __forceinline__ double hit_utility(double a, double b, int32_t Delta) {
     double q = 1.0, num = 1.0, den = 1.0;
-    const double ab = a + b;
+    double nb = b, nd = a + b;                              // b + j and a + b + j, advanced by exact additions
     for (int32_t j = 0; j < Delta; ++j) {
-        num *= b + (double)j;
-        den *= ab + (double)j;
+        num *= nb;
+        den *= nd;
+        nb += 1.0;
+        nd += 1.0;
         if ((j & 7) == 7) { q *= num / den; num = 1.0; den = 1.0; }
     }
     q *= num / den;
