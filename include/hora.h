@@ -62,7 +62,8 @@ enum { HORA_ADV_GRPO = 0, HORA_ADV_RLOO = 1 };
 /* Summary of one allocation; lives in DEVICE memory (64 bytes, 8-byte aligned). */
 typedef struct hora_alloc_info {
     int32_t status;        /* hora_status_t of the data-dependent checks */
-    int32_t reserved;
+    int32_t first_pass_bits; /* diagnostic: key bits the full-read pass resolved (23 when its sampled window held the
+                                threshold, else 13); 0 when B == 0 */
     double  lambda;        /* gain of the B-th best candidate (the selection threshold); 0 when B == 0 */
     int64_t n_above;       /* candidates strictly better than lambda (all taken) */
     int64_t n_tied;        /* candidates equal to lambda */

@@ -948,7 +948,7 @@ select_out(const double *__restrict__ alpha, const double *__restrict__ beta, do
             hdr->objective = s;
             if (info) {
                 info->status = status;
-                info->reserved = 0;
+                info->first_pass_bits = failed ? 0 : hdr->lv_bits[0];
                 info->lambda = failed ? 0.0 : hdr->lambda;
                 info->n_above = failed ? 0 : (int64_t)hdr->n_above;
                 info->n_tied = failed ? 0 : (int64_t)hdr->n_tied;
@@ -966,7 +966,7 @@ __global__ void write_empty(int64_t B, int64_t *offsets, hora_alloc_info *info) 
     if (offsets) offsets[0] = 0;
     if (info) {
         info->status = B > 0 ? HORA_ERR_INFEASIBLE : HORA_OK;
-        info->reserved = 0;
+        info->first_pass_bits = 0;
         info->lambda = 0.0;
         info->n_above = info->n_tied = info->n_tied_taken = 0;
         info->objective = 0.0;

@@ -33,7 +33,7 @@ class HoraError(RuntimeError):
 
 
 class hora_alloc_info(C.Structure):
-    _fields_ = [("status", C.c_int32), ("reserved", C.c_int32), ("lambda_", C.c_double),
+    _fields_ = [("status", C.c_int32), ("first_pass_bits", C.c_int32), ("lambda_", C.c_double),
                 ("n_above", C.c_int64), ("n_tied", C.c_int64), ("n_tied_taken", C.c_int64),
                 ("objective", C.c_double), ("sum_G", C.c_int64), ("sum_cap", C.c_int64)]
 
@@ -176,6 +176,7 @@ def hora_token_broadcast(adv, token_offsets, R, T, token_adv):
 @dataclass
 class AllocInfo:
     status: int
+    first_pass_bits: int
     lambda_: float
     n_above: int
     n_tied: int
@@ -189,7 +190,7 @@ def read_info(info_dev: torch.Tensor) -> AllocInfo:
     """Copy the 64-byte summary to the host (synchronises the current stream)."""
     raw = bytes(info_dev.cpu().numpy().tobytes())
     s = hora_alloc_info.from_buffer_copy(raw)
-    return AllocInfo(s.status, s.lambda_, s.n_above, s.n_tied, s.n_tied_taken, s.objective, s.sum_G, s.sum_cap)
+    return AllocInfo(s.status, s.first_pass_bits, s.lambda_, s.n_above, s.n_tied, s.n_tied_taken, s.objective, s.sum_G, s.sum_cap)
 
 
 class Allocator:

@@ -95,6 +95,7 @@ def run_and_compare(w, materialise=True):
     d, G, off, info = gu.gpu_allocate(w.alpha, w.beta, w.alpha0, w.beta0, w.c, w.G0, w.cap, w.ld, w.B,
                                       exact=w.exact_int, materialise=materialise)
     gu.assert_allocation_matches(w, d, G, off, info, d_o, lam_o, obj_o)
+    assert info.first_pass_bits == 23               # on these workloads the sampled window holds the threshold
     return d, G, off, info
 
 
@@ -192,6 +193,52 @@ def test_edge_budgets_and_caps():
     one[200] = 5
     d, G, off, info = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, one, ld, 4, exact=True)
     assert info.status == 0 and d[200] == 4 and d.sum() == 4
+
+
+@pytest.mark.parametrize("exact", [True, False])
+def test_allocation_when_the_sampled_window_misses(exact):
+    """The full-read pass refines 23 bits inside a window placed from a sample of every k-th row.  Here the
+    sampled rows (index multiple of 3) are all hopeless prompts and the others all saturated ones, so the
+    sample says nothing about the threshold and the window lands in the wrong place: the selection must
+    fall back to plain 13-bit digits and still reproduce the oracle."""
+    gu = _util()
+    N, G0, ld = 20000, 8, 96                      # N > 8192 rows, so only every 3rd row is sampled
+    idx = np.arange(N)
+    c = np.where(idx % 3 == 0, 0, G0).astype(np.int32)
+    cap = np.full(N, ld, np.int32)
+    rng = np.random.default_rng(5)
+    if exact:
+        alpha = beta = None
+    else:
+        alpha = np.exp(rng.uniform(np.log(0.5), np.log(2.0), N))
+        beta = np.exp(rng.uniform(np.log(0.5), np.log(2.0), N))
+    for B in (1000, 7 * N, 40 * N):
+        if exact:
+            d_o, _, lam, obj = orc.greedy_exact(None, None, 1.0, 1.0, c, G0, cap, B)
+        else:
+            d_o, _, lam, obj = orc.greedy_real(alpha, beta, 1.0, 1.0, c, G0, cap, B)
+        d, G, off, info = gu.gpu_allocate(alpha, beta, 1.0, 1.0, c, G0, cap, ld, B, exact=exact)
+        assert info.status == 0
+        assert info.first_pass_bits == 13            # the window did miss: this is the fallback being tested
+        np.testing.assert_array_equal(d, d_o)
+        assert abs(info.objective - obj) <= 1e-12 * obj
+
+
+def test_allocation_with_long_rows():
+    """ld > 256: several items per row in the full-read pass, several sketch chunks per row afterwards."""
+    gu = _util()
+    rng = np.random.default_rng(9)
+    N, G0, ld = 3000, 4, 700
+    alpha = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
+    beta = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    for B in (5000, 300000):
+        d_o, _, lam, obj = orc.greedy_real(alpha, beta, 1.0, 1.0, c, G0, cap, B)
+        d, G, off, info = gu.gpu_allocate(alpha, beta, 1.0, 1.0, c, G0, cap, ld, B, exact=False)
+        assert info.status == 0
+        np.testing.assert_array_equal(d, d_o)
+        assert abs(info.lambda_ - lam) <= 1e-12 * lam
 
 
 def test_allocation_status_codes():
