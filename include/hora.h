@@ -168,6 +168,36 @@ hora_status_t hora_allocate_static(const double *alpha, const double *beta, doub
                                    void *stream);
 
 /*
+ * hora_allocate_batched — many independent allocation problems in one call (the paper's appendix "Training
+ * configurations": Phase-B allocation is run on mini-batches of the training batch, e.g. four shards of 15
+ * prompts, each with its own budget, and Proposition 1 holds within each shard).
+ *
+ * Segment s covers prompts seg_offsets_host[s] .. seg_offsets_host[s+1]-1 and hands out budgets_host[s]
+ * rollouts among them, exactly as hora_allocate would on that segment alone (same gains bit for bit, same tie
+ * rules, same exact mode).  One CTA solves one segment in shared memory; no gains matrix is materialised.
+ *
+ *   alpha .. ld            as for hora_gains (device arrays over all N prompts)
+ *   seg_offsets_host       HOST array [S+1], non-decreasing, [0] == 0, [S] == N
+ *   budgets_host           HOST array [S], 0 <= budgets[s] <= sum of the segment's caps
+ *   delta, G               int32 [N] out;  group_offsets int64 [N+1] out over all prompts, may be NULL
+ *   info_dev               device array [S] of per-segment summaries (first_pass_bits is 0), may be NULL;
+ *                          data-dependent failures are per segment: that segment's status is set and its
+ *                          delta / G are zero, other segments are unaffected
+ *   workspace              device scratch, 256-byte aligned, hora_allocate_batched_workspace_bytes(N, S)
+ * Limits: a segment may hold at most 256 prompts and 176 KiB of keys (prompts * ld * 8 bytes); beyond that the
+ * call returns HORA_ERR_WORKSPACE and hora_allocate should be used for that problem.  The two host arrays are
+ * copied to the device during the call and may be reused as soon as it returns.
+ */
+size_t hora_allocate_batched_workspace_bytes(int64_t N, int64_t S);
+
+hora_status_t hora_allocate_batched(const double *alpha, const double *beta, double alpha0, double beta0,
+                                    const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar,
+                                    int64_t N, int32_t ld, const int64_t *seg_offsets_host,
+                                    const int64_t *budgets_host, int64_t S, uint32_t flags, int32_t *delta,
+                                    int32_t *G, int64_t *group_offsets, hora_alloc_info *info_dev,
+                                    void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * hora_group_advantage — group-relative advantages over ragged groups (Sec. 3.1 for GRPO; the RLOO
  * compatibility paragraph of Sec. 4 for the leave-one-out form).
  *

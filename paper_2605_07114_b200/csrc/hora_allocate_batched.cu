@@ -1,0 +1,427 @@
+// hora_allocate_batched: many small, independent allocation problems in one launch.
+//
+// The paper runs Phase-B allocation on mini-batches of the training batch (four shards of Gamma/4 = 15
+// prompts, each with its own share of the budget; appendix "Training configurations"), and Proposition 1
+// holds within each shard.  Here a shard ("segment") is a run of consecutive prompts with its own budget,
+// and one CTA solves one segment entirely in shared memory:
+//   1  gain rows of the segment's prompts, computed with the arithmetic of hora_gains (same bits), never
+//      written to global memory;
+//   2  the B_s-th largest key by a radix selection over the shared-memory keys (11-bit digits);
+//   3  per row the number of keys above and equal to the threshold (binary search in the sorted row);
+//   4  ties: in prompt order (fp64 equality), or, in exact mode, by exact rational comparison of the at
+//      most one candidate per row that lies within 2^-30 of the threshold (pairwise, 256-bit products);
+//   5  Delta, G, the segment's summary.
+// Group offsets over all prompts are an exclusive scan of G by two small kernels afterwards.
+#include <algorithm>
+
+#include "hora_common.cuh"
+#include "hora_exact.cuh"
+#include "hora_gains_chunk.cuh"
+
+namespace hora {
+
+constexpr int kBThreads = 256;
+constexpr int kBWarps = kBThreads / kWarp;
+constexpr int kBMaxRows = 256;                 // prompts per segment (one thread per prompt in the row phases)
+constexpr int kBBins = 2048;                   // 11-bit digits
+constexpr size_t kBMaxSmem = 200 * 1024;       // keys + bookkeeping must fit this
+constexpr int kScanRows = 1024;                // rows per CTA in the offsets scan
+
+struct BatchedSmemFixed {
+    unsigned int hist[kBBins];
+    double a[kBMaxRows], b[kBMaxRows];
+    U128 num[kBMaxRows], den[kBMaxRows];
+    int32_t cap[kBMaxRows], p_hi[kBMaxRows], tied[kBMaxRows], band[kBMaxRows];
+    long long warp_tmp[kBWarps];
+    double obj_tmp[kBWarps];
+    long long found[3];
+    double lam_exact;
+    int status;
+};
+
+__device__ __forceinline__ long long bblock_exclusive_sum(long long v, long long *total, long long *s_warp) {
+    const int lane = lane_id(), warp = threadIdx.x >> 5;
+    long long inc = v;
+#pragma unroll
+    for (int d = 1; d < kWarp; d <<= 1) {
+        const long long t = __shfl_up_sync(kFull, inc, d);
+        if (lane >= d) inc += t;
+    }
+    __syncthreads();
+    if (lane == kWarp - 1) s_warp[warp] = inc;
+    __syncthreads();
+    long long base = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < kBWarps; ++w) {
+        const long long x = s_warp[w];
+        if (w < warp) base += x;
+        tot += x;
+    }
+    *total = tot;
+    return base + inc - v;
+}
+
+// Scanning from the top bin down, the bin where the running count reaches `need` (1-based); the count of
+// the bins above it goes to *above_out.  All threads get the result.  -1 if need is out of range.
+__device__ int blocate_rank(BatchedSmemFixed &sm, int bins, long long need, long long *above_out) {
+    const int per = bins / kBThreads > 0 ? bins / kBThreads : 1;
+    const int top = bins - 1 - (int)threadIdx.x * per;
+    long long local = 0;
+    for (int j = 0; j < per; ++j)
+        if (top - j >= 0) local += sm.hist[top - j];
+    if (threadIdx.x == 0) sm.found[2] = 0;
+    long long total;
+    const long long above = bblock_exclusive_sum(local, &total, sm.warp_tmp);
+    if (need >= 1 && above < need && need <= above + local) {
+        long long run = above;
+        for (int j = 0; j < per && top - j >= 0; ++j) {
+            const long long cnt = sm.hist[top - j];
+            if (run + cnt >= need) {
+                sm.found[0] = top - j;
+                sm.found[1] = run;
+                sm.found[2] = 1;
+                break;
+            }
+            run += cnt;
+        }
+    }
+    __syncthreads();
+    const bool ok = sm.found[2] != 0;
+    const int digit = ok ? (int)sm.found[0] : -1;
+    *above_out = ok ? sm.found[1] : 0;
+    __syncthreads();
+    return digit;
+}
+
+template <int E>
+__global__ void __launch_bounds__(kBThreads)
+allocate_batched_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
+                        const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
+                        int32_t ld, const int64_t *__restrict__ seg_off, const int64_t *__restrict__ budgets, int64_t S,
+                        uint32_t flags, int32_t *__restrict__ delta, int32_t *__restrict__ G,
+                        hora_alloc_info *__restrict__ info) {
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    BatchedSmemFixed &sm = *reinterpret_cast<BatchedSmemFixed *>(s_raw);
+    unsigned long long *keys = reinterpret_cast<unsigned long long *>(s_raw + sizeof(BatchedSmemFixed));
+    const int lane = lane_id(), warp = threadIdx.x >> 5;
+    const bool exact = (flags & HORA_FLAG_EXACT_INT) != 0;
+    for (int64_t s = blockIdx.x; s < S; s += gridDim.x) {
+        const int64_t r0 = seg_off[s];
+        const int n = (int)(seg_off[s + 1] - r0);
+        const long long B = budgets[s];
+        __syncthreads();
+        if (threadIdx.x == 0) sm.status = (B < 0) ? HORA_ERR_INVALID_VALUE : HORA_OK;
+        __syncthreads();
+        // ---- 1: gain rows into shared memory (a warp per row) ----
+        for (int r = warp; r < n; r += kBWarps) {
+            const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, r0 + r);
+            if (!p.ok && lane == 0) sm.status = HORA_ERR_INVALID_VALUE;
+            const double a = p.ok ? p.a : 1.0, b = p.ok ? p.b : 1.0;
+            if (lane == 0) { sm.a[r] = a; sm.b[r] = b; sm.cap[r] = p.cap; }
+            double carry = 1.0;
+            double *out = reinterpret_cast<double *>(keys + (size_t)r * ld);
+            for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E)
+                gains_chunk<E, false, false>(a, b, a + b, p.cap, ld, k0, lane, carry, out, nullptr, nullptr);
+        }
+        __syncthreads();
+        long long sum_cap;
+        bblock_exclusive_sum(threadIdx.x < n ? sm.cap[threadIdx.x] : 0, &sum_cap, sm.warp_tmp);
+        if (threadIdx.x == 0 && sm.status == HORA_OK && B > sum_cap) sm.status = HORA_ERR_INFEASIBLE;
+        __syncthreads();
+        // ---- 2: the B-th largest key ----
+        unsigned long long prefix = 0;
+        long long need = B;
+        const int total = n * ld;
+        if (sm.status == HORA_OK && B > 0) {
+            for (int level = 0; level < 6; ++level) {             // 5 x 11 + 9 = 64 bits, from the top
+                const int w = level < 5 ? 11 : 9;
+                const int sh = level < 5 ? 53 - 11 * level : 0;
+                for (int t = threadIdx.x; t < kBBins; t += kBThreads) sm.hist[t] = 0;
+                __syncthreads();
+                for (int i = threadIdx.x; i < total; i += kBThreads) {
+                    const int r = i / ld, col = i - r * ld;
+                    if (col < sm.cap[r]) {
+                        const unsigned long long key = keys[i];
+                        const bool match = level == 0 || ((key >> (sh + w)) == (prefix >> (sh + w)));
+                        if (match) atomicAdd(&sm.hist[(key >> sh) & ((1u << w) - 1u)], 1u);
+                    }
+                }
+                __syncthreads();
+                long long above;
+                const int digit = blocate_rank(sm, 1 << w, need, &above);
+                prefix |= (unsigned long long)(digit < 0 ? 0 : digit) << sh;
+                need -= above;
+            }
+        }
+        const unsigned long long lam_key = prefix;
+        // ---- 3: per row, keys above and equal to the threshold ----
+        int my_hi = 0, my_tied = 0, my_cap = 0;
+        const unsigned long long *row = keys + (size_t)threadIdx.x * ld;
+        if (threadIdx.x < n && sm.status == HORA_OK && B > 0) {
+            my_cap = sm.cap[threadIdx.x];
+            int lo = 0, hi = my_cap;
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (row[mid] > lam_key) lo = mid + 1; else hi = mid;
+            }
+            my_hi = lo;
+            while (my_hi + my_tied < my_cap && row[my_hi + my_tied] == lam_key) ++my_tied;
+        }
+        // ---- 4: ties ----
+        int my_delta = 0;
+        long long n_above = 0, n_tied = 0, n_taken = 0;
+        double lambda = B > 0 ? __longlong_as_double((long long)lam_key) : 0.0;
+        if (!exact) {
+            long long tot_hi, tot_t;
+            bblock_exclusive_sum(my_hi, &tot_hi, sm.warp_tmp);
+            const long long pre_t = bblock_exclusive_sum(my_tied, &tot_t, sm.warp_tmp);
+            const long long R = B - tot_hi;
+            long long take = R - pre_t;
+            take = take < 0 ? 0 : (take > my_tied ? my_tied : take);
+            my_delta = my_hi + (int)take;
+            n_above = tot_hi; n_tied = tot_t; n_taken = R;
+        } else {
+            // the one candidate of this row, if any, within 2^-30 (relative) of the fp64 threshold
+            const double lam = __longlong_as_double((long long)lam_key);
+            const unsigned long long k_hi = (unsigned long long)__double_as_longlong(lam * (1.0 + 9.313225746154785e-10));
+            const unsigned long long k_lo = (unsigned long long)__double_as_longlong(lam * (1.0 - 9.313225746154785e-10));
+            int q = my_hi, has = 0, err = 0;
+            if (threadIdx.x < n && sm.status == HORA_OK && B > 0) {
+                const double al = alpha ? __ldg(alpha + r0 + threadIdx.x) : alpha0;
+                const double be = beta ? __ldg(beta + r0 + threadIdx.x) : beta0;
+                if (!(al >= 1.0 && be >= 1.0 && al == floor(al) && be == floor(be))) err = HORA_ERR_NOT_INTEGER;
+                else if (al + be + (double)G0 + (double)ld >= 1048576.0) err = HORA_ERR_EXACT_RANGE;
+                if (q > 0 && row[q - 1] <= k_hi) {
+                    --q;
+                    if (q > 0 && row[q - 1] <= k_hi) err = err ? err : HORA_ERR_EXACT_RANGE;
+                }
+                has = (q < my_cap) && (row[q] >= k_lo);
+                if (has && q + 1 < my_cap && row[q + 1] >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
+                if (has && !err) {
+                    U128 nu, de;
+                    if (!exact_gain((unsigned long long)sm.a[threadIdx.x], (unsigned long long)sm.b[threadIdx.x],
+                                    (unsigned long long)q + 1, nu, de)) err = HORA_ERR_EXACT_RANGE;
+                    sm.num[threadIdx.x] = nu;
+                    sm.den[threadIdx.x] = de;
+                }
+                if (err) atomicCAS(&sm.status, 0, err);
+            }
+            if (threadIdx.x < kBMaxRows) sm.band[threadIdx.x] = (threadIdx.x < n && has && !err) ? 1 : 0;
+            long long tot_q;
+            bblock_exclusive_sum(q, &tot_q, sm.warp_tmp);          // has a barrier: num/den/band are visible after it
+            const long long Rp = B - tot_q;                        // rollouts to hand out inside the band
+            int better = 0, equal = 0;
+            if (threadIdx.x < n && sm.band[threadIdx.x] && sm.status == HORA_OK) {
+                for (int u = 0; u < n; ++u) {
+                    if (!sm.band[u] || u == (int)threadIdx.x) continue;
+                    const int sgn = cmp_products(sm.num[u], sm.den[threadIdx.x], sm.num[threadIdx.x], sm.den[u]);
+                    better += (sgn > 0) || (sgn == 0 && u < (int)threadIdx.x);
+                    equal += (sgn == 0);
+                }
+                my_delta = q + (better < Rp ? 1 : 0);
+                if (better == Rp - 1) {                            // this row holds the B-th best candidate
+                    int strictly = 0;
+                    for (int u = 0; u < n; ++u)
+                        if (sm.band[u] && u != (int)threadIdx.x &&
+                            cmp_products(sm.num[u], sm.den[threadIdx.x], sm.num[threadIdx.x], sm.den[u]) > 0) ++strictly;
+                    sm.found[0] = tot_q + strictly;
+                    sm.found[1] = equal + 1;
+                    sm.found[2] = Rp - strictly;
+                    const U128 nu = sm.num[threadIdx.x], de = sm.den[threadIdx.x];
+                    lambda = ((double)nu.hi * 18446744073709551616.0 + (double)nu.lo) /
+                             ((double)de.hi * 18446744073709551616.0 + (double)de.lo);
+                    sm.lam_exact = lambda;
+                }
+            } else {
+                my_delta = q;
+            }
+            __syncthreads();
+            if (B > 0 && sm.status == HORA_OK) {
+                n_above = sm.found[0]; n_tied = sm.found[1]; n_taken = sm.found[2];
+                lambda = sm.lam_exact;
+            }
+            __syncthreads();
+        }
+        // ---- 5: outputs and summary ----
+        const int status = sm.status;
+        const bool failed = status != HORA_OK;
+        if (threadIdx.x < n) {
+            delta[r0 + threadIdx.x] = failed ? 0 : my_delta;
+            G[r0 + threadIdx.x] = failed ? 0 : G0 + my_delta;
+        }
+        double obj = 0.0;
+        if (!failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE) && threadIdx.x < n && my_delta > 0)
+            obj = hit_utility(sm.a[threadIdx.x], sm.b[threadIdx.x], my_delta);
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) obj += __shfl_xor_sync(kFull, obj, d);
+        __syncthreads();
+        if (lane == 0) sm.obj_tmp[warp] = obj;
+        __syncthreads();
+        if (threadIdx.x == 0 && info != nullptr) {
+            double tot = 0.0;
+            for (int w = 0; w < kBWarps; ++w) tot += sm.obj_tmp[w];
+            hora_alloc_info o;
+            o.status = status;
+            o.first_pass_bits = 0;
+            o.lambda = failed ? 0.0 : lambda;
+            o.n_above = failed ? 0 : n_above;
+            o.n_tied = failed ? 0 : n_tied;
+            o.n_tied_taken = failed ? 0 : n_taken;
+            o.objective = failed ? 0.0 : tot;
+            o.sum_G = failed ? 0 : (long long)n * G0 + B;
+            o.sum_cap = sum_cap;
+            info[s] = o;
+        }
+    }
+}
+
+// ---- group offsets: exclusive scan of G over all prompts ----
+struct ScanHeader { unsigned int ticket; unsigned int pad; };
+
+__global__ void __launch_bounds__(kBThreads)
+scan_block_sums(const int32_t *__restrict__ G, int64_t N, long long *bsum, int64_t NB, ScanHeader *hdr) {
+    __shared__ long long s_warp[kBWarps];
+    __shared__ bool s_last;
+    const int64_t row0 = (int64_t)blockIdx.x * kScanRows;
+    long long v = 0;
+    for (int q = 0; q < kScanRows / kBThreads; ++q) {
+        const int64_t row = row0 + q * kBThreads + threadIdx.x;
+        if (row < N) v += G[row];
+    }
+    long long tot;
+    bblock_exclusive_sum(v, &tot, s_warp);
+    if (threadIdx.x == 0) bsum[blockIdx.x] = tot;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&hdr->ticket, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    long long run = 0;
+    for (int64_t b0 = 0; b0 < NB; b0 += kBThreads) {
+        const int64_t b = b0 + threadIdx.x;
+        const long long x = b < NB ? __ldcg(bsum + b) : 0;
+        long long t;
+        const long long e = bblock_exclusive_sum(x, &t, s_warp);
+        if (b < NB) bsum[b] = run + e;
+        run += t;
+    }
+}
+
+__global__ void __launch_bounds__(kBThreads)
+scan_write_offsets(const int32_t *__restrict__ G, int64_t N, const long long *__restrict__ bpre,
+                   int64_t *__restrict__ offsets) {
+    __shared__ long long s_warp[kBWarps];
+    constexpr int kPer = kScanRows / kBThreads;
+    const int64_t row0 = (int64_t)blockIdx.x * kScanRows + (int64_t)threadIdx.x * kPer;
+    int g[kPer];
+    long long v = 0;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+        g[q] = row0 + q < N ? G[row0 + q] : 0;
+        v += g[q];
+    }
+    long long tot;
+    long long pre = bblock_exclusive_sum(v, &tot, s_warp) + bpre[blockIdx.x];
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+        if (row0 + q < N) offsets[row0 + q] = pre;
+        pre += g[q];
+        if (row0 + q == N - 1) offsets[N] = pre;
+    }
+}
+
+struct BatchedWorkspace {
+    int64_t *seg_off, *budgets;
+    long long *bsum;
+    ScanHeader *hdr;
+    size_t bytes;
+};
+
+static BatchedWorkspace carve_batched(void *base, int64_t N, int64_t S) {
+    BatchedWorkspace w{};
+    size_t o = 0;
+    char *p = static_cast<char *>(base);
+    auto take = [&](size_t n) { char *q = p ? p + o : nullptr; o = (o + n + 255) & ~(size_t)255; return q; };
+    const int64_t NB = (N + kScanRows - 1) / kScanRows;
+    w.hdr = reinterpret_cast<ScanHeader *>(take(sizeof(ScanHeader)));
+    w.seg_off = reinterpret_cast<int64_t *>(take(sizeof(int64_t) * (size_t)(S + 1)));
+    w.budgets = reinterpret_cast<int64_t *>(take(sizeof(int64_t) * (size_t)(S > 0 ? S : 1)));
+    w.bsum = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)(NB > 0 ? NB : 1)));
+    w.bytes = o;
+    return w;
+}
+
+}  // namespace hora
+
+extern "C" size_t hora_allocate_batched_workspace_bytes(int64_t N, int64_t S) {
+    if (N < 0 || S < 0) return 0;
+    return hora::carve_batched(nullptr, N, S).bytes;
+}
+
+extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double *beta, double alpha0, double beta0,
+                                               const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar,
+                                               int64_t N, int32_t ld, const int64_t *seg_offsets_host,
+                                               const int64_t *budgets_host, int64_t S, uint32_t flags, int32_t *delta,
+                                               int32_t *G, int64_t *group_offsets, hora_alloc_info *info_dev,
+                                               void *workspace, size_t workspace_bytes, void *stream) {
+    using namespace hora;
+    if (N < 0 || S < 0 || ld < 1 || G0 < 0) return HORA_ERR_INVALID_ARG;
+    if ((alpha == nullptr) != (beta == nullptr)) return HORA_ERR_INVALID_ARG;
+    if (alpha == nullptr && !(alpha0 > 0.0 && beta0 > 0.0 && alpha0 < 1.0e300 && beta0 < 1.0e300))
+        return HORA_ERR_INVALID_ARG;
+    if (cap == nullptr && (cap_scalar < 0 || cap_scalar > ld)) return HORA_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE)) return HORA_ERR_INVALID_ARG;
+    if (seg_offsets_host == nullptr || (S > 0 && budgets_host == nullptr)) return HORA_ERR_INVALID_ARG;
+    if (seg_offsets_host[0] != 0 || seg_offsets_host[S] != N) return HORA_ERR_INVALID_ARG;
+    int64_t max_rows = 0;
+    for (int64_t s = 0; s < S; ++s) {
+        const int64_t n = seg_offsets_host[s + 1] - seg_offsets_host[s];
+        if (n < 0 || budgets_host[s] < 0) return HORA_ERR_INVALID_ARG;
+        max_rows = std::max(max_rows, n);
+    }
+    const size_t smem = sizeof(BatchedSmemFixed) + (size_t)max_rows * (size_t)ld * sizeof(unsigned long long);
+    if (max_rows > kBMaxRows || smem > kBMaxSmem) return HORA_ERR_WORKSPACE;   // segment too large for one CTA
+    if (N > 0 && (c == nullptr || delta == nullptr || G == nullptr)) return HORA_ERR_INVALID_ARG;
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HORA_ERR_WORKSPACE;
+    const BatchedWorkspace w = carve_batched(workspace, N, S);
+    if (workspace_bytes < w.bytes) return HORA_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(w.hdr, 0, sizeof(ScanHeader), st) != cudaSuccess) return HORA_ERR_CUDA;
+    if (cudaMemcpyAsync(w.seg_off, seg_offsets_host, sizeof(int64_t) * (size_t)(S + 1), cudaMemcpyHostToDevice, st) !=
+        cudaSuccess)
+        return HORA_ERR_CUDA;
+    if (S > 0 && cudaMemcpyAsync(w.budgets, budgets_host, sizeof(int64_t) * (size_t)S, cudaMemcpyHostToDevice, st) !=
+                     cudaSuccess)
+        return HORA_ERR_CUDA;
+    int launches = 0;
+    if (S > 0 && N > 0) {
+        const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (220 * 1024) / smem));
+        const int grid = clamp_grid(S, per_sm);
+        auto launch = [&](auto kernel) -> cudaError_t {
+            cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            kernel<<<grid, kBThreads, smem, st>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, w.seg_off,
+                                                  w.budgets, S, flags, delta, G, info_dev);
+            return cudaGetLastError();
+        };
+        cudaError_t e;
+        if (ld > 128) e = launch(allocate_batched_kernel<8>);
+        else if (ld > 64) e = launch(allocate_batched_kernel<4>);
+        else e = launch(allocate_batched_kernel<2>);
+        if (e != cudaSuccess) return HORA_ERR_CUDA;
+        ++launches;
+    }
+    if (group_offsets != nullptr) {
+        if (N == 0) {
+            if (cudaMemsetAsync(group_offsets, 0, sizeof(int64_t), st) != cudaSuccess) return HORA_ERR_CUDA;
+        } else {
+            const int64_t NB = (N + kScanRows - 1) / kScanRows;
+            scan_block_sums<<<(int)NB, kBThreads, 0, st>>>(G, N, w.bsum, NB, w.hdr);
+            scan_write_offsets<<<(int)NB, kBThreads, 0, st>>>(G, N, w.bsum, group_offsets);
+            launches += 2;
+        }
+    }
+    count_launches(launches);
+    return cuda_ok(cudaGetLastError());
+}

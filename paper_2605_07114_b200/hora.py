@@ -23,7 +23,8 @@ ADV_GRPO, ADV_RLOO = 0, 1
 
 EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora_group_advantage",
            "hora_token_broadcast", "hora_status_string", "hora_version", "hora_launch_count",
-           "hora_allocate_static", "hora_allocate_static_capacity", "hora_allocate_profile_events")
+           "hora_allocate_static", "hora_allocate_static_capacity", "hora_allocate_profile_events",
+           "hora_allocate_batched", "hora_allocate_batched_workspace_bytes")
 
 
 class HoraError(RuntimeError):
@@ -60,6 +61,11 @@ def load() -> C.CDLL:
     L.hora_allocate_static.argtypes = [p, p, f64, f64, p, i32, p, i32, i64, i32, p, i64, u32, p, p, p, p, p]
     L.hora_allocate_static.restype = C.c_int
     L.hora_allocate_static_capacity.restype = C.c_size_t
+    L.hora_allocate_batched_workspace_bytes.argtypes = [i64, i64]
+    L.hora_allocate_batched_workspace_bytes.restype = C.c_size_t
+    L.hora_allocate_batched.argtypes = [p, p, f64, f64, p, i32, p, i32, i64, i32, p, p, i64, u32, p, p, p, p, p,
+                                        C.c_size_t, p]
+    L.hora_allocate_batched.restype = C.c_int
     L.hora_allocate_profile_events.argtypes = [p, p]
     L.hora_allocate_profile_events.restype = None
     L.hora_group_advantage.argtypes = [p, p, i64, i32, C.c_float, i32, p, p, p]
@@ -130,6 +136,40 @@ def hora_allocate(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gai
                               _ptr(info_dev, torch.uint8, "info_dev"), _ptr(workspace, torch.uint8, "workspace"),
                               0 if workspace is None else workspace.numel(), _stream())
     _check(rc, "hora_allocate")
+
+
+def hora_allocate_batched_workspace_bytes(N, S) -> int:
+    return int(load().hora_allocate_batched_workspace_bytes(N, S))
+
+
+def hora_allocate_batched(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, seg_offsets_host, budgets_host,
+                          flags, delta, G, group_offsets, info_dev, workspace):
+    """seg_offsets_host / budgets_host: host int64 arrays (numpy or CPU tensors); info_dev: uint8[S*64] on device."""
+    import numpy as np
+    seg = np.ascontiguousarray(np.asarray(seg_offsets_host), dtype=np.int64)
+    bud = np.ascontiguousarray(np.asarray(budgets_host), dtype=np.int64)
+    S = int(seg.shape[0]) - 1
+    if bud.shape[0] != S:
+        raise ValueError("budgets_host must have one entry per segment")
+    rc = load().hora_allocate_batched(_ptr(alpha, torch.float64, "alpha"), _ptr(beta, torch.float64, "beta"), alpha0,
+                                      beta0, _ptr(c, torch.int32, "c"), G0, _ptr(cap, torch.int32, "cap"), cap_scalar,
+                                      N, ld, seg.ctypes.data_as(C.c_void_p), bud.ctypes.data_as(C.c_void_p), S, flags,
+                                      _ptr(delta, torch.int32, "delta"), _ptr(G, torch.int32, "G"),
+                                      _ptr(group_offsets, torch.int64, "group_offsets"),
+                                      _ptr(info_dev, torch.uint8, "info_dev"), _ptr(workspace, torch.uint8, "workspace"),
+                                      0 if workspace is None else workspace.numel(), _stream())
+    _check(rc, "hora_allocate_batched")
+
+
+def read_infos(info_dev: torch.Tensor, S: int):
+    """Per-segment summaries of hora_allocate_batched (synchronises the current stream)."""
+    raw = info_dev.cpu().numpy().tobytes()
+    out = []
+    for s in range(S):
+        x = hora_alloc_info.from_buffer_copy(raw[s * INFO_BYTES:(s + 1) * INFO_BYTES])
+        out.append(AllocInfo(x.status, x.first_pass_bits, x.lambda_, x.n_above, x.n_tied, x.n_tied_taken, x.objective,
+                             x.sum_G, x.sum_cap))
+    return out
 
 
 def hora_allocate_profile_events(start_event, stop_event):

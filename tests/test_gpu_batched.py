@@ -1,0 +1,140 @@
+"""hora_allocate_batched against the oracle run segment by segment (GPU, through the C ABI)."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+from oracle import hora_oracle as orc  # noqa: E402
+
+
+def run_batched(alpha, beta, a0, b0, c, G0, cap, ld, seg, budgets, exact):
+    from paper_2605_07114_b200 import hora
+    dev = "cuda"
+    t = lambda x: None if x is None else torch.from_numpy(np.ascontiguousarray(x)).to(dev)
+    N, S = len(c), len(budgets)
+    delta = torch.full((N,), -1, dtype=torch.int32, device=dev)
+    G = torch.full((N,), -1, dtype=torch.int32, device=dev)
+    off = torch.full((N + 1,), -1, dtype=torch.int64, device=dev)
+    info = torch.zeros(max(S, 1) * hora.INFO_BYTES, dtype=torch.uint8, device=dev)
+    ws = torch.empty(max(hora.hora_allocate_batched_workspace_bytes(N, S), 256), dtype=torch.uint8, device=dev)
+    hora.hora_allocate_batched(t(alpha), t(beta), a0, b0, t(c), G0, t(cap), 0, N, ld, seg, budgets,
+                               hora.FLAG_EXACT_INT if exact else 0, delta, G, off, info, ws)
+    torch.cuda.synchronize()
+    return delta.cpu().numpy(), G.cpu().numpy(), off.cpu().numpy(), hora.read_infos(info, S)
+
+
+def oracle_segments(alpha, beta, a0, b0, c, G0, cap, seg, budgets, exact):
+    d = np.zeros(len(c), np.int32)
+    lam, obj = [], []
+    for s, B in enumerate(budgets):
+        sl = slice(int(seg[s]), int(seg[s + 1]))
+        al = None if alpha is None else alpha[sl]
+        be = None if beta is None else beta[sl]
+        if exact:
+            ds, _, (ln, ldn), o = orc.greedy_exact(al, be, a0, b0, c[sl], G0, cap[sl], int(B))
+            lam.append(ln / ldn if ldn else 0.0)
+        else:
+            ds, _, l, o = orc.greedy_real(al, be, a0, b0, c[sl], G0, cap[sl], int(B))
+            lam.append(l)
+        d[sl] = ds
+        obj.append(o)
+    return d, lam, obj
+
+
+def random_problem(rng, S, G0, ld, real, max_rows=40):
+    sizes = rng.integers(1, max_rows + 1, S)
+    sizes[rng.integers(0, S)] = 1
+    seg = np.zeros(S + 1, np.int64)
+    np.cumsum(sizes, out=seg[1:])
+    N = int(seg[-1])
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    alpha = beta = None
+    if real:
+        alpha = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
+        beta = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
+    budgets = np.zeros(S, np.int64)
+    for s in range(S):
+        tot = int(cap[seg[s]:seg[s + 1]].sum())
+        budgets[s] = rng.choice([0, tot, int(rng.integers(0, tot + 1))], p=[0.05, 0.05, 0.9])
+    return alpha, beta, c, cap, seg, budgets
+
+
+@pytest.mark.parametrize("G0,ld", [(2, 24), (4, 60), (8, 130), (8, 256)])
+@pytest.mark.parametrize("real", [False, True])
+def test_batched_matches_oracle_per_segment(G0, ld, real):
+    rng = np.random.default_rng(G0 * 1000 + ld + real)
+    alpha, beta, c, cap, seg, budgets = random_problem(rng, 300, G0, ld, real)
+    d, G, off, infos = run_batched(alpha, beta, 1.0, 1.0, c, G0, cap, ld, seg, budgets, exact=not real)
+    d_o, lam_o, obj_o = oracle_segments(alpha, beta, 1.0, 1.0, c, G0, cap, seg, budgets, exact=not real)
+    np.testing.assert_array_equal(d, d_o)
+    np.testing.assert_array_equal(G, G0 + d_o)
+    exp_off = np.zeros(len(c) + 1, np.int64)
+    np.cumsum(G.astype(np.int64), out=exp_off[1:])
+    np.testing.assert_array_equal(off, exp_off)
+    for s, inf in enumerate(infos):
+        assert inf.status == 0
+        B = int(budgets[s])
+        assert inf.sum_G == (seg[s + 1] - seg[s]) * G0 + B
+        assert inf.sum_cap == int(cap[seg[s]:seg[s + 1]].sum())
+        if B > 0:
+            assert abs(inf.objective - obj_o[s]) <= 1e-12 * abs(obj_o[s])
+            assert abs(inf.lambda_ - lam_o[s]) <= 1e-12 * lam_o[s]
+            assert inf.n_above + inf.n_tied_taken == B and 1 <= inf.n_tied_taken <= inf.n_tied
+
+
+def test_paper_shard_shape_and_agreement_with_single_problem_call():
+    """Four shards of 15 prompts, 360 rollouts each (G = 32, G0 = 8), uniform prior, exact ties; and each
+    shard solved alone by hora_allocate gives the same allocation."""
+    import gpu_util as gu
+    rng = np.random.default_rng(60)
+    G0, shard, B, ld = 8, 15, 360, 360
+    N = 4 * shard
+    c = rng.choice(G0 + 1, size=N, p=[0.15] + [0.34 / 7] * 7 + [0.51]).astype(np.int32)
+    cap = np.full(N, ld, np.int32)
+    seg = np.arange(0, N + 1, shard, dtype=np.int64)
+    budgets = np.full(4, B, np.int64)
+    d, G, off, infos = run_batched(None, None, 1.0, 1.0, c, G0, cap, ld, seg, budgets, exact=True)
+    d_o, _, _ = oracle_segments(None, None, 1.0, 1.0, c, G0, cap, seg, budgets, exact=True)
+    np.testing.assert_array_equal(d, d_o)
+    for s in range(4):
+        sl = slice(s * shard, (s + 1) * shard)
+        d1, _, _, info1 = gu.gpu_allocate(None, None, 1.0, 1.0, c[sl], G0, cap[sl], ld, B, exact=True)
+        np.testing.assert_array_equal(d[sl], d1)
+        assert infos[s].n_above == info1.n_above and infos[s].n_tied == info1.n_tied
+        assert abs(infos[s].objective - info1.objective) <= 1e-13 * info1.objective
+    assert d[c == 0].mean() > d[c == G0].mean()          # hopeless prompts get more than saturated ones
+
+
+def test_a_failing_segment_leaves_the_others_alone():
+    rng = np.random.default_rng(3)
+    alpha, beta, c, cap, seg, budgets = random_problem(rng, 20, 4, 32, real=True, max_rows=10)
+    budgets[5] = int(cap[seg[5]:seg[6]].sum()) + 1       # infeasible
+    alpha[seg[9]] = -2.0                                 # invalid prior in segment 9
+    d, G, off, infos = run_batched(alpha, beta, 1.0, 1.0, c, 4, cap, 32, seg, budgets, exact=False)
+    assert infos[5].status == 3 and not d[seg[5]:seg[6]].any() and not G[seg[5]:seg[6]].any()
+    assert infos[9].status == 2 and not d[seg[9]:seg[10]].any()
+    ok = [s for s in range(20) if s not in (5, 9)]
+    b2, a2 = budgets.copy(), alpha.copy()
+    a2[seg[9]] = 1.0
+    d_o, _, _ = oracle_segments(a2, beta, 1.0, 1.0, c, 4, cap, seg, b2 * 0 + np.where(np.arange(20) == 5, 0, b2), False)
+    for s in ok:
+        assert infos[s].status == 0
+        np.testing.assert_array_equal(d[seg[s]:seg[s + 1]], d_o[seg[s]:seg[s + 1]])
+
+
+def test_segments_beyond_the_per_cta_limits_are_refused():
+    from paper_2605_07114_b200 import hora
+    N, ld = 600, 64
+    c = np.zeros(N, np.int32)
+    cap = np.full(N, ld, np.int32)
+    with pytest.raises(hora.HoraError) as e:
+        run_batched(None, None, 1.0, 1.0, c, 4, cap, ld, np.array([0, 300, 600]), np.array([10, 10]), exact=True)
+    assert e.value.code == hora.ERR_WORKSPACE
+    with pytest.raises(hora.HoraError) as e:
+        run_batched(None, None, 1.0, 1.0, c, 4, cap, ld, np.array([0, 300, 500]), np.array([10, 10]), exact=True)
+    assert e.value.code == hora.ERR_INVALID_ARG
