@@ -317,11 +317,50 @@ def run_ours(args):
         "allocation": {"lambda": info.lambda_, "n_above": info.n_above, "n_tied": info.n_tied,
                        "objective": info.objective},
     }
+    if world == 1:
+        out["batched"] = bench_batched(torch, hora, wl, dev)
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_sample)
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def bench_batched(torch, hora, wl, dev, shards=65536, shard_prompts=15, per_prompt=24, reps=20):
+    """Secondary measurement: hora_allocate_batched on the shape the paper trains with (shards of 15 prompts,
+    G0 = 8, 24 extra rollouts per prompt, uniform prior, exact ties), many shards in one call."""
+    rng = np.random.default_rng(15)
+    G0, ld = 8, shard_prompts * per_prompt
+    N = shards * shard_prompts
+    c_h = rng.choice(G0 + 1, size=N, p=[0.15] + [0.34 / 7] * 7 + [0.51]).astype(np.int32)
+    c = torch.from_numpy(c_h).to(dev)
+    seg = np.arange(0, N + 1, shard_prompts, dtype=np.int64)
+    budgets = np.full(shards, ld, np.int64)
+    delta = torch.empty(N, dtype=torch.int32, device=dev)
+    G = torch.empty(N, dtype=torch.int32, device=dev)
+    off = torch.empty(N + 1, dtype=torch.int64, device=dev)
+    info = torch.zeros(shards * hora.INFO_BYTES, dtype=torch.uint8, device=dev)
+    ws = torch.empty(hora.hora_allocate_batched_workspace_bytes(N, shards), dtype=torch.uint8, device=dev)
+
+    def call():
+        hora.hora_allocate_batched(None, None, 1.0, 1.0, c, G0, None, ld, N, ld, seg, budgets, hora.FLAG_EXACT_INT,
+                                   delta, G, off, info, ws)
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    if int(delta.sum().item()) != shards * ld:
+        raise RuntimeError("batched allocation did not hand out the whole budget")
+    return {"call": "hora_allocate_batched", "shards": shards, "prompts_per_shard": shard_prompts, "G0": G0, "ld": ld,
+            "budget_per_shard": ld, "ms": round(ms, 4), "shards_per_s": shards / (ms * 1e-3),
+            "prompts_per_s": N / (ms * 1e-3), "candidates_per_s": N * ld / (ms * 1e-3),
+            "note": "gains are computed in shared memory and never written out: bound by fp64/integer issue, not HBM"}
 
 
 # ------------------------------------------------------------------------------- oracle timing

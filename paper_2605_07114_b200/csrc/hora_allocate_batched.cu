@@ -35,6 +35,7 @@ struct BatchedSmemFixed {
     long long warp_tmp[kBWarps];
     double obj_tmp[kBWarps];
     long long found[3];
+    unsigned long long list_count;
     double lam_exact;
     int status;
 };
@@ -131,19 +132,34 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         // ---- 2: the B-th largest key ----
         unsigned long long prefix = 0;
         long long need = B;
-        const int total = n * ld;
         if (sm.status == HORA_OK && B > 0) {
+            // Levels 0 and 1 (top 22 bits) sweep the keys row by row (a warp per row, no index division);
+            // what still matches after them is a handful of keys, which are copied to a short list that the
+            // remaining levels work on.  The list reuses the bin array's neighbour: the band flags are not
+            // live yet, so p_hi/tied/band (3 x 256 words) hold up to 384 keys; a longer list keeps sweeping.
+            unsigned long long *list = reinterpret_cast<unsigned long long *>(sm.p_hi);
+            constexpr int kListCap = 3 * kBMaxRows / 2;
+            int n_list = -1;                                       // -1: still sweeping the rows
             for (int level = 0; level < 6; ++level) {             // 5 x 11 + 9 = 64 bits, from the top
                 const int w = level < 5 ? 11 : 9;
                 const int sh = level < 5 ? 53 - 11 * level : 0;
                 for (int t = threadIdx.x; t < kBBins; t += kBThreads) sm.hist[t] = 0;
                 __syncthreads();
-                for (int i = threadIdx.x; i < total; i += kBThreads) {
-                    const int r = i / ld, col = i - r * ld;
-                    if (col < sm.cap[r]) {
-                        const unsigned long long key = keys[i];
-                        const bool match = level == 0 || ((key >> (sh + w)) == (prefix >> (sh + w)));
-                        if (match) atomicAdd(&sm.hist[(key >> sh) & ((1u << w) - 1u)], 1u);
+                if (n_list < 0) {
+                    for (int r = warp; r < n; r += kBWarps) {
+                        const unsigned long long *rk = keys + (size_t)r * ld;
+                        const int cp = sm.cap[r];
+                        for (int col = lane; col < cp; col += kWarp) {
+                            const unsigned long long key = rk[col];
+                            if (level == 0 || (key >> (sh + w)) == (prefix >> (sh + w)))
+                                atomicAdd(&sm.hist[(key >> sh) & ((1u << w) - 1u)], 1u);
+                        }
+                    }
+                } else {
+                    for (int i = threadIdx.x; i < n_list; i += kBThreads) {
+                        const unsigned long long key = list[i];
+                        if ((key >> (sh + w)) == (prefix >> (sh + w)))
+                            atomicAdd(&sm.hist[(key >> sh) & ((1u << w) - 1u)], 1u);
                     }
                 }
                 __syncthreads();
@@ -151,8 +167,26 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                 const int digit = blocate_rank(sm, 1 << w, need, &above);
                 prefix |= (unsigned long long)(digit < 0 ? 0 : digit) << sh;
                 need -= above;
+                // after this level: how many keys still match?  (the selected bin's count)
+                const long long left = digit < 0 ? 0 : (long long)sm.hist[digit];
+                if (n_list < 0 && level >= 1 && level < 5 && left <= kListCap) {
+                    if (threadIdx.x == 0) sm.list_count = 0;
+                    __syncthreads();
+                    for (int r = warp; r < n; r += kBWarps) {
+                        const unsigned long long *rk = keys + (size_t)r * ld;
+                        const int cp = sm.cap[r];
+                        for (int col = lane; col < cp; col += kWarp) {
+                            const unsigned long long key = rk[col];
+                            if ((key >> sh) == (prefix >> sh)) list[atomicAdd(&sm.list_count, 1ull)] = key;
+                        }
+                    }
+                    __syncthreads();
+                    n_list = (int)sm.list_count;
+                }
+                __syncthreads();
             }
         }
+        __syncthreads();
         const unsigned long long lam_key = prefix;
         // ---- 3: per row, keys above and equal to the threshold ----
         int my_hi = 0, my_tied = 0, my_cap = 0;
