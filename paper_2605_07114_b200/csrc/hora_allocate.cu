@@ -36,6 +36,7 @@
 
 #include "hora_common.cuh"
 #include "hora_exact.cuh"
+#include "hora_gains_chunk.cuh"
 
 namespace hora {
 
@@ -246,6 +247,25 @@ __device__ __forceinline__ void next_digit(int resolved, int *bits, int *shift) 
     *shift = 64 - resolved - w;
 }
 
+// Run by ONE CTA after the sample histogram is complete: scale the rank B to the sample and put the two-bin
+// window around the bin it falls in — towards the upper neighbour when the rank falls in the upper half of
+// that bin's count, else towards the lower one.
+__device__ void place_window(AllocHeader *hdr, const unsigned long long *hist, int64_t B, int64_t n_sample, int64_t N,
+                             long long *s_warp) {
+    long long need = (long long)((double)B * (double)n_sample / (double)N + 0.5);
+    const long long sample_cap = (long long)*(volatile unsigned long long *)&hdr->sample_cap;
+    if (need < 1) need = 1;
+    if (need > sample_cap) need = sample_cap;
+    long long above = 0, count = 0;
+    const int d = locate_rank(hist, kBins, need, &above, &count, s_warp);
+    if (d >= 0 && threadIdx.x == 0) {
+        const bool upper_half = 2 * (need - above) <= count;              // counting from the top of the bin
+        int lo = upper_half ? d : d - 1;
+        lo = lo < 0 ? 0 : (lo > kBins - kWinBins ? kBins - kWinBins : lo);
+        hdr->win_lo = lo;
+    }
+}
+
 // ---------------------------------------------------------------------------------------------------
 // Estimate: a warp per sampled row (every `every`-th row), histogram of the top 13 bits.  The last CTA
 // scales the rank B to the sample and places the two-bin window around the bin it falls in: towards the
@@ -278,21 +298,7 @@ select_estimate(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, 
     long long tot;
     block_exclusive_sum(capsum, &tot, s_warp);
     if (threadIdx.x == 0 && tot) atomicAdd(&hdr->sample_cap, (unsigned long long)tot);
-    if (last_block(&hdr->ticket[15])) {
-        // rank of the threshold within the sample
-        long long need = (long long)((double)B * (double)n_sample / (double)N + 0.5);
-        const long long sample_cap = (long long)*(volatile unsigned long long *)&hdr->sample_cap;
-        if (need < 1) need = 1;
-        if (need > sample_cap) need = sample_cap;
-        long long above = 0, count = 0;
-        const int d = locate_rank(hist, kBins, need, &above, &count, s_warp);
-        if (d >= 0 && threadIdx.x == 0) {
-            const bool upper_half = 2 * (need - above) <= count;          // counting from the top of the bin
-            int lo = upper_half ? d : d - 1;
-            lo = lo < 0 ? 0 : (lo > kBins - kWinBins ? kBins - kWinBins : lo);
-            hdr->win_lo = lo;
-        }
-    }
+    if (last_block(&hdr->ticket[15])) place_window(hdr, hist, B, n_sample, N, s_warp);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -304,6 +310,44 @@ select_estimate(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, 
 // non-negative and non-increasing (first key below +inf, every key <= its predecessor, compared as
 // unsigned integers), sums the caps, and writes the sketch: the top 16 bits of keys 0, 8, 16, ... (zero
 // beyond the cap).
+// End of the full-read pass (shared by the pass that reads a materialised matrix and by the fused pass that
+// produces the matrix): merge this CTA's histograms, add up the caps, and let the last CTA select the 13-bit
+// digit of the threshold and, on a window hit, its 23-bit prefix.
+__device__ void level0_finish(AllocHeader *hdr, unsigned long long *hist, unsigned long long *hist_fine,
+                              const unsigned int *s_hist, int win_lo, long long capsum, bool bad, int64_t B,
+                              long long *s_warp) {
+    if (bad) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);
+    __syncthreads();
+    flush_hist(s_hist, hist, kBins);
+    flush_hist(s_hist + kBins, hist_fine, kFineBins);
+    long long tot;
+    block_exclusive_sum(capsum, &tot, s_warp);
+    if (threadIdx.x == 0 && tot) atomicAdd(&hdr->sum_cap, (unsigned long long)tot);
+    if (last_block(&hdr->ticket[0])) {
+        const unsigned long long sum_cap = *(volatile unsigned long long *)&hdr->sum_cap;
+        // the 13-bit counts of the window bins are the sums of their fine bins
+        for (int wb = 0; wb < kWinBins; ++wb) {
+            long long part = 0;
+            for (int f = threadIdx.x; f < kFinePerBin; f += kSelThreads)
+                part += (long long)__ldcg(hist_fine + wb * kFinePerBin + f);
+            long long sum;
+            block_exclusive_sum(part, &sum, s_warp);
+            if (threadIdx.x == 0) hist[win_lo + wb] = (unsigned long long)sum;
+        }
+        if (threadIdx.x == 0) {
+            if ((unsigned long long)B > sum_cap) raise_status(&hdr->status, HORA_ERR_INFEASIBLE);
+            hdr->need = B;
+        }
+        __threadfence();
+        __syncthreads();
+        find_digit(hdr, hist, kBins, kDigitBits, 51, 0, false, s_warp);
+        const int d0 = hdr->sel_digit[0];
+        const unsigned w = (unsigned)(d0 - win_lo);
+        if (hdr->resolved == kDigitBits && w < (unsigned)kWinBins)        // inside the window: 10 more bits for free
+            find_digit(hdr, hist_fine + w * kFinePerBin, kFinePerBin, kFineBits, 51 - kFineBits, 0, true, s_warp);
+    }
+}
+
 template <int E>
 struct Level0Item {
     ulonglong2 v[E / 2];           // this lane's E consecutive keys, in pairs (E is even)
@@ -423,35 +467,144 @@ select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
         if (Bq.capi >= 0)
             level0_process<E>(Bq, item + stride, items_per_row, ld, lane, s_hist, win_lo, sketch, sk_ld, &capsum, &bad);
     }
-    if (bad) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);
+    level0_finish(hdr, hist, hist_fine, s_hist, win_lo, capsum, bad, B, s_warp);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Fused form of the full-read pass, used when the caller passes no gains matrix: the kernel that BUILDS the
+// rows (same arithmetic, same bits as hora_gains) counts the keys while they are still in registers, so the
+// matrix is written once and not read back in full.  The taps below plug into gains_chunk.
+
+// counts every valid key of the lane on its top 13 bits only (the sampled estimate)
+template <int E>
+struct CoarseTap {
+    unsigned long long key[E];
+    unsigned int *s_hist;
+    __device__ __forceinline__ void pair(int m, double g0, double g1) {
+        key[m] = (unsigned long long)__double_as_longlong(g0);
+        key[m + 1] = (unsigned long long)__double_as_longlong(g1);
+    }
+    __device__ __forceinline__ void finish(int32_t, int32_t k, int32_t capi, int32_t) {
+        const int valid = capi - k;
+#pragma unroll
+        for (int m = 0; m < E; ++m)
+            if (m < valid) atomicAdd(&s_hist[(unsigned)(key[m] >> 51)], 1u);
+    }
+};
+
+// the level-0 bookkeeping: window/coarse histogram and the sketch
+template <int E>
+struct Level0Tap {
+    unsigned long long key[E];
+    unsigned int *s_hist;
+    uint16_t *sk_row;              // sketch row of the prompt being built
+    int win_lo;
+    __device__ __forceinline__ void pair(int m, double g0, double g1) {
+        key[m] = (unsigned long long)__double_as_longlong(g0);
+        key[m + 1] = (unsigned long long)__double_as_longlong(g1);
+    }
+    __device__ __forceinline__ void count_key(unsigned long long k64) const {
+        const unsigned hi = (unsigned)(k64 >> 32);
+        const unsigned bin = hi >> 19;
+        const unsigned w = bin - (unsigned)win_lo;
+        const unsigned fine = kBins + w * kFinePerBin + ((hi >> (19 - kFineBits)) & (kFinePerBin - 1));
+        atomicAdd(&s_hist[w < (unsigned)kWinBins ? fine : bin], 1u);
+    }
+    __device__ __forceinline__ void finish(int32_t, int32_t k, int32_t capi, int32_t ld) {
+        if ((k & 7) == 0 && k < ld) sk_row[k >> 3] = (uint16_t)(key[0] >> 48);   // masked entries are 0.0: sketch 0
+        const int valid = capi - k;
+        const unsigned bin_first = (unsigned)(key[0] >> 51), bin_last = (unsigned)(key[E - 1] >> 51);
+        if (valid >= E && bin_first == bin_last && bin_first - (unsigned)win_lo >= (unsigned)kWinBins) {
+            atomicAdd(&s_hist[bin_first], (unsigned int)E);
+        } else {
+#pragma unroll
+            for (int m = 0; m < E; ++m)
+                if (m < valid) count_key(key[m]);
+        }
+    }
+};
+
+// Estimate for the fused pass: the sampled rows are computed, not read.
+template <int E>
+__global__ void __launch_bounds__(kSelThreads)
+select_estimate_fused(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
+                      const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
+                      int64_t N, int32_t ld, int64_t every, int64_t B, AllocHeader *hdr, unsigned long long *hist) {
+    __shared__ unsigned int s_hist[kBins];
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
+    __syncthreads();
+    const int lane = lane_id();
+    const int64_t n_sample = (N + every - 1) / every;
+    const int64_t warp0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5);
+    const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
+    long long capsum = 0;
+    CoarseTap<E> tap;
+    tap.s_hist = s_hist;
+    for (int64_t sidx = warp0; sidx < n_sample; sidx += stride) {
+        const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, sidx * every);
+        if (lane == 0) capsum += p.cap;
+        const double a = p.ok ? p.a : 1.0, b = p.ok ? p.b : 1.0;
+        double carry = 1.0;
+        for (int32_t k0 = 0; k0 < p.cap; k0 += kWarp * E)
+            gains_chunk<E, false, false>(a, b, a + b, p.cap, ld, k0, lane, carry, nullptr, nullptr, nullptr, tap);
+    }
     __syncthreads();
     flush_hist(s_hist, hist, kBins);
-    flush_hist(s_hist + kBins, hist_fine, kFineBins);
     long long tot;
     block_exclusive_sum(capsum, &tot, s_warp);
-    if (threadIdx.x == 0 && tot) atomicAdd(&hdr->sum_cap, (unsigned long long)tot);
-    if (last_block(&hdr->ticket[0])) {
-        const unsigned long long sum_cap = *(volatile unsigned long long *)&hdr->sum_cap;
-        // the 13-bit counts of the window bins are the sums of their fine bins
-        for (int wb = 0; wb < kWinBins; ++wb) {
-            long long part = 0;
-            for (int f = threadIdx.x; f < kFinePerBin; f += kSelThreads) part += (long long)__ldcg(hist_fine + wb * kFinePerBin + f);
-            long long sum;
-            block_exclusive_sum(part, &sum, s_warp);
-            if (threadIdx.x == 0) hist[win_lo + wb] = (unsigned long long)sum;
+    if (threadIdx.x == 0 && tot) atomicAdd(&hdr->sample_cap, (unsigned long long)tot);
+    if (last_block(&hdr->ticket[15])) place_window(hdr, hist, B, n_sample, N, s_warp);
+}
+
+// The fused full pass: builds the gains matrix (a warp per row, as hora_gains does) and does level 0's
+// counting on the way.  Rows are trusted to be sorted (they were just computed), so only the inputs are
+// validated.
+template <int E, bool VEC2>
+__global__ void __launch_bounds__(kSelThreads, 2)
+gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
+                   const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
+                   int64_t N, int32_t ld, double *__restrict__ gains, int64_t B, AllocHeader *hdr,
+                   unsigned long long *hist, unsigned long long *hist_fine, uint16_t *__restrict__ sketch,
+                   int32_t sk_ld) {
+    constexpr int P = E / 2;
+    constexpr bool kStaged = VEC2 && (P > 1);
+    extern __shared__ unsigned int s_hist[];               // kBins + kFineBins words (dynamic: 40 KiB)
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    __shared__ double2 s_stage[kStaged ? (kSelThreads / kWarp) * kWarp * P : 1];
+    for (int b = threadIdx.x; b < kBins + kFineBins; b += kSelThreads) s_hist[b] = 0;
+    __syncthreads();
+    const int lane = lane_id(), warp = threadIdx.x >> 5;
+    double2 *slab = s_stage + (kStaged ? warp * kWarp * P : 0);
+    double2 *wr = slab + lane * P;
+    const double2 *rd = slab + (lane ^ ((lane >> 3) & (P - 1)));
+    Level0Tap<E> tap;
+    tap.s_hist = s_hist;
+    tap.win_lo = hdr->win_lo;
+    const int64_t warp0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + warp;
+    const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
+    long long capsum = 0;
+    bool bad = false;
+    Posterior nxt;
+    nxt.ok = true; nxt.cap = 0; nxt.a = nxt.b = 1.0;
+    if (warp0 < N) nxt = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, warp0);
+    for (int64_t row = warp0; row < N; row += stride) {
+        const Posterior p = nxt;
+        if (row + stride < N) nxt = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row + stride);
+        bad |= !p.ok;
+        if (lane == 0) capsum += p.cap;
+        const double a = p.ok ? p.a : 1.0, b = p.ok ? p.b : 1.0;
+        double *out = gains + row * (int64_t)ld;
+        tap.sk_row = sketch + row * (int64_t)sk_ld;
+        double carry = 1.0;
+        for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E) {
+            if (k0 + kWarp * E <= p.cap)
+                gains_chunk<E, VEC2, true>(a, b, a + b, p.cap, ld, k0, lane, carry, out, wr, rd, tap);
+            else
+                gains_chunk<E, VEC2, false>(a, b, a + b, p.cap, ld, k0, lane, carry, out, wr, rd, tap);
         }
-        if (threadIdx.x == 0) {
-            if ((unsigned long long)B > sum_cap) raise_status(&hdr->status, HORA_ERR_INFEASIBLE);
-            hdr->need = B;
-        }
-        __threadfence();
-        __syncthreads();
-        find_digit(hdr, hist, kBins, kDigitBits, 51, 0, false, s_warp);
-        const int d0 = hdr->sel_digit[0];
-        const unsigned w = (unsigned)(d0 - win_lo);
-        if (hdr->resolved == kDigitBits && w < (unsigned)kWinBins)        // inside the window: 10 more bits for free
-            find_digit(hdr, hist_fine + w * kFinePerBin, kFinePerBin, kFineBits, 51 - kFineBits, 0, true, s_warp);
     }
+    level0_finish(hdr, hist, hist_fine, s_hist, tap.win_lo, capsum, bad, B, s_warp);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -915,6 +1068,26 @@ static void launch_level0(bool vec2, int grid, cudaStream_t s, const int32_t *ca
                                                              w.hist_fine, w.sketch, w.sk_ld);
 }
 
+constexpr size_t kFusedSmem = sizeof(unsigned int) * (kBins + kFineBins);
+
+template <int E>
+static cudaError_t launch_fused(bool vec2, bool estimate, int grid_est, int64_t every, int grid, cudaStream_t s,
+                                const double *alpha, const double *beta, double alpha0, double beta0, const int32_t *c,
+                                int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N, int32_t ld, int64_t B,
+                                const Workspace &w) {
+    if (estimate)
+        select_estimate_fused<E><<<grid_est, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N,
+                                                                  ld, every, B, w.hdr, w.hist_est);
+    auto go = [&](auto kernel) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmem);
+        if (e != cudaSuccess) return e;
+        kernel<<<grid, kSelThreads, kFusedSmem, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, w.gains,
+                                                     B, w.hdr, w.hist_coarse, w.hist_fine, w.sketch, w.sk_ld);
+        return cudaGetLastError();
+    };
+    return vec2 ? go(gains_level0_fused<E, true>) : go(gains_level0_fused<E, false>);
+}
+
 }  // namespace hora
 
 extern "C" void hora_allocate_profile_events(void *start_event, void *stop_event) {
@@ -960,31 +1133,37 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         const size_t tb = reinterpret_cast<char *>(w.rowslot) - reinterpret_cast<char *>(w.tkeys);
         if (cudaMemsetAsync(w.tkeys, 0, tb, s) != cudaSuccess) return HORA_ERR_CUDA;
     }
-    if (gains == nullptr) {
-        const hora_status_t st = launch_gains(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, w.gains,
-                                              &w.hdr->status, s);
-        if (st != HORA_OK) return st;
-        gains = w.gains;
-    }
+    const bool fused = gains == nullptr;                  // no matrix given: build it and count its keys in one pass
+    if (fused) gains = w.gains;
     const bool vec2 = (ld % 2 == 0) && ((reinterpret_cast<uintptr_t>(gains) & 15u) == 0);
     const int rows_per_cta = kSelThreads / kWarp;
-    if (B > 0) {
-        const int64_t every = (N + kSampleRows - 1) / kSampleRows;
-        const int64_t n_sample = (N + every - 1) / every;
-        select_estimate<<<clamp_grid((n_sample + rows_per_cta - 1) / rows_per_cta, 4), kSelThreads, 0, s>>>(
-            cap, cap_scalar, N, ld, every, gains, B, w.hdr, w.hist_est);
-    }
+    const int64_t every = (N + kSampleRows - 1) / kSampleRows;
+    const int64_t n_sample = (N + every - 1) / every;
+    const int grid_est = clamp_grid((n_sample + rows_per_cta - 1) / rows_per_cta, 4);
+    if (B > 0 && !fused)
+        select_estimate<<<grid_est, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, every, gains, B, w.hdr, w.hist_est);
     const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 4);
     const int grid1 = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     const cudaEvent_t prof_start = g_prof_start.load(std::memory_order_relaxed);
     const cudaEvent_t prof_stop = g_prof_stop.load(std::memory_order_relaxed);
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_start, s);
-    if (ld > 128)
+    if (fused) {
+        const int gridf = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 2);
+        cudaError_t e;
+        if (ld > 128)
+            e = launch_fused<8>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, w);
+        else if (ld > 64)
+            e = launch_fused<4>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, w);
+        else
+            e = launch_fused<2>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, w);
+        if (e != cudaSuccess) return HORA_ERR_CUDA;
+    } else if (ld > 128) {
         launch_level0<8>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
-    else if (ld > 64)
+    } else if (ld > 64) {
         launch_level0<4>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
-    else
+    } else {
         launch_level0<2>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
+    }
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_stop, s);
     const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     if (B > 0) {

@@ -7,11 +7,20 @@
 
 namespace hora {
 
+// A "tap" sees every pair of entries a lane produces, while they are still in registers, and is told
+// when the lane's part of the chunk is complete.  NoTap does nothing and costs nothing.
+struct NoTap {
+    __device__ __forceinline__ void pair(int, double, double) {}
+    __device__ __forceinline__ void finish(int32_t, int32_t, int32_t, int32_t) {}
+};
+
 // One chunk of 32*E entries of one row, starting at column k0.  FULL: the chunk lies entirely below the
-// row's cap and inside the row, so no entry needs masking.
-template <int E, bool VEC2, bool FULL>
+// row's cap and inside the row, so no entry needs masking.  `out` may be null when only the tap wants the
+// values (then nothing is stored).
+template <int E, bool VEC2, bool FULL, typename Tap = NoTap>
 __device__ __forceinline__ void gains_chunk(double a, double b, double ab, int32_t capi, int32_t ld, int32_t k0,
-                                            int lane, double &carry, double *__restrict__ out, double2 *wr, const double2 *rd) {
+                                            int lane, double &carry, double *__restrict__ out, double2 *wr,
+                                            const double2 *rd, Tap &&tap = Tap()) {
     constexpr int P = E / 2;                              // 16-byte chunks per lane
     constexpr bool kStaged = VEC2 && (P > 1);
     const int32_t k = k0 + lane * E;
@@ -47,15 +56,17 @@ __device__ __forceinline__ void gains_chunk(double a, double b, double ab, int32
             if (k + m >= capi) g0 = 0.0;
             if (k + m + 1 >= capi) g1 = 0.0;
         }
+        tap.pair(m, g0, g1);
         if (kStaged) {
             wr[(m >> 1) ^ ((lane >> (P == 4 ? 1 : 2)) & (P - 1))] = make_double2(g0, g1);   // (lane*P + p) >> 3
         } else if (VEC2) {
             if (FULL || k + m < ld) *reinterpret_cast<double2 *>(out + k + m) = make_double2(g0, g1);
-        } else {
+        } else if (out != nullptr) {
             if (FULL || k + m < ld) out[k + m] = g0;
             if (FULL || k + m + 1 < ld) out[k + m + 1] = g1;
         }
     }
+    tap.finish(k0, k, capi, ld);
     if (kStaged) {
         __syncwarp();
 #pragma unroll

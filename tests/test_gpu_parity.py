@@ -105,7 +105,8 @@ def test_allocation_matches_oracle(name, N):
     run_and_compare(wl.make(name, N))
 
 
-@pytest.mark.parametrize("name,N", [("cfg1", None), ("cfg2", 2048), ("cfg5", 5000)])
+@pytest.mark.parametrize("name,N", [("cfg1", None), ("cfg2", 2048), ("cfg5", 5000), ("cfg3", None), ("cfg4", 30000),
+                                    ("cfg5", 1 << 17)])
 def test_allocation_without_materialised_gains(name, N):
     run_and_compare(wl.make(name, N), materialise=False)
 
