@@ -490,6 +490,7 @@ struct CoarseTap {
         for (int m = 0; m < E; ++m)
             if (m < valid) atomicAdd(&s_hist[(unsigned)(key[m] >> 51)], 1u);
     }
+    __device__ __forceinline__ void begin_row(int64_t, int32_t) {}
 };
 
 // the level-0 bookkeeping: window/coarse histogram and the sketch
@@ -497,8 +498,15 @@ template <int E>
 struct Level0Tap {
     unsigned long long key[E];
     unsigned int *s_hist;
+    uint16_t *sketch;
     uint16_t *sk_row;              // sketch row of the prompt being built
+    int32_t sk_ld;
     int win_lo;
+    long long capsum;              // lane 0 of every warp: caps of the rows it built
+    __device__ __forceinline__ void begin_row(int64_t row, int32_t capi) {
+        sk_row = sketch + row * (int64_t)sk_ld;
+        if ((threadIdx.x & 31) == 0) capsum += capi;
+    }
     __device__ __forceinline__ void pair(int m, double g0, double g1) {
         key[m] = (unsigned long long)__double_as_longlong(g0);
         key[m + 1] = (unsigned long long)__double_as_longlong(g1);
@@ -557,9 +565,9 @@ select_estimate_fused(const double *__restrict__ alpha, const double *__restrict
     if (last_block(&hdr->ticket[15])) place_window(hdr, hist, B, n_sample, N, s_warp);
 }
 
-// The fused full pass: builds the gains matrix (a warp per row, as hora_gains does) and does level 0's
-// counting on the way.  Rows are trusted to be sorted (they were just computed), so only the inputs are
-// validated.
+// The fused full pass: the row loop of hora_gains (same staging, same arithmetic, same stores) with level 0's
+// counting tapped in.  Rows are trusted to be sorted (they were just computed), so only the inputs are
+// validated (the row loop raises the status for invalid priors, counts or caps).
 template <int E, bool VEC2>
 __global__ void __launch_bounds__(kSelThreads, 2)
 gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
@@ -567,44 +575,19 @@ gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ 
                    int64_t N, int32_t ld, double *__restrict__ gains, int64_t B, AllocHeader *hdr,
                    unsigned long long *hist, unsigned long long *hist_fine, uint16_t *__restrict__ sketch,
                    int32_t sk_ld) {
-    constexpr int P = E / 2;
-    constexpr bool kStaged = VEC2 && (P > 1);
     extern __shared__ unsigned int s_hist[];               // kBins + kFineBins words (dynamic: 40 KiB)
     __shared__ long long s_warp[kSelThreads / kWarp];
-    __shared__ double2 s_stage[kStaged ? (kSelThreads / kWarp) * kWarp * P : 1];
     for (int b = threadIdx.x; b < kBins + kFineBins; b += kSelThreads) s_hist[b] = 0;
     __syncthreads();
-    const int lane = lane_id(), warp = threadIdx.x >> 5;
-    double2 *slab = s_stage + (kStaged ? warp * kWarp * P : 0);
-    double2 *wr = slab + lane * P;
-    const double2 *rd = slab + (lane ^ ((lane >> 3) & (P - 1)));
     Level0Tap<E> tap;
     tap.s_hist = s_hist;
+    tap.sketch = sketch;
+    tap.sk_row = sketch;
+    tap.sk_ld = sk_ld;
     tap.win_lo = hdr->win_lo;
-    const int64_t warp0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + warp;
-    const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
-    long long capsum = 0;
-    bool bad = false;
-    Posterior nxt;
-    nxt.ok = true; nxt.cap = 0; nxt.a = nxt.b = 1.0;
-    if (warp0 < N) nxt = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, warp0);
-    for (int64_t row = warp0; row < N; row += stride) {
-        const Posterior p = nxt;
-        if (row + stride < N) nxt = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row + stride);
-        bad |= !p.ok;
-        if (lane == 0) capsum += p.cap;
-        const double a = p.ok ? p.a : 1.0, b = p.ok ? p.b : 1.0;
-        double *out = gains + row * (int64_t)ld;
-        tap.sk_row = sketch + row * (int64_t)sk_ld;
-        double carry = 1.0;
-        for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E) {
-            if (k0 + kWarp * E <= p.cap)
-                gains_chunk<E, VEC2, true>(a, b, a + b, p.cap, ld, k0, lane, carry, out, wr, rd, tap);
-            else
-                gains_chunk<E, VEC2, false>(a, b, a + b, p.cap, ld, k0, lane, carry, out, wr, rd, tap);
-        }
-    }
-    level0_finish(hdr, hist, hist_fine, s_hist, tap.win_lo, capsum, bad, B, s_warp);
+    tap.capsum = 0;
+    gains_rows_cta<E, VEC2>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, &hdr->status, tap);
+    level0_finish(hdr, hist, hist_fine, s_hist, tap.win_lo, tap.capsum, false, B, s_warp);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -1148,7 +1131,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     const cudaEvent_t prof_stop = g_prof_stop.load(std::memory_order_relaxed);
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_start, s);
     if (fused) {
-        const int gridf = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 2);
+        const int gridf = clamp_grid((N + kCtaRows - 1) / kCtaRows, 2);
         cudaError_t e;
         if (ld > 128)
             e = launch_fused<8>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, w);
