@@ -569,7 +569,7 @@ select_estimate_fused(const double *__restrict__ alpha, const double *__restrict
 // counting tapped in.  Rows are trusted to be sorted (they were just computed), so only the inputs are
 // validated (the row loop raises the status for invalid priors, counts or caps).
 template <int E, bool VEC2>
-__global__ void __launch_bounds__(kSelThreads, 2)
+__global__ void __launch_bounds__(kSelThreads, 3)
 gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
                    const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
                    int64_t N, int32_t ld, double *__restrict__ gains, int64_t B, AllocHeader *hdr,
@@ -1131,7 +1131,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     const cudaEvent_t prof_stop = g_prof_stop.load(std::memory_order_relaxed);
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_start, s);
     if (fused) {
-        const int gridf = clamp_grid((N + kCtaRows - 1) / kCtaRows, 2);
+        const int gridf = clamp_grid((N + kCtaRows - 1) / kCtaRows, 3);
         cudaError_t e;
         if (ld > 128)
             e = launch_fused<8>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, w);
