@@ -59,6 +59,8 @@ enum {
 
 enum { HORA_ADV_GRPO = 0, HORA_ADV_RLOO = 1 };
 
+enum { HORA_WEIGHT_PER_TOKEN = 0, HORA_WEIGHT_CONST_LENGTH = 1 };
+
 /* Summary of one allocation; lives in DEVICE memory (64 bytes, 8-byte aligned). */
 typedef struct hora_alloc_info {
     int32_t status;        /* hora_status_t of the data-dependent checks */
@@ -213,6 +215,27 @@ hora_status_t hora_allocate_batched(const double *alpha, const double *beta, dou
 hora_status_t hora_group_advantage(const float *rewards, const int64_t *group_offsets, int64_t N,
                                    int32_t mode, float eps, int32_t ddof, float *adv,
                                    int32_t *status_dev, void *stream);
+
+/*
+ * hora_rollout_weights — loss weight of every rollout under variable-size groups (Sec. 3.2, paragraph "Training
+ * objective with variable-size groups": in Eq. grpo-objective 1/G becomes 1/G_i, so every prompt weighs the
+ * same however many rollouts it was given).
+ *
+ *   HORA_WEIGHT_PER_TOKEN     weights[r] = 1 / (G_g * len_r)          the 1/G_i * 1/|o| of Eq. grpo-objective;
+ *                             0 for a zero-length rollout.  The tokens of one prompt then sum to weight 1.
+ *   HORA_WEIGHT_CONST_LENGTH  weights[r] = 1 / (G_g * length_const)   a length-free normalisation (the paper says
+ *                             its runs use one from Dr. GRPO but prints no formula; the constant is the caller's,
+ *                             e.g. the maximum response length)
+ * with g the group of rollout r, G_g = group_offsets[g+1] - group_offsets[g], len_r = token_offsets[r+1] -
+ * token_offsets[r].  One fp64 division, rounded to fp32.  hora_token_broadcast turns the result into per-token
+ * weights in the packed token layout.
+ *
+ *   group_offsets [N+1] int64, token_offsets [R+1] int64 with R = group_offsets[N] (may be NULL in the
+ *   CONST_LENGTH mode), weights [R] fp32 out, status_dev optional (INVALID_VALUE on decreasing offsets).
+ */
+hora_status_t hora_rollout_weights(const int64_t *group_offsets, int64_t N, const int64_t *token_offsets,
+                                   int32_t mode, float length_const, float *weights, int32_t *status_dev,
+                                   void *stream);
 
 /*
  * hora_token_broadcast — per-token advantages (Eq. grpo-objective: the advantage of a rollout does not

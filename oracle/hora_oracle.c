@@ -317,3 +317,24 @@ int oracle_token_broadcast(const float *adv, const int64_t *tok_off, int64_t R, 
     }
     return ORACLE_OK;
 }
+
+/* ----------------------- loss weights under variable-size groups (Sec. 3.2, last paragraph) */
+/* mode 0: 1/(G_g * len_r), the 1/G_i and 1/|o| of Eq. grpo-objective; mode 1: 1/(G_g * length_const) */
+int oracle_rollout_weights(const int64_t *goff, int64_t N, const int64_t *toff, int32_t mode, double length_const,
+                           float *weights)
+{
+    if (mode != 0 && mode != 1) return ORACLE_BAD_ARG;
+    for (int64_t g = 0; g < N; ++g) {
+        if (goff[g + 1] < goff[g]) return ORACLE_BAD_ARG;
+        double G = (double)(goff[g + 1] - goff[g]);
+        for (int64_t r = goff[g]; r < goff[g + 1]; ++r) {
+            double denom = G * length_const;
+            if (mode == 0) {
+                if (toff[r + 1] < toff[r]) return ORACLE_BAD_ARG;
+                denom = G * (double)(toff[r + 1] - toff[r]);
+            }
+            weights[r] = denom > 0.0 ? (float)(1.0 / denom) : 0.0f;
+        }
+    }
+    return ORACLE_OK;
+}

@@ -43,6 +43,7 @@ def lib():
                                           p, p, p, p, p]
         L.oracle_group_advantage.argtypes = [p, p, C.c_int64, C.c_int32, C.c_double, C.c_int32, p]
         L.oracle_token_broadcast.argtypes = [p, p, C.c_int64, p]
+        L.oracle_rollout_weights.argtypes = [p, C.c_int64, p, C.c_int32, C.c_double, p]
         _lib = L
     return _lib
 
@@ -130,4 +131,13 @@ def token_broadcast(adv, tok_off) -> np.ndarray:
     tok_off = np.ascontiguousarray(tok_off, dtype=np.int64)
     out = np.empty(int(tok_off[-1]), dtype=np.float32)
     _check(lib().oracle_token_broadcast(_ptr(adv), _ptr(tok_off), adv.shape[0], _ptr(out)))
+    return out
+
+
+def rollout_weights(goff, toff, mode: int, length_const: float = 1.0) -> np.ndarray:
+    """Loss weight per rollout: 1/(G_g len_r) (mode 0) or 1/(G_g length_const) (mode 1)."""
+    goff = np.ascontiguousarray(goff, dtype=np.int64)
+    toff = None if toff is None else np.ascontiguousarray(toff, dtype=np.int64)
+    out = np.zeros(int(goff[-1]), dtype=np.float32)
+    _check(lib().oracle_rollout_weights(_ptr(goff), goff.shape[0] - 1, _ptr(toff), mode, float(length_const), _ptr(out)))
     return out

@@ -20,11 +20,12 @@ OK, ERR_INVALID_ARG, ERR_INVALID_VALUE, ERR_INFEASIBLE, ERR_NOT_INTEGER, ERR_EXA
 FLAG_EXACT_INT = 1
 FLAG_SKIP_OBJECTIVE = 2
 ADV_GRPO, ADV_RLOO = 0, 1
+WEIGHT_PER_TOKEN, WEIGHT_CONST_LENGTH = 0, 1
 
 EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora_group_advantage",
            "hora_token_broadcast", "hora_status_string", "hora_version", "hora_launch_count",
            "hora_allocate_static", "hora_allocate_static_capacity", "hora_allocate_profile_events",
-           "hora_allocate_batched", "hora_allocate_batched_workspace_bytes")
+           "hora_allocate_batched", "hora_allocate_batched_workspace_bytes", "hora_rollout_weights")
 
 
 class HoraError(RuntimeError):
@@ -70,6 +71,8 @@ def load() -> C.CDLL:
     L.hora_allocate_profile_events.restype = None
     L.hora_group_advantage.argtypes = [p, p, i64, i32, C.c_float, i32, p, p, p]
     L.hora_group_advantage.restype = C.c_int
+    L.hora_rollout_weights.argtypes = [p, i64, p, i32, C.c_float, p, p, p]
+    L.hora_rollout_weights.restype = C.c_int
     L.hora_token_broadcast.argtypes = [p, p, i64, i64, p, p]
     L.hora_token_broadcast.restype = C.c_int
     L.hora_status_string.argtypes = [C.c_int]
@@ -203,6 +206,14 @@ def hora_group_advantage(rewards, group_offsets, N, mode, eps, ddof, adv, status
                                      _ptr(adv, torch.float32, "adv"), _ptr(status_dev, torch.int32, "status_dev"),
                                      _stream())
     _check(rc, "hora_group_advantage")
+
+
+def hora_rollout_weights(group_offsets, N, token_offsets, mode, length_const, weights, status_dev=None):
+    rc = load().hora_rollout_weights(_ptr(group_offsets, torch.int64, "group_offsets"), N,
+                                     _ptr(token_offsets, torch.int64, "token_offsets"), mode, length_const,
+                                     _ptr(weights, torch.float32, "weights"), _ptr(status_dev, torch.int32, "status_dev"),
+                                     _stream())
+    _check(rc, "hora_rollout_weights")
 
 
 def hora_token_broadcast(adv, token_offsets, R, T, token_adv):

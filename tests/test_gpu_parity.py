@@ -371,3 +371,35 @@ def test_token_broadcast_on_cfg3_layout_scaled():
     tok = w.token_offsets(len(r))
     got = gu.gpu_broadcast(adv, tok)
     np.testing.assert_array_equal(got.view(np.uint32), orc.token_broadcast(adv, tok).view(np.uint32))
+
+
+# ---------------------------------------------------------------------------------------- weights
+@pytest.mark.parametrize("mode", [0, 1])
+def test_rollout_weights_bitwise(mode):
+    from paper_2605_07114_b200 import hora
+    rng = np.random.default_rng(21 + mode)
+    sizes = rng.choice([0, 1, 2, 8, 9, 31, 32, 33, 100, 264, 1000], 3000)
+    goff = np.zeros(len(sizes) + 1, np.int64)
+    np.cumsum(sizes, out=goff[1:])
+    R = int(goff[-1])
+    lens = rng.integers(0, 2049, R)
+    toff = np.zeros(R + 1, np.int64)
+    np.cumsum(lens, out=toff[1:])
+    w = torch.full((R,), -1.0, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    hora.hora_rollout_weights(torch.from_numpy(goff).cuda(), len(sizes), torch.from_numpy(toff).cuda(), mode, 2048.0, w,
+                              status)
+    torch.cuda.synchronize()
+    exp = orc.rollout_weights(goff, toff, mode, 2048.0)
+    assert int(status.item()) == 0
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), exp.view(np.uint32))
+    # through the token broadcast: per-token weights of one prompt sum to 1 in the per-token mode
+    if mode == 0:
+        T = int(toff[-1])
+        tw = torch.empty(T, dtype=torch.float32, device="cuda")
+        hora.hora_token_broadcast(w, torch.from_numpy(toff).cuda(), R, T, tw)
+        per_rollout = np.add.reduceat(tw.cpu().numpy().astype(np.float64), toff[:-1][lens > 0])
+        g_of_r = np.repeat(np.arange(len(sizes)), sizes)[lens > 0]
+        per_prompt = np.bincount(g_of_r, weights=per_rollout, minlength=len(sizes))
+        full = np.array([sizes[g] > 0 and (lens[goff[g]:goff[g + 1]] > 0).all() for g in range(len(sizes))])
+        np.testing.assert_allclose(per_prompt[full], 1.0, rtol=1e-5)

@@ -388,6 +388,32 @@ def test_token_broadcast_is_repeat():
     np.testing.assert_array_equal(out.view(np.uint32), np.repeat(adv, lens).view(np.uint32))
 
 
+def test_rollout_weights_give_every_prompt_the_same_weight():
+    """Sec. 3.2: with 1/G_i in place of 1/G each prompt has equal weight however many rollouts it got.  Summed
+    over the tokens of a prompt, 1/(G_i |o|) gives exactly 1; the length-free form gives G_i/(G_i L) = 1/L per
+    prompt when summed over rollouts."""
+    rng = np.random.default_rng(12)
+    sizes = rng.integers(1, 40, 200)
+    goff = np.zeros(201, np.int64)
+    np.cumsum(sizes, out=goff[1:])
+    R = int(goff[-1])
+    lens = rng.integers(1, 500, R)
+    toff = np.zeros(R + 1, np.int64)
+    np.cumsum(lens, out=toff[1:])
+    w = orc.rollout_weights(goff, toff, 0).astype(np.float64)
+    per_prompt = np.add.reduceat(w * lens, goff[:-1])
+    np.testing.assert_allclose(per_prompt, 1.0, rtol=1e-6)
+    w1 = orc.rollout_weights(goff, None, 1, 2048.0).astype(np.float64)
+    np.testing.assert_allclose(np.add.reduceat(w1, goff[:-1]), 1.0 / 2048.0, rtol=1e-6)
+    # direct form on one group
+    np.testing.assert_allclose(w[:sizes[0]], 1.0 / (sizes[0] * lens[:sizes[0]]), rtol=1e-7)
+    lens0 = lens.copy()
+    lens0[3] = 0
+    toff0 = np.zeros(R + 1, np.int64)
+    np.cumsum(lens0, out=toff0[1:])
+    assert orc.rollout_weights(goff, toff0, 0)[3] == 0.0
+
+
 # ------------------------------------------------------------------ planted mistakes are caught
 def _mutant(kind):
     def marg(a, b, D):
