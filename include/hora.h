@@ -217,6 +217,40 @@ hora_status_t hora_group_advantage(const float *rewards, const int64_t *group_of
                                    int32_t *status_dev, void *stream);
 
 /*
+ * hora_learned_prior — prior parameters from a predictor's outputs (appendix "Prior-design predictor details",
+ * Eq. posterior-learned): alpha_i = s_i p_hat_i, beta_i = s_i (1 - p_hat_i); fed to hora_gains / hora_allocate,
+ * which add the Phase-A counts, they give the posterior of Eq. posterior-learned.  s_i = clamp(softplus(s_raw_i),
+ * 0.25, 16) when s_raw is given (the dual-head variants), else the fixed s_fixed (2 in the paper's single-head
+ * variants; s = 2 with p_hat = 1/2 is the uniform prior).
+ *   p_hat [N] fp64 in (0,1); s_raw [N] fp64 raw head output or NULL; alpha, beta [N] fp64 out;
+ *   status_dev optional: INVALID_VALUE if some p_hat is outside (0,1) (that prompt gets alpha = beta = 0).
+ *
+ * hora_beta_binomial_nll — the per-prompt training loss of those predictors (same appendix):
+ *   nll_i = -log( B(c_i + s_i p_hat_i, G0 - c_i + s_i (1 - p_hat_i)) / B(s_i p_hat_i, s_i (1 - p_hat_i)) )
+ * with s_i as above; log-Beta through lgamma in fp64.  c [N] int32 in [0, G0]; nll [N] fp64 out.
+ */
+hora_status_t hora_learned_prior(const double *p_hat, const double *s_raw, double s_fixed, int64_t N,
+                                 double *alpha, double *beta, int32_t *status_dev, void *stream);
+
+hora_status_t hora_beta_binomial_nll(const double *p_hat, const double *s_raw, double s_fixed, const int32_t *c,
+                                     int32_t G0, int64_t N, double *nll, int32_t *status_dev, void *stream);
+
+/*
+ * hora_pass_at_k — the unbiased Pass@K estimator (Eq. pass-k) averaged over prompts, for a grid of K values:
+ *   pass_at_k[j] = mean over the Q prompts of  1 - C(n - c_q, K_j) / C(n, K_j),
+ * c_q = correct samples among the n_samples drawn for prompt q.  Counts outside [0, n_samples] raise
+ * INVALID_VALUE in status_dev and are left out of the sums; a K_j outside [0, n_samples] raises
+ * INVALID_VALUE too and its output is 0 (C(n, K) is zero there, the estimator undefined).
+ *   c [Q] int32 device; K_dev [n_K] int32 device; pass_at_k [n_K] fp64 device out;
+ *   workspace: hora_pass_at_k_workspace_bytes(n_samples) bytes of device scratch, 8-byte aligned.
+ */
+size_t hora_pass_at_k_workspace_bytes(int32_t n_samples);
+
+hora_status_t hora_pass_at_k(const int32_t *c, int64_t Q, int32_t n_samples, const int32_t *K_dev, int32_t n_K,
+                             double *pass_at_k, int32_t *status_dev, void *workspace, size_t workspace_bytes,
+                             void *stream);
+
+/*
  * hora_rollout_weights — loss weight of every rollout under variable-size groups (Sec. 3.2, paragraph "Training
  * objective with variable-size groups": in Eq. grpo-objective 1/G becomes 1/G_i, so every prompt weighs the
  * same however many rollouts it was given).

@@ -25,7 +25,8 @@ WEIGHT_PER_TOKEN, WEIGHT_CONST_LENGTH = 0, 1
 EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora_group_advantage",
            "hora_token_broadcast", "hora_status_string", "hora_version", "hora_launch_count",
            "hora_allocate_static", "hora_allocate_static_capacity", "hora_allocate_profile_events",
-           "hora_allocate_batched", "hora_allocate_batched_workspace_bytes", "hora_rollout_weights")
+           "hora_allocate_batched", "hora_allocate_batched_workspace_bytes", "hora_rollout_weights",
+           "hora_learned_prior", "hora_beta_binomial_nll", "hora_pass_at_k", "hora_pass_at_k_workspace_bytes")
 
 
 class HoraError(RuntimeError):
@@ -71,6 +72,14 @@ def load() -> C.CDLL:
     L.hora_allocate_profile_events.restype = None
     L.hora_group_advantage.argtypes = [p, p, i64, i32, C.c_float, i32, p, p, p]
     L.hora_group_advantage.restype = C.c_int
+    L.hora_pass_at_k_workspace_bytes.argtypes = [i32]
+    L.hora_pass_at_k_workspace_bytes.restype = C.c_size_t
+    L.hora_pass_at_k.argtypes = [p, i64, i32, p, i32, p, p, p, C.c_size_t, p]
+    L.hora_pass_at_k.restype = C.c_int
+    L.hora_learned_prior.argtypes = [p, p, f64, i64, p, p, p, p]
+    L.hora_learned_prior.restype = C.c_int
+    L.hora_beta_binomial_nll.argtypes = [p, p, f64, p, i32, i64, p, p, p]
+    L.hora_beta_binomial_nll.restype = C.c_int
     L.hora_rollout_weights.argtypes = [p, i64, p, i32, C.c_float, p, p, p]
     L.hora_rollout_weights.restype = C.c_int
     L.hora_token_broadcast.argtypes = [p, p, i64, i64, p, p]
@@ -208,12 +217,39 @@ def hora_group_advantage(rewards, group_offsets, N, mode, eps, ddof, adv, status
     _check(rc, "hora_group_advantage")
 
 
+def hora_pass_at_k_workspace_bytes(n_samples) -> int:
+    return int(load().hora_pass_at_k_workspace_bytes(n_samples))
+
+
+def hora_pass_at_k(c, Q, n_samples, K_dev, n_K, pass_at_k, status_dev, workspace):
+    rc = load().hora_pass_at_k(_ptr(c, torch.int32, "c"), Q, n_samples, _ptr(K_dev, torch.int32, "K_dev"), n_K,
+                               _ptr(pass_at_k, torch.float64, "pass_at_k"), _ptr(status_dev, torch.int32, "status_dev"),
+                               _ptr(workspace, torch.uint8, "workspace"), 0 if workspace is None else workspace.numel(),
+                               _stream())
+    _check(rc, "hora_pass_at_k")
+
+
+def hora_learned_prior(p_hat, s_raw, s_fixed, N, alpha, beta, status_dev=None):
+    rc = load().hora_learned_prior(_ptr(p_hat, torch.float64, "p_hat"), _ptr(s_raw, torch.float64, "s_raw"), s_fixed, N,
+                                   _ptr(alpha, torch.float64, "alpha"), _ptr(beta, torch.float64, "beta"),
+                                   _ptr(status_dev, torch.int32, "status_dev"), _stream())
+    _check(rc, "hora_learned_prior")
+
+
+def hora_beta_binomial_nll(p_hat, s_raw, s_fixed, c, G0, N, nll, status_dev=None):
+    rc = load().hora_beta_binomial_nll(_ptr(p_hat, torch.float64, "p_hat"), _ptr(s_raw, torch.float64, "s_raw"), s_fixed,
+                                       _ptr(c, torch.int32, "c"), G0, N, _ptr(nll, torch.float64, "nll"),
+                                       _ptr(status_dev, torch.int32, "status_dev"), _stream())
+    _check(rc, "hora_beta_binomial_nll")
+
+
 def hora_rollout_weights(group_offsets, N, token_offsets, mode, length_const, weights, status_dev=None):
     rc = load().hora_rollout_weights(_ptr(group_offsets, torch.int64, "group_offsets"), N,
                                      _ptr(token_offsets, torch.int64, "token_offsets"), mode, length_const,
                                      _ptr(weights, torch.float32, "weights"), _ptr(status_dev, torch.int32, "status_dev"),
                                      _stream())
-    _check(rc, "hora_rollout_weights")
+    _check(rc, "hora_rollout_weights",
+           "hora_learned_prior", "hora_beta_binomial_nll", "hora_pass_at_k", "hora_pass_at_k_workspace_bytes")
 
 
 def hora_token_broadcast(adv, token_offsets, R, T, token_adv):

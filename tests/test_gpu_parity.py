@@ -403,3 +403,81 @@ def test_rollout_weights_bitwise(mode):
         per_prompt = np.bincount(g_of_r, weights=per_rollout, minlength=len(sizes))
         full = np.array([sizes[g] > 0 and (lens[goff[g]:goff[g + 1]] > 0).all() for g in range(len(sizes))])
         np.testing.assert_allclose(per_prompt[full], 1.0, rtol=1e-5)
+
+
+# ------------------------------------------------------------------------------------ learned prior
+def test_learned_prior_and_nll_match_oracle():
+    from oracle import prior
+    from paper_2605_07114_b200 import hora
+    rng = np.random.default_rng(33)
+    N, G0 = 5000, 8
+    p_hat = rng.uniform(0.001, 0.999, N)
+    s_raw = rng.uniform(-6, 20, N)
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    t = lambda x: torch.from_numpy(np.ascontiguousarray(x)).cuda()
+    for raw in (s_raw, None):
+        alpha = torch.empty(N, dtype=torch.float64, device="cuda")
+        beta = torch.empty(N, dtype=torch.float64, device="cuda")
+        nll = torch.empty(N, dtype=torch.float64, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        hora.hora_learned_prior(t(p_hat), None if raw is None else t(raw), 2.0, N, alpha, beta, status)
+        hora.hora_beta_binomial_nll(t(p_hat), None if raw is None else t(raw), 2.0, t(c), G0, N, nll, status)
+        torch.cuda.synchronize()
+        a_o, b_o = prior.learned_prior(p_hat, raw, 2.0)
+        assert int(status.item()) == 0
+        np.testing.assert_allclose(alpha.cpu().numpy(), a_o, rtol=1e-14)
+        np.testing.assert_allclose(beta.cpu().numpy(), b_o, rtol=1e-14)
+        np.testing.assert_allclose(nll.cpu().numpy(), prior.beta_binomial_nll(p_hat, c, G0, raw, 2.0), rtol=1e-11, atol=1e-12)
+    # the priors plug into the allocation: learned prior with s = 2, p_hat = 1/2 equals the uniform prior
+    import gpu_util as gu
+    alpha = torch.empty(64, dtype=torch.float64, device="cuda")
+    beta = torch.empty(64, dtype=torch.float64, device="cuda")
+    hora.hora_learned_prior(torch.full((64,), 0.5, dtype=torch.float64, device="cuda"), None, 2.0, 64, alpha, beta)
+    cc = rng.integers(0, 5, 64).astype(np.int32)
+    cap = np.full(64, 20, np.int32)
+    d1 = gu.gpu_allocate(alpha.cpu().numpy(), beta.cpu().numpy(), 1.0, 1.0, cc, 4, cap, 20, 300, exact=True)[0]
+    d2 = gu.gpu_allocate(None, None, 1.0, 1.0, cc, 4, cap, 20, 300, exact=True)[0]
+    np.testing.assert_array_equal(d1, d2)
+    bad = torch.tensor([0.5, 1.0, 0.2], dtype=torch.float64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    hora.hora_learned_prior(bad, None, 2.0, 3, alpha[:3], beta[:3], status)
+    assert int(status.item()) == 2
+
+
+# ------------------------------------------------------------------------------------ Pass@K estimator
+@pytest.mark.parametrize("Q,n", [(1, 1), (257, 16), (40000, 128), (3000, 1024)])
+def test_pass_at_k_matches_oracle(Q, n):
+    from oracle import passk
+    from paper_2605_07114_b200 import hora
+    rng = np.random.default_rng(Q + n)
+    p = rng.beta(0.5, 1.5, Q)                                   # many hard prompts, a tail of easy ones
+    c = rng.binomial(n, p).astype(np.int32)
+    Ks = sorted({min(k, n) for k in (1, 2, 4, 8, max(n // 2, 1), n)})
+    c_d = torch.from_numpy(c).cuda()
+    K_d = torch.tensor(Ks, dtype=torch.int32, device="cuda")
+    out = torch.full((len(Ks),), -1.0, dtype=torch.float64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(hora.hora_pass_at_k_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    hora.hora_pass_at_k(c_d, Q, n, K_d, len(Ks), out, status, ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    # 1 - prod of up to n ratios, each rounded once: absolute error below n * 2^-52, far inside 1e-12
+    np.testing.assert_allclose(out.cpu().numpy(), passk.pass_at_k(c, n, Ks), rtol=0, atol=1e-12)
+    again = torch.empty_like(out)
+    hora.hora_pass_at_k(c_d, Q, n, K_d, len(Ks), again, status, ws)
+    assert torch.equal(out, again)                              # fixed summation order
+
+
+def test_pass_at_k_rejects_bad_counts_and_k():
+    from paper_2605_07114_b200 import hora
+    n = 8
+    ws = torch.empty(hora.hora_pass_at_k_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    out = torch.empty(2, dtype=torch.float64, device="cuda")
+    for c, Ks in (([1, 9, 2], [1, 2]), ([1, 2, 3], [1, 9])):
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        hora.hora_pass_at_k(torch.tensor(c, dtype=torch.int32, device="cuda"), 3, n,
+                            torch.tensor(Ks, dtype=torch.int32, device="cuda"), 2, out, status, ws)
+        assert int(status.item()) == 2
+    with pytest.raises(hora.HoraError):
+        hora.hora_pass_at_k(torch.zeros(3, dtype=torch.int32, device="cuda"), 3, n,
+                            torch.ones(2, dtype=torch.int32, device="cuda"), 2, out, None, ws[:8])

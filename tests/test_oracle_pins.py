@@ -414,6 +414,36 @@ def test_rollout_weights_give_every_prompt_the_same_weight():
     assert orc.rollout_weights(goff, toff0, 0)[3] == 0.0
 
 
+def test_learned_prior_front_end_pins():
+    from oracle import prior
+    # s = 2, p_hat = 1/2 is the uniform Beta(1,1) prior (stated below Eq. posterior-learned)
+    a, b = prior.learned_prior([0.5], None, 2.0)
+    assert a[0] == 1.0 and b[0] == 1.0
+    # softplus and the clamp to [0.25, 16]
+    a, b = prior.learned_prior([0.25, 0.25, 0.25], [-50.0, 0.0, 50.0])
+    np.testing.assert_allclose(a + b, [0.25, math.log(2.0), 16.0], rtol=1e-15)
+    np.testing.assert_allclose(a / (a + b), 0.25, rtol=1e-15)
+    # one Phase-A draw: the Beta-Binomial probability of a success is the prior mean
+    for p_hat in (0.1, 0.5, 0.83):
+        for s in (0.3, 2.0, 11.0):
+            assert prior.beta_binomial_nll([p_hat], [1], 1, None, s)[0] == pytest.approx(-math.log(p_hat), rel=1e-12)
+            assert prior.beta_binomial_nll([p_hat], [0], 1, None, s)[0] == pytest.approx(-math.log(1 - p_hat), rel=1e-12)
+    # the Beta-Binomial pmf sums to one over c
+    G0 = 8
+    for p_hat, s in ((0.3, 2.0), (0.9, 0.25), (0.5, 16.0)):
+        nll = prior.beta_binomial_nll([p_hat] * (G0 + 1), list(range(G0 + 1)), G0, None, s)
+        total = sum(math.comb(G0, c) * math.exp(-nll[c]) for c in range(G0 + 1))
+        assert total == pytest.approx(1.0, rel=1e-12)
+    # uniform prior: every count is equally likely, pmf = 1/(G0+1)
+    nll = prior.beta_binomial_nll([0.5] * (G0 + 1), list(range(G0 + 1)), G0, None, 2.0)
+    for c in range(G0 + 1):
+        assert math.comb(G0, c) * math.exp(-nll[c]) == pytest.approx(1.0 / (G0 + 1), rel=1e-12)
+    # agreement with a library log-Beta
+    a, b = prior.learned_prior([0.37], None, 5.0)
+    assert prior.beta_binomial_nll([0.37], [3], 8, None, 5.0)[0] == pytest.approx(
+        -(special.betaln(3 + a[0], 5 + b[0]) - special.betaln(a[0], b[0])), rel=1e-12)
+
+
 # ------------------------------------------------------------------ planted mistakes are caught
 def _mutant(kind):
     def marg(a, b, D):
@@ -461,3 +491,28 @@ def test_pins_catch_wrong_tie_break_and_wrong_argmax():
         return d
 
     assert any(literal.objective(ab, greedy_by_mean(ab, cap, B)) < brute_force_best(ab, cap, B) for B in range(13))
+
+
+def test_pass_at_k_estimator_pins():
+    """Eq. pass-k: pinned by special cases, by brute force over K-subsets, and by unbiasedness."""
+    import itertools
+    from oracle import passk
+    n = 7
+    for c in range(n + 1):
+        assert passk.pass_at_k_one(n, c, 1) == Fraction(c, n)            # K = 1: the plain success rate
+        assert passk.pass_at_k_one(n, c, n) == (1 if c > 0 else 0)        # K = n: any correct sample at all
+        assert passk.pass_at_k_one(n, c, 0) == 0
+        for K in range(1, n + 1):
+            # brute force: fraction of K-subsets of the n samples that contain a correct one
+            marks = [1] * c + [0] * (n - c)
+            subsets = list(itertools.combinations(range(n), K))
+            hit = sum(1 for sub in subsets if any(marks[i] for i in sub))
+            assert passk.pass_at_k_one(n, c, K) == Fraction(hit, len(subsets))
+    for K in range(1, n + 1):
+        assert passk.pass_at_k_one(n, 0, K) == 0 and passk.pass_at_k_one(n, n, K) == 1
+    # unbiased: averaged over c ~ Binomial(n, p) it equals 1 - (1-p)^K exactly
+    p = Fraction(3, 10)
+    for K in (1, 2, 5, 7):
+        mean = sum(Fraction(math.comb(n, c)) * p**c * (1 - p)**(n - c) * passk.pass_at_k_one(n, c, K) for c in range(n + 1))
+        assert mean == 1 - (1 - p)**K
+    assert passk.pass_at_k([0, 7, 3], 7, [1, 7]) == [float(Fraction(10, 21)), float(Fraction(2, 3))]
