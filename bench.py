@@ -276,6 +276,36 @@ def run_ours(args):
         torch.cuda.empty_cache()
         al.gains = torch.empty((N, ld), dtype=torch.float64, device=dev)
 
+    # ---- token-level advantages of the broadcast rollouts: two calls against the one fused call ----
+    tok_cmp = None
+    if world == 1:
+        n_bc = int(np.searchsorted(off_h, R, side="left"))          # groups that cover the first R rollouts
+        check = torch.empty_like(token_adv)
+
+        def two_calls():
+            hora.hora_group_advantage(rewards, al.group_offsets, n_bc, w.adv_mode, eps, w.ddof, adv)
+            hora.hora_token_broadcast(adv, tok, R, T, token_adv)
+
+        def one_call():
+            hora.hora_group_advantage_tokens(rewards, al.group_offsets, N, tok, R, T, w.adv_mode, eps, w.ddof, check)
+        ms = []
+        for fn in (two_calls, one_call):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            nt = max(3, min(args.steps, 50))
+            a0.record()
+            for _ in range(nt):
+                fn()
+            a1.record()
+            torch.cuda.synchronize()
+            ms.append(a0.elapsed_time(a1) / nt)
+        if float((check - token_adv).abs().max()) > 1e-5:
+            raise RuntimeError("fused and two-call token advantages differ")
+        tok_cmp = {"rollouts": R, "tokens": T, "ms_two_calls": round(ms[0], 4), "ms_fused": round(ms[1], 4),
+                   "fused_gbs": round(4.0 * T / ms[1] / 1e6, 1)}
+
     # ---- end to end: pinned host inputs in, results out, every step ----
     e2e_steps = max(3, min(args.steps, 20))
     for _ in range(2):
@@ -347,6 +377,7 @@ def run_ours(args):
                        "objective": info.objective},
     }
     if fused_ms is not None:
+        out["token_advantages"] = tok_cmp
         out["fused_step"] = {"calls": "hora_allocate(gains=NULL)+hora_group_advantage+hora_token_broadcast",
                              "ms_per_step": round(fused_ms, 4), "prompts_per_s": N / (fused_ms * 1e-3),
                              "note": "same outputs; the matrix is written once inside the workspace and not read back in "

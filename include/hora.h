@@ -272,6 +272,25 @@ hora_status_t hora_rollout_weights(const int64_t *group_offsets, int64_t N, cons
                                    void *stream);
 
 /*
+ * hora_group_advantage_tokens — hora_group_advantage followed by hora_token_broadcast (and, when token_weight is
+ * given, hora_rollout_weights broadcast the same way) in one kernel, with no per-rollout array in between
+ * (Sec. 3.1, Eq. grpo-objective; Sec. 3.2 for the 1/G_i weight under variable-size groups):
+ *   token_adv[t]    = adv of the rollout that owns token t, adv as defined for hora_group_advantage
+ *   token_weight[t] = 1/(G_g len_r) (HORA_WEIGHT_PER_TOKEN) or 1/(G_g length_const) (HORA_WEIGHT_CONST_LENGTH)
+ * for tokens t < min(T, token_offsets[R]).  Rollout r belongs to the group g with group_offsets[g] <= r <
+ * group_offsets[g+1]; rollouts at or beyond group_offsets[N] get advantage and weight 0.
+ *   rewards [group_offsets[N]] fp32; group_offsets [N+1] int64 non-decreasing from 0; token_offsets [R+1] int64
+ *   non-decreasing from 0; token_adv [T] fp32 out; token_weight [T] fp32 out or NULL (weight_mode and
+ *   length_const are then ignored); status_dev optional (INVALID_VALUE on decreasing group offsets).
+ * All device pointers, caller-owned; enqueues one kernel on `stream`.
+ */
+hora_status_t hora_group_advantage_tokens(const float *rewards, const int64_t *group_offsets, int64_t N,
+                                          const int64_t *token_offsets, int64_t R, int64_t T, int32_t mode,
+                                          float eps, int32_t ddof, int32_t weight_mode, float length_const,
+                                          float *token_adv, float *token_weight, int32_t *status_dev,
+                                          void *stream);
+
+/*
  * hora_token_broadcast — per-token advantages (Eq. grpo-objective: the advantage of a rollout does not
  * depend on the token position).
  *

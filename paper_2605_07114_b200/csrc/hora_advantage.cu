@@ -18,7 +18,7 @@
 // A group longer than the slab is streamed from global memory instead (same arithmetic).
 // r - mean is exactly zero for a constant group (partial sums k*r are exact in fp64), so such groups
 // get exactly zero.  Every order of operations is fixed: results are bitwise reproducible.
-#include "hora_common.cuh"
+#include "hora_group_stats.cuh"
 
 namespace hora {
 
@@ -42,40 +42,13 @@ __device__ __forceinline__ void cp_async_4(float *smem_dst, const float *gmem_sr
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
-__device__ __forceinline__ double warp_sum(double v) {
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(kFull, v, d);
-    return v;
-}
-
 __device__ __forceinline__ int64_t shfl_i64(int64_t v, int src) { return __shfl_sync(kFull, v, src); }
-
-// scale of one group from its statistics (run by the lane that owns the group)
-__device__ __forceinline__ double group_scale(int32_t mode, double ss, int64_t n, int32_t ddof, double eps) {
-    if (mode == HORA_ADV_RLOO) return n > 1 ? (double)n / (double)(n - 1) : 0.0;
-    const double var = (n - ddof > 0) ? ss / (double)(n - ddof) : 0.0;
-    const double den = sqrt(var) + eps;
-    return den > 0.0 ? 1.0 / den : 0.0;
-}
 
 // One group streamed from global memory by the whole warp (groups longer than the slab).
 __device__ void advantage_streamed(const float *__restrict__ rewards, int64_t s, int64_t e, int32_t mode, double eps,
                                    int32_t ddof, float *__restrict__ adv, int lane) {
-    const int64_t n = e - s;
-    double part = 0.0;
-    for (int64_t j = s + lane; j < e; j += kWarp) part += (double)__ldg(rewards + j);
-    const double sum = warp_sum(part);
-    const double mean = sum / (double)n;
-    double ss = 0.0;
-    if (mode == HORA_ADV_GRPO) {
-        double sq = 0.0;
-        for (int64_t j = s + lane; j < e; j += kWarp) {
-            const double d = (double)__ldg(rewards + j) - mean;
-            sq += d * d;
-        }
-        ss = warp_sum(sq);
-    }
-    const double scale = group_scale(mode, ss, n, ddof, eps);
+    double mean, scale;
+    group_mean_scale(rewards, s, e, mode, eps, ddof, lane, mean, scale);
     for (int64_t j = s + lane; j < e; j += kWarp) adv[j] = (float)(((double)__ldg(rewards + j) - mean) * scale);
 }
 

@@ -26,7 +26,8 @@ EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora
            "hora_token_broadcast", "hora_status_string", "hora_version", "hora_launch_count",
            "hora_allocate_static", "hora_allocate_static_capacity", "hora_allocate_profile_events",
            "hora_allocate_batched", "hora_allocate_batched_workspace_bytes", "hora_rollout_weights",
-           "hora_learned_prior", "hora_beta_binomial_nll", "hora_pass_at_k", "hora_pass_at_k_workspace_bytes")
+           "hora_learned_prior", "hora_beta_binomial_nll", "hora_pass_at_k", "hora_pass_at_k_workspace_bytes",
+           "hora_group_advantage_tokens")
 
 
 class HoraError(RuntimeError):
@@ -72,6 +73,8 @@ def load() -> C.CDLL:
     L.hora_allocate_profile_events.restype = None
     L.hora_group_advantage.argtypes = [p, p, i64, i32, C.c_float, i32, p, p, p]
     L.hora_group_advantage.restype = C.c_int
+    L.hora_group_advantage_tokens.argtypes = [p, p, i64, p, i64, i64, i32, C.c_float, i32, i32, C.c_float, p, p, p, p]
+    L.hora_group_advantage_tokens.restype = C.c_int
     L.hora_pass_at_k_workspace_bytes.argtypes = [i32]
     L.hora_pass_at_k_workspace_bytes.restype = C.c_size_t
     L.hora_pass_at_k.argtypes = [p, i64, i32, p, i32, p, p, p, C.c_size_t, p]
@@ -217,6 +220,16 @@ def hora_group_advantage(rewards, group_offsets, N, mode, eps, ddof, adv, status
     _check(rc, "hora_group_advantage")
 
 
+def hora_group_advantage_tokens(rewards, group_offsets, N, token_offsets, R, T, mode, eps, ddof, token_adv,
+                                token_weight=None, weight_mode=WEIGHT_PER_TOKEN, length_const=1.0, status_dev=None):
+    rc = load().hora_group_advantage_tokens(
+        _ptr(rewards, torch.float32, "rewards"), _ptr(group_offsets, torch.int64, "group_offsets"), N,
+        _ptr(token_offsets, torch.int64, "token_offsets"), R, T, mode, eps, ddof, weight_mode, length_const,
+        _ptr(token_adv, torch.float32, "token_adv"), _ptr(token_weight, torch.float32, "token_weight"),
+        _ptr(status_dev, torch.int32, "status_dev"), _stream())
+    _check(rc, "hora_group_advantage_tokens")
+
+
 def hora_pass_at_k_workspace_bytes(n_samples) -> int:
     return int(load().hora_pass_at_k_workspace_bytes(n_samples))
 
@@ -248,8 +261,7 @@ def hora_rollout_weights(group_offsets, N, token_offsets, mode, length_const, we
                                      _ptr(token_offsets, torch.int64, "token_offsets"), mode, length_const,
                                      _ptr(weights, torch.float32, "weights"), _ptr(status_dev, torch.int32, "status_dev"),
                                      _stream())
-    _check(rc, "hora_rollout_weights",
-           "hora_learned_prior", "hora_beta_binomial_nll", "hora_pass_at_k", "hora_pass_at_k_workspace_bytes")
+    _check(rc, "hora_rollout_weights")
 
 
 def hora_token_broadcast(adv, token_offsets, R, T, token_adv):

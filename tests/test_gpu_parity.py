@@ -481,3 +481,74 @@ def test_pass_at_k_rejects_bad_counts_and_k():
     with pytest.raises(hora.HoraError):
         hora.hora_pass_at_k(torch.zeros(3, dtype=torch.int32, device="cuda"), 3, n,
                             torch.ones(2, dtype=torch.int32, device="cuda"), 2, out, None, ws[:8])
+
+
+# ------------------------------------------------------------------------ fused advantage -> tokens
+def _fused_case(rng, sizes, len_lo, len_hi, binary):
+    goff = np.zeros(len(sizes) + 1, np.int64)
+    np.cumsum(sizes, out=goff[1:])
+    R = int(goff[-1])
+    rewards = (rng.random(R) < 0.35).astype(np.float32) if binary else rng.choice([0.0, 0.5, 1.0], R).astype(np.float32)
+    lens = rng.integers(len_lo, len_hi + 1, R)
+    toff = np.zeros(R + 1, np.int64)
+    np.cumsum(lens, out=toff[1:])
+    return goff, rewards, toff
+
+
+@pytest.mark.parametrize("mode,ddof,wmode", [(0, 0, None), (0, 1, 0), (1, 0, 1), (1, 0, None)])
+@pytest.mark.parametrize("shape", ["mixed", "long_groups", "short_rollouts", "tiny"])
+def test_group_advantage_tokens_matches_oracle(mode, ddof, wmode, shape):
+    """Fused call == oracle advantage, then oracle broadcast (and oracle weights, broadcast), element by element."""
+    from paper_2605_07114_b200 import hora
+    rng = np.random.default_rng([mode, ddof, len(shape)])
+    if shape == "mixed":
+        sizes, lo, hi = rng.choice([0, 1, 2, 8, 9, 31, 32, 33, 100, 264], 1500), 0, 700
+    elif shape == "long_groups":
+        sizes, lo, hi = rng.choice([1024, 1500, 3000, 8], 40), 1, 300       # groups that span several chunks and stages
+    elif shape == "short_rollouts":
+        sizes, lo, hi = rng.choice([8, 32, 40], 6000), 0, 3                 # thousands of rollouts per chunk: many stage rounds
+    else:
+        sizes, lo, hi = np.array([3, 0, 2]), 1, 5
+    goff, rewards, toff = _fused_case(rng, sizes, lo, hi, binary=(mode == 0))
+    N, R, T = len(sizes), int(goff[-1]), int(toff[-1])
+    eps = 1e-6
+    for misalign in (0, 1):
+        buf = torch.full((T + 8,), -7.0, dtype=torch.float32, device="cuda")
+        wbuf = torch.full((T + 8,), -7.0, dtype=torch.float32, device="cuda")
+        out, wout = buf[misalign:misalign + T], wbuf[misalign:misalign + T]
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        hora.hora_group_advantage_tokens(torch.from_numpy(rewards).cuda(), torch.from_numpy(goff).cuda(), N,
+                                         torch.from_numpy(toff).cuda(), R, T, mode, eps, ddof, out,
+                                         None if wmode is None else wout, 0 if wmode is None else wmode, 512.0, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        adv = orc.group_advantage(rewards, goff, mode, eps, ddof)
+        np.testing.assert_allclose(out.cpu().numpy(), orc.token_broadcast(adv, toff), rtol=0, atol=1e-5)
+        assert float(buf[misalign + T:].min()) == -7.0 and (misalign == 0 or float(buf[0]) == -7.0)
+        if wmode is not None:
+            w = orc.rollout_weights(goff, toff, wmode, 512.0)
+            assert np.array_equal(wout.cpu().numpy().view(np.uint32), orc.token_broadcast(w, toff).view(np.uint32))
+
+
+def test_group_advantage_tokens_partial_cover():
+    """T below the token count stops early; rollouts beyond the last group get 0."""
+    from paper_2605_07114_b200 import hora
+    rng = np.random.default_rng(5)
+    goff, rewards, toff = _fused_case(rng, rng.choice([8, 32], 300), 1, 400, True)
+    N, R = 300, int(goff[-1])
+    T = int(toff[-1]) - 12345
+    out = torch.full((int(toff[-1]),), -7.0, dtype=torch.float32, device="cuda")
+    hora.hora_group_advantage_tokens(torch.from_numpy(rewards).cuda(), torch.from_numpy(goff).cuda(), N,
+                                     torch.from_numpy(toff).cuda(), R, T, 0, 1e-6, 0, out)
+    exp = orc.token_broadcast(orc.group_advantage(rewards, goff, 0, 1e-6, 0), toff)
+    got = out.cpu().numpy()
+    np.testing.assert_allclose(got[:T], exp[:T], rtol=0, atol=1e-5)
+    assert (got[T:] == -7.0).all()
+    # only the first 200 groups are described: later rollouts carry no advantage
+    out.fill_(-7.0)
+    hora.hora_group_advantage_tokens(torch.from_numpy(rewards).cuda(), torch.from_numpy(goff[:201].copy()).cuda(), 200,
+                                     torch.from_numpy(toff).cuda(), R, int(toff[-1]), 0, 1e-6, 0, out)
+    got = out.cpu().numpy()
+    cut = int(toff[goff[200]])
+    np.testing.assert_allclose(got[:cut], exp[:cut], rtol=0, atol=1e-5)
+    assert (got[cut:] == 0.0).all()
