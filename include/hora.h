@@ -236,6 +236,15 @@ hora_status_t hora_beta_binomial_nll(const double *p_hat, const double *s_raw, d
                                      int32_t G0, int64_t N, double *nll, int32_t *status_dev, void *stream);
 
 /*
+ * hora_allocation_share — how prompts and Phase-B budget split over the Phase-A success count (the statistic of
+ * Fig. 3, Sec. 4.1): for k = 0..G0, prompts[k] = #{i : c_i = k}, budget[k] = sum of delta_i over those prompts.
+ *   c, delta [N] int32 device; prompts, budget [G0+1] int64 device out (overwritten); 0 <= G0 <= 2047.
+ *   status_dev optional: INVALID_VALUE if some c_i is outside [0, G0] or some delta_i < 0 (that prompt is skipped).
+ */
+hora_status_t hora_allocation_share(const int32_t *c, const int32_t *delta, int64_t N, int32_t G0,
+                                    int64_t *prompts, int64_t *budget, int32_t *status_dev, void *stream);
+
+/*
  * hora_pass_at_k — the unbiased Pass@K estimator (Eq. pass-k) averaged over prompts, for a grid of K values:
  *   pass_at_k[j] = mean over the Q prompts of  1 - C(n - c_q, K_j) / C(n, K_j),
  * c_q = correct samples among the n_samples drawn for prompt q.  Counts outside [0, n_samples] raise

@@ -27,7 +27,7 @@ EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora
            "hora_allocate_static", "hora_allocate_static_capacity", "hora_allocate_profile_events",
            "hora_allocate_batched", "hora_allocate_batched_workspace_bytes", "hora_rollout_weights",
            "hora_learned_prior", "hora_beta_binomial_nll", "hora_pass_at_k", "hora_pass_at_k_workspace_bytes",
-           "hora_group_advantage_tokens")
+           "hora_group_advantage_tokens", "hora_allocation_share")
 
 
 class HoraError(RuntimeError):
@@ -75,6 +75,8 @@ def load() -> C.CDLL:
     L.hora_group_advantage.restype = C.c_int
     L.hora_group_advantage_tokens.argtypes = [p, p, i64, p, i64, i64, i32, C.c_float, i32, i32, C.c_float, p, p, p, p]
     L.hora_group_advantage_tokens.restype = C.c_int
+    L.hora_allocation_share.argtypes = [p, p, i64, i32, p, p, p, p]
+    L.hora_allocation_share.restype = C.c_int
     L.hora_pass_at_k_workspace_bytes.argtypes = [i32]
     L.hora_pass_at_k_workspace_bytes.restype = C.c_size_t
     L.hora_pass_at_k.argtypes = [p, i64, i32, p, i32, p, p, p, C.c_size_t, p]
@@ -228,6 +230,13 @@ def hora_group_advantage_tokens(rewards, group_offsets, N, token_offsets, R, T, 
         _ptr(token_adv, torch.float32, "token_adv"), _ptr(token_weight, torch.float32, "token_weight"),
         _ptr(status_dev, torch.int32, "status_dev"), _stream())
     _check(rc, "hora_group_advantage_tokens")
+
+
+def hora_allocation_share(c, delta, N, G0, prompts, budget, status_dev=None):
+    rc = load().hora_allocation_share(_ptr(c, torch.int32, "c"), _ptr(delta, torch.int32, "delta"), N, G0,
+                                      _ptr(prompts, torch.int64, "prompts"), _ptr(budget, torch.int64, "budget"),
+                                      _ptr(status_dev, torch.int32, "status_dev"), _stream())
+    _check(rc, "hora_allocation_share")
 
 
 def hora_pass_at_k_workspace_bytes(n_samples) -> int:

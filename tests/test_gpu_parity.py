@@ -552,3 +552,44 @@ def test_group_advantage_tokens_partial_cover():
     cut = int(toff[goff[200]])
     np.testing.assert_allclose(got[:cut], exp[:cut], rtol=0, atol=1e-5)
     assert (got[cut:] == 0.0).all()
+
+
+# ----------------------------------------------------------------------- allocation share (Fig. 3)
+@pytest.mark.parametrize("N,G0", [(0, 8), (1, 0), (77, 8), (100003, 8), (250000, 16), (50000, 2047)])
+def test_allocation_share_bit_exact(N, G0):
+    from oracle import share as share_orc
+    from paper_2605_07114_b200 import hora
+    rng = np.random.default_rng(N + G0)
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    d = rng.integers(0, 1025, N).astype(np.int32)
+    if N > 10:
+        d[:4] = 2**31 - 1                                   # sums beyond 32 bits
+        c[:4] = c[0]
+    prompts = torch.full((G0 + 1,), -1, dtype=torch.int64, device="cuda")
+    budget = torch.full((G0 + 1,), -1, dtype=torch.int64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    hora.hora_allocation_share(torch.from_numpy(c).cuda(), torch.from_numpy(d).cuda(), N, G0, prompts, budget, status)
+    torch.cuda.synchronize()
+    exp_p, exp_b = share_orc.allocation_share(c, d, G0)
+    assert int(status.item()) == 0
+    assert prompts.cpu().tolist() == exp_p and budget.cpu().tolist() == exp_b
+
+
+def test_allocation_share_of_an_allocation_and_bad_input():
+    from oracle import share as share_orc
+    from paper_2605_07114_b200 import hora
+    import gpu_util as gu
+    from paper_2605_07114_b200 import workloads as wl
+    w = wl.make("cfg2", 4096)
+    d = gu.gpu_allocate(w.alpha, w.beta, w.alpha0, w.beta0, w.c, w.G0, w.cap, w.ld, w.B, exact=w.exact_int)[0]
+    prompts = torch.empty(w.G0 + 1, dtype=torch.int64, device="cuda")
+    budget = torch.empty(w.G0 + 1, dtype=torch.int64, device="cuda")
+    hora.hora_allocation_share(torch.from_numpy(w.c).cuda(), torch.from_numpy(d).cuda(), w.N, w.G0, prompts, budget)
+    assert int(budget.sum()) == w.B and int(prompts.sum()) == w.N
+    assert (prompts.cpu().tolist(), budget.cpu().tolist()) == share_orc.allocation_share(w.c, d, w.G0)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    hora.hora_allocation_share(torch.tensor([0, 9, 1], dtype=torch.int32, device="cuda"),
+                               torch.tensor([1, 1, 1], dtype=torch.int32, device="cuda"), 3, 8, prompts, budget, status)
+    assert int(status.item()) == 2 and int(prompts.sum()) == 2
+    with pytest.raises(hora.HoraError):
+        hora.hora_allocation_share(None, None, 0, 4096, prompts, budget)

@@ -282,14 +282,17 @@ def test_budget_share_matches_paper_statistic():
     G0, shard, B = 8, 15, 15 * 24
     pmf = np.array([vals["c=0"][0]] + [(1 - vals["c=0"][0] - vals["c=8"][0]) / 7] * 7 + [vals["c=8"][0]])
     rng = np.random.default_rng(2024)
+    from oracle import share as share_orc
     got = np.zeros(G0 + 1)
     cnt = np.zeros(G0 + 1)
     cap = np.full(shard, B, np.int32)
     for _ in range(196 * 4):
         c = rng.choice(G0 + 1, size=shard, p=pmf).astype(np.int32)
         d = orc.greedy_exact(None, None, 1.0, 1.0, c, G0, cap, B)[0]
-        np.add.at(got, c, d)
-        np.add.at(cnt, c, 1)
+        prompts, budget = share_orc.allocation_share(c, d, G0)
+        assert sum(prompts) == shard and sum(budget) == B
+        got += budget
+        cnt += prompts
     share = got / got.sum()
     assert abs(share[0] - vals["c=0"][1]) < 0.04
     assert abs(share[8] - vals["c=8"][1]) < 0.04
@@ -516,3 +519,18 @@ def test_pass_at_k_estimator_pins():
         mean = sum(Fraction(math.comb(n, c)) * p**c * (1 - p)**(n - c) * passk.pass_at_k_one(n, c, K) for c in range(n + 1))
         assert mean == 1 - (1 - p)**K
     assert passk.pass_at_k([0, 7, 3], 7, [1, 7]) == [float(Fraction(10, 21)), float(Fraction(2, 3))]
+
+
+def test_allocation_share_statistic_pins():
+    """Fig. 3 statistic: hand example, and agreement with numpy's bincount (an independent routine)."""
+    from oracle import share as share_orc
+    prompts, budget = share_orc.allocation_share([0, 2, 2, 1, 0], [5, 1, 0, 3, 7], 2)
+    assert prompts == [2, 1, 2] and budget == [12, 3, 1]
+    rng = np.random.default_rng(8)
+    c = rng.integers(0, 9, 5000)
+    d = rng.integers(0, 100, 5000)
+    prompts, budget = share_orc.allocation_share(c, d, 8)
+    assert prompts == np.bincount(c, minlength=9).tolist()
+    assert budget == np.bincount(c, weights=d, minlength=9).astype(np.int64).tolist()
+    with pytest.raises(ValueError):
+        share_orc.allocation_share([3], [1], 2)
