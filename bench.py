@@ -237,6 +237,21 @@ def run_ours(args):
     if info.status != 0 or info.sum_G != total:
         raise RuntimeError("allocation changed during the timed loop")
 
+    # ---- where hora_allocate spends its time: events the library records at its stage boundaries ----
+    n_prof = max(3, min(args.steps, 20))
+    st_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(n_prof)]
+    for evs in st_ev:
+        for ev in evs:
+            ev.record()
+    for k in range(n_prof):
+        hora.hora_allocate_profile_stages([ev.cuda_event for ev in st_ev[k]])
+        step()
+    hora.hora_allocate_profile_stages(None)
+    torch.cuda.synchronize()
+    st = np.array([[evs[i].elapsed_time(evs[i + 1]) for i in range(6)] for evs in st_ev]).mean(axis=0)
+    alloc_stages = dict(zip(("estimate", "full_read_level0", "rows_level1", "threshold_list_or_digits",
+                             "closing_and_scan", "outputs"), (round(float(x), 4) for x in st)))
+
     # ---- the same step with the fused call: hora_allocate builds the matrix itself and counts on the way ----
     fused_ms = None
     if world == 1:
@@ -414,6 +429,7 @@ def run_ours(args):
                      "prompts_per_s": N / (pipe_ms * 1e-3), "candidate_gains_per_s": cand / (pipe_ms * 1e-3)},
         "tokens_per_s": T / (float(st_mean[3]) * 1e-3),
         "stages": stage_report,
+        "allocate_stages_ms": alloc_stages,
         "allocation": {"lambda": info.lambda_, "n_above": info.n_above, "n_tied": info.n_tied,
                        "objective": info.objective},
     }

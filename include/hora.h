@@ -322,6 +322,18 @@ hora_status_t hora_token_broadcast(const float *adv, const int64_t *token_offset
  */
 void hora_allocate_profile_events(void *start_event, void *stop_event);
 
+/*
+ * hora_allocate_profile_stages — measurement aid, no counterpart in the paper.  `events_host` is a HOST array of
+ * n <= 7 cudaEvent_t handles (timing enabled); every following hora_allocate / hora_allocate_static call records
+ * them on its stream at these points:  [0] entry (after the workspace is cleared), [1] after the sampled estimate,
+ * [2] after the full-read pass, [3] after the per-row pass (level 1), [4] after the threshold is complete (list
+ * selection, or the digit levels), [5] after the per-row closing and the block scan (and the exact tie ranking),
+ * [6] after the outputs are written.  Differences of consecutive events are the device times of the stages.
+ * A NULL handle skips its point; NULL or n = 0 switches everything off (the default).  Process-wide host
+ * setting; the array is read during this call only.
+ */
+void hora_allocate_profile_stages(void *const *events_host, int32_t n);
+
 const char *hora_status_string(hora_status_t status);   /* host: static string */
 int         hora_version(void);                         /* host: major*10000 + minor*100 + patch */
 uint64_t    hora_launch_count(void);                    /* host: kernels this library has launched so far in this

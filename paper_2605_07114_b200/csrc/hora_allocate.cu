@@ -14,12 +14,17 @@
 //             rows, sums the caps and writes a 2-byte sketch of every 8th key (its top 16 bits).
 //   level 1   a thread per row: a row is non-increasing, so its keys with the resolved prefix form ONE
 //             contiguous segment, which the sketch brackets to within 8 keys on each side; only the
-//             bracket is read, the segment [p_hi, p_lo) stored, its next 13 bits histogrammed, and rows
-//             whose segment is not empty are appended to a list.
-//   level 2-4 a thread per listed row narrows its segment by the digit just selected and histograms the
-//             next one (13 bits at a time until all 64 are resolved), then a last narrowing pass.
-//   sum       p_hi = #keys > lambda, p_lo - p_hi = #keys == lambda per row; block sums and their scan give
-//             n_above, n_tied and the exclusive prefixes over prompts; priors are validated here.
+//             bracket is read and the segment [p_hi, p_lo) stored.  The same pass validates the priors.
+//             What happens to the keys of the segments depends on how many there are (level 0 knows the
+//             exact count of keys with the resolved prefix):
+//   list      at most 65536 of them (the usual case after a window hit): level 1 appends them to a list
+//             and ONE CTA resolves the remaining bits over that list, with no further pass over rows.
+//   level 2-4 more than that (a missed window, or heavy ties): level 1 histograms the next 13 bits and
+//             lists the rows whose segment is not empty; a thread per listed row then narrows its segment
+//             by the digit just selected and histograms the next one, 13 bits at a time.
+//   sum       every non-empty segment is narrowed by the finished threshold: p_hi = #keys > lambda,
+//             p_lo - p_hi = #keys == lambda per row; block sums and their scan give n_above, n_tied and
+//             the exclusive prefixes over prompts.
 //   out       Delta_i = p_hi + (tied candidates of row i that fall within the first R = B - n_above tied
 //             candidates in prompt order); G_i, CSR offsets, objective.
 //
@@ -41,6 +46,8 @@
 namespace hora {
 
 constexpr int kLevels = 5;                   // level 0 (full read) + four digit levels
+constexpr int kListCap = 65536;              // candidates the single-CTA list selection accepts
+constexpr int kListThreads = 1024;
 constexpr int kBins = 8192;                  // 13-bit digits
 constexpr int kDigitBits = 13;
 constexpr int kWinBins = 2;                  // coarse bins covered by the fine window of level 0
@@ -71,7 +78,10 @@ struct AllocHeader {
     double objective;
     unsigned long long band_above;     // exact mode: candidates above the band
     unsigned int n_types;
-    unsigned int pad1;
+    unsigned int n_cand;               // list mode: keys appended by level 1
+    long long bin_count;               // keys that carry the prefix resolved so far
+    int32_t list_mode;                 // 1: the keys of level 1's segments go to the candidate list
+    int32_t pad1;
 };
 
 struct Workspace {
@@ -89,6 +99,7 @@ struct Workspace {
     unsigned long long *tkeys, *tcounts;   // [kTypeSlots]
     int32_t *tlabel;                   // [kTypeSlots]
     int32_t *rowslot;                  // [N]
+    unsigned long long *cand_key;      // [kListCap] list mode: every key that carries level 0's prefix
     double *gains;                     // [N*ld] when the caller passed none
     size_t bytes;
 };
@@ -113,6 +124,7 @@ static Workspace carve(void *base, int64_t N, int32_t ld, bool need_gains, bool 
     w.bsum_hi = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
     w.bsum_t = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
     w.objpart = reinterpret_cast<double *>(take(sizeof(double) * (size_t)NB));
+    w.cand_key = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kListCap));
     if (exact) {
         w.tkeys = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kTypeSlots));
         w.tcounts = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kTypeSlots));
@@ -162,18 +174,28 @@ __device__ __forceinline__ long long block_exclusive_sum(long long v, long long 
 // Run by ONE CTA.  Scanning from the top bin down, find the bin where the running count reaches `need`:
 //   count(bins above d) < need <= count(bins above d) + count(d).
 // Returns d (or -1 if need is out of range) to every thread, with the count above d in *above_out and the
-// count of d in *count_out.  Two stages so that no thread walks memory serially: every thread sums a
-// contiguous run of bins (independent loads) and a block scan picks the run that holds the crossing; then
-// the first warp loads that run's bins one per lane (`per` <= 32) and a warp scan pins the bin.
+// count of d in *count_out.  `bins` is a power of two and `hist` 16-byte aligned.  Two stages, neither of
+// which walks memory serially (a dependent chain of 32 loads from L2 cost 16 us here): every thread sums a
+// contiguous run of `per` bins, fetched by independent 16-byte loads that are all issued before the first
+// is used, and a block scan picks the run that holds the crossing; then the first warp loads that run's
+// bins one per lane (`per` <= 32) and a warp scan pins the bin.
 __device__ int locate_rank(const unsigned long long *hist, int bins, long long need, long long *above_out,
                            long long *count_out, long long *s_warp) {
     __shared__ long long s_found[3];                        // top bin of the run, count above the run, found flag
-    const int per = (bins + kSelThreads - 1) / kSelThreads; // <= 32 for bins <= 8192
+    const int per = (bins + kSelThreads - 1) / kSelThreads; // 1, or an even number <= 32 for bins <= 8192
     const int top = bins - 1 - (int)threadIdx.x * per;      // this thread's run: bins top, top-1, ..., top-per+1
     long long local = 0;
-#pragma unroll 8
-    for (int j = 0; j < per; ++j)
-        if (top - j >= 0) local += (long long)__ldcg(hist + top - j);
+    if (per == 1) {
+        if (top >= 0) local = (long long)__ldcg(hist + top);
+    } else {                                                // bins == kSelThreads * per: every run is complete
+        const ulonglong2 *run = reinterpret_cast<const ulonglong2 *>(hist + (top - per + 1));
+        const int nvec = per >> 1;
+        ulonglong2 v[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) v[u] = u < nvec ? __ldcg(run + u) : make_ulonglong2(0ull, 0ull);
+#pragma unroll
+        for (int u = 0; u < 16; ++u) local += (long long)(v[u].x + v[u].y);
+    }
     if (threadIdx.x == 0) s_found[2] = 0;
     long long total;
     const long long above = block_exclusive_sum(local, &total, s_warp);
@@ -229,6 +251,7 @@ __device__ void find_digit(AllocHeader *hdr, const unsigned long long *hist, int
         hdr->need -= above;
         hdr->prefix_key |= (unsigned long long)digit << shift;
         hdr->resolved += bits;
+        hdr->bin_count = count;
     }
     __syncthreads();
 }
@@ -288,9 +311,16 @@ select_estimate(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, 
         capi = capi < 0 ? 0 : (capi > ld ? ld : capi);
         if (lane == 0) capsum += capi;
         const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-        for (int32_t j = lane; j < capi; j += kWarp) {
-            const unsigned long long key = __ldg(keys + j);
-            atomicAdd(&s_hist[(int)(key >> 51) & (kBins - 1)], 1u);
+        for (int32_t k0 = 0; k0 < capi; k0 += 8 * kWarp) {      // eight coalesced loads in flight per lane
+            unsigned long long key[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int32_t j = k0 + u * kWarp + lane;
+                key[u] = j < capi ? __ldg(keys + j) : 0ull;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (k0 + u * kWarp + lane < capi) atomicAdd(&s_hist[(int)(key[u] >> 51) & (kBins - 1)], 1u);
         }
     }
     __syncthreads();
@@ -345,6 +375,7 @@ __device__ void level0_finish(AllocHeader *hdr, unsigned long long *hist, unsign
         const unsigned w = (unsigned)(d0 - win_lo);
         if (hdr->resolved == kDigitBits && w < (unsigned)kWinBins)        // inside the window: 10 more bits for free
             find_digit(hdr, hist_fine + w * kFinePerBin, kFinePerBin, kFineBits, 51 - kFineBits, 0, true, s_warp);
+        if (threadIdx.x == 0) hdr->list_mode = (hdr->resolved > 0 && hdr->bin_count <= (long long)kListCap) ? 1 : 0;
     }
 }
 
@@ -595,35 +626,55 @@ gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ 
 // P that prefix.  The sketch holds the top 16 bits of the first (largest) key of every group of 8 keys.
 // Compared at min(r, 16) bits: groups whose first key is above P form a prefix of G1 groups, groups whose
 // first key is above or equal a prefix of G2 >= G1 groups.  Every key with prefix P therefore sits in
-// groups G1-1 .. G2-1, and so does the boundary between "above" and "equal"; the thread walks only those
-// keys (a handful after a window hit), classifies them on all r bits and histograms the ones with
-// prefix P on the next digit.  Rows that keep a non-empty segment are appended to the active list.
-// A warp per row was tried first: with a million rows the per-row issue slots, not memory, set its time.
+// groups G1-1 .. G2-1, and so does the boundary between "above" and "equal"; the thread reads only those
+// keys (one or two groups after a window hit) and classifies them on all r bits.  The keys with prefix P
+// go to the candidate list (list mode: one slot reservation per CTA and 256 rows) or are histogrammed on
+// the next digit, their rows appended to the active list.
+// A warp per row was tried first: with a million rows the per-row issue slots, not memory, set its time;
+// for the same reason the sketch entries are compared two at a time (they are 15-bit numbers, so
+// (e | 0x8000) - p keeps bit 15 exactly when e >= p, in both halves of a word at once).
+__device__ __forceinline__ void sketch_count(unsigned w, unsigned mask2, unsigned Pp, unsigned &acc_ge,
+                                             unsigned &acc_gt) {
+    const unsigned d = ((w & mask2) | 0x80008000u) - Pp;      // per half: 0x8000 + e - p, never borrows
+    acc_ge += (d >> 15) & 0x00010001u;
+    acc_gt += ((d - 0x00010001u) >> 15) & 0x00010001u;        // e - p - 1 >= 0
+}
+
+template <bool VEC2>
 __global__ void __launch_bounds__(kSelThreads)
-select_level1(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
-              const double *__restrict__ gains, AllocHeader *hdr, unsigned long long *hist1,
+select_level1(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
+              const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N,
+              int32_t ld, const double *__restrict__ gains, AllocHeader *hdr, unsigned long long *hist1,
               const uint16_t *__restrict__ sketch, int32_t sk_ld, int2 *__restrict__ rowstate,
-              int32_t *__restrict__ active) {
+              int32_t *__restrict__ active, unsigned long long *__restrict__ cand_key) {
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
+    __shared__ unsigned int s_base;
     if (*(volatile int32_t *)&hdr->status != 0) return;
-    for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
-    __syncthreads();
+    const bool list = hdr->list_mode != 0;
+    if (!list) {
+        for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
+        __syncthreads();
+    }
     const int lane = lane_id();
-    const int r = hdr->resolved;
-    const unsigned long long P = hdr->prefix_key >> (64 - r);
+    const int r = hdr->resolved;                                 // 13 or 23: the prefix lies in the key's high word
+    const unsigned P = (unsigned)(hdr->prefix_key >> 32) >> (32 - r);
     const int sk_shift = r < 16 ? 16 - r : 0;                    // sketch entries compared at min(r, 16) bits
-    const unsigned Psk = (unsigned)((hdr->prefix_key >> 48) >> sk_shift);
+    const unsigned mask2 = ((0xFFFFu << sk_shift) & 0xFFFFu) * 0x00010001u;
+    const unsigned Pp = ((unsigned)(hdr->prefix_key >> 48) * 0x00010001u) & mask2;
     int bits, shift;
     next_digit(r, &bits, &shift);
     const unsigned long long digit_mask = (1ull << bits) - 1ull;
     const int64_t stride = (int64_t)gridDim.x * kSelThreads;
+    bool bad = false;
     for (int64_t base = (int64_t)blockIdx.x * kSelThreads; base < N; base += stride) {
         const int64_t row = base + threadIdx.x;
-        int32_t n_eq = 0;
+        int32_t p_hi = 0, n_eq = 0;
+        const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains);
         if (row < N) {
-            int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
-            capi = capi < 0 ? 0 : (capi > ld ? ld : capi);
+            const Posterior post = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row);
+            bad |= !post.ok;
+            const int32_t capi = post.cap;                       // 0 for an invalid row
             const int n_groups = (capi + 7) >> 3;
             // the sketch row is 16-byte aligned and padded to a multiple of 8 entries
             const uint4 *sk4 = reinterpret_cast<const uint4 *>(sketch + row * (int64_t)sk_ld);
@@ -633,78 +684,253 @@ select_level1(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
                     v[u] = (g0 + 8 * u < n_groups) ? __ldg(sk4 + (g0 >> 3) + u) : make_uint4(0u, 0u, 0u, 0u);
+                unsigned acc_ge = 0, acc_gt = 0;                 // two 16-bit counters each
+                if (g0 + 32 <= n_groups) {
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                    for (int u = 0; u < 4; ++u) {
+                        sketch_count(v[u].x, mask2, Pp, acc_ge, acc_gt);
+                        sketch_count(v[u].y, mask2, Pp, acc_ge, acc_gt);
+                        sketch_count(v[u].z, mask2, Pp, acc_ge, acc_gt);
+                        sketch_count(v[u].w, mask2, Pp, acc_ge, acc_gt);
+                    }
+                } else {                                         // ragged end: entries past the last group do not count
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int g = g0 + 8 * u + 2 * i;
-                        const unsigned e0 = (w[i] & 0xFFFFu) >> sk_shift, e1 = (w[i] >> 16) >> sk_shift;
-                        const bool v0 = g < n_groups, v1 = g + 1 < n_groups;
-                        G1 += (v0 && e0 > Psk) + (v1 && e1 > Psk);
-                        G2 += (v0 && e0 >= Psk) + (v1 && e1 >= Psk);
+                    for (int u = 0; u < 4; ++u) {
+                        const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int left = n_groups - (g0 + 8 * u + 2 * i);
+                            const unsigned valid = left >= 2 ? 0xFFFFFFFFu : (left == 1 ? 0x0000FFFFu : 0u);
+                            unsigned ge = 0, gt = 0;
+                            sketch_count(w[i], mask2, Pp, ge, gt);
+                            acc_ge += ge & valid & 0x00010001u;
+                            acc_gt += gt & valid & 0x00010001u;
+                        }
                     }
                 }
+                G1 += (int)((acc_gt & 0xFFFFu) + (acc_gt >> 16));
+                G2 += (int)((acc_ge & 0xFFFFu) + (acc_ge >> 16));
                 if (G2 < g0 + 32) break;                         // entries only decrease: the later ones are below P
             }
             const int32_t lo = G1 > 0 ? (G1 - 1) << 3 : 0;
             const int32_t hi = (G2 << 3) > capi ? capi : (G2 << 3);
-            const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+            keys += row * (int64_t)ld;
             int32_t n_gt = 0;
-            bool stop = false;
-            for (int32_t j0 = lo; j0 < hi && !stop; j0 += 8) {   // one group of 8 keys (independent loads) at a time
+            for (int32_t j0 = lo; j0 < hi; j0 += 8) {            // one group of 8 keys (independent loads) at a time
                 unsigned long long key[8];
+                if (VEC2) {                                      // j0 is a multiple of 8: 16-byte aligned in an aligned row
 #pragma unroll
-                for (int u = 0; u < 8; ++u) key[u] = (j0 + u < hi) ? __ldg(keys + j0 + u) : 0ull;
+                    for (int u = 0; u < 8; u += 2) {
+                        ulonglong2 t = make_ulonglong2(0ull, 0ull);
+                        if (j0 + u < hi) t = __ldg(reinterpret_cast<const ulonglong2 *>(keys + j0 + u));
+                        key[u] = t.x;
+                        key[u + 1] = t.y;
+                    }
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) key[u] = (j0 + u < hi) ? __ldg(keys + j0 + u) : 0ull;
+                }
+                int32_t eq_here = 0;
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                    const unsigned long long kp = key[u] >> (64 - r);
-                    if (j0 + u < hi && !stop) {
-                        if (kp > P) {
-                            ++n_gt;
-                        } else if (kp == P) {
-                            ++n_eq;
-                            atomicAdd(&s_hist[(key[u] >> shift) & digit_mask], 1u);
-                        } else {
-                            stop = true;                         // the row is sorted: nothing further can match
-                        }
-                    }
+                    const unsigned kp = (unsigned)(key[u] >> 32) >> (32 - r);
+                    const bool in = j0 + u < hi;
+                    n_gt += in && kp > P;
+                    const bool eq = in && kp == P;
+                    eq_here += eq;
+                    if (!list && eq) atomicAdd(&s_hist[(key[u] >> shift) & digit_mask], 1u);
+                }
+                n_eq += eq_here;
+                if (n_eq > 0 && eq_here == 0) break;             // the row is sorted: past the segment
+            }
+            p_hi = lo + n_gt;
+            rowstate[row] = make_int2(p_hi, p_hi + n_eq);
+        }
+        if (list) {
+            // one reservation per CTA and step; the order of the list does not matter to anything
+            long long tot;
+            const long long excl = block_exclusive_sum((long long)n_eq, &tot, s_warp);
+            if (tot > 0) {
+                if (threadIdx.x == 0) s_base = atomicAdd(&hdr->n_cand, (unsigned int)tot);
+                __syncthreads();
+                const long long slot = (long long)s_base + excl;
+                for (int32_t j = 0; j < n_eq; ++j) {
+                    const unsigned long long key = __ldg(keys + p_hi + j);
+                    if (slot + j < kListCap) cand_key[slot + j] = key;
+                    atomicAdd(hist1 + ((key >> shift) & digit_mask), 1ull);   // few keys: straight to global memory
                 }
             }
-            rowstate[row] = make_int2(lo + n_gt, lo + n_gt + n_eq);
-        }
-        // append the rows that keep a segment: one counter update per warp
-        const unsigned keep = __ballot_sync(kFull, n_eq > 0);
-        if (keep) {
-            unsigned int slot0 = 0;
-            if (lane == 0) slot0 = atomicAdd(&hdr->n_active, (unsigned int)__popc(keep));
-            slot0 = __shfl_sync(kFull, slot0, 0);
-            if (n_eq > 0) active[slot0 + __popc(keep & ((1u << lane) - 1u))] = (int32_t)row;
+        } else {
+            // append the rows that keep a segment: one counter update per warp
+            const unsigned keep = __ballot_sync(kFull, n_eq > 0);
+            if (keep) {
+                unsigned int slot0 = 0;
+                if (lane == 0) slot0 = atomicAdd(&hdr->n_active, (unsigned int)__popc(keep));
+                slot0 = __shfl_sync(kFull, slot0, 0);
+                if (n_eq > 0) active[slot0 + __popc(keep & ((1u << lane) - 1u))] = (int32_t)row;
+            }
         }
     }
+    if (bad) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);
+    if (list) return;
     __syncthreads();
     flush_hist(s_hist, hist1, 1 << bits);
     if (last_block(&hdr->ticket[1])) find_digit(hdr, hist1, 1 << bits, bits, shift, 1, false, s_warp);
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Levels 2..4 and the closing pass (level 5): a thread per ACTIVE row narrows the stored segment by the
-// digit selected one level up; for levels 2..4 the keys that remain are histogrammed on the next digit
-// and the last CTA selects it.  The active list is in no particular order; nothing here depends on it.
+// List mode: ONE CTA resolves the remaining bits of the threshold over the candidate list (every key that
+// carries level 0's prefix).  The first digit comes from the histogram level 1 accumulated; the keys that
+// carry it are usually a handful and are gathered into shared memory, over which the remaining digits are
+// found 13 bits per sweep.  Should more than kListSmall keys share that digit (ties), the sweeps run over
+// the list in global memory instead.
+constexpr int kListSmall = 1536;
+
+// digit search over a histogram in shared memory, run by the whole CTA: the bin where the count from the
+// top reaches `need`.  s_pick receives (digit, count above it, count of it); digit -1 if out of range.
+__device__ __forceinline__ void list_locate(const unsigned int *s_hist, int bins, long long need, long long *s_scan,
+                                            long long *s_pick) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per = (bins + kListThreads - 1) / kListThreads;    // thread t owns bins top, top-1, ..., top-per+1
+    const int top = bins - 1 - tid * per;
+    long long local = 0;
+    for (int j = 0; j < per; ++j)
+        if (top - j >= 0) local += s_hist[top - j];
+    long long inc = local;
+#pragma unroll
+    for (int d = 1; d < kWarp; d <<= 1) {
+        const long long t = __shfl_up_sync(kFull, inc, d);
+        if (lane >= d) inc += t;
+    }
+    if (lane == kWarp - 1) s_scan[warp] = inc;
+    if (tid == 0) s_pick[0] = -1;
+    __syncthreads();
+    long long above = inc - local;
+    for (int w = 0; w < warp; ++w) above += s_scan[w];
+    if (above < need && need <= above + local) {                 // at most one thread: the crossing is in its run
+        long long run = above;
+        for (int j = 0; j < per; ++j) {
+            const long long cnt = s_hist[top - j];
+            if (need <= run + cnt) {
+                s_pick[0] = top - j;
+                s_pick[1] = run;
+                s_pick[2] = cnt;
+                break;
+            }
+            run += cnt;
+        }
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kListThreads)
+select_list(AllocHeader *hdr, const unsigned long long *hist1, const unsigned long long *__restrict__ cand_key) {
+    __shared__ unsigned int s_hist[kBins];
+    __shared__ unsigned long long s_keys[kListSmall];
+    __shared__ long long s_scan[kListThreads / kWarp];
+    __shared__ long long s_pick[3];                              // digit, count above it, count of it
+    __shared__ unsigned int s_fill;
+    if (*(volatile int32_t *)&hdr->status != 0 || hdr->list_mode == 0) return;
+    const int tid = threadIdx.x;
+    unsigned int n = hdr->n_cand;
+    n = n < (unsigned)kListCap ? n : (unsigned)kListCap;
+    int resolved = hdr->resolved;
+    long long need = hdr->need;
+    unsigned long long prefix = hdr->prefix_key;
+    const int r0 = resolved;                                     // every key of the list agrees on these bits
+    // first digit: level 1 left its histogram in global memory
+    {
+        int bits, shift;
+        next_digit(resolved, &bits, &shift);
+        const int bins = 1 << bits;
+        for (int b = tid; b < bins; b += kListThreads) s_hist[b] = (unsigned int)__ldcg(hist1 + b);
+        if (tid == 0) s_fill = 0;
+        __syncthreads();
+        list_locate(s_hist, bins, need, s_scan, s_pick);
+        if (s_pick[0] < 0) return;                               // cannot happen: need lies within the list
+        need -= s_pick[1];
+        prefix |= (unsigned long long)s_pick[0] << shift;
+        resolved += bits;
+    }
+    const long long left = s_pick[2];                            // keys that carry the first digit
+    const unsigned long long *src = cand_key;
+    __syncthreads();
+    if (left <= kListSmall && resolved < 64) {                   // gather them; the later sweeps stay in shared memory
+        const int known = resolved - r0;
+        const unsigned long long want = (prefix << r0) >> (64 - known);
+        for (unsigned int i0 = 0; i0 < n; i0 += 8 * kListThreads) {
+            unsigned long long key[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const unsigned int i = i0 + u * kListThreads + tid;
+                key[u] = i < n ? cand_key[i] : 0ull;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const unsigned int i = i0 + u * kListThreads + tid;
+                if (i < n && (key[u] << r0) >> (64 - known) == want) {
+                    const unsigned int slot = atomicAdd(&s_fill, 1u);
+                    if (slot < (unsigned)kListSmall) s_keys[slot] = key[u];
+                }
+            }
+        }
+        __syncthreads();
+        n = s_fill < (unsigned)kListSmall ? s_fill : (unsigned)kListSmall;
+        src = s_keys;
+    }
+    while (resolved < 64) {
+        int bits, shift;
+        next_digit(resolved, &bits, &shift);
+        const int bins = 1 << bits;
+        for (int b = tid; b < bins; b += kListThreads) s_hist[b] = 0;
+        __syncthreads();
+        // keys that agree with the digits found so far in this kernel (bits r0 .. resolved-1)
+        const int known = resolved - r0;
+        const unsigned long long want = (prefix << r0) >> (64 - known);
+        for (unsigned int i0 = 0; i0 < n; i0 += 8 * kListThreads) {
+            unsigned long long key[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const unsigned int i = i0 + u * kListThreads + tid;
+                key[u] = i < n ? src[i] : 0ull;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const unsigned int i = i0 + u * kListThreads + tid;
+                if (i < n && (key[u] << r0) >> (64 - known) == want)
+                    atomicAdd(&s_hist[(key[u] >> shift) & (unsigned long long)(bins - 1)], 1u);
+            }
+        }
+        __syncthreads();
+        list_locate(s_hist, bins, need, s_scan, s_pick);
+        if (s_pick[0] < 0) break;                                // cannot happen
+        need -= s_pick[1];
+        prefix |= (unsigned long long)s_pick[0] << shift;
+        resolved += bits;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        hdr->prefix_key = prefix;
+        hdr->need = need;
+        hdr->resolved = resolved;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Levels 2..4 (only when the candidates were too many for the list): a thread per ACTIVE row narrows the
+// stored segment by the digit selected one level up; the keys that remain are histogrammed on the next
+// digit and the last CTA selects it.  The active list is in no particular order; nothing here depends on it.
 __global__ void __launch_bounds__(kSelThreads)
 select_refine(int32_t ld, const double *__restrict__ gains, int level, AllocHeader *hdr,
               unsigned long long *hist_all, int2 *__restrict__ rowstate, const int32_t *__restrict__ active) {
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
-    if (*(volatile int32_t *)&hdr->status != 0) return;
-    const bool closing = level >= kLevels;
+    if (*(volatile int32_t *)&hdr->status != 0 || hdr->list_mode != 0) return;
     int bits = 0, shift = 0;
-    if (!closing) next_digit(hdr->resolved, &bits, &shift);
+    next_digit(hdr->resolved, &bits, &shift);
     const int bins = 1 << bits;
-    if (!closing) {
-        for (int b = threadIdx.x; b < bins; b += kSelThreads) s_hist[b] = 0;
-        __syncthreads();
-    }
+    for (int b = threadIdx.x; b < bins; b += kSelThreads) s_hist[b] = 0;
+    __syncthreads();
     const int shift_prev = hdr->lv_shift[level - 1];
     const unsigned long long mask_prev = (1ull << hdr->lv_bits[level - 1]) - 1ull;
     const unsigned long long d_prev = (unsigned long long)hdr->sel_digit[level - 1];
@@ -723,7 +949,7 @@ select_refine(int32_t ld, const double *__restrict__ gains, int level, AllocHead
             if (dp > d_prev) {
                 new_hi = p + 1;
             } else if (dp == d_prev) {
-                if (!closing) atomicAdd(&s_hist[(key >> shift) & mask_cur], 1u);
+                atomicAdd(&s_hist[(key >> shift) & mask_cur], 1u);
             } else {
                 break;
             }
@@ -731,7 +957,6 @@ select_refine(int32_t ld, const double *__restrict__ gains, int level, AllocHead
         }
         if (new_hi != p_hi || p != p_end) rowstate[row] = make_int2(new_hi, p);
     }
-    if (closing) return;
     __syncthreads();
     flush_hist(s_hist, hist_all + (size_t)level * kBins, bins);
     if (last_block(&hdr->ticket[level]))
@@ -873,12 +1098,13 @@ exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ t
 
 // ---------------------------------------------------------------------------------------------------
 // Block sums of (p_hi, tied) in prompt order, and their exclusive scan by the last CTA.
-//   mode 0: rowstate is final    mode 2: apply the exact labels first
-// With `validate` the priors and counts of every prompt are checked here (a thread per row, coalesced).
+//   mode 0: first close every non-empty segment with the finished threshold    mode 2: apply the exact labels first
+// With `validate` the priors and counts of every prompt are checked here (only when level 1, which checks
+// them otherwise, did not run).
 __global__ void __launch_bounds__(kSelThreads)
 select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
            const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar, int validate,
-           int64_t N, int32_t ld, int mode, int64_t B, AllocHeader *hdr,
+           int64_t N, int32_t ld, const double *__restrict__ gains, int mode, int64_t B, AllocHeader *hdr,
            int2 *__restrict__ rowstate, const int32_t *__restrict__ rowslot, const int32_t *__restrict__ tlabel,
            long long *bsum_hi, long long *bsum_t, int64_t NB) {
     __shared__ long long s_warp[kSelThreads / kWarp];
@@ -886,21 +1112,45 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
     long long hi_sum = 0, t_sum = 0;
     if (!failed) {
         const int64_t row0 = (int64_t)blockIdx.x * kRowsPerBlock;
+        constexpr int kPer = kRowsPerBlock / kSelThreads;
+        int2 st[kPer];
+        int32_t slot[kPer];
+        bool ok = true;
 #pragma unroll
-        for (int q = 0; q < kRowsPerBlock / kSelThreads; ++q) {
+        for (int q = 0; q < kPer; ++q) {                      // every load of the thread is issued before any is used
             const int64_t row = row0 + q * kSelThreads + threadIdx.x;
-            if (row >= N) break;
-            if (validate && !load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row).ok)
-                raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);   // seen by the kernels that follow
-            int2 st = rowstate[row];
-            if (mode == 2) {
-                const int32_t slot = rowslot[row];
-                const int label = slot >= 0 ? tlabel[slot] : 0;
-                st = make_int2(st.x + (label == 2), st.x + (label == 2) + (label == 1));
-                rowstate[row] = st;
+            const int64_t rr = row < N ? row : N - 1;
+            st[q] = rowstate[rr];
+            slot[q] = mode == 2 ? rowslot[rr] : -1;
+            if (validate) ok &= load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, rr).ok;
+        }
+        if (!ok) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);   // seen by the kernels that follow
+        const unsigned long long lam = hdr->prefix_key;       // the threshold, once all 64 bits are resolved
+#pragma unroll
+        for (int q = 0; q < kPer; ++q) {
+            const int64_t row = row0 + q * kSelThreads + threadIdx.x;
+            if (row < N) {
+                if (mode == 0 && st[q].y > st[q].x) {         // close the segment: keys above / equal to the threshold
+                    const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+                    int32_t n_gt = 0, n_eq = 0;
+                    for (int32_t pp = st[q].x; pp < st[q].y; ++pp) {
+                        const unsigned long long key = __ldg(keys + pp);
+                        if (key > lam) ++n_gt;
+                        else if (key == lam) ++n_eq;
+                        else break;
+                    }
+                    const int2 fin = make_int2(st[q].x + n_gt, st[q].x + n_gt + n_eq);
+                    if (fin.x != st[q].x || fin.y != st[q].y) rowstate[row] = fin;
+                    st[q] = fin;
+                }
+                if (mode == 2) {
+                    const int label = slot[q] >= 0 ? tlabel[slot[q]] : 0;
+                    st[q] = make_int2(st[q].x + (label == 2), st[q].x + (label == 2) + (label == 1));
+                    rowstate[row] = st[q];
+                }
+                hi_sum += st[q].x;
+                t_sum += st[q].y - st[q].x;
             }
-            hi_sum += st.x;
-            t_sum += st.y - st.x;
         }
     }
     long long tot_hi, tot_t;
@@ -910,13 +1160,26 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
     if (last_block(&hdr->ticket[8 + mode])) {
         // exclusive scan of NB block sums, kSelThreads at a time, in index order
         long long run_hi = 0, run_t = 0;
-        for (int64_t b0 = 0; b0 < NB; b0 += kSelThreads) {
-            const int64_t b = b0 + threadIdx.x;
-            const long long vh = b < NB ? __ldcg(bsum_hi + b) : 0, vt = b < NB ? __ldcg(bsum_t + b) : 0;
+        constexpr int kRun = 4;                                 // consecutive block sums per thread
+        for (int64_t b0 = 0; b0 < NB; b0 += kRun * kSelThreads) {
+            const int64_t b = b0 + (int64_t)threadIdx.x * kRun;
+            long long vh[kRun], vt[kRun], sh = 0, st = 0;
+#pragma unroll
+            for (int u = 0; u < kRun; ++u) {
+                vh[u] = b + u < NB ? __ldcg(bsum_hi + b + u) : 0;
+                vt[u] = b + u < NB ? __ldcg(bsum_t + b + u) : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < kRun; ++u) { sh += vh[u]; st += vt[u]; }
             long long th, tt;
-            const long long eh = block_exclusive_sum(vh, &th, s_warp);
-            const long long et = block_exclusive_sum(vt, &tt, s_warp);
-            if (b < NB) { bsum_hi[b] = run_hi + eh; bsum_t[b] = run_t + et; }
+            long long eh = run_hi + block_exclusive_sum(sh, &th, s_warp);
+            long long et = run_t + block_exclusive_sum(st, &tt, s_warp);
+#pragma unroll
+            for (int u = 0; u < kRun; ++u) {
+                if (b + u < NB) { bsum_hi[b + u] = eh; bsum_t[b + u] = et; }
+                eh += vh[u];
+                et += vt[u];
+            }
             run_hi += th;
             run_t += tt;
         }
@@ -933,8 +1196,8 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
 __global__ void __launch_bounds__(kSelThreads)
 select_out(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
            const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N,
-           int32_t ld, int64_t B, uint32_t flags, AllocHeader *hdr, const int2 *__restrict__ rowstate,
-           const long long *__restrict__ bpre_hi, const long long *__restrict__ bpre_t, double *objpart, int64_t NB,
+           int32_t ld, const double *__restrict__ gains, int64_t B, uint32_t flags, AllocHeader *hdr,
+           const int2 *__restrict__ rowstate, const long long *__restrict__ bpre_hi, const long long *__restrict__ bpre_t, double *objpart, int64_t NB,
            int32_t *__restrict__ delta, int32_t *__restrict__ G, int64_t *__restrict__ offsets,
            hora_alloc_info *info) {
     __shared__ long long s_warp[kSelThreads / kWarp];
@@ -966,23 +1229,39 @@ select_out(const double *__restrict__ alpha, const double *__restrict__ beta, do
         pre_t += bpre_t[blockIdx.x];
     }
     const long long R = failed ? 0 : hdr->R;
+    int32_t d[kPer];
 #pragma unroll
     for (int q = 0; q < kPer; ++q) {
         const int64_t row = row0 + q;
+        d[q] = 0;
         if (row < N) {
             long long take = R - pre_t;
             take = take < 0 ? 0 : (take > tied[q] ? tied[q] : take);
-            const int32_t d = failed ? 0 : hi[q] + (int32_t)take;
-            delta[row] = d;
-            G[row] = failed ? 0 : G0 + d;
+            d[q] = failed ? 0 : hi[q] + (int32_t)take;
+            delta[row] = d[q];
+            G[row] = failed ? 0 : G0 + d[q];
             if (offsets) offsets[row] = failed ? 0 : row * (int64_t)G0 + pre_hi + (pre_t < R ? pre_t : R);
-            if (!failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE) && d > 0) {
-                const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row);
-                obj += hit_utility(p.a, p.b, d);
-            }
             pre_hi += hi[q];
             pre_t += tied[q];
         }
+    }
+    // Objective.  The product in U_i(Delta) = 1 - prod_{j<Delta} (b+j)/(a+b+j) is the row's own entry
+    // g_i(Delta) times (b + Delta - 1) / a  (Eq. marginal), so one load replaces Delta multiplications.
+    if (!failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE)) {
+        double g[kPer], pa[kPer], pb[kPer];
+#pragma unroll
+        for (int q = 0; q < kPer; ++q) {                      // all loads first
+            const int64_t row = row0 + q;
+            const bool use = row < N && d[q] > 0;
+            const int64_t rr = use ? row : 0;
+            const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, rr);
+            pa[q] = p.a;
+            pb[q] = p.b;
+            g[q] = use ? __ldg(gains + rr * (int64_t)ld + (d[q] - 1)) : 0.0;
+        }
+#pragma unroll
+        for (int q = 0; q < kPer; ++q)
+            if (row0 + q < N && d[q] > 0) obj += 1.0 - g[q] * (pb[q] + (double)(d[q] - 1)) / pa[q];
     }
     if (offsets && blockIdx.x == gridDim.x - 1 && threadIdx.x == kSelThreads - 1)
         offsets[N] = failed ? 0 : N * (int64_t)G0 + B;
@@ -1037,8 +1316,16 @@ __global__ void write_empty(int64_t B, int64_t *offsets, hora_alloc_info *info) 
     }
 }
 
-// Optional profiling aid (see hora_allocate_profile_events): events recorded around the full-read pass.
+// Optional profiling aids (see hora_allocate_profile_events / hora_allocate_profile_stages): events recorded
+// around the full-read pass, and after each stage of the call.
 static std::atomic<cudaEvent_t> g_prof_start{nullptr}, g_prof_stop{nullptr};
+constexpr int kStageEvents = 7;
+static std::atomic<cudaEvent_t> g_stage_ev[kStageEvents];
+
+static inline void mark_stage(int k, cudaStream_t s) {
+    const cudaEvent_t ev = g_stage_ev[k].load(std::memory_order_relaxed);
+    if (ev != nullptr) cudaEventRecord(ev, s);
+}
 
 template <int E>
 static void launch_level0(bool vec2, int grid, cudaStream_t s, const int32_t *cap, int32_t cap_scalar, int64_t N,
@@ -1076,6 +1363,12 @@ static cudaError_t launch_fused(bool vec2, bool estimate, int grid_est, int64_t 
 extern "C" void hora_allocate_profile_events(void *start_event, void *stop_event) {
     hora::g_prof_start.store(static_cast<cudaEvent_t>(start_event), std::memory_order_relaxed);
     hora::g_prof_stop.store(static_cast<cudaEvent_t>(stop_event), std::memory_order_relaxed);
+}
+
+extern "C" void hora_allocate_profile_stages(void *const *events_host, int32_t n) {
+    for (int k = 0; k < hora::kStageEvents; ++k)
+        hora::g_stage_ev[k].store(events_host != nullptr && k < n ? static_cast<cudaEvent_t>(events_host[k]) : nullptr,
+                                  std::memory_order_relaxed);
 }
 
 extern "C" size_t hora_allocate_workspace_bytes(int64_t N, int32_t ld, int32_t gains_is_null, uint32_t flags) {
@@ -1123,12 +1416,14 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     const int64_t every = (N + kSampleRows - 1) / kSampleRows;
     const int64_t n_sample = (N + every - 1) / every;
     const int grid_est = clamp_grid((n_sample + rows_per_cta - 1) / rows_per_cta, 4);
+    mark_stage(0, s);
     if (B > 0 && !fused)
         select_estimate<<<grid_est, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, every, gains, B, w.hdr, w.hist_est);
     const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 4);
     const int grid1 = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     const cudaEvent_t prof_start = g_prof_start.load(std::memory_order_relaxed);
     const cudaEvent_t prof_stop = g_prof_stop.load(std::memory_order_relaxed);
+    if (!fused) mark_stage(1, s);                         // (the fused pass launches its own estimate)
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_start, s);
     if (fused) {
         const int gridf = clamp_grid((N + kCtaRows - 1) / kCtaRows, 3);
@@ -1148,30 +1443,42 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         launch_level0<2>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
     }
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_stop, s);
+    mark_stage(2, s);
     const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     if (B > 0) {
-        select_level1<<<grid1, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, w.hdr, w.hist_lv + kBins, w.sketch,
-                                                    w.sk_ld, w.rowstate, w.active);
-        for (int level = 2; level <= kLevels; ++level)     // levels 2..4, then the closing pass
+        if (vec2)
+            select_level1<true><<<grid1, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains,
+                                                              w.hdr, w.hist_lv + kBins, w.sketch, w.sk_ld, w.rowstate,
+                                                              w.active, w.cand_key);
+        else
+            select_level1<false><<<grid1, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains,
+                                                               w.hdr, w.hist_lv + kBins, w.sketch, w.sk_ld, w.rowstate,
+                                                               w.active, w.cand_key);
+        mark_stage(3, s);
+        select_list<<<1, kListThreads, 0, s>>>(w.hdr, w.hist_lv + kBins, w.cand_key);
+        for (int level = 2; level < kLevels; ++level)      // levels 2..4: stand down at once in list mode
             select_refine<<<2 * kSmCount, kSelThreads, 0, s>>>(ld, gains, level, w.hdr, w.hist_lv, w.rowstate, w.active);
-        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 1, N, ld, 0, B, w.hdr,
-                                                   w.rowstate, nullptr, nullptr, w.bsum_hi, w.bsum_t, NB);
+        mark_stage(4, s);
+        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 0, N, ld, gains, 0, B,
+                                                   w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi, w.bsum_t, NB);
         if (exact) {
             exact_collect<<<grid_rows, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
                                                             gains, w.hdr, w.rowstate, w.rowslot, w.tkeys, w.tcounts);
             exact_rank<<<1, 1024, 0, s>>>(B, w.hdr, w.tkeys, w.tcounts, w.tlabel);
-            select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 0, N, ld, 2, B,
+            select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 0, N, ld, gains, 2, B,
                                                        w.hdr, w.rowstate, w.rowslot, w.tlabel, w.bsum_hi, w.bsum_t, NB);
         }
     } else {
         if (cudaMemsetAsync(w.rowstate, 0, sizeof(int2) * (size_t)N, s) != cudaSuccess) return HORA_ERR_CUDA;
-        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 1, N, ld, 0, B, w.hdr,
-                                                   w.rowstate, nullptr, nullptr, w.bsum_hi, w.bsum_t, NB);
+        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 1, N, ld, gains, 0, B,
+                                                   w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi, w.bsum_t, NB);
     }
-    select_out<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, flags, w.hdr,
+    mark_stage(5, s);
+    select_out<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, flags, w.hdr,
                                                w.rowstate, w.bsum_hi, w.bsum_t, w.objpart, NB, delta, G, group_offsets,
                                                info_dev);
-    count_launches(B > 0 ? (exact ? 13 : 10) : 3);
+    mark_stage(6, s);
+    count_launches(B > 0 ? (exact ? 12 : 9) : 3);
     return cuda_ok(cudaGetLastError());
 }
 

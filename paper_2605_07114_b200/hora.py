@@ -24,7 +24,7 @@ WEIGHT_PER_TOKEN, WEIGHT_CONST_LENGTH = 0, 1
 
 EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora_group_advantage",
            "hora_token_broadcast", "hora_status_string", "hora_version", "hora_launch_count",
-           "hora_allocate_static", "hora_allocate_static_capacity", "hora_allocate_profile_events",
+           "hora_allocate_static", "hora_allocate_static_capacity", "hora_allocate_profile_events", "hora_allocate_profile_stages",
            "hora_allocate_batched", "hora_allocate_batched_workspace_bytes", "hora_rollout_weights",
            "hora_learned_prior", "hora_beta_binomial_nll", "hora_pass_at_k", "hora_pass_at_k_workspace_bytes",
            "hora_group_advantage_tokens", "hora_allocation_share")
@@ -71,6 +71,8 @@ def load() -> C.CDLL:
     L.hora_allocate_batched.restype = C.c_int
     L.hora_allocate_profile_events.argtypes = [p, p]
     L.hora_allocate_profile_events.restype = None
+    L.hora_allocate_profile_stages.argtypes = [C.POINTER(C.c_void_p), C.c_int32]
+    L.hora_allocate_profile_stages.restype = None
     L.hora_group_advantage.argtypes = [p, p, i64, i32, C.c_float, i32, p, p, p]
     L.hora_group_advantage.restype = C.c_int
     L.hora_group_advantage_tokens.argtypes = [p, p, i64, p, i64, i64, i32, C.c_float, i32, i32, C.c_float, p, p, p, p]
@@ -194,6 +196,16 @@ def hora_allocate_profile_events(start_event, stop_event):
     selection kernel of every following hora_allocate call."""
     load().hora_allocate_profile_events(None if start_event is None else C.c_void_p(int(start_event)),
                                         None if stop_event is None else C.c_void_p(int(stop_event)))
+
+
+def hora_allocate_profile_stages(events):
+    """Record the given events (raw cudaEvent_t handles as ints; at most 7; None or empty to switch off) at the
+    stage boundaries of every following hora_allocate call."""
+    if not events:
+        load().hora_allocate_profile_stages(None, 0)
+        return
+    arr = (C.c_void_p * len(events))(*[C.c_void_p(int(e)) if e is not None else None for e in events])
+    load().hora_allocate_profile_stages(arr, len(events))
 
 
 def hora_allocate_static_capacity() -> int:
