@@ -3,19 +3,20 @@
 // A warp takes 32 consecutive groups at a time; lane i reads group i's two offsets (one coalesced load)
 // and owns that group's statistics, so the per-group scalar work (mean, variance, square root,
 // reciprocal — fp64) is done once per group by one lane.  The rewards of those groups are one contiguous
-// run of memory.  As many whole groups as fit 1536 elements form a batch; a lane loads the batch as up to
-// twelve 16-byte pieces (all in flight together: that is what hides DRAM latency here) and KEEPS them in
-// registers, 128 elements of the batch per "row" of the warp, regardless of where the group boundaries fall:
-//   statistics  per row four ballots (which rewards are 1.0) give every lane the number of ones before its
-//               four elements; that count and the lane's own four bits go to shared memory as one word,
+// run of memory.  As many whole groups as fit 1536 elements form a batch, staged in a per-warp shared-memory
+// slab by asynchronous 16-byte copies (up to twelve per lane, all in flight together: that is what hides DRAM
+// latency here) and handled in "rows" of 128 elements, a lane four consecutive elements of each row,
+// regardless of where the group boundaries fall:
+//   statistics  a warp scan (shared by four rows, one byte each) gives every lane the number of ones before
+//               its four elements; that count and the lane's own four bits go to shared memory as one word,
 //               so lane i gets its group's number of ones from two lookups, at its start and end offsets.
 //               A group of 0/1 rewards (the verifiable-reward case) is finished there: sum = k,
 //               sum (r - m)^2 = k (n - k) / n exactly, and its two possible advantages — of a 0 and of a 1 —
 //               are computed once, in fp64, rounded to fp32 once.
 //   output      a bitmap of group starts with running counts maps every element to its group; the element
 //               picks one of its group's two values; 16-byte stores.
-// If any reward of the batch is neither 0.0 nor 1.0 the batch takes the general route instead: the rows go
-// to a shared-memory slab, each group is summed in fp64 by the whole warp (fixed butterfly), its squared
+// If any reward of the batch is neither 0.0 nor 1.0 the batch takes the general route instead: each group
+// is summed in fp64 by the whole warp (fixed butterfly), its squared
 // deviations taken in a second sweep (the two-pass form), and every element evaluated as
 // adv = (r - mean) * scale in fp64, scale = 1 / (std + eps) for GRPO, n / (n - 1) for RLOO
 // (r - (S - r)/(n-1) = (r - S/n) n/(n-1)); for a 0/1 group both routes perform the same operations.
@@ -32,7 +33,7 @@ constexpr int kSlab = kRows * 128;                            // 1536 elements
 constexpr unsigned kOne = 0x3F800000u;                        // bit pattern of 1.0f
 
 struct __align__(16) AdvWarpSmem {
-    float buf[kSlab];                                         // general route only
+    float buf[kSlab];                                         // the staged batch
     unsigned int pre[kSlab / 4 + 4];                          // per 4 elements: (ones before them << 4) | their own bits
     unsigned int starts[kSlab / 32];                          // one bit per element: a non-empty group starts here
     int cum_starts[kSlab / 32];                               // exclusive running counts per word
@@ -74,10 +75,22 @@ __device__ __forceinline__ int ones_before(const unsigned int *pre, int pos) {
     return (int)(w >> 4) + __popc(w & ((1u << (pos & 3)) - 1u));
 }
 
-// VEC4: rewards and adv are 16-byte aligned, so a batch is read and written in 16-byte pieces starting at
+// Asynchronous 16-byte global -> shared copy (the data does not pass through registers or L1).
+__device__ __forceinline__ void cp_async_16(float *smem_dst, const float *gmem_src) {
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// group (in the order of the batch's non-empty groups) of element el, through the start bitmap
+__device__ __forceinline__ int rank_of(const AdvWarpSmem &sm, int el) {
+    return sm.cum_starts[el >> 5] + __popc(sm.starts[el >> 5] & (0xFFFFFFFFu >> (31 - (el & 31)))) - 1;
+}
+
+// VEC4: rewards and adv are 16-byte aligned, so a batch is staged and written in 16-byte pieces starting at
 // the 4-element boundary at or below its first element.
 template <bool VEC4>
-__global__ void __launch_bounds__(kAdvWarps *kWarp, 2)
+__global__ void __launch_bounds__(kAdvWarps *kWarp, 3)
 group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restrict__ off, int64_t N, int32_t mode,
                        double eps, int32_t ddof, float *__restrict__ adv, int32_t *status_dev) {
     extern __shared__ __align__(16) unsigned char s_raw[];
@@ -123,52 +136,65 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
             if (span == lead) { done += nfit; continue; }     // only empty groups
             const int my_rs = mine ? (int)(my_s - start) : 0, my_re = mine ? (int)rel_end : 0;
             const int n_rows = (span + 127) >> 7;
-            // ---- load: every piece of the batch in flight at once, then held in registers ----
-            float4 v[kRows];
-#pragma unroll
-            for (int j = 0; j < kRows; ++j) {
-                v[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                const int e0 = 128 * j + 4 * lane;
-                if (j < n_rows && e0 < span) {
-                    const int64_t e = start + e0;
-                    if (VEC4 && e + 4 <= n_all) {
-                        v[j] = __ldg(reinterpret_cast<const float4 *>(rewards + e));
-                    } else {
-                        if (e < n_all) v[j].x = __ldg(rewards + e);
-                        if (e + 1 < n_all) v[j].y = __ldg(rewards + e + 1);
-                        if (e + 2 < n_all) v[j].z = __ldg(rewards + e + 2);
-                        if (e + 3 < n_all) v[j].w = __ldg(rewards + e + 3);
-                    }
+            // ---- stage: every piece of the batch in flight at once; pieces past the batch read as zeros ----
+            const bool tail = start + 128 * (int64_t)n_rows > n_all;   // the last pieces may cross the end of the array
+            if (VEC4 && !tail) {
+                const float *src = rewards + start + 4 * lane;
+                for (int j = 0; j < n_rows; ++j) {
+                    if (128 * j + 4 * lane < span) cp_async_16(&sm.buf[128 * j + 4 * lane], src + 128 * j);
+                    else *reinterpret_cast<float4 *>(&sm.buf[128 * j + 4 * lane]) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                 }
+                cp_async_wait_all();
+            } else {
+                for (int j = lane; j < 128 * n_rows; j += kWarp)
+                    sm.buf[j] = (j < span && start + j < n_all) ? __ldg(rewards + start + j) : 0.0f;
             }
+            __syncwarp();
             // ---- which rewards are 1.0 (packed prefix words); is anything neither 0.0 nor 1.0? ----
+            // A lane takes four consecutive elements of each 128-element row.  Four rows share one warp scan:
+            // their per-lane counts (at most 4 each, 128 per row) sit in the four bytes of a word.
+            // r (r - 1) is +0.0 exactly for r = 0.0 and r = 1.0 and for nothing else.
             unsigned other = 0;
             int carry = 0;
+            for (int j0 = 0; j0 < n_rows; j0 += 4) {
+                unsigned own[4], packed = 0;
 #pragma unroll
-            for (int j = 0; j < kRows; ++j) {
-                if (j < n_rows) {
-                    const unsigned ux = __float_as_uint(v[j].x), uy = __float_as_uint(v[j].y);
-                    const unsigned uz = __float_as_uint(v[j].z), uw = __float_as_uint(v[j].w);
-                    other |= min(ux, ux ^ kOne) | min(uy, uy ^ kOne) | min(uz, uz ^ kOne) | min(uw, uw ^ kOne);
-                    const unsigned bx = __ballot_sync(kFull, ux == kOne), by = __ballot_sync(kFull, uy == kOne);
-                    const unsigned bz = __ballot_sync(kFull, uz == kOne), bw = __ballot_sync(kFull, uw == kOne);
-                    const int before = carry + __popc(bx & lt) + __popc(by & lt) + __popc(bz & lt) + __popc(bw & lt);
-                    const unsigned own = (ux == kOne ? 1u : 0u) | (uy == kOne ? 2u : 0u) | (uz == kOne ? 4u : 0u) |
-                                         (uw == kOne ? 8u : 0u);
-                    sm.pre[32 * j + lane] = ((unsigned)before << 4) | own;
-                    carry += __popc(bx) + __popc(by) + __popc(bz) + __popc(bw);
+                for (int q = 0; q < 4; ++q) {
+                    own[q] = 0;
+                    if (j0 + q < n_rows) {
+                        const float4 x = *reinterpret_cast<const float4 *>(&sm.buf[128 * (j0 + q) + 4 * lane]);
+                        other |= __float_as_uint(fmaf(x.x, x.x, -x.x)) | __float_as_uint(fmaf(x.y, x.y, -x.y)) |
+                                 __float_as_uint(fmaf(x.z, x.z, -x.z)) | __float_as_uint(fmaf(x.w, x.w, -x.w));
+                        own[q] = (x.x == 1.0f ? 1u : 0u) | (x.y == 1.0f ? 2u : 0u) | (x.z == 1.0f ? 4u : 0u) |
+                                 (x.w == 1.0f ? 8u : 0u);
+                    }
+                    packed |= (unsigned)__popc(own[q]) << (8 * q);
+                }
+                unsigned inc = packed;
+#pragma unroll
+                for (int d = 1; d < kWarp; d <<= 1) {
+                    const unsigned t = __shfl_up_sync(kFull, inc, d);
+                    if (lane >= d) inc += t;
+                }
+                const unsigned excl = inc - packed;            // byte-wise: no byte ever borrows
+                const unsigned tot = __shfl_sync(kFull, inc, kWarp - 1);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (j0 + q < n_rows)
+                        sm.pre[32 * (j0 + q) + lane] = ((unsigned)(carry + (int)((excl >> (8 * q)) & 0xFFu)) << 4) | own[q];
+                    carry += (int)((tot >> (8 * q)) & 0xFFu);
                 }
             }
             if (lane == 0) sm.pre[32 * n_rows] = (unsigned)carry << 4;
             const bool general = __any_sync(kFull, other != 0u);
             // ---- group starts (non-empty groups only: they have distinct starts) and their order ----
-            for (int w = lane; w < kSlab / 32; w += kWarp) sm.starts[w] = 0u;
+            for (int w = lane; w < 4 * n_rows; w += kWarp) sm.starts[w] = 0u;
             __syncwarp();
             const bool nonempty = mine && my_re > my_rs;
             if (nonempty) atomicOr(&sm.starts[my_rs >> 5], 1u << (my_rs & 31));
             const int my_rank = __popc(__ballot_sync(kFull, nonempty) & lt);
             __syncwarp();
-            running_counts(sm.starts, sm.cum_starts, n_rows * 4, lane);
+            running_counts(sm.starts, sm.cum_starts, 4 * n_rows, lane);
             __syncwarp();
             const double dn = (double)my_n;
             if (!general) {
@@ -179,42 +205,39 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
                 const double scale = group_scale(mode, ss, my_n, ddof, eps);
                 if (nonempty) sm.two[my_rank] = make_float2((float)((0.0 - mean) * scale), (float)((1.0 - mean) * scale));
                 __syncwarp();
-                // ---- output: element -> group through the start bitmap ----
-#pragma unroll
-                for (int j = 0; j < kRows; ++j) {
+                // ---- output: element -> group through the start bitmap; whole 16-byte pieces here ----
+                float *dst4 = adv + start + 4 * lane;
+                for (int j = 0; j < n_rows; ++j) {
                     const int e0 = 128 * j + 4 * lane;
-                    if (j < n_rows && e0 < span) {
+                    if (VEC4 && e0 >= lead && e0 + 4 <= span) {
+                        const float4 x = *reinterpret_cast<const float4 *>(&sm.buf[e0]);
                         const int bit = e0 & 31;
-                        const unsigned sw = sm.starts[e0 >> 5];
-                        const int r0 = sm.cum_starts[e0 >> 5] + __popc(sw & (0xFFFFFFFFu >> (31 - bit))) - 1;
-                        const int r1 = r0 + (int)((sw >> (bit + 1)) & 1u);
-                        const int r2 = r1 + (int)((sw >> (bit + 2)) & 1u);
-                        const int r3 = r2 + (int)((sw >> (bit + 3)) & 1u);
-                        // rank -1: an element before the batch's first group, loaded but never stored
-                        const float2 a0 = sm.two[max(r0, 0)], a1 = sm.two[max(r1, 0)], a2 = sm.two[max(r2, 0)],
-                                     a3 = sm.two[r3];
+                        const unsigned word = sm.starts[e0 >> 5], sw = word >> bit;
+                        const int r0 = sm.cum_starts[e0 >> 5] + __popc(word & (0xFFFFFFFFu >> (31 - bit))) - 1;
+                        const int r1 = r0 + (int)((sw >> 1) & 1u);
+                        const int r2 = r1 + (int)((sw >> 2) & 1u);
+                        const int r3 = r2 + (int)((sw >> 3) & 1u);
+                        const float2 a0 = sm.two[r0], a1 = sm.two[r1], a2 = sm.two[r2], a3 = sm.two[r3];
                         float4 o;
-                        o.x = __float_as_uint(v[j].x) == kOne ? a0.y : a0.x;
-                        o.y = __float_as_uint(v[j].y) == kOne ? a1.y : a1.x;
-                        o.z = __float_as_uint(v[j].z) == kOne ? a2.y : a2.x;
-                        o.w = __float_as_uint(v[j].w) == kOne ? a3.y : a3.x;
-                        float *dst = adv + start + e0;
-                        if (VEC4 && e0 >= lead && e0 + 4 <= span) {
-                            *reinterpret_cast<float4 *>(dst) = o;
-                        } else {
-                            if (e0 >= lead && e0 < span) dst[0] = o.x;
-                            if (e0 + 1 >= lead && e0 + 1 < span) dst[1] = o.y;
-                            if (e0 + 2 >= lead && e0 + 2 < span) dst[2] = o.z;
-                            if (e0 + 3 >= lead && e0 + 3 < span) dst[3] = o.w;
-                        }
+                        o.x = x.x == 1.0f ? a0.y : a0.x;
+                        o.y = x.y == 1.0f ? a1.y : a1.x;
+                        o.z = x.z == 1.0f ? a2.y : a2.x;
+                        o.w = x.w == 1.0f ? a3.y : a3.x;
+                        *reinterpret_cast<float4 *>(dst4 + 128 * j) = o;
                     }
                 }
+                // ragged ends (at most 3 elements after `lead` and 3 before `span`; everything when the pointers
+                // are not 16-byte aligned): one element per lane and step
+                const int head_end = VEC4 ? min(span, (lead + 3) & ~3) : span;
+                const int tail_beg = VEC4 ? max(head_end, span & ~3) : span;
+                const int n_rag = (head_end - lead) + (span - tail_beg);
+                for (int i = lane; i < n_rag; i += kWarp) {
+                    const int el = i < head_end - lead ? lead + i : tail_beg + (i - (head_end - lead));
+                    const float2 a = sm.two[rank_of(sm, el)];
+                    adv[start + el] = sm.buf[el] == 1.0f ? a.y : a.x;
+                }
             } else {
-                // ---- general route: rows to the slab, whole-warp two-pass sums per group ----
-#pragma unroll
-                for (int j = 0; j < kRows; ++j)
-                    if (j < n_rows) *reinterpret_cast<float4 *>(&sm.buf[128 * j + 4 * lane]) = v[j];
-                __syncwarp();
+                // ---- general route: whole-warp two-pass sums per group over the slab ----
                 double my_mean = 0.0, my_ss = 0.0;
                 for (int i = done; i <= last; ++i) {
                     const int s = __shfl_sync(kFull, my_rs, i), e = __shfl_sync(kFull, my_re, i);
@@ -238,21 +261,9 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
                     sm.scale[my_rank] = group_scale(mode, my_ss, my_n, ddof, eps);
                 }
                 __syncwarp();
-#pragma unroll
-                for (int j = 0; j < kRows; ++j) {
-                    const int e0 = 128 * j + 4 * lane;
-                    if (j < n_rows && e0 < span) {
-                        const float val[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const int el = e0 + q;
-                            if (el >= lead && el < span) {
-                                const int r = sm.cum_starts[el >> 5] +
-                                              __popc(sm.starts[el >> 5] & (0xFFFFFFFFu >> (31 - (el & 31)))) - 1;
-                                adv[start + el] = (float)(((double)val[q] - sm.mean[r]) * sm.scale[r]);
-                            }
-                        }
-                    }
+                for (int el = lead + lane; el < span; el += kWarp) {
+                    const int r = rank_of(sm, el);
+                    adv[start + el] = (float)(((double)sm.buf[el] - sm.mean[r]) * sm.scale[r]);
                 }
             }
             __syncwarp();
@@ -273,7 +284,7 @@ extern "C" hora_status_t hora_group_advantage(const float *rewards, const int64_
     if (group_offsets == nullptr || rewards == nullptr || adv == nullptr) return HORA_ERR_INVALID_ARG;
     const bool vec4 = ((reinterpret_cast<uintptr_t>(rewards) | reinterpret_cast<uintptr_t>(adv)) & 15u) == 0;
     const int64_t n_blocks = (N + kWarp - 1) / kWarp;
-    const int grid = clamp_grid((n_blocks + kAdvWarps - 1) / kAdvWarps, 2);
+    const int grid = clamp_grid((n_blocks + kAdvWarps - 1) / kAdvWarps, 3);
     auto go = [&](auto kernel) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAdvSmem);
         if (e != cudaSuccess) return e;

@@ -6,10 +6,9 @@
 // block-wide k-ary search over the CSR offsets, then works in rounds: it stages the next kStage
 // rollouts in shared memory — offsets as 32-bit distances from the chunk start, advantages as they
 // are — and writes every token those rollouts cover.  Tokens are visited in 128-token windows on an
-// absolute 128-aligned grid, one window per warp per step, one 16-byte st.global.cs per lane.  A
-// warp keeps a forward-only rollout cursor; when the whole window lies inside one rollout (the
-// usual case for responses of tens to thousands of tokens) the lanes store one broadcast value and
-// never look at the offsets.  Cost per token does not depend on the length mix; the only global
+// absolute 128-aligned grid, one 16-byte st.global.cs per lane and window; a warp takes a contiguous run
+// of windows, so while it is inside one rollout (the usual case for responses of tens to thousands of
+// tokens) it stores one broadcast value window after window and never looks at the offsets.  Cost per token does not depend on the length mix; the only global
 // reads are 8 B of offset and 4 B of advantage per rollout.
 #include "hora_broadcast.cuh"
 

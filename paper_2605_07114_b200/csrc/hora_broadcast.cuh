@@ -35,24 +35,47 @@ static __device__ int64_t block_find_rollout(const int64_t *__restrict__ off, in
 }
 
 // Writes s_val[j] over the tokens of staged rollout j, for the chunk-relative tokens [t, t_end) (t_end =
-// s_rel[n_stage]).  Tokens are visited in 128-token windows on an absolute 128-aligned grid, one window per warp
-// per step; a window that lies inside one rollout is one broadcast 16-byte store per lane.
+// s_rel[n_stage]).  Tokens are visited in 128-token windows on an absolute 128-aligned grid; each warp takes a
+// contiguous run of windows, so that it stays inside one rollout for many windows in a row: there the loop is
+// one broadcast 16-byte store per lane and window and nothing else.  Only the window in which a rollout ends
+// walks the offsets.
 template <bool VEC4>
 __device__ __forceinline__ void write_staged(const int32_t *s_rel, const float *s_val, int n_stage, int32_t t,
                                              int32_t t_end, int warp, int lane, float *__restrict__ dst) {
-    int cur = 0;                                    // warp-uniform, forward only: s_rel[cur] <= window start
-    for (int32_t w0 = (t & ~(kWarpTokens - 1)) + warp * kWarpTokens; w0 < t_end; w0 += kStepTokens) {
+    const int32_t first = t & ~(kWarpTokens - 1);
+    const int32_t n_win = (t_end - first + kWarpTokens - 1) / kWarpTokens;
+    const int32_t share = (n_win + kBcWarps - 1) / kBcWarps;
+    int32_t w0 = first + warp * share * kWarpTokens;
+    int32_t w_end = w0 + share * kWarpTokens;                    // end of this warp's run of windows
+    if (w_end > first + n_win * kWarpTokens) w_end = first + n_win * kWarpTokens;
+    if (w0 >= w_end) return;
+    int cur = 0;                                                 // warp-uniform: largest j with s_rel[j] <= w0 (else 0)
+    for (int lo = 0, hi = n_stage - 1; lo <= hi;) {
+        const int mid = (lo + hi) >> 1;
+        if (s_rel[mid] <= w0) { cur = mid; lo = mid + 1; } else { hi = mid - 1; }
+    }
+    while (w0 < w_end) {
         while (cur + 1 < n_stage && s_rel[cur + 1] <= w0) ++cur;
-        const int32_t t0 = w0 + lane * 4;
-        if (w0 >= t && w0 + kWarpTokens <= t_end && s_rel[cur + 1] >= w0 + kWarpTokens) {
-            const float v = s_val[cur];             // the whole window lies inside rollout `cur`
-            if (VEC4) {
-                __stcs(reinterpret_cast<float4 *>(dst + t0), make_float4(v, v, v, v));
-            } else {
-                dst[t0] = v; dst[t0 + 1] = v; dst[t0 + 2] = v; dst[t0 + 3] = v;
+        // whole windows inside rollout `cur` (and inside [t, t_end)), starting at w0
+        int32_t stop = s_rel[cur + 1] < t_end ? s_rel[cur + 1] : t_end;
+        if (stop > w_end) stop = w_end;
+        int32_t n_full = (VEC4 && w0 >= t && stop > w0) ? (stop - w0) / kWarpTokens : 0;
+        if (n_full > 0) {
+            const float v = s_val[cur];
+            const float4 vv = make_float4(v, v, v, v);
+            float4 *p = reinterpret_cast<float4 *>(dst + w0) + lane;
+            w0 += n_full * kWarpTokens;
+            for (; n_full >= 4; n_full -= 4, p += 4 * (kWarpTokens / 4)) {
+                __stcs(p, vv);
+                __stcs(p + kWarpTokens / 4, vv);
+                __stcs(p + 2 * (kWarpTokens / 4), vv);
+                __stcs(p + 3 * (kWarpTokens / 4), vv);
             }
+            for (; n_full > 0; --n_full, p += kWarpTokens / 4) __stcs(p, vv);
             continue;
         }
+        // the window at w0 holds a rollout boundary, or an end of [t, t_end): every lane finds its own rollouts
+        const int32_t t0 = w0 + lane * 4;
         int r = cur;
         float v[4];
 #pragma unroll
@@ -67,6 +90,7 @@ __device__ __forceinline__ void write_staged(const int32_t *s_rel, const float *
             for (int q = 0; q < 4; ++q)
                 if (t0 + q >= t && t0 + q < t_end) dst[t0 + q] = v[q];
         }
+        w0 += kWarpTokens;
     }
 }
 
