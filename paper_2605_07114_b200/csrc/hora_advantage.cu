@@ -30,7 +30,6 @@ namespace hora {
 constexpr int kAdvWarps = 8;
 constexpr int kRows = 12;                                     // 128-element rows a batch may span
 constexpr int kSlab = kRows * 128;                            // 1536 elements
-constexpr unsigned kOne = 0x3F800000u;                        // bit pattern of 1.0f
 
 struct __align__(16) AdvWarpSmem {
     float buf[kSlab];                                         // the staged batch

@@ -105,10 +105,7 @@ extern "C" hora_status_t hora_group_advantage_tokens(const float *rewards, const
         return HORA_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(token_adv) & 3u) || (reinterpret_cast<uintptr_t>(token_weight) & 3u))
         return HORA_ERR_INVALID_ARG;
-    const int64_t max_ctas = (int64_t)kSmCount * 8;
-    int64_t chunk = (T + max_ctas - 1) / max_ctas;
-    chunk = (chunk + kStepTokens - 1) / kStepTokens * kStepTokens;
-    if (chunk > kMaxChunk) chunk = kMaxChunk;
+    const int64_t chunk = token_chunk(T);
     const int64_t grid = (T + chunk - 1) / chunk;
     if (grid > 0x7FFFFFFF) return HORA_ERR_INVALID_ARG;
     const bool vec4 = ((reinterpret_cast<uintptr_t>(token_adv) | reinterpret_cast<uintptr_t>(token_weight)) & 15u) == 0;

@@ -1,8 +1,8 @@
 // hora_token_broadcast: replicate each rollout's advantage over its tokens (Eq. grpo-objective: the
 // per-token advantage has no dependence on the token position).
 //
-// Output-centric streaming write.  The token axis is cut into one contiguous chunk per CTA (a
-// multiple of 1024 tokens).  A CTA locates the rollout that contains its first token with a
+// Output-centric streaming write.  The token axis is cut into contiguous chunks, one per CTA (a
+// multiple of 1024 tokens, at most 65536).  A CTA locates the rollout that contains its first token with a
 // block-wide k-ary search over the CSR offsets, then works in rounds: it stages the next kStage
 // rollouts in shared memory — offsets as 32-bit distances from the chunk start, advantages as they
 // are — and writes every token those rollouts cover.  Tokens are visited in 128-token windows on an
@@ -56,10 +56,7 @@ extern "C" hora_status_t hora_token_broadcast(const float *adv, const int64_t *t
     if (R == 0 || T == 0) return HORA_OK;
     if (adv == nullptr || token_offsets == nullptr || token_adv == nullptr) return HORA_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(token_adv) & 3u) return HORA_ERR_INVALID_ARG;
-    const int64_t max_ctas = (int64_t)kSmCount * 8;
-    int64_t chunk = (T + max_ctas - 1) / max_ctas;
-    chunk = (chunk + kStepTokens - 1) / kStepTokens * kStepTokens;
-    if (chunk > kMaxChunk) chunk = kMaxChunk;
+    const int64_t chunk = token_chunk(T);
     const int64_t grid = (T + chunk - 1) / chunk;
     if (grid > 0x7FFFFFFF) return HORA_ERR_INVALID_ARG;
     const bool vec4 = (reinterpret_cast<uintptr_t>(token_adv) & 15u) == 0;
