@@ -249,8 +249,8 @@ def run_ours(args):
     hora.hora_allocate_profile_stages(None)
     torch.cuda.synchronize()
     st = np.array([[evs[i].elapsed_time(evs[i + 1]) for i in range(6)] for evs in st_ev]).mean(axis=0)
-    alloc_stages = dict(zip(("estimate", "full_read_level0", "rows_level1", "threshold_list_or_digits",
-                             "closing_and_scan", "outputs"), (round(float(x), 4) for x in st)))
+    alloc_stages = dict(zip(("estimate", "full_read_level0", "rows_level1", "tail_threshold_and_scan",
+                             "exact_ranking", "outputs"), (round(float(x), 4) for x in st)))
 
     # ---- the same step with the fused call: hora_allocate builds the matrix itself and counts on the way ----
     fused_ms = None

@@ -326,8 +326,8 @@ void hora_allocate_profile_events(void *start_event, void *stop_event);
  * hora_allocate_profile_stages — measurement aid, no counterpart in the paper.  `events_host` is a HOST array of
  * n <= 7 cudaEvent_t handles (timing enabled); every following hora_allocate / hora_allocate_static call records
  * them on its stream at these points:  [0] entry (after the workspace is cleared), [1] after the sampled estimate,
- * [2] after the full-read pass, [3] after the per-row pass (level 1), [4] after the threshold is complete (list
- * selection, or the digit levels), [5] after the per-row closing and the block scan (and the exact tie ranking),
+ * [2] after the full-read pass, [3] after the per-row pass (level 1), [4] after the tail (threshold complete,
+ * prefixes over prompts formed), [5] after the exact tie ranking (right after [4] when that does not run),
  * [6] after the outputs are written.  Differences of consecutive events are the device times of the stages.
  * A NULL handle skips its point; NULL or n = 0 switches everything off (the default).  Process-wide host
  * setting; the array is read during this call only.

@@ -17,18 +17,21 @@
 //             bracket is read and the segment [p_hi, p_lo) stored.  The same pass validates the priors.
 //             What happens to the keys of the segments depends on how many there are (level 0 knows the
 //             exact count of keys with the resolved prefix):
-//   list      at most 65536 of them (the usual case after a window hit): level 1 appends them to a list
-//             and ONE CTA resolves the remaining bits over that list, with no further pass over rows.
-//   level 2-4 more than that (a missed window, or heavy ties): level 1 histograms the next 13 bits and
-//             lists the rows whose segment is not empty; a thread per listed row then narrows its segment
-//             by the digit just selected and histograms the next one, 13 bits at a time.
-//   sum       every non-empty segment is narrowed by the finished threshold: p_hi = #keys > lambda,
-//             p_lo - p_hi = #keys == lambda per row; block sums and their scan give n_above, n_tied and
-//             the exclusive prefixes over prompts.
-//   out       Delta_i = p_hi + (tied candidates of row i that fall within the first R = B - n_above tied
-//             candidates in prompt order); G_i, CSR offsets, objective.
+//   tail      ONE cooperative launch finishes the threshold and the prefixes over prompts:
+//     list    at most 65536 such keys (the usual case after a window hit): level 1 appended them to a list
+//             and accumulated per-block sums of its provisional counts; one CTA resolves the remaining bits
+//             over the list, corrects the block sums by the listed keys above / equal to the threshold and
+//             scans them.  No further pass over rows.
+//     digits  more than that (a missed window, or heavy ties): level 1 histogrammed the next 13 bits and
+//             listed the rows whose segment is not empty; all CTAs narrow the listed rows' segments digit by
+//             digit (13 bits at a time, a grid-wide barrier between levels), close them with the finished
+//             threshold, form the block sums and scan them.
+//   out       p_hi = #keys > lambda, tied = #keys == lambda per row (segments left open by the list route are
+//             closed here); Delta_i = p_hi + (tied candidates of row i that fall within the first
+//             R = B - n_above tied candidates in prompt order); G_i, CSR offsets, objective.
 //
-// No kernel waits on another CTA: every "last CTA" step uses an atomic ticket after a fence.
+// Outside the cooperative tail no kernel waits on another CTA: every "last CTA" step uses an atomic ticket
+// after a fence; inside it the only waits are the runtime's grid-wide barriers.
 //
 // Exact mode (integer priors).  After the fp64 selection, candidates within a relative band of 2^-30
 // around lambda (far wider than the fp64 evaluation error, far narrower than the gap between two
@@ -37,6 +40,8 @@
 // by 256-bit cross multiplication of num/den = a (b)_a / (b+Delta-1)_{a+1}  (or the equivalent
 // a (b)_{Delta-1} / (a+b)_Delta when that has fewer factors), and the threshold class is found by
 // walking the ranked types.  Rows are relabelled above / tied / below and the same sum/out steps run.
+#include <cooperative_groups.h>
+
 #include <atomic>
 
 #include "hora_common.cuh"
@@ -47,14 +52,15 @@ namespace hora {
 
 constexpr int kLevels = 5;                   // level 0 (full read) + four digit levels
 constexpr int kListCap = 65536;              // candidates the single-CTA list selection accepts
-constexpr int kListThreads = 1024;
+constexpr int kListSmall = 1536;               // keys of the list that later sweeps keep in shared memory
+constexpr int kTailPerSm = 4;                 // CTAs of the cooperative tail per SM
 constexpr int kBins = 8192;                  // 13-bit digits
 constexpr int kDigitBits = 13;
 constexpr int kWinBins = 2;                  // coarse bins covered by the fine window of level 0
 constexpr int kFineBits = 10;                // extra bits resolved inside the window
 constexpr int kFinePerBin = 1 << kFineBits;
 constexpr int kFineBins = kWinBins * kFinePerBin;
-constexpr int kSampleRows = 8192;            // rows read by the estimate pass
+constexpr int kSampleRows = 4096;            // rows read by the estimate pass
 constexpr int kSelThreads = 256;
 constexpr int kRowsPerBlock = 1024;          // rows per CTA in the sum / out kernels (4 per thread)
 constexpr int kTypeSlots = 4096;             // hash slots for exact tie types
@@ -94,12 +100,14 @@ struct Workspace {
     uint16_t *sketch;                  // [N][sk_ld] top 16 bits of keys 0, 8, 16, ... of each row
     int32_t sk_ld;
     int32_t *active;                   // [N] rows with a non-empty segment
-    long long *bsum_hi, *bsum_t;       // [NB] block sums, overwritten by exclusive prefixes
+    long long *bsum_hi, *bsum_t;       // [NB] sums over blocks of kRowsPerBlock prompts, overwritten by exclusive prefixes
     double *objpart;                   // [NB]
     unsigned long long *tkeys, *tcounts;   // [kTypeSlots]
     int32_t *tlabel;                   // [kTypeSlots]
     int32_t *rowslot;                  // [N]
     unsigned long long *cand_key;      // [kListCap] list mode: every key that carries level 0's prefix
+    int32_t *cand_row;                 // [kListCap] and its row
+    double *objrow;                    // [N] U_i(Delta_i) where level 1 could evaluate it, else negative
     double *gains;                     // [N*ld] when the caller passed none
     size_t bytes;
 };
@@ -117,14 +125,16 @@ static Workspace carve(void *base, int64_t N, int32_t ld, bool need_gains, bool 
     w.hist_coarse = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kBins));
     w.hist_fine = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kFineBins));
     w.hist_lv = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kLevels * kBins));
+    w.bsum_hi = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
+    w.bsum_t = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
     w.rowstate = reinterpret_cast<int2 *>(take(sizeof(int2) * (size_t)N));          // everything before this is zeroed per call
     w.sk_ld = ((ld + 7) / 8 + 7) & ~7;
     w.sketch = reinterpret_cast<uint16_t *>(take(sizeof(uint16_t) * (size_t)N * (size_t)w.sk_ld));
     w.active = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (size_t)N));
-    w.bsum_hi = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
-    w.bsum_t = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
     w.objpart = reinterpret_cast<double *>(take(sizeof(double) * (size_t)NB));
     w.cand_key = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kListCap));
+    w.cand_row = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * kListCap));
+    w.objrow = reinterpret_cast<double *>(take(sizeof(double) * (size_t)N));
     if (exact) {
         w.tkeys = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kTypeSlots));
         w.tcounts = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kTypeSlots));
@@ -621,6 +631,13 @@ gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ 
     level0_finish(hdr, hist, hist_fine, s_hist, tap.win_lo, tap.capsum, false, B, s_warp);
 }
 
+// U_i(Delta) from the row's own entry: the product in U_i(Delta) = 1 - prod_{j<Delta} (b+j)/(a+b+j) is
+// g_i(Delta) (b + Delta - 1) / a  (Eq. marginal), so one load replaces Delta multiplications.  Every operation
+// is pinned to one rounding so that the value does not depend on which kernel evaluates it.
+__device__ __forceinline__ double utility_from_gain(double g, double a, double b, int32_t Delta) {
+    return __dsub_rn(1.0, __ddiv_rn(__dmul_rn(g, __dadd_rn(b, (double)(Delta - 1))), a));
+}
+
 // ---------------------------------------------------------------------------------------------------
 // Level 1: a thread per row.  r bits of the threshold are known (23 after a window hit, else 13); call
 // P that prefix.  The sketch holds the top 16 bits of the first (largest) key of every group of 8 keys.
@@ -646,7 +663,8 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
               const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N,
               int32_t ld, const double *__restrict__ gains, AllocHeader *hdr, unsigned long long *hist1,
               const uint16_t *__restrict__ sketch, int32_t sk_ld, int2 *__restrict__ rowstate,
-              int32_t *__restrict__ active, unsigned long long *__restrict__ cand_key) {
+              int32_t *__restrict__ active, unsigned long long *__restrict__ cand_key,
+              int32_t *__restrict__ cand_row, long long *bsum_hi, double *__restrict__ objrow) {
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     __shared__ unsigned int s_base;
@@ -745,18 +763,33 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
             }
             p_hi = lo + n_gt;
             rowstate[row] = make_int2(p_hi, p_hi + n_eq);
+            if (objrow != nullptr) {
+                // no key in the threshold's bin: Delta_i = p_hi is final, and g_i(Delta_i) was just read (L1)
+                double u = -1.0;                                 // otherwise: evaluated by the output pass
+                if (n_eq == 0)
+                    u = p_hi > 0 ? utility_from_gain(__longlong_as_double((long long)__ldg(keys + p_hi - 1)), post.a, post.b, p_hi)
+                                 : 0.0;
+                objrow[row] = u;
+            }
         }
         if (list) {
+            // one block scan gives the step's sum of p_hi (upper half) and the slots of its keys (lower half);
             // one reservation per CTA and step; the order of the list does not matter to anything
             long long tot;
-            const long long excl = block_exclusive_sum((long long)n_eq, &tot, s_warp);
-            if (tot > 0) {
-                if (threadIdx.x == 0) s_base = atomicAdd(&hdr->n_cand, (unsigned int)tot);
+            const long long excl = block_exclusive_sum(((long long)p_hi << 32) | (long long)n_eq, &tot, s_warp);
+            if (threadIdx.x == 0 && (tot >> 32) != 0)
+                atomicAdd(reinterpret_cast<unsigned long long *>(bsum_hi) + base / kRowsPerBlock, (unsigned long long)(tot >> 32));
+            const unsigned int n_new = (unsigned int)(tot & 0xFFFFFFFFll);
+            if (n_new > 0) {
+                if (threadIdx.x == 0) s_base = atomicAdd(&hdr->n_cand, n_new);
                 __syncthreads();
-                const long long slot = (long long)s_base + excl;
+                const long long slot = (long long)s_base + (excl & 0xFFFFFFFFll);
                 for (int32_t j = 0; j < n_eq; ++j) {
                     const unsigned long long key = __ldg(keys + p_hi + j);
-                    if (slot + j < kListCap) cand_key[slot + j] = key;
+                    if (slot + j < kListCap) {
+                        cand_key[slot + j] = key;
+                        cand_row[slot + j] = (int32_t)row;
+                    }
                     atomicAdd(hist1 + ((key >> shift) & digit_mask), 1ull);   // few keys: straight to global memory
                 }
             }
@@ -779,35 +812,34 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
 }
 
 // ---------------------------------------------------------------------------------------------------
-// List mode: ONE CTA resolves the remaining bits of the threshold over the candidate list (every key that
-// carries level 0's prefix).  The first digit comes from the histogram level 1 accumulated; the keys that
-// carry it are usually a handful and are gathered into shared memory, over which the remaining digits are
-// found 13 bits per sweep.  Should more than kListSmall keys share that digit (ties), the sweeps run over
-// the list in global memory instead.
-constexpr int kListSmall = 1536;
+// The tail: one cooperative launch (every CTA resident at once) that finishes the threshold and leaves, for
+// the output pass, the exclusive prefixes of (#keys > lambda, #keys == lambda) over blocks of 1024 prompts.
 
-// digit search over a histogram in shared memory, run by the whole CTA: the bin where the count from the
-// top reaches `need`.  s_pick receives (digit, count above it, count of it); digit -1 if out of range.
-__device__ __forceinline__ void list_locate(const unsigned int *s_hist, int bins, long long need, long long *s_scan,
-                                            long long *s_pick) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int per = (bins + kListThreads - 1) / kListThreads;    // thread t owns bins top, top-1, ..., top-per+1
-    const int top = bins - 1 - tid * per;
+// Close a row's segment with the finished threshold: keys above it, keys equal to it.
+__device__ __forceinline__ int2 close_segment(const unsigned long long *__restrict__ keys, int2 st, unsigned long long lam) {
+    int32_t n_gt = 0, n_eq = 0;
+    for (int32_t pp = st.x; pp < st.y; ++pp) {
+        const unsigned long long key = __ldg(keys + pp);
+        if (key > lam) ++n_gt;
+        else if (key == lam) ++n_eq;
+        else break;
+    }
+    return make_int2(st.x + n_gt, st.x + n_gt + n_eq);
+}
+
+// Digit search over a histogram in SHARED memory, run by one CTA: the bin where the count from the top
+// reaches `need`.  s_pick receives (digit, count above it, count of it); digit -1 if need is out of range.
+__device__ __forceinline__ void locate_rank_shared(const unsigned int *s_hist, int bins, long long need, long long *s_warp,
+                                                   long long *s_pick) {
+    const int per = (bins + kSelThreads - 1) / kSelThreads;      // thread t owns bins top, top-1, ..., top-per+1
+    const int top = bins - 1 - (int)threadIdx.x * per;
     long long local = 0;
     for (int j = 0; j < per; ++j)
         if (top - j >= 0) local += s_hist[top - j];
-    long long inc = local;
-#pragma unroll
-    for (int d = 1; d < kWarp; d <<= 1) {
-        const long long t = __shfl_up_sync(kFull, inc, d);
-        if (lane >= d) inc += t;
-    }
-    if (lane == kWarp - 1) s_scan[warp] = inc;
-    if (tid == 0) s_pick[0] = -1;
-    __syncthreads();
-    long long above = inc - local;
-    for (int w = 0; w < warp; ++w) above += s_scan[w];
-    if (above < need && need <= above + local) {                 // at most one thread: the crossing is in its run
+    if (threadIdx.x == 0) s_pick[0] = -1;
+    long long total;
+    const long long above = block_exclusive_sum(local, &total, s_warp);
+    if (need >= 1 && above < need && need <= above + local) {    // at most one thread: the crossing is in its run
         long long run = above;
         for (int j = 0; j < per; ++j) {
             const long long cnt = s_hist[top - j];
@@ -823,52 +855,84 @@ __device__ __forceinline__ void list_locate(const unsigned int *s_hist, int bins
     __syncthreads();
 }
 
-__global__ void __launch_bounds__(kListThreads)
-select_list(AllocHeader *hdr, const unsigned long long *hist1, const unsigned long long *__restrict__ cand_key) {
-    __shared__ unsigned int s_hist[kBins];
-    __shared__ unsigned long long s_keys[kListSmall];
-    __shared__ long long s_scan[kListThreads / kWarp];
+// Exclusive scan of the block sums (plus, in list mode, the corrections held in shared memory for blocks
+// [b0, b0 + n_here)), kSelThreads * 4 entries per step, in index order; run by one CTA.
+__device__ void scan_block_sums(long long *bsum_hi, long long *bsum_t, int64_t b0, int64_t n_here,
+                                const unsigned int *s_fix_hi, const unsigned int *s_fix_t, long long &run_hi,
+                                long long &run_t, long long *s_warp) {
+    constexpr int kRun = 4;                                      // consecutive block sums per thread
+    for (int64_t c0 = 0; c0 < n_here; c0 += kRun * kSelThreads) {
+        const int64_t c = c0 + (int64_t)threadIdx.x * kRun;
+        long long vh[kRun], vt[kRun], sh = 0, st = 0;
+#pragma unroll
+        for (int u = 0; u < kRun; ++u) {
+            const bool in = c + u < n_here;
+            vh[u] = in ? __ldcg(bsum_hi + b0 + c + u) + (s_fix_hi ? (long long)s_fix_hi[c + u] : 0) : 0;
+            vt[u] = in ? __ldcg(bsum_t + b0 + c + u) + (s_fix_t ? (long long)s_fix_t[c + u] : 0) : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < kRun; ++u) { sh += vh[u]; st += vt[u]; }
+        long long th, tt;
+        long long eh = run_hi + block_exclusive_sum(sh, &th, s_warp);
+        long long et = run_t + block_exclusive_sum(st, &tt, s_warp);
+#pragma unroll
+        for (int u = 0; u < kRun; ++u) {
+            if (c + u < n_here) { bsum_hi[b0 + c + u] = eh; bsum_t[b0 + c + u] = et; }
+            eh += vh[u];
+            et += vt[u];
+        }
+        run_hi += th;
+        run_t += tt;
+    }
+}
+
+// List route, run by ONE CTA: the first digit comes from the histogram level 1 accumulated in global memory;
+// the keys that carry it are usually a handful and are gathered into shared memory, over which the remaining
+// digits are found 13 bits per sweep.  Should more than kListSmall keys share that digit (ties), the sweeps
+// run over the list in global memory instead.  Then the block sums are corrected and scanned.
+__device__ void tail_list(int64_t B, AllocHeader *hdr, const unsigned long long *hist1,
+                          const unsigned long long *__restrict__ cand_key, const int32_t *__restrict__ cand_row,
+                          long long *bsum_hi, long long *bsum_t, int64_t NB, unsigned int *s_hist,
+                          unsigned long long *s_keys, long long *s_warp) {
     __shared__ long long s_pick[3];                              // digit, count above it, count of it
     __shared__ unsigned int s_fill;
-    if (*(volatile int32_t *)&hdr->status != 0 || hdr->list_mode == 0) return;
     const int tid = threadIdx.x;
-    unsigned int n = hdr->n_cand;
-    n = n < (unsigned)kListCap ? n : (unsigned)kListCap;
+    unsigned int n_all = hdr->n_cand;
+    n_all = n_all < (unsigned)kListCap ? n_all : (unsigned)kListCap;
     int resolved = hdr->resolved;
     long long need = hdr->need;
     unsigned long long prefix = hdr->prefix_key;
     const int r0 = resolved;                                     // every key of the list agrees on these bits
-    // first digit: level 1 left its histogram in global memory
+    long long left;                                              // keys that carry every digit found so far
     {
         int bits, shift;
         next_digit(resolved, &bits, &shift);
-        const int bins = 1 << bits;
-        for (int b = tid; b < bins; b += kListThreads) s_hist[b] = (unsigned int)__ldcg(hist1 + b);
-        if (tid == 0) s_fill = 0;
-        __syncthreads();
-        list_locate(s_hist, bins, need, s_scan, s_pick);
-        if (s_pick[0] < 0) return;                               // cannot happen: need lies within the list
-        need -= s_pick[1];
-        prefix |= (unsigned long long)s_pick[0] << shift;
+        long long above = 0, count = 0;
+        const int digit = locate_rank(hist1, 1 << bits, need, &above, &count, s_warp);
+        if (digit < 0) return;                                   // cannot happen: need lies within the list
+        need -= above;
+        prefix |= (unsigned long long)digit << shift;
         resolved += bits;
+        left = count;
     }
-    const long long left = s_pick[2];                            // keys that carry the first digit
     const unsigned long long *src = cand_key;
+    unsigned int n = n_all;
+    if (tid == 0) s_fill = 0;
     __syncthreads();
     if (left <= kListSmall && resolved < 64) {                   // gather them; the later sweeps stay in shared memory
         const int known = resolved - r0;
         const unsigned long long want = (prefix << r0) >> (64 - known);
-        for (unsigned int i0 = 0; i0 < n; i0 += 8 * kListThreads) {
+        for (unsigned int i0 = 0; i0 < n_all; i0 += 8 * kSelThreads) {
             unsigned long long key[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const unsigned int i = i0 + u * kListThreads + tid;
-                key[u] = i < n ? cand_key[i] : 0ull;
+                const unsigned int i = i0 + u * kSelThreads + tid;
+                key[u] = i < n_all ? cand_key[i] : 0ull;
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const unsigned int i = i0 + u * kListThreads + tid;
-                if (i < n && (key[u] << r0) >> (64 - known) == want) {
+                const unsigned int i = i0 + u * kSelThreads + tid;
+                if (i < n_all && (key[u] << r0) >> (64 - known) == want) {
                     const unsigned int slot = atomicAdd(&s_fill, 1u);
                     if (slot < (unsigned)kListSmall) s_keys[slot] = key[u];
                 }
@@ -878,89 +942,208 @@ select_list(AllocHeader *hdr, const unsigned long long *hist1, const unsigned lo
         n = s_fill < (unsigned)kListSmall ? s_fill : (unsigned)kListSmall;
         src = s_keys;
     }
+    if (src == s_keys && n <= (unsigned)kSelThreads && resolved < 64) {
+        // a handful of keys left: rank them directly — the threshold is the key k with
+        // #(keys > k) < need <= #(keys >= k); equal keys write the same answer
+        if (tid == 0) s_pick[0] = -1;
+        __syncthreads();
+        if ((unsigned)tid < n) {
+            const unsigned long long mine = s_keys[tid];
+            long long gt = 0, ge = 0;
+            for (unsigned int j = 0; j < n; ++j) {
+                const unsigned long long other = s_keys[j];
+                gt += other > mine;
+                ge += other >= mine;
+            }
+            if (gt < need && need <= ge) {
+                s_pick[0] = (long long)mine;
+                s_pick[1] = gt;
+                s_pick[2] = ge - gt;
+            }
+        }
+        __syncthreads();
+        if (s_pick[0] < 0) return;                               // cannot happen (keys are non-negative doubles)
+        prefix = (unsigned long long)s_pick[0];
+        need -= s_pick[1];
+        left = s_pick[2];
+        resolved = 64;
+        __syncthreads();
+    }
     while (resolved < 64) {
         int bits, shift;
         next_digit(resolved, &bits, &shift);
         const int bins = 1 << bits;
-        for (int b = tid; b < bins; b += kListThreads) s_hist[b] = 0;
+        for (int b = tid; b < bins; b += kSelThreads) s_hist[b] = 0;
         __syncthreads();
         // keys that agree with the digits found so far in this kernel (bits r0 .. resolved-1)
         const int known = resolved - r0;
         const unsigned long long want = (prefix << r0) >> (64 - known);
-        for (unsigned int i0 = 0; i0 < n; i0 += 8 * kListThreads) {
+        for (unsigned int i0 = 0; i0 < n; i0 += 8 * kSelThreads) {
             unsigned long long key[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const unsigned int i = i0 + u * kListThreads + tid;
+                const unsigned int i = i0 + u * kSelThreads + tid;
                 key[u] = i < n ? src[i] : 0ull;
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const unsigned int i = i0 + u * kListThreads + tid;
+                const unsigned int i = i0 + u * kSelThreads + tid;
                 if (i < n && (key[u] << r0) >> (64 - known) == want)
                     atomicAdd(&s_hist[(key[u] >> shift) & (unsigned long long)(bins - 1)], 1u);
             }
         }
         __syncthreads();
-        list_locate(s_hist, bins, need, s_scan, s_pick);
-        if (s_pick[0] < 0) break;                                // cannot happen
+        locate_rank_shared(s_hist, bins, need, s_warp, s_pick);
+        if (s_pick[0] < 0) return;                               // cannot happen
         need -= s_pick[1];
         prefix |= (unsigned long long)s_pick[0] << shift;
         resolved += bits;
+        left = s_pick[2];
+        __syncthreads();
+    }
+    // The threshold is `prefix`; `need` of the `left` keys equal to it are taken.  Block sums: level 1 added up
+    // its provisional p_hi (keys above the 23-bit prefix); the listed keys above / equal to the threshold
+    // complete them, 4096 blocks at a time through shared-memory counters.
+    unsigned int *s_fix_hi = s_hist, *s_fix_t = s_hist + kBins / 2;
+    long long run_hi = 0, run_t = 0;
+    for (int64_t b0 = 0; b0 < NB; b0 += kBins / 2) {
+        const int64_t n_here = NB - b0 < kBins / 2 ? NB - b0 : kBins / 2;
+        for (int b = tid; b < kBins; b += kSelThreads) s_hist[b] = 0;
+        __syncthreads();
+        for (unsigned int i0 = 0; i0 < n_all; i0 += 8 * kSelThreads) {
+            unsigned long long key[8];
+            int32_t row[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const unsigned int i = i0 + u * kSelThreads + tid;
+                key[u] = i < n_all ? cand_key[i] : 0ull;
+                row[u] = i < n_all ? cand_row[i] : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const unsigned int i = i0 + u * kSelThreads + tid;
+                const int64_t blk = (int64_t)row[u] / kRowsPerBlock - b0;
+                if (i < n_all && blk >= 0 && blk < n_here) {
+                    if (key[u] > prefix) atomicAdd(&s_fix_hi[blk], 1u);
+                    else if (key[u] == prefix) atomicAdd(&s_fix_t[blk], 1u);
+                }
+            }
+        }
+        __syncthreads();
+        scan_block_sums(bsum_hi, bsum_t, b0, n_here, s_fix_hi, s_fix_t, run_hi, run_t, s_warp);
         __syncthreads();
     }
     if (tid == 0) {
         hdr->prefix_key = prefix;
         hdr->need = need;
         hdr->resolved = resolved;
+        hdr->n_above = (unsigned long long)run_hi;
+        hdr->n_tied = (unsigned long long)run_t;
+        hdr->R = B - run_hi;
+        hdr->lambda = __longlong_as_double((long long)prefix);
     }
 }
 
-// ---------------------------------------------------------------------------------------------------
-// Levels 2..4 (only when the candidates were too many for the list): a thread per ACTIVE row narrows the
-// stored segment by the digit selected one level up; the keys that remain are histogrammed on the next
-// digit and the last CTA selects it.  The active list is in no particular order; nothing here depends on it.
-__global__ void __launch_bounds__(kSelThreads)
-select_refine(int32_t ld, const double *__restrict__ gains, int level, AllocHeader *hdr,
-              unsigned long long *hist_all, int2 *__restrict__ rowstate, const int32_t *__restrict__ active) {
-    __shared__ unsigned int s_hist[kBins];
-    __shared__ long long s_warp[kSelThreads / kWarp];
-    if (*(volatile int32_t *)&hdr->status != 0 || hdr->list_mode != 0) return;
-    int bits = 0, shift = 0;
-    next_digit(hdr->resolved, &bits, &shift);
-    const int bins = 1 << bits;
-    for (int b = threadIdx.x; b < bins; b += kSelThreads) s_hist[b] = 0;
-    __syncthreads();
-    const int shift_prev = hdr->lv_shift[level - 1];
-    const unsigned long long mask_prev = (1ull << hdr->lv_bits[level - 1]) - 1ull;
-    const unsigned long long d_prev = (unsigned long long)hdr->sel_digit[level - 1];
-    const unsigned long long mask_cur = (unsigned long long)bins - 1ull;
+// Digit route, all CTAs: levels 2..4 (a thread per ACTIVE row narrows the stored segment by the digit selected
+// one level up; the keys that remain are histogrammed on the next digit, which CTA 0 selects between two
+// grid-wide barriers), then every segment is closed with the finished threshold, the block sums formed and
+// scanned.  The active list is in no particular order; nothing here depends on it.
+__device__ void tail_digits(int64_t N, int32_t ld, const double *__restrict__ gains, int64_t B, AllocHeader *hdr,
+                            unsigned long long *hist_all, int2 *__restrict__ rowstate,
+                            const int32_t *__restrict__ active, long long *bsum_hi, long long *bsum_t, int64_t NB,
+                            unsigned int *s_hist, long long *s_warp) {
+    cooperative_groups::grid_group grid = cooperative_groups::this_grid();
     const unsigned int n_active = hdr->n_active;
     const unsigned int stride = gridDim.x * kSelThreads;
-    for (unsigned int idx = blockIdx.x * kSelThreads + threadIdx.x; idx < n_active; idx += stride) {
-        const int64_t row = active[idx];
-        const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-        const int2 st = rowstate[row];
-        const int32_t p_hi = st.x, p_end = st.y;
-        int32_t p = p_hi, new_hi = p_hi;
-        while (p < p_end) {
-            const unsigned long long key = __ldg(keys + p);
-            const unsigned long long dp = (key >> shift_prev) & mask_prev;
-            if (dp > d_prev) {
-                new_hi = p + 1;
-            } else if (dp == d_prev) {
-                atomicAdd(&s_hist[(key >> shift) & mask_cur], 1u);
-            } else {
-                break;
+    for (int level = 2; level < kLevels; ++level) {
+        int bits = 0, shift = 0;
+        next_digit(*(volatile int32_t *)&hdr->resolved, &bits, &shift);
+        const int bins = 1 << bits;
+        for (int b = threadIdx.x; b < bins; b += kSelThreads) s_hist[b] = 0;
+        __syncthreads();
+        const int shift_prev = *(volatile int32_t *)&hdr->lv_shift[level - 1];
+        const unsigned long long mask_prev = (1ull << *(volatile int32_t *)&hdr->lv_bits[level - 1]) - 1ull;
+        const unsigned long long d_prev = (unsigned long long)*(volatile int32_t *)&hdr->sel_digit[level - 1];
+        const unsigned long long mask_cur = (unsigned long long)bins - 1ull;
+        for (unsigned int idx = blockIdx.x * kSelThreads + threadIdx.x; idx < n_active; idx += stride) {
+            const int64_t row = active[idx];
+            const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+            const int2 st = __ldcg(rowstate + row);
+            const int32_t p_hi = st.x, p_end = st.y;
+            int32_t p = p_hi, new_hi = p_hi;
+            while (p < p_end) {
+                const unsigned long long key = __ldg(keys + p);
+                const unsigned long long dp = (key >> shift_prev) & mask_prev;
+                if (dp > d_prev) {
+                    new_hi = p + 1;
+                } else if (dp == d_prev) {
+                    atomicAdd(&s_hist[(key >> shift) & mask_cur], 1u);
+                } else {
+                    break;
+                }
+                ++p;
             }
-            ++p;
+            if (new_hi != p_hi || p != p_end) rowstate[row] = make_int2(new_hi, p);
         }
-        if (new_hi != p_hi || p != p_end) rowstate[row] = make_int2(new_hi, p);
+        __syncthreads();
+        flush_hist(s_hist, hist_all + (size_t)level * kBins, bins);
+        grid.sync();
+        if (blockIdx.x == 0) {
+            find_digit(hdr, hist_all + (size_t)level * kBins, bins, bits, shift, level, false, s_warp);
+            __threadfence();
+        }
+        grid.sync();
     }
-    __syncthreads();
-    flush_hist(s_hist, hist_all + (size_t)level * kBins, bins);
-    if (last_block(&hdr->ticket[level]))
-        find_digit(hdr, hist_all + (size_t)level * kBins, bins, bits, shift, level, false, s_warp);
+    // close every segment and add up blocks of kRowsPerBlock prompts
+    const unsigned long long lam = *(volatile unsigned long long *)&hdr->prefix_key;
+    for (int64_t blk = blockIdx.x; blk < NB; blk += gridDim.x) {
+        long long hi_sum = 0, t_sum = 0;
+#pragma unroll
+        for (int q = 0; q < kRowsPerBlock / kSelThreads; ++q) {
+            const int64_t row = blk * kRowsPerBlock + q * kSelThreads + threadIdx.x;
+            if (row < N) {
+                int2 st = __ldcg(rowstate + row);
+                if (st.y > st.x) {
+                    const int2 fin = close_segment(reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld, st, lam);
+                    if (fin.x != st.x || fin.y != st.y) rowstate[row] = fin;
+                    st = fin;
+                }
+                hi_sum += st.x;
+                t_sum += st.y - st.x;
+            }
+        }
+        long long tot_hi, tot_t;
+        block_exclusive_sum(hi_sum, &tot_hi, s_warp);
+        block_exclusive_sum(t_sum, &tot_t, s_warp);
+        if (threadIdx.x == 0) { bsum_hi[blk] = tot_hi; bsum_t[blk] = tot_t; }
+    }
+    grid.sync();
+    if (blockIdx.x == 0) {
+        long long run_hi = 0, run_t = 0;
+        scan_block_sums(bsum_hi, bsum_t, 0, NB, nullptr, nullptr, run_hi, run_t, s_warp);
+        if (threadIdx.x == 0) {
+            hdr->n_above = (unsigned long long)run_hi;
+            hdr->n_tied = (unsigned long long)run_t;
+            hdr->R = B - run_hi;
+            hdr->lambda = __longlong_as_double((long long)lam);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kSelThreads, kTailPerSm)
+select_tail(int64_t N, int32_t ld, const double *__restrict__ gains, int64_t B, AllocHeader *hdr,
+            unsigned long long *hist_all, int2 *__restrict__ rowstate, const int32_t *__restrict__ active,
+            long long *bsum_hi, long long *bsum_t, int64_t NB, const unsigned long long *__restrict__ cand_key,
+            const int32_t *__restrict__ cand_row) {
+    __shared__ unsigned int s_hist[kBins];
+    __shared__ unsigned long long s_keys[kListSmall];
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    if (*(volatile int32_t *)&hdr->status != 0) return;         // the same answer in every CTA: nobody waits at a barrier
+    if (hdr->list_mode != 0) {
+        if (blockIdx.x == 0) tail_list(B, hdr, hist_all + kBins, cand_key, cand_row, bsum_hi, bsum_t, NB, s_hist, s_keys, s_warp);
+        return;
+    }
+    tail_digits(N, ld, gains, B, hdr, hist_all, rowstate, active, bsum_hi, bsum_t, NB, s_hist, s_warp);
 }
 
 // (exact 128/256-bit helpers: hora_exact.cuh)
@@ -979,7 +1162,9 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
               int32_t *__restrict__ rowslot, unsigned long long *tkeys, unsigned long long *tcounts) {
     __shared__ long long s_warp[kSelThreads / kWarp];
     if (*(volatile int32_t *)&hdr->status != 0) return;
-    const double lam = __longlong_as_double((long long)hdr->prefix_key);
+    const unsigned long long lam_key = hdr->prefix_key;
+    const bool list = hdr->list_mode != 0;
+    const double lam = __longlong_as_double((long long)lam_key);
     const double delta_rel = 9.313225746154785e-10;   // 2^-30
     const unsigned long long k_hi = (unsigned long long)__double_as_longlong(lam * (1.0 + delta_rel));
     const unsigned long long k_lo = (unsigned long long)__double_as_longlong(lam * (1.0 - delta_rel));
@@ -998,7 +1183,8 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
             if (!(al >= 1.0 && be >= 1.0 && al == floor(al) && be == floor(be))) err = HORA_ERR_NOT_INTEGER;
             else if (al + be + (double)G0 + (double)ld >= 1048576.0) err = err ? err : HORA_ERR_EXACT_RANGE;
             const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-            const int2 st = rowstate[row];
+            int2 st = rowstate[row];
+            if (list && st.y > st.x) st = close_segment(keys, st, lam_key);   // the list route leaves segments open
             q = st.x;                                         // #keys > lambda
             if (q > 0 && __ldg(keys + q - 1) <= k_hi) {
                 --q;
@@ -1097,10 +1283,9 @@ exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ t
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Block sums of (p_hi, tied) in prompt order, and their exclusive scan by the last CTA.
-//   mode 0: first close every non-empty segment with the finished threshold    mode 2: apply the exact labels first
-// With `validate` the priors and counts of every prompt are checked here (only when level 1, which checks
-// them otherwise, did not run).
+// Block sums of (p_hi, tied) in prompt order, and their exclusive scan by the last CTA; used where the tail
+// did not run (B == 0: mode 0) or its result is relabelled (exact mode: mode 2, apply the labels first).
+// With `validate` the priors and counts of every prompt are checked here (level 1 checks them otherwise).
 __global__ void __launch_bounds__(kSelThreads)
 select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
            const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar, int validate,
@@ -1125,24 +1310,10 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
             if (validate) ok &= load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, rr).ok;
         }
         if (!ok) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);   // seen by the kernels that follow
-        const unsigned long long lam = hdr->prefix_key;       // the threshold, once all 64 bits are resolved
 #pragma unroll
         for (int q = 0; q < kPer; ++q) {
             const int64_t row = row0 + q * kSelThreads + threadIdx.x;
             if (row < N) {
-                if (mode == 0 && st[q].y > st[q].x) {         // close the segment: keys above / equal to the threshold
-                    const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-                    int32_t n_gt = 0, n_eq = 0;
-                    for (int32_t pp = st[q].x; pp < st[q].y; ++pp) {
-                        const unsigned long long key = __ldg(keys + pp);
-                        if (key > lam) ++n_gt;
-                        else if (key == lam) ++n_eq;
-                        else break;
-                    }
-                    const int2 fin = make_int2(st[q].x + n_gt, st[q].x + n_gt + n_eq);
-                    if (fin.x != st[q].x || fin.y != st[q].y) rowstate[row] = fin;
-                    st[q] = fin;
-                }
                 if (mode == 2) {
                     const int label = slot[q] >= 0 ? tlabel[slot[q]] : 0;
                     st[q] = make_int2(st[q].x + (label == 2), st[q].x + (label == 2) + (label == 1));
@@ -1158,31 +1329,8 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
     block_exclusive_sum(t_sum, &tot_t, s_warp);
     if (threadIdx.x == 0) { bsum_hi[blockIdx.x] = tot_hi; bsum_t[blockIdx.x] = tot_t; }
     if (last_block(&hdr->ticket[8 + mode])) {
-        // exclusive scan of NB block sums, kSelThreads at a time, in index order
         long long run_hi = 0, run_t = 0;
-        constexpr int kRun = 4;                                 // consecutive block sums per thread
-        for (int64_t b0 = 0; b0 < NB; b0 += kRun * kSelThreads) {
-            const int64_t b = b0 + (int64_t)threadIdx.x * kRun;
-            long long vh[kRun], vt[kRun], sh = 0, st = 0;
-#pragma unroll
-            for (int u = 0; u < kRun; ++u) {
-                vh[u] = b + u < NB ? __ldcg(bsum_hi + b + u) : 0;
-                vt[u] = b + u < NB ? __ldcg(bsum_t + b + u) : 0;
-            }
-#pragma unroll
-            for (int u = 0; u < kRun; ++u) { sh += vh[u]; st += vt[u]; }
-            long long th, tt;
-            long long eh = run_hi + block_exclusive_sum(sh, &th, s_warp);
-            long long et = run_t + block_exclusive_sum(st, &tt, s_warp);
-#pragma unroll
-            for (int u = 0; u < kRun; ++u) {
-                if (b + u < NB) { bsum_hi[b + u] = eh; bsum_t[b + u] = et; }
-                eh += vh[u];
-                et += vt[u];
-            }
-            run_hi += th;
-            run_t += tt;
-        }
+        scan_block_sums(bsum_hi, bsum_t, 0, NB, nullptr, nullptr, run_hi, run_t, s_warp);
         if (threadIdx.x == 0 && !failed) {
             hdr->n_above = (unsigned long long)run_hi;
             hdr->n_tied = (unsigned long long)run_t;
@@ -1192,76 +1340,110 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
     }
 }
 
-// Outputs.  A CTA owns kRowsPerBlock consecutive prompts, a thread four consecutive ones.
+// Outputs.  A CTA owns kRowsPerBlock consecutive prompts, a thread four consecutive ones (16-byte loads and
+// stores where the caller's arrays are 16-byte aligned: `vec`).  `objrow` (may be null) holds the utilities
+// level 1 already evaluated; a negative entry, or no array, means "evaluate here".
 __global__ void __launch_bounds__(kSelThreads)
 select_out(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
            const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N,
            int32_t ld, const double *__restrict__ gains, int64_t B, uint32_t flags, AllocHeader *hdr,
-           const int2 *__restrict__ rowstate, const long long *__restrict__ bpre_hi, const long long *__restrict__ bpre_t, double *objpart, int64_t NB,
-           int32_t *__restrict__ delta, int32_t *__restrict__ G, int64_t *__restrict__ offsets,
-           hora_alloc_info *info) {
+           const int2 *__restrict__ rowstate, const double *__restrict__ objrow, const long long *__restrict__ bpre_hi,
+           const long long *__restrict__ bpre_t, double *objpart, int64_t NB, int32_t *__restrict__ delta,
+           int32_t *__restrict__ G, int64_t *__restrict__ offsets, int vec, hora_alloc_info *info) {
     __shared__ long long s_warp[kSelThreads / kWarp];
     __shared__ double s_obj[kSelThreads / kWarp];
     const int32_t status = *(volatile int32_t *)&hdr->status;
     const bool failed = status != 0;
     constexpr int kPer = kRowsPerBlock / kSelThreads;
+    static_assert(kPer == 4, "a thread owns four consecutive prompts");
     const int64_t row0 = (int64_t)blockIdx.x * kRowsPerBlock + (int64_t)threadIdx.x * kPer;
+    const bool whole = row0 + kPer <= N;                      // all four prompts exist
+    // the list route of the tail leaves the segments as level 1 found them (exact mode has closed them since)
+    const bool open = !failed && hdr->list_mode != 0 && !(flags & HORA_FLAG_EXACT_INT);
+    const unsigned long long lam_key = hdr->prefix_key;
+    const bool want_obj = !failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE);
+    // every load that does not depend on another is issued here
+    int2 st[kPer];
+    double o[kPer];
+    if (whole) {
+        const int4 s01 = *reinterpret_cast<const int4 *>(rowstate + row0), s23 = *reinterpret_cast<const int4 *>(rowstate + row0 + 2);
+        st[0] = make_int2(s01.x, s01.y); st[1] = make_int2(s01.z, s01.w);
+        st[2] = make_int2(s23.x, s23.y); st[3] = make_int2(s23.z, s23.w);
+    } else {
+#pragma unroll
+        for (int q = 0; q < kPer; ++q) st[q] = row0 + q < N ? rowstate[row0 + q] : make_int2(0, 0);
+    }
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) o[q] = -1.0;
+    if (want_obj && objrow != nullptr) {
+        if (whole) {
+            const double2 o01 = *reinterpret_cast<const double2 *>(objrow + row0), o23 = *reinterpret_cast<const double2 *>(objrow + row0 + 2);
+            o[0] = o01.x; o[1] = o01.y; o[2] = o23.x; o[3] = o23.y;
+        } else {
+#pragma unroll
+            for (int q = 0; q < kPer; ++q) if (row0 + q < N) o[q] = objrow[row0 + q];
+        }
+    }
+    const long long blk_hi = failed ? 0 : bpre_hi[blockIdx.x], blk_t = failed ? 0 : bpre_t[blockIdx.x];
+    const long long R = failed ? 0 : hdr->R;
     int32_t hi[kPer], tied[kPer];
     long long hi_sum = 0, t_sum = 0;
 #pragma unroll
     for (int q = 0; q < kPer; ++q) {
-        hi[q] = 0;
-        tied[q] = 0;
-        if (!failed && row0 + q < N) {
-            const int2 st = rowstate[row0 + q];
-            hi[q] = st.x;
-            tied[q] = st.y - st.x;
-        }
+        if (failed) st[q] = make_int2(0, 0);
+        if (open && st[q].y > st[q].x)
+            st[q] = close_segment(reinterpret_cast<const unsigned long long *>(gains) + (row0 + q) * (int64_t)ld, st[q], lam_key);
+        hi[q] = st[q].x;
+        tied[q] = st[q].y - st[q].x;
         hi_sum += hi[q];
         t_sum += tied[q];
     }
     long long th, tt;
-    long long pre_hi = block_exclusive_sum(hi_sum, &th, s_warp);
-    long long pre_t = block_exclusive_sum(t_sum, &tt, s_warp);
-    double obj = 0.0;
-    if (!failed) {
-        pre_hi += bpre_hi[blockIdx.x];
-        pre_t += bpre_t[blockIdx.x];
-    }
-    const long long R = failed ? 0 : hdr->R;
+    long long pre_hi = blk_hi + block_exclusive_sum(hi_sum, &th, s_warp);
+    long long pre_t = blk_t + block_exclusive_sum(t_sum, &tt, s_warp);
     int32_t d[kPer];
+    int64_t of[kPer];
 #pragma unroll
     for (int q = 0; q < kPer; ++q) {
-        const int64_t row = row0 + q;
-        d[q] = 0;
-        if (row < N) {
-            long long take = R - pre_t;
-            take = take < 0 ? 0 : (take > tied[q] ? tied[q] : take);
-            d[q] = failed ? 0 : hi[q] + (int32_t)take;
-            delta[row] = d[q];
-            G[row] = failed ? 0 : G0 + d[q];
-            if (offsets) offsets[row] = failed ? 0 : row * (int64_t)G0 + pre_hi + (pre_t < R ? pre_t : R);
-            pre_hi += hi[q];
-            pre_t += tied[q];
+        long long take = R - pre_t;
+        take = take < 0 ? 0 : (take > tied[q] ? tied[q] : take);
+        d[q] = hi[q] + (int32_t)take;
+        of[q] = failed ? 0 : (row0 + q) * (int64_t)G0 + pre_hi + (pre_t < R ? pre_t : R);
+        pre_hi += hi[q];
+        pre_t += tied[q];
+    }
+    if (whole && vec) {
+        *reinterpret_cast<int4 *>(delta + row0) = make_int4(d[0], d[1], d[2], d[3]);
+        *reinterpret_cast<int4 *>(G + row0) = failed ? make_int4(0, 0, 0, 0) : make_int4(G0 + d[0], G0 + d[1], G0 + d[2], G0 + d[3]);
+        if (offsets) {
+            *reinterpret_cast<longlong2 *>(offsets + row0) = make_longlong2(of[0], of[1]);
+            *reinterpret_cast<longlong2 *>(offsets + row0 + 2) = make_longlong2(of[2], of[3]);
+        }
+    } else {
+#pragma unroll
+        for (int q = 0; q < kPer; ++q) {
+            if (row0 + q < N) {
+                delta[row0 + q] = d[q];
+                G[row0 + q] = failed ? 0 : G0 + d[q];
+                if (offsets) offsets[row0 + q] = of[q];
+            }
         }
     }
-    // Objective.  The product in U_i(Delta) = 1 - prod_{j<Delta} (b+j)/(a+b+j) is the row's own entry
-    // g_i(Delta) times (b + Delta - 1) / a  (Eq. marginal), so one load replaces Delta multiplications.
-    if (!failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE)) {
-        double g[kPer], pa[kPer], pb[kPer];
+    // Objective: level 1's values where they stand (the row had no key in the threshold's bin, so its Delta was
+    // final there); the other rows are evaluated here, from the row's own entry g_i(Delta).
+    double obj = 0.0;
+    if (want_obj) {
 #pragma unroll
-        for (int q = 0; q < kPer; ++q) {                      // all loads first
-            const int64_t row = row0 + q;
-            const bool use = row < N && d[q] > 0;
-            const int64_t rr = use ? row : 0;
-            const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, rr);
-            pa[q] = p.a;
-            pb[q] = p.b;
-            g[q] = use ? __ldg(gains + rr * (int64_t)ld + (d[q] - 1)) : 0.0;
+        for (int q = 0; q < kPer; ++q) {
+            if (row0 + q < N && d[q] > 0) {
+                double u = o[q];
+                if (u < 0.0) {
+                    const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row0 + q);
+                    u = utility_from_gain(__ldg(gains + (row0 + q) * (int64_t)ld + (d[q] - 1)), p.a, p.b, d[q]);
+                }
+                obj += u;
+            }
         }
-#pragma unroll
-        for (int q = 0; q < kPer; ++q)
-            if (row0 + q < N && d[q] > 0) obj += 1.0 - g[q] * (pb[q] + (double)(d[q] - 1)) / pa[q];
     }
     if (offsets && blockIdx.x == gridDim.x - 1 && threadIdx.x == kSelThreads - 1)
         offsets[N] = failed ? 0 : N * (int64_t)G0 + B;
@@ -1358,6 +1540,25 @@ static cudaError_t launch_fused(bool vec2, bool estimate, int grid_est, int64_t 
     return vec2 ? go(gains_level0_fused<E, true>) : go(gains_level0_fused<E, false>);
 }
 
+// CTAs of the cooperative tail on the current device: what fits at once, at most kTailPerSm per SM (0 on failure).
+// Looked up once per device.
+static int tail_grid_size() {
+    constexpr int kMaxDev = 64;
+    static std::atomic<int> cached[kMaxDev];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return 0;
+    int g = cached[dev].load(std::memory_order_acquire);
+    if (g > 0) return g;
+    int coop = 0, sms = 0, per_sm = 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_tail, kSelThreads, 0) != cudaSuccess || per_sm <= 0)
+        return 0;
+    g = sms * (per_sm < kTailPerSm ? per_sm : kTailPerSm);
+    cached[dev].store(g, std::memory_order_release);
+    return g;
+}
+
 }  // namespace hora
 
 extern "C" void hora_allocate_profile_events(void *start_event, void *stop_event) {
@@ -1445,22 +1646,38 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_stop, s);
     mark_stage(2, s);
     const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
+    // utilities of the rows whose Delta is final after level 1 are evaluated there (not in exact mode, where the
+    // tie ranking may still move a row's Delta)
+    double *objrow = (B > 0 && !exact && !(flags & HORA_FLAG_SKIP_OBJECTIVE)) ? w.objrow : nullptr;
     if (B > 0) {
         if (vec2)
             select_level1<true><<<grid1, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains,
                                                               w.hdr, w.hist_lv + kBins, w.sketch, w.sk_ld, w.rowstate,
-                                                              w.active, w.cand_key);
+                                                              w.active, w.cand_key, w.cand_row, w.bsum_hi, objrow);
         else
             select_level1<false><<<grid1, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains,
                                                                w.hdr, w.hist_lv + kBins, w.sketch, w.sk_ld, w.rowstate,
-                                                               w.active, w.cand_key);
+                                                               w.active, w.cand_key, w.cand_row, w.bsum_hi, objrow);
         mark_stage(3, s);
-        select_list<<<1, kListThreads, 0, s>>>(w.hdr, w.hist_lv + kBins, w.cand_key);
-        for (int level = 2; level < kLevels; ++level)      // levels 2..4: stand down at once in list mode
-            select_refine<<<2 * kSmCount, kSelThreads, 0, s>>>(ld, gains, level, w.hdr, w.hist_lv, w.rowstate, w.active);
+        {
+            // the cooperative tail: every CTA must be resident at once, so the grid is what the device can hold
+            const int tail_grid = tail_grid_size();
+            if (tail_grid <= 0) return HORA_ERR_CUDA;
+            int64_t N_ = N, B_ = B, NB_ = NB;
+            int32_t ld_ = ld;
+            AllocHeader *hdr_ = w.hdr;
+            unsigned long long *hist_ = w.hist_lv;
+            int2 *rowstate_ = w.rowstate;
+            const int32_t *active_ = w.active;
+            long long *bhi_ = w.bsum_hi, *bt_ = w.bsum_t;
+            const unsigned long long *ck_ = w.cand_key;
+            const int32_t *cr_ = w.cand_row;
+            void *args[] = {&N_, &ld_, &gains, &B_, &hdr_, &hist_, &rowstate_, &active_, &bhi_, &bt_, &NB_, &ck_, &cr_};
+            if (cudaLaunchCooperativeKernel(reinterpret_cast<void *>(select_tail), dim3(tail_grid), dim3(kSelThreads), args,
+                                            0, s) != cudaSuccess)
+                return HORA_ERR_CUDA;
+        }
         mark_stage(4, s);
-        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 0, N, ld, gains, 0, B,
-                                                   w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi, w.bsum_t, NB);
         if (exact) {
             exact_collect<<<grid_rows, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
                                                             gains, w.hdr, w.rowstate, w.rowslot, w.tkeys, w.tcounts);
@@ -1474,11 +1691,13 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
                                                    w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi, w.bsum_t, NB);
     }
     mark_stage(5, s);
+    const int out_vec = ((reinterpret_cast<uintptr_t>(delta) | reinterpret_cast<uintptr_t>(G) |
+                          reinterpret_cast<uintptr_t>(group_offsets)) & 15u) == 0;
     select_out<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, flags, w.hdr,
-                                               w.rowstate, w.bsum_hi, w.bsum_t, w.objpart, NB, delta, G, group_offsets,
-                                               info_dev);
+                                               w.rowstate, objrow, w.bsum_hi, w.bsum_t, w.objpart, NB, delta, G,
+                                               group_offsets, out_vec, info_dev);
     mark_stage(6, s);
-    count_launches(B > 0 ? (exact ? 12 : 9) : 3);
+    count_launches(B > 0 ? (exact ? 8 : 5) : 3);
     return cuda_ok(cudaGetLastError());
 }
 

@@ -199,13 +199,13 @@ def test_edge_budgets_and_caps():
 @pytest.mark.parametrize("exact", [True, False])
 def test_allocation_when_the_sampled_window_misses(exact):
     """The full-read pass refines 23 bits inside a window placed from a sample of every k-th row.  Here the
-    sampled rows (index multiple of 3) are all hopeless prompts and the others all saturated ones, so the
+    sampled rows (index multiple of 5) are all hopeless prompts and the others all saturated ones, so the
     sample says nothing about the threshold and the window lands in the wrong place: the selection must
     fall back to plain 13-bit digits and still reproduce the oracle."""
     gu = _util()
-    N, G0, ld = 20000, 8, 96                      # N > 8192 rows, so only every 3rd row is sampled
+    N, G0, ld = 20000, 8, 96                      # N > 4096 rows: every ceil(N / 4096) = 5th row is sampled
     idx = np.arange(N)
-    c = np.where(idx % 3 == 0, 0, G0).astype(np.int32)
+    c = np.where(idx % 5 == 0, 0, G0).astype(np.int32)
     cap = np.full(N, ld, np.int32)
     rng = np.random.default_rng(5)
     if exact:
