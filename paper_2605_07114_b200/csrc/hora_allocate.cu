@@ -4,19 +4,21 @@
 // Keys.  A gain is a non-negative finite double, so its bit pattern orders like the value.  The 64-bit
 // key of the B-th largest gain is resolved from the top, a digit at a time:
 //
-//   estimate  every S-th row (about 8192 rows) is read and histogrammed on the top 13 bits; the scaled rank
-//             says in which two adjacent 13-bit bins the threshold almost surely lies (the "window").
-//   level 0   one coalesced read of the whole matrix (a warp per row-item, two items in flight).  Keys
-//             outside the window are counted per 13-bit bin, keys inside it per 23-bit bin (1024 fine bins
-//             per window bin), all in shared memory, then merged into global histograms.  The last CTA to
-//             finish locates the 13-bit digit of the threshold and, if it is inside the window, its 23-bit
-//             prefix; otherwise the selection simply goes on from 13 bits.  The same pass validates the
-//             rows, sums the caps and writes a 2-byte sketch of every 8th key (its top 16 bits).
+//   estimate  every S-th row (about 4096 rows) is read and histogrammed on the top 13 bits; the scaled rank
+//             says in which two adjacent 13-bit bins the threshold almost surely lies (the "window"), and,
+//             interpolated inside its bin, roughly where: a guessed threshold.
+//   level 0   one coalesced read of the whole matrix (a warp per row-item, two items in flight).  Only the
+//             window is looked at closely: keys inside it are counted per 23-bit bin (2048 fine bins in
+//             shared memory), keys above the guess are counted per row (stored for level 1) and in all.
+//             The last CTA to finish knows from those counts whether the B-th key lies inside the window
+//             and, if so, its 23-bit prefix.  If not (a sample that misleads), a plain pass histograms
+//             every key on 13 bits and the selection goes on from there.  The full read also validates the
+//             rows and sums the caps.
 //   level 1   a thread per row: a row is non-increasing, so its keys with the resolved prefix form ONE
-//             contiguous segment, which the sketch brackets to within 8 keys on each side; only the
-//             bracket is read and the segment [p_hi, p_lo) stored.  The same pass validates the priors.
-//             What happens to the keys of the segments depends on how many there are (level 0 knows the
-//             exact count of keys with the resolved prefix):
+//             contiguous segment [p_hi, p_lo), and p_hi is within a key or two of the stored guess: the
+//             thread reads the eight keys around the guess (widening, then a binary search over the row, if
+//             they do not settle it) and stores the segment.  The same pass validates the priors and
+//             evaluates the utility of every row whose segment is empty (its Delta is final).
 //   tail      ONE cooperative launch finishes the threshold and the prefixes over prompts:
 //     list    at most 65536 such keys (the usual case after a window hit): level 1 appended them to a list
 //             and accumulated per-block sums of its provisional counts; one CTA resolves the remaining bits
@@ -72,11 +74,14 @@ struct AllocHeader {
     int32_t resolved;                  // key bits resolved so far, from the top
     unsigned int ticket[16];
     unsigned long long sum_cap;
+    unsigned long long sum_pguess;     // keys above the guessed threshold, over all rows
     unsigned long long prefix_key;     // the resolved bits in place (the threshold once all 64 are resolved)
     long long need;                    // rank of the threshold inside the current bin (1-based)
     int32_t lv_shift[8], lv_bits[8], sel_digit[8];   // per level: position, width and value of its digit
     int32_t win_lo;                    // first 13-bit bin of level 0's fine window
+    unsigned int guess_hi;             // guessed threshold: a key counts as "above" when its high word exceeds this
     unsigned int n_active;             // rows with a non-empty segment after level 1
+    int32_t l0_miss;                   // 1: the B-th key is not inside level 0's window (the plain 13-bit pass runs)
     unsigned long long sample_cap;     // sum of the caps of the sampled rows
     unsigned long long n_above, n_tied;
     long long R;                       // tied candidates to take
@@ -97,8 +102,7 @@ struct Workspace {
     unsigned long long *hist_fine;     // [kFineBins] level 0, 23-bit bins inside the window
     unsigned long long *hist_lv;       // [kLevels][kBins] levels 1..4 (slot 0 unused)
     int2 *rowstate;                    // [N] (p_hi, p_lo)
-    uint16_t *sketch;                  // [N][sk_ld] top 16 bits of keys 0, 8, 16, ... of each row
-    int32_t sk_ld;
+    unsigned int *pguess;              // [N] keys of the row above the guessed threshold
     int32_t *active;                   // [N] rows with a non-empty segment
     long long *bsum_hi, *bsum_t;       // [NB] sums over blocks of kRowsPerBlock prompts, overwritten by exclusive prefixes
     double *objpart;                   // [NB]
@@ -128,8 +132,7 @@ static Workspace carve(void *base, int64_t N, int32_t ld, bool need_gains, bool 
     w.bsum_hi = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
     w.bsum_t = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)NB));
     w.rowstate = reinterpret_cast<int2 *>(take(sizeof(int2) * (size_t)N));          // everything before this is zeroed per call
-    w.sk_ld = ((ld + 7) / 8 + 7) & ~7;
-    w.sketch = reinterpret_cast<uint16_t *>(take(sizeof(uint16_t) * (size_t)N * (size_t)w.sk_ld));
+    w.pguess = reinterpret_cast<unsigned int *>(take(sizeof(unsigned int) * (size_t)N));
     w.active = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (size_t)N));
     w.objpart = reinterpret_cast<double *>(take(sizeof(double) * (size_t)NB));
     w.cand_key = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * kListCap));
@@ -282,7 +285,8 @@ __device__ __forceinline__ void next_digit(int resolved, int *bits, int *shift) 
 
 // Run by ONE CTA after the sample histogram is complete: scale the rank B to the sample and put the two-bin
 // window around the bin it falls in — towards the upper neighbour when the rank falls in the upper half of
-// that bin's count, else towards the lower one.
+// that bin's count, else towards the lower one — and interpolate a guessed threshold inside that bin.  Both
+// are hints: a poor one costs time, never correctness.
 __device__ void place_window(AllocHeader *hdr, const unsigned long long *hist, int64_t B, int64_t n_sample, int64_t N,
                              long long *s_warp) {
     long long need = (long long)((double)B * (double)n_sample / (double)N + 0.5);
@@ -296,6 +300,11 @@ __device__ void place_window(AllocHeader *hdr, const unsigned long long *hist, i
         int lo = upper_half ? d : d - 1;
         lo = lo < 0 ? 0 : (lo > kBins - kWinBins ? kBins - kWinBins : lo);
         hdr->win_lo = lo;
+        // the guess: the rank's position inside bin d, counted from the top, on a linear scale of the key bits
+        // (bin d holds the high words [d << 19, (d + 1) << 19))
+        const double f = ((double)(need - above) - 0.5) / (double)(count > 0 ? count : 1);
+        const unsigned int down = (unsigned int)(f * 524288.0);
+        hdr->guess_hi = ((unsigned int)(d + 1) << 19) - (down < 524288u ? down : 524287u) - 1u;
     }
 }
 
@@ -344,48 +353,91 @@ select_estimate(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, 
 // ---------------------------------------------------------------------------------------------------
 // Level 0: the one full read.  The matrix is cut into items of 32*E consecutive keys of one row; a warp
 // takes one item at a time and a lane E consecutive keys of it, and the loads of the NEXT item are
-// issued before the current one is processed.  The row is sorted, so a lane's keys usually fall into
-// one 13-bit bin: if that bin is outside the window, one shared-memory atomic counts all E; keys inside
-// the window are counted one by one in the 23-bit bins.  The pass also checks that the row is finite,
-// non-negative and non-increasing (first key below +inf, every key <= its predecessor, compared as
-// unsigned integers), sums the caps, and writes the sketch: the top 16 bits of keys 0, 8, 16, ... (zero
-// beyond the cap).
+// issued before the current one is processed.
+//
+// What is counted.  Only the window matters: the keys ABOVE it (one number) and the keys INSIDE it, per
+// 23-bit bin (2048 fine bins in shared memory).  A row is sorted, so a lane's E keys lie wholly above the
+// window, wholly below it, or (about ten lanes of a 256-key row) need a look at each key.  The per-key look
+// also counts the keys above the guessed threshold; summed over the row that count is stored for level 1,
+// and summed over everything it gives the number of keys above the window:
+//     #above window = #above guess - #(window keys above the guess)      (the guess lies inside the window).
+// The last CTA then knows whether the B-th key falls inside the window — almost always — and if so in which
+// fine bin: 23 bits of the threshold.  If not, a second pass (select_level0_full) builds the plain 13-bit
+// histogram of everything and the selection goes on from 13 bits.
+// A histogram of all 8192 13-bit bins in the same pass was the first design; it cost an index computation and
+// a shared-memory atomic for nearly every key (a row crosses some forty 13-bit bins), 2.4 times the
+// instructions, and those, not memory, set the time.
+// The pass also checks that the row is finite, non-negative and non-increasing and sums the caps.
+
+// E sorted keys of one lane, as high words; `valid` of them exist (the rest were read as 0).  Counts the window
+// keys in s_fine and returns how many keys are above the guess.  ts = prefix23 - W0 is negative below the window
+// and >= kFineBins above it; the guess is t_guess in [0, kFineBins).
+template <int E>
+__device__ __forceinline__ int window_count(const unsigned (&h)[E], int valid, unsigned W0, int t_guess,
+                                            unsigned int *s_fine) {
+    const int ts_first = (int)(h[0] >> 9) - (int)W0, ts_last = (int)(h[E - 1] >> 9) - (int)W0;
+    if (valid >= E && ts_last >= kFineBins) return E;      // the whole lane above the window
+    if (ts_first < 0 || valid <= 0) return 0;              // the whole lane below it
+    int above = 0;
+#pragma unroll
+    for (int m = 0; m < E; ++m) {
+        const int ts = (int)(h[m] >> 9) - (int)W0;
+        if (m < valid) {
+            if ((unsigned)ts < (unsigned)kFineBins) atomicAdd(&s_fine[ts], 1u);
+            above += ts > t_guess;
+        }
+    }
+    return above;
+}
+
 // End of the full-read pass (shared by the pass that reads a materialised matrix and by the fused pass that
-// produces the matrix): merge this CTA's histograms, add up the caps, and let the last CTA select the 13-bit
-// digit of the threshold and, on a window hit, its 23-bit prefix.
-__device__ void level0_finish(AllocHeader *hdr, unsigned long long *hist, unsigned long long *hist_fine,
-                              const unsigned int *s_hist, int win_lo, long long capsum, bool bad, int64_t B,
-                              long long *s_warp) {
+// produces the matrix): merge this CTA's window histogram, add up the caps and the counts above the guess, and
+// let the last CTA locate the threshold's 23-bit prefix inside the window, or declare a miss.
+__device__ void level0_finish(AllocHeader *hdr, unsigned long long *hist_fine, const unsigned int *s_fine, unsigned W0,
+                              int t_guess, long long capsum, long long sum_pg, bool bad, int64_t B, long long *s_warp) {
     if (bad) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);
     __syncthreads();
-    flush_hist(s_hist, hist, kBins);
-    flush_hist(s_hist + kBins, hist_fine, kFineBins);
+    flush_hist(s_fine, hist_fine, kFineBins);
     long long tot;
     block_exclusive_sum(capsum, &tot, s_warp);
     if (threadIdx.x == 0 && tot) atomicAdd(&hdr->sum_cap, (unsigned long long)tot);
+    block_exclusive_sum(sum_pg, &tot, s_warp);
+    if (threadIdx.x == 0 && tot) atomicAdd(&hdr->sum_pguess, (unsigned long long)tot);
     if (last_block(&hdr->ticket[0])) {
         const unsigned long long sum_cap = *(volatile unsigned long long *)&hdr->sum_cap;
-        // the 13-bit counts of the window bins are the sums of their fine bins
-        for (int wb = 0; wb < kWinBins; ++wb) {
-            long long part = 0;
-            for (int f = threadIdx.x; f < kFinePerBin; f += kSelThreads)
-                part += (long long)__ldcg(hist_fine + wb * kFinePerBin + f);
-            long long sum;
-            block_exclusive_sum(part, &sum, s_warp);
-            if (threadIdx.x == 0) hist[win_lo + wb] = (unsigned long long)sum;
+        const long long above_guess = (long long)*(volatile unsigned long long *)&hdr->sum_pguess;
+        // window keys in all, and those above the guess
+        long long part_all = 0, part_up = 0;
+        for (int f = threadIdx.x; f < kFineBins; f += kSelThreads) {
+            const long long v = (long long)__ldcg(hist_fine + f);
+            part_all += v;
+            if (f > t_guess) part_up += v;
         }
+        long long in_window, up;
+        block_exclusive_sum(part_all, &in_window, s_warp);
+        block_exclusive_sum(part_up, &up, s_warp);
+        const long long above_window = above_guess - up;
+        const long long need_w = B - above_window;               // rank of the threshold inside the window
+        const bool hit = B >= 1 && need_w >= 1 && need_w <= in_window;
+        if (threadIdx.x == 0 && (unsigned long long)B > sum_cap) raise_status(&hdr->status, HORA_ERR_INFEASIBLE);
+        long long above = 0, count = 0;
+        const int t = hit ? locate_rank(hist_fine, kFineBins, need_w, &above, &count, s_warp) : -1;
         if (threadIdx.x == 0) {
-            if ((unsigned long long)B > sum_cap) raise_status(&hdr->status, HORA_ERR_INFEASIBLE);
-            hdr->need = B;
+            if (t >= 0) {
+                const unsigned long long prefix23 = (unsigned long long)W0 + (unsigned long long)t;
+                hdr->sel_digit[0] = (int32_t)prefix23;
+                hdr->lv_bits[0] = kDigitBits + kFineBits;
+                hdr->lv_shift[0] = 64 - (kDigitBits + kFineBits);
+                hdr->need = need_w - above;
+                hdr->prefix_key = prefix23 << (64 - (kDigitBits + kFineBits));
+                hdr->resolved = kDigitBits + kFineBits;
+                hdr->bin_count = count;
+                hdr->list_mode = count <= (long long)kListCap ? 1 : 0;
+            } else {
+                hdr->need = B;
+                hdr->l0_miss = B >= 1 ? 1 : 0;                   // the plain 13-bit pass takes over
+            }
         }
-        __threadfence();
-        __syncthreads();
-        find_digit(hdr, hist, kBins, kDigitBits, 51, 0, false, s_warp);
-        const int d0 = hdr->sel_digit[0];
-        const unsigned w = (unsigned)(d0 - win_lo);
-        if (hdr->resolved == kDigitBits && w < (unsigned)kWinBins)        // inside the window: 10 more bits for free
-            find_digit(hdr, hist_fine + w * kFinePerBin, kFinePerBin, kFineBits, 51 - kFineBits, 0, true, s_warp);
-        if (threadIdx.x == 0) hdr->list_mode = (hdr->resolved > 0 && hdr->bin_count <= (long long)kListCap) ? 1 : 0;
     }
 }
 
@@ -433,82 +485,107 @@ __device__ __forceinline__ void level0_fetch(Level0Item<E> &it, const int32_t *_
 
 template <int E>
 __device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t item, int32_t items_per_row,
-                                               int32_t ld, int lane, unsigned int *s_hist, int win_lo,
-                                               uint16_t *__restrict__ sketch, int32_t sk_ld,
-                                               long long *capsum, bool *bad) {
+                                               int lane, unsigned int *s_fine, unsigned W0, int t_guess,
+                                               unsigned int *__restrict__ pguess, long long *capsum, long long *sum_pg,
+                                               bool *bad) {
     const int64_t row = items_per_row == 1 ? item : item / items_per_row;
     const int32_t k0 = (int32_t)(item - row * items_per_row) * (kWarp * E);
     const int32_t k = k0 + lane * E;
     if (lane == 0 && k0 == 0) *capsum += it.capi;
-    // order check; keys past the cap were read as 0, below every valid key, so a ragged item is no special case
+    // Order check, on the values: !(next <= prev) also catches a NaN on either side; keys past the cap were read
+    // as 0.0, below every valid key, so a ragged item is no special case.  The first key of a row must be finite
+    // (lane 0 compares it with the largest finite double), and no key may carry a sign bit (that includes -0.0).
     unsigned long long before = __shfl_up_sync(kFull, it.v[E / 2 - 1].y, 1);
     if (lane == 0) before = it.before;
-    bool wrong = it.v[0].x > before;
+    bool wrong = !(__longlong_as_double((long long)it.v[0].x) <= __longlong_as_double((long long)before));
+    unsigned signs = 0;
+    unsigned h[E];
 #pragma unroll
     for (int p = 0; p < E / 2; ++p) {
-        wrong |= it.v[p].y > it.v[p].x;
-        if (p > 0) wrong |= it.v[p].x > it.v[p - 1].y;
+        const double x = __longlong_as_double((long long)it.v[p].x), y = __longlong_as_double((long long)it.v[p].y);
+        wrong |= !(y <= x);
+        if (p > 0) wrong |= !(x <= __longlong_as_double((long long)it.v[p - 1].y));
+        h[2 * p] = (unsigned)(it.v[p].x >> 32);
+        h[2 * p + 1] = (unsigned)(it.v[p].y >> 32);
+        signs |= h[2 * p] | h[2 * p + 1];
     }
-    *bad |= wrong;
-    if ((k & 7) == 0 && k < ld) sketch[row * (int64_t)sk_ld + (k >> 3)] = (uint16_t)(it.v[0].x >> 48);
-    // one key: a 23-bit bin inside the window, a 13-bit bin outside it.  The two histograms are one array
-    // (fine bins after the coarse ones), so the choice is an index select, not a branch.
-    auto count_key = [&](unsigned long long key) {
-        const unsigned hi = (unsigned)(key >> 32);
-        const unsigned bin = hi >> 19;
-        const unsigned w = bin - (unsigned)win_lo;
-        const unsigned fine = kBins + w * kFinePerBin + ((hi >> (19 - kFineBits)) & (kFinePerBin - 1));
-        atomicAdd(&s_hist[w < (unsigned)kWinBins ? fine : bin], 1u);
-    };
-    const int bin_first = (int)(it.v[0].x >> 51), bin_last = (int)(it.v[E / 2 - 1].y >> 51);
-    if (k0 + kWarp * E <= it.capi) {                           // full item: every lane has E valid keys
-        if (bin_first == bin_last && (unsigned)(bin_first - win_lo) >= (unsigned)kWinBins) {
-            atomicAdd(&s_hist[bin_first], (unsigned int)E);
-        } else {
-#pragma unroll
-            for (int p = 0; p < E / 2; ++p) {
-                count_key(it.v[p].x);
-                count_key(it.v[p].y);
-            }
-        }
-    } else {
-        const int valid = it.capi - k;                         // may be <= 0 or > E
-#pragma unroll
-        for (int p = 0; p < E / 2; ++p) {
-            if (2 * p < valid) count_key(it.v[p].x);
-            if (2 * p + 1 < valid) count_key(it.v[p].y);
-        }
+    *bad |= wrong || (signs >> 31) != 0u;
+    const int above_lane = window_count<E>(h, it.capi - k, W0, t_guess, s_fine);
+    const int above = __reduce_add_sync(kFull, above_lane);
+    if (lane == 0) {
+        *sum_pg += above;
+        if (items_per_row == 1) pguess[row] = (unsigned int)above;
+        else if (above) atomicAdd(pguess + row, (unsigned int)above);   // several items per row: cleared by the host
     }
 }
 
 template <int E, bool VEC2>
-__global__ void __launch_bounds__(kSelThreads, 4)
+__global__ void __launch_bounds__(kSelThreads, 3)
 select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
-              const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist,
-              unsigned long long *hist_fine, uint16_t *__restrict__ sketch, int32_t sk_ld) {
-    __shared__ unsigned int s_hist[kBins + kFineBins];     // 13-bit bins, then the window's 23-bit bins
+              const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist_fine,
+              unsigned int *__restrict__ pguess) {
+    __shared__ unsigned int s_fine[kFineBins];             // the window's 23-bit bins
     __shared__ long long s_warp[kSelThreads / kWarp];
-    for (int b = threadIdx.x; b < kBins + kFineBins; b += kSelThreads) s_hist[b] = 0;
+    for (int b = threadIdx.x; b < kFineBins; b += kSelThreads) s_fine[b] = 0;
     __syncthreads();
     const int lane = lane_id();
-    const int win_lo = hdr->win_lo;
+    const unsigned W0 = (unsigned)hdr->win_lo << kFineBits;
+    int t_guess = (int)(hdr->guess_hi >> 9) - (int)W0;
+    t_guess = t_guess < 0 ? 0 : (t_guess >= kFineBins ? kFineBins - 1 : t_guess);
     const int32_t items_per_row = (ld + kWarp * E - 1) / (kWarp * E);
     const int64_t n_items = N * items_per_row;
     const int64_t item0 = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5);
     const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
-    long long capsum = 0;
+    long long capsum = 0, sum_pg = 0;
     bool bad = false;
     // two items in flight, in two fixed register sets (no copies): A is processed while B's loads land
     Level0Item<E> A, Bq;
     level0_fetch<E, VEC2>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item0, lane, &bad);
     for (int64_t item = item0; item < n_items; item += 2 * stride) {
         level0_fetch<E, VEC2>(Bq, cap, cap_scalar, n_items, items_per_row, ld, gains, item + stride, lane, &bad);
-        level0_process<E>(A, item, items_per_row, ld, lane, s_hist, win_lo, sketch, sk_ld, &capsum, &bad);
+        level0_process<E>(A, item, items_per_row, lane, s_fine, W0, t_guess, pguess, &capsum, &sum_pg, &bad);
         level0_fetch<E, VEC2>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item + 2 * stride, lane, &bad);
         if (Bq.capi >= 0)
-            level0_process<E>(Bq, item + stride, items_per_row, ld, lane, s_hist, win_lo, sketch, sk_ld, &capsum, &bad);
+            level0_process<E>(Bq, item + stride, items_per_row, lane, s_fine, W0, t_guess, pguess, &capsum, &sum_pg, &bad);
     }
-    level0_finish(hdr, hist, hist_fine, s_hist, win_lo, capsum, bad, B, s_warp);
+    level0_finish(hdr, hist_fine, s_fine, W0, t_guess, capsum, sum_pg, bad, B, s_warp);
+}
+
+// The plain pass, for the rare case that the window missed: a warp per row, every key counted on its top 13
+// bits; the last CTA selects that digit and the selection goes on from there.  (The counts above the guess
+// that level 0 stored mean little then; level 1 falls back to searching the rows.)
+__global__ void __launch_bounds__(kSelThreads)
+select_level0_full(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
+                   const double *__restrict__ gains, AllocHeader *hdr, unsigned long long *hist) {
+    __shared__ unsigned int s_hist[kBins];
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    if (*(volatile int32_t *)&hdr->status != 0 || hdr->l0_miss == 0) return;
+    for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
+    __syncthreads();
+    const int lane = lane_id();
+    const int64_t stride = (int64_t)gridDim.x * (kSelThreads / kWarp);
+    for (int64_t row = (int64_t)blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5); row < N; row += stride) {
+        int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
+        capi = capi < 0 ? 0 : (capi > ld ? ld : capi);
+        const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
+        for (int32_t k0 = 0; k0 < capi; k0 += 8 * kWarp) {      // eight coalesced loads in flight per lane
+            unsigned long long key[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int32_t j = k0 + u * kWarp + lane;
+                key[u] = j < capi ? __ldg(keys + j) : 0ull;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (k0 + u * kWarp + lane < capi) atomicAdd(&s_hist[(int)(key[u] >> 51) & (kBins - 1)], 1u);
+        }
+    }
+    __syncthreads();
+    flush_hist(s_hist, hist, kBins);
+    if (last_block(&hdr->ticket[14])) {
+        find_digit(hdr, hist, kBins, kDigitBits, 51, 0, false, s_warp);
+        if (threadIdx.x == 0) hdr->list_mode = (hdr->resolved > 0 && hdr->bin_count <= (long long)kListCap) ? 1 : 0;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -534,42 +611,35 @@ struct CoarseTap {
     __device__ __forceinline__ void begin_row(int64_t, int32_t) {}
 };
 
-// the level-0 bookkeeping: window/coarse histogram and the sketch
+// the level-0 bookkeeping: window histogram and the count of keys above the guessed threshold
 template <int E>
 struct Level0Tap {
     unsigned long long key[E];
-    unsigned int *s_hist;
-    uint16_t *sketch;
-    uint16_t *sk_row;              // sketch row of the prompt being built
-    int32_t sk_ld;
-    int win_lo;
+    unsigned int *s_fine;
+    unsigned int *pguess;
+    unsigned int *pg_row;          // the count of the prompt being built
+    unsigned W0;
+    int t_guess;
+    unsigned int row_above;        // lane 0: keys above the guess in the chunks of this row so far
+    long long sum_pg;              // lane 0: the same over all rows of this warp
     long long capsum;              // lane 0 of every warp: caps of the rows it built
     __device__ __forceinline__ void begin_row(int64_t row, int32_t capi) {
-        sk_row = sketch + row * (int64_t)sk_ld;
+        pg_row = pguess + row;
+        row_above = 0;
         if ((threadIdx.x & 31) == 0) capsum += capi;
     }
     __device__ __forceinline__ void pair(int m, double g0, double g1) {
         key[m] = (unsigned long long)__double_as_longlong(g0);
         key[m + 1] = (unsigned long long)__double_as_longlong(g1);
     }
-    __device__ __forceinline__ void count_key(unsigned long long k64) const {
-        const unsigned hi = (unsigned)(k64 >> 32);
-        const unsigned bin = hi >> 19;
-        const unsigned w = bin - (unsigned)win_lo;
-        const unsigned fine = kBins + w * kFinePerBin + ((hi >> (19 - kFineBits)) & (kFinePerBin - 1));
-        atomicAdd(&s_hist[w < (unsigned)kWinBins ? fine : bin], 1u);
-    }
-    __device__ __forceinline__ void finish(int32_t, int32_t k, int32_t capi, int32_t ld) {
-        if ((k & 7) == 0 && k < ld) sk_row[k >> 3] = (uint16_t)(key[0] >> 48);   // masked entries are 0.0: sketch 0
-        const int valid = capi - k;
-        const unsigned bin_first = (unsigned)(key[0] >> 51), bin_last = (unsigned)(key[E - 1] >> 51);
-        if (valid >= E && bin_first == bin_last && bin_first - (unsigned)win_lo >= (unsigned)kWinBins) {
-            atomicAdd(&s_hist[bin_first], (unsigned int)E);
-        } else {
+    __device__ __forceinline__ void finish(int32_t, int32_t k, int32_t capi, int32_t) {
+        unsigned h[E];
 #pragma unroll
-            for (int m = 0; m < E; ++m)
-                if (m < valid) count_key(key[m]);
-        }
+        for (int m = 0; m < E; ++m) h[m] = (unsigned)(key[m] >> 32);
+        const int above = __reduce_add_sync(kFull, window_count<E>(h, capi - k, W0, t_guess, s_fine));
+        row_above += (unsigned int)above;
+        sum_pg += above;
+        if ((threadIdx.x & 31) == 0) *pg_row = row_above;      // the row's chunks come one after another in this warp
     }
 };
 
@@ -614,21 +684,24 @@ __global__ void __launch_bounds__(kSelThreads, 3)
 gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
                    const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
                    int64_t N, int32_t ld, double *__restrict__ gains, int64_t B, AllocHeader *hdr,
-                   unsigned long long *hist, unsigned long long *hist_fine, uint16_t *__restrict__ sketch,
-                   int32_t sk_ld) {
-    extern __shared__ unsigned int s_hist[];               // kBins + kFineBins words (dynamic: 40 KiB)
+                   unsigned long long *hist_fine, unsigned int *__restrict__ pguess) {
+    __shared__ unsigned int s_fine[kFineBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
-    for (int b = threadIdx.x; b < kBins + kFineBins; b += kSelThreads) s_hist[b] = 0;
+    for (int b = threadIdx.x; b < kFineBins; b += kSelThreads) s_fine[b] = 0;
     __syncthreads();
     Level0Tap<E> tap;
-    tap.s_hist = s_hist;
-    tap.sketch = sketch;
-    tap.sk_row = sketch;
-    tap.sk_ld = sk_ld;
-    tap.win_lo = hdr->win_lo;
+    tap.s_fine = s_fine;
+    tap.pguess = pguess;
+    tap.pg_row = pguess;
+    tap.W0 = (unsigned)hdr->win_lo << kFineBits;
+    const int t_guess = (int)(hdr->guess_hi >> 9) - (int)tap.W0;
+    tap.t_guess = t_guess < 0 ? 0 : (t_guess >= kFineBins ? kFineBins - 1 : t_guess);
+    tap.row_above = 0;
+    tap.sum_pg = 0;
     tap.capsum = 0;
     gains_rows_cta<E, VEC2>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, &hdr->status, tap);
-    level0_finish(hdr, hist, hist_fine, s_hist, tap.win_lo, tap.capsum, false, B, s_warp);
+    level0_finish(hdr, hist_fine, s_fine, tap.W0, tap.t_guess, tap.capsum, (threadIdx.x & 31) == 0 ? tap.sum_pg : 0, false, B,
+                  s_warp);
 }
 
 // U_i(Delta) from the row's own entry: the product in U_i(Delta) = 1 - prod_{j<Delta} (b+j)/(a+b+j) is
@@ -639,22 +712,30 @@ __device__ __forceinline__ double utility_from_gain(double g, double a, double b
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Level 1: a thread per row.  r bits of the threshold are known (23 after a window hit, else 13); call
-// P that prefix.  The sketch holds the top 16 bits of the first (largest) key of every group of 8 keys.
-// Compared at min(r, 16) bits: groups whose first key is above P form a prefix of G1 groups, groups whose
-// first key is above or equal a prefix of G2 >= G1 groups.  Every key with prefix P therefore sits in
-// groups G1-1 .. G2-1, and so does the boundary between "above" and "equal"; the thread reads only those
-// keys (one or two groups after a window hit) and classifies them on all r bits.  The keys with prefix P
-// go to the candidate list (list mode: one slot reservation per CTA and 256 rows) or are histogrammed on
-// the next digit, their rows appended to the active list.
-// A warp per row was tried first: with a million rows the per-row issue slots, not memory, set its time;
-// for the same reason the sketch entries are compared two at a time (they are 15-bit numbers, so
-// (e | 0x8000) - p keeps bit 15 exactly when e >= p, in both halves of a word at once).
-__device__ __forceinline__ void sketch_count(unsigned w, unsigned mask2, unsigned Pp, unsigned &acc_ge,
-                                             unsigned &acc_gt) {
-    const unsigned d = ((w & mask2) | 0x80008000u) - Pp;      // per half: 0x8000 + e - p, never borrows
-    acc_ge += (d >> 15) & 0x00010001u;
-    acc_gt += ((d - 0x00010001u) >> 15) & 0x00010001u;        // e - p - 1 >= 0
+// Level 1: a thread per row.  r bits of the threshold are known (23 after a window hit, else 13); call P that
+// prefix.  The row is non-increasing, so with p_hi = #keys above P and p_lo = #keys above or equal, the keys
+// that carry P are the segment [p_hi, p_lo).  Level 0 left a guess of p_hi (the keys above a threshold
+// interpolated from the sample); the thread reads the 8 keys around it — two sectors — and is done when the
+// first of them is above P (or is the row's first key) and the last of them is below P (or is the row's
+// last).  Otherwise it widens the range a few times, and after that two binary searches over the row find
+// the segment.  The keys of the segment go to the candidate list (list mode: one slot reservation per warp
+// that has any) or are histogrammed on the next digit, their rows appended to the active list.
+// A per-row sketch of every 8th key, written by level 0 and scanned here, was the first design: the scan
+// cost more issue slots (700 instructions per row) and memory (200 bytes per row) than the whole search here.
+
+// prefix of a key: its top r bits, r <= 32
+__device__ __forceinline__ unsigned key_prefix(unsigned long long key, int r) { return (unsigned)(key >> 32) >> (32 - r); }
+
+// first index in [0, n) whose prefix is <= P (STRICT false) or < P (STRICT true); n if none
+template <bool STRICT>
+__device__ __forceinline__ int32_t first_not_above(const unsigned long long *__restrict__ keys, int32_t n, unsigned P, int r) {
+    int32_t lo = 0, hi = n;
+    while (lo < hi) {
+        const int32_t mid = (lo + hi) >> 1;
+        const unsigned kp = key_prefix(__ldg(keys + mid), r);
+        if (STRICT ? kp >= P : kp > P) lo = mid + 1; else hi = mid;
+    }
+    return lo;
 }
 
 template <bool VEC2>
@@ -662,12 +743,11 @@ __global__ void __launch_bounds__(kSelThreads)
 select_level1(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
               const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N,
               int32_t ld, const double *__restrict__ gains, AllocHeader *hdr, unsigned long long *hist1,
-              const uint16_t *__restrict__ sketch, int32_t sk_ld, int2 *__restrict__ rowstate,
+              const unsigned int *__restrict__ pguess, int2 *__restrict__ rowstate,
               int32_t *__restrict__ active, unsigned long long *__restrict__ cand_key,
               int32_t *__restrict__ cand_row, long long *bsum_hi, double *__restrict__ objrow) {
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
-    __shared__ unsigned int s_base;
     if (*(volatile int32_t *)&hdr->status != 0) return;
     const bool list = hdr->list_mode != 0;
     if (!list) {
@@ -677,9 +757,6 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
     const int lane = lane_id();
     const int r = hdr->resolved;                                 // 13 or 23: the prefix lies in the key's high word
     const unsigned P = (unsigned)(hdr->prefix_key >> 32) >> (32 - r);
-    const int sk_shift = r < 16 ? 16 - r : 0;                    // sketch entries compared at min(r, 16) bits
-    const unsigned mask2 = ((0xFFFFu << sk_shift) & 0xFFFFu) * 0x00010001u;
-    const unsigned Pp = ((unsigned)(hdr->prefix_key >> 48) * 0x00010001u) & mask2;
     int bits, shift;
     next_digit(r, &bits, &shift);
     const unsigned long long digit_mask = (1ull << bits) - 1ull;
@@ -690,78 +767,83 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
         int32_t p_hi = 0, n_eq = 0;
         const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains);
         if (row < N) {
+            const unsigned int guess = __ldg(pguess + row);
             const Posterior post = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row);
             bad |= !post.ok;
             const int32_t capi = post.cap;                       // 0 for an invalid row
-            const int n_groups = (capi + 7) >> 3;
-            // the sketch row is 16-byte aligned and padded to a multiple of 8 entries
-            const uint4 *sk4 = reinterpret_cast<const uint4 *>(sketch + row * (int64_t)sk_ld);
-            int G1 = 0, G2 = 0;
-            for (int g0 = 0; g0 < n_groups; g0 += 32) {          // 32 entries (four independent 16-byte loads) at a time
-                uint4 v[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    v[u] = (g0 + 8 * u < n_groups) ? __ldg(sk4 + (g0 >> 3) + u) : make_uint4(0u, 0u, 0u, 0u);
-                unsigned acc_ge = 0, acc_gt = 0;                 // two 16-bit counters each
-                if (g0 + 32 <= n_groups) {
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        sketch_count(v[u].x, mask2, Pp, acc_ge, acc_gt);
-                        sketch_count(v[u].y, mask2, Pp, acc_ge, acc_gt);
-                        sketch_count(v[u].z, mask2, Pp, acc_ge, acc_gt);
-                        sketch_count(v[u].w, mask2, Pp, acc_ge, acc_gt);
-                    }
-                } else {                                         // ragged end: entries past the last group do not count
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int left = n_groups - (g0 + 8 * u + 2 * i);
-                            const unsigned valid = left >= 2 ? 0xFFFFFFFFu : (left == 1 ? 0x0000FFFFu : 0u);
-                            unsigned ge = 0, gt = 0;
-                            sketch_count(w[i], mask2, Pp, ge, gt);
-                            acc_ge += ge & valid & 0x00010001u;
-                            acc_gt += gt & valid & 0x00010001u;
-                        }
-                    }
-                }
-                G1 += (int)((acc_gt & 0xFFFFu) + (acc_gt >> 16));
-                G2 += (int)((acc_ge & 0xFFFFu) + (acc_ge >> 16));
-                if (G2 < g0 + 32) break;                         // entries only decrease: the later ones are below P
-            }
-            const int32_t lo = G1 > 0 ? (G1 - 1) << 3 : 0;
-            const int32_t hi = (G2 << 3) > capi ? capi : (G2 << 3);
             keys += row * (int64_t)ld;
+            // the 8 keys around the guess, from a 4-key boundary (two whole sectors of an aligned row), at
+            // least two keys on either side of it
+            const int32_t j0 = guess < (unsigned)capi ? (int32_t)guess : capi;
+            int32_t ws = (j0 > 2 ? j0 - 2 : 0) & ~3;
+            int32_t we = ws + 8 < capi ? ws + 8 : capi;
             int32_t n_gt = 0;
-            for (int32_t j0 = lo; j0 < hi; j0 += 8) {            // one group of 8 keys (independent loads) at a time
-                unsigned long long key[8];
-                if (VEC2) {                                      // j0 is a multiple of 8: 16-byte aligned in an aligned row
+            unsigned kp_first = 0, kp_last = 0;
+            {
+                unsigned kp[8];
+                if (VEC2) {
 #pragma unroll
                     for (int u = 0; u < 8; u += 2) {
                         ulonglong2 t = make_ulonglong2(0ull, 0ull);
-                        if (j0 + u < hi) t = __ldg(reinterpret_cast<const ulonglong2 *>(keys + j0 + u));
-                        key[u] = t.x;
-                        key[u + 1] = t.y;
+                        if (ws + u < we) t = __ldg(reinterpret_cast<const ulonglong2 *>(keys + ws + u));
+                        kp[u] = key_prefix(t.x, r);
+                        kp[u + 1] = key_prefix(t.y, r);
                     }
                 } else {
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) key[u] = (j0 + u < hi) ? __ldg(keys + j0 + u) : 0ull;
+                    for (int u = 0; u < 8; ++u) kp[u] = ws + u < we ? key_prefix(__ldg(keys + ws + u), r) : 0u;
                 }
-                int32_t eq_here = 0;
+                kp_first = kp[0];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                    const unsigned kp = (unsigned)(key[u] >> 32) >> (32 - r);
-                    const bool in = j0 + u < hi;
-                    n_gt += in && kp > P;
-                    const bool eq = in && kp == P;
-                    eq_here += eq;
-                    if (!list && eq) atomicAdd(&s_hist[(key[u] >> shift) & digit_mask], 1u);
+                    const bool in = ws + u < we;
+                    n_gt += in && kp[u] > P;
+                    n_eq += in && kp[u] == P;
+                    if (ws + u == we - 1) kp_last = kp[u];
                 }
-                n_eq += eq_here;
-                if (n_eq > 0 && eq_here == 0) break;             // the row is sorted: past the segment
             }
-            p_hi = lo + n_gt;
+            // done when everything before the keys read is above P and everything after them below it;
+            // else widen by 8 keys on the open side, a few times, before falling back to a search of the row
+            bool left_ok = ws == 0 || (we > ws && kp_first > P);
+            bool right_ok = we == capi || kp_last < P;
+            for (int widen = 0; widen < 3 && !(left_ok && right_ok); ++widen) {
+                if (!left_ok) {                                  // the 8 keys before (independent loads)
+                    unsigned kp[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) kp[u] = ws - 1 - u >= 0 ? key_prefix(__ldg(keys + ws - 1 - u), r) : 0u;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (ws - 1 - u >= 0) {
+                            n_gt += kp[u] > P;
+                            n_eq += kp[u] == P;
+                            kp_first = kp[u];
+                        }
+                    }
+                    ws = ws > 8 ? ws - 8 : 0;
+                    left_ok = ws == 0 || kp_first > P;
+                }
+                if (!right_ok) {                                 // the 8 keys after
+                    unsigned kp[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) kp[u] = we + u < capi ? key_prefix(__ldg(keys + we + u), r) : 0u;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (we + u < capi) {
+                            n_gt += kp[u] > P;
+                            n_eq += kp[u] == P;
+                            kp_last = kp[u];
+                        }
+                    }
+                    we = we + 8 < capi ? we + 8 : capi;
+                    right_ok = we == capi || kp_last < P;
+                }
+            }
+            if (left_ok && right_ok) {
+                p_hi = ws + n_gt;
+            } else {                                             // a poor guess, or a long segment
+                p_hi = first_not_above<false>(keys, capi, P, r);
+                n_eq = first_not_above<true>(keys + p_hi, capi - p_hi, P, r);
+            }
             rowstate[row] = make_int2(p_hi, p_hi + n_eq);
             if (objrow != nullptr) {
                 // no key in the threshold's bin: Delta_i = p_hi is final, and g_i(Delta_i) was just read (L1)
@@ -771,19 +853,29 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
                                  : 0.0;
                 objrow[row] = u;
             }
+            if (!list)                                           // digit route: the segment's keys on the next digit
+                for (int32_t j = 0; j < n_eq; ++j)
+                    atomicAdd(&s_hist[(__ldg(keys + p_hi + j) >> shift) & digit_mask], 1u);
         }
         if (list) {
-            // one block scan gives the step's sum of p_hi (upper half) and the slots of its keys (lower half);
-            // one reservation per CTA and step; the order of the list does not matter to anything
-            long long tot;
-            const long long excl = block_exclusive_sum(((long long)p_hi << 32) | (long long)n_eq, &tot, s_warp);
-            if (threadIdx.x == 0 && (tot >> 32) != 0)
-                atomicAdd(reinterpret_cast<unsigned long long *>(bsum_hi) + base / kRowsPerBlock, (unsigned long long)(tot >> 32));
-            const unsigned int n_new = (unsigned int)(tot & 0xFFFFFFFFll);
-            if (n_new > 0) {
-                if (threadIdx.x == 0) s_base = atomicAdd(&hdr->n_cand, n_new);
-                __syncthreads();
-                const long long slot = (long long)s_base + (excl & 0xFFFFFFFFll);
+            // per warp: one addition to the block sum of p_hi, one slot reservation for the warp's keys (the
+            // order of the list does not matter to anything).  Nothing here waits for another warp.
+            const int hi_sum = __reduce_add_sync(kFull, p_hi);
+            if (lane == 0 && hi_sum != 0)
+                atomicAdd(reinterpret_cast<unsigned long long *>(bsum_hi) + base / kRowsPerBlock, (unsigned long long)hi_sum);
+            const unsigned has = __ballot_sync(kFull, n_eq > 0);
+            if (has) {
+                int inc = n_eq;                                  // inclusive scan of n_eq over the warp
+#pragma unroll
+                for (int d = 1; d < kWarp; d <<= 1) {
+                    const int t = __shfl_up_sync(kFull, inc, d);
+                    if (lane >= d) inc += t;
+                }
+                const int n_new = __shfl_sync(kFull, inc, kWarp - 1);
+                unsigned int slot0 = 0;
+                if (lane == 0) slot0 = atomicAdd(&hdr->n_cand, (unsigned int)n_new);
+                slot0 = __shfl_sync(kFull, slot0, 0);
+                const long long slot = (long long)slot0 + (inc - n_eq);
                 for (int32_t j = 0; j < n_eq; ++j) {
                     const unsigned long long key = __ldg(keys + p_hi + j);
                     if (slot + j < kListCap) {
@@ -1513,14 +1605,10 @@ template <int E>
 static void launch_level0(bool vec2, int grid, cudaStream_t s, const int32_t *cap, int32_t cap_scalar, int64_t N,
                           int32_t ld, const double *gains, int64_t B, const Workspace &w) {
     if (vec2)
-        select_level0<E, true><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_coarse,
-                                                            w.hist_fine, w.sketch, w.sk_ld);
+        select_level0<E, true><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_fine, w.pguess);
     else
-        select_level0<E, false><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_coarse,
-                                                             w.hist_fine, w.sketch, w.sk_ld);
+        select_level0<E, false><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_fine, w.pguess);
 }
-
-constexpr size_t kFusedSmem = sizeof(unsigned int) * (kBins + kFineBins);
 
 template <int E>
 static cudaError_t launch_fused(bool vec2, bool estimate, int grid_est, int64_t every, int grid, cudaStream_t s,
@@ -1530,14 +1618,13 @@ static cudaError_t launch_fused(bool vec2, bool estimate, int grid_est, int64_t 
     if (estimate)
         select_estimate_fused<E><<<grid_est, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N,
                                                                   ld, every, B, w.hdr, w.hist_est);
-    auto go = [&](auto kernel) -> cudaError_t {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmem);
-        if (e != cudaSuccess) return e;
-        kernel<<<grid, kSelThreads, kFusedSmem, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, w.gains,
-                                                     B, w.hdr, w.hist_coarse, w.hist_fine, w.sketch, w.sk_ld);
-        return cudaGetLastError();
-    };
-    return vec2 ? go(gains_level0_fused<E, true>) : go(gains_level0_fused<E, false>);
+    if (vec2)
+        gains_level0_fused<E, true><<<grid, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
+                                                                 w.gains, B, w.hdr, w.hist_fine, w.pguess);
+    else
+        gains_level0_fused<E, false><<<grid, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
+                                                                  w.gains, B, w.hdr, w.hist_fine, w.pguess);
+    return cudaGetLastError();
 }
 
 // CTAs of the cooperative tail on the current device: what fits at once, at most kTailPerSm per SM (0 on failure).
@@ -1611,6 +1698,8 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         if (cudaMemsetAsync(w.tkeys, 0, tb, s) != cudaSuccess) return HORA_ERR_CUDA;
     }
     const bool fused = gains == nullptr;                  // no matrix given: build it and count its keys in one pass
+    if (!fused && ld > 256 && B > 0)                      // rows of several items add up their counts with atomics
+        if (cudaMemsetAsync(w.pguess, 0, sizeof(unsigned int) * (size_t)N, s) != cudaSuccess) return HORA_ERR_CUDA;
     if (fused) gains = w.gains;
     const bool vec2 = (ld % 2 == 0) && ((reinterpret_cast<uintptr_t>(gains) & 15u) == 0);
     const int rows_per_cta = kSelThreads / kWarp;
@@ -1620,7 +1709,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     mark_stage(0, s);
     if (B > 0 && !fused)
         select_estimate<<<grid_est, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, every, gains, B, w.hdr, w.hist_est);
-    const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 4);
+    const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 3);
     const int grid1 = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     const cudaEvent_t prof_start = g_prof_start.load(std::memory_order_relaxed);
     const cudaEvent_t prof_stop = g_prof_stop.load(std::memory_order_relaxed);
@@ -1644,6 +1733,8 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         launch_level0<2>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
     }
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_stop, s);
+    if (B > 0)                                            // stands down at once unless the window missed
+        select_level0_full<<<grid0, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, w.hdr, w.hist_coarse);
     mark_stage(2, s);
     const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     // utilities of the rows whose Delta is final after level 1 are evaluated there (not in exact mode, where the
@@ -1652,11 +1743,11 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     if (B > 0) {
         if (vec2)
             select_level1<true><<<grid1, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains,
-                                                              w.hdr, w.hist_lv + kBins, w.sketch, w.sk_ld, w.rowstate,
+                                                              w.hdr, w.hist_lv + kBins, w.pguess, w.rowstate,
                                                               w.active, w.cand_key, w.cand_row, w.bsum_hi, objrow);
         else
             select_level1<false><<<grid1, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains,
-                                                               w.hdr, w.hist_lv + kBins, w.sketch, w.sk_ld, w.rowstate,
+                                                               w.hdr, w.hist_lv + kBins, w.pguess, w.rowstate,
                                                                w.active, w.cand_key, w.cand_row, w.bsum_hi, objrow);
         mark_stage(3, s);
         {
@@ -1697,7 +1788,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
                                                w.rowstate, objrow, w.bsum_hi, w.bsum_t, w.objpart, NB, delta, G,
                                                group_offsets, out_vec, info_dev);
     mark_stage(6, s);
-    count_launches(B > 0 ? (exact ? 8 : 5) : 3);
+    count_launches(B > 0 ? (exact ? 9 : 6) : 3);
     return cuda_ok(cudaGetLastError());
 }
 
