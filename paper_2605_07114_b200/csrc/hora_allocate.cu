@@ -56,6 +56,8 @@ constexpr int kLevels = 5;                   // level 0 (full read) + four digit
 constexpr int kListCap = 65536;              // candidates the single-CTA list selection accepts
 constexpr int kListSmall = 1536;               // keys of the list that later sweeps keep in shared memory
 constexpr int kTailPerSm = 4;                 // CTAs of the cooperative tail per SM
+constexpr int kLevel1PerSm = 5;               // CTAs of level 1 per SM: the grid is exactly one resident wave (a sixth
+                                              // CTA per SM that has to wait for a slot cost 25 us of 77 at 2^20 rows)
 constexpr int kBins = 8192;                  // 13-bit digits
 constexpr int kDigitBits = 13;
 constexpr int kWinBins = 2;                  // coarse bins covered by the fine window of level 0
@@ -739,7 +741,7 @@ __device__ __forceinline__ int32_t first_not_above(const unsigned long long *__r
 }
 
 template <bool VEC2>
-__global__ void __launch_bounds__(kSelThreads)
+__global__ void __launch_bounds__(kSelThreads, kLevel1PerSm)
 select_level1(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
               const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N,
               int32_t ld, const double *__restrict__ gains, AllocHeader *hdr, unsigned long long *hist1,
@@ -1710,7 +1712,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     if (B > 0 && !fused)
         select_estimate<<<grid_est, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, every, gains, B, w.hdr, w.hist_est);
     const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 3);
-    const int grid1 = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
+    const int grid1 = clamp_grid((N + kSelThreads - 1) / kSelThreads, kLevel1PerSm);
     const cudaEvent_t prof_start = g_prof_start.load(std::memory_order_relaxed);
     const cudaEvent_t prof_stop = g_prof_stop.load(std::memory_order_relaxed);
     if (!fused) mark_stage(1, s);                         // (the fused pass launches its own estimate)
