@@ -104,7 +104,7 @@ hora_status_t hora_gains(const double *alpha, const double *beta, double alpha0,
  * current marginal gain" without running them one by one: because every row of gains decreases,
  * that result is the set of the B largest candidates g_i(Delta), Delta <= cap_i.  The call finds the
  * B-th largest value lambda by a multi-level radix selection on the 64-bit patterns of the gains
- * (one full read of the matrix, then per-row segment refinement), counts per row the candidates
+ * (one full read of the matrix, then a short look at each row around a guessed position), counts per row the candidates
  * above lambda, and gives the remaining B - n_above rollouts to the tied candidates in order of
  * increasing prompt index (then increasing Delta).  Outputs:
  *
@@ -152,10 +152,11 @@ hora_status_t hora_allocate(const double *alpha, const double *beta, double alph
  *
  *   - Size limit: hora_allocate_workspace_bytes(N, ld, gains == NULL, flags) must not exceed
  *     hora_allocate_static_capacity(); otherwise HORA_ERR_WORKSPACE is returned and nothing is enqueued.
- *     With a materialised gains matrix and ld = 256 that admits about 1e5 prompts; with gains == NULL the
+ *     With a materialised gains matrix that admits about 2.5e5 prompts; with gains == NULL the
  *     matrix itself must fit, so only small problems (N*ld*8 bytes well under 8 MiB) qualify.
  *   - First use: the first call on each device looks up the array's device address (cudaGetSymbolAddress)
- *     with that device current, and caches it.  Make that first call outside any stream capture.
+ *     with that device current, and caches it (as hora_allocate caches, per device, how many thread blocks of
+ *     its cooperative kernel fit at once).  Make that first call outside any stream capture.
  *   - Sharing: every call on a device uses the same array.  It keeps whatever the previous call left there;
  *     each call clears the parts it needs zeroed before using them, so back-to-back calls on one stream
  *     are fine.  Two calls that overlap on the GPU (different streams, or different host threads without
