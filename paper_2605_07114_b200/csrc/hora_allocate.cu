@@ -358,8 +358,8 @@ select_estimate(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, 
 // issued before the current one is processed.
 //
 // What is counted.  Only the window matters: the keys ABOVE it (one number) and the keys INSIDE it, per
-// 23-bit bin (2048 fine bins in shared memory).  A row is sorted, so a lane's E keys lie wholly above the
-// window, wholly below it, or (about ten lanes of a 256-key row) need a look at each key.  The per-key look
+// 23-bit bin (2048 fine bins in shared memory).  A row is sorted, so a 64-key slice of it lies wholly above the
+// window, wholly below it, or (one or two slices of a 256-key row) needs a look at each key.  The per-key look
 // also counts the keys above the guessed threshold; summed over the row that count is stored for level 1,
 // and summed over everything it gives the number of keys above the window:
 //     #above window = #above guess - #(window keys above the guess)      (the guess lies inside the window).
@@ -443,9 +443,14 @@ __device__ void level0_finish(AllocHeader *hdr, unsigned long long *hist_fine, c
     }
 }
 
+// One item in registers.  The item is cut into E/2 slices of 64 consecutive keys; of every slice a lane holds
+// the pair of keys 2*lane, 2*lane + 1 (one 16-byte load, 512 contiguous bytes per warp instruction).  A slice is
+// thus spread over all lanes, and one that lies wholly above or wholly below the window is settled by a vote
+// instead of a look at each key; with E consecutive keys per lane the ten lanes of a row that intersect the
+// window made every warp run the per-key code for all its keys (121 of 250 instructions per row).
 template <int E>
 struct Level0Item {
-    ulonglong2 v[E / 2];           // this lane's E consecutive keys, in pairs (E is even)
+    ulonglong2 v[E / 2];           // slice p: keys k0 + 64 p + 2 lane, + 1
     unsigned long long before;     // lane 0 only: the key just before this item (or the largest finite key)
     int32_t capi;                  // the row's cap; -1 marks "no item"
 };
@@ -461,28 +466,48 @@ __device__ __forceinline__ void level0_fetch(Level0Item<E> &it, const int32_t *_
     int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
     if (capi < 0 || capi > ld) { *bad = true; capi = 0; }
     it.capi = capi;
-    const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-    const int32_t k = k0 + lane * E;
+    const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld + k0 + 2 * lane;
     if (VEC2 && k0 + kWarp * E <= capi) {                      // the whole item lies below the cap: plain loads
 #pragma unroll
-        for (int p = 0; p < E / 2; ++p) it.v[p] = __ldg(reinterpret_cast<const ulonglong2 *>(keys + k) + p);
+        for (int p = 0; p < E / 2; ++p) it.v[p] = __ldg(reinterpret_cast<const ulonglong2 *>(keys) + 32 * p);
     } else {                                                   // ragged: keys past the cap read as 0
 #pragma unroll
         for (int p = 0; p < E / 2; ++p) {
+            const int32_t k = k0 + 64 * p + 2 * lane;
             it.v[p] = make_ulonglong2(0ull, 0ull);
             if (VEC2) {
-                if (k + 2 * p < capi) {
-                    it.v[p] = __ldg(reinterpret_cast<const ulonglong2 *>(keys + k) + p);
-                    if (k + 2 * p + 1 >= capi) it.v[p].y = 0ull;
+                if (k < capi) {
+                    it.v[p] = __ldg(reinterpret_cast<const ulonglong2 *>(keys) + 32 * p);
+                    if (k + 1 >= capi) it.v[p].y = 0ull;
                 }
             } else {
-                if (k + 2 * p < capi) it.v[p].x = __ldg(keys + k + 2 * p);
-                if (k + 2 * p + 1 < capi) it.v[p].y = __ldg(keys + k + 2 * p + 1);
+                if (k < capi) it.v[p].x = __ldg(keys + 64 * p);
+                if (k + 1 < capi) it.v[p].y = __ldg(keys + 64 * p + 1);
             }
         }
     }
     it.before = kKeyInf - 1;
-    if (lane == 0 && k0 > 0 && k0 < capi) it.before = __ldg(keys + k0 - 1);
+    if (lane == 0 && k0 > 0 && k0 < capi) it.before = __ldg(keys - 1);
+}
+
+// Exact order check of an item, on the values: !(next <= prev) also catches a NaN on either side.  Keys past the
+// cap were read as 0.0, below every valid key.  Used for ragged items and wherever the quick check on the high
+// words found two equal ones.
+template <int E>
+__device__ __forceinline__ bool level0_order_exact(const Level0Item<E> &it, int lane) {
+    bool wrong = false;
+    double prev_y = 0.0;                                       // lane 31: its y of the previous slice
+#pragma unroll
+    for (int p = 0; p < E / 2; ++p) {
+        const double x = __longlong_as_double((long long)it.v[p].x), y = __longlong_as_double((long long)it.v[p].y);
+        const double nx = __longlong_as_double((long long)__shfl_sync(kFull, it.v[p].x, (lane + 1) & 31));
+        wrong |= !(y <= x);
+        if (lane < 31) wrong |= !(nx <= y);                    // the next lane's x follows this lane's y
+        else if (p > 0) wrong |= !(nx <= prev_y);              // lane 0's x of this slice follows lane 31's y of the last
+        prev_y = y;
+    }
+    if (lane == 0) wrong |= !(__longlong_as_double((long long)it.v[0].x) <= __longlong_as_double((long long)it.before));
+    return wrong;
 }
 
 template <int E>
@@ -492,28 +517,70 @@ __device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t 
                                                bool *bad) {
     const int64_t row = items_per_row == 1 ? item : item / items_per_row;
     const int32_t k0 = (int32_t)(item - row * items_per_row) * (kWarp * E);
-    const int32_t k = k0 + lane * E;
+    const int32_t nvalid = it.capi - k0;                       // keys of this item below the cap (may be <= 0 or > 32 E)
+    const bool full = nvalid >= kWarp * E;
     if (lane == 0 && k0 == 0) *capsum += it.capi;
-    // Order check, on the values: !(next <= prev) also catches a NaN on either side; keys past the cap were read
-    // as 0.0, below every valid key, so a ragged item is no special case.  The first key of a row must be finite
-    // (lane 0 compares it with the largest finite double), and no key may carry a sign bit (that includes -0.0).
-    unsigned long long before = __shfl_up_sync(kFull, it.v[E / 2 - 1].y, 1);
-    if (lane == 0) before = it.before;
-    bool wrong = !(__longlong_as_double((long long)it.v[0].x) <= __longlong_as_double((long long)before));
-    unsigned signs = 0;
-    unsigned h[E];
+    unsigned hx[E / 2], hy[E / 2];
 #pragma unroll
     for (int p = 0; p < E / 2; ++p) {
-        const double x = __longlong_as_double((long long)it.v[p].x), y = __longlong_as_double((long long)it.v[p].y);
-        wrong |= !(y <= x);
-        if (p > 0) wrong |= !(x <= __longlong_as_double((long long)it.v[p - 1].y));
-        h[2 * p] = (unsigned)(it.v[p].x >> 32);
-        h[2 * p + 1] = (unsigned)(it.v[p].y >> 32);
-        signs |= h[2 * p] | h[2 * p + 1];
+        hx[p] = (unsigned)(it.v[p].x >> 32);
+        hy[p] = (unsigned)(it.v[p].y >> 32);
     }
-    *bad |= wrong || (signs >> 31) != 0u;
-    const int above_lane = window_count<E>(h, it.capi - k, W0, t_guess, s_fine);
-    const int above = __reduce_add_sync(kFull, above_lane);
+    // Order check.  The high words of valid keys order like the keys (a sign bit or a NaN shows as a high word
+    // above its predecessor's, the first key being held against the largest finite double); only where two
+    // neighbours have EQUAL high words do the low words matter, and then the exact check runs.  A row of
+    // hora_gains never has such neighbours (consecutive entries differ by more than 1 part in 2^11).
+    if (full) {
+        bool viol = false, ties = false;
+        unsigned prev_hy = 0;
+#pragma unroll
+        for (int p = 0; p < E / 2; ++p) {
+            const unsigned nh = __shfl_sync(kFull, hx[p], (lane + 1) & 31);
+            viol |= hy[p] > hx[p];
+            ties |= hy[p] == hx[p];
+            const unsigned mine = lane < 31 ? hy[p] : prev_hy;  // lane 31 holds lane 0's x against its last slice's y
+            if (lane < 31 || p > 0) {
+                viol |= nh > mine;
+                ties |= nh == mine;
+            }
+            prev_hy = hy[p];
+        }
+        if (lane == 0) {
+            const unsigned bh = (unsigned)(it.before >> 32);
+            viol |= hx[0] > bh;
+            ties |= hx[0] == bh;
+        }
+        if (__any_sync(kFull, ties)) viol |= level0_order_exact<E>(it, lane);
+        *bad |= viol;
+    } else {
+        unsigned signs = 0;
+#pragma unroll
+        for (int p = 0; p < E / 2; ++p) signs |= hx[p] | hy[p];
+        *bad |= level0_order_exact<E>(it, lane) || (signs >> 31) != 0u;
+    }
+    // Window: ts = prefix23 - W0 is negative below the window and >= kFineBins above it.  Slices come in
+    // descending order, so after one that lies wholly below the window nothing is left to count.
+    int above = 0;
+#pragma unroll
+    for (int p = 0; p < E / 2; ++p) {
+        const int tsx = (int)(hx[p] >> 9) - (int)W0, tsy = (int)(hy[p] >> 9) - (int)W0;
+        const int32_t kk = 64 * p + 2 * lane;
+        const bool vx = full || kk < nvalid, vy = full || kk + 1 < nvalid;
+        if (__all_sync(kFull, vy && tsy >= kFineBins)) {       // the slice lies above the window (hence above the guess)
+            above += 2;
+            continue;
+        }
+        if (__all_sync(kFull, !vx || tsx < 0)) break;          // ... or wholly below it
+        if (vx) {
+            if ((unsigned)tsx < (unsigned)kFineBins) atomicAdd(&s_fine[tsx], 1u);
+            above += tsx > t_guess;
+        }
+        if (vy) {
+            if ((unsigned)tsy < (unsigned)kFineBins) atomicAdd(&s_fine[tsy], 1u);
+            above += tsy > t_guess;
+        }
+    }
+    above = __reduce_add_sync(kFull, above);
     if (lane == 0) {
         *sum_pg += above;
         if (items_per_row == 1) pguess[row] = (unsigned int)above;
