@@ -455,14 +455,14 @@ struct Level0Item {
     int32_t capi;                  // the row's cap; -1 marks "no item"
 };
 
-template <int E, bool VEC2>
+template <int E, bool VEC2, bool ONE>
 __device__ __forceinline__ void level0_fetch(Level0Item<E> &it, const int32_t *__restrict__ cap, int32_t cap_scalar,
                                              int64_t n_items, int32_t items_per_row, int32_t ld,
                                              const double *__restrict__ gains, int64_t item, int lane, bool *bad) {
     it.capi = -1;
     if (item >= n_items) return;
-    const int64_t row = items_per_row == 1 ? item : item / items_per_row;
-    const int32_t k0 = (int32_t)(item - row * items_per_row) * (kWarp * E);
+    const int64_t row = ONE ? item : item / items_per_row;     // ONE: an item is a whole row (no 64-bit division)
+    const int32_t k0 = ONE ? 0 : (int32_t)(item - row * items_per_row) * (kWarp * E);
     int32_t capi = cap ? __ldg(cap + row) : cap_scalar;
     if (capi < 0 || capi > ld) { *bad = true; capi = 0; }
     it.capi = capi;
@@ -510,13 +510,13 @@ __device__ __forceinline__ bool level0_order_exact(const Level0Item<E> &it, int 
     return wrong;
 }
 
-template <int E>
+template <int E, bool ONE>
 __device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t item, int32_t items_per_row,
                                                int lane, unsigned int *s_fine, unsigned W0, int t_guess,
                                                unsigned int *__restrict__ pguess, long long *capsum, long long *sum_pg,
                                                bool *bad) {
-    const int64_t row = items_per_row == 1 ? item : item / items_per_row;
-    const int32_t k0 = (int32_t)(item - row * items_per_row) * (kWarp * E);
+    const int64_t row = ONE ? item : item / items_per_row;
+    const int32_t k0 = ONE ? 0 : (int32_t)(item - row * items_per_row) * (kWarp * E);
     const int32_t nvalid = it.capi - k0;                       // keys of this item below the cap (may be <= 0 or > 32 E)
     const bool full = nvalid >= kWarp * E;
     if (lane == 0 && k0 == 0) *capsum += it.capi;
@@ -583,12 +583,12 @@ __device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t 
     above = __reduce_add_sync(kFull, above);
     if (lane == 0) {
         *sum_pg += above;
-        if (items_per_row == 1) pguess[row] = (unsigned int)above;
+        if (ONE) pguess[row] = (unsigned int)above;
         else if (above) atomicAdd(pguess + row, (unsigned int)above);   // several items per row: cleared by the host
     }
 }
 
-template <int E, bool VEC2>
+template <int E, bool VEC2, bool ONE>
 __global__ void __launch_bounds__(kSelThreads, 3)
 select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
               const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist_fine,
@@ -609,13 +609,13 @@ select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
     bool bad = false;
     // two items in flight, in two fixed register sets (no copies): A is processed while B's loads land
     Level0Item<E> A, Bq;
-    level0_fetch<E, VEC2>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item0, lane, &bad);
+    level0_fetch<E, VEC2, ONE>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item0, lane, &bad);
     for (int64_t item = item0; item < n_items; item += 2 * stride) {
-        level0_fetch<E, VEC2>(Bq, cap, cap_scalar, n_items, items_per_row, ld, gains, item + stride, lane, &bad);
-        level0_process<E>(A, item, items_per_row, lane, s_fine, W0, t_guess, pguess, &capsum, &sum_pg, &bad);
-        level0_fetch<E, VEC2>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item + 2 * stride, lane, &bad);
+        level0_fetch<E, VEC2, ONE>(Bq, cap, cap_scalar, n_items, items_per_row, ld, gains, item + stride, lane, &bad);
+        level0_process<E, ONE>(A, item, items_per_row, lane, s_fine, W0, t_guess, pguess, &capsum, &sum_pg, &bad);
+        level0_fetch<E, VEC2, ONE>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item + 2 * stride, lane, &bad);
         if (Bq.capi >= 0)
-            level0_process<E>(Bq, item + stride, items_per_row, lane, s_fine, W0, t_guess, pguess, &capsum, &sum_pg, &bad);
+            level0_process<E, ONE>(Bq, item + stride, items_per_row, lane, s_fine, W0, t_guess, pguess, &capsum, &sum_pg, &bad);
     }
     level0_finish(hdr, hist_fine, s_fine, W0, t_guess, capsum, sum_pg, bad, B, s_warp);
 }
@@ -1673,10 +1673,10 @@ static inline void mark_stage(int k, cudaStream_t s) {
 template <int E>
 static void launch_level0(bool vec2, int grid, cudaStream_t s, const int32_t *cap, int32_t cap_scalar, int64_t N,
                           int32_t ld, const double *gains, int64_t B, const Workspace &w) {
-    if (vec2)
-        select_level0<E, true><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_fine, w.pguess);
-    else
-        select_level0<E, false><<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_fine, w.pguess);
+    const bool one = ld <= kWarp * E;                     // an item is a whole row
+    auto go = [&](auto kernel) { kernel<<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_fine, w.pguess); };
+    if (vec2) { if (one) go(select_level0<E, true, true>); else go(select_level0<E, true, false>); }
+    else { if (one) go(select_level0<E, false, true>); else go(select_level0<E, false, false>); }
 }
 
 template <int E>
