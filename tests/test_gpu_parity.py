@@ -260,6 +260,85 @@ def test_allocation_status_codes():
     assert info.status == 2 and not d.any()
 
 
+@pytest.mark.parametrize("ld,cap_value", [(256, 256), (256, 200), (96, 96), (40, 33)])
+def test_allocation_validates_a_given_gains_matrix(ld, cap_value):
+    """hora_allocate checks the matrix it is given: every row finite, non-negative and non-increasing up to its
+    cap.  Equal neighbours are allowed; a disorder that shows only in the low 32 bits of two keys with equal
+    high words, a NaN, an infinity, a negative value and a negative zero are not."""
+    from paper_2605_07114_b200 import hora
+    N, G0, B = 300, 4, 700
+    rng = np.random.default_rng(ld + cap_value)
+    alpha, beta = rng.uniform(0.5, 3.0, N), rng.uniform(0.5, 3.0, N)
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    al = hora.Allocator(N, ld, G0, exact_int=False)
+    a_d, b_d, c_d = gu_dev(alpha), gu_dev(beta), gu_dev(c)
+    hora.hora_gains(a_d, b_d, 1.0, 1.0, c_d, G0, None, cap_value, N, ld, al.gains)
+    torch.cuda.synchronize()
+    clean = al.gains.clone()
+
+    def status_with(edit):
+        al.gains.copy_(clean)
+        edit(al.gains)
+        hora.hora_allocate(a_d, b_d, 1.0, 1.0, c_d, G0, None, cap_value, N, ld, al.gains, B, al.flags, al.delta, al.G,
+                           al.group_offsets, al.info, al.workspace)
+        torch.cuda.synchronize()
+        return al.read_info().status, al.delta.cpu().numpy()
+
+    def bits(g):
+        return g.view(torch.int64)
+
+    st, d = status_with(lambda g: None)
+    assert st == 0 and d.sum() == B
+    j = cap_value // 2                                    # a column well inside every row
+    # equal neighbours: still non-increasing
+    def tie(g): g[7, j + 1] = g[7, j]
+    st, d = status_with(tie)
+    assert st == 0 and d.sum() == B
+    # same high word, low word one step UP: increasing by one unit in the last place
+    def lo_up(g): bits(g)[11, j + 1] = bits(g)[11, j] + 1
+    assert status_with(lo_up)[0] == 2
+    # plainly increasing, at a slice boundary of the full-read pass too
+    def swap(g): g[13, j], g[13, j + 1] = g[13, j + 1].clone(), g[13, j].clone()
+    assert status_with(swap)[0] == 2
+    if cap_value > 66:
+        def at_64(g): g[17, 64] = g[17, 62]
+        assert status_with(at_64)[0] == 2
+    for bad in (float("nan"), float("inf"), -1.0e-3, -0.0):
+        def put(g, bad=bad): g[19, cap_value - 1] = bad
+        st, d = status_with(put)
+        assert st == 2 and not d.any(), bad
+    def first_inf(g): g[23, 0] = float("inf")
+    assert status_with(first_inf)[0] == 2
+
+
+def test_allocate_stage_events_are_recorded_in_order():
+    """hora_allocate_profile_stages: the seven events land on the call's stream in stage order, and switching
+    the aid off stops the recording."""
+    from paper_2605_07114_b200 import hora
+    w = wl.make("cfg2", 2048)
+    al = hora.Allocator(w.N, w.ld, w.G0, exact_int=False)
+    args = (gu_dev(w.alpha), gu_dev(w.beta), 1.0, 1.0, gu_dev(w.c), gu_dev(w.cap), 0, w.B)
+    al.run(*args)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(7)]
+    for e in evs:
+        e.record()
+    torch.cuda.synchronize()
+    hora.hora_allocate_profile_stages([e.cuda_event for e in evs])
+    try:
+        al.run(*args)
+    finally:
+        hora.hora_allocate_profile_stages(None)
+    torch.cuda.synchronize()
+    gaps = [evs[i].elapsed_time(evs[i + 1]) for i in range(6)]
+    assert all(g >= 0.0 for g in gaps) and sum(gaps) > 0.0
+    assert al.read_info().status == 0
+    tail = torch.cuda.Event(enable_timing=True)
+    tail.record()
+    al.run(*args)                                         # recording is off: the old events keep their times
+    torch.cuda.synchronize()
+    assert evs[6].elapsed_time(tail) >= 0.0
+
+
 def test_allocation_host_errors():
     from paper_2605_07114_b200 import hora
     N, ld = 10, 8
@@ -282,6 +361,10 @@ def test_allocation_is_reproducible():
     b = gu.gpu_allocate(w.alpha, w.beta, 1.0, 1.0, w.c, w.G0, w.cap, w.ld, w.B, exact=False)
     np.testing.assert_array_equal(a[0], b[0])
     assert np.float64(a[3].objective).view(np.uint64) == np.float64(b[3].objective).view(np.uint64)
+
+
+def gu_dev(a):
+    return _util().dev(a)
 
 
 # ------------------------------------------------------------------------------------- advantages
