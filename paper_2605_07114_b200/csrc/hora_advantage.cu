@@ -37,8 +37,12 @@ struct __align__(16) AdvWarpSmem {
     unsigned int starts[kSlab / 32];                          // one bit per element: a non-empty group starts here
     int cum_starts[kSlab / 32];                               // exclusive running counts per word
     float2 two[kWarp];                                        // per non-empty group, in order: advantage of a 0, of a 1
-    double mean[kWarp], scale[kWarp];                         // per non-empty group, in order (general route)
+    // general route: mean and scale per non-empty group, in order; they take the place of `pre`, which only the
+    // 0/1 route reads
+    __device__ __forceinline__ double *mean() { return reinterpret_cast<double *>(pre); }
+    __device__ __forceinline__ double *scale() { return reinterpret_cast<double *>(pre) + kWarp; }
 };
+static_assert(sizeof(unsigned int) * (kSlab / 4 + 4) >= 2 * kWarp * sizeof(double), "mean and scale fit in pre");
 constexpr size_t kAdvSmem = sizeof(AdvWarpSmem) * kAdvWarps;
 
 __device__ __forceinline__ int64_t shfl_i64(int64_t v, int src) { return __shfl_sync(kFull, v, src); }
@@ -256,13 +260,13 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
                     if (lane == i) { my_mean = mean; my_ss = ss; }
                 }
                 if (nonempty) {
-                    sm.mean[my_rank] = my_mean;
-                    sm.scale[my_rank] = group_scale(mode, my_ss, my_n, ddof, eps);
+                    sm.mean()[my_rank] = my_mean;
+                    sm.scale()[my_rank] = group_scale(mode, my_ss, my_n, ddof, eps);
                 }
                 __syncwarp();
                 for (int el = lead + lane; el < span; el += kWarp) {
                     const int r = rank_of(sm, el);
-                    adv[start + el] = (float)(((double)sm.buf[el] - sm.mean[r]) * sm.scale[r]);
+                    adv[start + el] = (float)(((double)sm.buf[el] - sm.mean()[r]) * sm.scale()[r]);
                 }
             }
             __syncwarp();

@@ -226,7 +226,7 @@ def test_allocation_when_the_sampled_window_misses(exact):
 
 
 def test_allocation_with_long_rows():
-    """ld > 256: several items per row in the full-read pass, several sketch chunks per row afterwards."""
+    """ld > 256: several items per row in the full-read pass, whose counts above the guess add up per row."""
     gu = _util()
     rng = np.random.default_rng(9)
     N, G0, ld = 3000, 4, 700
@@ -240,6 +240,42 @@ def test_allocation_with_long_rows():
         assert info.status == 0
         np.testing.assert_array_equal(d, d_o)
         assert abs(info.lambda_ - lam) <= 1e-12 * lam
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_allocation_on_random_shapes(seed):
+    """Random sizes, row lengths (odd ones too: no 16-byte loads), caps and budgets, real and integer priors,
+    with the matrix given and built inside: Delta, G, offsets and the objective against the oracle."""
+    gu = _util()
+    rng = np.random.default_rng(1000 + seed)
+    N = int(rng.integers(1, 6000))
+    ld = int(rng.choice([1, 2, 7, 31, 64, 65, 100, 128, 129, 255, 256, 257, 300, 513]))
+    G0 = int(rng.integers(1, 9))
+    exact = bool(seed % 2)
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    if seed % 3 == 0:
+        cap[:] = ld
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    if exact:
+        alpha = rng.integers(1, 4, N).astype(np.float64)
+        beta = rng.integers(1, 4, N).astype(np.float64)
+    else:
+        alpha = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
+        beta = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
+    total = int(cap.sum())
+    for B in sorted({0, 1, total // 3, total - 1 if total > 0 else 0, total}):
+        if exact:
+            d_o, _, lam, obj = orc.greedy_exact(alpha, beta, 1.0, 1.0, c, G0, cap, B)
+        else:
+            d_o, _, lam, obj = orc.greedy_real(alpha, beta, 1.0, 1.0, c, G0, cap, B)
+        for materialise in (True, False):
+            d, G, off, info = gu.gpu_allocate(alpha, beta, 1.0, 1.0, c, G0, cap, ld, B, exact=exact,
+                                              materialise=materialise)
+            assert info.status == 0, (N, ld, G0, B, materialise)
+            np.testing.assert_array_equal(d, d_o)
+            np.testing.assert_array_equal(G, G0 + d_o)
+            np.testing.assert_array_equal(off, np.concatenate(([0], np.cumsum(G0 + d_o.astype(np.int64)))))
+            assert abs(info.objective - obj) <= 1e-12 * max(abs(obj), 1e-300)
 
 
 def test_allocation_status_codes():
