@@ -284,8 +284,12 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
             G[r0 + threadIdx.x] = failed ? 0 : G0 + my_delta;
         }
         double obj = 0.0;
+        // U_i(Delta) from the row's own entry in shared memory: the product in U = 1 - prod_{j<Delta} (b+j)/(a+b+j)
+        // is g_i(Delta) (b + Delta - 1) / a  (Eq. marginal); the product loop itself took up to Delta iterations of
+        // the slowest lane
         if (!failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE) && threadIdx.x < n && my_delta > 0)
-            obj = hit_utility(sm.a[threadIdx.x], sm.b[threadIdx.x], my_delta);
+            obj = 1.0 - __longlong_as_double((long long)row[my_delta - 1]) *
+                            (sm.b[threadIdx.x] + (double)(my_delta - 1)) / sm.a[threadIdx.x];
 #pragma unroll
         for (int d = 16; d >= 1; d >>= 1) obj += __shfl_xor_sync(kFull, obj, d);
         __syncthreads();
