@@ -27,11 +27,11 @@ constexpr int kBBins = 2048;                   // 11-bit digits
 constexpr size_t kBMaxSmem = 200 * 1024;       // keys + bookkeeping must fit this
 constexpr int kScanRows = 1024;                // rows per CTA in the offsets scan
 
+constexpr int kBListCap = 256;                 // keys of the short list the late digit levels work on
+
 struct BatchedSmemFixed {
     unsigned int hist[kBBins];
-    double a[kBMaxRows], b[kBMaxRows];
-    U128 num[kBMaxRows], den[kBMaxRows];
-    int32_t cap[kBMaxRows], p_hi[kBMaxRows], tied[kBMaxRows], band[kBMaxRows];
+    unsigned long long list[kBListCap];
     long long warp_tmp[kBWarps];
     double obj_tmp[kBWarps];
     long long found[3];
@@ -39,6 +39,26 @@ struct BatchedSmemFixed {
     double lam_exact;
     int status;
 };
+
+// Per-prompt arrays of a segment, carved behind the fixed part for the longest segment of the call (so that
+// calls with short segments — the paper's 15 prompts — leave shared memory for a fourth CTA per SM).
+struct BatchedRows {
+    double *a, *b;
+    U128 *num, *den;
+    int32_t *cap, *band;
+};
+constexpr size_t kBRowBytes = 2 * sizeof(double) + 2 * sizeof(U128) + 2 * sizeof(int32_t);   // 56 bytes per prompt
+
+__device__ __forceinline__ BatchedRows carve_rows(unsigned char *base, int rows_cap) {
+    BatchedRows r;
+    r.num = reinterpret_cast<U128 *>(base);
+    r.den = r.num + rows_cap;
+    r.a = reinterpret_cast<double *>(r.den + rows_cap);
+    r.b = r.a + rows_cap;
+    r.cap = reinterpret_cast<int32_t *>(r.b + rows_cap);
+    r.band = r.cap + rows_cap;
+    return r;
+}
 
 __device__ __forceinline__ long long bblock_exclusive_sum(long long v, long long *total, long long *s_warp) {
     const int lane = lane_id(), warp = threadIdx.x >> 5;
@@ -99,11 +119,13 @@ __global__ void __launch_bounds__(kBThreads)
 allocate_batched_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
                         const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
                         int32_t ld, const int64_t *__restrict__ seg_off, const int64_t *__restrict__ budgets, int64_t S,
-                        uint32_t flags, int32_t *__restrict__ delta, int32_t *__restrict__ G,
+                        uint32_t flags, int32_t rows_cap, int32_t *__restrict__ delta, int32_t *__restrict__ G,
                         hora_alloc_info *__restrict__ info) {
     extern __shared__ __align__(16) unsigned char s_raw[];
     BatchedSmemFixed &sm = *reinterpret_cast<BatchedSmemFixed *>(s_raw);
-    unsigned long long *keys = reinterpret_cast<unsigned long long *>(s_raw + sizeof(BatchedSmemFixed));
+    const BatchedRows rw = carve_rows(s_raw + sizeof(BatchedSmemFixed), rows_cap);
+    unsigned long long *keys =
+        reinterpret_cast<unsigned long long *>(s_raw + sizeof(BatchedSmemFixed) + (size_t)rows_cap * kBRowBytes);
     const int lane = lane_id(), warp = threadIdx.x >> 5;
     const bool exact = (flags & HORA_FLAG_EXACT_INT) != 0;
     for (int64_t s = blockIdx.x; s < S; s += gridDim.x) {
@@ -118,7 +140,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
             const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, r0 + r);
             if (!p.ok && lane == 0) sm.status = HORA_ERR_INVALID_VALUE;
             const double a = p.ok ? p.a : 1.0, b = p.ok ? p.b : 1.0;
-            if (lane == 0) { sm.a[r] = a; sm.b[r] = b; sm.cap[r] = p.cap; }
+            if (lane == 0) { rw.a[r] = a; rw.b[r] = b; rw.cap[r] = p.cap; }
             double carry = 1.0;
             double *out = reinterpret_cast<double *>(keys + (size_t)r * ld);
             for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E)
@@ -126,7 +148,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         }
         __syncthreads();
         long long sum_cap;
-        bblock_exclusive_sum(threadIdx.x < n ? sm.cap[threadIdx.x] : 0, &sum_cap, sm.warp_tmp);
+        bblock_exclusive_sum(threadIdx.x < n ? rw.cap[threadIdx.x] : 0, &sum_cap, sm.warp_tmp);
         if (threadIdx.x == 0 && sm.status == HORA_OK && B > sum_cap) sm.status = HORA_ERR_INFEASIBLE;
         __syncthreads();
         // ---- 2: the B-th largest key ----
@@ -135,10 +157,9 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         if (sm.status == HORA_OK && B > 0) {
             // Levels 0 and 1 (top 22 bits) sweep the keys row by row (a warp per row, no index division);
             // what still matches after them is a handful of keys, which are copied to a short list that the
-            // remaining levels work on.  The list reuses the bin array's neighbour: the band flags are not
-            // live yet, so p_hi/tied/band (3 x 256 words) hold up to 384 keys; a longer list keeps sweeping.
-            unsigned long long *list = reinterpret_cast<unsigned long long *>(sm.p_hi);
-            constexpr int kListCap = 3 * kBMaxRows / 2;
+            // remaining levels work on (up to kBListCap keys; a longer list keeps sweeping).
+            unsigned long long *list = sm.list;
+            constexpr int kListCap = kBListCap;
             int n_list = -1;                                       // -1: still sweeping the rows
             for (int level = 0; level < 6; ++level) {             // 5 x 11 + 9 = 64 bits, from the top
                 const int w = level < 5 ? 11 : 9;
@@ -148,7 +169,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                 if (n_list < 0) {
                     for (int r = warp; r < n; r += kBWarps) {
                         const unsigned long long *rk = keys + (size_t)r * ld;
-                        const int cp = sm.cap[r];
+                        const int cp = rw.cap[r];
                         for (int col = lane; col < cp; col += kWarp) {
                             const unsigned long long key = rk[col];
                             if (level == 0 || (key >> (sh + w)) == (prefix >> (sh + w)))
@@ -174,7 +195,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                     __syncthreads();
                     for (int r = warp; r < n; r += kBWarps) {
                         const unsigned long long *rk = keys + (size_t)r * ld;
-                        const int cp = sm.cap[r];
+                        const int cp = rw.cap[r];
                         for (int col = lane; col < cp; col += kWarp) {
                             const unsigned long long key = rk[col];
                             if ((key >> sh) == (prefix >> sh)) list[atomicAdd(&sm.list_count, 1ull)] = key;
@@ -192,7 +213,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         int my_hi = 0, my_tied = 0, my_cap = 0;
         const unsigned long long *row = keys + (size_t)threadIdx.x * ld;
         if (threadIdx.x < n && sm.status == HORA_OK && B > 0) {
-            my_cap = sm.cap[threadIdx.x];
+            my_cap = rw.cap[threadIdx.x];
             int lo = 0, hi = my_cap;
             while (lo < hi) {
                 const int mid = (lo + hi) >> 1;
@@ -233,22 +254,22 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                 if (has && q + 1 < my_cap && row[q + 1] >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
                 if (has && !err) {
                     U128 nu, de;
-                    if (!exact_gain((unsigned long long)sm.a[threadIdx.x], (unsigned long long)sm.b[threadIdx.x],
+                    if (!exact_gain((unsigned long long)rw.a[threadIdx.x], (unsigned long long)rw.b[threadIdx.x],
                                     (unsigned long long)q + 1, nu, de)) err = HORA_ERR_EXACT_RANGE;
-                    sm.num[threadIdx.x] = nu;
-                    sm.den[threadIdx.x] = de;
+                    rw.num[threadIdx.x] = nu;
+                    rw.den[threadIdx.x] = de;
                 }
                 if (err) atomicCAS(&sm.status, 0, err);
             }
-            if (threadIdx.x < kBMaxRows) sm.band[threadIdx.x] = (threadIdx.x < n && has && !err) ? 1 : 0;
+            if ((int)threadIdx.x < rows_cap) rw.band[threadIdx.x] = (threadIdx.x < n && has && !err) ? 1 : 0;
             long long tot_q;
             bblock_exclusive_sum(q, &tot_q, sm.warp_tmp);          // has a barrier: num/den/band are visible after it
             const long long Rp = B - tot_q;                        // rollouts to hand out inside the band
             int better = 0, equal = 0;
-            if (threadIdx.x < n && sm.band[threadIdx.x] && sm.status == HORA_OK) {
+            if (threadIdx.x < n && rw.band[threadIdx.x] && sm.status == HORA_OK) {
                 for (int u = 0; u < n; ++u) {
-                    if (!sm.band[u] || u == (int)threadIdx.x) continue;
-                    const int sgn = cmp_products(sm.num[u], sm.den[threadIdx.x], sm.num[threadIdx.x], sm.den[u]);
+                    if (!rw.band[u] || u == (int)threadIdx.x) continue;
+                    const int sgn = cmp_products(rw.num[u], rw.den[threadIdx.x], rw.num[threadIdx.x], rw.den[u]);
                     better += (sgn > 0) || (sgn == 0 && u < (int)threadIdx.x);
                     equal += (sgn == 0);
                 }
@@ -256,12 +277,12 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                 if (better == Rp - 1) {                            // this row holds the B-th best candidate
                     int strictly = 0;
                     for (int u = 0; u < n; ++u)
-                        if (sm.band[u] && u != (int)threadIdx.x &&
-                            cmp_products(sm.num[u], sm.den[threadIdx.x], sm.num[threadIdx.x], sm.den[u]) > 0) ++strictly;
+                        if (rw.band[u] && u != (int)threadIdx.x &&
+                            cmp_products(rw.num[u], rw.den[threadIdx.x], rw.num[threadIdx.x], rw.den[u]) > 0) ++strictly;
                     sm.found[0] = tot_q + strictly;
                     sm.found[1] = equal + 1;
                     sm.found[2] = Rp - strictly;
-                    const U128 nu = sm.num[threadIdx.x], de = sm.den[threadIdx.x];
+                    const U128 nu = rw.num[threadIdx.x], de = rw.den[threadIdx.x];
                     lambda = ((double)nu.hi * 18446744073709551616.0 + (double)nu.lo) /
                              ((double)de.hi * 18446744073709551616.0 + (double)de.lo);
                     sm.lam_exact = lambda;
@@ -289,7 +310,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         // the slowest lane
         if (!failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE) && threadIdx.x < n && my_delta > 0)
             obj = 1.0 - __longlong_as_double((long long)row[my_delta - 1]) *
-                            (sm.b[threadIdx.x] + (double)(my_delta - 1)) / sm.a[threadIdx.x];
+                            (rw.b[threadIdx.x] + (double)(my_delta - 1)) / rw.a[threadIdx.x];
 #pragma unroll
         for (int d = 16; d >= 1; d >>= 1) obj += __shfl_xor_sync(kFull, obj, d);
         __syncthreads();
@@ -418,7 +439,9 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
         if (n < 0 || budgets_host[s] < 0) return HORA_ERR_INVALID_ARG;
         max_rows = std::max(max_rows, n);
     }
-    const size_t smem = sizeof(BatchedSmemFixed) + (size_t)max_rows * (size_t)ld * sizeof(unsigned long long);
+    const int32_t rows_cap = (int32_t)((max_rows + 3) & ~(int64_t)3);
+    const size_t smem = sizeof(BatchedSmemFixed) + (size_t)rows_cap * kBRowBytes +
+                        (size_t)max_rows * (size_t)ld * sizeof(unsigned long long);
     if (max_rows > kBMaxRows || smem > kBMaxSmem) return HORA_ERR_WORKSPACE;   // segment too large for one CTA
     if (N > 0 && (c == nullptr || delta == nullptr || G == nullptr)) return HORA_ERR_INVALID_ARG;
     if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HORA_ERR_WORKSPACE;
@@ -434,13 +457,14 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
         return HORA_ERR_CUDA;
     int launches = 0;
     if (S > 0 && N > 0) {
-        const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (220 * 1024) / smem));
+        // 227 KiB of shared memory per SM, 1 KiB of it reserved per resident CTA
+        const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (227 * 1024) / (smem + 1024)));
         const int grid = clamp_grid(S, per_sm);
         auto launch = [&](auto kernel) -> cudaError_t {
             cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
             kernel<<<grid, kBThreads, smem, st>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, w.seg_off,
-                                                  w.budgets, S, flags, delta, G, info_dev);
+                                                  w.budgets, S, flags, rows_cap, delta, G, info_dev);
             return cudaGetLastError();
         };
         cudaError_t e;
