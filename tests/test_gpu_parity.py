@@ -444,6 +444,30 @@ def test_group_advantage_on_workload_groups():
         assert np.abs(sums).max() < 1e-3                          # advantages of a group sum to zero
 
 
+@pytest.mark.parametrize("mis_in,mis_out", [(0, 0), (1, 0), (0, 3), (2, 2)])
+def test_group_advantage_with_unaligned_buffers_stays_in_bounds(mis_in, mis_out):
+    """Rewards and advantages that do not start on a 16-byte boundary (no vector path), and a guard band around
+    the output: nothing before the first or after the last element is written."""
+    from paper_2605_07114_b200 import hora
+    rng = np.random.default_rng(10 * mis_in + mis_out)
+    r, off = ragged(rng, 3000, [0, 1, 5, 8, 31, 32, 33, 100, 264, 2000], [0.0, 1.0])
+    total = int(off[-1])
+    rbuf = torch.zeros(total + 8, dtype=torch.float32, device="cuda")
+    obuf = torch.full((total + 16,), float("nan"), dtype=torch.float32, device="cuda")
+    rin = rbuf[mis_in:mis_in + total]
+    rin.copy_(torch.from_numpy(r))
+    out = obuf[4 + mis_out:4 + mis_out + total]
+    for mode in (0, 1):
+        obuf.fill_(float("nan"))
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        hora.hora_group_advantage(rin, torch.from_numpy(off).cuda(), len(off) - 1, mode, 1e-6, 0, out, status)
+        torch.cuda.synchronize()
+        exp = orc.group_advantage(r, off, mode, float(np.float32(1e-6)), 0)
+        assert int(status.item()) == 0
+        np.testing.assert_allclose(out.cpu().numpy(), exp, rtol=0, atol=1e-5)
+        assert torch.isnan(obuf[:4 + mis_out]).all() and torch.isnan(obuf[4 + mis_out + total:]).all()
+
+
 def test_group_advantage_flags_decreasing_offsets():
     gu = _util()
     r = np.ones(10, np.float32)
