@@ -45,6 +45,7 @@
 #include <cooperative_groups.h>
 
 #include <atomic>
+#include <type_traits>
 
 #include "hora_common.cuh"
 #include "hora_exact.cuh"
@@ -530,33 +531,37 @@ __device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t 
     // above its predecessor's, the first key being held against the largest finite double); only where two
     // neighbours have EQUAL high words do the low words matter, and then the exact check runs.  A row of
     // hora_gains never has such neighbours (consecutive entries differ by more than 1 part in 2^11).
-    if (full) {
+    // Keys past the cap were read as 0: they can never show as a violation (0 is above nothing), and they are
+    // kept out of the tie test by their index (a test that whole items skip).
+    {
         bool viol = false, ties = false;
-        unsigned prev_hy = 0;
+        auto quick = [&](auto whole) {
+            constexpr bool kWhole = decltype(whole)::value;
+            unsigned prev_hy = 0;
 #pragma unroll
-        for (int p = 0; p < E / 2; ++p) {
-            const unsigned nh = __shfl_sync(kFull, hx[p], (lane + 1) & 31);
-            viol |= hy[p] > hx[p];
-            ties |= hy[p] == hx[p];
-            const unsigned mine = lane < 31 ? hy[p] : prev_hy;  // lane 31 holds lane 0's x against its last slice's y
-            if (lane < 31 || p > 0) {
-                viol |= nh > mine;
-                ties |= nh == mine;
+            for (int p = 0; p < E / 2; ++p) {
+                const int32_t kk = 64 * p + 2 * lane;
+                const unsigned nh = __shfl_sync(kFull, hx[p], (lane + 1) & 31);
+                viol |= hy[p] > hx[p];
+                ties |= hy[p] == hx[p] && (kWhole || kk + 1 < nvalid);
+                // the key after this pair: the next lane's x; lane 31 holds lane 0's x against its last slice's y
+                const unsigned mine = lane < 31 ? hy[p] : prev_hy;
+                const int32_t next_k = lane < 31 ? kk + 2 : 64 * p;
+                if (lane < 31 || p > 0) {
+                    viol |= nh > mine;
+                    ties |= nh == mine && (kWhole || next_k < nvalid);
+                }
+                prev_hy = hy[p];
             }
-            prev_hy = hy[p];
-        }
+        };
+        if (full) quick(std::true_type{}); else quick(std::false_type{});
         if (lane == 0) {
             const unsigned bh = (unsigned)(it.before >> 32);
             viol |= hx[0] > bh;
-            ties |= hx[0] == bh;
+            ties |= hx[0] == bh && nvalid > 0;
         }
         if (__any_sync(kFull, ties)) viol |= level0_order_exact<E>(it, lane);
         *bad |= viol;
-    } else {
-        unsigned signs = 0;
-#pragma unroll
-        for (int p = 0; p < E / 2; ++p) signs |= hx[p] | hy[p];
-        *bad |= level0_order_exact<E>(it, lane) || (signs >> 31) != 0u;
     }
     // Window: ts = prefix23 - W0 is negative below the window and >= kFineBins above it.  Slices come in
     // descending order, so after one that lies wholly below the window nothing is left to count.
@@ -588,8 +593,12 @@ __device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t 
     }
 }
 
+// CTAs per SM of the full-read pass: what the registers allow (two items of 16 E bytes per lane in flight)
+template <int E>
+constexpr int level0_per_sm() { return E == 8 ? 3 : 5; }
+
 template <int E, bool VEC2, bool ONE>
-__global__ void __launch_bounds__(kSelThreads, 3)
+__global__ void __launch_bounds__(kSelThreads, level0_per_sm<E>())
 select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
               const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist_fine,
               unsigned int *__restrict__ pguess) {
@@ -1674,6 +1683,8 @@ template <int E>
 static void launch_level0(bool vec2, int grid, cudaStream_t s, const int32_t *cap, int32_t cap_scalar, int64_t N,
                           int32_t ld, const double *gains, int64_t B, const Workspace &w) {
     const bool one = ld <= kWarp * E;                     // an item is a whole row
+    grid = clamp_grid((N * ((ld + kWarp * E - 1) / (kWarp * E)) + kSelThreads / kWarp - 1) / (kSelThreads / kWarp),
+                      level0_per_sm<E>());                // exactly what is resident at once
     auto go = [&](auto kernel) { kernel<<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_fine, w.pguess); };
     if (vec2) { if (one) go(select_level0<E, true, true>); else go(select_level0<E, true, false>); }
     else { if (one) go(select_level0<E, false, true>); else go(select_level0<E, false, false>); }
