@@ -127,6 +127,8 @@ hora_status_t hora_gains(const double *alpha, const double *beta, double alpha0,
  *                    contents are undefined on entry and on exit
  * Data-dependent failures (INVALID_VALUE, INFEASIBLE, NOT_INTEGER, EXACT_RANGE) set info_dev->status and
  * leave delta, G and group_offsets all zero.
+ * One of the call's kernels is launched cooperatively (all its thread blocks resident at once, sized per device
+ * on first use); a device or context without cooperative launch makes the call return HORA_ERR_CUDA.
  */
 size_t hora_allocate_workspace_bytes(int64_t N, int32_t ld, int32_t gains_is_null, uint32_t flags);
 
