@@ -104,6 +104,16 @@ def test_utility_beta_ratio_and_telescoping(a, b):
         assert u == pytest.approx(uf, rel=1e-15, abs=1e-18)
 
 
+@pytest.mark.parametrize("a,b", REAL_AB)
+def test_utility_from_the_marginal_itself(a, b):
+    """The product inside U(Delta) is M(Delta - 1) (b + Delta - 1) / a (Eq. marginal, Eq. hit-utility), so
+    U(Delta) = 1 - g(Delta) (b + Delta - 1) / a: exact in rationals, and to rounding in the oracle's floats."""
+    fa, fb = Fraction(a), Fraction(b)
+    for D in (1, 2, 3, 17, 100, 256):
+        assert literal.utility(fa, fb, D) == 1 - literal.marginals(fa, fb, D)[D - 1] * (fb + D - 1) / fa
+        assert orc.utility_one(a, b, D) == pytest.approx(1.0 - orc.gain_one(a, b, D) * (b + D - 1) / a, rel=1e-13, abs=1e-15)
+
+
 def test_utility_uniform_prior_no_success_closed_form():
     """Beta(1,1), c = 0: a = 1, b = G0 + 1, U(Delta) = Delta / (Delta + G0 + 1)."""
     for G0 in (2, 4, 8):
