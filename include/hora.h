@@ -122,6 +122,7 @@ hora_status_t hora_gains(const double *alpha, const double *beta, double alpha0,
  *   alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld   as for hora_gains
  *   gains            [N*ld] the matrix hora_gains wrote for the same inputs, or NULL to have it built
  *                    inside the workspace (the workspace must then be sized with gains_is_null = 1)
+ *   N                at most 2^31 - 1 prompts per call (HORA_ERR_INVALID_ARG beyond)
  *   B                number of Phase-B rollouts, 0 <= B <= sum_i cap_i
  *   workspace        device scratch, 256-byte aligned, at least hora_allocate_workspace_bytes(...);
  *                    contents are undefined on entry and on exit

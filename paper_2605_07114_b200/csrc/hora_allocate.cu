@@ -1751,6 +1751,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
                                        size_t workspace_bytes, void *stream) {
     using namespace hora;
     if (N < 0 || ld < 1 || G0 < 0 || B < 0) return HORA_ERR_INVALID_ARG;
+    if (N > 0x7FFFFFFFll) return HORA_ERR_INVALID_ARG;     // row indices are kept in 32 bits
     if ((alpha == nullptr) != (beta == nullptr)) return HORA_ERR_INVALID_ARG;
     if (alpha == nullptr && !(alpha0 > 0.0 && beta0 > 0.0 && alpha0 < 1.0e300 && beta0 < 1.0e300))
         return HORA_ERR_INVALID_ARG;
