@@ -199,6 +199,13 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    # ---- before any timing counts: the oracle's pass over (a prefix of) this batch, and the four calls held
+    # against it, output by output.  The same pass is the CPU baseline reported beside the result. ----
+    ref = parity = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        ref = oracle_pass(w, min(args.cpu_sample, N))
+        parity = check_against_oracle(torch, hora, dev, ref)
+
     warmup = max(args.warmup, 3)
     for _ in range(warmup):
         step()
@@ -474,8 +481,9 @@ def run_ours(args):
                              "note": "the same four calls captured once in a CUDA graph and replayed"}
     if world == 1:
         out["batched"] = bench_batched(torch, hora, wl, dev)
-    if world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(w, args.cpu_sample)
+    if ref is not None:
+        out["cpu_baseline"] = cpu_baseline(w, args.cpu_sample, ref)
+        out["parity"] = parity
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -519,9 +527,9 @@ def bench_batched(torch, hora, wl, dev, shards=65536, shard_prompts=15, per_prom
 
 
 # ------------------------------------------------------------------------------- oracle timing
-def oracle_step(w, n):
+def oracle_pass(w, n):
     """The oracle, as it stands, on the first n prompts of the workload (budget scaled with n).
-    Returns the seconds spent inside oracle calls (input generation excluded)."""
+    Returns the seconds spent inside oracle calls (input generation excluded) and what it computed."""
     from oracle import hora_oracle as orc
     sl = slice(0, n)
     alpha, beta, c, cap = w.alpha[sl], w.beta[sl], w.c[sl], w.cap[sl]
@@ -538,17 +546,78 @@ def oracle_step(w, n):
     tok = sub.token_offsets(R)
     t2 = time.perf_counter()
     adv = orc.group_advantage(rewards, off, w.adv_mode, float(np.float32(w.eps)), w.ddof)
-    orc.token_broadcast(adv[:R], tok)
+    token_adv = orc.token_broadcast(adv[:R], tok)
     t3 = time.perf_counter()
-    return (t1 - t0) + (t3 - t2)
+    return {"seconds": (t1 - t0) + (t3 - t2), "n": n, "B": B, "delta": d, "G": G, "lambda": lam, "objective": obj,
+            "offsets": off, "rewards": rewards, "adv": adv, "R": R, "token_offsets": tok, "token_adv": token_adv,
+            "workload": sub}
 
 
-def cpu_baseline(w, n):
+def oracle_step(w, n):
+    return oracle_pass(w, n)["seconds"]
+
+
+def cpu_baseline(w, n, ref=None):
     n = min(n, w.N)
-    secs = oracle_step(w, n)
+    secs = (ref if ref is not None else oracle_pass(w, n))["seconds"]
     return {"value": n / secs, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(secs, 2),
             "sample": f"first {n} of {w.N} prompts of {WORKLOAD} (budget and token count scaled by the same factor), "
                       "one pass: long-double gain rows, heap greedy, group advantages, token repeat"}
+
+
+def check_against_oracle(torch, hora, dev, ref, band=1e-12):
+    """Runs the four calls on the prompts the oracle pass covered and compares every output with the oracle's:
+    Delta may differ only on candidates whose oracle gain is within `band` (relative) of the oracle threshold,
+    G and the offsets must follow from Delta, lambda and the objective agree to 1e-12 relative, advantages to
+    1e-5 absolute (on the oracle's group layout), the token broadcast bitwise.  Raises on any violation."""
+    from oracle import hora_oracle as orc
+    w = ref["workload"]
+    n, ld, G0, B = ref["n"], w.ld, w.G0, ref["B"]
+    alpha, beta = torch.from_numpy(w.alpha).to(dev), torch.from_numpy(w.beta).to(dev)
+    c = torch.from_numpy(w.c).to(dev)
+    al = hora.Allocator(n, ld, G0, exact_int=False, device=dev)
+    al.run(alpha, beta, w.alpha0, w.beta0, c, None, ld, B)
+    info = al.read_info()
+    if info.status != 0:
+        raise RuntimeError(f"parity check: allocation failed: {hora.status_string(info.status)}")
+    d = al.delta.cpu().numpy()
+    if int(d.astype(np.int64).sum()) != B or (d < 0).any() or (d > w.cap).any():
+        raise RuntimeError("parity check: Delta is not a feasible allocation")
+    if not np.array_equal(al.G.cpu().numpy(), G0 + d):
+        raise RuntimeError("parity check: G != G0 + Delta")
+    off = np.zeros(n + 1, np.int64)
+    np.cumsum((G0 + d).astype(np.int64), out=off[1:])
+    if not np.array_equal(al.group_offsets.cpu().numpy(), off):
+        raise RuntimeError("parity check: group offsets are not the prefix sums of G")
+    lam = ref["lambda"]
+    differ = np.nonzero(d != ref["delta"])[0]
+    in_band = 0
+    for i in differ:
+        lo, hi = sorted((int(d[i]), int(ref["delta"][i])))
+        a_i, b_i = float(w.alpha[i]) + int(w.c[i]), float(w.beta[i]) + (G0 - int(w.c[i]))
+        for D in range(lo + 1, hi + 1):
+            g = orc.gain_one(a_i, b_i, D)
+            if abs(g - lam) > band * lam:
+                raise RuntimeError(f"parity check: Delta differs outside the band at prompt {i}, candidate {D}")
+            in_band += 1
+    if abs(info.lambda_ - lam) > 1e-12 * lam or abs(info.objective - ref["objective"]) > 1e-12 * ref["objective"]:
+        raise RuntimeError("parity check: threshold or objective differ from the oracle's")
+    rewards = torch.from_numpy(ref["rewards"]).to(dev)
+    off_o = torch.from_numpy(ref["offsets"]).to(dev)
+    adv = torch.empty_like(rewards)
+    hora.hora_group_advantage(rewards, off_o, n, w.adv_mode, float(w.eps), w.ddof, adv)
+    adv_err = float(np.abs(adv.cpu().numpy().astype(np.float64) - ref["adv"].astype(np.float64)).max())
+    if not adv_err <= 1e-5:
+        raise RuntimeError(f"parity check: advantages differ by {adv_err}")
+    R, tok_h = ref["R"], ref["token_offsets"]
+    T = int(tok_h[-1])
+    token_adv = torch.empty(T, dtype=torch.float32, device=dev)
+    hora.hora_token_broadcast(torch.from_numpy(ref["adv"][:R].copy()).to(dev), torch.from_numpy(tok_h).to(dev), R, T,
+                              token_adv)
+    if not np.array_equal(token_adv.cpu().numpy().view(np.uint32), ref["token_adv"].view(np.uint32)):
+        raise RuntimeError("parity check: token broadcast differs")
+    return {"parity_checked": True, "prompts": n, "delta_differences": int(len(differ)),
+            "band_differences": in_band, "adv_max_abs_err": adv_err, "tokens_compared": T}
 
 
 def reference_sample_size(steps: int, warmup: int, N: int) -> int:

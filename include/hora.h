@@ -49,7 +49,9 @@ typedef enum hora_status {
     HORA_ERR_NOT_INTEGER = 4,    /* HORA_FLAG_EXACT_INT given but some alpha_i or beta_i is not a positive integer */
     HORA_ERR_EXACT_RANGE = 5,    /* exact path: parameters too large for 128-bit integers or too many tie types */
     HORA_ERR_WORKSPACE = 6,      /* workspace missing, misaligned (needs 256 B) or too small */
-    HORA_ERR_CUDA = 7            /* a CUDA runtime call or kernel launch failed */
+    HORA_ERR_CUDA = 7,           /* a CUDA runtime call or kernel launch failed */
+    HORA_ERR_INTERNAL = 8        /* device data: a consistency check inside the selection failed (a fault of the
+                                    library, never of the inputs); reported like the other data-dependent errors */
 } hora_status_t;
 
 enum {
@@ -126,7 +128,7 @@ hora_status_t hora_gains(const double *alpha, const double *beta, double alpha0,
  *   B                number of Phase-B rollouts, 0 <= B <= sum_i cap_i
  *   workspace        device scratch, 256-byte aligned, at least hora_allocate_workspace_bytes(...);
  *                    contents are undefined on entry and on exit
- * Data-dependent failures (INVALID_VALUE, INFEASIBLE, NOT_INTEGER, EXACT_RANGE) set info_dev->status and
+ * Data-dependent failures (INVALID_VALUE, INFEASIBLE, NOT_INTEGER, EXACT_RANGE, INTERNAL) set info_dev->status and
  * leave delta, G and group_offsets all zero.
  * One of the call's kernels is launched cooperatively (all its thread blocks resident at once, sized per device
  * on first use); a device or context without cooperative launch makes the call return HORA_ERR_CUDA.
@@ -159,7 +161,9 @@ hora_status_t hora_allocate(const double *alpha, const double *beta, double alph
  *     matrix itself must fit, so only small problems (N*ld*8 bytes well under 8 MiB) qualify.
  *   - First use: the first call on each device looks up the array's device address (cudaGetSymbolAddress)
  *     with that device current, and caches it (as hora_allocate caches, per device, how many thread blocks of
- *     its cooperative kernel fit at once).  Make that first call outside any stream capture.
+ *     its cooperative kernel fit at once).  Make that first call outside any stream capture.  The cached
+ *     address belongs to the device's context: after cudaDeviceReset it is stale, and the library must be
+ *     reloaded before the call is used again.
  *   - Sharing: every call on a device uses the same array.  It keeps whatever the previous call left there;
  *     each call clears the parts it needs zeroed before using them, so back-to-back calls on one stream
  *     are fine.  Two calls that overlap on the GPU (different streams, or different host threads without

@@ -35,7 +35,7 @@ def utility(a: Fraction, b: Fraction, Delta: int) -> Fraction:
 
 
 def greedy(ab: Sequence[Tuple[Fraction, Fraction]], cap: Sequence[int], B: int) -> List[int]:
-    """Algorithm 1, Phase B, line by line in spirit: B times, give one rollout to the prompt with
+    """The greedy rule of Algorithm 1, Phase B: B times, give one rollout to the prompt with
     the largest current marginal gain.  Ties go to the lowest prompt index (``max`` over an
     ascending scan with a strict comparison); prompts at their cap are not eligible."""
     N = len(ab)

@@ -3,7 +3,7 @@
 Appendix "Prior-design predictor details": Eq. posterior-learned with the confidence s parametrised through a
 softplus and clamped to [0.25, 16] (fixed s = 2 for the single-head variants), and the per-prompt Beta-Binomial
 negative log-likelihood.  Pinned in tests/test_oracle_pins.py by the s = 2, p_hat = 1/2 collapse to the uniform
-prior, by closed forms (G0 = 1), by normalisation over c, and by the large-s limit (the binomial NLL)."""
+prior, by closed forms (G0 = 1), by normalisation over c, and by the large-s limit (the binomial NLL, approached like 1/s)."""
 from __future__ import annotations
 
 import math

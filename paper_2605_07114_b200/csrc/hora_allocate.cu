@@ -1079,7 +1079,10 @@ __device__ void tail_list(int64_t B, AllocHeader *hdr, const unsigned long long 
         next_digit(resolved, &bits, &shift);
         long long above = 0, count = 0;
         const int digit = locate_rank(hist1, 1 << bits, need, &above, &count, s_warp);
-        if (digit < 0) return;                                   // cannot happen: need lies within the list
+        if (digit < 0) {                                         // the rank must lie within the list: an internal fault
+            if (tid == 0) raise_status(&hdr->status, HORA_ERR_INTERNAL);
+            return;
+        }
         need -= above;
         prefix |= (unsigned long long)digit << shift;
         resolved += bits;
@@ -1132,7 +1135,10 @@ __device__ void tail_list(int64_t B, AllocHeader *hdr, const unsigned long long 
             }
         }
         __syncthreads();
-        if (s_pick[0] < 0) return;                               // cannot happen (keys are non-negative doubles)
+        if (s_pick[0] < 0) {                                     // keys are non-negative doubles: an internal fault
+            if (tid == 0) raise_status(&hdr->status, HORA_ERR_INTERNAL);
+            return;
+        }
         prefix = (unsigned long long)s_pick[0];
         need -= s_pick[1];
         left = s_pick[2];
@@ -1164,7 +1170,10 @@ __device__ void tail_list(int64_t B, AllocHeader *hdr, const unsigned long long 
         }
         __syncthreads();
         locate_rank_shared(s_hist, bins, need, s_warp, s_pick);
-        if (s_pick[0] < 0) return;                               // cannot happen
+        if (s_pick[0] < 0) {                                     // the rank left the histogram: an internal fault
+            if (tid == 0) raise_status(&hdr->status, HORA_ERR_INTERNAL);
+            return;
+        }
         need -= s_pick[1];
         prefix |= (unsigned long long)s_pick[0] << shift;
         resolved += bits;
@@ -1408,8 +1417,9 @@ exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ t
     __shared__ int s_slot[kMaxTypes];
     __shared__ int s_n;
     __shared__ int s_err;
+    __shared__ unsigned long long s_writer;
     if (hdr->status != 0) return;
-    if (threadIdx.x == 0) { s_n = 0; s_err = 0; }
+    if (threadIdx.x == 0) { s_n = 0; s_err = 0; s_writer = ~0ull; }
     __syncthreads();
     for (int h = threadIdx.x; h < kTypeSlots; h += blockDim.x) {
         tlabel[h] = 0;
@@ -1444,12 +1454,19 @@ exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ t
         if (above + equal < Rp) label = 2;
         else if (above < Rp) label = 1;
         tlabel[s_slot[t]] = label;
-        if (label == 1) {          // every member of the threshold class writes the same values
+        if (label == 1) {
+            // Members of the threshold class agree on R, but their unreduced num/den differ, and so may the
+            // last bit of the quotient below: the member with the smallest packed type (a, b, Delta) alone
+            // reports lambda (table slots depend on the insertion order, types do not).
             hdr->R = Rp - above;
-            hdr->lambda = ((double)s_num[t].hi * 18446744073709551616.0 + (double)s_num[t].lo) /
-                          ((double)s_den[t].hi * 18446744073709551616.0 + (double)s_den[t].lo);
+            atomicMin(&s_writer, tkeys[s_slot[t]]);
         }
     }
+    __syncthreads();
+    for (int t = threadIdx.x; t < n; t += blockDim.x)
+        if (tkeys[s_slot[t]] == s_writer)
+            hdr->lambda = ((double)s_num[t].hi * 18446744073709551616.0 + (double)s_num[t].lo) /
+                          ((double)s_den[t].hi * 18446744073709551616.0 + (double)s_den[t].lo);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -1654,6 +1671,9 @@ select_out(const double *__restrict__ alpha, const double *__restrict__ beta, do
     }
 }
 
+// Marks the call failed from the host's side (a launch that could not be made after others were enqueued).
+__global__ void fail_call(AllocHeader *hdr, int32_t code) { raise_status(&hdr->status, code); }
+
 // N == 0: nothing to select; still produce a well-defined summary.
 __global__ void write_empty(int64_t B, int64_t *offsets, hora_alloc_info *info) {
     if (offsets) offsets[0] = 0;
@@ -1770,6 +1790,11 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     const Workspace w = carve(workspace, N, ld, gains == nullptr, exact);
     if (workspace_bytes < w.bytes) return HORA_ERR_WORKSPACE;
     const int64_t NB = (N + kRowsPerBlock - 1) / kRowsPerBlock;
+    // the cooperative tail: every CTA must be resident at once, so the grid is what the device can hold; asked
+    // before anything is enqueued, so that a device without cooperative launch leaves the outputs untouched
+    const int tail_grid = B > 0 ? tail_grid_size() : 0;
+    if (B > 0 && tail_grid <= 0) return HORA_ERR_CUDA;
+    bool launch_failed = false;
 
     // header and histograms are contiguous at the start of the workspace
     const size_t zero_bytes = reinterpret_cast<char *>(w.rowstate) - reinterpret_cast<char *>(w.hdr);
@@ -1832,9 +1857,6 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
                                                                w.active, w.cand_key, w.cand_row, w.bsum_hi, objrow);
         mark_stage(3, s);
         {
-            // the cooperative tail: every CTA must be resident at once, so the grid is what the device can hold
-            const int tail_grid = tail_grid_size();
-            if (tail_grid <= 0) return HORA_ERR_CUDA;
             int64_t N_ = N, B_ = B, NB_ = NB;
             int32_t ld_ = ld;
             AllocHeader *hdr_ = w.hdr;
@@ -1846,8 +1868,13 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
             const int32_t *cr_ = w.cand_row;
             void *args[] = {&N_, &ld_, &gains, &B_, &hdr_, &hist_, &rowstate_, &active_, &bhi_, &bt_, &NB_, &ck_, &cr_};
             if (cudaLaunchCooperativeKernel(reinterpret_cast<void *>(select_tail), dim3(tail_grid), dim3(kSelThreads), args,
-                                            0, s) != cudaSuccess)
-                return HORA_ERR_CUDA;
+                                            0, s) != cudaSuccess) {
+                // the passes before it are already enqueued: mark the call failed on the device, so that the
+                // output pass below leaves zeroed outputs and the status in info_dev
+                (void)cudaGetLastError();
+                fail_call<<<1, 1, 0, s>>>(w.hdr, HORA_ERR_CUDA);
+                launch_failed = true;
+            }
         }
         mark_stage(4, s);
         if (exact) {
@@ -1870,6 +1897,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
                                                group_offsets, out_vec, info_dev);
     mark_stage(6, s);
     count_launches(B > 0 ? (exact ? 9 : 6) : 3);
+    if (launch_failed) return HORA_ERR_CUDA;
     return cuda_ok(cudaGetLastError());
 }
 

@@ -18,10 +18,11 @@ extern "C" const char *hora_status_string(hora_status_t status) {
         case HORA_ERR_EXACT_RANGE: return "exact mode: parameters out of range";
         case HORA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case HORA_ERR_CUDA: return "CUDA runtime error";
+        case HORA_ERR_INTERNAL: return "internal consistency check failed";
     }
     return "unknown status";
 }
 
-extern "C" int hora_version(void) { return 100; }
+extern "C" int hora_version(void) { return 200; }
 
 extern "C" uint64_t hora_launch_count(void) { return hora::g_launches.load(std::memory_order_relaxed); }

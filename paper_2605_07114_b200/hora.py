@@ -16,7 +16,8 @@ import torch
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhora.so")
 
-OK, ERR_INVALID_ARG, ERR_INVALID_VALUE, ERR_INFEASIBLE, ERR_NOT_INTEGER, ERR_EXACT_RANGE, ERR_WORKSPACE, ERR_CUDA = range(8)
+(OK, ERR_INVALID_ARG, ERR_INVALID_VALUE, ERR_INFEASIBLE, ERR_NOT_INTEGER, ERR_EXACT_RANGE, ERR_WORKSPACE, ERR_CUDA,
+ ERR_INTERNAL) = range(9)
 FLAG_EXACT_INT = 1
 FLAG_SKIP_OBJECTIVE = 2
 ADV_GRPO, ADV_RLOO = 0, 1

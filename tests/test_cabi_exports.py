@@ -72,3 +72,22 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     assert lib.hora_group_advantage(None, None, 5, 7, 0.0, 0, None, None, None) == 1                # unknown mode
     assert lib.hora_group_advantage(None, None, 5, 0, 0.0, 2, None, None, None) == 1                # ddof
     assert lib.hora_group_advantage(None, None, 0, 0, 0.0, 0, None, None, None) == 0
+
+
+def test_allocate_refuses_what_the_host_can_see(lib):
+    """hora_allocate: more than 2^31 - 1 prompts (row indices are kept in 32 bits), negative sizes, a cap above
+    ld and unknown flags are refused with INVALID_ARG before the device is touched."""
+    i64, i32, f64, p, u32 = ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.c_void_p, ctypes.c_uint32
+    lib.hora_allocate.argtypes = [p, p, f64, f64, p, i32, p, i32, i64, i32, p, i64, u32, p, p, p, p, p, ctypes.c_size_t, p]
+
+    def call(N=10, ld=8, G0=4, B=5, cap_scalar=8, flags=0, alpha0=1.0):
+        return lib.hora_allocate(None, None, alpha0, 1.0, None, G0, None, cap_scalar, N, ld, None, B, flags, None, None,
+                                 None, None, None, 0, None)
+
+    assert call(N=1 << 31) == 1
+    assert call(N=(1 << 31) + 12345) == 1
+    assert call(N=-1) == 1 and call(ld=0) == 1 and call(G0=-1) == 1 and call(B=-1) == 1
+    assert call(cap_scalar=9) == 1 and call(flags=64) == 1 and call(alpha0=0.0) == 1
+    assert call(N=(1 << 31) - 1) == 1          # in range, but c / delta / G are missing
+    lib.hora_status_string.restype = ctypes.c_char_p
+    assert b"internal" in lib.hora_status_string(8)

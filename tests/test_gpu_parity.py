@@ -196,8 +196,9 @@ def test_edge_budgets_and_caps():
     assert info.status == 0 and d[200] == 4 and d.sum() == 4
 
 
+@pytest.mark.parametrize("materialise", [True, False])
 @pytest.mark.parametrize("exact", [True, False])
-def test_allocation_when_the_sampled_window_misses(exact):
+def test_allocation_when_the_sampled_window_misses(exact, materialise):
     """The full-read pass refines 23 bits inside a window placed from a sample of every k-th row.  Here the
     sampled rows (index multiple of 5) are all hopeless prompts and the others all saturated ones, so the
     sample says nothing about the threshold and the window lands in the wrong place: the selection must
@@ -218,11 +219,33 @@ def test_allocation_when_the_sampled_window_misses(exact):
             d_o, _, lam, obj = orc.greedy_exact(None, None, 1.0, 1.0, c, G0, cap, B)
         else:
             d_o, _, lam, obj = orc.greedy_real(alpha, beta, 1.0, 1.0, c, G0, cap, B)
-        d, G, off, info = gu.gpu_allocate(alpha, beta, 1.0, 1.0, c, G0, cap, ld, B, exact=exact)
+        d, G, off, info = gu.gpu_allocate(alpha, beta, 1.0, 1.0, c, G0, cap, ld, B, exact=exact,
+                                          materialise=materialise)
         assert info.status == 0
         assert info.first_pass_bits == 13            # the window did miss: this is the fallback being tested
         np.testing.assert_array_equal(d, d_o)
         assert abs(info.objective - obj) <= 1e-12 * obj
+
+
+@pytest.mark.parametrize("materialise", [True, False])
+@pytest.mark.parametrize("exact", [True, False])
+def test_heavy_ties_take_the_digit_route_at_moderate_size(exact, materialise):
+    """One posterior class, 2^17 prompts: the threshold is a value that 131072 candidates share, more than the
+    candidate list holds, so the tail narrows the rows digit by digit — with the matrix given and with the
+    matrix built inside the call.  The result is a pure index tie-break."""
+    gu = _util()
+    N, G0, ld = 1 << 17, 4, 24
+    c = np.zeros(N, np.int32)
+    cap = np.full(N, ld, np.int32)
+    cap[::7] = 5                                     # some rows end before the threshold's column
+    B = 9 * N + 4321
+    d_o, _, lam, obj = orc.greedy_exact(None, None, 1.0, 1.0, c, G0, cap, B)
+    d, G, off, info = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, cap, ld, B, exact=exact, materialise=materialise)
+    assert info.status == 0
+    assert info.n_tied > 65536                       # what forces the digit route
+    np.testing.assert_array_equal(d, d_o)
+    np.testing.assert_array_equal(off, np.concatenate(([0], np.cumsum(G0 + d_o.astype(np.int64)))))
+    assert abs(info.objective - obj) <= 1e-12 * obj
 
 
 def test_allocation_with_long_rows():

@@ -451,6 +451,12 @@ def test_learned_prior_front_end_pins():
     nll = prior.beta_binomial_nll([0.5] * (G0 + 1), list(range(G0 + 1)), G0, None, 2.0)
     for c in range(G0 + 1):
         assert math.comb(G0, c) * math.exp(-nll[c]) == pytest.approx(1.0 / (G0 + 1), rel=1e-12)
+    # large confidence: the posterior over the success rate collapses on p_hat and the loss tends to the binomial
+    # negative log-likelihood -[c log p_hat + (G0 - c) log(1 - p_hat)], with an error that shrinks like 1/s
+    for p_hat, c in ((0.3, 2), (0.71, 8), (0.5, 0)):
+        binom = -(c * math.log(p_hat) + (G0 - c) * math.log(1 - p_hat))
+        err = [abs(prior.beta_binomial_nll([p_hat], [c], G0, None, s)[0] - binom) for s in (1e3, 1e4, 1e5)]
+        assert err[2] < 1e-3 * binom and err[0] > 5 * err[1] > 25 * err[2]
     # agreement with a library log-Beta
     a, b = prior.learned_prior([0.37], None, 5.0)
     assert prior.beta_binomial_nll([0.37], [3], 8, None, 5.0)[0] == pytest.approx(
