@@ -47,7 +47,8 @@ typedef enum hora_status {
                                     a gain row that is not finite/non-negative/non-increasing, offsets that decrease */
     HORA_ERR_INFEASIBLE = 3,     /* B > sum_i cap_i */
     HORA_ERR_NOT_INTEGER = 4,    /* HORA_FLAG_EXACT_INT given but some alpha_i or beta_i is not a positive integer */
-    HORA_ERR_EXACT_RANGE = 5,    /* exact path: parameters too large for 128-bit integers or too many tie types */
+    HORA_ERR_EXACT_RANGE = 5,    /* exact path: a near-threshold gain does not fit the 512-bit exact form (see
+                                    hora_allocate), alpha+beta+G0+ld >= 2^20, or more than 1024 distinct tie types */
     HORA_ERR_WORKSPACE = 6,      /* workspace missing, misaligned (needs 256 B) or too small */
     HORA_ERR_CUDA = 7,           /* a CUDA runtime call or kernel launch failed */
     HORA_ERR_INTERNAL = 8        /* device data: a consistency check inside the selection failed (a fault of the
@@ -118,8 +119,13 @@ hora_status_t hora_gains(const double *alpha, const double *beta, double alpha0,
  * Ties.  Without HORA_FLAG_EXACT_INT a tie is equality of the fp64 gains as hora_gains computes
  * them.  With HORA_FLAG_EXACT_INT (every alpha_i, beta_i a positive integer) candidates within a
  * relative band of 2^-30 around the fp64 threshold are re-ranked on exact integers
- * (g = a*(b)_a / (b+Delta-1)_{a+1} compared by 256-bit cross multiplication), so a tie is an exact
- * rational equality and the result equals exact greedy with lowest-index tie-breaking.
+ * (g = a*(b)_a / (b+Delta-1)_{a+1}, or the equal a*(b)_{Delta-1} / (a+b)_Delta when that has fewer factors,
+ * numerator and denominator in 512 bits, compared by cross multiplication), so a tie is an exact rational
+ * equality and the result equals exact greedy with lowest-index tie-breaking.  Guaranteed range of the exact
+ * form: with m = min(a_i + 1, Delta) factors, each below a_i + b_i + Delta, m * log2(a_i + b_i + Delta) <= 512 —
+ * e.g. any posterior with a_i <= 50 up to Delta = 1000 (this covers G0 = 16 and learned priors with
+ * alpha_i + beta_i <= 16), or any a_i at all up to Delta = 25.  Only candidates near the threshold are ever
+ * formed exactly; one that does not fit raises HORA_ERR_EXACT_RANGE (nothing wraps).
  *
  *   alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld   as for hora_gains
  *   gains            [N*ld] the matrix hora_gains wrote for the same inputs, or NULL to have it built
@@ -131,7 +137,9 @@ hora_status_t hora_gains(const double *alpha, const double *beta, double alpha0,
  * Data-dependent failures (INVALID_VALUE, INFEASIBLE, NOT_INTEGER, EXACT_RANGE, INTERNAL) set info_dev->status and
  * leave delta, G and group_offsets all zero.
  * One of the call's kernels is launched cooperatively (all its thread blocks resident at once, sized per device
- * on first use); a device or context without cooperative launch makes the call return HORA_ERR_CUDA.
+ * on first use); a device or context without cooperative launch makes the call return HORA_ERR_CUDA before
+ * anything is enqueued.  Should that launch fail after the earlier passes were enqueued, the call still returns
+ * HORA_ERR_CUDA, with zeroed delta / G / group_offsets and the code in info_dev->status.
  */
 size_t hora_allocate_workspace_bytes(int64_t N, int32_t ld, int32_t gains_is_null, uint32_t flags);
 

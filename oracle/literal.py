@@ -55,5 +55,30 @@ def greedy(ab: Sequence[Tuple[Fraction, Fraction]], cap: Sequence[int], B: int) 
     return delta
 
 
+def greedy_heap(ab: Sequence[Tuple[Fraction, Fraction]], cap: Sequence[int], B: int):
+    """The same B greedy steps with the argmax kept in a binary heap (key: gain descending, prompt index
+    ascending), in unbounded Python integers: for sizes the O(B*N) scan above is too slow for, and for integer
+    posteriors whose exact gains outgrow any fixed word size.  Returns (delta, gain of the last rollout given)."""
+    import heapq
+    N = len(ab)
+    if B > sum(cap):
+        raise ValueError("infeasible")
+    delta = [0] * N
+    heap = [(-(a / (a + b)), i) for i, (a, b) in enumerate(ab) if cap[i] > 0]
+    heapq.heapify(heap)
+    last = Fraction(0)
+    for _ in range(B):
+        neg, i = heap[0]
+        last = -neg
+        a, b = ab[i]
+        l = delta[i]
+        delta[i] = l + 1
+        if delta[i] < cap[i]:
+            heapq.heapreplace(heap, (neg * (b + l) / (a + b + l + 1), i))
+        else:
+            heapq.heappop(heap)
+    return delta, last
+
+
 def objective(ab, delta) -> Fraction:
     return sum((utility(a, b, d) for (a, b), d in zip(ab, delta)), Fraction(0))

@@ -39,7 +39,7 @@
 // around lambda (far wider than the fp64 evaluation error, far narrower than the gap between two
 // entries of one row) are the only ones whose exact rank is in doubt.  Each row has at most one.
 // Their types (a, b, Delta) are collected in a small hash table with instance counts, ranked exactly
-// by 256-bit cross multiplication of num/den = a (b)_a / (b+Delta-1)_{a+1}  (or the equivalent
+// by cross multiplication in 1024-bit integers of num/den = a (b)_a / (b+Delta-1)_{a+1}  (or the equivalent
 // a (b)_{Delta-1} / (a+b)_Delta when that has fewer factors), and the threshold class is found by
 // walking the ranked types.  Rows are relabelled above / tied / below and the same sum/out steps run.
 #include <cooperative_groups.h>
@@ -1325,7 +1325,7 @@ select_tail(int64_t N, int32_t ld, const double *__restrict__ gains, int64_t B, 
     tail_digits(N, ld, gains, B, hdr, hist_all, rowstate, active, bsum_hi, bsum_t, NB, s_hist, s_warp);
 }
 
-// (exact 128/256-bit helpers: hora_exact.cuh)
+// (exact multi-word integer helpers: hora_exact.cuh)
 
 __device__ __forceinline__ unsigned long long pack_type(unsigned long long a, unsigned long long b, unsigned long long D) {
     return (a << 43) | (b << 22) | D;   // a, b < 2^21, D < 2^22
@@ -1409,12 +1409,18 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
 
 // Exact mode, step 2 (one CTA): rank the collected types exactly and label them.
 //   label 2: strictly better than the threshold class (taken)   1: threshold class   0: worse
-__global__ void __launch_bounds__(1024)
+// Numerators and denominators (512 bits each) live in dynamic shared memory: kExactRankSmem bytes.
+constexpr int kExactRankThreads = 256;
+constexpr size_t kExactRankSmem = (size_t)kMaxTypes * (2 * sizeof(UBig) + sizeof(unsigned long long) + sizeof(int));
+
+__global__ void __launch_bounds__(kExactRankThreads)
 exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ tkeys,
            const unsigned long long *__restrict__ tcounts, int32_t *__restrict__ tlabel) {
-    __shared__ U128 s_num[kMaxTypes], s_den[kMaxTypes];
-    __shared__ unsigned long long s_cnt[kMaxTypes];
-    __shared__ int s_slot[kMaxTypes];
+    extern __shared__ __align__(16) unsigned char s_rank_raw[];
+    UBig *s_num = reinterpret_cast<UBig *>(s_rank_raw);
+    UBig *s_den = s_num + kMaxTypes;
+    unsigned long long *s_cnt = reinterpret_cast<unsigned long long *>(s_den + kMaxTypes);
+    int *s_slot = reinterpret_cast<int *>(s_cnt + kMaxTypes);
     __shared__ int s_n;
     __shared__ int s_err;
     __shared__ unsigned long long s_writer;
@@ -1427,7 +1433,7 @@ exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ t
         if (key != 0ull) {
             const int j = atomicAdd(&s_n, 1);
             if (j < kMaxTypes) {
-                U128 nu, de;
+                UBig nu, de;
                 if (!exact_gain(key >> 43, (key >> 22) & 0x1FFFFFull, key & 0x3FFFFFull, nu, de)) s_err = 1;
                 s_num[j] = nu;
                 s_den[j] = de;
@@ -1464,9 +1470,7 @@ exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ t
     }
     __syncthreads();
     for (int t = threadIdx.x; t < n; t += blockDim.x)
-        if (tkeys[s_slot[t]] == s_writer)
-            hdr->lambda = ((double)s_num[t].hi * 18446744073709551616.0 + (double)s_num[t].lo) /
-                          ((double)s_den[t].hi * 18446744073709551616.0 + (double)s_den[t].lo);
+        if (tkeys[s_slot[t]] == s_writer) hdr->lambda = ratio_double(s_num[t], s_den[t]);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -1880,7 +1884,10 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         if (exact) {
             exact_collect<<<grid_rows, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
                                                             gains, w.hdr, w.rowstate, w.rowslot, w.tkeys, w.tcounts);
-            exact_rank<<<1, 1024, 0, s>>>(B, w.hdr, w.tkeys, w.tcounts, w.tlabel);
+            if (cudaFuncSetAttribute(exact_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kExactRankSmem) !=
+                cudaSuccess)
+                launch_failed = true;
+            exact_rank<<<1, kExactRankThreads, kExactRankSmem, s>>>(B, w.hdr, w.tkeys, w.tcounts, w.tlabel);
             select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 0, N, ld, gains, 2, B,
                                                        w.hdr, w.rowstate, w.rowslot, w.tlabel, w.bsum_hi, w.bsum_t, NB);
         }

@@ -9,7 +9,7 @@
 //   2  the B_s-th largest key by a radix selection over the shared-memory keys (11-bit digits);
 //   3  per row the number of keys above and equal to the threshold (binary search in the sorted row);
 //   4  ties: in prompt order (fp64 equality), or, in exact mode, by exact rational comparison of the at
-//      most one candidate per row that lies within 2^-30 of the threshold (pairwise, 256-bit products);
+//      most one candidate per row that lies within 2^-30 of the threshold (pairwise, cross-multiplied);
 //   5  Delta, G, the segment's summary.
 // Group offsets over all prompts are an exclusive scan of G by two small kernels afterwards.
 #include <algorithm>
@@ -44,14 +44,14 @@ struct BatchedSmemFixed {
 // calls with short segments — the paper's 15 prompts — leave shared memory for a fourth CTA per SM).
 struct BatchedRows {
     double *a, *b;
-    U128 *num, *den;
+    UBig *num, *den;
     int32_t *cap, *band;
 };
-constexpr size_t kBRowBytes = 2 * sizeof(double) + 2 * sizeof(U128) + 2 * sizeof(int32_t);   // 56 bytes per prompt
+constexpr size_t kBRowBytes = 2 * sizeof(double) + 2 * sizeof(UBig) + 2 * sizeof(int32_t);   // 152 bytes per prompt
 
 __device__ __forceinline__ BatchedRows carve_rows(unsigned char *base, int rows_cap) {
     BatchedRows r;
-    r.num = reinterpret_cast<U128 *>(base);
+    r.num = reinterpret_cast<UBig *>(base);
     r.den = r.num + rows_cap;
     r.a = reinterpret_cast<double *>(r.den + rows_cap);
     r.b = r.a + rows_cap;
@@ -253,7 +253,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                 has = (q < my_cap) && (row[q] >= k_lo);
                 if (has && q + 1 < my_cap && row[q + 1] >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
                 if (has && !err) {
-                    U128 nu, de;
+                    UBig nu, de;
                     if (!exact_gain((unsigned long long)rw.a[threadIdx.x], (unsigned long long)rw.b[threadIdx.x],
                                     (unsigned long long)q + 1, nu, de)) err = HORA_ERR_EXACT_RANGE;
                     rw.num[threadIdx.x] = nu;
@@ -282,9 +282,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                     sm.found[0] = tot_q + strictly;
                     sm.found[1] = equal + 1;
                     sm.found[2] = Rp - strictly;
-                    const U128 nu = rw.num[threadIdx.x], de = rw.den[threadIdx.x];
-                    lambda = ((double)nu.hi * 18446744073709551616.0 + (double)nu.lo) /
-                             ((double)de.hi * 18446744073709551616.0 + (double)de.lo);
+                    lambda = ratio_double(rw.num[threadIdx.x], rw.den[threadIdx.x]);
                     sm.lam_exact = lambda;
                 }
             } else {

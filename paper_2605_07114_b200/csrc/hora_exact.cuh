@@ -1,61 +1,79 @@
-// Exact integer arithmetic for the tie path (unsigned 128-bit values as two words, 256-bit products) and
-// the product form of the hit utility; shared by the single-problem and the batched allocation kernels.
+// Exact integer arithmetic for the tie path and the product form of the hit utility; shared by the
+// single-problem and the batched allocation kernels.
+//
+// For an integer posterior (a, b) the gain of Eq. marginal is a ratio of two products of small integers,
+//     g(Delta) = a (b)_a / (b + Delta - 1)_{a+1}          (x)_k = x (x+1) ... (x+k-1)
+//              = a (b)_{Delta-1} / (a + b)_Delta           (the same value; fewer factors when Delta <= a)
+// Numerator and denominator are held unreduced in kLimbs 64-bit words (512 bits); two gains are compared by
+// cross multiplication with 1024-bit products formed column by column, so nothing is ever rounded.  Whatever
+// does not fit is reported (never wrapped): m = min(a + 1, Delta) factors, each below a + b + Delta, must
+// satisfy m log2(a + b + Delta) <= 512 — any a <= 50 with Delta up to 1000, or any a at all with Delta <= 25.
 #pragma once
 
 #include "hora_common.cuh"
 
 namespace hora {
 
-// Exact arithmetic helpers (unsigned 128-bit as two words; overflow is reported, never wrapped).
-struct U128 { unsigned long long lo, hi; };
+constexpr int kLimbs = 8;
+struct UBig { unsigned long long w[kLimbs]; };              // little-endian words
 
-__device__ __forceinline__ bool mul_small(U128 &x, unsigned long long m) {   // returns false on overflow
-    const unsigned long long lo = x.lo * m, carry = __umul64hi(x.lo, m);
-    const unsigned long long hi = x.hi * m;
-    const bool ovf = (__umul64hi(x.hi, m) != 0) || (hi + carry < hi);
-    x.lo = lo;
-    x.hi = hi + carry;
-    return !ovf;
+__device__ __forceinline__ void set_small(UBig &x, unsigned long long v) {
+    x.w[0] = v;
+#pragma unroll
+    for (int i = 1; i < kLimbs; ++i) x.w[i] = 0ull;
 }
 
-// 128 x 128 -> 256 bit product, little-endian words
-__device__ __forceinline__ void mul_wide(const U128 &p, const U128 &q, unsigned long long r[4]) {
-    const unsigned long long a0 = p.lo, a1 = p.hi, b0 = q.lo, b1 = q.hi;
-    r[0] = a0 * b0;
-    const unsigned long long t1 = __umul64hi(a0, b0);
-    const unsigned long long l01 = a0 * b1, h01 = __umul64hi(a0, b1);
-    const unsigned long long l10 = a1 * b0, h10 = __umul64hi(a1, b0);
-    const unsigned long long s = t1 + l01;
-    unsigned long long c1 = s < t1;
-    const unsigned long long s2 = s + l10;
-    c1 += s2 < s;
-    r[1] = s2;
-    const unsigned long long l11 = a1 * b1, h11 = __umul64hi(a1, b1);
-    const unsigned long long q2 = h01 + h10;
-    unsigned long long c2 = q2 < h01;
-    const unsigned long long q3 = q2 + l11;
-    c2 += q3 < q2;
-    const unsigned long long q4 = q3 + c1;
-    c2 += q4 < q3;
-    r[2] = q4;
-    r[3] = h11 + c2;
-}
-
-// sign of x*y - u*v with full 256-bit products
-__device__ __forceinline__ int cmp_products(const U128 &x, const U128 &y, const U128 &u, const U128 &v) {
-    unsigned long long L[4], Rr[4];
-    mul_wide(x, y, L);
-    mul_wide(u, v, Rr);
-    for (int i = 3; i >= 0; --i) {
-        if (L[i] != Rr[i]) return L[i] > Rr[i] ? 1 : -1;
+// x *= m; returns false if the product does not fit (x is then meaningless)
+__device__ __forceinline__ bool mul_small(UBig &x, unsigned long long m) {
+    unsigned long long carry = 0ull;
+#pragma unroll
+    for (int i = 0; i < kLimbs; ++i) {
+        const unsigned long long lo = x.w[i] * m, hi = __umul64hi(x.w[i], m);
+        const unsigned long long s = lo + carry;
+        x.w[i] = s;
+        carry = hi + (s < lo ? 1ull : 0ull);                 // hi <= 2^64 - 2: no wrap
     }
-    return 0;
+    return carry == 0ull;
 }
 
-// Exact gain of type (a, b, Delta) as num/den (not reduced).  Returns false if 128 bits do not suffice.
-__device__ __forceinline__ bool exact_gain(unsigned long long a, unsigned long long b, unsigned long long Delta, U128 &num, U128 &den) {
-    num.lo = a; num.hi = 0;
-    den.lo = 1; den.hi = 0;
+// (c2, c1, c0) += p * q, a 192-bit accumulator
+__device__ __forceinline__ void mac192(unsigned long long &c0, unsigned long long &c1, unsigned long long &c2,
+                                       unsigned long long p, unsigned long long q) {
+    const unsigned long long lo = p * q, hi = __umul64hi(p, q);
+    c0 += lo;
+    const unsigned long long k0 = c0 < lo ? 1ull : 0ull;
+    const unsigned long long t = hi + k0;                    // hi <= 2^64 - 2: no wrap
+    c1 += t;
+    c2 += c1 < t ? 1ull : 0ull;
+}
+
+// sign of x*y - u*v.  The two 1024-bit products are formed a 64-bit column at a time from the bottom (three
+// words of running carry each), and the most significant column in which they differ decides.
+__device__ __forceinline__ int cmp_products(const UBig &x, const UBig &y, const UBig &u, const UBig &v) {
+    unsigned long long l0 = 0, l1 = 0, l2 = 0, r0 = 0, r1 = 0, r2 = 0;
+    int sign = 0;
+#pragma unroll
+    for (int k = 0; k < 2 * kLimbs; ++k) {
+#pragma unroll
+        for (int i = 0; i < kLimbs; ++i) {
+            const int j = k - i;
+            if (j >= 0 && j < kLimbs) {
+                mac192(l0, l1, l2, x.w[i], y.w[j]);
+                mac192(r0, r1, r2, u.w[i], v.w[j]);
+            }
+        }
+        if (l0 != r0) sign = l0 > r0 ? 1 : -1;
+        l0 = l1; l1 = l2; l2 = 0;
+        r0 = r1; r1 = r2; r2 = 0;
+    }
+    return sign;
+}
+
+// Exact gain of type (a, b, Delta) as num/den (not reduced).  Returns false if kLimbs words do not suffice.
+__device__ __forceinline__ bool exact_gain(unsigned long long a, unsigned long long b, unsigned long long Delta, UBig &num,
+                                           UBig &den) {
+    set_small(num, a);
+    set_small(den, 1ull);
     bool ok = true;
     if (a + 1 <= Delta) {               // a (b)_a / (b+Delta-1)_{a+1}
         for (unsigned long long k = 0; k < a && ok; ++k) ok = mul_small(num, b + k);
@@ -66,6 +84,17 @@ __device__ __forceinline__ bool exact_gain(unsigned long long a, unsigned long l
     }
     return ok;
 }
+
+// nearest double of a kLimbs-word integer, up to the rounding of the partial sums (used for reporting only)
+__device__ __forceinline__ double to_double(const UBig &x) {
+    double v = 0.0;
+#pragma unroll
+    for (int i = kLimbs - 1; i >= 0; --i) v = v * 18446744073709551616.0 + (double)x.w[i];
+    return v;
+}
+
+// num/den as a double (2^512 is far inside the range of a double; a handful of roundings, reporting only)
+__device__ __forceinline__ double ratio_double(const UBig &num, const UBig &den) { return to_double(num) / to_double(den); }
 
 // U(Delta) = 1 - prod_{j<Delta} (b+j)/(a+b+j)  (Eq. appendix-hit-closed-form written as a product)
 __device__ __forceinline__ double hit_utility(double a, double b, int32_t Delta) {

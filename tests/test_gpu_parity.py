@@ -157,6 +157,87 @@ def test_per_prompt_integer_priors_exact():
         np.testing.assert_array_equal(d, d_o)
 
 
+def _exact_oracle_any_width(alpha, beta, a0, b0, c, G0, cap, B):
+    """Exact greedy: the C oracle while its 128-bit reduced fractions suffice, else the Python-integer heap."""
+    from fractions import Fraction
+    from oracle import literal
+    try:
+        return orc.greedy_exact(alpha, beta, a0, b0, c, G0, cap, B)[0]
+    except orc.OracleError as e:
+        assert e.code == orc.OVERFLOW
+    al = np.full(len(c), a0) if alpha is None else alpha
+    be = np.full(len(c), b0) if beta is None else beta
+    ab = [literal.posterior(int(x), int(y), int(ci), G0) for x, y, ci in zip(al, be, c)]
+    return np.array(literal.greedy_heap(ab, [int(x) for x in cap], int(B))[0], np.int32)
+
+
+@pytest.mark.parametrize("prior_max,G0,ld", [(20, 8, 256), (40, 8, 256), (16, 16, 256), (3, 4, 1000)])
+def test_strong_integer_priors_exact(prior_max, G0, ld):
+    """Integer priors well beyond the uniform one: the exact numerators and denominators of the near-threshold
+    candidates outgrow 128 bits (a = 28 at Delta = 250 needs about 240), and the result must still be exact greedy."""
+    gu = _util()
+    rng = np.random.default_rng(prior_max * 100 + G0)
+    N = 400
+    alpha = rng.integers(1, prior_max + 1, N).astype(np.float64)
+    beta = rng.integers(1, prior_max + 1, N).astype(np.float64)
+    alpha[::3], beta[::3] = alpha[0], beta[0]            # repeated priors: exact ties between prompts
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    c[::3] = c[0]
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    total = int(cap.sum())
+    for B in (1, N, total // 4, total // 2, total - 5):
+        d_o = _exact_oracle_any_width(alpha, beta, 1.0, 1.0, c, G0, cap, B)
+        d, G, off, info = gu.gpu_allocate(alpha, beta, 1.0, 1.0, c, G0, cap, ld, B, exact=True)
+        assert info.status == 0, (B, info)
+        np.testing.assert_array_equal(d, d_o, err_msg=f"B={B}")
+
+
+def test_threshold_on_candidates_wider_than_128_bits():
+    """G0 = 16 with the uniform prior (the paper's G0 ablation, Table allocator-g0): a prompt with every Phase-A
+    rollout correct has a = 17, b = 1, and g(Delta) = 17 * 17! / (Delta)_18, whose denominator passes 2^128 near
+    Delta = 140.  Budgets that put the threshold on such candidates, alone and tied across classes, must
+    reproduce exact greedy with the lowest-index tie-break."""
+    gu = _util()
+    from fractions import Fraction
+    from oracle import literal
+    G0, ld, N = 16, 256, 300
+    rng = np.random.default_rng(16)
+    c = np.where(rng.random(N) < 0.5, G0, rng.integers(0, G0 + 1, N)).astype(np.int32)
+    cap = np.full(N, ld, np.int32)
+    # budgets whose threshold lies on a c = 16 candidate with Delta >= 150: take every candidate at least as good as
+    # g_{c=16}(Delta*), minus a few so that the last ones are handed out by index
+    ab = [literal.posterior(1, 1, int(ci), G0) for ci in c]
+    rows = {int(k): literal.marginals(*literal.posterior(1, 1, int(k), G0), ld) for k in set(c.tolist())}
+    for D_star in (150, 201, 256):
+        lam = rows[G0][D_star - 1]
+        B = sum(sum(1 for g in rows[int(ci)] if g >= lam) for ci in c) - 7
+        d_o, lam_o = literal.greedy_heap(ab, [ld] * N, B)
+        unreduced = 1
+        for k in range(18):
+            unreduced *= D_star + k                   # (Delta)_18, the denominator as the GPU path forms it
+        assert lam_o == lam and unreduced.bit_length() > 128
+        d, G, off, info = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, cap, ld, B, exact=True)
+        assert info.status == 0
+        np.testing.assert_array_equal(d, np.array(d_o, np.int32))
+        assert info.lambda_ == pytest.approx(float(lam), rel=1e-12)
+        d2, _, _, info2 = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, cap, ld, B, exact=True, materialise=False)
+        assert info2.status == 0
+        np.testing.assert_array_equal(d2, d)
+
+
+def test_exact_range_is_reported_not_wrapped():
+    """A posterior too strong for the 512-bit exact form (a about 5000 at Delta about 500) must give EXACT_RANGE and
+    zeroed outputs, never a wrong allocation."""
+    gu = _util()
+    N, G0, ld = 64, 4, 600
+    alpha = np.full(N, 5000.0)
+    beta = np.full(N, 3.0)
+    c = np.full(N, 2, np.int32)
+    cap = np.full(N, ld, np.int32)
+    d, G, off, info = gu.gpu_allocate(alpha, beta, 1.0, 1.0, c, G0, cap, ld, 500 * N + 3, exact=True)
+    assert info.status == 5 and not d.any() and not G.any()
+
+
 def test_single_class_is_pure_index_tie_break():
     gu = _util()
     N, G0, ld = 1000, 4, 8

@@ -206,6 +206,48 @@ def test_greedy_is_optimal_and_tie_broken_small(case):
     assert float(literal.objective(ab, [int(x) for x in d_r])) == pytest.approx(float(brute_force_best(ab, cap, B)), rel=1e-14)
 
 
+@pytest.mark.parametrize("case", small_integer_cases()[:30])
+def test_heap_greedy_in_python_integers_small(case):
+    """literal.greedy_heap against the O(B*N) scan, the global sort (a different algorithm) and brute force."""
+    G0, al, be, c, cap, B = case
+    ab = [literal.posterior(al, be, ci, G0) for ci in c]
+    d, lam = literal.greedy_heap(ab, cap, B)
+    assert d == literal.greedy(ab, cap, B) == sorted_top_B(ab, cap, B)
+    assert literal.objective(ab, d) == brute_force_best(ab, cap, B)
+    if B > 0:
+        assert lam == min(literal.marginals(a, b, x)[x - 1] for (a, b), x in zip(ab, d) if x > 0)
+
+
+def test_heap_greedy_beyond_128_bits():
+    """Strong integer priors (alpha, beta up to 64, G0 = 8, up to 300 extra rollouts): for the larger budgets the
+    reduced fractions no longer fit the C oracle's 128-bit words (it says so), the Python-integer heap carries on.  Pins: the global sort under
+    (gain desc, index asc, Delta asc), the exchange certificate (Eq. appendix-exchange-condition), and agreement
+    with the C oracle on the budgets it can still do."""
+    rng = np.random.default_rng(20)
+    N, G0, ld = 40, 8, 300
+    alpha = rng.integers(1, 65, N)
+    beta = rng.integers(1, 65, N)
+    c = rng.integers(0, G0 + 1, N)
+    cap = [int(x) for x in rng.integers(0, ld + 1, N)]
+    ab = [literal.posterior(int(al), int(be), int(ci), G0) for al, be, ci in zip(alpha, beta, c)]
+    gf = lambda a, b, D: literal.marginals(a, b, D)[D - 1]
+    overflowed = 0
+    for B in (1, 50, 700, sum(cap) // 2, sum(cap) - 3):
+        d, lam = literal.greedy_heap(ab, cap, B)
+        assert sum(d) == B and all(0 <= x <= cp for x, cp in zip(d, cap))
+        assert d == sorted_top_B(ab, cap, B)
+        assert exchange_certificate(gf, ab, cap, d)
+        assert lam == min(gf(a, b, x) for (a, b), x in zip(ab, d) if x > 0)
+        try:
+            d_c = orc.greedy_exact(alpha.astype(np.float64), beta.astype(np.float64), 1.0, 1.0, c.astype(np.int32), G0,
+                                   np.array(cap, np.int32), B)[0]
+            assert list(d_c) == d
+        except orc.OracleError as e:
+            assert e.code == orc.OVERFLOW
+            overflowed += 1
+    assert overflowed > 0                        # this case does leave the 128-bit range
+
+
 def test_worked_example_fixture():
     G0, c, cap = 2, (0, 1, 2, 0), (3, 3, 3, 3)
     ab = [literal.posterior(1, 1, ci, G0) for ci in c]
