@@ -57,7 +57,10 @@ typedef enum hora_status {
 
 enum {
     HORA_FLAG_EXACT_INT = 1u,      /* priors are integer-valued: decide ties by exact rational equality */
-    HORA_FLAG_SKIP_OBJECTIVE = 2u  /* do not compute hora_alloc_info.objective (left 0) */
+    HORA_FLAG_SKIP_OBJECTIVE = 2u, /* do not compute hora_alloc_info.objective (left 0) */
+    HORA_FLAG_SHARED_INT_PRIOR = 4u /* sizing hint for hora_allocate_workspace_bytes: the call will pass alpha == beta ==
+                                      NULL with integer alpha0, beta0, HORA_FLAG_EXACT_INT and gains == NULL (see the
+                                      rank-based route under hora_allocate); ignored by the calls themselves */
 };
 
 enum { HORA_ADV_GRPO = 0, HORA_ADV_RLOO = 1 };
@@ -68,7 +71,7 @@ enum { HORA_WEIGHT_PER_TOKEN = 0, HORA_WEIGHT_CONST_LENGTH = 1 };
 typedef struct hora_alloc_info {
     int32_t status;        /* hora_status_t of the data-dependent checks */
     int32_t first_pass_bits; /* diagnostic: key bits the full-read pass resolved (23 when its sampled window held the
-                                threshold, else 13); 0 when B == 0 */
+                                threshold, else 13); 0 when B == 0; -1 when the rank-based route ran (no key pass) */
     double  lambda;        /* gain of the B-th best candidate (the selection threshold); 0 when B == 0 */
     int64_t n_above;       /* candidates strictly better than lambda (all taken) */
     int64_t n_tied;        /* candidates equal to lambda */
@@ -126,6 +129,14 @@ hora_status_t hora_gains(const double *alpha, const double *beta, double alpha0,
  * e.g. any posterior with a_i <= 50 up to Delta = 1000 (this covers G0 = 16 and learned priors with
  * alpha_i + beta_i <= 16), or any a_i at all up to Delta = 25.  Only candidates near the threshold are ever
  * formed exactly; one that does not fit raises HORA_ERR_EXACT_RANGE (nothing wraps).
+ *
+ * Rank-based route.  With ONE integer prior for all prompts (alpha == beta == NULL, alpha0 and beta0 positive
+ * integers), HORA_FLAG_EXACT_INT and gains == NULL there are only G0 + 1 posteriors and at most (G0 + 1) * ld distinct
+ * candidate values.  When (G0 + 1) * ld <= 8192 the call ranks those values once, exactly, counts the prompts per
+ * (c_i, cap_i) in one pass and selects on integer ranks: no matrix is built, 8 bytes are read per prompt per pass
+ * (three passes), and the result is exact greedy by construction.  The workspace this route needs is small and
+ * independent of ld: pass HORA_FLAG_SHARED_INT_PRIOR to hora_allocate_workspace_bytes to size for it (a workspace
+ * sized without that flag is always large enough).  info_dev->lambda is then the fp64 gain of the threshold type.
  *
  *   alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld   as for hora_gains
  *   gains            [N*ld] the matrix hora_gains wrote for the same inputs, or NULL to have it built

@@ -47,9 +47,11 @@
 #include <atomic>
 #include <type_traits>
 
+#include "hora_block.cuh"
 #include "hora_common.cuh"
 #include "hora_exact.cuh"
 #include "hora_gains_chunk.cuh"
+#include "hora_rank.cuh"
 
 namespace hora {
 
@@ -66,8 +68,6 @@ constexpr int kFineBits = 10;                // extra bits resolved inside the w
 constexpr int kFinePerBin = 1 << kFineBits;
 constexpr int kFineBins = kWinBins * kFinePerBin;
 constexpr int kSampleRows = 4096;            // rows read by the estimate pass
-constexpr int kSelThreads = 256;
-constexpr int kRowsPerBlock = 1024;          // rows per CTA in the sum / out kernels (4 per thread)
 constexpr int kTypeSlots = 4096;             // hash slots for exact tie types
 constexpr int kMaxTypes = 1024;              // distinct types the exact ranking accepts
 constexpr unsigned long long kKeyInf = 0x7FF0000000000000ull;
@@ -150,107 +150,6 @@ static Workspace carve(void *base, int64_t N, int32_t ld, bool need_gains, bool 
     if (need_gains) w.gains = reinterpret_cast<double *>(take(sizeof(double) * (size_t)N * (size_t)ld));
     w.bytes = o;
     return w;
-}
-
-// ---------------------------------------------------------------------------------------------------
-// "Last CTA" ticket: returns true in exactly one CTA, after every other CTA's global writes are visible.
-__device__ __forceinline__ bool last_block(unsigned int *ticket) {
-    __shared__ bool s_last;
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
-    __syncthreads();
-    if (s_last) __threadfence();
-    return s_last;
-}
-
-// Block-wide exclusive sum over kSelThreads values (long long), also returns the total.
-__device__ __forceinline__ long long block_exclusive_sum(long long v, long long *total, long long *s_warp) {
-    const int lane = lane_id(), warp = threadIdx.x >> 5;
-    long long inc = v;
-#pragma unroll
-    for (int d = 1; d < kWarp; d <<= 1) {
-        const long long t = __shfl_up_sync(kFull, inc, d);
-        if (lane >= d) inc += t;
-    }
-    __syncthreads();
-    if (lane == kWarp - 1) s_warp[warp] = inc;
-    __syncthreads();
-    long long base = 0, tot = 0;
-#pragma unroll
-    for (int w = 0; w < kSelThreads / kWarp; ++w) {
-        const long long x = s_warp[w];
-        if (w < warp) base += x;
-        tot += x;
-    }
-    *total = tot;
-    return base + inc - v;
-}
-
-// Run by ONE CTA.  Scanning from the top bin down, find the bin where the running count reaches `need`:
-//   count(bins above d) < need <= count(bins above d) + count(d).
-// Returns d (or -1 if need is out of range) to every thread, with the count above d in *above_out and the
-// count of d in *count_out.  `bins` is a power of two and `hist` 16-byte aligned.  Two stages, neither of
-// which walks memory serially (a dependent chain of 32 loads from L2 cost 16 us here): every thread sums a
-// contiguous run of `per` bins, fetched by independent 16-byte loads that are all issued before the first
-// is used, and a block scan picks the run that holds the crossing; then the first warp loads that run's
-// bins one per lane (`per` <= 32) and a warp scan pins the bin.
-__device__ int locate_rank(const unsigned long long *hist, int bins, long long need, long long *above_out,
-                           long long *count_out, long long *s_warp) {
-    __shared__ long long s_found[3];                        // top bin of the run, count above the run, found flag
-    const int per = (bins + kSelThreads - 1) / kSelThreads; // 1, or an even number <= 32 for bins <= 8192
-    const int top = bins - 1 - (int)threadIdx.x * per;      // this thread's run: bins top, top-1, ..., top-per+1
-    long long local = 0;
-    if (per == 1) {
-        if (top >= 0) local = (long long)__ldcg(hist + top);
-    } else {                                                // bins == kSelThreads * per: every run is complete
-        const ulonglong2 *run = reinterpret_cast<const ulonglong2 *>(hist + (top - per + 1));
-        const int nvec = per >> 1;
-        ulonglong2 v[16];
-#pragma unroll
-        for (int u = 0; u < 16; ++u) v[u] = u < nvec ? __ldcg(run + u) : make_ulonglong2(0ull, 0ull);
-#pragma unroll
-        for (int u = 0; u < 16; ++u) local += (long long)(v[u].x + v[u].y);
-    }
-    if (threadIdx.x == 0) s_found[2] = 0;
-    long long total;
-    const long long above = block_exclusive_sum(local, &total, s_warp);
-    if (need >= 1 && above < need && need <= above + local) {
-        s_found[0] = top;
-        s_found[1] = above;
-        s_found[2] = 1;
-    }
-    __syncthreads();
-    int digit = -1;
-    const bool found = s_found[2] != 0;
-    const int run_top = (int)s_found[0];
-    const long long run_above = s_found[1];
-    __syncthreads();                                        // everyone has read the run before it is overwritten
-    if (found) {
-        if (threadIdx.x < kWarp) {
-            const int lane = threadIdx.x;
-            const int bin = run_top - lane;
-            const long long cnt = (lane < per && bin >= 0) ? (long long)__ldcg(hist + bin) : 0;
-            long long inc = cnt;
-#pragma unroll
-            for (int d = 1; d < kWarp; d <<= 1) {
-                const long long t = __shfl_up_sync(kFull, inc, d);
-                if (lane >= d) inc += t;
-            }
-            const bool here = run_above + inc - cnt < need && need <= run_above + inc;
-            if (here) {
-                s_found[0] = bin;
-                s_found[1] = run_above + inc - cnt;
-                s_found[2] = cnt;
-            }
-        }
-        __syncthreads();
-        digit = (int)s_found[0];
-        *above_out = s_found[1];
-        *count_out = s_found[2];
-    }
-    __syncthreads();
-    return digit;
 }
 
 // Run by ONE CTA: select the next digit of the threshold from hist[0..bins), bins a power of two; the digit
@@ -782,13 +681,6 @@ gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ 
                   s_warp);
 }
 
-// U_i(Delta) from the row's own entry: the product in U_i(Delta) = 1 - prod_{j<Delta} (b+j)/(a+b+j) is
-// g_i(Delta) (b + Delta - 1) / a  (Eq. marginal), so one load replaces Delta multiplications.  Every operation
-// is pinned to one rounding so that the value does not depend on which kernel evaluates it.
-__device__ __forceinline__ double utility_from_gain(double g, double a, double b, int32_t Delta) {
-    return __dsub_rn(1.0, __ddiv_rn(__dmul_rn(g, __dadd_rn(b, (double)(Delta - 1))), a));
-}
-
 // ---------------------------------------------------------------------------------------------------
 // Level 1: a thread per row.  r bits of the threshold are known (23 after a window hit, else 13); call P that
 // prefix.  The row is non-increasing, so with p_hi = #keys above P and p_lo = #keys above or equal, the keys
@@ -995,65 +887,6 @@ __device__ __forceinline__ int2 close_segment(const unsigned long long *__restri
         else break;
     }
     return make_int2(st.x + n_gt, st.x + n_gt + n_eq);
-}
-
-// Digit search over a histogram in SHARED memory, run by one CTA: the bin where the count from the top
-// reaches `need`.  s_pick receives (digit, count above it, count of it); digit -1 if need is out of range.
-__device__ __forceinline__ void locate_rank_shared(const unsigned int *s_hist, int bins, long long need, long long *s_warp,
-                                                   long long *s_pick) {
-    const int per = (bins + kSelThreads - 1) / kSelThreads;      // thread t owns bins top, top-1, ..., top-per+1
-    const int top = bins - 1 - (int)threadIdx.x * per;
-    long long local = 0;
-    for (int j = 0; j < per; ++j)
-        if (top - j >= 0) local += s_hist[top - j];
-    if (threadIdx.x == 0) s_pick[0] = -1;
-    long long total;
-    const long long above = block_exclusive_sum(local, &total, s_warp);
-    if (need >= 1 && above < need && need <= above + local) {    // at most one thread: the crossing is in its run
-        long long run = above;
-        for (int j = 0; j < per; ++j) {
-            const long long cnt = s_hist[top - j];
-            if (need <= run + cnt) {
-                s_pick[0] = top - j;
-                s_pick[1] = run;
-                s_pick[2] = cnt;
-                break;
-            }
-            run += cnt;
-        }
-    }
-    __syncthreads();
-}
-
-// Exclusive scan of the block sums (plus, in list mode, the corrections held in shared memory for blocks
-// [b0, b0 + n_here)), kSelThreads * 4 entries per step, in index order; run by one CTA.
-__device__ void scan_block_sums(long long *bsum_hi, long long *bsum_t, int64_t b0, int64_t n_here,
-                                const unsigned int *s_fix_hi, const unsigned int *s_fix_t, long long &run_hi,
-                                long long &run_t, long long *s_warp) {
-    constexpr int kRun = 4;                                      // consecutive block sums per thread
-    for (int64_t c0 = 0; c0 < n_here; c0 += kRun * kSelThreads) {
-        const int64_t c = c0 + (int64_t)threadIdx.x * kRun;
-        long long vh[kRun], vt[kRun], sh = 0, st = 0;
-#pragma unroll
-        for (int u = 0; u < kRun; ++u) {
-            const bool in = c + u < n_here;
-            vh[u] = in ? __ldcg(bsum_hi + b0 + c + u) + (s_fix_hi ? (long long)s_fix_hi[c + u] : 0) : 0;
-            vt[u] = in ? __ldcg(bsum_t + b0 + c + u) + (s_fix_t ? (long long)s_fix_t[c + u] : 0) : 0;
-        }
-#pragma unroll
-        for (int u = 0; u < kRun; ++u) { sh += vh[u]; st += vt[u]; }
-        long long th, tt;
-        long long eh = run_hi + block_exclusive_sum(sh, &th, s_warp);
-        long long et = run_t + block_exclusive_sum(st, &tt, s_warp);
-#pragma unroll
-        for (int u = 0; u < kRun; ++u) {
-            if (c + u < n_here) { bsum_hi[b0 + c + u] = eh; bsum_t[b0 + c + u] = et; }
-            eh += vh[u];
-            et += vt[u];
-        }
-        run_hi += th;
-        run_t += tt;
-    }
 }
 
 // List route, run by ONE CTA: the first digit comes from the histogram level 1 accumulated in global memory;
@@ -1765,6 +1598,10 @@ extern "C" void hora_allocate_profile_stages(void *const *events_host, int32_t n
 
 extern "C" size_t hora_allocate_workspace_bytes(int64_t N, int32_t ld, int32_t gains_is_null, uint32_t flags) {
     if (N < 0 || ld < 1) return 0;
+    // the caller promises a shared integer prior, exact ties and no matrix: the rank-based route, which needs
+    // neither the matrix nor anything per candidate
+    if ((flags & HORA_FLAG_SHARED_INT_PRIOR) && (flags & HORA_FLAG_EXACT_INT) && gains_is_null != 0)
+        return hora::rank_allocate_workspace_bound(N);
     return hora::carve(nullptr, N, ld, gains_is_null != 0, (flags & HORA_FLAG_EXACT_INT) != 0).bytes;
 }
 
@@ -1780,7 +1617,8 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     if (alpha == nullptr && !(alpha0 > 0.0 && beta0 > 0.0 && alpha0 < 1.0e300 && beta0 < 1.0e300))
         return HORA_ERR_INVALID_ARG;
     if (cap == nullptr && (cap_scalar < 0 || cap_scalar > ld)) return HORA_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE)) return HORA_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE | HORA_FLAG_SHARED_INT_PRIOR))
+        return HORA_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (N == 0) {
         write_empty<<<1, 1, 0, s>>>(B, group_offsets, info_dev);
@@ -1791,6 +1629,11 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     if (gains != nullptr && (reinterpret_cast<uintptr_t>(gains) & 7u)) return HORA_ERR_INVALID_ARG;
     const bool exact = (flags & HORA_FLAG_EXACT_INT) != 0;
     if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HORA_ERR_WORKSPACE;
+    // One integer prior for all prompts, exact ties, no matrix given: at most (G0 + 1) * ld distinct candidate
+    // values, ranked once; the selection runs on ranks and on counts of (c_i, cap_i) and builds no matrix.
+    if (exact && alpha == nullptr && gains == nullptr && rank_route_applies(alpha0, beta0, G0, ld))
+        return launch_rank_allocate(alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, flags, delta, G, group_offsets,
+                                    info_dev, workspace, workspace_bytes, s, mark_stage);
     const Workspace w = carve(workspace, N, ld, gains == nullptr, exact);
     if (workspace_bytes < w.bytes) return HORA_ERR_WORKSPACE;
     const int64_t NB = (N + kRowsPerBlock - 1) / kRowsPerBlock;

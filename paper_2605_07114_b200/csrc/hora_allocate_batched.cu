@@ -14,13 +14,15 @@
 // Group offsets over all prompts are an exclusive scan of G by two small kernels afterwards.
 #include <algorithm>
 
+#include "hora_block.cuh"
 #include "hora_common.cuh"
 #include "hora_exact.cuh"
 #include "hora_gains_chunk.cuh"
+#include "hora_rank.cuh"
 
 namespace hora {
 
-constexpr int kBThreads = 256;
+constexpr int kBThreads = kSelThreads;        // the shared block helpers are written for this many threads
 constexpr int kBWarps = kBThreads / kWarp;
 constexpr int kBMaxRows = 256;                 // prompts per segment (one thread per prompt in the row phases)
 constexpr int kBBins = 2048;                   // 11-bit digits
@@ -60,28 +62,6 @@ __device__ __forceinline__ BatchedRows carve_rows(unsigned char *base, int rows_
     return r;
 }
 
-__device__ __forceinline__ long long bblock_exclusive_sum(long long v, long long *total, long long *s_warp) {
-    const int lane = lane_id(), warp = threadIdx.x >> 5;
-    long long inc = v;
-#pragma unroll
-    for (int d = 1; d < kWarp; d <<= 1) {
-        const long long t = __shfl_up_sync(kFull, inc, d);
-        if (lane >= d) inc += t;
-    }
-    __syncthreads();
-    if (lane == kWarp - 1) s_warp[warp] = inc;
-    __syncthreads();
-    long long base = 0, tot = 0;
-#pragma unroll
-    for (int w = 0; w < kBWarps; ++w) {
-        const long long x = s_warp[w];
-        if (w < warp) base += x;
-        tot += x;
-    }
-    *total = tot;
-    return base + inc - v;
-}
-
 // Scanning from the top bin down, the bin where the running count reaches `need` (1-based); the count of
 // the bins above it goes to *above_out.  All threads get the result.  -1 if need is out of range.
 __device__ int blocate_rank(BatchedSmemFixed &sm, int bins, long long need, long long *above_out) {
@@ -92,7 +72,7 @@ __device__ int blocate_rank(BatchedSmemFixed &sm, int bins, long long need, long
         if (top - j >= 0) local += sm.hist[top - j];
     if (threadIdx.x == 0) sm.found[2] = 0;
     long long total;
-    const long long above = bblock_exclusive_sum(local, &total, sm.warp_tmp);
+    const long long above = block_exclusive_sum(local, &total, sm.warp_tmp);
     if (need >= 1 && above < need && need <= above + local) {
         long long run = above;
         for (int j = 0; j < per && top - j >= 0; ++j) {
@@ -148,7 +128,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         }
         __syncthreads();
         long long sum_cap;
-        bblock_exclusive_sum(threadIdx.x < n ? rw.cap[threadIdx.x] : 0, &sum_cap, sm.warp_tmp);
+        block_exclusive_sum(threadIdx.x < n ? rw.cap[threadIdx.x] : 0, &sum_cap, sm.warp_tmp);
         if (threadIdx.x == 0 && sm.status == HORA_OK && B > sum_cap) sm.status = HORA_ERR_INFEASIBLE;
         __syncthreads();
         // ---- 2: the B-th largest key ----
@@ -228,8 +208,8 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         double lambda = B > 0 ? __longlong_as_double((long long)lam_key) : 0.0;
         if (!exact) {
             long long tot_hi, tot_t;
-            bblock_exclusive_sum(my_hi, &tot_hi, sm.warp_tmp);
-            const long long pre_t = bblock_exclusive_sum(my_tied, &tot_t, sm.warp_tmp);
+            block_exclusive_sum(my_hi, &tot_hi, sm.warp_tmp);
+            const long long pre_t = block_exclusive_sum(my_tied, &tot_t, sm.warp_tmp);
             const long long R = B - tot_hi;
             long long take = R - pre_t;
             take = take < 0 ? 0 : (take > my_tied ? my_tied : take);
@@ -263,7 +243,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
             }
             if ((int)threadIdx.x < rows_cap) rw.band[threadIdx.x] = (threadIdx.x < n && has && !err) ? 1 : 0;
             long long tot_q;
-            bblock_exclusive_sum(q, &tot_q, sm.warp_tmp);          // has a barrier: num/den/band are visible after it
+            block_exclusive_sum(q, &tot_q, sm.warp_tmp);          // has a barrier: num/den/band are visible after it
             const long long Rp = B - tot_q;                        // rollouts to hand out inside the band
             int better = 0, equal = 0;
             if (threadIdx.x < n && rw.band[threadIdx.x] && sm.status == HORA_OK) {
@@ -346,7 +326,7 @@ scan_block_sums(const int32_t *__restrict__ G, int64_t N, long long *bsum, int64
         if (row < N) v += G[row];
     }
     long long tot;
-    bblock_exclusive_sum(v, &tot, s_warp);
+    block_exclusive_sum(v, &tot, s_warp);
     if (threadIdx.x == 0) bsum[blockIdx.x] = tot;
     __threadfence();
     __syncthreads();
@@ -359,7 +339,7 @@ scan_block_sums(const int32_t *__restrict__ G, int64_t N, long long *bsum, int64
         const int64_t b = b0 + threadIdx.x;
         const long long x = b < NB ? __ldcg(bsum + b) : 0;
         long long t;
-        const long long e = bblock_exclusive_sum(x, &t, s_warp);
+        const long long e = block_exclusive_sum(x, &t, s_warp);
         if (b < NB) bsum[b] = run + e;
         run += t;
     }
@@ -379,7 +359,7 @@ scan_write_offsets(const int32_t *__restrict__ G, int64_t N, const long long *__
         v += g[q];
     }
     long long tot;
-    long long pre = bblock_exclusive_sum(v, &tot, s_warp) + bpre[blockIdx.x];
+    long long pre = block_exclusive_sum(v, &tot, s_warp) + bpre[blockIdx.x];
 #pragma unroll
     for (int q = 0; q < kPer; ++q) {
         if (row0 + q < N) offsets[row0 + q] = pre;
@@ -388,10 +368,15 @@ scan_write_offsets(const int32_t *__restrict__ G, int64_t N, const long long *__
     }
 }
 
+// room for the rank tables of the shared-integer-prior route (its size does not depend on N or S)
+constexpr size_t kBRankReserve = ((size_t)5 << 19) + 4096;     // 2.5 MiB: 2 MiB of positions + the per-type tables
+
 struct BatchedWorkspace {
     int64_t *seg_off, *budgets;
     long long *bsum;
     ScanHeader *hdr;
+    int32_t *table_status;
+    void *tables;
     size_t bytes;
 };
 
@@ -405,6 +390,8 @@ static BatchedWorkspace carve_batched(void *base, int64_t N, int64_t S) {
     w.seg_off = reinterpret_cast<int64_t *>(take(sizeof(int64_t) * (size_t)(S + 1)));
     w.budgets = reinterpret_cast<int64_t *>(take(sizeof(int64_t) * (size_t)(S > 0 ? S : 1)));
     w.bsum = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)(NB > 0 ? NB : 1)));
+    w.table_status = reinterpret_cast<int32_t *>(take(sizeof(int32_t)));
+    w.tables = take(kBRankReserve);
     w.bytes = o;
     return w;
 }
@@ -428,7 +415,8 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
     if (alpha == nullptr && !(alpha0 > 0.0 && beta0 > 0.0 && alpha0 < 1.0e300 && beta0 < 1.0e300))
         return HORA_ERR_INVALID_ARG;
     if (cap == nullptr && (cap_scalar < 0 || cap_scalar > ld)) return HORA_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE)) return HORA_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE | HORA_FLAG_SHARED_INT_PRIOR))
+        return HORA_ERR_INVALID_ARG;
     if (seg_offsets_host == nullptr || (S > 0 && budgets_host == nullptr)) return HORA_ERR_INVALID_ARG;
     if (seg_offsets_host[0] != 0 || seg_offsets_host[S] != N) return HORA_ERR_INVALID_ARG;
     int64_t max_rows = 0;
@@ -440,7 +428,11 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
     const int32_t rows_cap = (int32_t)((max_rows + 3) & ~(int64_t)3);
     const size_t smem = sizeof(BatchedSmemFixed) + (size_t)rows_cap * kBRowBytes +
                         (size_t)max_rows * (size_t)ld * sizeof(unsigned long long);
-    if (max_rows > kBMaxRows || smem > kBMaxSmem) return HORA_ERR_WORKSPACE;   // segment too large for one CTA
+    // One integer prior for all prompts and exact ties: the candidate values are ranked once for all segments
+    // and every segment is solved on integer ranks by one warp (no shared-memory keys, no segment size limit).
+    const bool by_rank = (flags & HORA_FLAG_EXACT_INT) && alpha == nullptr && rank_route_applies(alpha0, beta0, G0, ld) &&
+                         rank_pos_applies(G0, ld) && rank_tables_bytes(G0, ld, true) <= kBRankReserve;
+    if (!by_rank && (max_rows > kBMaxRows || smem > kBMaxSmem)) return HORA_ERR_WORKSPACE;   // segment too large for one CTA
     if (N > 0 && (c == nullptr || delta == nullptr || G == nullptr)) return HORA_ERR_INVALID_ARG;
     if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HORA_ERR_WORKSPACE;
     const BatchedWorkspace w = carve_batched(workspace, N, S);
@@ -454,7 +446,16 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
                      cudaSuccess)
         return HORA_ERR_CUDA;
     int launches = 0;
-    if (S > 0 && N > 0) {
+    if (S > 0 && N > 0 && by_rank) {
+        if (cudaMemsetAsync(w.table_status, 0, sizeof(int32_t), st) != cudaSuccess) return HORA_ERR_CUDA;
+        const RankTables t = rank_tables_carve(w.tables, G0, ld, true);
+        const int tl = launch_rank_tables(alpha0, beta0, G0, ld, t, w.table_status, st);
+        if (tl < 0) return HORA_ERR_CUDA;
+        if (launch_rank_batched(c, G0, cap, cap_scalar, ld, w.seg_off, w.budgets, S, flags, t, w.table_status, delta, G,
+                                info_dev, st) != HORA_OK)
+            return HORA_ERR_CUDA;
+        launches += tl + 1;
+    } else if (S > 0 && N > 0) {
         // 227 KiB of shared memory per SM, 1 KiB of it reserved per resident CTA
         const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (227 * 1024) / (smem + 1024)));
         const int grid = clamp_grid(S, per_sm);

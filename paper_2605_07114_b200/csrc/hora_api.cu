@@ -6,6 +6,18 @@
 namespace hora {
 static std::atomic<unsigned long long> g_launches{0};
 void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+int sm_count() {
+    constexpr int kMaxDev = 64, kFallback = 148;           // B200, should the query fail
+    static std::atomic<int> cached[kMaxDev];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return kFallback;
+    int n = cached[dev].load(std::memory_order_acquire);
+    if (n > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return kFallback;
+    cached[dev].store(n, std::memory_order_release);
+    return n;
+}
 }  // namespace hora
 
 extern "C" const char *hora_status_string(hora_status_t status) {

@@ -18,7 +18,7 @@ constexpr int64_t kFrontChunk = 1 << 16;                // tokens per CTA when t
 // write rate is 6.3 TB/s against 5.5 TB/s for one long chunk per CTA slot (the same bytes spread over 1184
 // distant streams).  Short token axes fall back to one chunk per CTA slot.
 inline int64_t token_chunk(int64_t T) {
-    const int64_t max_ctas = (int64_t)kSmCount * 8;
+    const int64_t max_ctas = (int64_t)sm_count() * 8;
     int64_t chunk = (T + max_ctas - 1) / max_ctas;
     if (chunk > kFrontChunk) chunk = kFrontChunk;
     chunk = (chunk + kStepTokens - 1) / kStepTokens * kStepTokens;

@@ -10,7 +10,6 @@ namespace hora {
 
 constexpr int kWarp = 32;
 constexpr unsigned kFull = 0xFFFFFFFFu;
-constexpr int kSmCount = 148;              // B200: grids are sized in multiples of this
 
 // First data-dependent error wins; later kernels of the same call see it and stand down.
 __device__ __forceinline__ void raise_status(int32_t *status, int32_t code) {
@@ -47,8 +46,12 @@ __device__ __forceinline__ Posterior load_posterior(const double *alpha, const d
 
 inline hora_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? HORA_OK : HORA_ERR_CUDA; }
 
+// Multiprocessors of the current device (148 on B200), looked up once per device; persistent grids are sized
+// in multiples of it.
+int sm_count();
+
 inline int clamp_grid(int64_t want, int per_sm) {
-    const int64_t cap = (int64_t)kSmCount * per_sm;
+    const int64_t cap = (int64_t)sm_count() * per_sm;
     if (want < 1) want = 1;
     return (int)(want < cap ? want : cap);
 }

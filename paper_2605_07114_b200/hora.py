@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(HERE, "libhora.so")
  ERR_INTERNAL) = range(9)
 FLAG_EXACT_INT = 1
 FLAG_SKIP_OBJECTIVE = 2
+FLAG_SHARED_INT_PRIOR = 4
 ADV_GRPO, ADV_RLOO = 0, 1
 WEIGHT_PER_TOKEN, WEIGHT_CONST_LENGTH = 0, 1
 
@@ -318,9 +319,10 @@ class Allocator:
     """Owns the device buffers of one allocation problem shape (N, ld) and runs gains -> allocate."""
 
     def __init__(self, N: int, ld: int, G0: int, *, exact_int: bool = False, skip_objective: bool = False,
-                 materialise: bool = True, device="cuda"):
+                 materialise: bool = True, shared_int_prior: bool = False, device="cuda"):
         self.N, self.ld, self.G0 = N, ld, G0
-        self.flags = (FLAG_EXACT_INT if exact_int else 0) | (FLAG_SKIP_OBJECTIVE if skip_objective else 0)
+        self.flags = (FLAG_EXACT_INT if exact_int else 0) | (FLAG_SKIP_OBJECTIVE if skip_objective else 0) | \
+                     (FLAG_SHARED_INT_PRIOR if shared_int_prior else 0)
         self.materialise = materialise
         dev = torch.device(device)
         self.gains = torch.empty((N, ld), dtype=torch.float64, device=dev) if materialise else None

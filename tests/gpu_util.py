@@ -30,10 +30,11 @@ def gpu_gains(alpha, beta, alpha0, beta0, c, G0, cap, ld, cap_scalar=None):
 
 
 def gpu_allocate(alpha, beta, alpha0, beta0, c, G0, cap, ld, B, *, exact, materialise=True, cap_scalar=None,
-                 skip_objective=False):
-    """Returns (delta, G, offsets, info)."""
+                 skip_objective=False, shared_int_prior=False):
+    """Returns (delta, G, offsets, info).  shared_int_prior sizes the workspace for the rank-based route only."""
     N = len(c)
-    al = hora.Allocator(N, ld, G0, exact_int=exact, materialise=materialise, skip_objective=skip_objective)
+    al = hora.Allocator(N, ld, G0, exact_int=exact, materialise=materialise, skip_objective=skip_objective,
+                        shared_int_prior=shared_int_prior)
     al.delta.fill_(-1)
     al.G.fill_(-1)
     al.group_offsets.fill_(-1)

@@ -45,7 +45,7 @@ def oracle_segments(alpha, beta, a0, b0, c, G0, cap, seg, budgets, exact):
     return d, lam, obj
 
 
-def random_problem(rng, S, G0, ld, real, max_rows=40):
+def random_problem(rng, S, G0, ld, real, max_rows=40, int_priors=False):
     sizes = rng.integers(1, max_rows + 1, S)
     sizes[rng.integers(0, S)] = 1
     seg = np.zeros(S + 1, np.int64)
@@ -57,6 +57,9 @@ def random_problem(rng, S, G0, ld, real, max_rows=40):
     if real:
         alpha = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
         beta = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
+    elif int_priors:
+        alpha = rng.integers(1, 4, N).astype(np.float64)
+        beta = rng.integers(1, 4, N).astype(np.float64)
     budgets = np.zeros(S, np.int64)
     for s in range(S):
         tot = int(cap[seg[s]:seg[s + 1]].sum())
@@ -65,10 +68,13 @@ def random_problem(rng, S, G0, ld, real, max_rows=40):
 
 
 @pytest.mark.parametrize("G0,ld", [(2, 24), (4, 60), (8, 130), (8, 256)])
-@pytest.mark.parametrize("real", [False, True])
-def test_batched_matches_oracle_per_segment(G0, ld, real):
+@pytest.mark.parametrize("prior", ["shared", "integer", "real"])
+def test_batched_matches_oracle_per_segment(G0, ld, prior):
+    """shared: one Beta(1,1) prior, exact ties (solved on exact ranks, a warp per segment); integer: per-prompt
+    integer priors, exact ties (a CTA per segment, keys in shared memory); real: per-prompt real priors."""
+    real = prior == "real"
     rng = np.random.default_rng(G0 * 1000 + ld + real)
-    alpha, beta, c, cap, seg, budgets = random_problem(rng, 300, G0, ld, real)
+    alpha, beta, c, cap, seg, budgets = random_problem(rng, 300, G0, ld, real, int_priors=prior == "integer")
     d, G, off, infos = run_batched(alpha, beta, 1.0, 1.0, c, G0, cap, ld, seg, budgets, exact=not real)
     d_o, lam_o, obj_o = oracle_segments(alpha, beta, 1.0, 1.0, c, G0, cap, seg, budgets, exact=not real)
     np.testing.assert_array_equal(d, d_o)
@@ -132,9 +138,55 @@ def test_segments_beyond_the_per_cta_limits_are_refused():
     N, ld = 600, 64
     c = np.zeros(N, np.int32)
     cap = np.full(N, ld, np.int32)
-    with pytest.raises(hora.HoraError) as e:
-        run_batched(None, None, 1.0, 1.0, c, 4, cap, ld, np.array([0, 300, 600]), np.array([10, 10]), exact=True)
+    with pytest.raises(hora.HoraError) as e:            # fp64 ties: a CTA per segment, 256 prompts at most
+        run_batched(None, None, 1.0, 1.0, c, 4, cap, ld, np.array([0, 300, 600]), np.array([10, 10]), exact=False)
     assert e.value.code == hora.ERR_WORKSPACE
     with pytest.raises(hora.HoraError) as e:
         run_batched(None, None, 1.0, 1.0, c, 4, cap, ld, np.array([0, 300, 500]), np.array([10, 10]), exact=True)
     assert e.value.code == hora.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("a0,b0", [(1.0, 1.0), (2.0, 3.0)])
+def test_shared_integer_prior_has_no_segment_size_limit(a0, b0):
+    """One integer prior and exact ties: segments are solved on ranks by one warp each, whatever their size
+    (1, 31, 32, 33, 300 and 2000 prompts here), empty segments included."""
+    rng = np.random.default_rng(int(a0 * 10 + b0))
+    G0, ld = 8, 96
+    sizes = np.array([1, 31, 0, 32, 33, 300, 2000, 15, 0, 64])
+    seg = np.zeros(len(sizes) + 1, np.int64)
+    np.cumsum(sizes, out=seg[1:])
+    N = int(seg[-1])
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    budgets = np.array([int(rng.integers(0, int(cap[seg[s]:seg[s + 1]].sum()) + 1)) for s in range(len(sizes))], np.int64)
+    d, G, off, infos = run_batched(None, None, a0, b0, c, G0, cap, ld, seg, budgets, exact=True)
+    d_o, lam_o, obj_o = oracle_segments(None, None, a0, b0, c, G0, cap, seg, budgets, exact=True)
+    np.testing.assert_array_equal(d, d_o)
+    np.testing.assert_array_equal(off, np.concatenate(([0], np.cumsum(G0 + d_o.astype(np.int64)))))
+    for s, inf in enumerate(infos):
+        assert inf.status == 0 and inf.sum_cap == int(cap[seg[s]:seg[s + 1]].sum())
+        if budgets[s] > 0:
+            assert abs(inf.objective - obj_o[s]) <= 1e-12 * abs(obj_o[s])
+            assert abs(inf.lambda_ - lam_o[s]) <= 1e-12 * lam_o[s]
+            assert inf.n_above + inf.n_tied_taken == budgets[s] and 1 <= inf.n_tied_taken <= inf.n_tied
+
+
+def test_shared_prior_segments_fail_one_by_one():
+    rng = np.random.default_rng(12)
+    G0, ld, S = 4, 20, 12
+    seg = np.arange(0, 15 * S + 1, 15, dtype=np.int64)
+    N = int(seg[-1])
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    budgets = np.full(S, 40, np.int64)
+    budgets[3] = int(cap[seg[3]:seg[4]].sum()) + 1       # infeasible
+    c[seg[7] + 2] = G0 + 1                               # a count outside [0, G0]
+    d, G, off, infos = run_batched(None, None, 1.0, 1.0, c, G0, cap, ld, seg, budgets, exact=True)
+    assert infos[3].status == 3 and infos[7].status == 2
+    assert not d[seg[3]:seg[4]].any() and not G[seg[7]:seg[8]].any()
+    for s in range(S):
+        if s in (3, 7):
+            continue
+        sl = slice(int(seg[s]), int(seg[s + 1]))
+        assert infos[s].status == 0
+        np.testing.assert_array_equal(d[sl], orc.greedy_exact(None, None, 1.0, 1.0, c[sl], G0, cap[sl], 40)[0])

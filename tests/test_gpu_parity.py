@@ -95,7 +95,10 @@ def run_and_compare(w, materialise=True):
     d, G, off, info = gu.gpu_allocate(w.alpha, w.beta, w.alpha0, w.beta0, w.c, w.G0, w.cap, w.ld, w.B,
                                       exact=w.exact_int, materialise=materialise)
     gu.assert_allocation_matches(w, d, G, off, info, d_o, lam_o, obj_o)
-    assert info.first_pass_bits == 23               # on these workloads the sampled window holds the threshold
+    if w.exact_int and w.alpha is None and not materialise and (w.G0 + 1) * w.ld <= 8192:
+        assert info.first_pass_bits == -1           # one integer prior, no matrix: the rank-based route ran
+    else:
+        assert info.first_pass_bits == 23           # on these workloads the sampled window holds the threshold
     return d, G, off, info
 
 
@@ -291,7 +294,7 @@ def test_allocation_when_the_sampled_window_misses(exact, materialise):
     cap = np.full(N, ld, np.int32)
     rng = np.random.default_rng(5)
     if exact:
-        alpha = beta = None
+        alpha = beta = np.ones(N)                    # per-prompt arrays: the key-based selection, not the rank route
     else:
         alpha = np.exp(rng.uniform(np.log(0.5), np.log(2.0), N))
         beta = np.exp(rng.uniform(np.log(0.5), np.log(2.0), N))
@@ -321,8 +324,9 @@ def test_heavy_ties_take_the_digit_route_at_moderate_size(exact, materialise):
     cap[::7] = 5                                     # some rows end before the threshold's column
     B = 9 * N + 4321
     d_o, _, lam, obj = orc.greedy_exact(None, None, 1.0, 1.0, c, G0, cap, B)
-    d, G, off, info = gu.gpu_allocate(None, None, 1.0, 1.0, c, G0, cap, ld, B, exact=exact, materialise=materialise)
-    assert info.status == 0
+    ones = np.ones(N)                                # per-prompt arrays: the key-based selection, not the rank route
+    d, G, off, info = gu.gpu_allocate(ones, ones, 1.0, 1.0, c, G0, cap, ld, B, exact=exact, materialise=materialise)
+    assert info.status == 0 and info.first_pass_bits in (13, 23)
     assert info.n_tied > 65536                       # what forces the digit route
     np.testing.assert_array_equal(d, d_o)
     np.testing.assert_array_equal(off, np.concatenate(([0], np.cumsum(G0 + d_o.astype(np.int64)))))
