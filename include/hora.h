@@ -197,6 +197,31 @@ hora_status_t hora_allocate_static(const double *alpha, const double *beta, doub
                                    void *stream);
 
 /*
+ * hora_allocate_hard_first — the comparison allocator of Sec. 4.2 (paragraph "Comparison with the hard-first heuristic",
+ * Table allocator-g0): after the G0 pre-rollouts the whole Phase-B budget goes to the prompts none of whose
+ * pre-rollouts was correct (c_i = 0).  The paper prints no split rule; the one taken here is the plainest even
+ * split: the budget is dealt one rollout at a time, round-robin in prompt order, to the c_i = 0 prompts that are
+ * still below their cap, so they all end within one rollout of each other (or at their caps) and the earlier
+ * prompts hold the extra ones.  What the c_i = 0 prompts cannot absorb (all at their caps, or no such prompt in
+ * the batch) is dealt the same way to the remaining prompts, which makes the rule the uniform split when no
+ * prompt has c_i = 0.  No prior enters: the rule looks at c_i and cap_i only.
+ *
+ *   c, G0, cap, cap_scalar, N, ld   as for hora_gains (ld <= 8192 here); B as for hora_allocate
+ *   delta, G, group_offsets         as for hora_allocate
+ *   info_dev                        status, n_above (rollouts dealt in full rounds), n_tied (prompts that could take
+ *                                   one more in the last, partial round), n_tied_taken (those that did), sum_G, sum_cap;
+ *                                   lambda and objective are 0, first_pass_bits is -1 (0 when B == 0)
+ *   workspace                       hora_allocate_hard_first_workspace_bytes(N, ld) bytes, 256-byte aligned
+ * Data-dependent failures (INVALID_VALUE for c_i outside [0, G0] or cap_i outside [0, ld]; INFEASIBLE for
+ * B > sum_i cap_i) set info_dev->status and leave delta, G and group_offsets zero.
+ */
+size_t hora_allocate_hard_first_workspace_bytes(int64_t N, int32_t ld);
+
+hora_status_t hora_allocate_hard_first(const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N,
+                                       int32_t ld, int64_t B, int32_t *delta, int32_t *G, int64_t *group_offsets,
+                                       hora_alloc_info *info_dev, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * hora_allocate_batched — many independent allocation problems in one call (the paper's appendix "Training
  * configurations": Phase-B allocation is run on mini-batches of the training batch, e.g. four shards of 15
  * prompts, each with its own budget, and Proposition 1 holds within each shard).

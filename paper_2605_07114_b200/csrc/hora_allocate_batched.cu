@@ -46,16 +46,13 @@ struct BatchedSmemFixed {
 // calls with short segments — the paper's 15 prompts — leave shared memory for a fourth CTA per SM).
 struct BatchedRows {
     double *a, *b;
-    UBig *num, *den;
-    int32_t *cap, *band;
+    int32_t *cap, *band;           // band: Delta of the row's near-threshold candidate (exact mode), 0 if it has none
 };
-constexpr size_t kBRowBytes = 2 * sizeof(double) + 2 * sizeof(UBig) + 2 * sizeof(int32_t);   // 152 bytes per prompt
+constexpr size_t kBRowBytes = 2 * sizeof(double) + 2 * sizeof(int32_t);   // 24 bytes per prompt
 
 __device__ __forceinline__ BatchedRows carve_rows(unsigned char *base, int rows_cap) {
     BatchedRows r;
-    r.num = reinterpret_cast<UBig *>(base);
-    r.den = r.num + rows_cap;
-    r.a = reinterpret_cast<double *>(r.den + rows_cap);
+    r.a = reinterpret_cast<double *>(base);
     r.b = r.a + rows_cap;
     r.cap = reinterpret_cast<int32_t *>(r.b + rows_cap);
     r.band = r.cap + rows_cap;
@@ -232,38 +229,39 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                 }
                 has = (q < my_cap) && (row[q] >= k_lo);
                 if (has && q + 1 < my_cap && row[q + 1] >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
-                if (has && !err) {
-                    UBig nu, de;
-                    if (!exact_gain((unsigned long long)rw.a[threadIdx.x], (unsigned long long)rw.b[threadIdx.x],
-                                    (unsigned long long)q + 1, nu, de)) err = HORA_ERR_EXACT_RANGE;
-                    rw.num[threadIdx.x] = nu;
-                    rw.den[threadIdx.x] = de;
-                }
                 if (err) atomicCAS(&sm.status, 0, err);
             }
-            if ((int)threadIdx.x < rows_cap) rw.band[threadIdx.x] = (threadIdx.x < n && has && !err) ? 1 : 0;
+            if ((int)threadIdx.x < rows_cap) rw.band[threadIdx.x] = (threadIdx.x < n && has && !err) ? q + 1 : 0;
             long long tot_q;
-            block_exclusive_sum(q, &tot_q, sm.warp_tmp);          // has a barrier: num/den/band are visible after it
+            block_exclusive_sum(q, &tot_q, sm.warp_tmp);           // has a barrier: band is visible after it
             const long long Rp = B - tot_q;                        // rollouts to hand out inside the band
             int better = 0, equal = 0;
             if (threadIdx.x < n && rw.band[threadIdx.x] && sm.status == HORA_OK) {
+                // exact rank of this row's candidate among the band candidates: equal types need no arithmetic,
+                // different ones are compared as exact fractions
+                const unsigned long long a_t = (unsigned long long)rw.a[threadIdx.x], b_t = (unsigned long long)rw.b[threadIdx.x];
+                const unsigned long long D_t = (unsigned long long)rw.band[threadIdx.x];
+                bool ovf = false;
+                int strictly = 0;
                 for (int u = 0; u < n; ++u) {
                     if (!rw.band[u] || u == (int)threadIdx.x) continue;
-                    const int sgn = cmp_products(rw.num[u], rw.den[threadIdx.x], rw.num[threadIdx.x], rw.den[u]);
+                    const unsigned long long a_u = (unsigned long long)rw.a[u], b_u = (unsigned long long)rw.b[u];
+                    const unsigned long long D_u = (unsigned long long)rw.band[u];
+                    const int sgn = (a_u == a_t && b_u == b_t && D_u == D_t)
+                                        ? 0 : exact_compare_types(a_u, b_u, D_u, a_t, b_t, D_t, &ovf);
+                    strictly += sgn > 0;
                     better += (sgn > 0) || (sgn == 0 && u < (int)threadIdx.x);
                     equal += (sgn == 0);
                 }
+                if (ovf) atomicCAS(&sm.status, 0, (int)HORA_ERR_EXACT_RANGE);
                 my_delta = q + (better < Rp ? 1 : 0);
                 if (better == Rp - 1) {                            // this row holds the B-th best candidate
-                    int strictly = 0;
-                    for (int u = 0; u < n; ++u)
-                        if (rw.band[u] && u != (int)threadIdx.x &&
-                            cmp_products(rw.num[u], rw.den[threadIdx.x], rw.num[threadIdx.x], rw.den[u]) > 0) ++strictly;
                     sm.found[0] = tot_q + strictly;
                     sm.found[1] = equal + 1;
                     sm.found[2] = Rp - strictly;
-                    lambda = ratio_double(rw.num[threadIdx.x], rw.den[threadIdx.x]);
-                    sm.lam_exact = lambda;
+                    UBig nu, de;
+                    if (exact_gain(a_t, b_t, D_t, nu, de)) sm.lam_exact = ratio_double(nu, de);
+                    else atomicCAS(&sm.status, 0, (int)HORA_ERR_EXACT_RANGE);
                 }
             } else {
                 my_delta = q;

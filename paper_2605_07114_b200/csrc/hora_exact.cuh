@@ -15,19 +15,23 @@
 namespace hora {
 
 constexpr int kLimbs = 8;
-struct UBig { unsigned long long w[kLimbs]; };              // little-endian words
+template <int L>
+struct UBigT { unsigned long long w[L]; };                  // little-endian words
+using UBig = UBigT<kLimbs>;
 
-__device__ __forceinline__ void set_small(UBig &x, unsigned long long v) {
+template <int L>
+__device__ __forceinline__ void set_small(UBigT<L> &x, unsigned long long v) {
     x.w[0] = v;
 #pragma unroll
-    for (int i = 1; i < kLimbs; ++i) x.w[i] = 0ull;
+    for (int i = 1; i < L; ++i) x.w[i] = 0ull;
 }
 
 // x *= m; returns false if the product does not fit (x is then meaningless)
-__device__ __forceinline__ bool mul_small(UBig &x, unsigned long long m) {
+template <int L>
+__device__ __forceinline__ bool mul_small(UBigT<L> &x, unsigned long long m) {
     unsigned long long carry = 0ull;
 #pragma unroll
-    for (int i = 0; i < kLimbs; ++i) {
+    for (int i = 0; i < L; ++i) {
         const unsigned long long lo = x.w[i] * m, hi = __umul64hi(x.w[i], m);
         const unsigned long long s = lo + carry;
         x.w[i] = s;
@@ -47,17 +51,18 @@ __device__ __forceinline__ void mac192(unsigned long long &c0, unsigned long lon
     c2 += c1 < t ? 1ull : 0ull;
 }
 
-// sign of x*y - u*v.  The two 1024-bit products are formed a 64-bit column at a time from the bottom (three
+// sign of x*y - u*v.  The two double-width products are formed a 64-bit column at a time from the bottom (three
 // words of running carry each), and the most significant column in which they differ decides.
-__device__ __forceinline__ int cmp_products(const UBig &x, const UBig &y, const UBig &u, const UBig &v) {
+template <int L>
+__device__ __forceinline__ int cmp_products(const UBigT<L> &x, const UBigT<L> &y, const UBigT<L> &u, const UBigT<L> &v) {
     unsigned long long l0 = 0, l1 = 0, l2 = 0, r0 = 0, r1 = 0, r2 = 0;
     int sign = 0;
 #pragma unroll
-    for (int k = 0; k < 2 * kLimbs; ++k) {
+    for (int k = 0; k < 2 * L; ++k) {
 #pragma unroll
-        for (int i = 0; i < kLimbs; ++i) {
+        for (int i = 0; i < L; ++i) {
             const int j = k - i;
-            if (j >= 0 && j < kLimbs) {
+            if (j >= 0 && j < L) {
                 mac192(l0, l1, l2, x.w[i], y.w[j]);
                 mac192(r0, r1, r2, u.w[i], v.w[j]);
             }
@@ -69,9 +74,10 @@ __device__ __forceinline__ int cmp_products(const UBig &x, const UBig &y, const 
     return sign;
 }
 
-// Exact gain of type (a, b, Delta) as num/den (not reduced).  Returns false if kLimbs words do not suffice.
-__device__ __forceinline__ bool exact_gain(unsigned long long a, unsigned long long b, unsigned long long Delta, UBig &num,
-                                           UBig &den) {
+// Exact gain of type (a, b, Delta) as num/den (not reduced).  Returns false if L words do not suffice.
+template <int L>
+__device__ __forceinline__ bool exact_gain(unsigned long long a, unsigned long long b, unsigned long long Delta,
+                                           UBigT<L> &num, UBigT<L> &den) {
     set_small(num, a);
     set_small(den, 1ull);
     bool ok = true;
@@ -83,6 +89,23 @@ __device__ __forceinline__ bool exact_gain(unsigned long long a, unsigned long l
         for (unsigned long long j = 0; j < Delta && ok; ++j) ok = mul_small(den, a + b + j);
     }
     return ok;
+}
+
+// sign of g_{a1,b1}(D1) - g_{a2,b2}(D2) on exact fractions: in 128-bit words when both fit (the usual case, a
+// fraction of the work), else in the full width; *overflow is set when that does not suffice either
+static __device__ __noinline__ int exact_compare_types(unsigned long long a1, unsigned long long b1, unsigned long long D1,
+                                                unsigned long long a2, unsigned long long b2, unsigned long long D2,
+                                                bool *overflow) {
+    {
+        UBigT<2> n1, d1, n2, d2;
+        if (exact_gain(a1, b1, D1, n1, d1) && exact_gain(a2, b2, D2, n2, d2)) return cmp_products(n1, d2, n2, d1);
+    }
+    UBig n1, d1, n2, d2;
+    if (!exact_gain(a1, b1, D1, n1, d1) || !exact_gain(a2, b2, D2, n2, d2)) {
+        *overflow = true;
+        return 0;
+    }
+    return cmp_products(n1, d2, n2, d1);
 }
 
 // nearest double of a kLimbs-word integer, up to the rounding of the partial sums (used for reporting only)

@@ -16,8 +16,9 @@
 //            candidates above the threshold and whether the next one is tied with it.  The objective comes from
 //            the same histogram (every prompt of bin (c, cap) gets the same Delta, up to the tied rollouts, each
 //            of which adds exactly lambda).
-//   sums/out two passes over (c_i, cap_i) again: block sums of (above, tied) and their scan, then Delta, G and
-//            the CSR offsets with the first R tied prompts in index order taking one more.
+//   sums/out two passes over (c_i, cap_i) again: sums of (above, tied) per 256 prompts and per CTA, then — every
+//            CTA adding up the sums before its own — Delta, G and the CSR offsets, the first R tied prompts in
+//            index order taking one more.  Neither pass has a barrier in its loop or a serial scan behind it.
 //
 // The batched form (hora_allocate_batched with the same kind of prior) ranks once for all segments and gives a
 // warp to each segment: the threshold rank is bisected with a table pos[c][r] = #{Delta : rank_c(Delta) < r}, so
@@ -76,18 +77,6 @@ RankTables rank_tables_carve(void *base, int32_t G0, int32_t ld, bool with_pos) 
 
 // ---------------------------------------------------------------------------------------------------
 // Tables.
-
-// sign of g_{a1,b1}(D1) - g_{a2,b2}(D2) on exact fractions; *overflow is set when 512 bits do not suffice
-__device__ __noinline__ int exact_compare_types(unsigned long long a1, unsigned long long b1, unsigned long long D1,
-                                                unsigned long long a2, unsigned long long b2, unsigned long long D2,
-                                                bool *overflow) {
-    UBig n1, d1, n2, d2;
-    if (!exact_gain(a1, b1, D1, n1, d1) || !exact_gain(a2, b2, D2, n2, d2)) {
-        *overflow = true;
-        return 0;
-    }
-    return cmp_products(n1, d2, n2, d1);
-}
 
 // Every CTA builds the whole table of fp64 gains in shared memory (a warp per class row: a few hundred
 // instructions), then a thread ranks one type.
@@ -198,6 +187,9 @@ int launch_rank_tables(double alpha0, double beta0, int32_t G0, int32_t ld, cons
 // ---------------------------------------------------------------------------------------------------
 // Single problem.
 
+constexpr int kRankTask = 256;          // prompts a warp handles at a time in the sum / output passes (2 x 128)
+constexpr int kRankMaxCtas = 4096;      // CTAs of those passes (each owns a contiguous run of tasks)
+
 struct RankHeader {
     int32_t status;
     unsigned int ticket[3];
@@ -212,7 +204,8 @@ struct RankWorkspace {
     RankHeader *hdr;
     unsigned long long *H;             // [C][ld+1] prompts per (c, cap)
     unsigned long long *bucket;        // [bins] instances by rank, stored top down: slot bins-1-rank
-    long long *bsum_hi, *bsum_t;       // [NB]
+    int2 *tsum;                        // [NT] (above, tied) summed over each task of kRankTask prompts
+    long long *super_hi, *super_t;     // [kRankMaxCtas] the same summed over each CTA's run of tasks
     int32_t *class_tab;                // [C] (candidates above the threshold << 1) | next one is tied
     RankTables tab;
     int32_t bins;
@@ -229,7 +222,7 @@ static int rank_bins(int32_t G0, int32_t ld) {
 static RankWorkspace rank_carve(void *base, int64_t N, int32_t G0, int32_t ld) {
     RankWorkspace w{};
     const size_t C = (size_t)G0 + 1;
-    const int64_t NB = (N + kRowsPerBlock - 1) / kRowsPerBlock;
+    const int64_t NT = (N + kRankTask - 1) / kRankTask;
     w.bins = rank_bins(G0, ld);
     size_t o = 0;
     char *p = static_cast<char *>(base);
@@ -238,8 +231,9 @@ static RankWorkspace rank_carve(void *base, int64_t N, int32_t G0, int32_t ld) {
     w.H = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * C * ((size_t)ld + 1)));
     w.bucket = reinterpret_cast<unsigned long long *>(take(sizeof(unsigned long long) * (size_t)w.bins));
     w.zero_bytes = o;                                        // everything before this is cleared per call
-    w.bsum_hi = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)(NB > 0 ? NB : 1)));
-    w.bsum_t = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)(NB > 0 ? NB : 1)));
+    w.tsum = reinterpret_cast<int2 *>(take(sizeof(int2) * (size_t)(NT > 0 ? NT : 1)));
+    w.super_hi = reinterpret_cast<long long *>(take(sizeof(long long) * kRankMaxCtas));
+    w.super_t = reinterpret_cast<long long *>(take(sizeof(long long) * kRankMaxCtas));
     w.class_tab = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * C));
     const size_t tb = rank_tables_bytes(G0, ld, false);
     char *tbase = take(tb);
@@ -253,44 +247,151 @@ size_t rank_allocate_workspace_bytes(int64_t N, int32_t G0, int32_t ld) { return
 
 // Upper bound over every (G0, ld) the route accepts: what a caller reserves who only knows N.
 size_t rank_allocate_workspace_bound(int64_t N) {
-    const size_t T = kRankMaxTypes, NB = (size_t)((N + kRowsPerBlock - 1) / kRowsPerBlock) + 1;
+    const size_t T = kRankMaxTypes, NT = (size_t)((N + kRankTask - 1) / kRankTask) + 1;
     // C (ld + 1) <= 2 T, C <= T, bins <= T; each array rounded up to 256 bytes
-    return rk_align(sizeof(RankHeader)) + rk_align(8 * 2 * T) + rk_align(8 * T) + 2 * rk_align(8 * NB) + rk_align(4 * T) +
+    return rk_align(sizeof(RankHeader)) + rk_align(8 * 2 * T) + rk_align(8 * T) + rk_align(8 * NT) +
+           2 * rk_align(8 * kRankMaxCtas) + rk_align(4 * T) +
            rk_align(4 * T) + rk_align(8 * T) + rk_align(8 * 2 * T) + rk_align(8 * T) + 4096;
 }
 
-// (c_i, cap_i) of prompt i, validated; bin = -1 for an invalid or missing prompt
-__device__ __forceinline__ int rank_bin(const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap,
-                                        int32_t cap_scalar, int32_t ld, int64_t i, int64_t N, bool *bad) {
-    if (i >= N) return -1;
-    const int32_t ci = __ldg(c + i);
-    const int32_t cp = cap ? __ldg(cap + i) : cap_scalar;
-    if (ci < 0 || ci > G0 || cp < 0 || cp > ld) { *bad = true; return -1; }
-    return ci * (ld + 1) + cp;
+// Four consecutive prompts, (c_i, cap_i) each: two 16-byte loads where the arrays allow (`vec`), else scalar loads.
+// A prompt at or beyond N reads as c = -1 (no bin, not an error).
+struct RankQuad { int32_t c[4], cap[4]; };
+
+__device__ __forceinline__ void rank_load_quad(RankQuad &q, const int32_t *__restrict__ c, const int32_t *__restrict__ cap,
+                                               int32_t cap_scalar, int64_t p, int64_t N, bool vec) {
+    if (vec && p + 4 <= N) {
+        const int4 cv = __ldg(reinterpret_cast<const int4 *>(c + p));
+        q.c[0] = cv.x; q.c[1] = cv.y; q.c[2] = cv.z; q.c[3] = cv.w;
+        if (cap) {
+            const int4 pv = __ldg(reinterpret_cast<const int4 *>(cap + p));
+            q.cap[0] = pv.x; q.cap[1] = pv.y; q.cap[2] = pv.z; q.cap[3] = pv.w;
+        } else {
+            q.cap[0] = q.cap[1] = q.cap[2] = q.cap[3] = cap_scalar;
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            q.c[k] = p + k < N ? __ldg(c + p + k) : -1;
+            q.cap[k] = (p + k < N && cap) ? __ldg(cap + p + k) : cap_scalar;
+        }
+    }
 }
 
-__global__ void __launch_bounds__(kSelThreads)
+// (candidates above the threshold, tied candidate) of a prompt from its class entry; zeros for a missing prompt
+__device__ __forceinline__ void rank_row_state(int32_t ci, int32_t cp, const int32_t *s_class, int tiers, int *hi,
+                                               int *tied) {
+    *hi = 0;
+    *tied = 0;
+    if (ci < 0) return;
+    const int e = s_class[tiers ? (ci > 0) : ci], above = e >> 1;   // tiers: two classes only, c = 0 and c > 0
+    *hi = cp < above ? cp : above;
+    *tied = (e & 1) && cp > above;
+}
+
+// Tail of the hard-first heuristic (Sec. 4.2, "Comparison with the hard-first heuristic"), run by the last CTA of
+// the counting pass over the two-class histogram H[tier][cap], tier 0 = prompts with c = 0.  The budget is dealt
+// one rollout at a time, round-robin in prompt order, to the tier-0 prompts that are below their cap; what they
+// cannot absorb is dealt the same way to the others.  Dealing round-robin fills every prompt of the active tier
+// to a common level L (or its cap) and gives the first R prompts with cap > L one more:
+//     f(L) = sum_i min(cap_i, L) <= budget of the tier < f(L + 1),   R = budget - f(L).
+// The class table then reads exactly like the rank route's (level, "has a tied candidate"), so the same sum and
+// output passes finish the job.
+__device__ void hard_first_tail(const RankWorkspace &w, int32_t ld, int64_t B, long long *s_warp) {
+    RankHeader *hdr = w.hdr;
+    const unsigned long long *H0 = w.H, *H1 = w.H + (ld + 1);
+    long long part0 = 0, part1 = 0;
+    for (int cp = threadIdx.x; cp <= ld; cp += kSelThreads) {
+        part0 += (long long)__ldcg(H0 + cp) * cp;
+        part1 += (long long)__ldcg(H1 + cp) * cp;
+    }
+    long long cap0, cap1;
+    block_exclusive_sum(part0, &cap0, s_warp);
+    block_exclusive_sum(part1, &cap1, s_warp);
+    if (threadIdx.x == 0) {
+        hdr->sum_cap = (unsigned long long)(cap0 + cap1);
+        if (B > cap0 + cap1) raise_status(&hdr->status, HORA_ERR_INFEASIBLE);
+    }
+    __syncthreads();
+    if (*(volatile int32_t *)&hdr->status != 0) return;
+    const int tier = B <= cap0 ? 0 : 1;                      // the tier the level is sought in
+    const long long Bt = tier == 0 ? B : B - cap0;
+    const unsigned long long *Ht = tier == 0 ? H0 : H1;
+    auto filled = [&](int L) -> long long {                  // f(L), every thread gets it
+        long long part = 0;
+        for (int cp = threadIdx.x; cp <= ld; cp += kSelThreads) part += (long long)__ldcg(Ht + cp) * (cp < L ? cp : L);
+        long long tot;
+        block_exclusive_sum(part, &tot, s_warp);
+        return tot;
+    };
+    int lo = 0, hi = ld;                                     // largest L with f(L) <= Bt  (f(0) = 0 <= Bt)
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (filled(mid) <= Bt) lo = mid; else hi = mid - 1;
+    }
+    const int L = lo;
+    const long long used = filled(L);
+    long long part = 0;
+    for (int cp = threadIdx.x; cp <= ld; cp += kSelThreads)
+        if (cp > L) part += (long long)__ldcg(Ht + cp);
+    long long above_level;                                   // prompts of the tier that can take one more
+    block_exclusive_sum(part, &above_level, s_warp);
+    if (threadIdx.x == 0) {
+        const int active = (L << 1) | (above_level > 0 ? 1 : 0);
+        w.class_tab[tier] = active;
+        w.class_tab[1 - tier] = tier == 0 ? 0 : (ld << 1);  // the others get nothing / tier 0 is filled to its caps
+        hdr->rstar = L;
+        hdr->R = Bt - used;
+        hdr->n_above = (unsigned long long)(B - (Bt - used));
+        hdr->n_tied = (unsigned long long)above_level;
+        hdr->lambda = 0.0;
+        hdr->objective = 0.0;
+    }
+}
+
+// HARD: the hard-first heuristic instead of the hit-utility ranks — two classes only (c = 0, c > 0), and the tail
+// finds a water level instead of a threshold rank (hard_first_tail).
+template <bool HARD>
+__global__ void __launch_bounds__(kSelThreads, 8)
 rank_count_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
-                  int64_t N, int32_t ld, int64_t B, uint32_t flags, RankWorkspace w) {
+                  int64_t N, int32_t ld, int64_t B, uint32_t flags, int vec, RankWorkspace w) {
     extern __shared__ __align__(16) unsigned char s_rank_cnt[];
     unsigned int *s_hist = reinterpret_cast<unsigned int *>(s_rank_cnt);
     __shared__ long long s_warp[kSelThreads / kWarp];
     __shared__ double s_obj[kSelThreads / kWarp];
-    const int C = G0 + 1, n_h = C * (ld + 1);
+    const int C = HARD ? 2 : G0 + 1, n_h = C * (ld + 1);
     const int lane = lane_id(), warp = threadIdx.x >> 5;
     for (int b = threadIdx.x; b < n_h; b += kSelThreads) s_hist[b] = 0;
     __syncthreads();
     bool bad = false;
-    const int64_t stride = (int64_t)gridDim.x * kSelThreads * 4;
-    for (int64_t base = (int64_t)blockIdx.x * kSelThreads * 4; base < N; base += stride) {
-        int bin[4];
+    // a handful of bins: one shared-memory update per distinct bin per warp (the lanes would otherwise serialise
+    // on a few addresses)
+    const bool few_bins = n_h <= 64;
+    auto tally = [&](const RankQuad &q, int64_t p) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) bin[u] = rank_bin(c, G0, cap, cap_scalar, ld, base + u * kSelThreads + threadIdx.x, N, &bad);
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {                       // one shared-memory update per distinct bin per warp
-            const unsigned peers = __match_any_sync(kFull, bin[u]);
-            if (bin[u] >= 0 && lane == __ffs(peers) - 1) atomicAdd(&s_hist[bin[u]], (unsigned)__popc(peers));
+        for (int k = 0; k < 4; ++k) {
+            int bin = -1;
+            if (p + k < N) {                                 // (a prompt beyond N was read as c = -1: not an error)
+                if (q.c[k] < 0 || q.c[k] > G0 || q.cap[k] < 0 || q.cap[k] > ld) bad = true;
+                else bin = (HARD ? (q.c[k] > 0) : q.c[k]) * (ld + 1) + q.cap[k];
+            }
+            if (few_bins) {                                  // (the match costs more than it saves on a wide table)
+                const unsigned peers = __match_any_sync(kFull, bin);
+                if (bin >= 0 && lane == __ffs(peers) - 1) atomicAdd(&s_hist[bin], (unsigned)__popc(peers));
+            } else if (bin >= 0) {
+                atomicAdd(&s_hist[bin], 1u);
+            }
         }
+    };
+    // two quads in flight per thread
+    const int64_t stride = (int64_t)gridDim.x * kSelThreads * 4;
+    for (int64_t base = (int64_t)blockIdx.x * kSelThreads * 4; base < N; base += 2 * stride) {   // uniform per CTA
+        const int64_t p = base + threadIdx.x * 4;
+        RankQuad q0, q1;
+        rank_load_quad(q0, c, cap, cap_scalar, p, N, vec != 0);
+        rank_load_quad(q1, c, cap, cap_scalar, p + stride, N, vec != 0);
+        tally(q0, p);
+        tally(q1, p + stride);
     }
     if (bad) raise_status(&w.hdr->status, HORA_ERR_INVALID_VALUE);
     __syncthreads();
@@ -299,6 +400,10 @@ rank_count_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__re
         if (v) atomicAdd(w.H + b, (unsigned long long)v);
     }
     if (!last_block(&w.hdr->ticket[0])) return;
+    if (HARD) {
+        hard_first_tail(w, ld, B, s_warp);
+        return;
+    }
 
     // ---- the last CTA: from the histogram to the threshold ----
     RankHeader *hdr = w.hdr;
@@ -387,107 +492,157 @@ rank_count_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__re
     }
 }
 
-// (candidates above the threshold, tied candidate) of a prompt from its class entry
-__device__ __forceinline__ void rank_row_state(int bin, int32_t ld, const int32_t *s_class, int *hi, int *tied) {
-    *hi = 0;
-    *tied = 0;
-    if (bin < 0) return;
-    const int cls = bin / (ld + 1), cp = bin - cls * (ld + 1);
-    const int e = s_class[cls], above = e >> 1;
-    *hi = cp < above ? cp : above;
-    *tied = (e & 1) && cp > above;
+// The prompts are cut into tasks of kRankTask; CTA k owns the contiguous tasks [k m, (k+1) m) and its warps take
+// them in turn.  A lane holds 4 consecutive prompts of each 128 (two 16-byte loads), so a task is two steps.
+__device__ __forceinline__ void rank_task_state(const RankQuad (&q)[2], const int32_t *s_class, int tiers,
+                                                int (&hi)[2][4], int (&tied)[2][4]) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) rank_row_state(q[h].c[k], q[h].cap[k], s_class, tiers, &hi[h][k], &tied[h][k]);
 }
 
-// Block sums of (above, tied) over blocks of kRowsPerBlock prompts; the last CTA scans them.
-__global__ void __launch_bounds__(kSelThreads)
-rank_sums_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
-                 int64_t N, int32_t ld, RankWorkspace w, int64_t NB) {
+// Sums of (above, tied) per task and per CTA.  No barrier inside the loop, no ticket at the end.
+__global__ void __launch_bounds__(kSelThreads, 4)
+rank_sums_kernel(const int32_t *__restrict__ c, int32_t n_class, int tiers, const int32_t *__restrict__ cap,
+                 int32_t cap_scalar, int64_t N, int vec, RankWorkspace w, int64_t NT, int64_t m) {
     extern __shared__ __align__(16) unsigned char s_rank_cls[];
     int32_t *s_class = reinterpret_cast<int32_t *>(s_rank_cls);
-    __shared__ long long s_warp[kSelThreads / kWarp];
-    const bool failed = *(volatile int32_t *)&w.hdr->status != 0;
-    long long hi_sum = 0, t_sum = 0;
-    if (!failed) {
-        for (int k = threadIdx.x; k <= G0; k += kSelThreads) s_class[k] = w.class_tab[k];
-        __syncthreads();
-        const int64_t row0 = (int64_t)blockIdx.x * kRowsPerBlock + (int64_t)threadIdx.x * 4;
-        bool bad = false;
+    __shared__ long long s_acc[2][kSelThreads / kWarp];
+    if (*(volatile int32_t *)&w.hdr->status != 0) return;    // the output pass writes zeros and reads none of this
+    const int lane = lane_id(), warp = threadIdx.x >> 5;
+    for (int k = threadIdx.x; k < n_class; k += kSelThreads) s_class[k] = w.class_tab[k];
+    __syncthreads();
+    const int64_t t0 = (int64_t)blockIdx.x * m, t1 = t0 + m < NT ? t0 + m : NT;
+    long long acc_hi = 0, acc_t = 0;
+    for (int64_t t = t0 + warp; t < t1; t += kSelThreads / kWarp) {
+        RankQuad q[2];
+        rank_load_quad(q[0], c, cap, cap_scalar, t * kRankTask + lane * 4, N, vec != 0);
+        rank_load_quad(q[1], c, cap, cap_scalar, t * kRankTask + 128 + lane * 4, N, vec != 0);
+        int hi[2][4], tied[2][4], hs = 0, ts = 0;
+        rank_task_state(q, s_class, tiers, hi, tied);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            int hi, tied;
-            rank_row_state(rank_bin(c, G0, cap, cap_scalar, ld, row0 + q, N, &bad), ld, s_class, &hi, &tied);
-            hi_sum += hi;
-            t_sum += tied;
-        }
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { hs += hi[h][k]; ts += tied[h][k]; }
+        hs = __reduce_add_sync(kFull, hs);                   // at most 256 * ld < 2^31
+        ts = __reduce_add_sync(kFull, ts);
+        if (lane == 0) w.tsum[t] = make_int2(hs, ts);
+        acc_hi += hs;
+        acc_t += ts;
     }
-    long long tot_hi, tot_t;
-    block_exclusive_sum(hi_sum, &tot_hi, s_warp);
-    block_exclusive_sum(t_sum, &tot_t, s_warp);
-    if (threadIdx.x == 0) { w.bsum_hi[blockIdx.x] = tot_hi; w.bsum_t[blockIdx.x] = tot_t; }
-    if (last_block(&w.hdr->ticket[1])) {
-        long long run_hi = 0, run_t = 0;
-        scan_block_sums(w.bsum_hi, w.bsum_t, 0, NB, nullptr, nullptr, run_hi, run_t, s_warp);
+    if (lane == 0) { s_acc[0][warp] = acc_hi; s_acc[1][warp] = acc_t; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long a = 0, b = 0;
+        for (int k = 0; k < kSelThreads / kWarp; ++k) { a += s_acc[0][k]; b += s_acc[1][k]; }
+        w.super_hi[blockIdx.x] = a;
+        w.super_t[blockIdx.x] = b;
     }
 }
 
-// Outputs: a thread owns four consecutive prompts (16-byte stores where the arrays allow: `vec`).
-__global__ void __launch_bounds__(kSelThreads)
-rank_out_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
-                int64_t N, int32_t ld, int64_t B, RankWorkspace w, int32_t *__restrict__ delta, int32_t *__restrict__ G,
-                int64_t *__restrict__ offsets, int vec, hora_alloc_info *info) {
+// Outputs.  CTA k adds up the sums of the CTAs before it, then each warp walks the CTA's tasks eight at a time:
+// lanes 0..7 fetch the eight task sums, a 3-step scan gives the warp the prefix of its own task and the total
+// of the eight, and the warp writes its 256 prompts (16-byte stores where the arrays allow: `vec_out`).
+__global__ void __launch_bounds__(kSelThreads, 3)
+rank_out_kernel(const int32_t *__restrict__ c, int32_t G0, int32_t n_class, int tiers, const int32_t *__restrict__ cap,
+                int32_t cap_scalar, int64_t N, int64_t B, int vec, RankWorkspace w, int64_t NT, int64_t m,
+                int32_t *__restrict__ delta,
+                int32_t *__restrict__ G, int64_t *__restrict__ offsets, int vec_out, hora_alloc_info *info) {
     extern __shared__ __align__(16) unsigned char s_rank_cls[];
     int32_t *s_class = reinterpret_cast<int32_t *>(s_rank_cls);
     __shared__ long long s_warp[kSelThreads / kWarp];
     const RankHeader *hdr = w.hdr;
     const int32_t status = *(volatile int32_t *)&hdr->status;
     const bool failed = status != 0;
-    if (!failed)
-        for (int k = threadIdx.x; k <= G0; k += kSelThreads) s_class[k] = w.class_tab[k];
+    const int lane = lane_id(), warp = threadIdx.x >> 5;
+    long long base_hi = 0, base_t = 0;
+    if (!failed) {
+        for (int k = threadIdx.x; k < n_class; k += kSelThreads) s_class[k] = w.class_tab[k];
+        long long ph = 0, pt = 0;
+        for (int k = threadIdx.x; k < (int)blockIdx.x; k += kSelThreads) { ph += w.super_hi[k]; pt += w.super_t[k]; }
+        block_exclusive_sum(ph, &base_hi, s_warp);
+        block_exclusive_sum(pt, &base_t, s_warp);
+    }
     __syncthreads();
-    const int64_t row0 = (int64_t)blockIdx.x * kRowsPerBlock + (int64_t)threadIdx.x * 4;
-    const bool whole = row0 + 4 <= N;
-    int hi[4], tied[4];
-    long long hi_sum = 0, t_sum = 0;
-    bool bad = false;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        hi[q] = tied[q] = 0;
-        if (!failed) rank_row_state(rank_bin(c, G0, cap, cap_scalar, ld, row0 + q, N, &bad), ld, s_class, &hi[q], &tied[q]);
-        hi_sum += hi[q];
-        t_sum += tied[q];
-    }
-    const long long blk_hi = failed ? 0 : w.bsum_hi[blockIdx.x], blk_t = failed ? 0 : w.bsum_t[blockIdx.x];
     const long long R = failed ? 0 : hdr->R;
-    long long th, tt;
-    long long pre_hi = blk_hi + block_exclusive_sum(hi_sum, &th, s_warp);
-    long long pre_t = blk_t + block_exclusive_sum(t_sum, &tt, s_warp);
-    int32_t d[4];
-    int64_t of[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        d[q] = hi[q] + ((tied[q] && pre_t < R) ? 1 : 0);
-        of[q] = failed ? 0 : (row0 + q) * (int64_t)G0 + pre_hi + (pre_t < R ? pre_t : R);
-        pre_hi += hi[q];
-        pre_t += tied[q];
-    }
-    if (whole && vec) {
-        *reinterpret_cast<int4 *>(delta + row0) = make_int4(d[0], d[1], d[2], d[3]);
-        *reinterpret_cast<int4 *>(G + row0) = failed ? make_int4(0, 0, 0, 0) : make_int4(G0 + d[0], G0 + d[1], G0 + d[2], G0 + d[3]);
-        if (offsets) {
-            *reinterpret_cast<longlong2 *>(offsets + row0) = make_longlong2(of[0], of[1]);
-            *reinterpret_cast<longlong2 *>(offsets + row0 + 2) = make_longlong2(of[2], of[3]);
+    const int64_t t0 = (int64_t)blockIdx.x * m, t1 = t0 + m < NT ? t0 + m : NT;
+    long long run_hi = base_hi, run_t = base_t;
+    for (int64_t tc = t0; tc < t1; tc += kSelThreads / kWarp) {
+        const int64_t t = tc + warp;
+        RankQuad q[2];
+        if (!failed && t < t1) {
+            rank_load_quad(q[0], c, cap, cap_scalar, t * kRankTask + lane * 4, N, vec != 0);
+            rank_load_quad(q[1], c, cap, cap_scalar, t * kRankTask + 128 + lane * 4, N, vec != 0);
         }
-    } else {
+        int2 v = make_int2(0, 0);
+        if (!failed && lane < kSelThreads / kWarp && tc + lane < t1) v = w.tsum[tc + lane];
+        int2 inc = v;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            if (row0 + q < N) {
-                delta[row0 + q] = d[q];
-                G[row0 + q] = failed ? 0 : G0 + d[q];
-                if (offsets) offsets[row0 + q] = of[q];
+        for (int d = 1; d < kSelThreads / kWarp; d <<= 1) {
+            const int x = __shfl_up_sync(kFull, inc.x, d), y = __shfl_up_sync(kFull, inc.y, d);
+            if (lane >= d) { inc.x += x; inc.y += y; }
+        }
+        const int before_hi = __shfl_sync(kFull, inc.x - v.x, warp), before_t = __shfl_sync(kFull, inc.y - v.y, warp);
+        const int chunk_hi = __shfl_sync(kFull, inc.x, kSelThreads / kWarp - 1), chunk_t = __shfl_sync(kFull, inc.y, kSelThreads / kWarp - 1);
+        if (t < t1) {
+            long long pre_hi = run_hi + before_hi, pre_t = run_t + before_t;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int64_t row0 = t * kRankTask + h * 128 + lane * 4;
+                int hi[4], tied[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    hi[k] = tied[k] = 0;
+                    if (!failed) rank_row_state(q[h].c[k], q[h].cap[k], s_class, tiers, &hi[k], &tied[k]);
+                }
+                const int hs = hi[0] + hi[1] + hi[2] + hi[3], ts = tied[0] + tied[1] + tied[2] + tied[3];
+                // exclusive prefix over the lanes of (above, tied), packed: tied <= 4 per lane, 128 per step;
+                // above <= 4 ld < 2^16 per lane, 2^21 per step
+                const int packed = (hs << 8) | ts;
+                int sc = packed;
+#pragma unroll
+                for (int d = 1; d < kWarp; d <<= 1) {
+                    const int x = __shfl_up_sync(kFull, sc, d);
+                    if (lane >= d) sc += x;
+                }
+                const int excl = sc - packed, total = __shfl_sync(kFull, sc, kWarp - 1);
+                long long ph = pre_hi + (excl >> 8), pt = pre_t + (excl & 0xFF);
+                int32_t d4[4];
+                int64_t of[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    d4[k] = hi[k] + ((tied[k] && pt < R) ? 1 : 0);
+                    of[k] = failed ? 0 : (row0 + k) * (int64_t)G0 + ph + (pt < R ? pt : R);
+                    ph += hi[k];
+                    pt += tied[k];
+                }
+                if (row0 + 4 <= N && vec_out) {
+                    *reinterpret_cast<int4 *>(delta + row0) = make_int4(d4[0], d4[1], d4[2], d4[3]);
+                    *reinterpret_cast<int4 *>(G + row0) =
+                        failed ? make_int4(0, 0, 0, 0) : make_int4(G0 + d4[0], G0 + d4[1], G0 + d4[2], G0 + d4[3]);
+                    if (offsets) {
+                        *reinterpret_cast<longlong2 *>(offsets + row0) = make_longlong2(of[0], of[1]);
+                        *reinterpret_cast<longlong2 *>(offsets + row0 + 2) = make_longlong2(of[2], of[3]);
+                    }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        if (row0 + k < N) {
+                            delta[row0 + k] = d4[k];
+                            G[row0 + k] = failed ? 0 : G0 + d4[k];
+                            if (offsets) offsets[row0 + k] = of[k];
+                        }
+                    }
+                }
+                pre_hi += total >> 8;
+                pre_t += total & 0xFF;
             }
         }
+        run_hi += chunk_hi;
+        run_t += chunk_t;
     }
-    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == kSelThreads - 1) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
         if (offsets) offsets[N] = failed ? 0 : N * (int64_t)G0 + B;
         if (info) {
             info->status = status;
@@ -503,39 +658,51 @@ rank_out_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__rest
     }
 }
 
+// The three passes over (c_i, cap_i) shared by the rank route and the hard-first heuristic.
+template <bool HARD>
+static hora_status_t launch_rank_passes(const RankWorkspace &w, const int32_t *c, int32_t G0, const int32_t *cap,
+                                        int32_t cap_scalar, int64_t N, int32_t ld, int64_t B, uint32_t flags,
+                                        int32_t *delta, int32_t *G, int64_t *group_offsets, hora_alloc_info *info_dev,
+                                        cudaStream_t s, void (*mark)(int, cudaStream_t)) {
+    const int C = HARD ? 2 : G0 + 1;
+    const size_t smem_h = sizeof(unsigned int) * (size_t)C * ((size_t)ld + 1);
+    if (smem_h > 48 * 1024 && cudaFuncSetAttribute(rank_count_kernel<HARD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)smem_h) != cudaSuccess)
+        return HORA_ERR_CUDA;
+    const int vec = ((reinterpret_cast<uintptr_t>(c) | reinterpret_cast<uintptr_t>(cap)) & 15u) == 0;
+    const int per_sm = (int)std::fmax(1.0, std::fmin(8.0, std::floor(200.0 * 1024.0 / (double)(smem_h + 1024))));
+    const int grid = clamp_grid((N + 8 * kSelThreads - 1) / (8 * kSelThreads), per_sm);
+    rank_count_kernel<HARD><<<grid, kSelThreads, smem_h, s>>>(c, G0, cap, cap_scalar, N, ld, B, flags, vec, w);
+    if (mark) { mark(2, s); mark(3, s); }
+    const size_t smem_c = sizeof(int32_t) * (size_t)C;
+    const int warps = kSelThreads / kWarp;
+    const int64_t NT = (N + kRankTask - 1) / kRankTask;
+    int grid_b = clamp_grid((NT + warps - 1) / warps, 3);       // what the output pass keeps resident
+    if (grid_b > kRankMaxCtas) grid_b = kRankMaxCtas;
+    const int64_t m = (NT + grid_b - 1) / grid_b;            // tasks per CTA, a contiguous run
+    rank_sums_kernel<<<grid_b, kSelThreads, smem_c, s>>>(c, C, HARD ? 1 : 0, cap, cap_scalar, N, vec, w, NT, m);
+    if (mark) { mark(4, s); mark(5, s); }
+    const int out_vec = ((reinterpret_cast<uintptr_t>(delta) | reinterpret_cast<uintptr_t>(G) |
+                          reinterpret_cast<uintptr_t>(group_offsets)) & 15u) == 0;
+    rank_out_kernel<<<grid_b, kSelThreads, smem_c, s>>>(c, G0, C, HARD ? 1 : 0, cap, cap_scalar, N, B, vec, w, NT, m, delta,
+                                                        G, group_offsets, out_vec, info_dev);
+    if (mark) mark(6, s);
+    return cuda_ok(cudaGetLastError());
+}
+
 hora_status_t launch_rank_allocate(double alpha0, double beta0, const int32_t *c, int32_t G0, const int32_t *cap,
                                    int32_t cap_scalar, int64_t N, int32_t ld, int64_t B, uint32_t flags, int32_t *delta,
                                    int32_t *G, int64_t *group_offsets, hora_alloc_info *info_dev, void *workspace,
                                    size_t workspace_bytes, cudaStream_t s, void (*mark)(int, cudaStream_t)) {
     const RankWorkspace w = rank_carve(workspace, N, G0, ld);
     if (workspace_bytes < w.bytes) return HORA_ERR_WORKSPACE;
-    const int64_t NB = (N + kRowsPerBlock - 1) / kRowsPerBlock;
-    const int C = G0 + 1;
     if (cudaMemsetAsync(w.hdr, 0, w.zero_bytes, s) != cudaSuccess) return HORA_ERR_CUDA;
     mark(0, s);
     const int tl = launch_rank_tables(alpha0, beta0, G0, ld, w.tab, &w.hdr->status, s);
     if (tl < 0) return HORA_ERR_CUDA;
     mark(1, s);
-    const size_t smem_h = sizeof(unsigned int) * (size_t)C * ((size_t)ld + 1);
-    if (smem_h > 48 * 1024 &&
-        cudaFuncSetAttribute(rank_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_h) != cudaSuccess)
-        return HORA_ERR_CUDA;
-    const int per_sm = smem_h > 32 * 1024 ? 2 : 4;
-    const int grid = clamp_grid((N + 4 * kSelThreads - 1) / (4 * kSelThreads), per_sm);
-    rank_count_kernel<<<grid, kSelThreads, smem_h, s>>>(c, G0, cap, cap_scalar, N, ld, B, flags, w);
-    mark(2, s);
-    mark(3, s);
-    const size_t smem_c = sizeof(int32_t) * (size_t)C;
-    rank_sums_kernel<<<(int)NB, kSelThreads, smem_c, s>>>(c, G0, cap, cap_scalar, N, ld, w, NB);
-    mark(4, s);
-    mark(5, s);
-    const int out_vec = ((reinterpret_cast<uintptr_t>(delta) | reinterpret_cast<uintptr_t>(G) |
-                          reinterpret_cast<uintptr_t>(group_offsets)) & 15u) == 0;
-    rank_out_kernel<<<(int)NB, kSelThreads, smem_c, s>>>(c, G0, cap, cap_scalar, N, ld, B, w, delta, G, group_offsets,
-                                                        out_vec, info_dev);
-    mark(6, s);
     count_launches(tl + 3);
-    return cuda_ok(cudaGetLastError());
+    return launch_rank_passes<false>(w, c, G0, cap, cap_scalar, N, ld, B, flags, delta, G, group_offsets, info_dev, s, mark);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -662,4 +829,46 @@ hora_status_t launch_rank_batched(const int32_t *c, int32_t G0, const int32_t *c
     return cuda_ok(cudaGetLastError());
 }
 
+// N == 0 for the hard-first call: nothing to hand out
+__global__ void hard_first_empty(int64_t B, int64_t *offsets, hora_alloc_info *info) {
+    if (offsets) offsets[0] = 0;
+    if (info) {
+        info->status = B > 0 ? HORA_ERR_INFEASIBLE : HORA_OK;
+        info->first_pass_bits = 0;
+        info->lambda = 0.0;
+        info->n_above = info->n_tied = info->n_tied_taken = 0;
+        info->objective = 0.0;
+        info->sum_G = 0;
+        info->sum_cap = 0;
+    }
+}
+
 }  // namespace hora
+
+extern "C" size_t hora_allocate_hard_first_workspace_bytes(int64_t N, int32_t ld) {
+    if (N < 0 || ld < 1 || ld > hora::kRankMaxTypes) return 0;
+    return hora::rank_carve(nullptr, N, 1, ld).bytes;       // two classes; the table area (a few KB) stays unused
+}
+
+extern "C" hora_status_t hora_allocate_hard_first(const int32_t *c, int32_t G0, const int32_t *cap, int32_t cap_scalar,
+                                                  int64_t N, int32_t ld, int64_t B, int32_t *delta, int32_t *G,
+                                                  int64_t *group_offsets, hora_alloc_info *info_dev, void *workspace,
+                                                  size_t workspace_bytes, void *stream) {
+    using namespace hora;
+    if (N < 0 || N > 0x7FFFFFFFll || ld < 1 || ld > kRankMaxTypes || G0 < 0 || B < 0) return HORA_ERR_INVALID_ARG;
+    if (cap == nullptr && (cap_scalar < 0 || cap_scalar > ld)) return HORA_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (N == 0) {
+        hard_first_empty<<<1, 1, 0, s>>>(B, group_offsets, info_dev);
+        count_launches(1);
+        return cuda_ok(cudaGetLastError());
+    }
+    if (c == nullptr || delta == nullptr || G == nullptr) return HORA_ERR_INVALID_ARG;
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HORA_ERR_WORKSPACE;
+    const RankWorkspace w = rank_carve(workspace, N, 1, ld);
+    if (workspace_bytes < w.bytes) return HORA_ERR_WORKSPACE;
+    if (cudaMemsetAsync(w.hdr, 0, w.zero_bytes, s) != cudaSuccess) return HORA_ERR_CUDA;
+    count_launches(3);
+    return launch_rank_passes<true>(w, c, G0, cap, cap_scalar, N, ld, B, HORA_FLAG_SKIP_OBJECTIVE, delta, G, group_offsets,
+                                    info_dev, s, nullptr);
+}

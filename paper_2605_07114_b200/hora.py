@@ -29,7 +29,8 @@ EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora
            "hora_allocate_static", "hora_allocate_static_capacity", "hora_allocate_profile_events", "hora_allocate_profile_stages",
            "hora_allocate_batched", "hora_allocate_batched_workspace_bytes", "hora_rollout_weights",
            "hora_learned_prior", "hora_beta_binomial_nll", "hora_pass_at_k", "hora_pass_at_k_workspace_bytes",
-           "hora_group_advantage_tokens", "hora_allocation_share")
+           "hora_group_advantage_tokens", "hora_allocation_share", "hora_allocate_hard_first",
+           "hora_allocate_hard_first_workspace_bytes")
 
 
 class HoraError(RuntimeError):
@@ -66,6 +67,10 @@ def load() -> C.CDLL:
     L.hora_allocate_static.argtypes = [p, p, f64, f64, p, i32, p, i32, i64, i32, p, i64, u32, p, p, p, p, p]
     L.hora_allocate_static.restype = C.c_int
     L.hora_allocate_static_capacity.restype = C.c_size_t
+    L.hora_allocate_hard_first_workspace_bytes.argtypes = [i64, i32]
+    L.hora_allocate_hard_first_workspace_bytes.restype = C.c_size_t
+    L.hora_allocate_hard_first.argtypes = [p, i32, p, i32, i64, i32, i64, p, p, p, p, p, C.c_size_t, p]
+    L.hora_allocate_hard_first.restype = C.c_int
     L.hora_allocate_batched_workspace_bytes.argtypes = [i64, i64]
     L.hora_allocate_batched_workspace_bytes.restype = C.c_size_t
     L.hora_allocate_batched.argtypes = [p, p, f64, f64, p, i32, p, i32, i64, i32, p, p, i64, u32, p, p, p, p, p,
@@ -157,6 +162,19 @@ def hora_allocate(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gai
                               _ptr(info_dev, torch.uint8, "info_dev"), _ptr(workspace, torch.uint8, "workspace"),
                               0 if workspace is None else workspace.numel(), _stream())
     _check(rc, "hora_allocate")
+
+
+def hora_allocate_hard_first_workspace_bytes(N, ld) -> int:
+    return int(load().hora_allocate_hard_first_workspace_bytes(N, ld))
+
+
+def hora_allocate_hard_first(c, G0, cap, cap_scalar, N, ld, B, delta, G, group_offsets, info_dev, workspace):
+    rc = load().hora_allocate_hard_first(_ptr(c, torch.int32, "c"), G0, _ptr(cap, torch.int32, "cap"), cap_scalar, N, ld, B,
+                                         _ptr(delta, torch.int32, "delta"), _ptr(G, torch.int32, "G"),
+                                         _ptr(group_offsets, torch.int64, "group_offsets"),
+                                         _ptr(info_dev, torch.uint8, "info_dev"), _ptr(workspace, torch.uint8, "workspace"),
+                                         0 if workspace is None else workspace.numel(), _stream())
+    _check(rc, "hora_allocate_hard_first")
 
 
 def hora_allocate_batched_workspace_bytes(N, S) -> int:

@@ -120,10 +120,11 @@ def test_status_codes_and_zeroed_outputs():
     cap = np.full(N, ld, np.int32)
     d, G, off, info = rank_allocate(1.0, 1.0, c, G0, cap, ld, N * ld + 1)
     assert info.status == 3 and not d.any() and not G.any() and not off.any()
-    c2 = c.copy()
-    c2[77] = G0 + 1
-    d, G, off, info = rank_allocate(1.0, 1.0, c2, G0, cap, ld, 50)
-    assert info.status == 2 and not d.any() and not G.any()
+    for bad_c in (G0 + 1, -1, -5):
+        c2 = c.copy()
+        c2[77] = bad_c
+        d, G, off, info = rank_allocate(1.0, 1.0, c2, G0, cap, ld, 50)
+        assert info.status == 2 and not d.any() and not G.any()
     cap2 = cap.copy()
     cap2[400] = ld + 1
     d, G, off, info = rank_allocate(1.0, 1.0, c, G0, cap2, ld, 50)

@@ -592,3 +592,49 @@ def test_allocation_share_statistic_pins():
     assert budget == np.bincount(c, weights=d, minlength=9).astype(np.int64).tolist()
     with pytest.raises(ValueError):
         share_orc.allocation_share([3], [1], 2)
+
+
+# ------------------------------------------------------------------ hard-first heuristic (Sec. 4.2)
+def test_hard_first_pins():
+    """The comparison allocator of Sec. 4.2 under the even-split reading: a hand example, the invariants of an even
+    split, the closed form of the water level, and the fall-through cases."""
+    from oracle import hard_first as hf
+    # hand example: prompts 0, 2, 5 have c = 0; caps 3, 9, 1, 9, 9, 9; 6 rollouts: rounds (0,2,5), (0,5), (0) -> 3, 1, 2
+    c = [0, 1, 0, 4, 2, 0]
+    cap = [3, 9, 1, 9, 9, 9]
+    assert hf.hard_first(c, cap, 6) == [3, 0, 1, 0, 0, 2]
+    assert hf.hard_first(c, cap, 7) == [3, 0, 1, 0, 0, 3]
+    # the c = 0 prompts hold 3 + 1 + 9 = 13; the 14th and 15th rollout fall through to prompts 1 and 3
+    assert hf.hard_first(c, cap, 13) == [3, 0, 1, 0, 0, 9]
+    assert hf.hard_first(c, cap, 15) == [3, 1, 1, 1, 0, 9]
+    # no c = 0 prompt at all: the uniform split, remainder to the lowest indices
+    assert hf.hard_first([1, 2, 3, 1], [9, 9, 9, 9], 10) == [3, 3, 2, 2]
+    with pytest.raises(ValueError):
+        hf.hard_first(c, cap, sum(cap) + 1)
+    rng = np.random.default_rng(42)
+    for _ in range(200):
+        N = int(rng.integers(1, 30))
+        G0 = int(rng.integers(1, 6))
+        cc = [int(x) for x in rng.integers(0, G0 + 1, N)]
+        cp = [int(x) for x in rng.integers(0, 12, N)]
+        B = int(rng.integers(0, sum(cp) + 1))
+        d = hf.hard_first(cc, cp, B)
+        assert sum(d) == B and all(0 <= x <= y for x, y in zip(d, cp))
+        hard = [i for i in range(N) if cc[i] == 0]
+        rest = [i for i in range(N) if cc[i] != 0]
+        hard_room = sum(cp[i] for i in hard)
+        if B <= hard_room:
+            assert all(d[i] == 0 for i in rest)                       # only c = 0 prompts receive budget
+            tier, Bt = hard, B
+        else:
+            assert all(d[i] == cp[i] for i in hard)                   # they are full before anyone else gets any
+            tier, Bt = rest, B - hard_room
+        # water level: the largest L with sum_i min(cap_i, L) <= Bt; everyone sits at min(cap, L) or one above,
+        # and the ones above are the lowest-index prompts with room
+        L = max(l for l in range(0, 13) if sum(min(cp[i], l) for i in tier) <= Bt)
+        R = Bt - sum(min(cp[i], L) for i in tier)
+        extra = [i for i in tier if cp[i] > L][:R]
+        assert len(extra) == R
+        for i in tier:
+            assert d[i] == min(cp[i], L) + (1 if i in extra else 0)
+
