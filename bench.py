@@ -36,6 +36,12 @@ WORKLOAD = "cfg4"
 BCAST_ROLLOUTS = 262144
 FALLBACK_HBM_GBS = 6650.0
 
+NOMINAL_HBM_GBS = 8000.0                  # datasheet figure, context beside the measured peak
+PIPELINE_TARGET_FRAC = 0.60               # the stated bar for the allocation + advantage pipeline at cfg4
+# fp64 operations per candidate gain as the method states them (recurrence after Eq. marginal:
+# M(l+1) = M(l) (b + l) / (a + b + l + 1): two additions, one multiplication, one division)
+FP64_OPS_PER_CANDIDATE = 4
+
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
 # under profiles/ (taken at N = 131072 and scaled by the row count: the traffic is proportional to it);
 # None = no usable capture (for gains_kernel the small case leaves a large share of its output in L2).
@@ -108,6 +114,20 @@ def physical_gpu_index(local_rank: int) -> int:
         except Exception:
             return local_rank
     return local_rank
+
+
+def time_events(torch, fn, reps: int, warm: int = 3) -> float:
+    """Mean milliseconds per call of fn, CUDA events on the current stream, after `warm` untimed calls."""
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
 
 
 def shard_seed(rank: int) -> int:
@@ -231,10 +251,17 @@ def run_ours(args):
     t1.record()
     hora.hora_allocate_profile_events(None, None)
     barrier()
-    clocks = sampler.stop()
     launches = hora.hora_launch_count() - launches0
     ms_total = max_over_ranks(t0.elapsed_time(t1), world, dev)
     ms_step = ms_total / args.steps
+    # a short timed region gives the clock sampler only a few samples: the same step loop goes on, untimed, until
+    # the sampler has seen about 0.3 s of this load
+    extra_steps = max(0, int(0.3 / (ms_step * 1e-3)) - args.steps)
+    for _ in range(extra_steps):
+        step()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    clocks["covers"] = f"the {args.steps} timed steps and {extra_steps} further identical steps"
     stages = np.array([[ev[i].elapsed_time(ev[i + 1]) for i in range(4)] for ev in stage_ev])
     st_mean = stages.mean(axis=0)
     st_min = stages.min(axis=0)
@@ -296,9 +323,12 @@ def run_ours(args):
         torch.cuda.empty_cache()
         alf = hora.Allocator(N, ld, G0, exact_int=False, materialise=False, device=dev)
 
-        def step_fused():
+        def fused_allocate():
             hora.hora_allocate(alpha, beta, 1.0, 1.0, c, G0, None, cap_scalar, N, ld, None, B, alf.flags, alf.delta,
                                alf.G, alf.group_offsets, alf.info, alf.workspace)
+
+        def step_fused():
+            fused_allocate()
             hora.hora_group_advantage(rewards, alf.group_offsets, N, w.adv_mode, eps, w.ddof, adv)
             hora.hora_token_broadcast(adv, tok, R, T, token_adv)
         for _ in range(3):
@@ -312,6 +342,7 @@ def run_ours(args):
         f1.record()
         torch.cuda.synchronize()
         fused_ms = f0.elapsed_time(f1) / nf
+        fused_alloc_ms = time_events(torch, fused_allocate, nf)
         if not torch.equal(alf.delta, al.delta):
             raise RuntimeError("fused and two-call allocations differ")
         del alf
@@ -470,17 +501,39 @@ def run_ours(args):
         "allocation": {"lambda": info.lambda_, "n_above": info.n_above, "n_tied": info.n_tied,
                        "objective": info.objective},
     }
+    out["pipeline"].update({"target_frac": PIPELINE_TARGET_FRAC,
+                            "frac_of_nominal_hbm": round(pipe_bytes / (pipe_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 4),
+                            "nominal_hbm_gbs": NOMINAL_HBM_GBS})
+    fp64 = None
+    if world == 1:
+        fp64 = measure_fp64_peak(torch, hora, dev)
+        out["peak_fp64_tflops"] = fp64
     if fused_ms is not None:
         out["token_advantages"] = tok_cmp
+        flops = FP64_OPS_PER_CANDIDATE * cand
+        ach = flops / (fused_alloc_ms * 1e-3) / 1e12
         out["fused_step"] = {"calls": "hora_allocate(gains=NULL)+hora_group_advantage+hora_token_broadcast",
                              "ms_per_step": round(fused_ms, 4), "prompts_per_s": N / (fused_ms * 1e-3),
+                             "hora_allocate_ms": round(fused_alloc_ms, 4),
+                             "roofline": {"bound": "alu", "kernel": "hora_allocate(gains=NULL): rows computed and counted "
+                                          "in one pass (gains_level0_fused and the passes behind it)",
+                                          "achieved": round(ach, 3), "peak": fp64["value"], "unit": "TFLOP/s",
+                                          "frac": round(ach / fp64["value"], 4), "traffic": None,
+                                          "algorithmic_flops_per_launch": int(flops),
+                                          "flops_per_candidate": FP64_OPS_PER_CANDIDATE,
+                                          "peak_kind": "measured fp64 FMA rate (hora_fp64_probe), 2 flop per FMA"},
+                             "hbm_view": {"bytes_written_once": int(cand * 8), "gbs": round(cand * 8 / (fused_alloc_ms * 1e-3) / 1e9, 1),
+                                          "frac_of_hbm_peak": round(cand * 8 / (fused_alloc_ms * 1e-3) / 1e9 / peak, 4),
+                                          "note": "the call still writes the matrix once into its workspace; against "
+                                                  "that one write it runs at this fraction of the measured copy peak"},
                              "note": "same outputs; the matrix is written once inside the workspace and not read back in "
                                      "full, so this step moves 2.15 GB less than the four-call step timed above"}
     if graph_ms is not None:
         out["graph_step"] = {"ms_per_step": round(graph_ms, 4), "prompts_per_s": N / (graph_ms * 1e-3),
                              "note": "the same four calls captured once in a CUDA graph and replayed"}
     if world == 1:
-        out["batched"] = bench_batched(torch, hora, wl, dev)
+        out["batched"] = bench_batched(torch, hora, wl, dev, peak, fp64["value"])
+        out["configs"] = bench_configs(torch, hora, wl, dev, peak)
     if ref is not None:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_sample, ref)
         out["parity"] = parity
@@ -489,9 +542,27 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def bench_batched(torch, hora, wl, dev, shards=65536, shard_prompts=15, per_prompt=24, reps=20):
+def measure_fp64_peak(torch, hora, dev, iters=4096, reps=5):
+    """fp64 rate of this GPU from the library's FMA probe: best of `reps` launches, 2 flop per FMA."""
+    sink = torch.zeros(1, dtype=torch.float64, device=dev)
+    hora.hora_fp64_probe(256, sink)
+    torch.cuda.synchronize()
+    best = 0.0
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fmas = hora.hora_fp64_probe(iters, sink)
+        e1.record()
+        torch.cuda.synchronize()
+        best = max(best, 2.0 * fmas / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+    return {"value": round(best, 2), "unit": "TFLOP/s", "how": f"hora_fp64_probe: 8 independent FMA chains per thread, "
+            f"{iters} steps, 8 CTAs of 256 threads per SM, best of {reps}; flop = 2 per FMA"}
+
+
+def bench_batched(torch, hora, wl, dev, hbm_peak, fp64_peak, shards=65536, shard_prompts=15, per_prompt=24, reps=20):
     """Secondary measurement: hora_allocate_batched on the shape the paper trains with (shards of 15 prompts,
-    G0 = 8, 24 extra rollouts per prompt, uniform prior, exact ties), many shards in one call."""
+    G0 = 8, 24 extra rollouts per prompt, exact ties), many shards in one call: with the paper's uniform prior
+    (solved on exact ranks, a warp per shard) and with per-prompt real priors (a CTA per shard, rows in shared memory)."""
     rng = np.random.default_rng(15)
     G0, ld = 8, shard_prompts * per_prompt
     N = shards * shard_prompts
@@ -505,25 +576,123 @@ def bench_batched(torch, hora, wl, dev, shards=65536, shard_prompts=15, per_prom
     info = torch.zeros(shards * hora.INFO_BYTES, dtype=torch.uint8, device=dev)
     ws = torch.empty(hora.hora_allocate_batched_workspace_bytes(N, shards), dtype=torch.uint8, device=dev)
 
-    def call():
+    def uniform():
         hora.hora_allocate_batched(None, None, 1.0, 1.0, c, G0, None, ld, N, ld, seg, budgets, hora.FLAG_EXACT_INT,
                                    delta, G, off, info, ws)
-    for _ in range(3):
-        call()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
-        call()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / reps
+    ms = time_events(torch, uniform, reps)
     if int(delta.sum().item()) != shards * ld:
         raise RuntimeError("batched allocation did not hand out the whole budget")
-    return {"call": "hora_allocate_batched", "shards": shards, "prompts_per_shard": shard_prompts, "G0": G0, "ld": ld,
-            "budget_per_shard": ld, "ms": round(ms, 4), "shards_per_s": shards / (ms * 1e-3),
-            "prompts_per_s": N / (ms * 1e-3), "candidates_per_s": N * ld / (ms * 1e-3),
-            "note": "gains are computed in shared memory and never written out: bound by fp64/integer issue, not HBM"}
+    # algorithmic traffic of the uniform-prior form: 4 B of c in, Delta, G (8 B) and an offset (8 B) out per
+    # prompt, a 16-byte segment entry in and a 64-byte summary out per shard
+    by = N * 20 + shards * 80
+    out = {"call": "hora_allocate_batched", "shards": shards, "prompts_per_shard": shard_prompts, "G0": G0, "ld": ld,
+           "budget_per_shard": ld, "prior": "uniform Beta(1,1), exact ties (rank-based route)", "ms": round(ms, 4),
+           "shards_per_s": shards / (ms * 1e-3), "prompts_per_s": N / (ms * 1e-3), "candidates_per_s": N * ld / (ms * 1e-3),
+           "roofline": {"bound": "hbm", "kernel": "whole call (rank tables, one warp per shard, offsets scan; the segment "
+                        "table is copied from host memory inside the call)", "achieved": round(by / (ms * 1e-3) / 1e9, 1),
+                        "peak": hbm_peak, "unit": "GB/s", "frac": round(by / (ms * 1e-3) / 1e9 / hbm_peak, 4), "traffic": None,
+                        "algorithmic_bytes_per_launch": int(by),
+                        "note": "a few tens of MB per call: launch latency and the host-to-device copy of the segment "
+                                "table set the time, not bandwidth"}}
+    # per-prompt real priors on a quarter of the shards (the general path)
+    s2 = shards // 4
+    n2 = s2 * shard_prompts
+    al = torch.from_numpy(np.exp(rng.uniform(np.log(0.05), np.log(20), n2))).to(dev)
+    be = torch.from_numpy(np.exp(rng.uniform(np.log(0.05), np.log(20), n2))).to(dev)
+
+    def real():
+        hora.hora_allocate_batched(al, be, 1.0, 1.0, c[:n2], G0, None, ld, n2, ld, seg[:s2 + 1], budgets[:s2], 0,
+                                   delta[:n2], G[:n2], off[:n2 + 1], info[:s2 * hora.INFO_BYTES], ws)
+    ms2 = time_events(torch, real, max(3, reps // 4))
+    flops = FP64_OPS_PER_CANDIDATE * n2 * ld
+    ach = flops / (ms2 * 1e-3) / 1e12
+    out["real_priors"] = {"shards": s2, "ms": round(ms2, 4), "shards_per_s": s2 / (ms2 * 1e-3),
+                          "prompts_per_s": n2 / (ms2 * 1e-3),
+                          "roofline": {"bound": "alu", "kernel": "allocate_batched_kernel (rows built in shared memory, "
+                                       "selection by digit sweeps)", "achieved": round(ach, 3), "peak": fp64_peak,
+                                       "unit": "TFLOP/s", "frac": round(ach / fp64_peak, 4), "traffic": None,
+                                       "algorithmic_flops_per_launch": int(flops),
+                                       "flops_per_candidate": FP64_OPS_PER_CANDIDATE}}
+    return out
+
+
+def bench_configs(torch, hora, wl, dev, peak):
+    """The other named workloads (parity cases of the test-suite), event-timed here so that their numbers come from
+    the same run: hora_gains + hora_allocate with the matrix, the rank-based route where the prior is the shared
+    integer one, the advantages over the resulting groups, and for cfg3 the broadcast to its 2.7e8 tokens."""
+    res = {}
+    for name in ("cfg1", "cfg2", "cfg3", "cfg5"):
+        w = wl.make(name)
+        N, ld, G0, B = w.N, w.ld, w.G0, w.B
+        t = lambda x: None if x is None else torch.from_numpy(x).to(dev)
+        alpha, beta, c, cap = t(w.alpha), t(w.beta), t(w.c), t(w.cap)
+        al = hora.Allocator(N, ld, G0, exact_int=w.exact_int, device=dev)
+        reps = 50 if N <= (1 << 16) else 10
+
+        def gains():
+            hora.hora_gains(alpha, beta, w.alpha0, w.beta0, c, G0, cap, 0, N, ld, al.gains)
+
+        def allocate():
+            hora.hora_allocate(alpha, beta, w.alpha0, w.beta0, c, G0, cap, 0, N, ld, al.gains, B, al.flags, al.delta, al.G,
+                               al.group_offsets, al.info, al.workspace)
+        g_ms = time_events(torch, gains, reps)
+        a_ms = time_events(torch, allocate, reps)
+        if al.read_info().status != 0:
+            raise RuntimeError(f"{name}: allocation failed")
+        cand = N * ld
+        entry = {"N": N, "ld": ld, "G0": G0, "B": B, "prior": "shared Beta(1,1), exact ties" if w.exact_int else "per-prompt real",
+                 "hora_gains_us": round(g_ms * 1e3, 1), "hora_allocate_us": round(a_ms * 1e3, 1)}
+        if w.exact_int:
+            ar = hora.Allocator(N, ld, G0, exact_int=True, materialise=False, shared_int_prior=True, device=dev)
+
+            def on_ranks():
+                hora.hora_allocate(None, None, w.alpha0, w.beta0, c, G0, cap, 0, N, ld, None, B, ar.flags, ar.delta, ar.G,
+                                   ar.group_offsets, ar.info, ar.workspace)
+            r_ms = time_events(torch, on_ranks, reps)
+            if not torch.equal(ar.delta, al.delta):
+                raise RuntimeError(f"{name}: the rank-based route and the matrix route disagree")
+            entry["hora_allocate_on_ranks_us"] = round(r_ms * 1e3, 1)
+            entry["on_ranks_bytes"] = int(N * 24 + N * 16)           # three reads of (c, cap), Delta, G, offset out
+            entry["on_ranks_gbs"] = round(entry["on_ranks_bytes"] / (r_ms * 1e-3) / 1e9, 1)
+            del ar
+        off_h = al.group_offsets.cpu().numpy()
+        rewards_h = w.rewards(off_h)
+        rewards = torch.from_numpy(rewards_h).to(dev)
+        adv = torch.empty_like(rewards)
+
+        def advantage():
+            hora.hora_group_advantage(rewards, al.group_offsets, N, w.adv_mode, float(w.eps), w.ddof, adv)
+        v_ms = time_events(torch, advantage, reps)
+        entry["hora_group_advantage_us"] = round(v_ms * 1e3, 1)
+        entry["rollouts"] = int(off_h[-1])
+        if N >= (1 << 20):                                           # large enough for bandwidth to mean something
+            bg, ba = cand * 8 + N * 20, cand * 8 + N * 36
+            bv = int(off_h[-1]) * 8 + (N + 1) * 8
+            entry["gbs"] = {"hora_gains": round(bg / (g_ms * 1e-3) / 1e9, 1), "hora_allocate": round(ba / (a_ms * 1e-3) / 1e9, 1),
+                            "hora_group_advantage": round(bv / (v_ms * 1e-3) / 1e9, 1)}
+            entry["frac_of_hbm_peak"] = {k: round(v / peak, 4) for k, v in entry["gbs"].items()}
+        else:
+            entry["note"] = "launch- and latency-bound at this size: microseconds per call, bandwidth figures would mean nothing"
+        if w.with_tokens:
+            Rn = int(off_h[-1])
+            tok_h = w.token_offsets(Rn)
+            T = int(tok_h[-1])
+            tok = torch.from_numpy(tok_h).to(dev)
+            token_adv = torch.empty(T, dtype=torch.float32, device=dev)
+
+            def broadcast():
+                hora.hora_token_broadcast(adv, tok, Rn, T, token_adv)
+            b_ms = time_events(torch, broadcast, 20)
+            bb = T * 4 + Rn * 12
+            entry["hora_token_broadcast"] = {"tokens": T, "ms": round(b_ms, 4), "tokens_per_s": T / (b_ms * 1e-3),
+                                             "gbs": round(bb / (b_ms * 1e-3) / 1e9, 1),
+                                             "frac_of_hbm_peak": round(bb / (b_ms * 1e-3) / 1e9 / peak, 4)}
+            del tok, token_adv
+        res[name] = entry
+        del al, rewards, adv
+        torch.cuda.empty_cache()
+    res["parity"] = "each of these workloads is compared with the oracle, at full size, by the test-suite (tests/test_gpu_parity.py, tests/test_gpu_fullsize.py, tests/test_gpu_rank_route.py)"
+    return res
 
 
 # ------------------------------------------------------------------------------- oracle timing
@@ -557,12 +726,57 @@ def oracle_step(w, n):
     return oracle_pass(w, n)["seconds"]
 
 
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_all_cores(ref, n_gain_rows=1 << 17):
+    """The parts of the oracle that split over prompts with no interaction — gain rows, group advantages, token
+    repeat — run as they stand on every host core (one thread per core, each on its own contiguous slice; the C
+    routines release the interpreter lock).  The heap greedy is one sequential loop and stays on one core."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import hora_oracle as orc
+    w = ref["workload"]
+    cores = host_cores()
+    n = min(n_gain_rows, ref["n"])
+
+    def split(total):
+        edges = np.linspace(0, total, cores + 1).astype(np.int64)
+        return [(int(edges[k]), int(edges[k + 1])) for k in range(cores) if edges[k + 1] > edges[k]]
+
+    def run(jobs):
+        t0 = time.perf_counter()
+        with ThreadPoolExecutor(max_workers=cores) as ex:
+            list(ex.map(lambda f: f(), jobs))
+        return time.perf_counter() - t0
+    t_gains = run([lambda a=a, b=b: orc.gains(w.alpha[a:b], w.beta[a:b], w.alpha0, w.beta0, w.c[a:b], w.G0, w.cap[a:b], w.ld)
+                   for a, b in split(n)])
+    off, rewards = ref["offsets"], ref["rewards"]
+    eps = float(np.float32(w.eps))
+    t_adv = run([lambda a=a, b=b: orc.group_advantage(rewards[off[a]:off[b]], off[a:b + 1] - off[a], w.adv_mode, eps, w.ddof)
+                 for a, b in split(ref["n"])])
+    tok, R = ref["token_offsets"], ref["R"]
+    t_bc = run([lambda a=a, b=b: orc.token_broadcast(ref["adv"][a:b], tok[a:b + 1] - tok[a]) for a, b in split(R)])
+    return {"cores": cores, "gain_rows_per_s": n / t_gains, "candidate_gains_per_s": n * w.ld / t_gains,
+            "advantage_rollouts_per_s": len(rewards) / t_adv, "broadcast_tokens_per_s": int(tok[-1]) / t_bc,
+            "seconds": {"gains": round(t_gains, 3), "advantage": round(t_adv, 3), "broadcast": round(t_bc, 3)},
+            "sample": f"gain rows of the first {n} prompts; advantages of all {len(rewards)} rollouts of the oracle pass; "
+                      f"broadcast of {R} rollouts to {int(tok[-1])} tokens",
+            "note": "the heap greedy (Algorithm 1's loop) is sequential: it is timed on one core in `value`"}
+
+
 def cpu_baseline(w, n, ref=None):
     n = min(n, w.N)
-    secs = (ref if ref is not None else oracle_pass(w, n))["seconds"]
-    return {"value": n / secs, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(secs, 2),
-            "sample": f"first {n} of {w.N} prompts of {WORKLOAD} (budget and token count scaled by the same factor), "
-                      "one pass: long-double gain rows, heap greedy, group advantages, token repeat"}
+    ref = ref if ref is not None else oracle_pass(w, n)
+    secs = ref["seconds"]
+    out = {"value": n / secs, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(secs, 2),
+           "sample": f"first {n} of {w.N} prompts of {WORKLOAD} (budget and token count scaled by the same factor), "
+                     "one pass: long-double gain rows, heap greedy, group advantages, token repeat"}
+    out["all_cores"] = oracle_all_cores(ref)
+    return out
 
 
 def check_against_oracle(torch, hora, dev, ref, band=1e-12):
@@ -620,12 +834,23 @@ def check_against_oracle(torch, hora, dev, ref, band=1e-12):
             "band_differences": in_band, "adv_max_abs_err": adv_err, "tokens_compared": T}
 
 
-def reference_sample_size(steps: int, warmup: int, N: int) -> int:
-    """Prompts per oracle step so that the whole run stays near 100 s of CPU work."""
-    budget_prompts = 5.0e6
-    n = int(budget_prompts / max(1, steps + warmup))
+REFERENCE_CPU_SECONDS = 150.0             # what the whole --impl reference run may cost
+ORACLE_US_PER_PROMPT = 15.0               # measured on this machine's hosts at cfg4 (14.9 s for 2^20 prompts)
+
+
+def reference_sample_size(steps: int, warmup: int, N: int):
+    """Prompts per oracle step: the whole workload when steps + warm-up of it fit the time allowed for this arm,
+    else the largest power of two that does.  Returns (n, reason)."""
+    per_step = REFERENCE_CPU_SECONDS / max(1, steps + warmup)
+    if N * ORACLE_US_PER_PROMPT * 1e-6 <= per_step:
+        return N, "the whole workload per step"
+    n = int(per_step / (ORACLE_US_PER_PROMPT * 1e-6))
     n = 1 << (max(n, 1).bit_length() - 1)
-    return max(1024, min(1 << 19, n, N))
+    n = max(1024, min(n, N))
+    return n, (f"one oracle pass over all {N} prompts takes about {N * ORACLE_US_PER_PROMPT * 1e-6:.0f} s on one host core; "
+               f"{steps} + {warmup} of them would take {(steps + warmup) * N * ORACLE_US_PER_PROMPT * 1e-6 / 60:.0f} min, so each "
+               f"step covers the first {n} prompts (budget and tokens scaled); run with fewer steps (steps + warmup <= "
+               f"{int(REFERENCE_CPU_SECONDS / (N * ORACLE_US_PER_PROMPT * 1e-6))}) for the whole workload per step")
 
 
 def run_reference(args):
@@ -636,7 +861,7 @@ def run_reference(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     w = wl.make(WORKLOAD, args.prompts, seed=shard_seed(0))
     steps, warm = args.steps, args.warmup
-    n = reference_sample_size(steps, warm, w.N)
+    n, why = reference_sample_size(steps, warm, w.N)
     for _ in range(warm):
         oracle_step(w, n)
     secs = [oracle_step(w, n) for _ in range(steps)]
@@ -647,7 +872,7 @@ def run_reference(args):
         "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f80", "data": "synthetic",
         "config": {"workload": f"{WORKLOAD}: each step is the first {n} of {w.N} prompts (budget and tokens scaled), "
-                               "CPU oracle, one host thread"},
+                               "CPU oracle, one host thread", "same_workload_as_repo_arm": n == w.N, "sample_reason": why},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "sample": f"first {n} prompts of {WORKLOAD} per step"},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},

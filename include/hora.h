@@ -386,6 +386,16 @@ void hora_allocate_profile_events(void *start_event, void *stop_event);
  */
 void hora_allocate_profile_stages(void *const *events_host, int32_t n);
 
+/*
+ * hora_fp64_probe — measurement aid, no counterpart in the paper.  Enqueues one kernel that does nothing but
+ * independent fp64 fused multiply-adds (8 chains per thread, 8 CTAs of 256 threads per multiprocessor, `iters`
+ * steps per chain) and returns how many FMAs that launch performs (0 on a bad argument or a failed launch).
+ * Timed with events by the caller it gives the device's fp64 rate: 2 * FMAs / seconds flop/s, the peak that
+ * kernels bound by plain fp64 arithmetic are held against.  sink_dev: one double in device memory (never written
+ * in practice; it only keeps the arithmetic alive).
+ */
+uint64_t hora_fp64_probe(int32_t iters, double *sink_dev, void *stream);
+
 const char *hora_status_string(hora_status_t status);   /* host: static string */
 int         hora_version(void);                         /* host: major*10000 + minor*100 + patch */
 uint64_t    hora_launch_count(void);                    /* host: kernels this library has launched so far in this

@@ -30,7 +30,7 @@ EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora
            "hora_allocate_batched", "hora_allocate_batched_workspace_bytes", "hora_rollout_weights",
            "hora_learned_prior", "hora_beta_binomial_nll", "hora_pass_at_k", "hora_pass_at_k_workspace_bytes",
            "hora_group_advantage_tokens", "hora_allocation_share", "hora_allocate_hard_first",
-           "hora_allocate_hard_first_workspace_bytes")
+           "hora_allocate_hard_first_workspace_bytes", "hora_fp64_probe")
 
 
 class HoraError(RuntimeError):
@@ -98,6 +98,8 @@ def load() -> C.CDLL:
     L.hora_rollout_weights.restype = C.c_int
     L.hora_token_broadcast.argtypes = [p, p, i64, i64, p, p]
     L.hora_token_broadcast.restype = C.c_int
+    L.hora_fp64_probe.argtypes = [i32, p, p]
+    L.hora_fp64_probe.restype = C.c_uint64
     L.hora_status_string.argtypes = [C.c_int]
     L.hora_status_string.restype = C.c_char_p
     L.hora_version.restype = C.c_int
@@ -209,6 +211,14 @@ def read_infos(info_dev: torch.Tensor, S: int):
         out.append(AllocInfo(x.status, x.first_pass_bits, x.lambda_, x.n_above, x.n_tied, x.n_tied_taken, x.objective,
                              x.sum_G, x.sum_cap))
     return out
+
+
+def hora_fp64_probe(iters, sink_dev) -> int:
+    """Enqueue the fp64 FMA probe kernel; returns the number of FMAs it performs (time it with events)."""
+    n = int(load().hora_fp64_probe(iters, _ptr(sink_dev, torch.float64, "sink_dev"), _stream()))
+    if n == 0:
+        raise HoraError(ERR_CUDA, "hora_fp64_probe")
+    return n
 
 
 def hora_allocate_profile_events(start_event, stop_event):

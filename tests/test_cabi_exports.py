@@ -11,7 +11,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def declared_functions():
     src = open(os.path.join(ROOT, "include", "hora.h")).read()
     src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    names = re.findall(r"\b(hora_[a-z_]+)\s*\(", src)
+    names = re.findall(r"\b(hora_[a-z0-9_]+)\s*\(", src)
     return sorted(set(names))
 
 
