@@ -16,7 +16,7 @@
 //   output      a bitmap of group starts with running counts maps every element to its group; the element
 //               picks one of its group's two values; 16-byte stores.
 // If any reward of the batch is neither 0.0 nor 1.0 the batch takes the general route instead: each group
-// is summed in fp64 by the whole warp (fixed butterfly), its squared
+// is summed in fp64 by a sub-warp of 4, 8 or 32 lanes (fixed butterfly), its squared
 // deviations taken in a second sweep (the two-pass form), and every element evaluated as
 // adv = (r - mean) * scale in fp64, scale = 1 / (std + eps) for GRPO, n / (n - 1) for RLOO
 // (r - (S - r)/(n-1) = (r - S/n) n/(n-1)); for a 0/1 group both routes perform the same operations.
@@ -37,12 +37,7 @@ struct __align__(16) AdvWarpSmem {
     unsigned int starts[kSlab / 32];                          // one bit per element: a non-empty group starts here
     int cum_starts[kSlab / 32];                               // exclusive running counts per word
     float2 two[kWarp];                                        // per non-empty group, in order: advantage of a 0, of a 1
-    // general route: mean and scale per non-empty group, in order; they take the place of `pre`, which only the
-    // 0/1 route reads
-    __device__ __forceinline__ double *mean() { return reinterpret_cast<double *>(pre); }
-    __device__ __forceinline__ double *scale() { return reinterpret_cast<double *>(pre) + kWarp; }
 };
-static_assert(sizeof(unsigned int) * (kSlab / 4 + 4) >= 2 * kWarp * sizeof(double), "mean and scale fit in pre");
 constexpr size_t kAdvSmem = sizeof(AdvWarpSmem) * kAdvWarps;
 
 __device__ __forceinline__ int64_t shfl_i64(int64_t v, int src) { return __shfl_sync(kFull, v, src); }
@@ -88,6 +83,53 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 // group (in the order of the batch's non-empty groups) of element el, through the start bitmap
 __device__ __forceinline__ int rank_of(const AdvWarpSmem &sm, int el) {
     return sm.cum_starts[el >> 5] + __popc(sm.starts[el >> 5] & (0xFFFFFFFFu >> (31 - (el & 31)))) - 1;
+}
+
+// General rewards, one staged batch: groups done .. last of the warp's 32 (lane g owns group g; my_rs, my_re are
+// its bounds inside the slab).  The warp is split into sub-warps of W lanes and a sub-warp walks one group, W
+// elements a step: the sum (hence the mean), then for GRPO the squared deviations (the two-pass form), both in
+// fp64 with a fixed butterfly over the W lanes; the lane that owns the group turns them into its scale; a last
+// walk replaces every staged reward by (r - mean) * scale.  A whole warp per group, the first form of this route,
+// left 27 of 32 lanes idle on groups of five.
+template <int W>
+__device__ __forceinline__ void general_batch(float *buf, int done, int last, int my_rs, int my_re, int64_t my_n,
+                                              int32_t mode, double eps, int32_t ddof, int lane) {
+    constexpr int kPer = kWarp / W;                           // groups per pass
+    const int sub = lane / W, sl = lane % W;
+    const int n_pass = (last - done + kPer) / kPer;
+    const bool mine = lane >= done && lane <= last;
+    const int my_pass = mine ? (lane - done) / kPer : -1, my_src = mine ? ((lane - done) % kPer) * W : 0;
+    double mean_mine = 0.0, ss_mine = 0.0;
+    for (int p = 0; p < n_pass; ++p) {
+        const int g = done + p * kPer + sub;
+        const int s = __shfl_sync(kFull, my_rs, g & 31), e = __shfl_sync(kFull, my_re, g & 31);
+        double part = 0.0;
+        if (g <= last)
+            for (int j = s + sl; j < e; j += W) part += (double)buf[j];
+#pragma unroll
+        for (int d = 1; d < W; d <<= 1) part += __shfl_xor_sync(kFull, part, d);
+        const double mean = e > s ? part / (double)(e - s) : 0.0;
+        double sq = 0.0;
+        if (mode == HORA_ADV_GRPO) {
+            if (g <= last)
+                for (int j = s + sl; j < e; j += W) {
+                    const double dv = (double)buf[j] - mean;
+                    sq += dv * dv;
+                }
+#pragma unroll
+            for (int d = 1; d < W; d <<= 1) sq += __shfl_xor_sync(kFull, sq, d);
+        }
+        const double tm = __shfl_sync(kFull, mean, my_src), ts = __shfl_sync(kFull, sq, my_src);
+        if (p == my_pass) { mean_mine = tm; ss_mine = ts; }
+    }
+    const double scale_mine = group_scale(mode, ss_mine, my_n, ddof, eps);
+    for (int p = 0; p < n_pass; ++p) {
+        const int g = done + p * kPer + sub;
+        const int s = __shfl_sync(kFull, my_rs, g & 31), e = __shfl_sync(kFull, my_re, g & 31);
+        const double M = __shfl_sync(kFull, mean_mine, g & 31), S = __shfl_sync(kFull, scale_mine, g & 31);
+        if (g <= last)
+            for (int j = s + sl; j < e; j += W) buf[j] = (float)(((double)buf[j] - M) * S);
+    }
 }
 
 // VEC4: rewards and adv are 16-byte aligned, so a batch is staged and written in 16-byte pieces starting at
@@ -240,33 +282,28 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
                     adv[start + el] = sm.buf[el] == 1.0f ? a.y : a.x;
                 }
             } else {
-                // ---- general route: whole-warp two-pass sums per group over the slab ----
-                double my_mean = 0.0, my_ss = 0.0;
-                for (int i = done; i <= last; ++i) {
-                    const int s = __shfl_sync(kFull, my_rs, i), e = __shfl_sync(kFull, my_re, i);
-                    if (e <= s) continue;
-                    double part = 0.0;
-                    for (int j = s + lane; j < e; j += kWarp) part += (double)sm.buf[j];
-                    const double mean = warp_sum(part) / (double)(e - s);
-                    double ss = 0.0;
-                    if (mode == HORA_ADV_GRPO) {
-                        double sq = 0.0;
-                        for (int j = s + lane; j < e; j += kWarp) {
-                            const double d = (double)sm.buf[j] - mean;
-                            sq += d * d;
-                        }
-                        ss = warp_sum(sq);
-                    }
-                    if (lane == i) { my_mean = mean; my_ss = ss; }
-                }
-                if (nonempty) {
-                    sm.mean()[my_rank] = my_mean;
-                    sm.scale()[my_rank] = group_scale(mode, my_ss, my_n, ddof, eps);
-                }
+                // ---- general route: sub-warps of W lanes walk one group each over the slab (W by the batch's mean
+                // group size); two walks for the statistics, a third overwrites every reward by its advantage ----
+                const int mean_size = (span - lead) / nfit;
+                if (mean_size > 48) general_batch<32>(sm.buf, done, last, my_rs, my_re, my_n, mode, eps, ddof, lane);
+                else if (mean_size > 10) general_batch<8>(sm.buf, done, last, my_rs, my_re, my_n, mode, eps, ddof, lane);
+                else general_batch<4>(sm.buf, done, last, my_rs, my_re, my_n, mode, eps, ddof, lane);
                 __syncwarp();
-                for (int el = lead + lane; el < span; el += kWarp) {
-                    const int r = rank_of(sm, el);
-                    adv[start + el] = (float)(((double)sm.buf[el] - sm.mean()[r]) * sm.scale()[r]);
+                // the slab leaves in 16-byte pieces, the ragged ends one element per lane and step
+                if (VEC4) {
+                    float *dst4 = adv + start + 4 * lane;
+                    for (int j = 0; j < n_rows; ++j) {
+                        const int e0 = 128 * j + 4 * lane;
+                        if (e0 >= lead && e0 + 4 <= span)
+                            *reinterpret_cast<float4 *>(dst4 + 128 * j) = *reinterpret_cast<const float4 *>(&sm.buf[e0]);
+                    }
+                }
+                const int head_end = VEC4 ? min(span, (lead + 3) & ~3) : span;
+                const int tail_beg = VEC4 ? max(head_end, span & ~3) : span;
+                const int n_rag = (head_end - lead) + (span - tail_beg);
+                for (int i = lane; i < n_rag; i += kWarp) {
+                    const int el = i < head_end - lead ? lead + i : tail_beg + (i - (head_end - lead));
+                    adv[start + el] = sm.buf[el];
                 }
             }
             __syncwarp();

@@ -732,13 +732,30 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
     const unsigned long long digit_mask = (1ull << bits) - 1ull;
     const int64_t stride = (int64_t)gridDim.x * kSelThreads;
     bool bad = false;
+    // The inputs of a thread's NEXT row (guess, prior, count, cap) are fetched while the current row's keys are
+    // being looked at.
+    struct RowInputs { double al, be; int32_t ci, capi; unsigned int guess; };
+    auto fetch_inputs = [&](int64_t row) {
+        RowInputs in;
+        in.al = alpha0; in.be = beta0; in.ci = 0; in.capi = cap_scalar; in.guess = 0;
+        if (row < N) {
+            in.guess = __ldg(pguess + row);
+            if (alpha) { in.al = __ldg(alpha + row); in.be = __ldg(beta + row); }
+            in.ci = __ldg(c + row);
+            if (cap) in.capi = __ldg(cap + row);
+        }
+        return in;
+    };
+    RowInputs nxt = fetch_inputs((int64_t)blockIdx.x * kSelThreads + threadIdx.x);
     for (int64_t base = (int64_t)blockIdx.x * kSelThreads; base < N; base += stride) {
         const int64_t row = base + threadIdx.x;
         int32_t p_hi = 0, n_eq = 0;
         const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains);
+        const RowInputs cur = nxt;
+        nxt = fetch_inputs(row + stride);
         if (row < N) {
-            const unsigned int guess = __ldg(pguess + row);
-            const Posterior post = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row);
+            const unsigned int guess = cur.guess;
+            const Posterior post = make_posterior(cur.al, cur.be, cur.ci, cur.capi, G0, ld);
             bad |= !post.ok;
             const int32_t capi = post.cap;                       // 0 for an invalid row
             keys += row * (int64_t)ld;
@@ -1658,7 +1675,8 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     const int rows_per_cta = kSelThreads / kWarp;
     const int64_t every = (N + kSampleRows - 1) / kSampleRows;
     const int64_t n_sample = (N + every - 1) / every;
-    const int grid_est = clamp_grid((n_sample + rows_per_cta - 1) / rows_per_cta, 4);
+    // two rows per warp: half as many CTAs flush their histogram into the same few hundred global bins
+    const int grid_est = clamp_grid((n_sample + 2 * rows_per_cta - 1) / (2 * rows_per_cta), 2);
     mark_stage(0, s);
     if (B > 0 && !fused)
         select_estimate<<<grid_est, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, every, gains, B, w.hdr, w.hist_est);

@@ -28,20 +28,24 @@ struct Posterior {
     bool ok;
 };
 
-__device__ __forceinline__ Posterior load_posterior(const double *alpha, const double *beta, double alpha0,
-                                                    double beta0, const int32_t *c, int32_t G0,
-                                                    const int32_t *cap, int32_t cap_scalar, int32_t ld, int64_t i) {
+// The posterior and its checks from a prompt's raw inputs (already in registers).
+__device__ __forceinline__ Posterior make_posterior(double al, double be, int32_t ci, int32_t capi, int32_t G0, int32_t ld) {
     Posterior p;
-    const double al = alpha ? __ldg(alpha + i) : alpha0;
-    const double be = beta ? __ldg(beta + i) : beta0;
-    const int32_t ci = __ldg(c + i);
-    p.cap = cap ? __ldg(cap + i) : cap_scalar;
+    p.cap = capi;
     p.ok = (al > 0.0) && (be > 0.0) && (al < 1.0e300) && (be < 1.0e300) && (ci >= 0) && (ci <= G0) &&
            (p.cap >= 0) && (p.cap <= ld);
     p.a = al + (double)ci;
     p.b = be + (double)(G0 - ci);
     if (!p.ok) p.cap = 0;
     return p;
+}
+
+__device__ __forceinline__ Posterior load_posterior(const double *alpha, const double *beta, double alpha0,
+                                                    double beta0, const int32_t *c, int32_t G0,
+                                                    const int32_t *cap, int32_t cap_scalar, int32_t ld, int64_t i) {
+    const double al = alpha ? __ldg(alpha + i) : alpha0;
+    const double be = beta ? __ldg(beta + i) : beta0;
+    return make_posterior(al, be, __ldg(c + i), cap ? __ldg(cap + i) : cap_scalar, G0, ld);
 }
 
 inline hora_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? HORA_OK : HORA_ERR_CUDA; }
