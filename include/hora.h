@@ -369,8 +369,9 @@ hora_status_t hora_token_broadcast(const float *adv, const int64_t *token_offset
  * handles (created by the caller with timing enabled), every following hora_allocate / hora_allocate_static
  * call records `start_event` just before and `stop_event` just after the launch of its full-read selection
  * pass (the kernel that reads the whole gains matrix) on the call's stream, so that kernel can be timed on
- * the device without a profiler.  Pass NULLs to switch it off (the default).  Process-wide host setting; set
- * it from the thread that issues the calls.
+ * the device without a profiler.  Pass NULLs to switch it off (the default).  The setting belongs to the calling
+ * host thread: only hora_allocate calls issued by that thread record the events, so allocations running at the
+ * same time from other threads (on other streams) are not touched.
  */
 void hora_allocate_profile_events(void *start_event, void *stop_event);
 
@@ -381,8 +382,10 @@ void hora_allocate_profile_events(void *start_event, void *stop_event);
  * [2] after the full-read pass, [3] after the per-row pass (level 1), [4] after the tail (threshold complete,
  * prefixes over prompts formed), [5] after the exact tie ranking (right after [4] when that does not run),
  * [6] after the outputs are written.  Differences of consecutive events are the device times of the stages.
- * A NULL handle skips its point; NULL or n = 0 switches everything off (the default).  Process-wide host
- * setting; the array is read during this call only.
+ * A NULL handle skips its point; NULL or n = 0 switches everything off (the default).  Per host thread, like
+ * hora_allocate_profile_events; the array is read during this call only.  On the rank-based route the points are
+ * [0] entry, [1] after the rank tables, [2] = [3] after the counting pass, [4] = [5] after the sums, [6] after the
+ * outputs.
  */
 void hora_allocate_profile_stages(void *const *events_host, int32_t n);
 

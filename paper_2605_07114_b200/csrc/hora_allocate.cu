@@ -1544,12 +1544,14 @@ __global__ void write_empty(int64_t B, int64_t *offsets, hora_alloc_info *info) 
 
 // Optional profiling aids (see hora_allocate_profile_events / hora_allocate_profile_stages): events recorded
 // around the full-read pass, and after each stage of the call.
-static std::atomic<cudaEvent_t> g_prof_start{nullptr}, g_prof_stop{nullptr};
+// The handles are kept per host thread: only calls issued by the thread that set them record anything, so calls
+// running concurrently from other threads (on other streams) are left alone.
+static thread_local cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 constexpr int kStageEvents = 7;
-static std::atomic<cudaEvent_t> g_stage_ev[kStageEvents];
+static thread_local cudaEvent_t g_stage_ev[kStageEvents] = {};
 
 static inline void mark_stage(int k, cudaStream_t s) {
-    const cudaEvent_t ev = g_stage_ev[k].load(std::memory_order_relaxed);
+    const cudaEvent_t ev = g_stage_ev[k];
     if (ev != nullptr) cudaEventRecord(ev, s);
 }
 
@@ -1603,14 +1605,13 @@ static int tail_grid_size() {
 }  // namespace hora
 
 extern "C" void hora_allocate_profile_events(void *start_event, void *stop_event) {
-    hora::g_prof_start.store(static_cast<cudaEvent_t>(start_event), std::memory_order_relaxed);
-    hora::g_prof_stop.store(static_cast<cudaEvent_t>(stop_event), std::memory_order_relaxed);
+    hora::g_prof_start = static_cast<cudaEvent_t>(start_event);
+    hora::g_prof_stop = static_cast<cudaEvent_t>(stop_event);
 }
 
 extern "C" void hora_allocate_profile_stages(void *const *events_host, int32_t n) {
     for (int k = 0; k < hora::kStageEvents; ++k)
-        hora::g_stage_ev[k].store(events_host != nullptr && k < n ? static_cast<cudaEvent_t>(events_host[k]) : nullptr,
-                                  std::memory_order_relaxed);
+        hora::g_stage_ev[k] = events_host != nullptr && k < n ? static_cast<cudaEvent_t>(events_host[k]) : nullptr;
 }
 
 extern "C" size_t hora_allocate_workspace_bytes(int64_t N, int32_t ld, int32_t gains_is_null, uint32_t flags) {
@@ -1682,8 +1683,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         select_estimate<<<grid_est, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, every, gains, B, w.hdr, w.hist_est);
     const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 3);
     const int grid1 = clamp_grid((N + kSelThreads - 1) / kSelThreads, kLevel1PerSm);
-    const cudaEvent_t prof_start = g_prof_start.load(std::memory_order_relaxed);
-    const cudaEvent_t prof_stop = g_prof_stop.load(std::memory_order_relaxed);
+    const cudaEvent_t prof_start = g_prof_start, prof_stop = g_prof_stop;
     if (!fused) mark_stage(1, s);                         // (the fused pass launches its own estimate)
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_start, s);
     if (fused) {
@@ -1694,7 +1694,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         else if (ld > 64)
             e = launch_fused<4>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, w);
         else
-            e = launch_fused<2>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, w);
+            e = launch_fused<8>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, w);
         if (e != cudaSuccess) return HORA_ERR_CUDA;
     } else if (ld > 128) {
         launch_level0<8>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);

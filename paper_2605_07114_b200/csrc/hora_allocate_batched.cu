@@ -467,7 +467,7 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
         cudaError_t e;
         if (ld > 128) e = launch(allocate_batched_kernel<8>);
         else if (ld > 64) e = launch(allocate_batched_kernel<4>);
-        else e = launch(allocate_batched_kernel<2>);
+        else e = launch(allocate_batched_kernel<8>);   // short rows: as hora_gains builds them (8 entries a lane)
         if (e != cudaSuccess) return HORA_ERR_CUDA;
         ++launches;
     }

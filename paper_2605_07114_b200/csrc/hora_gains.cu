@@ -14,27 +14,30 @@
 namespace hora {
 
 // The kernel is the shared row loop with no tap attached.
-template <int E, bool VEC2>
+// LG: lanes per row.  Rows of at most 64 entries are built four (LG = 8) or eight (LG = 4) to a warp, so that a
+// warp still produces 256 entries per scan and per reciprocal: a whole warp on a 64-entry row spent as many
+// instructions per row as on a 256-entry one, and those, not the memory system, set the time (2.9 TB/s).
+template <int E, bool VEC2, int LG>
 __global__ void __launch_bounds__(kGainsWarps *kWarp, 3)
 gains_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
              const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
              int64_t N, int32_t ld, double *__restrict__ gains, int32_t *status_dev) {
     NoTap tap;
-    gains_rows_cta<E, VEC2>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, tap);
+    gains_rows_cta<E, VEC2, NoTap, LG>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, tap);
 }
 
-template <int E>
+template <int E, int LG>
 static hora_status_t launch_e(const double *alpha, const double *beta, double alpha0, double beta0, const int32_t *c,
                               int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N, int32_t ld, double *gains,
                               int32_t *status_dev, cudaStream_t stream) {
     const int grid = clamp_grid((N + kCtaRows - 1) / kCtaRows, 3);
     const bool vec2 = (ld % 2 == 0) && ((reinterpret_cast<uintptr_t>(gains) & 15u) == 0);
     if (vec2)
-        gains_kernel<E, true><<<grid, kGainsWarps * kWarp, 0, stream>>>(alpha, beta, alpha0, beta0, c, G0, cap,
-                                                                        cap_scalar, N, ld, gains, status_dev);
+        gains_kernel<E, true, LG><<<grid, kGainsWarps * kWarp, 0, stream>>>(alpha, beta, alpha0, beta0, c, G0, cap,
+                                                                            cap_scalar, N, ld, gains, status_dev);
     else
-        gains_kernel<E, false><<<grid, kGainsWarps * kWarp, 0, stream>>>(alpha, beta, alpha0, beta0, c, G0, cap,
-                                                                         cap_scalar, N, ld, gains, status_dev);
+        gains_kernel<E, false, LG><<<grid, kGainsWarps * kWarp, 0, stream>>>(alpha, beta, alpha0, beta0, c, G0, cap,
+                                                                             cap_scalar, N, ld, gains, status_dev);
     count_launches(1);
     return cuda_ok(cudaGetLastError());
 }
@@ -43,10 +46,12 @@ hora_status_t launch_gains(const double *alpha, const double *beta, double alpha
                            int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N, int32_t ld, double *gains,
                            int32_t *status_dev, cudaStream_t stream) {
     if (ld > 128)
-        return launch_e<8>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
+        return launch_e<8, kWarp>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
     if (ld > 64)
-        return launch_e<4>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
-    return launch_e<2>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
+        return launch_e<4, kWarp>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
+    if (ld > 32)
+        return launch_e<8, 8>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
+    return launch_e<8, 4>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
 }
 
 }  // namespace hora

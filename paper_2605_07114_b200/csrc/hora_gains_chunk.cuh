@@ -18,12 +18,23 @@ struct NoTap {
 // One chunk of 32*E entries of one row, starting at column k0.  FULL: the chunk lies entirely below the
 // row's cap and inside the row, so no entry needs masking.  `out` may be null when only the tap wants the
 // values (then nothing is stored).
-template <int E, bool VEC2, bool FULL, typename Tap = NoTap>
+//
+// LG < 32: packed rows.  The warp holds 32 / LG rows at once, LG lanes each (a, b, capi and `out` then differ
+// from group to group, `lane` is the lane's position inside its group, and the scan runs over the group only).
+// A lane's entries depend on the lanes before it in its row and on nothing else, so a row computed by a group
+// of LG lanes has the same bits as the same row computed by a whole warp whose other lanes lie past its end.
+// `tile_ld`: the staged store path treats the warp's 32 * E entries as one run of memory starting at `out` (rows
+// of exactly LG * E entries, packed) and writes the first tile_ld of them; for a single row it is ld.
+// STAGE: results leave through the swizzled shared-memory slab (the default wherever 16-byte stores are possible and
+// a lane has more than one of them); packed rows that are shorter than LG * E entries, hence not back to back in
+// memory, store directly instead.
+template <int E, bool VEC2, bool FULL, typename Tap = NoTap, int LG = kWarp, bool STAGE = VEC2 && (E > 2)>
 __device__ __forceinline__ void gains_chunk(double a, double b, double ab, int32_t capi, int32_t ld, int32_t k0,
                                             int lane, double &carry, double *__restrict__ out, double2 *wr,
-                                            const double2 *rd, Tap &&tap = Tap()) {
+                                            const double2 *rd, Tap &&tap = Tap(), int32_t tile_ld = -1) {
     constexpr int P = E / 2;                              // 16-byte chunks per lane
-    constexpr bool kStaged = VEC2 && (P > 1);
+    constexpr bool kStaged = STAGE;
+    static_assert(!STAGE || (VEC2 && P > 1), "staging needs 16-byte stores and more than one of them per lane");
     const int32_t k = k0 + lane * E;
     // factors of entries k .. k+E-1: num = a (k = 0) or b + k - 1, then +1 each; den = a + b + k, then +1 each
     const double x = b + (double)(k - 1), y = ab + (double)k;
@@ -38,13 +49,13 @@ __device__ __forceinline__ void gains_chunk(double a, double b, double ab, int32
     const double r = 1.0 / S[0];
     double inc = pt * r;                                  // this lane's E-factor product
 #pragma unroll
-    for (int d = 1; d < kWarp; d <<= 1) {
-        const double t = shfl_up_f64(inc, d);
+    for (int d = 1; d < LG; d <<= 1) {
+        const double t = __shfl_up_sync(kFull, inc, d, LG);
         if (lane >= d) inc *= t;
     }
-    double excl = shfl_up_f64(inc, 1);
+    double excl = __shfl_up_sync(kFull, inc, 1, LG);
     if (lane == 0) excl = 1.0;
-    const double total = shfl_idx_f64(inc, kWarp - 1);
+    const double total = __shfl_sync(kFull, inc, LG - 1, LG);
     double pm = (carry * excl * r) * n0;                  // running numerator product times everything shared
     carry *= total;
 #pragma unroll
@@ -59,7 +70,8 @@ __device__ __forceinline__ void gains_chunk(double a, double b, double ab, int32
         }
         tap.pair(m, g0, g1);
         if (kStaged) {
-            wr[(m >> 1) ^ ((lane >> (P == 4 ? 1 : 2)) & (P - 1))] = make_double2(g0, g1);   // (lane*P + p) >> 3
+            const int wl = LG == kWarp ? lane : (int)(threadIdx.x & (kWarp - 1));   // position in the warp's tile
+            wr[(m >> 1) ^ ((wl >> (P == 4 ? 1 : 2)) & (P - 1))] = make_double2(g0, g1);   // (wl*P + p) >> 3
         } else if (VEC2) {
             if (FULL || k + m < ld) *reinterpret_cast<double2 *>(out + k + m) = make_double2(g0, g1);
         } else if (out != nullptr) {
@@ -70,11 +82,13 @@ __device__ __forceinline__ void gains_chunk(double a, double b, double ab, int32
     tap.finish(k0, k, capi, ld);
     if (kStaged) {
         __syncwarp();
+        const int wl = LG == kWarp ? lane : (int)(threadIdx.x & (kWarp - 1));
+        const int32_t bound = LG == kWarp ? ld : tile_ld;
 #pragma unroll
         for (int q = 0; q < P; ++q) {
             const double2 v = rd[q * kWarp];
-            const int32_t col = k0 + 2 * (q * kWarp + lane);
-            if (FULL || col < ld) *reinterpret_cast<double2 *>(out + col) = v;
+            const int32_t col = k0 + 2 * (q * kWarp + wl);
+            if ((FULL && LG == kWarp) || col < bound) *reinterpret_cast<double2 *>(out + col) = v;
         }
         __syncwarp();
     }
@@ -86,7 +100,8 @@ constexpr int kCtaRows = kGainsWarps * kTile; // rows a CTA stages per step
 
 // A CTA stages the posterior parameters of 64 consecutive rows in shared memory (one coalesced load per
 // array, issued one step ahead and parked in registers meanwhile); each warp then takes 8 of those rows.
-template <int E, bool VEC2, typename Tap>
+// LG < 32 (rows of at most LG * E entries): a warp builds 32 / LG rows at a time, LG lanes a row (no tap then).
+template <int E, bool VEC2, typename Tap, int LG = kWarp>
 __device__ __forceinline__ void gains_rows_cta(const double *__restrict__ alpha, const double *__restrict__ beta,
                                                double alpha0, double beta0, const int32_t *__restrict__ c, int32_t G0,
                                                const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N,
@@ -130,6 +145,30 @@ __device__ __forceinline__ void gains_rows_cta(const double *__restrict__ alpha,
         __syncthreads();                                  // buf was last read two steps ago: safe to have overwritten it
         nxt = fetch(step + gridDim.x);
         const int64_t row0 = step * kCtaRows + warp * kTile;
+        if (LG < kWarp) {
+            // packed rows: group g of the warp builds row row0 + i + g
+            constexpr int R = kWarp / LG;
+            const int grp = lane / LG, gl = lane % LG;
+            const bool back_to_back = VEC2 && E > 2 && ld == LG * E;   // the rows of a tile are one run of memory
+            for (int i = 0; i < kTile && row0 + i < N; i += R) {
+                const int64_t row = row0 + i + grp;
+                const bool live = row < N;
+                const int idx = warp * kTile + i + grp;
+                const double a = s_a[buf][idx], b = s_b[buf][idx];
+                const int32_t capi = live ? s_cap[buf][idx] : 0;
+                double carry = 1.0;
+                if (back_to_back) {
+                    const int64_t rows_here = N - (row0 + i) < R ? N - (row0 + i) : R;
+                    gains_chunk<E, VEC2, false, NoTap, LG, VEC2 && (E > 2)>(a, b, a + b, capi, ld, 0, gl, carry,
+                                                                          gains + (row0 + i) * (int64_t)ld, wr, rd,
+                                                                          NoTap(), (int32_t)(rows_here * ld));
+                } else {
+                    gains_chunk<E, VEC2, false, NoTap, LG, false>(a, b, a + b, capi, live ? ld : 0, 0, gl, carry,
+                                                                 gains + (live ? row : 0) * (int64_t)ld, nullptr, nullptr);
+                }
+            }
+            continue;
+        }
         for (int i = 0; i < kTile && row0 + i < N; ++i) {
             const double a = s_a[buf][warp * kTile + i], b = s_b[buf][warp * kTile + i];
             const int32_t capi = s_cap[buf][warp * kTile + i];

@@ -172,7 +172,7 @@ int launch_rank_tables(double alpha0, double beta0, int32_t G0, int32_t ld, cons
     bool ok;
     if (ld > 128) ok = go(rank_table_kernel<8>);
     else if (ld > 64) ok = go(rank_table_kernel<4>);
-    else ok = go(rank_table_kernel<2>);
+    else ok = go(rank_table_kernel<8>);                       // short rows: as hora_gains builds them
     if (!ok) return -1;
     int launches = 1;
     if (t.pos != nullptr) {

@@ -844,3 +844,45 @@ def test_allocation_share_of_an_allocation_and_bad_input():
     assert int(status.item()) == 2 and int(prompts.sum()) == 2
     with pytest.raises(hora.HoraError):
         hora.hora_allocation_share(None, None, 0, 4096, prompts, budget)
+
+
+# ------------------------------------------------------------------------------- concurrency
+def test_two_allocations_on_two_streams_with_their_own_workspaces():
+    """Calls on different streams may overlap as long as they share neither outputs nor workspaces: two different
+    problems are enqueued alternately on two streams, several rounds, from two host threads, and each result is held
+    against the oracle (and against the same problem run alone)."""
+    import threading
+    from paper_2605_07114_b200 import hora
+    gu = _util()
+    probs = []
+    for name, N in (("cfg4", 40000), ("cfg5", 60000)):
+        w = wl.make(name, N)
+        d_o, G_o, lam_o, obj_o = gu.oracle_allocate(w)
+        al = hora.Allocator(w.N, w.ld, w.G0, exact_int=w.exact_int)
+        dev = lambda x: None if x is None else gu.dev(x)
+        probs.append(dict(w=w, al=al, args=(dev(w.alpha), dev(w.beta), 1.0, 1.0, dev(w.c), dev(w.cap), 0, w.B),
+                          oracle=(d_o, lam_o, obj_o), stream=torch.cuda.Stream()))
+    torch.cuda.synchronize()
+    errors = []
+
+    def worker(p):
+        try:
+            with torch.cuda.stream(p["stream"]):
+                for _ in range(6):
+                    p["al"].delta.fill_(-1)
+                    p["al"].run(*p["args"])
+        except Exception as exc:                                 # pragma: no cover - reported below
+            errors.append(exc)
+
+    threads = [threading.Thread(target=worker, args=(p,)) for p in probs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    for p in probs:
+        al, w = p["al"], p["w"]
+        d_o, lam_o, obj_o = p["oracle"]
+        gu.assert_allocation_matches(w, al.delta.cpu().numpy(), al.G.cpu().numpy(), al.group_offsets.cpu().numpy(),
+                                     al.read_info(), d_o, lam_o, obj_o)
