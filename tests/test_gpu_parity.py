@@ -404,7 +404,7 @@ def test_allocation_status_codes():
     assert info.status == 2 and not d.any()
 
 
-@pytest.mark.parametrize("ld,cap_value", [(256, 256), (256, 200), (96, 96), (40, 33)])
+@pytest.mark.parametrize("ld,cap_value", [(256, 256), (256, 200), (96, 96), (40, 33), (64, 64), (64, 50)])
 def test_allocation_validates_a_given_gains_matrix(ld, cap_value):
     """hora_allocate checks the matrix it is given: every row finite, non-negative and non-increasing up to its
     cap.  Equal neighbours are allowed; a disorder that shows only in the low 32 bits of two keys with equal
