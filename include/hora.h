@@ -399,6 +399,18 @@ void hora_allocate_profile_stages(void *const *events_host, int32_t n);
  */
 uint64_t hora_fp64_probe(int32_t iters, double *sink_dev, void *stream);
 
+/*
+ * hora_checked_violation — verification aid, no counterpart in the paper.  The library can be built a second time
+ * with -DHORA_CHECKED (python -m paper_2605_07114_b200.build --checked writes libhora_checked.so): every access of
+ * the allocation, batched-allocation and advantage kernels whose index is computed from device data then checks
+ * that index against the size of its array; a violation is recorded (never trapped: the access goes to a scratch
+ * slot and the kernel runs on).  This call synchronises the device and returns 0 if no check has failed since the
+ * last call, else (file id << 20) | source line of the first failure (file ids: 1 hora_allocate.cu,
+ * 2 hora_allocate_batched.cu, 3 hora_advantage.cu, 4 hora_rank.cu); the record is cleared.  The normal build has no
+ * checks and returns -1; -2 reports a failed synchronisation.
+ */
+int32_t hora_checked_violation(void);
+
 const char *hora_status_string(hora_status_t status);   /* host: static string */
 int         hora_version(void);                         /* host: major*10000 + minor*100 + patch */
 uint64_t    hora_launch_count(void);                    /* host: kernels this library has launched so far in this

@@ -23,7 +23,11 @@
 // A group longer than a batch is streamed from global memory (same arithmetic).
 // r - mean is exactly zero for a constant group (partial sums k*r are exact in fp64), so such groups
 // get exactly zero.  Every order of operations is fixed: results are bitwise reproducible.
+#define HORA_FILE_ID 3
+#include "hora_checked.cuh"
 #include "hora_group_stats.cuh"
+
+HORA_CHECKED_REGISTER()
 
 namespace hora {
 
@@ -69,7 +73,7 @@ __device__ __forceinline__ void running_counts(const unsigned int *word, int *cu
 
 // ones among elements [0, pos) of the batch, from the packed prefix words
 __device__ __forceinline__ int ones_before(const unsigned int *pre, int pos) {
-    const unsigned w = pre[pos >> 2];
+    const unsigned w = HORA_AT(pre, pos >> 2, kSlab / 4 + 4);
     return (int)(w >> 4) + __popc(w & ((1u << (pos & 3)) - 1u));
 }
 
@@ -105,7 +109,7 @@ __device__ __forceinline__ void general_batch(float *buf, int done, int last, in
         const int s = __shfl_sync(kFull, my_rs, g & 31), e = __shfl_sync(kFull, my_re, g & 31);
         double part = 0.0;
         if (g <= last)
-            for (int j = s + sl; j < e; j += W) part += (double)buf[j];
+            for (int j = s + sl; j < e; j += W) part += (double)HORA_AT(buf, j, kSlab);
 #pragma unroll
         for (int d = 1; d < W; d <<= 1) part += __shfl_xor_sync(kFull, part, d);
         const double mean = e > s ? part / (double)(e - s) : 0.0;
@@ -113,7 +117,7 @@ __device__ __forceinline__ void general_batch(float *buf, int done, int last, in
         if (mode == HORA_ADV_GRPO) {
             if (g <= last)
                 for (int j = s + sl; j < e; j += W) {
-                    const double dv = (double)buf[j] - mean;
+                    const double dv = (double)HORA_AT(buf, j, kSlab) - mean;
                     sq += dv * dv;
                 }
 #pragma unroll
@@ -128,7 +132,7 @@ __device__ __forceinline__ void general_batch(float *buf, int done, int last, in
         const int s = __shfl_sync(kFull, my_rs, g & 31), e = __shfl_sync(kFull, my_re, g & 31);
         const double M = __shfl_sync(kFull, mean_mine, g & 31), S = __shfl_sync(kFull, scale_mine, g & 31);
         if (g <= last)
-            for (int j = s + sl; j < e; j += W) buf[j] = (float)(((double)buf[j] - M) * S);
+            for (int j = s + sl; j < e; j += W) HORA_AT(buf, j, kSlab) = (float)(((double)HORA_AT(buf, j, kSlab) - M) * S);
     }
 }
 
@@ -186,13 +190,13 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
             if (VEC4 && !tail) {
                 const float *src = rewards + start + 4 * lane;
                 for (int j = 0; j < n_rows; ++j) {
-                    if (128 * j + 4 * lane < span) cp_async_16(&sm.buf[128 * j + 4 * lane], src + 128 * j);
+                    if (128 * j + 4 * lane < span) cp_async_16(&HORA_AT(sm.buf, 128 * j + 4 * lane, kSlab - 3), src + 128 * j);
                     else *reinterpret_cast<float4 *>(&sm.buf[128 * j + 4 * lane]) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                 }
                 cp_async_wait_all();
             } else {
                 for (int j = lane; j < 128 * n_rows; j += kWarp)
-                    sm.buf[j] = (j < span && start + j < n_all) ? __ldg(rewards + start + j) : 0.0f;
+                    HORA_AT(sm.buf, j, kSlab) = (j < span && start + j < n_all) ? __ldg(&HORA_AT(rewards, start + j, n_all)) : 0.0f;
             }
             __syncwarp();
             // ---- which rewards are 1.0 (packed prefix words); is anything neither 0.0 nor 1.0? ----
@@ -236,7 +240,7 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
             for (int w = lane; w < 4 * n_rows; w += kWarp) sm.starts[w] = 0u;
             __syncwarp();
             const bool nonempty = mine && my_re > my_rs;
-            if (nonempty) atomicOr(&sm.starts[my_rs >> 5], 1u << (my_rs & 31));
+            if (nonempty) atomicOr(&HORA_AT(sm.starts, my_rs >> 5, kSlab / 32), 1u << (my_rs & 31));
             const int my_rank = __popc(__ballot_sync(kFull, nonempty) & lt);
             __syncwarp();
             running_counts(sm.starts, sm.cum_starts, 4 * n_rows, lane);
@@ -248,7 +252,7 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
                 const double mean = my_n > 0 ? k / dn : 0.0;
                 const double ss = k * (dn - k) / (my_n > 0 ? dn : 1.0);
                 const double scale = group_scale(mode, ss, my_n, ddof, eps);
-                if (nonempty) sm.two[my_rank] = make_float2((float)((0.0 - mean) * scale), (float)((1.0 - mean) * scale));
+                if (nonempty) HORA_AT(sm.two, my_rank, kWarp) = make_float2((float)((0.0 - mean) * scale), (float)((1.0 - mean) * scale));
                 __syncwarp();
                 // ---- output: element -> group through the start bitmap; whole 16-byte pieces here ----
                 float *dst4 = adv + start + 4 * lane;
@@ -262,13 +266,14 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
                         const int r1 = r0 + (int)((sw >> 1) & 1u);
                         const int r2 = r1 + (int)((sw >> 2) & 1u);
                         const int r3 = r2 + (int)((sw >> 3) & 1u);
-                        const float2 a0 = sm.two[r0], a1 = sm.two[r1], a2 = sm.two[r2], a3 = sm.two[r3];
+                        const float2 a0 = HORA_AT(sm.two, r0, kWarp), a1 = HORA_AT(sm.two, r1, kWarp), a2 = HORA_AT(sm.two, r2, kWarp),
+                                     a3 = HORA_AT(sm.two, r3, kWarp);
                         float4 o;
                         o.x = x.x == 1.0f ? a0.y : a0.x;
                         o.y = x.y == 1.0f ? a1.y : a1.x;
                         o.z = x.z == 1.0f ? a2.y : a2.x;
                         o.w = x.w == 1.0f ? a3.y : a3.x;
-                        *reinterpret_cast<float4 *>(dst4 + 128 * j) = o;
+                        *reinterpret_cast<float4 *>(&HORA_AT(dst4, 128 * j, n_all - start - 4 * lane - 3)) = o;
                     }
                 }
                 // ragged ends (at most 3 elements after `lead` and 3 before `span`; everything when the pointers
@@ -278,8 +283,8 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
                 const int n_rag = (head_end - lead) + (span - tail_beg);
                 for (int i = lane; i < n_rag; i += kWarp) {
                     const int el = i < head_end - lead ? lead + i : tail_beg + (i - (head_end - lead));
-                    const float2 a = sm.two[rank_of(sm, el)];
-                    adv[start + el] = sm.buf[el] == 1.0f ? a.y : a.x;
+                    const float2 a = HORA_AT(sm.two, rank_of(sm, el), kWarp);
+                    HORA_AT(adv, start + el, n_all) = HORA_AT(sm.buf, el, kSlab) == 1.0f ? a.y : a.x;
                 }
             } else {
                 // ---- general route: sub-warps of W lanes walk one group each over the slab (W by the batch's mean
@@ -295,7 +300,8 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
                     for (int j = 0; j < n_rows; ++j) {
                         const int e0 = 128 * j + 4 * lane;
                         if (e0 >= lead && e0 + 4 <= span)
-                            *reinterpret_cast<float4 *>(dst4 + 128 * j) = *reinterpret_cast<const float4 *>(&sm.buf[e0]);
+                            *reinterpret_cast<float4 *>(&HORA_AT(dst4, 128 * j, n_all - start - 4 * lane - 3)) =
+                                *reinterpret_cast<const float4 *>(&HORA_AT(sm.buf, e0, kSlab - 3));
                     }
                 }
                 const int head_end = VEC4 ? min(span, (lead + 3) & ~3) : span;
@@ -303,7 +309,7 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
                 const int n_rag = (head_end - lead) + (span - tail_beg);
                 for (int i = lane; i < n_rag; i += kWarp) {
                     const int el = i < head_end - lead ? lead + i : tail_beg + (i - (head_end - lead));
-                    adv[start + el] = sm.buf[el];
+                    HORA_AT(adv, start + el, n_all) = HORA_AT(sm.buf, el, kSlab);
                 }
             }
             __syncwarp();

@@ -47,11 +47,15 @@
 #include <atomic>
 #include <type_traits>
 
+#define HORA_FILE_ID 1
 #include "hora_block.cuh"
+#include "hora_checked.cuh"
 #include "hora_common.cuh"
 #include "hora_exact.cuh"
 #include "hora_gains_chunk.cuh"
 #include "hora_rank.cuh"
+
+HORA_CHECKED_REGISTER()
 
 namespace hora {
 
@@ -285,7 +289,7 @@ __device__ __forceinline__ int window_count(const unsigned (&h)[E], int valid, u
     for (int m = 0; m < E; ++m) {
         const int ts = (int)(h[m] >> 9) - (int)W0;
         if (m < valid) {
-            if ((unsigned)ts < (unsigned)kFineBins) atomicAdd(&s_fine[ts], 1u);
+            if ((unsigned)ts < (unsigned)kFineBins) atomicAdd(&HORA_AT(s_fine, ts, kFineBins), 1u);
             above += ts > t_guess;
         }
     }
@@ -476,11 +480,11 @@ __device__ __forceinline__ void level0_process(const Level0Item<E> &it, int64_t 
         }
         if (__all_sync(kFull, !vx || tsx < 0)) break;          // ... or wholly below it
         if (vx) {
-            if ((unsigned)tsx < (unsigned)kFineBins) atomicAdd(&s_fine[tsx], 1u);
+            if ((unsigned)tsx < (unsigned)kFineBins) atomicAdd(&HORA_AT(s_fine, tsx, kFineBins), 1u);
             above += tsx > t_guess;
         }
         if (vy) {
-            if ((unsigned)tsy < (unsigned)kFineBins) atomicAdd(&s_fine[tsy], 1u);
+            if ((unsigned)tsy < (unsigned)kFineBins) atomicAdd(&HORA_AT(s_fine, tsy, kFineBins), 1u);
             above += tsy > t_guess;
         }
     }
@@ -702,7 +706,7 @@ __device__ __forceinline__ int32_t first_not_above(const unsigned long long *__r
     int32_t lo = 0, hi = n;
     while (lo < hi) {
         const int32_t mid = (lo + hi) >> 1;
-        const unsigned kp = key_prefix(__ldg(keys + mid), r);
+        const unsigned kp = key_prefix(__ldg(&HORA_AT(keys, mid, n)), r);
         if (STRICT ? kp >= P : kp > P) lo = mid + 1; else hi = mid;
     }
     return lo;
@@ -772,13 +776,13 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
 #pragma unroll
                     for (int u = 0; u < 8; u += 2) {
                         ulonglong2 t = make_ulonglong2(0ull, 0ull);
-                        if (ws + u < we) t = __ldg(reinterpret_cast<const ulonglong2 *>(keys + ws + u));
+                        if (ws + u < we) t = __ldg(reinterpret_cast<const ulonglong2 *>(&HORA_AT(keys, ws + u, ld - 1)));
                         kp[u] = key_prefix(t.x, r);
                         kp[u + 1] = key_prefix(t.y, r);
                     }
                 } else {
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) kp[u] = ws + u < we ? key_prefix(__ldg(keys + ws + u), r) : 0u;
+                    for (int u = 0; u < 8; ++u) kp[u] = ws + u < we ? key_prefix(__ldg(&HORA_AT(keys, ws + u, ld)), r) : 0u;
                 }
                 kp_first = kp[0];
 #pragma unroll
@@ -797,7 +801,7 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
                 if (!left_ok) {                                  // the 8 keys before (independent loads)
                     unsigned kp[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) kp[u] = ws - 1 - u >= 0 ? key_prefix(__ldg(keys + ws - 1 - u), r) : 0u;
+                    for (int u = 0; u < 8; ++u) kp[u] = ws - 1 - u >= 0 ? key_prefix(__ldg(&HORA_AT(keys, ws - 1 - u, ld)), r) : 0u;
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
                         if (ws - 1 - u >= 0) {
@@ -812,7 +816,7 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
                 if (!right_ok) {                                 // the 8 keys after
                     unsigned kp[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) kp[u] = we + u < capi ? key_prefix(__ldg(keys + we + u), r) : 0u;
+                    for (int u = 0; u < 8; ++u) kp[u] = we + u < capi ? key_prefix(__ldg(&HORA_AT(keys, we + u, ld)), r) : 0u;
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
                         if (we + u < capi) {
@@ -836,13 +840,13 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
                 // no key in the threshold's bin: Delta_i = p_hi is final, and g_i(Delta_i) was just read (L1)
                 double u = -1.0;                                 // otherwise: evaluated by the output pass
                 if (n_eq == 0)
-                    u = p_hi > 0 ? utility_from_gain(__longlong_as_double((long long)__ldg(keys + p_hi - 1)), post.a, post.b, p_hi)
+                    u = p_hi > 0 ? utility_from_gain(__longlong_as_double((long long)__ldg(&HORA_AT(keys, p_hi - 1, ld))), post.a, post.b, p_hi)
                                  : 0.0;
                 objrow[row] = u;
             }
             if (!list)                                           // digit route: the segment's keys on the next digit
                 for (int32_t j = 0; j < n_eq; ++j)
-                    atomicAdd(&s_hist[(__ldg(keys + p_hi + j) >> shift) & digit_mask], 1u);
+                    atomicAdd(&HORA_AT(s_hist, (__ldg(&HORA_AT(keys, p_hi + j, ld)) >> shift) & digit_mask, kBins), 1u);
         }
         if (list) {
             // per warp: one addition to the block sum of p_hi, one slot reservation for the warp's keys (the
@@ -864,10 +868,10 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
                 slot0 = __shfl_sync(kFull, slot0, 0);
                 const long long slot = (long long)slot0 + (inc - n_eq);
                 for (int32_t j = 0; j < n_eq; ++j) {
-                    const unsigned long long key = __ldg(keys + p_hi + j);
+                    const unsigned long long key = __ldg(&HORA_AT(keys, p_hi + j, ld));
                     if (slot + j < kListCap) {
-                        cand_key[slot + j] = key;
-                        cand_row[slot + j] = (int32_t)row;
+                        HORA_AT(cand_key, slot + j, kListCap) = key;
+                        HORA_AT(cand_row, slot + j, kListCap) = (int32_t)row;
                     }
                     atomicAdd(hist1 + ((key >> shift) & digit_mask), 1ull);   // few keys: straight to global memory
                 }
@@ -879,7 +883,7 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
                 unsigned int slot0 = 0;
                 if (lane == 0) slot0 = atomicAdd(&hdr->n_active, (unsigned int)__popc(keep));
                 slot0 = __shfl_sync(kFull, slot0, 0);
-                if (n_eq > 0) active[slot0 + __popc(keep & ((1u << lane) - 1u))] = (int32_t)row;
+                if (n_eq > 0) HORA_AT(active, slot0 + __popc(keep & ((1u << lane) - 1u)), N) = (int32_t)row;
             }
         }
     }
@@ -895,10 +899,11 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
 // the output pass, the exclusive prefixes of (#keys > lambda, #keys == lambda) over blocks of 1024 prompts.
 
 // Close a row's segment with the finished threshold: keys above it, keys equal to it.
-__device__ __forceinline__ int2 close_segment(const unsigned long long *__restrict__ keys, int2 st, unsigned long long lam) {
+__device__ __forceinline__ int2 close_segment(const unsigned long long *__restrict__ keys, int2 st, unsigned long long lam,
+                                              int32_t ld) {
     int32_t n_gt = 0, n_eq = 0;
     for (int32_t pp = st.x; pp < st.y; ++pp) {
-        const unsigned long long key = __ldg(keys + pp);
+        const unsigned long long key = __ldg(&HORA_AT(keys, pp, ld));
         if (key > lam) ++n_gt;
         else if (key == lam) ++n_eq;
         else break;
@@ -957,7 +962,7 @@ __device__ void tail_list(int64_t B, AllocHeader *hdr, const unsigned long long 
                 const unsigned int i = i0 + u * kSelThreads + tid;
                 if (i < n_all && (key[u] << r0) >> (64 - known) == want) {
                     const unsigned int slot = atomicAdd(&s_fill, 1u);
-                    if (slot < (unsigned)kListSmall) s_keys[slot] = key[u];
+                    if (slot < (unsigned)kListSmall) HORA_AT(s_keys, slot, kListSmall) = key[u];
                 }
             }
         }
@@ -1053,8 +1058,8 @@ __device__ void tail_list(int64_t B, AllocHeader *hdr, const unsigned long long 
                 const unsigned int i = i0 + u * kSelThreads + tid;
                 const int64_t blk = (int64_t)row[u] / kRowsPerBlock - b0;
                 if (i < n_all && blk >= 0 && blk < n_here) {
-                    if (key[u] > prefix) atomicAdd(&s_fix_hi[blk], 1u);
-                    else if (key[u] == prefix) atomicAdd(&s_fix_t[blk], 1u);
+                    if (key[u] > prefix) atomicAdd(&HORA_AT(s_fix_hi, blk, kBins / 2), 1u);
+                    else if (key[u] == prefix) atomicAdd(&HORA_AT(s_fix_t, blk, kBins / 2), 1u);
                 }
             }
         }
@@ -1095,24 +1100,24 @@ __device__ void tail_digits(int64_t N, int32_t ld, const double *__restrict__ ga
         const unsigned long long d_prev = (unsigned long long)*(volatile int32_t *)&hdr->sel_digit[level - 1];
         const unsigned long long mask_cur = (unsigned long long)bins - 1ull;
         for (unsigned int idx = blockIdx.x * kSelThreads + threadIdx.x; idx < n_active; idx += stride) {
-            const int64_t row = active[idx];
+            const int64_t row = HORA_AT(active, idx, N);
             const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
-            const int2 st = __ldcg(rowstate + row);
+            const int2 st = __ldcg(&HORA_AT(rowstate, row, N));
             const int32_t p_hi = st.x, p_end = st.y;
             int32_t p = p_hi, new_hi = p_hi;
             while (p < p_end) {
-                const unsigned long long key = __ldg(keys + p);
+                const unsigned long long key = __ldg(&HORA_AT(keys, p, ld));
                 const unsigned long long dp = (key >> shift_prev) & mask_prev;
                 if (dp > d_prev) {
                     new_hi = p + 1;
                 } else if (dp == d_prev) {
-                    atomicAdd(&s_hist[(key >> shift) & mask_cur], 1u);
+                    atomicAdd(&HORA_AT(s_hist, (key >> shift) & mask_cur, kBins), 1u);
                 } else {
                     break;
                 }
                 ++p;
             }
-            if (new_hi != p_hi || p != p_end) rowstate[row] = make_int2(new_hi, p);
+            if (new_hi != p_hi || p != p_end) HORA_AT(rowstate, row, N) = make_int2(new_hi, p);
         }
         __syncthreads();
         flush_hist(s_hist, hist_all + (size_t)level * kBins, bins);
@@ -1133,7 +1138,7 @@ __device__ void tail_digits(int64_t N, int32_t ld, const double *__restrict__ ga
             if (row < N) {
                 int2 st = __ldcg(rowstate + row);
                 if (st.y > st.x) {
-                    const int2 fin = close_segment(reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld, st, lam);
+                    const int2 fin = close_segment(reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld, st, lam, ld);
                     if (fin.x != st.x || fin.y != st.y) rowstate[row] = fin;
                     st = fin;
                 }
@@ -1213,14 +1218,14 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
             else if (al + be + (double)G0 + (double)ld >= 1048576.0) err = err ? err : HORA_ERR_EXACT_RANGE;
             const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
             int2 st = rowstate[row];
-            if (list && st.y > st.x) st = close_segment(keys, st, lam_key);   // the list route leaves segments open
+            if (list && st.y > st.x) st = close_segment(keys, st, lam_key, ld);   // the list route leaves segments open
             q = st.x;                                         // #keys > lambda
-            if (q > 0 && __ldg(keys + q - 1) <= k_hi) {
+            if (q > 0 && __ldg(&HORA_AT(keys, q - 1, ld)) <= k_hi) {
                 --q;
-                if (q > 0 && __ldg(keys + q - 1) <= k_hi) err = err ? err : HORA_ERR_EXACT_RANGE;
+                if (q > 0 && __ldg(&HORA_AT(keys, q - 1, ld)) <= k_hi) err = err ? err : HORA_ERR_EXACT_RANGE;
             }
-            const bool has = (q < capi) && (__ldg(keys + q) >= k_lo);
-            if (has && q + 1 < capi && __ldg(keys + q + 1) >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
+            const bool has = (q < capi) && (__ldg(&HORA_AT(keys, q, ld)) >= k_lo);
+            if (has && q + 1 < capi && __ldg(&HORA_AT(keys, q + 1, ld)) >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
             if (has && !err)
                 tkey = pack_type((unsigned long long)al + ci, (unsigned long long)be + (G0 - ci), (unsigned long long)q + 1);
             above += q;
@@ -1233,7 +1238,7 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
             if (lane == leader) {
                 unsigned int h = (unsigned int)((tkey * 0x9E3779B97F4A7C15ull) >> 52) & (kTypeSlots - 1);
                 for (int probe = 0; probe < kTypeSlots; ++probe) {
-                    const unsigned long long old = atomicCAS(tkeys + h, 0ull, tkey);
+                    const unsigned long long old = atomicCAS(&HORA_AT(tkeys, h, kTypeSlots), 0ull, tkey);
                     if (old == 0ull || old == tkey) {
                         if (old == 0ull) atomicAdd(&hdr->n_types, 1u);
                         slot = (int32_t)h;
@@ -1241,7 +1246,7 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
                     }
                     h = (h + 1) & (kTypeSlots - 1);
                 }
-                if (slot >= 0) atomicAdd(tcounts + slot, (unsigned long long)__popc(peers));
+                if (slot >= 0) atomicAdd(&HORA_AT(tcounts, slot, kTypeSlots), (unsigned long long)__popc(peers));
                 else err = err ? err : HORA_ERR_EXACT_RANGE;
             }
             slot = __shfl_sync(peers, slot, leader);
@@ -1309,7 +1314,7 @@ exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ t
         int label = 0;
         if (above + equal < Rp) label = 2;
         else if (above < Rp) label = 1;
-        tlabel[s_slot[t]] = label;
+        HORA_AT(tlabel, s_slot[t], kTypeSlots) = label;
         if (label == 1) {
             // Members of the threshold class agree on R, but their unreduced num/den differ, and so may the
             // last bit of the quotient below: the member with the smallest packed type (a, b, Delta) alone
@@ -1356,7 +1361,7 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
             const int64_t row = row0 + q * kSelThreads + threadIdx.x;
             if (row < N) {
                 if (mode == 2) {
-                    const int label = slot[q] >= 0 ? tlabel[slot[q]] : 0;
+                    const int label = slot[q] >= 0 ? HORA_AT(tlabel, slot[q], kTypeSlots) : 0;
                     st[q] = make_int2(st[q].x + (label == 2), st[q].x + (label == 2) + (label == 1));
                     rowstate[row] = st[q];
                 }
@@ -1433,7 +1438,7 @@ select_out(const double *__restrict__ alpha, const double *__restrict__ beta, do
     for (int q = 0; q < kPer; ++q) {
         if (failed) st[q] = make_int2(0, 0);
         if (open && st[q].y > st[q].x)
-            st[q] = close_segment(reinterpret_cast<const unsigned long long *>(gains) + (row0 + q) * (int64_t)ld, st[q], lam_key);
+            st[q] = close_segment(reinterpret_cast<const unsigned long long *>(gains) + (row0 + q) * (int64_t)ld, st[q], lam_key, ld);
         hi[q] = st[q].x;
         tied[q] = st[q].y - st[q].x;
         hi_sum += hi[q];
@@ -1480,7 +1485,7 @@ select_out(const double *__restrict__ alpha, const double *__restrict__ beta, do
                 double u = o[q];
                 if (u < 0.0) {
                     const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, row0 + q);
-                    u = utility_from_gain(__ldg(gains + (row0 + q) * (int64_t)ld + (d[q] - 1)), p.a, p.b, d[q]);
+                    u = utility_from_gain(__ldg(&HORA_AT(gains, (row0 + q) * (int64_t)ld + (d[q] - 1), N * (int64_t)ld)), p.a, p.b, d[q]);
                 }
                 obj += u;
             }

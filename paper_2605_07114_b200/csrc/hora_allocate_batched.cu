@@ -6,7 +6,8 @@
 // and one CTA solves one segment entirely in shared memory:
 //   1  gain rows of the segment's prompts, computed with the arithmetic of hora_gains (same bits), never
 //      written to global memory;
-//   2  the B_s-th largest key by a radix selection over the shared-memory keys (11-bit digits);
+//   2  the B_s-th largest key, built bit by bit from the top by one warp: a step is a binary search per sorted
+//      row (inside a range that every step narrows) and one warp sum;
 //   3  per row the number of keys above and equal to the threshold (binary search in the sorted row);
 //   4  ties: in prompt order (fp64 equality), or, in exact mode, by exact rational comparison of the at
 //      most one candidate per row that lies within 2^-30 of the threshold (pairwise, cross-multiplied);
@@ -14,30 +15,29 @@
 // Group offsets over all prompts are an exclusive scan of G by two small kernels afterwards.
 #include <algorithm>
 
+#define HORA_FILE_ID 2
 #include "hora_block.cuh"
+#include "hora_checked.cuh"
 #include "hora_common.cuh"
 #include "hora_exact.cuh"
 #include "hora_gains_chunk.cuh"
 #include "hora_rank.cuh"
+
+HORA_CHECKED_REGISTER()
 
 namespace hora {
 
 constexpr int kBThreads = kSelThreads;        // the shared block helpers are written for this many threads
 constexpr int kBWarps = kBThreads / kWarp;
 constexpr int kBMaxRows = 256;                 // prompts per segment (one thread per prompt in the row phases)
-constexpr int kBBins = 2048;                   // 11-bit digits
 constexpr size_t kBMaxSmem = 200 * 1024;       // keys + bookkeeping must fit this
 constexpr int kScanRows = 1024;                // rows per CTA in the offsets scan
 
-constexpr int kBListCap = 256;                 // keys of the short list the late digit levels work on
-
 struct BatchedSmemFixed {
-    unsigned int hist[kBBins];
-    unsigned long long list[kBListCap];
+    unsigned long long lam_key;
     long long warp_tmp[kBWarps];
     double obj_tmp[kBWarps];
     long long found[3];
-    unsigned long long list_count;
     double lam_exact;
     int status;
 };
@@ -47,8 +47,10 @@ struct BatchedSmemFixed {
 struct BatchedRows {
     double *a, *b;
     int32_t *cap, *band;           // band: Delta of the row's near-threshold candidate (exact mode), 0 if it has none
+    int32_t *lo, *hi;              // selection: the row's count of keys >= the threshold lies in [lo, hi]
+    int32_t *cnt2, *cnt3;          // selection: the row's counts for the second and third trial value of a step
 };
-constexpr size_t kBRowBytes = 2 * sizeof(double) + 2 * sizeof(int32_t);   // 24 bytes per prompt
+constexpr size_t kBRowBytes = 2 * sizeof(double) + 6 * sizeof(int32_t);   // 40 bytes per prompt
 
 __device__ __forceinline__ BatchedRows carve_rows(unsigned char *base, int rows_cap) {
     BatchedRows r;
@@ -56,43 +58,15 @@ __device__ __forceinline__ BatchedRows carve_rows(unsigned char *base, int rows_
     r.b = r.a + rows_cap;
     r.cap = reinterpret_cast<int32_t *>(r.b + rows_cap);
     r.band = r.cap + rows_cap;
+    r.lo = r.band + rows_cap;
+    r.hi = r.lo + rows_cap;
+    r.cnt2 = r.hi + rows_cap;
+    r.cnt3 = r.cnt2 + rows_cap;
     return r;
 }
 
-// Scanning from the top bin down, the bin where the running count reaches `need` (1-based); the count of
-// the bins above it goes to *above_out.  All threads get the result.  -1 if need is out of range.
-__device__ int blocate_rank(BatchedSmemFixed &sm, int bins, long long need, long long *above_out) {
-    const int per = bins / kBThreads > 0 ? bins / kBThreads : 1;
-    const int top = bins - 1 - (int)threadIdx.x * per;
-    long long local = 0;
-    for (int j = 0; j < per; ++j)
-        if (top - j >= 0) local += sm.hist[top - j];
-    if (threadIdx.x == 0) sm.found[2] = 0;
-    long long total;
-    const long long above = block_exclusive_sum(local, &total, sm.warp_tmp);
-    if (need >= 1 && above < need && need <= above + local) {
-        long long run = above;
-        for (int j = 0; j < per && top - j >= 0; ++j) {
-            const long long cnt = sm.hist[top - j];
-            if (run + cnt >= need) {
-                sm.found[0] = top - j;
-                sm.found[1] = run;
-                sm.found[2] = 1;
-                break;
-            }
-            run += cnt;
-        }
-    }
-    __syncthreads();
-    const bool ok = sm.found[2] != 0;
-    const int digit = ok ? (int)sm.found[0] : -1;
-    *above_out = ok ? sm.found[1] : 0;
-    __syncthreads();
-    return digit;
-}
-
 template <int E>
-__global__ void __launch_bounds__(kBThreads)
+__global__ void __launch_bounds__(kBThreads, 3)
 allocate_batched_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
                         const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
                         int32_t ld, const int64_t *__restrict__ seg_off, const int64_t *__restrict__ budgets, int64_t S,
@@ -113,8 +87,10 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         if (threadIdx.x == 0) sm.status = (B < 0) ? HORA_ERR_INVALID_VALUE : HORA_OK;
         __syncthreads();
         // ---- 1: gain rows into shared memory (a warp per row) ----
+        Posterior nxt = warp < n ? load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, r0 + warp) : Posterior{};
         for (int r = warp; r < n; r += kBWarps) {
-            const Posterior p = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, r0 + r);
+            const Posterior p = nxt;                          // the next row's inputs are fetched while this row is built
+            if (r + kBWarps < n) nxt = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, r0 + r + kBWarps);
             if (!p.ok && lane == 0) sm.status = HORA_ERR_INVALID_VALUE;
             const double a = p.ok ? p.a : 1.0, b = p.ok ? p.b : 1.0;
             if (lane == 0) { rw.a[r] = a; rw.b[r] = b; rw.cap[r] = p.cap; }
@@ -128,63 +104,80 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         block_exclusive_sum(threadIdx.x < n ? rw.cap[threadIdx.x] : 0, &sum_cap, sm.warp_tmp);
         if (threadIdx.x == 0 && sm.status == HORA_OK && B > sum_cap) sm.status = HORA_ERR_INFEASIBLE;
         __syncthreads();
-        // ---- 2: the B-th largest key ----
-        unsigned long long prefix = 0;
-        long long need = B;
-        if (sm.status == HORA_OK && B > 0) {
-            // Levels 0 and 1 (top 22 bits) sweep the keys row by row (a warp per row, no index division);
-            // what still matches after them is a handful of keys, which are copied to a short list that the
-            // remaining levels work on (up to kBListCap keys; a longer list keeps sweeping).
-            unsigned long long *list = sm.list;
-            constexpr int kListCap = kBListCap;
-            int n_list = -1;                                       // -1: still sweeping the rows
-            for (int level = 0; level < 6; ++level) {             // 5 x 11 + 9 = 64 bits, from the top
-                const int w = level < 5 ? 11 : 9;
-                const int sh = level < 5 ? 53 - 11 * level : 0;
-                for (int t = threadIdx.x; t < kBBins; t += kBThreads) sm.hist[t] = 0;
-                __syncthreads();
-                if (n_list < 0) {
-                    for (int r = warp; r < n; r += kBWarps) {
-                        const unsigned long long *rk = keys + (size_t)r * ld;
-                        const int cp = rw.cap[r];
-                        for (int col = lane; col < cp; col += kWarp) {
-                            const unsigned long long key = rk[col];
-                            if (level == 0 || (key >> (sh + w)) == (prefix >> (sh + w)))
-                                atomicAdd(&sm.hist[(key >> sh) & ((1u << w) - 1u)], 1u);
-                        }
-                    }
-                } else {
-                    for (int i = threadIdx.x; i < n_list; i += kBThreads) {
-                        const unsigned long long key = list[i];
-                        if ((key >> (sh + w)) == (prefix >> (sh + w)))
-                            atomicAdd(&sm.hist[(key >> sh) & ((1u << w) - 1u)], 1u);
-                    }
+        // ---- 2: the B-th largest key, by warp 0 ----
+        // The key is built from its top bits down, two bits a step: with p the bits so far, the three trial values
+        // p | 1, p | 2, p | 3 (at the step's position) are counted at once — how many keys are >= each — and the
+        // largest one that still has B keys at or above it gives the two bits.  A lane owns rows lane, lane + 32,
+        // ...; a row is sorted, so a count is one binary search, and it can only move inside [lo, hi], which every
+        // step narrows from both sides: after a few steps a search is a probe or two.  The bits that all keys share
+        // (the sign, most of the exponent) are taken from the largest and the smallest key directly.  About thirty
+        // steps of (three searches in flight, three warp sums) replace six histogram sweeps over every key with
+        // block-wide barriers between them.
+        if (warp == 0 && sm.status == HORA_OK && B > 0) {
+            unsigned long long kmax = 0ull, kmin = ~0ull;
+            for (int r = lane; r < n; r += kWarp) {
+                const int cp = rw.cap[r];
+                rw.lo[r] = 0;
+                rw.hi[r] = cp;
+                if (cp > 0) {
+                    const unsigned long long first = keys[(size_t)r * ld], last_k = keys[(size_t)r * ld + cp - 1];
+                    kmax = first > kmax ? first : kmax;
+                    kmin = last_k < kmin ? last_k : kmin;
                 }
-                __syncthreads();
-                long long above;
-                const int digit = blocate_rank(sm, 1 << w, need, &above);
-                prefix |= (unsigned long long)(digit < 0 ? 0 : digit) << sh;
-                need -= above;
-                // after this level: how many keys still match?  (the selected bin's count)
-                const long long left = digit < 0 ? 0 : (long long)sm.hist[digit];
-                if (n_list < 0 && level >= 1 && level < 5 && left <= kListCap) {
-                    if (threadIdx.x == 0) sm.list_count = 0;
-                    __syncthreads();
-                    for (int r = warp; r < n; r += kBWarps) {
-                        const unsigned long long *rk = keys + (size_t)r * ld;
-                        const int cp = rw.cap[r];
-                        for (int col = lane; col < cp; col += kWarp) {
-                            const unsigned long long key = rk[col];
-                            if ((key >> sh) == (prefix >> sh)) list[atomicAdd(&sm.list_count, 1ull)] = key;
-                        }
-                    }
-                    __syncthreads();
-                    n_list = (int)sm.list_count;
-                }
-                __syncthreads();
             }
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) {
+                const unsigned long long a = __shfl_xor_sync(kFull, kmax, d), z = __shfl_xor_sync(kFull, kmin, d);
+                kmax = a > kmax ? a : kmax;
+                kmin = z < kmin ? z : kmin;
+            }
+            // bits above `top` are the same in every key (B <= the number of keys, so the threshold is one of them)
+            int top = 63 - __clzll((long long)((kmax ^ kmin) | 1ull));
+            top |= 1;                                          // steps take bits (top, top - 1), ..., (1, 0)
+            unsigned long long prefix = top >= 63 ? 0ull : (kmax >> (top + 1)) << (top + 1);
+#pragma unroll 1
+            for (int bit = top; bit >= 1; bit -= 2) {
+                const unsigned long long t1 = prefix | (1ull << (bit - 1)), t2 = prefix | (2ull << (bit - 1)),
+                                         t3 = prefix | (3ull << (bit - 1));
+                int c1 = 0, c2 = 0, c3 = 0;
+#pragma unroll 1
+                for (int r = lane; r < n; r += kWarp) {
+                    const unsigned long long *rk = keys + (size_t)r * ld;
+                    const int lo = rw.lo[r], hi = rw.hi[r];
+                    int a1 = lo, z1 = hi, a2 = lo, z2 = hi, a3 = lo, z3 = hi;   // first position whose key is below t_k
+                    while (a1 < z1 || a2 < z2 || a3 < z3) {
+                        const int m1 = (a1 + z1) >> 1, m2 = (a2 + z2) >> 1, m3 = (a3 + z3) >> 1;
+                        const unsigned long long k1 = HORA_AT(rk, m1 < hi ? m1 : lo, ld), k2 = HORA_AT(rk, m2 < hi ? m2 : lo, ld),
+                                                 k3 = HORA_AT(rk, m3 < hi ? m3 : lo, ld);
+                        if (a1 < z1) { if (k1 >= t1) a1 = m1 + 1; else z1 = m1; }
+                        if (a2 < z2) { if (k2 >= t2) a2 = m2 + 1; else z2 = m2; }
+                        if (a3 < z3) { if (k3 >= t3) a3 = m3 + 1; else z3 = m3; }
+                    }
+                    c1 += a1; c2 += a2; c3 += a3;
+                    rw.band[r] = a1;                           // (scratch until the tie step)
+                    rw.cnt2[r] = a2;
+                    rw.cnt3[r] = a3;
+                }
+                c1 = __reduce_add_sync(kFull, c1);            // at most 22528 keys in a segment
+                c2 = __reduce_add_sync(kFull, c2);
+                c3 = __reduce_add_sync(kFull, c3);
+                // counts decrease with the trial value: take the largest trial that still has B keys at or above it
+                const int pick = (long long)c3 >= B ? 3 : ((long long)c2 >= B ? 2 : ((long long)c1 >= B ? 1 : 0));
+                prefix |= (unsigned long long)pick << (bit - 1);
+#pragma unroll 1
+                for (int r = lane; r < n; r += kWarp) {
+                    const int a1 = rw.band[r], a2 = rw.cnt2[r], a3 = rw.cnt3[r];
+                    // #keys >= threshold lies between the count of the next larger trial and that of the picked one
+                    if (pick == 3) rw.hi[r] = a3;
+                    else if (pick == 2) { rw.lo[r] = a3; rw.hi[r] = a2; }
+                    else if (pick == 1) { rw.lo[r] = a2; rw.hi[r] = a1; }
+                    else rw.lo[r] = a1;
+                }
+            }
+            if (lane == 0) sm.lam_key = prefix;
         }
         __syncthreads();
+        const unsigned long long prefix = sm.lam_key;
         const unsigned long long lam_key = prefix;
         // ---- 3: per row, keys above and equal to the threshold ----
         int my_hi = 0, my_tied = 0, my_cap = 0;
@@ -194,10 +187,10 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
             int lo = 0, hi = my_cap;
             while (lo < hi) {
                 const int mid = (lo + hi) >> 1;
-                if (row[mid] > lam_key) lo = mid + 1; else hi = mid;
+                if (HORA_AT(row, mid, ld) > lam_key) lo = mid + 1; else hi = mid;
             }
             my_hi = lo;
-            while (my_hi + my_tied < my_cap && row[my_hi + my_tied] == lam_key) ++my_tied;
+            while (my_hi + my_tied < my_cap && HORA_AT(row, my_hi + my_tied, ld) == lam_key) ++my_tied;
         }
         // ---- 4: ties ----
         int my_delta = 0;
@@ -223,12 +216,12 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                 const double be = beta ? __ldg(beta + r0 + threadIdx.x) : beta0;
                 if (!(al >= 1.0 && be >= 1.0 && al == floor(al) && be == floor(be))) err = HORA_ERR_NOT_INTEGER;
                 else if (al + be + (double)G0 + (double)ld >= 1048576.0) err = HORA_ERR_EXACT_RANGE;
-                if (q > 0 && row[q - 1] <= k_hi) {
+                if (q > 0 && HORA_AT(row, q - 1, ld) <= k_hi) {
                     --q;
-                    if (q > 0 && row[q - 1] <= k_hi) err = err ? err : HORA_ERR_EXACT_RANGE;
+                    if (q > 0 && HORA_AT(row, q - 1, ld) <= k_hi) err = err ? err : HORA_ERR_EXACT_RANGE;
                 }
-                has = (q < my_cap) && (row[q] >= k_lo);
-                if (has && q + 1 < my_cap && row[q + 1] >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
+                has = (q < my_cap) && (HORA_AT(row, q, ld) >= k_lo);
+                if (has && q + 1 < my_cap && HORA_AT(row, q + 1, ld) >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
                 if (err) atomicCAS(&sm.status, 0, err);
             }
             if ((int)threadIdx.x < rows_cap) rw.band[threadIdx.x] = (threadIdx.x < n && has && !err) ? q + 1 : 0;
@@ -259,8 +252,8 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                     sm.found[0] = tot_q + strictly;
                     sm.found[1] = equal + 1;
                     sm.found[2] = Rp - strictly;
-                    UBig nu, de;
-                    if (exact_gain(a_t, b_t, D_t, nu, de)) sm.lam_exact = ratio_double(nu, de);
+                    double lam_x = 0.0;
+                    if (exact_gain_as_double(a_t, b_t, D_t, &lam_x)) sm.lam_exact = lam_x;
                     else atomicCAS(&sm.status, 0, (int)HORA_ERR_EXACT_RANGE);
                 }
             } else {
@@ -285,7 +278,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         // is g_i(Delta) (b + Delta - 1) / a  (Eq. marginal); the product loop itself took up to Delta iterations of
         // the slowest lane
         if (!failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE) && threadIdx.x < n && my_delta > 0)
-            obj = 1.0 - __longlong_as_double((long long)row[my_delta - 1]) *
+            obj = 1.0 - __longlong_as_double((long long)HORA_AT(row, my_delta - 1, ld)) *
                             (rw.b[threadIdx.x] + (double)(my_delta - 1)) / rw.a[threadIdx.x];
 #pragma unroll
         for (int d = 16; d >= 1; d >>= 1) obj += __shfl_xor_sync(kFull, obj, d);

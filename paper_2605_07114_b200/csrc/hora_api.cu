@@ -20,6 +20,31 @@ int sm_count() {
 }
 }  // namespace hora
 
+#ifdef HORA_CHECKED
+namespace hora {
+constexpr int kMaxCheckedUnits = 16;
+static unsigned (*g_check_fetch[kMaxCheckedUnits])();
+static int g_check_units = 0;
+void register_check_word(unsigned (*fetch_and_clear)()) {
+    if (g_check_units < kMaxCheckedUnits) g_check_fetch[g_check_units++] = fetch_and_clear;
+}
+}  // namespace hora
+#endif
+
+extern "C" int32_t hora_checked_violation(void) {
+#ifdef HORA_CHECKED
+    if (cudaDeviceSynchronize() != cudaSuccess) return -2;
+    int32_t first = 0;
+    for (int k = 0; k < hora::g_check_units; ++k) {
+        const unsigned v = hora::g_check_fetch[k]();          // reads and clears every unit's word
+        if (v != 0u && first == 0) first = (int32_t)v;
+    }
+    return first;
+#else
+    return -1;
+#endif
+}
+
 extern "C" const char *hora_status_string(hora_status_t status) {
     switch (status) {
         case HORA_OK: return "ok";

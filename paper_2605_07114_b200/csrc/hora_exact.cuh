@@ -119,6 +119,16 @@ __device__ __forceinline__ double to_double(const UBig &x) {
 // num/den as a double (2^512 is far inside the range of a double; a handful of roundings, reporting only)
 __device__ __forceinline__ double ratio_double(const UBig &num, const UBig &den) { return to_double(num) / to_double(den); }
 
+// g_{a,b}(Delta) as the double nearest its exact fraction (reporting only); false if the fraction does not fit.
+// Kept out of line: the callers are large kernels that need it once per problem.
+static __device__ __noinline__ bool exact_gain_as_double(unsigned long long a, unsigned long long b, unsigned long long Delta,
+                                                         double *out) {
+    UBig nu, de;
+    if (!exact_gain(a, b, Delta, nu, de)) return false;
+    *out = ratio_double(nu, de);
+    return true;
+}
+
 // U(Delta) = 1 - prod_{j<Delta} (b+j)/(a+b+j)  (Eq. appendix-hit-closed-form written as a product)
 __device__ __forceinline__ double hit_utility(double a, double b, int32_t Delta) {
     double q = 1.0, num = 1.0, den = 1.0;

@@ -25,10 +25,14 @@
 // one step costs one lookup per prompt and one warp reduction.
 #include <cmath>
 
+#define HORA_FILE_ID 4
 #include "hora_block.cuh"
+#include "hora_checked.cuh"
 #include "hora_exact.cuh"
 #include "hora_gains_chunk.cuh"
 #include "hora_rank.cuh"
+
+HORA_CHECKED_REGISTER()
 
 namespace hora {
 
@@ -135,7 +139,7 @@ rank_table_kernel(double alpha0, double beta0, int32_t G0, int32_t ld, RankTable
     if (overflow) raise_status(status, HORA_ERR_EXACT_RANGE);
     t.rank[id] = rank;
     t.gain[id] = g0;
-    if (first_of_class) t.lam[rank] = g0;
+    if (first_of_class) HORA_AT(t.lam, rank, T) = g0;
     t.util[(size_t)c * (ld + 1) + j + 1] = utility_from_gain(g0, alpha0 + (double)c, beta0 + (double)(G0 - c), j + 1);
     if (j == 0) t.util[(size_t)c * (ld + 1)] = 0.0;
 }
@@ -279,12 +283,12 @@ __device__ __forceinline__ void rank_load_quad(RankQuad &q, const int32_t *__res
 }
 
 // (candidates above the threshold, tied candidate) of a prompt from its class entry; zeros for a missing prompt
-__device__ __forceinline__ void rank_row_state(int32_t ci, int32_t cp, const int32_t *s_class, int tiers, int *hi,
-                                               int *tied) {
+__device__ __forceinline__ void rank_row_state(int32_t ci, int32_t cp, const int32_t *s_class, int n_class, int tiers,
+                                               int *hi, int *tied) {
     *hi = 0;
     *tied = 0;
     if (ci < 0) return;
-    const int e = s_class[tiers ? (ci > 0) : ci], above = e >> 1;   // tiers: two classes only, c = 0 and c > 0
+    const int e = HORA_AT(s_class, tiers ? (ci > 0) : ci, n_class), above = e >> 1;   // tiers: two classes only, c = 0 and c > 0
     *hi = cp < above ? cp : above;
     *tied = (e & 1) && cp > above;
 }
@@ -377,9 +381,9 @@ rank_count_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__re
             }
             if (few_bins) {                                  // (the match costs more than it saves on a wide table)
                 const unsigned peers = __match_any_sync(kFull, bin);
-                if (bin >= 0 && lane == __ffs(peers) - 1) atomicAdd(&s_hist[bin], (unsigned)__popc(peers));
+                if (bin >= 0 && lane == __ffs(peers) - 1) atomicAdd(&HORA_AT(s_hist, bin, n_h), (unsigned)__popc(peers));
             } else if (bin >= 0) {
-                atomicAdd(&s_hist[bin], 1u);
+                atomicAdd(&HORA_AT(s_hist, bin, n_h), 1u);
             }
         }
     };
@@ -432,7 +436,7 @@ rank_count_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__re
                 if (lane >= d) inc += x;
             }
             const long long cnt = carry + inc;
-            if (D >= 1 && cnt > 0) atomicAdd(w.bucket + (w.bins - 1 - __ldg(rrow + D - 1)), (unsigned long long)cnt);
+            if (D >= 1 && cnt > 0) atomicAdd(&HORA_AT(w.bucket, w.bins - 1 - __ldg(rrow + D - 1), w.bins), (unsigned long long)cnt);
             carry += __shfl_sync(kFull, inc, kWarp - 1);
         }
     }
@@ -494,12 +498,12 @@ rank_count_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__re
 
 // The prompts are cut into tasks of kRankTask; CTA k owns the contiguous tasks [k m, (k+1) m) and its warps take
 // them in turn.  A lane holds 4 consecutive prompts of each 128 (two 16-byte loads), so a task is two steps.
-__device__ __forceinline__ void rank_task_state(const RankQuad (&q)[2], const int32_t *s_class, int tiers,
+__device__ __forceinline__ void rank_task_state(const RankQuad (&q)[2], const int32_t *s_class, int n_class, int tiers,
                                                 int (&hi)[2][4], int (&tied)[2][4]) {
 #pragma unroll
     for (int h = 0; h < 2; ++h)
 #pragma unroll
-        for (int k = 0; k < 4; ++k) rank_row_state(q[h].c[k], q[h].cap[k], s_class, tiers, &hi[h][k], &tied[h][k]);
+        for (int k = 0; k < 4; ++k) rank_row_state(q[h].c[k], q[h].cap[k], s_class, n_class, tiers, &hi[h][k], &tied[h][k]);
 }
 
 // Sums of (above, tied) per task and per CTA.  No barrier inside the loop, no ticket at the end.
@@ -520,7 +524,7 @@ rank_sums_kernel(const int32_t *__restrict__ c, int32_t n_class, int tiers, cons
         rank_load_quad(q[0], c, cap, cap_scalar, t * kRankTask + lane * 4, N, vec != 0);
         rank_load_quad(q[1], c, cap, cap_scalar, t * kRankTask + 128 + lane * 4, N, vec != 0);
         int hi[2][4], tied[2][4], hs = 0, ts = 0;
-        rank_task_state(q, s_class, tiers, hi, tied);
+        rank_task_state(q, s_class, n_class, tiers, hi, tied);
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -594,7 +598,7 @@ rank_out_kernel(const int32_t *__restrict__ c, int32_t G0, int32_t n_class, int 
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     hi[k] = tied[k] = 0;
-                    if (!failed) rank_row_state(q[h].c[k], q[h].cap[k], s_class, tiers, &hi[k], &tied[k]);
+                    if (!failed) rank_row_state(q[h].c[k], q[h].cap[k], s_class, n_class, tiers, &hi[k], &tied[k]);
                 }
                 const int hs = hi[0] + hi[1] + hi[2] + hi[3], ts = tied[0] + tied[1] + tied[2] + tied[3];
                 // exclusive prefix over the lanes of (above, tied), packed: tied <= 4 per lane, 128 per step;
@@ -746,14 +750,14 @@ rank_batched_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__
         // candidates of the segment whose rank is below r: sum_i min(cap_i, pos[c_i][r])
         auto count_below = [&](int r) -> long long {
             if (small) {
-                const int p = (int)__ldg(t.pos + (size_t)my_c * (T + 1) + r);
+                const int p = (int)__ldg(&HORA_AT(t.pos, (size_t)my_c * (T + 1) + r, (size_t)(G0 + 1) * (T + 1)));
                 return (long long)__reduce_add_sync(kFull, p < my_cap ? p : my_cap);
             }
             long long part = 0;
             for (int64_t i = lane; i < n; i += kWarp) {
                 const int ci = __ldg(c + r0 + i);
                 const int cp = cap ? __ldg(cap + r0 + i) : cap_scalar;
-                const int p = (int)__ldg(t.pos + (size_t)ci * (T + 1) + r);
+                const int p = (int)__ldg(&HORA_AT(t.pos, (size_t)ci * (T + 1) + r, (size_t)(G0 + 1) * (T + 1)));
                 part += p < cp ? p : cp;
             }
 #pragma unroll
@@ -796,7 +800,8 @@ rank_batched_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__
             if (i < n) {
                 delta[r0 + i] = status ? 0 : d_i;
                 G[r0 + i] = status ? 0 : G0 + d_i;
-                if (!status && !(flags & HORA_FLAG_SKIP_OBJECTIVE)) obj += __ldg(t.util + (size_t)ci * (ld + 1) + d_i);
+                if (!status && !(flags & HORA_FLAG_SKIP_OBJECTIVE))
+                    obj += __ldg(&HORA_AT(t.util, (size_t)ci * (ld + 1) + d_i, (size_t)(G0 + 1) * (ld + 1)));
             }
             pre_t += __popc(tmask);
         }

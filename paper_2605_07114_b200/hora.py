@@ -30,7 +30,7 @@ EXPORTS = ("hora_gains", "hora_allocate_workspace_bytes", "hora_allocate", "hora
            "hora_allocate_batched", "hora_allocate_batched_workspace_bytes", "hora_rollout_weights",
            "hora_learned_prior", "hora_beta_binomial_nll", "hora_pass_at_k", "hora_pass_at_k_workspace_bytes",
            "hora_group_advantage_tokens", "hora_allocation_share", "hora_allocate_hard_first",
-           "hora_allocate_hard_first_workspace_bytes", "hora_fp64_probe")
+           "hora_allocate_hard_first_workspace_bytes", "hora_fp64_probe", "hora_checked_violation")
 
 
 class HoraError(RuntimeError):
@@ -49,14 +49,25 @@ INFO_BYTES = C.sizeof(hora_alloc_info)
 _lib = None
 
 
+def use_library(path: Optional[str]) -> None:
+    """Bind the module to another build of the same library (e.g. the checked one), or back to the default (None).
+    Takes effect at the next call."""
+    global _lib, _lib_path
+    _lib = None
+    _lib_path = path or LIB_PATH
+
+
+_lib_path = LIB_PATH
+
+
 def load() -> C.CDLL:
     """Load the CUDA library built in-tree.  Raises if it is not there: nothing else can do its work."""
     global _lib
     if _lib is not None:
         return _lib
-    if not os.path.exists(LIB_PATH):
-        raise FileNotFoundError(f"{LIB_PATH} not found: build it with `python -m paper_2605_07114_b200.build`")
-    L = C.CDLL(LIB_PATH)
+    if not os.path.exists(_lib_path):
+        raise FileNotFoundError(f"{_lib_path} not found: build it with `python -m paper_2605_07114_b200.build`")
+    L = C.CDLL(_lib_path)
     p, i32, i64, f64, u32 = C.c_void_p, C.c_int32, C.c_int64, C.c_double, C.c_uint32
     L.hora_gains.argtypes = [p, p, f64, f64, p, i32, p, i32, i64, i32, p, p, p]
     L.hora_gains.restype = C.c_int
@@ -98,6 +109,7 @@ def load() -> C.CDLL:
     L.hora_rollout_weights.restype = C.c_int
     L.hora_token_broadcast.argtypes = [p, p, i64, i64, p, p]
     L.hora_token_broadcast.restype = C.c_int
+    L.hora_checked_violation.restype = C.c_int32
     L.hora_fp64_probe.argtypes = [i32, p, p]
     L.hora_fp64_probe.restype = C.c_uint64
     L.hora_status_string.argtypes = [C.c_int]
@@ -211,6 +223,12 @@ def read_infos(info_dev: torch.Tensor, S: int):
         out.append(AllocInfo(x.status, x.first_pass_bits, x.lambda_, x.n_above, x.n_tied, x.n_tied_taken, x.objective,
                              x.sum_G, x.sum_cap))
     return out
+
+
+def hora_checked_violation() -> int:
+    """0: no index check failed since the last call; > 0: (file id << 20) | line of the first failure; -1: this is
+    not the checked build."""
+    return int(load().hora_checked_violation())
 
 
 def hora_fp64_probe(iters, sink_dev) -> int:

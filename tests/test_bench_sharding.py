@@ -56,7 +56,11 @@ def test_reference_arm_runs_on_rank_zero_only():
 def test_reference_sample_size_is_bounded():
     sys.path.insert(0, ROOT)
     import bench
-    for steps, warm in ((1, 0), (20, 5), (200, 10), (5000, 10)):
-        n = bench.reference_sample_size(steps, warm, 1 << 20)
-        assert 1024 <= n <= 1 << 19 and n & (n - 1) == 0
-        assert n * (steps + warm) <= 5.0e6 or n == 1024
+    N = 1 << 20
+    for steps, warm in ((1, 0), (5, 2), (20, 5), (200, 10), (5000, 10)):
+        n, why = bench.reference_sample_size(steps, warm, N)
+        assert 1024 <= n <= N and n & (n - 1) == 0 and why
+        # the whole run stays within the CPU time allowed for this arm (or sits at the floor of 1024 prompts)
+        assert n * (steps + warm) * bench.ORACLE_US_PER_PROMPT * 1e-6 <= bench.REFERENCE_CPU_SECONDS or n == 1024
+    # few enough steps: every step is the whole workload, the same one the repository's arm times
+    assert bench.reference_sample_size(5, 2, N)[0] == N
