@@ -177,7 +177,9 @@ hora_status_t hora_allocate(const double *alpha, const double *beta, double alph
  *   - Size limit: hora_allocate_workspace_bytes(N, ld, gains == NULL, flags) must not exceed
  *     hora_allocate_static_capacity(); otherwise HORA_ERR_WORKSPACE is returned and nothing is enqueued.
  *     With a materialised gains matrix that admits about 2.5e5 prompts; with gains == NULL the
- *     matrix itself must fit, so only small problems (N*ld*8 bytes well under 8 MiB) qualify.
+ *     matrix itself must fit, so only small problems (N*ld*8 bytes well under 8 MiB) qualify — except on the
+ *     rank-based route (one integer prior, HORA_FLAG_EXACT_INT, gains == NULL), which builds no matrix: pass
+ *     HORA_FLAG_SHARED_INT_PRIOR as well and the need is about 0.6 MiB + 8 bytes per 256 prompts.
  *   - First use: the first call on each device looks up the array's device address (cudaGetSymbolAddress)
  *     with that device current, and caches it (as hora_allocate caches, per device, how many thread blocks of
  *     its cooperative kernel fit at once).  Make that first call outside any stream capture.  The cached

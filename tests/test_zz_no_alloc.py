@@ -58,6 +58,35 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
     _run_both(wl.make("cfg1"), B=777)          # and back to the first shape with another budget
 
 
+def test_static_scratch_serves_the_rank_route_at_sizes_no_matrix_would_fit():
+    """One integer prior, exact ties, no matrix: the route that builds none needs well under the built-in 8 MiB even
+    for 2^18 prompts (a matrix of that problem would take 128 MiB).  Twice in a row, against the workspace call."""
+    from paper_2605_07114_b200 import hora
+    dev = "cuda"
+    flags = hora.FLAG_EXACT_INT | hora.FLAG_SHARED_INT_PRIOR
+    for N, B_per in ((1 << 18, 3), (100_001, 2)):
+        w = wl.make("cfg5", N)
+        c, cap = torch.from_numpy(w.c).to(dev), torch.from_numpy(w.cap).to(dev)
+        assert hora.hora_allocate_workspace_bytes(N, w.ld, True, flags) <= hora.hora_allocate_static_capacity()
+        res = []
+        for static in (False, True):
+            d = torch.full((N,), -1, dtype=torch.int32, device=dev)
+            G = torch.full((N,), -1, dtype=torch.int32, device=dev)
+            off = torch.full((N + 1,), -1, dtype=torch.int64, device=dev)
+            info = torch.zeros(hora.INFO_BYTES, dtype=torch.uint8, device=dev)
+            if static:
+                hora.hora_allocate_static(None, None, 1.0, 1.0, c, w.G0, cap, 0, N, w.ld, None, B_per * N, flags, d, G, off, info)
+            else:
+                ws = torch.empty(hora.hora_allocate_workspace_bytes(N, w.ld, True, flags), dtype=torch.uint8, device=dev)
+                hora.hora_allocate(None, None, 1.0, 1.0, c, w.G0, cap, 0, N, w.ld, None, B_per * N, flags, d, G, off, info, ws)
+            torch.cuda.synchronize()
+            res.append((d, G, off, hora.read_info(info)))
+        (d0, G0_, off0, a), (d1, G1, off1, b) = res
+        assert a.status == 0 and b.status == 0 and a.first_pass_bits == -1 and b.first_pass_bits == -1
+        assert torch.equal(d0, d1) and torch.equal(G0_, G1) and torch.equal(off0, off1) and int(d1.sum()) == B_per * N
+        assert (a.n_above, a.n_tied, a.n_tied_taken, a.lambda_, a.objective) == (b.n_above, b.n_tied, b.n_tied_taken, b.lambda_, b.objective)
+
+
 def test_static_scratch_rejects_problems_beyond_its_capacity():
     from paper_2605_07114_b200 import hora
     N, ld = 1 << 20, 256
