@@ -42,6 +42,10 @@
 // by cross multiplication in 1024-bit integers of num/den = a (b)_a / (b+Delta-1)_{a+1}  (or the equivalent
 // a (b)_{Delta-1} / (a+b)_Delta when that has fewer factors), and the threshold class is found by
 // walking the ranked types.  Rows are relabelled above / tied / below and the same sum/out steps run.
+//
+// One integer prior for all prompts, exact ties, no matrix given: none of the above runs.  The at most
+// (G0 + 1) * ld distinct candidate values are ranked once and the selection works on ranks and on counts of
+// (c_i, cap_i): hora_rank.cu.
 #include <cooperative_groups.h>
 
 #include <atomic>
