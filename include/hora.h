@@ -58,9 +58,10 @@ typedef enum hora_status {
 enum {
     HORA_FLAG_EXACT_INT = 1u,      /* priors are integer-valued: decide ties by exact rational equality */
     HORA_FLAG_SKIP_OBJECTIVE = 2u, /* do not compute hora_alloc_info.objective (left 0) */
-    HORA_FLAG_SHARED_INT_PRIOR = 4u /* sizing hint for hora_allocate_workspace_bytes: the call will pass alpha == beta ==
-                                      NULL with integer alpha0, beta0, HORA_FLAG_EXACT_INT and gains == NULL (see the
-                                      rank-based route under hora_allocate); ignored by the calls themselves */
+    HORA_FLAG_SHARED_PRIOR = 4u,   /* sizing hint for hora_allocate_workspace_bytes: the call will pass alpha == beta ==
+                                      NULL and gains == NULL (see the rank-based route under hora_allocate); ignored
+                                      by the calls themselves */
+    HORA_FLAG_SHARED_INT_PRIOR = 4u /* the same flag under the name of its first use (an integer prior, exact ties) */
 };
 
 enum { HORA_ADV_GRPO = 0, HORA_ADV_RLOO = 1 };
@@ -130,13 +131,16 @@ hora_status_t hora_gains(const double *alpha, const double *beta, double alpha0,
  * alpha_i + beta_i <= 16), or any a_i at all up to Delta = 25.  Only candidates near the threshold are ever
  * formed exactly; one that does not fit raises HORA_ERR_EXACT_RANGE (nothing wraps).
  *
- * Rank-based route.  With ONE integer prior for all prompts (alpha == beta == NULL, alpha0 and beta0 positive
- * integers), HORA_FLAG_EXACT_INT and gains == NULL there are only G0 + 1 posteriors and at most (G0 + 1) * ld distinct
- * candidate values.  When (G0 + 1) * ld <= 8192 the call ranks those values once, exactly, counts the prompts per
- * (c_i, cap_i) in one pass and selects on integer ranks: no matrix is built, 8 bytes are read per prompt per pass
- * (three passes), and the result is exact greedy by construction.  The workspace this route needs is small and
- * independent of ld: pass HORA_FLAG_SHARED_INT_PRIOR to hora_allocate_workspace_bytes to size for it (a workspace
- * sized without that flag is always large enough).  info_dev->lambda is then the fp64 gain of the threshold type.
+ * Rank-based route.  With ONE prior for all prompts (alpha == beta == NULL) and gains == NULL there are only G0 + 1
+ * posteriors and at most (G0 + 1) * ld distinct candidate values.  When (G0 + 1) * ld <= 8192 (and alpha0 + beta0 +
+ * G0 + ld < 2^20) the call ranks those values once, counts the prompts per (c_i, cap_i) in one pass and selects on
+ * integer ranks: no matrix is built, 8 bytes are read per prompt per pass (three passes).  With HORA_FLAG_EXACT_INT
+ * (alpha0, beta0 positive integers whose exact forms fit 512 bits) the ranking is exact and the result is exact
+ * greedy by construction; without the flag the values are ranked as the doubles hora_gains would write, equal
+ * doubles tie, and the result is what the key-based selection gives on that matrix.  The workspace this route
+ * needs is small and independent of ld: pass HORA_FLAG_SHARED_PRIOR to hora_allocate_workspace_bytes to size for
+ * it (a workspace sized without that flag is always large enough).  info_dev->lambda is then the fp64 gain of the
+ * threshold type.
  *
  *   alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld   as for hora_gains
  *   gains            [N*ld] the matrix hora_gains wrote for the same inputs, or NULL to have it built
@@ -178,8 +182,8 @@ hora_status_t hora_allocate(const double *alpha, const double *beta, double alph
  *     hora_allocate_static_capacity(); otherwise HORA_ERR_WORKSPACE is returned and nothing is enqueued.
  *     With a materialised gains matrix that admits about 2.5e5 prompts; with gains == NULL the
  *     matrix itself must fit, so only small problems (N*ld*8 bytes well under 8 MiB) qualify — except on the
- *     rank-based route (one integer prior, HORA_FLAG_EXACT_INT, gains == NULL), which builds no matrix: pass
- *     HORA_FLAG_SHARED_INT_PRIOR as well and the need is about 0.6 MiB + 8 bytes per 256 prompts.
+ *     rank-based route (one prior for all prompts, gains == NULL), which builds no matrix: pass
+ *     HORA_FLAG_SHARED_PRIOR as well and the need is about 0.6 MiB + 8 bytes per 256 prompts.
  *   - First use: the first call on each device looks up the array's device address (cudaGetSymbolAddress)
  *     with that device current, and caches it (as hora_allocate caches, per device, how many thread blocks of
  *     its cooperative kernel fit at once).  Make that first call outside any stream capture.  The cached
@@ -230,7 +234,8 @@ hora_status_t hora_allocate_hard_first(const int32_t *c, int32_t G0, const int32
  *
  * Segment s covers prompts seg_offsets_host[s] .. seg_offsets_host[s+1]-1 and hands out budgets_host[s]
  * rollouts among them, exactly as hora_allocate would on that segment alone (same gains bit for bit, same tie
- * rules, same exact mode).  One CTA solves one segment in shared memory; no gains matrix is materialised.
+ * rules, same exact mode).  One CTA solves one segment in shared memory (one warp on precomputed ranks when the
+ * prior is shared); no gains matrix is materialised.
  *
  *   alpha .. ld            as for hora_gains (device arrays over all N prompts)
  *   seg_offsets_host       HOST array [S+1], non-decreasing, [0] == 0, [S] == N
@@ -241,7 +246,10 @@ hora_status_t hora_allocate_hard_first(const int32_t *c, int32_t G0, const int32
  *                          delta / G are zero, other segments are unaffected
  *   workspace              device scratch, 256-byte aligned, hora_allocate_batched_workspace_bytes(N, S)
  * Limits: a segment may hold at most 256 prompts and 176 KiB of keys (prompts * ld * 8 bytes); beyond that the
- * call returns HORA_ERR_WORKSPACE and hora_allocate should be used for that problem.  The two host arrays are
+ * call returns HORA_ERR_WORKSPACE and hora_allocate should be used for that problem.  With ONE prior for all
+ * prompts (alpha == beta == NULL) and (G0 + 1) * ld <= 8192 neither limit applies: the candidate values are ranked
+ * once for all segments (as under hora_allocate's rank-based route, exactly or as doubles by the tie mode) and
+ * every segment is solved on ranks by one warp, whatever its size.  The two host arrays are
  * copied to the device during the call and may be reused as soon as it returns.
  */
 size_t hora_allocate_batched_workspace_bytes(int64_t N, int64_t S);

@@ -43,7 +43,7 @@
 // a (b)_{Delta-1} / (a+b)_Delta when that has fewer factors), and the threshold class is found by
 // walking the ranked types.  Rows are relabelled above / tied / below and the same sum/out steps run.
 //
-// One integer prior for all prompts, exact ties, no matrix given: none of the above runs.  The at most
+// One prior for all prompts and no matrix given: none of the above runs.  The at most
 // (G0 + 1) * ld distinct candidate values are ranked once and the selection works on ranks and on counts of
 // (c_i, cap_i): hora_rank.cu.
 #include <cooperative_groups.h>
@@ -1627,7 +1627,7 @@ extern "C" size_t hora_allocate_workspace_bytes(int64_t N, int32_t ld, int32_t g
     if (N < 0 || ld < 1) return 0;
     // the caller promises a shared integer prior, exact ties and no matrix: the rank-based route, which needs
     // neither the matrix nor anything per candidate
-    if ((flags & HORA_FLAG_SHARED_INT_PRIOR) && (flags & HORA_FLAG_EXACT_INT) && gains_is_null != 0)
+    if ((flags & HORA_FLAG_SHARED_PRIOR) && gains_is_null != 0)
         return hora::rank_allocate_workspace_bound(N);
     return hora::carve(nullptr, N, ld, gains_is_null != 0, (flags & HORA_FLAG_EXACT_INT) != 0).bytes;
 }
@@ -1644,7 +1644,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     if (alpha == nullptr && !(alpha0 > 0.0 && beta0 > 0.0 && alpha0 < 1.0e300 && beta0 < 1.0e300))
         return HORA_ERR_INVALID_ARG;
     if (cap == nullptr && (cap_scalar < 0 || cap_scalar > ld)) return HORA_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE | HORA_FLAG_SHARED_INT_PRIOR))
+    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE | HORA_FLAG_SHARED_PRIOR))
         return HORA_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (N == 0) {
@@ -1656,9 +1656,10 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     if (gains != nullptr && (reinterpret_cast<uintptr_t>(gains) & 7u)) return HORA_ERR_INVALID_ARG;
     const bool exact = (flags & HORA_FLAG_EXACT_INT) != 0;
     if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HORA_ERR_WORKSPACE;
-    // One integer prior for all prompts, exact ties, no matrix given: at most (G0 + 1) * ld distinct candidate
-    // values, ranked once; the selection runs on ranks and on counts of (c_i, cap_i) and builds no matrix.
-    if (exact && alpha == nullptr && gains == nullptr && rank_route_applies(alpha0, beta0, G0, ld))
+    // One prior for all prompts and no matrix given: at most (G0 + 1) * ld distinct candidate values, ranked once
+    // (exactly for an integer prior with HORA_FLAG_EXACT_INT, else as the doubles hora_gains would write); the
+    // selection runs on ranks and on counts of (c_i, cap_i) and builds no matrix.
+    if (alpha == nullptr && gains == nullptr && rank_route_applies(alpha0, beta0, G0, ld, exact))
         return launch_rank_allocate(alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, flags, delta, G, group_offsets,
                                     info_dev, workspace, workspace_bytes, s, mark_stage);
     const Workspace w = carve(workspace, N, ld, gains == nullptr, exact);

@@ -406,7 +406,7 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
     if (alpha == nullptr && !(alpha0 > 0.0 && beta0 > 0.0 && alpha0 < 1.0e300 && beta0 < 1.0e300))
         return HORA_ERR_INVALID_ARG;
     if (cap == nullptr && (cap_scalar < 0 || cap_scalar > ld)) return HORA_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE | HORA_FLAG_SHARED_INT_PRIOR))
+    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE | HORA_FLAG_SHARED_PRIOR))
         return HORA_ERR_INVALID_ARG;
     if (seg_offsets_host == nullptr || (S > 0 && budgets_host == nullptr)) return HORA_ERR_INVALID_ARG;
     if (seg_offsets_host[0] != 0 || seg_offsets_host[S] != N) return HORA_ERR_INVALID_ARG;
@@ -419,9 +419,11 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
     const int32_t rows_cap = (int32_t)((max_rows + 3) & ~(int64_t)3);
     const size_t smem = sizeof(BatchedSmemFixed) + (size_t)rows_cap * kBRowBytes +
                         (size_t)max_rows * (size_t)ld * sizeof(unsigned long long);
-    // One integer prior for all prompts and exact ties: the candidate values are ranked once for all segments
-    // and every segment is solved on integer ranks by one warp (no shared-memory keys, no segment size limit).
-    const bool by_rank = (flags & HORA_FLAG_EXACT_INT) && alpha == nullptr && rank_route_applies(alpha0, beta0, G0, ld) &&
+    // One prior for all prompts: the candidate values are ranked once for all segments (exactly, or as doubles,
+    // by the tie mode) and every segment is solved on integer ranks by one warp (no shared-memory keys, no
+    // segment size limit).
+    const bool exact_ties = (flags & HORA_FLAG_EXACT_INT) != 0;
+    const bool by_rank = alpha == nullptr && rank_route_applies(alpha0, beta0, G0, ld, exact_ties) &&
                          rank_pos_applies(G0, ld) && rank_tables_bytes(G0, ld, true) <= kBRankReserve;
     if (!by_rank && (max_rows > kBMaxRows || smem > kBMaxSmem)) return HORA_ERR_WORKSPACE;   // segment too large for one CTA
     if (N > 0 && (c == nullptr || delta == nullptr || G == nullptr)) return HORA_ERR_INVALID_ARG;
@@ -440,7 +442,7 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
     if (S > 0 && N > 0 && by_rank) {
         if (cudaMemsetAsync(w.table_status, 0, sizeof(int32_t), st) != cudaSuccess) return HORA_ERR_CUDA;
         const RankTables t = rank_tables_carve(w.tables, G0, ld, true);
-        const int tl = launch_rank_tables(alpha0, beta0, G0, ld, t, w.table_status, st);
+        const int tl = launch_rank_tables(alpha0, beta0, G0, ld, exact_ties, t, w.table_status, st);
         if (tl < 0) return HORA_ERR_CUDA;
         if (launch_rank_batched(c, G0, cap, cap_scalar, ld, w.seg_off, w.budgets, S, flags, t, w.table_status, delta, G,
                                 info_dev, st) != HORA_OK)

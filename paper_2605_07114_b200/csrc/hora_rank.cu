@@ -40,12 +40,13 @@ constexpr double kRankBand = 9.313225746154785e-10;       // 2^-30
 
 static inline size_t rk_align(size_t x) { return (x + 255) & ~(size_t)255; }
 
-bool rank_route_applies(double alpha0, double beta0, int32_t G0, int32_t ld) {
-    if (!(alpha0 >= 1.0 && beta0 >= 1.0 && alpha0 == std::floor(alpha0) && beta0 == std::floor(beta0))) return false;
-    if (G0 < 0 || ld < 1) return false;
+bool rank_route_applies(double alpha0, double beta0, int32_t G0, int32_t ld, bool exact) {
+    if (!(alpha0 > 0.0 && beta0 > 0.0) || G0 < 0 || ld < 1) return false;
     const double top = alpha0 + beta0 + (double)G0 + (double)ld;
-    if (top >= 1048576.0) return false;
+    if (!(top < 1048576.0)) return false;
     if ((int64_t)(G0 + 1) * (int64_t)ld > kRankMaxTypes) return false;
+    if (!exact) return true;                                // ties are equal doubles: nothing else to ask of the prior
+    if (!(alpha0 >= 1.0 && beta0 >= 1.0 && alpha0 == std::floor(alpha0) && beta0 == std::floor(beta0))) return false;
     // every exact form a (b)_a / (b+Delta-1)_{a+1} or a (b)_{Delta-1} / (a+b)_Delta of the table fits 512 bits
     const double factors = std::fmin(alpha0 + (double)G0 + 1.0, (double)ld);
     return factors * std::log2(top) <= 500.0;
@@ -84,7 +85,10 @@ RankTables rank_tables_carve(void *base, int32_t G0, int32_t ld, bool with_pos) 
 
 // Every CTA builds the whole table of fp64 gains in shared memory (a warp per class row: a few hundred
 // instructions), then a thread ranks one type.
-template <int E>
+// EXACT: two types whose doubles are within 2^-30 of each other are compared as exact fractions (integer prior);
+// otherwise the doubles themselves are the order and equal doubles are ties, which is how the key-based selection
+// of hora_allocate treats a matrix of hora_gains without HORA_FLAG_EXACT_INT.
+template <int E, bool EXACT>
 __global__ void __launch_bounds__(kSelThreads)
 rank_table_kernel(double alpha0, double beta0, int32_t G0, int32_t ld, RankTables t, int32_t *status) {
     extern __shared__ __align__(16) unsigned char s_rank_tab[];
@@ -116,7 +120,10 @@ rank_table_kernel(double alpha0, double beta0, int32_t G0, int32_t ld, RankTable
             const int mid = (lo + hi) >> 1;
             const double x = row[mid];
             bool above;
-            if (x > up) above = true;
+            if (!EXACT) {
+                above = x > g0;
+                tie_seen |= x == g0;
+            } else if (x > up) above = true;
             else if (x < dn) above = false;
             else {
                 const int sgn = exact_compare_types(a2, b2, (unsigned long long)mid + 1, a, b, (unsigned long long)j + 1, &overflow);
@@ -130,7 +137,9 @@ rank_table_kernel(double alpha0, double beta0, int32_t G0, int32_t ld, RankTable
         // have compared it: look at column lo itself
         if (c2 < c && lo < ld) {
             const double x = row[lo];
-            if (x <= up && x >= dn) {
+            if (!EXACT) {
+                if (x == g0) first_of_class = false;
+            } else if (x <= up && x >= dn) {
                 if (tie_seen || exact_compare_types(a2, b2, (unsigned long long)lo + 1, a, b, (unsigned long long)j + 1, &overflow) == 0)
                     first_of_class = false;
             }
@@ -161,8 +170,8 @@ rank_pos_kernel(int32_t G0, int32_t ld, RankTables t) {
     t.pos[id] = (uint16_t)lo;
 }
 
-int launch_rank_tables(double alpha0, double beta0, int32_t G0, int32_t ld, const RankTables &t, int32_t *status,
-                       cudaStream_t s) {
+int launch_rank_tables(double alpha0, double beta0, int32_t G0, int32_t ld, bool exact, const RankTables &t,
+                       int32_t *status, cudaStream_t s) {
     const int C = G0 + 1, T = C * ld;
     const size_t smem = sizeof(double) * (size_t)T;
     const int grid = (T + kSelThreads - 1) / kSelThreads;
@@ -174,9 +183,15 @@ int launch_rank_tables(double alpha0, double beta0, int32_t G0, int32_t ld, cons
         return cudaGetLastError() == cudaSuccess;
     };
     bool ok;
-    if (ld > 128) ok = go(rank_table_kernel<8>);
-    else if (ld > 64) ok = go(rank_table_kernel<4>);
-    else ok = go(rank_table_kernel<8>);                       // short rows: as hora_gains builds them
+    if (exact) {
+        if (ld > 128) ok = go(rank_table_kernel<8, true>);
+        else if (ld > 64) ok = go(rank_table_kernel<4, true>);
+        else ok = go(rank_table_kernel<8, true>);             // short rows: as hora_gains builds them
+    } else {
+        if (ld > 128) ok = go(rank_table_kernel<8, false>);
+        else if (ld > 64) ok = go(rank_table_kernel<4, false>);
+        else ok = go(rank_table_kernel<8, false>);
+    }
     if (!ok) return -1;
     int launches = 1;
     if (t.pos != nullptr) {
@@ -702,7 +717,7 @@ hora_status_t launch_rank_allocate(double alpha0, double beta0, const int32_t *c
     if (workspace_bytes < w.bytes) return HORA_ERR_WORKSPACE;
     if (cudaMemsetAsync(w.hdr, 0, w.zero_bytes, s) != cudaSuccess) return HORA_ERR_CUDA;
     mark(0, s);
-    const int tl = launch_rank_tables(alpha0, beta0, G0, ld, w.tab, &w.hdr->status, s);
+    const int tl = launch_rank_tables(alpha0, beta0, G0, ld, (flags & HORA_FLAG_EXACT_INT) != 0, w.tab, &w.hdr->status, s);
     if (tl < 0) return HORA_ERR_CUDA;
     mark(1, s);
     count_launches(tl + 3);

@@ -22,8 +22,9 @@ struct RankTables {
     uint16_t *pos;        // [C][T+1]    pos[c][r] = #{Delta : rank_c(Delta) < r}; null when not built
 };
 
-// Host: does the route apply to this prior and shape?  (integer prior, T within bounds, exact forms within 512 bits)
-bool rank_route_applies(double alpha0, double beta0, int32_t G0, int32_t ld);
+// Host: does the route apply to this prior and shape?  (T within bounds; exact ties: integer prior whose exact forms
+// fit 512 bits; fp64 ties: any prior)
+bool rank_route_applies(double alpha0, double beta0, int32_t G0, int32_t ld, bool exact);
 bool rank_pos_applies(int32_t G0, int32_t ld);
 
 // Bytes of the tables (256-byte granularity) and their carving out of `base`.
@@ -32,8 +33,8 @@ RankTables rank_tables_carve(void *base, int32_t G0, int32_t ld, bool with_pos);
 
 // Enqueue the kernels that fill the tables; `status` (device) receives HORA_ERR_EXACT_RANGE should an exact
 // comparison not fit (the host check makes that unreachable).  Returns the number of launches, or -1 on failure.
-int launch_rank_tables(double alpha0, double beta0, int32_t G0, int32_t ld, const RankTables &t, int32_t *status,
-                       cudaStream_t s);
+int launch_rank_tables(double alpha0, double beta0, int32_t G0, int32_t ld, bool exact, const RankTables &t,
+                       int32_t *status, cudaStream_t s);
 
 // The single-problem route of hora_allocate.
 size_t rank_allocate_workspace_bytes(int64_t N, int32_t G0, int32_t ld);

@@ -138,8 +138,9 @@ def test_segments_beyond_the_per_cta_limits_are_refused():
     N, ld = 600, 64
     c = np.zeros(N, np.int32)
     cap = np.full(N, ld, np.int32)
-    with pytest.raises(hora.HoraError) as e:            # fp64 ties: a CTA per segment, 256 prompts at most
-        run_batched(None, None, 1.0, 1.0, c, 4, cap, ld, np.array([0, 300, 600]), np.array([10, 10]), exact=False)
+    ones = np.ones(N)
+    with pytest.raises(hora.HoraError) as e:            # per-prompt priors: a CTA per segment, 256 prompts at most
+        run_batched(ones, ones, 1.0, 1.0, c, 4, cap, ld, np.array([0, 300, 600]), np.array([10, 10]), exact=False)
     assert e.value.code == hora.ERR_WORKSPACE
     with pytest.raises(hora.HoraError) as e:
         run_batched(None, None, 1.0, 1.0, c, 4, cap, ld, np.array([0, 300, 500]), np.array([10, 10]), exact=True)
@@ -169,6 +170,32 @@ def test_shared_integer_prior_has_no_segment_size_limit(a0, b0):
             assert abs(inf.objective - obj_o[s]) <= 1e-12 * abs(obj_o[s])
             assert abs(inf.lambda_ - lam_o[s]) <= 1e-12 * lam_o[s]
             assert inf.n_above + inf.n_tied_taken == budgets[s] and 1 <= inf.n_tied_taken <= inf.n_tied
+
+
+@pytest.mark.parametrize("a0,b0", [(1.0, 1.0), (0.37, 2.9)])
+def test_shared_prior_with_fp64_ties_matches_the_per_prompt_form(a0, b0):
+    """Without the exact flag a shared prior is ranked as doubles: the result must be what the per-prompt form of the
+    same call (the same prior in arrays: a CTA per segment on its own rows) gives, bit for bit, and the oracle's
+    within its band."""
+    rng = np.random.default_rng(5)
+    G0, ld = 8, 60
+    sizes = rng.integers(1, 40, 200)
+    seg = np.zeros(len(sizes) + 1, np.int64)
+    np.cumsum(sizes, out=seg[1:])
+    N = int(seg[-1])
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    budgets = np.array([int(rng.integers(0, int(cap[seg[s]:seg[s + 1]].sum()) + 1)) for s in range(len(sizes))], np.int64)
+    d, G, off, infos = run_batched(None, None, a0, b0, c, G0, cap, ld, seg, budgets, exact=False)
+    d2, G2, off2, infos2 = run_batched(np.full(N, a0), np.full(N, b0), 1.0, 1.0, c, G0, cap, ld, seg, budgets, exact=False)
+    np.testing.assert_array_equal(d, d2)
+    np.testing.assert_array_equal(off, off2)
+    for x, y in zip(infos, infos2):
+        assert (x.status, x.n_above, x.n_tied, x.n_tied_taken) == (y.status, y.n_above, y.n_tied, y.n_tied_taken)
+        assert x.lambda_ == y.lambda_ and abs(x.objective - y.objective) <= 1e-12 * max(abs(y.objective), 1e-300)
+    if a0 != 1.0:                                        # a real prior: no ties, the oracle's allocation is the only one
+        d_o, _, _ = oracle_segments(np.full(N, a0), np.full(N, b0), 1.0, 1.0, c, G0, cap, seg, budgets, exact=False)
+        np.testing.assert_array_equal(d, d_o)
 
 
 def test_shared_prior_segments_fail_one_by_one():

@@ -145,6 +145,34 @@ def test_route_agrees_with_the_general_exact_path():
     assert abs(i1.lambda_ - i2.lambda_) <= 1e-13 * i1.lambda_ and abs(i1.objective - i2.objective) <= 1e-12 * i1.objective
 
 
+@pytest.mark.parametrize("a0,b0", [(1.0, 1.0), (2.0, 5.0), (0.5, 0.5), (3.7, 0.21)])
+def test_fp64_ties_on_ranks_equal_the_key_based_selection(a0, b0):
+    """Without the exact flag the shared prior's candidate values are ranked as the doubles hora_gains writes, equal
+    doubles tie: Delta, the tie counts and the threshold must be those of the key-based selection on the
+    materialised matrix, bit for bit; for a real prior (no ties) also the oracle's."""
+    gu = _gu()
+    rng = np.random.default_rng(int(a0 * 100 + b0 * 10))
+    N, G0, ld = 20011, 6, 90
+    c = rng.integers(0, G0 + 1, N).astype(np.int32)
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    total = int(cap.sum())
+    for B in (0, 1, total // 5, total // 2, total - 1, total):
+        d1, G1, off1, i1 = gu.gpu_allocate(None, None, a0, b0, c, G0, cap, ld, B, exact=False, materialise=True)
+        d2, G2, off2, i2 = gu.gpu_allocate(None, None, a0, b0, c, G0, cap, ld, B, exact=False, materialise=False,
+                                           shared_int_prior=True)
+        assert i1.status == 0 and i2.status == 0
+        assert i2.first_pass_bits == (-1 if B > 0 else 0) and i1.first_pass_bits in (0, 13, 23)
+        np.testing.assert_array_equal(d1, d2, err_msg=f"B={B}")
+        np.testing.assert_array_equal(off1, off2)
+        assert (i1.n_above, i1.n_tied, i1.n_tied_taken) == (i2.n_above, i2.n_tied, i2.n_tied_taken)
+        assert i1.lambda_ == i2.lambda_
+        assert abs(i1.objective - i2.objective) <= 1e-12 * max(abs(i1.objective), 1e-300)
+        if a0 != np.floor(a0) and B > 0:
+            d_o, _, lam_o, obj_o = orc.greedy_real(None, None, a0, b0, c, G0, cap, B)
+            np.testing.assert_array_equal(d2, d_o)
+            assert abs(i2.lambda_ - lam_o) <= 1e-12 * lam_o and abs(i2.objective - obj_o) <= 1e-12 * obj_o
+
+
 def test_shapes_outside_the_route_fall_back_to_the_general_path():
     """(G0 + 1) * ld above 8192 types: the call builds the matrix as before (needs the full-size workspace)."""
     gu = _gu()
