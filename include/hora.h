@@ -61,7 +61,9 @@ enum {
     HORA_FLAG_SHARED_PRIOR = 4u,   /* sizing hint for hora_allocate_workspace_bytes: the call will pass alpha == beta ==
                                       NULL and gains == NULL (see the rank-based route under hora_allocate); ignored
                                       by the calls themselves */
-    HORA_FLAG_SHARED_INT_PRIOR = 4u /* the same flag under the name of its first use (an integer prior, exact ties) */
+    HORA_FLAG_SHARED_INT_PRIOR = 4u, /* the same flag under the name of its first use (an integer prior, exact ties) */
+    HORA_FLAG_HARD_FIRST = 8u      /* hora_allocate_batched only: every segment by the hard-first rule of
+                                      hora_allocate_hard_first instead of the hit-utility optimum (priors unused) */
 };
 
 enum { HORA_ADV_GRPO = 0, HORA_ADV_RLOO = 1 };
@@ -235,7 +237,9 @@ hora_status_t hora_allocate_hard_first(const int32_t *c, int32_t G0, const int32
  * Segment s covers prompts seg_offsets_host[s] .. seg_offsets_host[s+1]-1 and hands out budgets_host[s]
  * rollouts among them, exactly as hora_allocate would on that segment alone (same gains bit for bit, same tie
  * rules, same exact mode).  One CTA solves one segment in shared memory (one warp on precomputed ranks when the
- * prior is shared); no gains matrix is materialised.
+ * prior is shared); no gains matrix is materialised.  With HORA_FLAG_HARD_FIRST every segment is allocated by the
+ * comparison rule of hora_allocate_hard_first instead (the form the paper's ablation ran it in: per shard); the
+ * priors are then unused, lambda and objective are 0, and no segment size limit applies.
  *
  *   alpha .. ld            as for hora_gains (device arrays over all N prompts)
  *   seg_offsets_host       HOST array [S+1], non-decreasing, [0] == 0, [S] == N

@@ -362,6 +362,105 @@ scan_write_offsets(const int32_t *__restrict__ G, int64_t N, const long long *__
 // room for the rank tables of the shared-integer-prior route (its size does not depend on N or S)
 constexpr size_t kBRankReserve = ((size_t)5 << 19) + 4096;     // 2.5 MiB: 2 MiB of positions + the per-type tables
 
+// The hard-first rule (Sec. 4.2, "Comparison with the hard-first heuristic") per segment, a warp per segment: the
+// segment's budget is dealt round-robin in prompt order to its prompts with c = 0 that are below their cap, the
+// rest of it the same way to the other prompts.  Dealing round-robin fills the active class to a common level L
+// (or each prompt's cap) and gives the first R prompts with cap > L one more:
+//     f(L) = sum_i min(cap_i, L) <= budget of the class < f(L + 1),   R = budget - f(L);
+// L comes out of a bisection whose step is one pass over the segment's caps and one warp sum.
+__global__ void __launch_bounds__(kBThreads)
+hard_first_batched_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
+                          int32_t ld, const int64_t *__restrict__ seg_off, const int64_t *__restrict__ budgets, int64_t S,
+                          int32_t *__restrict__ delta, int32_t *__restrict__ G, hora_alloc_info *__restrict__ info) {
+    const int lane = lane_id();
+    const int64_t warp0 = (int64_t)blockIdx.x * kBWarps + (threadIdx.x >> 5);
+    const int64_t n_warps = (int64_t)gridDim.x * kBWarps;
+    auto warp_sum = [](long long v) {
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(kFull, v, d);
+        return v;
+    };
+    for (int64_t s = warp0; s < S; s += n_warps) {
+        const int64_t r0 = __ldg(seg_off + s);
+        const int64_t n = __ldg(seg_off + s + 1) - r0;
+        const long long B = __ldg(budgets + s);
+        // prompt i of the segment: (tier, cap) with tier 0 for c = 0; -1 marks an invalid prompt
+        auto fetch = [&](int64_t i, int *tier, int *cp) {
+            const int ci = __ldg(c + r0 + i);
+            *cp = cap ? __ldg(cap + r0 + i) : cap_scalar;
+            *tier = (ci < 0 || ci > G0 || *cp < 0 || *cp > ld) ? -1 : (ci > 0);
+        };
+        long long cap0 = 0, cap1 = 0;
+        bool bad = false;
+        for (int64_t i = lane; i < n; i += kWarp) {
+            int tier, cp;
+            fetch(i, &tier, &cp);
+            bad |= tier < 0;
+            if (tier == 0) cap0 += cp; else if (tier == 1) cap1 += cp;
+        }
+        cap0 = warp_sum(cap0);
+        cap1 = warp_sum(cap1);
+        int status = HORA_OK;
+        if (__any_sync(kFull, bad) || B < 0) status = HORA_ERR_INVALID_VALUE;
+        else if (B > cap0 + cap1) status = HORA_ERR_INFEASIBLE;
+        const int active = B <= cap0 ? 0 : 1;                  // the class in which the level is sought
+        const long long Bt = active == 0 ? B : B - cap0;
+        auto filled = [&](int L) {                             // f(L) over the active class
+            long long part = 0;
+            for (int64_t i = lane; i < n; i += kWarp) {
+                int tier, cp;
+                fetch(i, &tier, &cp);
+                if (tier == active) part += cp < L ? cp : L;
+            }
+            return warp_sum(part);
+        };
+        int L = 0;
+        long long used = 0;
+        if (!status) {
+            int lo = 0, hi = ld;                               // largest L with f(L) <= Bt
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (filled(mid) <= Bt) lo = mid; else hi = mid - 1;
+            }
+            L = lo;
+            used = filled(L);
+        }
+        const long long R = Bt - used;
+        long long before = 0, n_room = 0;                      // prompts with room above the level, in index order
+        for (int64_t i0 = 0; i0 < n; i0 += kWarp) {
+            const int64_t i = i0 + lane;
+            int tier = -1, cp = 0;
+            if (i < n) fetch(i, &tier, &cp);
+            const bool in_active = !status && tier == active;
+            const bool room = in_active && cp > L;
+            const unsigned m = __ballot_sync(kFull, room);
+            const long long rank = before + __popc(m & ((1u << lane) - 1u));
+            int d = 0;
+            if (in_active) d = (cp < L ? cp : L) + ((room && rank < R) ? 1 : 0);
+            else if (!status && tier == 0) d = cp;            // the level is in the other class: c = 0 prompts are full
+            if (i < n) {
+                delta[r0 + i] = d;
+                G[r0 + i] = status ? 0 : G0 + d;
+            }
+            before += __popc(m);
+            n_room += __popc(m);
+        }
+        if (lane == 0 && info != nullptr) {
+            hora_alloc_info o;
+            o.status = status;
+            o.first_pass_bits = 0;
+            o.lambda = 0.0;
+            o.n_above = status ? 0 : B - R;
+            o.n_tied = status ? 0 : n_room;
+            o.n_tied_taken = status ? 0 : R;
+            o.objective = 0.0;
+            o.sum_G = status ? 0 : n * (long long)G0 + B;
+            o.sum_cap = cap0 + cap1;
+            info[s] = o;
+        }
+    }
+}
+
 struct BatchedWorkspace {
     int64_t *seg_off, *budgets;
     long long *bsum;
@@ -406,8 +505,9 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
     if (alpha == nullptr && !(alpha0 > 0.0 && beta0 > 0.0 && alpha0 < 1.0e300 && beta0 < 1.0e300))
         return HORA_ERR_INVALID_ARG;
     if (cap == nullptr && (cap_scalar < 0 || cap_scalar > ld)) return HORA_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE | HORA_FLAG_SHARED_PRIOR))
+    if (flags & ~(uint32_t)(HORA_FLAG_EXACT_INT | HORA_FLAG_SKIP_OBJECTIVE | HORA_FLAG_SHARED_PRIOR | HORA_FLAG_HARD_FIRST))
         return HORA_ERR_INVALID_ARG;
+    const bool hard_first = (flags & HORA_FLAG_HARD_FIRST) != 0;   // the comparison rule: the priors play no part
     if (seg_offsets_host == nullptr || (S > 0 && budgets_host == nullptr)) return HORA_ERR_INVALID_ARG;
     if (seg_offsets_host[0] != 0 || seg_offsets_host[S] != N) return HORA_ERR_INVALID_ARG;
     int64_t max_rows = 0;
@@ -425,7 +525,8 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
     const bool exact_ties = (flags & HORA_FLAG_EXACT_INT) != 0;
     const bool by_rank = alpha == nullptr && rank_route_applies(alpha0, beta0, G0, ld, exact_ties) &&
                          rank_pos_applies(G0, ld) && rank_tables_bytes(G0, ld, true) <= kBRankReserve;
-    if (!by_rank && (max_rows > kBMaxRows || smem > kBMaxSmem)) return HORA_ERR_WORKSPACE;   // segment too large for one CTA
+    if (!by_rank && !hard_first && (max_rows > kBMaxRows || smem > kBMaxSmem))
+        return HORA_ERR_WORKSPACE;                            // segment too large for one CTA
     if (N > 0 && (c == nullptr || delta == nullptr || G == nullptr)) return HORA_ERR_INVALID_ARG;
     if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HORA_ERR_WORKSPACE;
     const BatchedWorkspace w = carve_batched(workspace, N, S);
@@ -439,7 +540,12 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
                      cudaSuccess)
         return HORA_ERR_CUDA;
     int launches = 0;
-    if (S > 0 && N > 0 && by_rank) {
+    if (S > 0 && N > 0 && hard_first) {
+        hard_first_batched_kernel<<<clamp_grid((S + kBWarps - 1) / kBWarps, 8), kBThreads, 0, st>>>(
+            c, G0, cap, cap_scalar, ld, w.seg_off, w.budgets, S, delta, G, info_dev);
+        if (cudaGetLastError() != cudaSuccess) return HORA_ERR_CUDA;
+        ++launches;
+    } else if (S > 0 && N > 0 && by_rank) {
         if (cudaMemsetAsync(w.table_status, 0, sizeof(int32_t), st) != cudaSuccess) return HORA_ERR_CUDA;
         const RankTables t = rank_tables_carve(w.tables, G0, ld, true);
         const int tl = launch_rank_tables(alpha0, beta0, G0, ld, exact_ties, t, w.table_status, st);

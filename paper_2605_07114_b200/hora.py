@@ -21,6 +21,7 @@ LIB_PATH = os.path.join(HERE, "libhora.so")
 FLAG_EXACT_INT = 1
 FLAG_SKIP_OBJECTIVE = 2
 FLAG_SHARED_PRIOR = 4
+FLAG_HARD_FIRST = 8
 FLAG_SHARED_INT_PRIOR = 4            # the same flag under the name of its first use
 ADV_GRPO, ADV_RLOO = 0, 1
 WEIGHT_PER_TOKEN, WEIGHT_CONST_LENGTH = 0, 1

@@ -91,3 +91,51 @@ def test_scalar_cap_and_status_codes():
     cap[5] = ld + 1
     d, G, off, info = run(c, G0, cap, ld, 100)
     assert info.status == 2 and not d.any()
+
+
+def test_hard_first_per_segment():
+    """hora_allocate_batched with HORA_FLAG_HARD_FIRST: every segment by the comparison rule, against the plain loops
+    run segment by segment (segments of 0, 1, 15, 32, 33 and 700 prompts; budgets below, at and above what the c = 0
+    prompts can take; an infeasible and an invalid segment that leave the others alone)."""
+    from paper_2605_07114_b200 import hora
+    rng = np.random.default_rng(321)
+    G0, ld = 8, 40
+    sizes = np.array([15] * 40 + [0, 1, 32, 33, 700, 15, 15])
+    seg = np.zeros(len(sizes) + 1, np.int64)
+    np.cumsum(sizes, out=seg[1:])
+    N, S = int(seg[-1]), len(sizes)
+    c = np.where(rng.random(N) < 0.2, 0, rng.integers(1, G0 + 1, N)).astype(np.int32)
+    cap = rng.integers(0, ld + 1, N).astype(np.int32)
+    budgets = np.zeros(S, np.int64)
+    for s in range(S):
+        sl = slice(int(seg[s]), int(seg[s + 1]))
+        hard, total = int(cap[sl][c[sl] == 0].sum()), int(cap[sl].sum())
+        budgets[s] = [0, hard // 2, hard, min(hard + 3, total), total, int(rng.integers(0, total + 1))][s % 6]
+    budgets[S - 2] = int(cap[seg[S - 2]:seg[S - 1]].sum()) + 1          # infeasible
+    c[seg[S - 1] + 4] = G0 + 3                                           # invalid count in the last segment
+    dev = "cuda"
+    t = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(dev)
+    delta = torch.full((N,), -1, dtype=torch.int32, device=dev)
+    G = torch.full((N,), -1, dtype=torch.int32, device=dev)
+    off = torch.full((N + 1,), -1, dtype=torch.int64, device=dev)
+    info = torch.zeros(S * hora.INFO_BYTES, dtype=torch.uint8, device=dev)
+    ws = torch.empty(hora.hora_allocate_batched_workspace_bytes(N, S), dtype=torch.uint8, device=dev)
+    hora.hora_allocate_batched(None, None, 1.0, 1.0, t(c), G0, t(cap), 0, N, ld, seg, budgets, hora.FLAG_HARD_FIRST, delta, G,
+                               off, info, ws)
+    torch.cuda.synchronize()
+    d, infos = delta.cpu().numpy(), hora.read_infos(info, S)
+    exp = np.zeros(N, np.int32)
+    for s in range(S):
+        sl = slice(int(seg[s]), int(seg[s + 1]))
+        if s == S - 2:
+            assert infos[s].status == 3
+        elif s == S - 1:
+            assert infos[s].status == 2
+        else:
+            assert infos[s].status == 0
+            exp[sl] = hf.hard_first([int(x) for x in c[sl]], [int(x) for x in cap[sl]], int(budgets[s]))
+            assert infos[s].n_above + infos[s].n_tied_taken == budgets[s] and infos[s].sum_cap == int(cap[sl].sum())
+    np.testing.assert_array_equal(d, exp)
+    Gx = np.where(np.repeat([i.status == 0 for i in infos], sizes), G0 + exp, 0)
+    np.testing.assert_array_equal(G.cpu().numpy(), Gx)
+    np.testing.assert_array_equal(off.cpu().numpy(), np.concatenate(([0], np.cumsum(Gx.astype(np.int64)))))
