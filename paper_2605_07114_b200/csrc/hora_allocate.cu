@@ -596,22 +596,25 @@ struct CoarseTap {
     __device__ __forceinline__ void begin_row(int64_t, int32_t) {}
 };
 
-// the level-0 bookkeeping: window histogram and the count of keys above the guessed threshold
-template <int E>
+// the level-0 bookkeeping: window histogram and the count of keys above the guessed threshold.  LG lanes build a
+// row (32 for long rows; 16, 8 or 4 when several short rows share the warp): the counts are summed over the
+// row's own lanes, and the first lane of a row keeps its totals.
+template <int E, int LG>
 struct Level0Tap {
     unsigned long long key[E];
     unsigned int *s_fine;
     unsigned int *pguess;
-    unsigned int *pg_row;          // the count of the prompt being built
+    unsigned int *pg_row;          // the count of the prompt being built (null: the row does not exist)
     unsigned W0;
     int t_guess;
-    unsigned int row_above;        // lane 0: keys above the guess in the chunks of this row so far
-    long long sum_pg;              // lane 0: the same over all rows of this warp
-    long long capsum;              // lane 0 of every warp: caps of the rows it built
+    unsigned int row_above;        // first lane of the row: keys above the guess in the chunks of this row so far
+    long long sum_pg;              // first lane of a row: the same over all rows it led
+    long long capsum;              // first lane of a row: caps of the rows it led
+    __device__ __forceinline__ bool leader() const { return (threadIdx.x & (LG - 1)) == 0; }
     __device__ __forceinline__ void begin_row(int64_t row, int32_t capi) {
-        pg_row = pguess + row;
+        pg_row = row >= 0 ? pguess + row : nullptr;
         row_above = 0;
-        if ((threadIdx.x & 31) == 0) capsum += capi;
+        if (leader()) capsum += capi;
     }
     __device__ __forceinline__ void pair(int m, double g0, double g1) {
         key[m] = (unsigned long long)__double_as_longlong(g0);
@@ -621,10 +624,16 @@ struct Level0Tap {
         unsigned h[E];
 #pragma unroll
         for (int m = 0; m < E; ++m) h[m] = (unsigned)(key[m] >> 32);
-        const int above = __reduce_add_sync(kFull, window_count<E>(h, capi - k, W0, t_guess, s_fine));
+        int above = window_count<E>(h, capi - k, W0, t_guess, s_fine);
+        if (LG == kWarp) {
+            above = __reduce_add_sync(kFull, above);
+        } else {
+#pragma unroll
+            for (int d = 1; d < LG; d <<= 1) above += __shfl_xor_sync(kFull, above, d);
+        }
         row_above += (unsigned int)above;
         sum_pg += above;
-        if ((threadIdx.x & 31) == 0) *pg_row = row_above;      // the row's chunks come one after another in this warp
+        if (leader() && pg_row != nullptr) *pg_row = row_above;   // the row's chunks come one after another in these lanes
     }
 };
 
@@ -664,7 +673,7 @@ select_estimate_fused(const double *__restrict__ alpha, const double *__restrict
 // The fused full pass: the row loop of hora_gains (same staging, same arithmetic, same stores) with level 0's
 // counting tapped in.  Rows are trusted to be sorted (they were just computed), so only the inputs are
 // validated (the row loop raises the status for invalid priors, counts or caps).
-template <int E, bool VEC2>
+template <int E, bool VEC2, int LG>
 __global__ void __launch_bounds__(kSelThreads, 3)
 gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
                    const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
@@ -674,7 +683,7 @@ gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ 
     __shared__ long long s_warp[kSelThreads / kWarp];
     for (int b = threadIdx.x; b < kFineBins; b += kSelThreads) s_fine[b] = 0;
     __syncthreads();
-    Level0Tap<E> tap;
+    Level0Tap<E, LG> tap;
     tap.s_fine = s_fine;
     tap.pguess = pguess;
     tap.pg_row = pguess;
@@ -684,9 +693,9 @@ gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ 
     tap.row_above = 0;
     tap.sum_pg = 0;
     tap.capsum = 0;
-    gains_rows_cta<E, VEC2>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, &hdr->status, tap);
-    level0_finish(hdr, hist_fine, s_fine, tap.W0, tap.t_guess, tap.capsum, (threadIdx.x & 31) == 0 ? tap.sum_pg : 0, false, B,
-                  s_warp);
+    gains_rows_cta<E, VEC2, Level0Tap<E, LG>, LG>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, &hdr->status, tap);
+    level0_finish(hdr, hist_fine, s_fine, tap.W0, tap.t_guess, tap.leader() ? tap.capsum : 0, tap.leader() ? tap.sum_pg : 0,
+                  false, B, s_warp);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -1583,12 +1592,15 @@ static cudaError_t launch_fused(bool vec2, bool estimate, int grid_est, int64_t 
     if (estimate)
         select_estimate_fused<E><<<grid_est, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N,
                                                                   ld, every, B, w.hdr, w.hist_est);
-    if (vec2)
-        gains_level0_fused<E, true><<<grid, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
-                                                                 w.gains, B, w.hdr, w.hist_fine, w.pguess);
-    else
-        gains_level0_fused<E, false><<<grid, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
-                                                                  w.gains, B, w.hdr, w.hist_fine, w.pguess);
+    auto go = [&](auto kernel) {
+        kernel<<<grid, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, w.gains, B, w.hdr,
+                                            w.hist_fine, w.pguess);
+    };
+    // lanes per row as in hora_gains: short rows share a warp
+    if (ld > 128) { if (vec2) go(gains_level0_fused<E, true, kWarp>); else go(gains_level0_fused<E, false, kWarp>); }
+    else if (ld > 64) { if (vec2) go(gains_level0_fused<E, true, 16>); else go(gains_level0_fused<E, false, 16>); }
+    else if (ld > 32) { if (vec2) go(gains_level0_fused<E, true, 8>); else go(gains_level0_fused<E, false, 8>); }
+    else { if (vec2) go(gains_level0_fused<E, true, 4>); else go(gains_level0_fused<E, false, 4>); }
     return cudaGetLastError();
 }
 
@@ -1698,14 +1710,9 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_start, s);
     if (fused) {
         const int gridf = clamp_grid((N + kCtaRows - 1) / kCtaRows, 3);
-        cudaError_t e;
-        if (ld > 128)
-            e = launch_fused<8>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, w);
-        else if (ld > 64)
-            e = launch_fused<4>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, w);
-        else
-            e = launch_fused<8>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, B, w);
-        if (e != cudaSuccess) return HORA_ERR_CUDA;
+        if (launch_fused<8>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
+                            B, w) != cudaSuccess)
+            return HORA_ERR_CUDA;
     } else if (ld > 128) {
         launch_level0<8>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
     } else if (ld > 64) {

@@ -565,11 +565,7 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
                                                   w.budgets, S, flags, rows_cap, delta, G, info_dev);
             return cudaGetLastError();
         };
-        cudaError_t e;
-        if (ld > 128) e = launch(allocate_batched_kernel<8>);
-        else if (ld > 64) e = launch(allocate_batched_kernel<4>);
-        else e = launch(allocate_batched_kernel<8>);   // short rows: as hora_gains builds them (8 entries a lane)
-        if (e != cudaSuccess) return HORA_ERR_CUDA;
+        if (launch(allocate_batched_kernel<8>) != cudaSuccess) return HORA_ERR_CUDA;   // 8 entries a lane, as hora_gains
         ++launches;
     }
     if (group_offsets != nullptr) {

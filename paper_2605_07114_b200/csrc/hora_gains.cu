@@ -14,9 +14,10 @@
 namespace hora {
 
 // The kernel is the shared row loop with no tap attached.
-// LG: lanes per row.  Rows of at most 64 entries are built four (LG = 8) or eight (LG = 4) to a warp, so that a
-// warp still produces 256 entries per scan and per reciprocal: a whole warp on a 64-entry row spent as many
-// instructions per row as on a 256-entry one, and those, not the memory system, set the time (2.9 TB/s).
+// LG: lanes per row.  Rows of at most 128 entries are built two (LG = 16), four (LG = 8) or eight (LG = 4) to a
+// warp, so that a warp still produces 256 entries per scan and per reciprocal: a whole warp on a 64-entry row
+// spent as many instructions per row as on a 256-entry one, and those, not the memory system, set the time
+// (2.9 TB/s at 64 entries, 4.3 TB/s at 128).  A lane always holds 8 consecutive entries.
 template <int E, bool VEC2, int LG>
 __global__ void __launch_bounds__(kGainsWarps *kWarp, 3)
 gains_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
@@ -48,7 +49,7 @@ hora_status_t launch_gains(const double *alpha, const double *beta, double alpha
     if (ld > 128)
         return launch_e<8, kWarp>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
     if (ld > 64)
-        return launch_e<4, kWarp>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
+        return launch_e<8, 16>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
     if (ld > 32)
         return launch_e<8, 8>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);
     return launch_e<8, 4>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, stream);

@@ -100,7 +100,8 @@ constexpr int kCtaRows = kGainsWarps * kTile; // rows a CTA stages per step
 
 // A CTA stages the posterior parameters of 64 consecutive rows in shared memory (one coalesced load per
 // array, issued one step ahead and parked in registers meanwhile); each warp then takes 8 of those rows.
-// LG < 32 (rows of at most LG * E entries): a warp builds 32 / LG rows at a time, LG lanes a row (no tap then).
+// LG < 32 (rows of at most LG * E entries): a warp builds 32 / LG rows at a time, LG lanes a row; a tap is told
+// begin_row(-1, 0) for the rows of the last tile that do not exist.
 template <int E, bool VEC2, typename Tap, int LG = kWarp>
 __device__ __forceinline__ void gains_rows_cta(const double *__restrict__ alpha, const double *__restrict__ beta,
                                                double alpha0, double beta0, const int32_t *__restrict__ c, int32_t G0,
@@ -145,7 +146,7 @@ __device__ __forceinline__ void gains_rows_cta(const double *__restrict__ alpha,
         __syncthreads();                                  // buf was last read two steps ago: safe to have overwritten it
         nxt = fetch(step + gridDim.x);
         const int64_t row0 = step * kCtaRows + warp * kTile;
-        if (LG < kWarp) {
+        if constexpr (LG < kWarp) {
             // packed rows: group g of the warp builds row row0 + i + g
             constexpr int R = kWarp / LG;
             const int grp = lane / LG, gl = lane % LG;
@@ -157,30 +158,31 @@ __device__ __forceinline__ void gains_rows_cta(const double *__restrict__ alpha,
                 const double a = s_a[buf][idx], b = s_b[buf][idx];
                 const int32_t capi = live ? s_cap[buf][idx] : 0;
                 double carry = 1.0;
+                tap.begin_row(live ? row : -1, capi);
                 if (back_to_back) {
                     const int64_t rows_here = N - (row0 + i) < R ? N - (row0 + i) : R;
-                    gains_chunk<E, VEC2, false, NoTap, LG, VEC2 && (E > 2)>(a, b, a + b, capi, ld, 0, gl, carry,
-                                                                          gains + (row0 + i) * (int64_t)ld, wr, rd,
-                                                                          NoTap(), (int32_t)(rows_here * ld));
+                    gains_chunk<E, VEC2, false, Tap &, LG, VEC2 && (E > 2)>(a, b, a + b, capi, ld, 0, gl, carry,
+                                                                          gains + (row0 + i) * (int64_t)ld, wr, rd, tap,
+                                                                          (int32_t)(rows_here * ld));
                 } else {
-                    gains_chunk<E, VEC2, false, NoTap, LG, false>(a, b, a + b, capi, live ? ld : 0, 0, gl, carry,
-                                                                 gains + (live ? row : 0) * (int64_t)ld, nullptr, nullptr);
+                    gains_chunk<E, VEC2, false, Tap &, LG, false>(a, b, a + b, capi, live ? ld : 0, 0, gl, carry,
+                                                                 gains + (live ? row : 0) * (int64_t)ld, nullptr, nullptr, tap);
                 }
             }
-            continue;
-        }
-        for (int i = 0; i < kTile && row0 + i < N; ++i) {
-            const double a = s_a[buf][warp * kTile + i], b = s_b[buf][warp * kTile + i];
-            const int32_t capi = s_cap[buf][warp * kTile + i];
-            const double ab = a + b;
-            double *out = gains + (row0 + i) * (int64_t)ld;
-            tap.begin_row(row0 + i, capi);
-            double carry = 1.0;
-            for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E) {
-                if (k0 + kWarp * E <= capi)               // capi <= ld: the chunk is inside the row as well
-                    gains_chunk<E, VEC2, true>(a, b, ab, capi, ld, k0, lane, carry, out, wr, rd, tap);
-                else
-                    gains_chunk<E, VEC2, false>(a, b, ab, capi, ld, k0, lane, carry, out, wr, rd, tap);
+        } else {
+            for (int i = 0; i < kTile && row0 + i < N; ++i) {
+                const double a = s_a[buf][warp * kTile + i], b = s_b[buf][warp * kTile + i];
+                const int32_t capi = s_cap[buf][warp * kTile + i];
+                const double ab = a + b;
+                double *out = gains + (row0 + i) * (int64_t)ld;
+                tap.begin_row(row0 + i, capi);
+                double carry = 1.0;
+                for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E) {
+                    if (k0 + kWarp * E <= capi)           // capi <= ld: the chunk is inside the row as well
+                        gains_chunk<E, VEC2, true>(a, b, ab, capi, ld, k0, lane, carry, out, wr, rd, tap);
+                    else
+                        gains_chunk<E, VEC2, false>(a, b, ab, capi, ld, k0, lane, carry, out, wr, rd, tap);
+                }
             }
         }
     }

@@ -183,15 +183,8 @@ int launch_rank_tables(double alpha0, double beta0, int32_t G0, int32_t ld, bool
         return cudaGetLastError() == cudaSuccess;
     };
     bool ok;
-    if (exact) {
-        if (ld > 128) ok = go(rank_table_kernel<8, true>);
-        else if (ld > 64) ok = go(rank_table_kernel<4, true>);
-        else ok = go(rank_table_kernel<8, true>);             // short rows: as hora_gains builds them
-    } else {
-        if (ld > 128) ok = go(rank_table_kernel<8, false>);
-        else if (ld > 64) ok = go(rank_table_kernel<4, false>);
-        else ok = go(rank_table_kernel<8, false>);
-    }
+    if (exact) ok = go(rank_table_kernel<8, true>);          // 8 entries a lane at every ld, as hora_gains builds rows
+    else ok = go(rank_table_kernel<8, false>);
     if (!ok) return -1;
     int launches = 1;
     if (t.pos != nullptr) {
