@@ -536,6 +536,172 @@ select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
     level0_finish(hdr, hist_fine, s_fine, W0, t_guess, capsum, sum_pg, bad, B, s_warp);
 }
 
+// ---------------------------------------------------------------------------------------------------
+// The full-read pass for rows of at most 128 keys: LG = 16, 8 or 4 lanes take a row (of at most 8 LG keys) and a
+// warp takes 32 / LG consecutive rows at a time, every row with its own cap, its own order check and its own count
+// above the guess.  With a warp per row, a 64-key row cost as many warp instructions as a 256-key one (the cap,
+// the votes, the reduction and the row's count are per row) and the pass read 2.4 TB/s.
+// A lane holds 8 consecutive keys of its row, so all but one of its order checks stay inside the lane; the caps
+// are fetched one item further ahead than the keys, whose loads they gate.
+template <int LG>
+struct Level0Short {
+    unsigned long long key[8];     // keys 8 gl .. 8 gl + 7 of the lane's row (gl = its place among the row's lanes);
+                                   // keys past the cap read as 0
+    int32_t capi;                  // the cap of the lane's row (0 for a row past the end); -1 marks "no item"
+};
+
+// what every item of the pass needs, worked out once (items and rows are counted in 32 bits: N < 2^31)
+struct Level0ShortPass {
+    const int32_t *cap;
+    int32_t cap_scalar, N, n_items, ld;
+    const unsigned long long *keys;
+    unsigned int *pguess;
+    unsigned fine_shared;          // shared-window address of the fine histogram
+    unsigned base;                 // first high word of the window
+    unsigned above_from;           // first high word above the guess
+};
+
+// 16 zero bytes: where a lane's chunk lies past the cap it reads these instead (a select on the address and an
+// unconditional load, where a conditional load compiled to a branch of its own per chunk)
+__device__ __align__(16) const unsigned long long g_zero_chunk[2] = {0ull, 0ull};
+
+// the cap of the lane's row of `item`, without a branch: the load is taken at a row that exists
+template <int LG>
+__device__ __forceinline__ int32_t level0_short_cap(const Level0ShortPass &ps, int32_t item, int lane, unsigned *bad) {
+    const int32_t row = item * (kWarp / LG) + lane / LG;
+    const bool there = row < ps.N;                             // (an item past the end has no row that is)
+    int32_t capi = ps.cap_scalar;
+    if (ps.cap != nullptr) capi = __ldg(ps.cap + (there ? row : 0));
+    const bool ok = (unsigned)capi <= (unsigned)ps.ld;
+    *bad |= (unsigned)(there && !ok);
+    capi = there && ok ? capi : 0;
+    return item < ps.n_items ? capi : -1;
+}
+
+template <int LG, bool VEC2>
+__device__ __forceinline__ void level0_short_fetch(Level0Short<LG> &it, const Level0ShortPass &ps, int32_t capi,
+                                                   int32_t item, int lane) {
+    it.capi = capi;
+    const int gl = lane & (LG - 1);
+    const int32_t row = item * (kWarp / LG) + lane / LG;
+    const int32_t nvalid = capi - 8 * gl;                      // <= 0 for "no item" and for a row past the end
+    const unsigned long long *keys = ps.keys + ((int64_t)row * ps.ld + 8 * gl);   // (used only where nvalid > 0)
+#pragma unroll
+    for (int j = 0; j < 8; j += 2) {
+        if (VEC2) {
+            const ulonglong2 t = __ldg(reinterpret_cast<const ulonglong2 *>(j < nvalid ? keys + j : g_zero_chunk));
+            it.key[j] = t.x;
+            it.key[j + 1] = j + 1 < nvalid ? t.y : 0ull;
+        } else {
+            it.key[j] = __ldg(j < nvalid ? keys + j : g_zero_chunk);
+            it.key[j + 1] = __ldg(j + 1 < nvalid ? keys + j + 1 : g_zero_chunk);
+        }
+    }
+}
+
+// fine[d >> 9] += 1 where d < limit, as one predicated instruction (an `if` around the atomic compiled to a
+// branch per key); the address is formed for every key and used only under the predicate
+__device__ __forceinline__ void count_if_below(unsigned fine_shared, unsigned d, unsigned limit) {
+    const unsigned addr = fine_shared + (d >> 9) * 4u;
+    asm volatile("{\n .reg .pred p;\n setp.lt.u32 p, %1, %2;\n @p red.shared.add.u32 [%0], 1;\n}" ::"r"(addr), "r"(d), "r"(limit)
+                 : "memory");
+}
+
+template <int LG>
+__device__ __forceinline__ void level0_short_process(const Level0Short<LG> &it, const Level0ShortPass &ps, int32_t item,
+                                                     int lane, int32_t *capsum, int32_t *sum_pg, unsigned *bad) {
+    const int gl = lane & (LG - 1);
+    const int32_t row = item * (kWarp / LG) + lane / LG;
+    const int32_t nvalid = it.capi - 8 * gl;
+    // Order: the bit patterns of finite non-negative doubles order like the values, and anything else (a sign bit,
+    // an infinity, a NaN) is a pattern above the largest finite one: it either exceeds its predecessor or is the
+    // row's first key, which is held against that bound.  Keys past the cap are 0 and exceed nothing.
+    {
+        bool viol = false;
+#pragma unroll
+        for (int j = 0; j < 7; ++j) viol |= it.key[j + 1] > it.key[j];
+        const unsigned long long nx = __shfl_down_sync(kFull, it.key[0], 1);
+        viol |= gl < LG - 1 && nx > it.key[7];                 // the next lane of the same row
+        viol |= gl == 0 && it.key[0] > kKeyInf - 1;
+        *bad |= (unsigned)viol;
+    }
+    // Window, on the high words: d = h - (first pattern of the window) wraps far above the window's width for a
+    // key below it (so does a key past the cap, read as 0, unless the window is the lowest one: then such keys are
+    // kept out by their index); a key is above the guess from the first pattern of the bin after the guess on.
+    int above = 0;
+    auto count = [&](auto lowest) {
+        constexpr bool kLowest = decltype(lowest)::value;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const unsigned h = (unsigned)(it.key[j] >> 32);
+            const unsigned d = h - ps.base;
+#ifdef HORA_CHECKED
+            if ((!kLowest || j < nvalid) && d < ((unsigned)kFineBins << 9)) {
+                unsigned int *fine = reinterpret_cast<unsigned int *>(__cvta_shared_to_generic(ps.fine_shared));
+                atomicAdd(&HORA_AT(fine, d >> 9, kFineBins), 1u);
+            }
+#else
+            // (the lowest window: a key past the cap, read as 0, must not count: its d is pushed out of range)
+            count_if_below(ps.fine_shared, kLowest && j >= nvalid ? 0xFFFFFFFFu : d, (unsigned)kFineBins << 9);
+#endif
+            above += (h >= ps.above_from) && (!kLowest || j < nvalid);
+        }
+    };
+    if (ps.base != 0) count(std::false_type{}); else count(std::true_type{});
+#pragma unroll
+    for (int d = 1; d < LG; d <<= 1) above += __shfl_xor_sync(kFull, above, d);
+    if (gl == 0 && row < ps.N) {
+        *capsum += it.capi;
+        *sum_pg += above;
+        ps.pguess[row] = (unsigned int)above;
+    }
+}
+
+template <int LG, bool VEC2>
+__global__ void __launch_bounds__(kSelThreads, 3)
+select_level0_short(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
+                    const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist_fine,
+                    unsigned int *__restrict__ pguess) {
+    __shared__ unsigned int s_fine[kFineBins];
+    __shared__ long long s_warp[kSelThreads / kWarp];
+    for (int b = threadIdx.x; b < kFineBins; b += kSelThreads) s_fine[b] = 0;
+    __syncthreads();
+    const int lane = lane_id();
+    const unsigned W0 = (unsigned)hdr->win_lo << kFineBits;
+    int t_guess = (int)(hdr->guess_hi >> 9) - (int)W0;
+    t_guess = t_guess < 0 ? 0 : (t_guess >= kFineBins ? kFineBins - 1 : t_guess);
+    constexpr int R = kWarp / LG;
+    Level0ShortPass ps;
+    ps.cap = cap;
+    ps.cap_scalar = cap_scalar;
+    ps.N = (int32_t)N;
+    ps.n_items = (int32_t)((N + R - 1) / R);
+    ps.ld = ld;
+    ps.keys = reinterpret_cast<const unsigned long long *>(gains);
+    ps.pguess = pguess;
+    ps.fine_shared = (unsigned)__cvta_generic_to_shared(s_fine);
+    ps.base = W0 << 9;
+    const unsigned long long g64 = ((unsigned long long)W0 + (unsigned)t_guess + 1ull) << 9;
+    ps.above_from = g64 > 0xFFFFFFFFull ? 0xFFFFFFFFu : (unsigned)g64;   // (no valid key is that high)
+    const int32_t item0 = (int32_t)(blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5));
+    const int32_t stride = (int32_t)(gridDim.x * (kSelThreads / kWarp));   // (item + 3 stride stays far below 2^31)
+    int32_t capsum = 0, sum_pg = 0;                            // per thread: at most 2^31 / (32 * a wave of warps)
+    unsigned bad = 0;
+    // two items in flight, in two fixed register sets, as in select_level0; caps one item further ahead
+    Level0Short<LG> A, Bq;
+    int32_t cap_b = level0_short_cap<LG>(ps, item0 + stride, lane, &bad);
+    level0_short_fetch<LG, VEC2>(A, ps, level0_short_cap<LG>(ps, item0, lane, &bad), item0, lane);
+    for (int32_t item = item0; item < ps.n_items; item += 2 * stride) {
+        const int32_t cap_a = level0_short_cap<LG>(ps, item + 2 * stride, lane, &bad);
+        level0_short_fetch<LG, VEC2>(Bq, ps, cap_b, item + stride, lane);
+        level0_short_process<LG>(A, ps, item, lane, &capsum, &sum_pg, &bad);
+        cap_b = level0_short_cap<LG>(ps, item + 3 * stride, lane, &bad);
+        level0_short_fetch<LG, VEC2>(A, ps, cap_a, item + 2 * stride, lane);
+        if (Bq.capi >= 0) level0_short_process<LG>(Bq, ps, item + stride, lane, &capsum, &sum_pg, &bad);
+    }
+    level0_finish(hdr, hist_fine, s_fine, W0, t_guess, capsum, sum_pg, bad != 0, B, s_warp);
+}
+
 // The plain pass, for the rare case that the window missed: a warp per row, every key counted on its top 13
 // bits; the last CTA selects that digit and the selection goes on from there.  (The counts above the guess
 // that level 0 stored mean little then; level 1 falls back to searching the rows.)
@@ -1715,10 +1881,15 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
             return HORA_ERR_CUDA;
     } else if (ld > 128) {
         launch_level0<8>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
-    } else if (ld > 64) {
-        launch_level0<4>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
-    } else {
-        launch_level0<2>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
+    } else {                                              // short rows share a warp
+        auto go = [&](auto kernel, int lg) {
+            const int64_t items = (N + kWarp / lg - 1) / (kWarp / lg);
+            kernel<<<clamp_grid((items + rows_per_cta - 1) / rows_per_cta, 3), kSelThreads, 0, s>>>(
+                cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_fine, w.pguess);
+        };
+        if (ld > 64) { if (vec2) go(select_level0_short<16, true>, 16); else go(select_level0_short<16, false>, 16); }
+        else if (ld > 32) { if (vec2) go(select_level0_short<8, true>, 8); else go(select_level0_short<8, false>, 8); }
+        else { if (vec2) go(select_level0_short<4, true>, 4); else go(select_level0_short<4, false>, 4); }
     }
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_stop, s);
     if (B > 0)                                            // stands down at once unless the window missed
