@@ -279,24 +279,52 @@ select_estimate(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, 
 // instructions, and those, not memory, set the time.
 // The pass also checks that the row is finite, non-negative and non-increasing and sums the caps.
 
-// E sorted keys of one lane, as high words; `valid` of them exist (the rest were read as 0).  Counts the window
-// keys in s_fine and returns how many keys are above the guess.  ts = prefix23 - W0 is negative below the window
-// and >= kFineBins above it; the guess is t_guess in [0, kFineBins).
-template <int E>
-__device__ __forceinline__ int window_count(const unsigned (&h)[E], int valid, unsigned W0, int t_guess,
-                                            unsigned int *s_fine) {
-    const int ts_first = (int)(h[0] >> 9) - (int)W0, ts_last = (int)(h[E - 1] >> 9) - (int)W0;
-    if (valid >= E && ts_last >= kFineBins) return E;      // the whole lane above the window
-    if (ts_first < 0 || valid <= 0) return 0;              // the whole lane below it
-    int above = 0;
-#pragma unroll
-    for (int m = 0; m < E; ++m) {
-        const int ts = (int)(h[m] >> 9) - (int)W0;
-        if (m < valid) {
-            if ((unsigned)ts < (unsigned)kFineBins) atomicAdd(&HORA_AT(s_fine, ts, kFineBins), 1u);
-            above += ts > t_guess;
-        }
+// The window as the per-key code sees it: d = h - base is below `kFineBins << 9` exactly for the high words h of
+// window keys (it wraps far above that for a key below the window; so does a key past the cap, which every caller
+// presents as 0, unless the window is the lowest one: then such keys are kept out by their index), and a key is
+// above the guess from the first pattern of the bin after the guess on.
+struct WindowView {
+    unsigned fine_shared;          // shared-window address of the fine histogram
+    unsigned base;                 // first high word of the window
+    unsigned above_from;           // first high word above the guess
+    __device__ __forceinline__ void set(unsigned int *s_fine, unsigned W0, int t_guess) {
+        fine_shared = (unsigned)__cvta_generic_to_shared(s_fine);
+        base = W0 << 9;
+        const unsigned long long g64 = ((unsigned long long)W0 + (unsigned)t_guess + 1ull) << 9;
+        above_from = g64 > 0xFFFFFFFFull ? 0xFFFFFFFFu : (unsigned)g64;   // (no valid key is that high)
     }
+};
+
+// fine[d >> 9] += 1 where d < limit, as one predicated instruction (an `if` around the atomic compiled to a
+// branch per key); the address is formed for every key and used only under the predicate
+__device__ __forceinline__ void count_if_below(unsigned fine_shared, unsigned d, unsigned limit) {
+    const unsigned addr = fine_shared + (d >> 9) * 4u;
+    asm volatile("{\n .reg .pred p;\n setp.lt.u32 p, %1, %2;\n @p red.shared.add.u32 [%0], 1;\n}" ::"r"(addr), "r"(d), "r"(limit)
+                 : "memory");
+}
+
+// E keys of one lane, as high words; the first `nvalid` exist, the rest are 0.  Counts the window keys in the fine
+// histogram and returns how many keys are above the guess.  No branch but the one on the window's position.
+template <int E>
+__device__ __forceinline__ int window_count(const unsigned (&h)[E], int nvalid, const WindowView &wv) {
+    int above = 0;
+    auto count = [&](auto lowest) {
+        constexpr bool kLowest = decltype(lowest)::value;
+#pragma unroll
+        for (int j = 0; j < E; ++j) {
+            const unsigned d = h[j] - wv.base;
+#ifdef HORA_CHECKED
+            if ((!kLowest || j < nvalid) && d < ((unsigned)kFineBins << 9)) {
+                unsigned int *fine = reinterpret_cast<unsigned int *>(__cvta_shared_to_generic(wv.fine_shared));
+                atomicAdd(&HORA_AT(fine, d >> 9, kFineBins), 1u);
+            }
+#else
+            count_if_below(wv.fine_shared, kLowest && j >= nvalid ? 0xFFFFFFFFu : d, (unsigned)kFineBins << 9);
+#endif
+            above += (h[j] >= wv.above_from) && (!kLowest || j < nvalid);
+        }
+    };
+    if (wv.base != 0) count(std::false_type{}); else count(std::true_type{});
     return above;
 }
 
@@ -556,9 +584,7 @@ struct Level0ShortPass {
     int32_t cap_scalar, N, n_items, ld;
     const unsigned long long *keys;
     unsigned int *pguess;
-    unsigned fine_shared;          // shared-window address of the fine histogram
-    unsigned base;                 // first high word of the window
-    unsigned above_from;           // first high word above the guess
+    WindowView wv;
 };
 
 // 16 zero bytes: where a lane's chunk lies past the cap it reads these instead (a select on the address and an
@@ -599,14 +625,6 @@ __device__ __forceinline__ void level0_short_fetch(Level0Short<LG> &it, const Le
     }
 }
 
-// fine[d >> 9] += 1 where d < limit, as one predicated instruction (an `if` around the atomic compiled to a
-// branch per key); the address is formed for every key and used only under the predicate
-__device__ __forceinline__ void count_if_below(unsigned fine_shared, unsigned d, unsigned limit) {
-    const unsigned addr = fine_shared + (d >> 9) * 4u;
-    asm volatile("{\n .reg .pred p;\n setp.lt.u32 p, %1, %2;\n @p red.shared.add.u32 [%0], 1;\n}" ::"r"(addr), "r"(d), "r"(limit)
-                 : "memory");
-}
-
 template <int LG>
 __device__ __forceinline__ void level0_short_process(const Level0Short<LG> &it, const Level0ShortPass &ps, int32_t item,
                                                      int lane, int32_t *capsum, int32_t *sum_pg, unsigned *bad) {
@@ -625,29 +643,10 @@ __device__ __forceinline__ void level0_short_process(const Level0Short<LG> &it, 
         viol |= gl == 0 && it.key[0] > kKeyInf - 1;
         *bad |= (unsigned)viol;
     }
-    // Window, on the high words: d = h - (first pattern of the window) wraps far above the window's width for a
-    // key below it (so does a key past the cap, read as 0, unless the window is the lowest one: then such keys are
-    // kept out by their index); a key is above the guess from the first pattern of the bin after the guess on.
-    int above = 0;
-    auto count = [&](auto lowest) {
-        constexpr bool kLowest = decltype(lowest)::value;
+    unsigned h[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const unsigned h = (unsigned)(it.key[j] >> 32);
-            const unsigned d = h - ps.base;
-#ifdef HORA_CHECKED
-            if ((!kLowest || j < nvalid) && d < ((unsigned)kFineBins << 9)) {
-                unsigned int *fine = reinterpret_cast<unsigned int *>(__cvta_shared_to_generic(ps.fine_shared));
-                atomicAdd(&HORA_AT(fine, d >> 9, kFineBins), 1u);
-            }
-#else
-            // (the lowest window: a key past the cap, read as 0, must not count: its d is pushed out of range)
-            count_if_below(ps.fine_shared, kLowest && j >= nvalid ? 0xFFFFFFFFu : d, (unsigned)kFineBins << 9);
-#endif
-            above += (h >= ps.above_from) && (!kLowest || j < nvalid);
-        }
-    };
-    if (ps.base != 0) count(std::false_type{}); else count(std::true_type{});
+    for (int j = 0; j < 8; ++j) h[j] = (unsigned)(it.key[j] >> 32);
+    int above = window_count<8>(h, nvalid, ps.wv);
 #pragma unroll
     for (int d = 1; d < LG; d <<= 1) above += __shfl_xor_sync(kFull, above, d);
     if (gl == 0 && row < ps.N) {
@@ -679,10 +678,7 @@ select_level0_short(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t
     ps.ld = ld;
     ps.keys = reinterpret_cast<const unsigned long long *>(gains);
     ps.pguess = pguess;
-    ps.fine_shared = (unsigned)__cvta_generic_to_shared(s_fine);
-    ps.base = W0 << 9;
-    const unsigned long long g64 = ((unsigned long long)W0 + (unsigned)t_guess + 1ull) << 9;
-    ps.above_from = g64 > 0xFFFFFFFFull ? 0xFFFFFFFFu : (unsigned)g64;   // (no valid key is that high)
+    ps.wv.set(s_fine, W0, t_guess);
     const int32_t item0 = (int32_t)(blockIdx.x * (kSelThreads / kWarp) + (threadIdx.x >> 5));
     const int32_t stride = (int32_t)(gridDim.x * (kSelThreads / kWarp));   // (item + 3 stride stays far below 2^31)
     int32_t capsum = 0, sum_pg = 0;                            // per thread: at most 2^31 / (32 * a wave of warps)
@@ -768,7 +764,7 @@ struct CoarseTap {
 template <int E, int LG>
 struct Level0Tap {
     unsigned long long key[E];
-    unsigned int *s_fine;
+    WindowView wv;
     unsigned int *pguess;
     unsigned int *pg_row;          // the count of the prompt being built (null: the row does not exist)
     unsigned W0;
@@ -790,7 +786,7 @@ struct Level0Tap {
         unsigned h[E];
 #pragma unroll
         for (int m = 0; m < E; ++m) h[m] = (unsigned)(key[m] >> 32);
-        int above = window_count<E>(h, capi - k, W0, t_guess, s_fine);
+        int above = window_count<E>(h, capi - k, wv);
         if (LG == kWarp) {
             above = __reduce_add_sync(kFull, above);
         } else {
@@ -850,12 +846,12 @@ gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ 
     for (int b = threadIdx.x; b < kFineBins; b += kSelThreads) s_fine[b] = 0;
     __syncthreads();
     Level0Tap<E, LG> tap;
-    tap.s_fine = s_fine;
     tap.pguess = pguess;
     tap.pg_row = pguess;
     tap.W0 = (unsigned)hdr->win_lo << kFineBits;
     const int t_guess = (int)(hdr->guess_hi >> 9) - (int)tap.W0;
     tap.t_guess = t_guess < 0 ? 0 : (t_guess >= kFineBins ? kFineBins - 1 : t_guess);
+    tap.wv.set(s_fine, tap.W0, tap.t_guess);
     tap.row_above = 0;
     tap.sum_pg = 0;
     tap.capsum = 0;
@@ -1879,15 +1875,17 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         if (launch_fused<8>(vec2, B > 0, grid_est, every, gridf, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
                             B, w) != cudaSuccess)
             return HORA_ERR_CUDA;
-    } else if (ld > 128) {
+    } else if (ld > 256 || (ld > 128 && cap == nullptr && cap_scalar == ld)) {
+        // long rows, and whole rows of up to 256 keys (slices settled by votes: 0.35 against 0.37 ms at 2^20 x 256)
         launch_level0<8>(vec2, grid0, s, cap, cap_scalar, N, ld, gains, B, w);
-    } else {                                              // short rows share a warp
+    } else {                                              // short rows share a warp; ragged ones of up to 256 keys
         auto go = [&](auto kernel, int lg) {
             const int64_t items = (N + kWarp / lg - 1) / (kWarp / lg);
             kernel<<<clamp_grid((items + rows_per_cta - 1) / rows_per_cta, 3), kSelThreads, 0, s>>>(
                 cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_fine, w.pguess);
         };
-        if (ld > 64) { if (vec2) go(select_level0_short<16, true>, 16); else go(select_level0_short<16, false>, 16); }
+        if (ld > 128) { if (vec2) go(select_level0_short<32, true>, 32); else go(select_level0_short<32, false>, 32); }
+        else if (ld > 64) { if (vec2) go(select_level0_short<16, true>, 16); else go(select_level0_short<16, false>, 16); }
         else if (ld > 32) { if (vec2) go(select_level0_short<8, true>, 8); else go(select_level0_short<8, false>, 8); }
         else { if (vec2) go(select_level0_short<4, true>, 4); else go(select_level0_short<4, false>, 4); }
     }
