@@ -142,6 +142,7 @@ template <bool VEC4>
 __global__ void __launch_bounds__(kAdvWarps *kWarp, 3)
 group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restrict__ off, int64_t N, int32_t mode,
                        double eps, int32_t ddof, float *__restrict__ adv, int32_t *status_dev) {
+    pdl_enter();
     extern __shared__ __align__(16) unsigned char s_raw[];
     AdvWarpSmem &sm = reinterpret_cast<AdvWarpSmem *>(s_raw)[threadIdx.x >> 5];
     const int lane = lane_id();
@@ -150,14 +151,22 @@ group_advantage_kernel(const float *__restrict__ rewards, const int64_t *__restr
     const int64_t stride = (int64_t)gridDim.x * kAdvWarps;
     const int64_t n_blocks = (N + kWarp - 1) / kWarp;
     const int64_t n_all = __ldg(off + N);                     // nothing is read at or beyond this element
+    // a lane's two offsets of the warp's NEXT 32 groups are fetched while the current ones are worked on
+    auto fetch_offsets = [&](int64_t blk, int64_t &s, int64_t &e) {
+        s = e = 0;
+        const int64_t g = blk * kWarp + lane;
+        if (blk < n_blocks && g < N) {
+            s = __ldg(off + g);
+            e = __ldg(off + g + 1);
+        }
+    };
+    int64_t nxt_s, nxt_e;
+    fetch_offsets(warp0, nxt_s, nxt_e);
     for (int64_t blk = warp0; blk < n_blocks; blk += stride) {
         const int64_t g0 = blk * kWarp;
         const int ng = (int)((N - g0 < kWarp) ? N - g0 : kWarp);
-        int64_t my_s = 0, my_e = 0;
-        if (lane < ng) {
-            my_s = __ldg(off + g0 + lane);
-            my_e = __ldg(off + g0 + lane + 1);
-        }
+        int64_t my_s = nxt_s, my_e = nxt_e;
+        fetch_offsets(blk + stride, nxt_s, nxt_e);
         if (my_e < my_s || my_s < 0 || my_e > n_all) {
             raise_status(status_dev, HORA_ERR_INVALID_VALUE);
             my_e = my_s = 0;                                  // treat as empty: nothing is read or written for it
@@ -334,9 +343,8 @@ extern "C" hora_status_t hora_group_advantage(const float *rewards, const int64_
     auto go = [&](auto kernel) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAdvSmem);
         if (e != cudaSuccess) return e;
-        kernel<<<grid, kAdvWarps * kWarp, kAdvSmem, static_cast<cudaStream_t>(stream)>>>(rewards, group_offsets, N, mode,
-                                                                                         (double)eps, ddof, adv, status_dev);
-        return cudaSuccess;
+        return launch_pdl(kernel, grid, kAdvWarps * kWarp, kAdvSmem, static_cast<cudaStream_t>(stream), rewards, group_offsets,
+                          N, mode, (double)eps, ddof, adv, status_dev);
     };
     if ((vec4 ? go(group_advantage_kernel<true>) : go(group_advantage_kernel<false>)) != cudaSuccess) return HORA_ERR_CUDA;
     count_launches(1);

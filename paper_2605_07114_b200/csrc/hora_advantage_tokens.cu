@@ -22,6 +22,7 @@ advantage_tokens_kernel(const float *__restrict__ rewards, const int64_t *__rest
                         const int64_t *__restrict__ off, int64_t R, int64_t T, int64_t chunk, int32_t mode, double eps,
                         int32_t ddof, int32_t weight_mode, double length_const, float *__restrict__ out,
                         float *__restrict__ out_w, int32_t *status_dev) {
+    pdl_enter();
     __shared__ int32_t s_rel[kStage + 1];
     __shared__ float s_adv[kStage];
     __shared__ float s_w[WEIGHT ? kStage : 1];
@@ -111,10 +112,9 @@ extern "C" hora_status_t hora_group_advantage_tokens(const float *rewards, const
     const bool vec4 = ((reinterpret_cast<uintptr_t>(token_adv) | reinterpret_cast<uintptr_t>(token_weight)) & 15u) == 0;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 #define HORA_LAUNCH_AT(V, W)                                                                                        \
-    advantage_tokens_kernel<V, W><<<(int)grid, kBcThreads, 0, st>>>(rewards, group_offsets, N, token_offsets, R, T, \
-                                                                     chunk, mode, (double)eps, ddof, weight_mode,    \
-                                                                     (double)length_const, token_adv, token_weight,  \
-                                                                     status_dev)
+    launch_pdl(advantage_tokens_kernel<V, W>, (int)grid, kBcThreads, 0, st, rewards, group_offsets, N, token_offsets, \
+               R, T, chunk, mode, (double)eps, ddof, weight_mode, (double)length_const, token_adv, token_weight,      \
+               status_dev)
     if (token_weight != nullptr) { if (vec4) HORA_LAUNCH_AT(true, true); else HORA_LAUNCH_AT(false, true); }
     else                         { if (vec4) HORA_LAUNCH_AT(true, false); else HORA_LAUNCH_AT(false, false); }
 #undef HORA_LAUNCH_AT

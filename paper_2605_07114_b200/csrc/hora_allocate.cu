@@ -225,6 +225,7 @@ __device__ void place_window(AllocHeader *hdr, const unsigned long long *hist, i
 __global__ void __launch_bounds__(kSelThreads)
 select_estimate(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld, int64_t every,
                 const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist) {
+    pdl_enter();
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
@@ -537,6 +538,7 @@ __global__ void __launch_bounds__(kSelThreads, level0_per_sm<E>())
 select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
               const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist_fine,
               unsigned int *__restrict__ pguess) {
+    pdl_enter();
     __shared__ unsigned int s_fine[kFineBins];             // the window's 23-bit bins
     __shared__ long long s_warp[kSelThreads / kWarp];
     for (int b = threadIdx.x; b < kFineBins; b += kSelThreads) s_fine[b] = 0;
@@ -661,6 +663,7 @@ __global__ void __launch_bounds__(kSelThreads, 3)
 select_level0_short(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
                     const double *__restrict__ gains, int64_t B, AllocHeader *hdr, unsigned long long *hist_fine,
                     unsigned int *__restrict__ pguess) {
+    pdl_enter();
     __shared__ unsigned int s_fine[kFineBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     for (int b = threadIdx.x; b < kFineBins; b += kSelThreads) s_fine[b] = 0;
@@ -704,6 +707,7 @@ select_level0_short(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t
 __global__ void __launch_bounds__(kSelThreads)
 select_level0_full(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, int32_t ld,
                    const double *__restrict__ gains, AllocHeader *hdr, unsigned long long *hist) {
+    pdl_enter();
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     if (*(volatile int32_t *)&hdr->status != 0 || hdr->l0_miss == 0) return;
@@ -805,6 +809,7 @@ __global__ void __launch_bounds__(kSelThreads)
 select_estimate_fused(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
                       const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
                       int64_t N, int32_t ld, int64_t every, int64_t B, AllocHeader *hdr, unsigned long long *hist) {
+    pdl_enter();
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
@@ -841,6 +846,7 @@ gains_level0_fused(const double *__restrict__ alpha, const double *__restrict__ 
                    const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
                    int64_t N, int32_t ld, double *__restrict__ gains, int64_t B, AllocHeader *hdr,
                    unsigned long long *hist_fine, unsigned int *__restrict__ pguess) {
+    pdl_enter();
     __shared__ unsigned int s_fine[kFineBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     for (int b = threadIdx.x; b < kFineBins; b += kSelThreads) s_fine[b] = 0;
@@ -895,6 +901,7 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
               const unsigned int *__restrict__ pguess, int2 *__restrict__ rowstate,
               int32_t *__restrict__ active, unsigned long long *__restrict__ cand_key,
               int32_t *__restrict__ cand_row, long long *bsum_hi, double *__restrict__ objrow) {
+    pdl_enter();
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     if (*(volatile int32_t *)&hdr->status != 0) return;
@@ -1344,6 +1351,7 @@ select_tail(int64_t N, int32_t ld, const double *__restrict__ gains, int64_t B, 
             unsigned long long *hist_all, int2 *__restrict__ rowstate, const int32_t *__restrict__ active,
             long long *bsum_hi, long long *bsum_t, int64_t NB, const unsigned long long *__restrict__ cand_key,
             const int32_t *__restrict__ cand_row) {
+    pdl_enter();
     __shared__ unsigned int s_hist[kBins];
     __shared__ unsigned long long s_keys[kListSmall];
     __shared__ long long s_warp[kSelThreads / kWarp];
@@ -1369,6 +1377,7 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
               const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
               int64_t N, int32_t ld, const double *__restrict__ gains, AllocHeader *hdr, int2 *__restrict__ rowstate,
               int32_t *__restrict__ rowslot, unsigned long long *tkeys, unsigned long long *tcounts) {
+    pdl_enter();
     __shared__ long long s_warp[kSelThreads / kWarp];
     if (*(volatile int32_t *)&hdr->status != 0) return;
     const unsigned long long lam_key = hdr->prefix_key;
@@ -1446,6 +1455,7 @@ constexpr size_t kExactRankSmem = (size_t)kMaxTypes * (2 * sizeof(UBig) + sizeof
 __global__ void __launch_bounds__(kExactRankThreads)
 exact_rank(int64_t B, AllocHeader *hdr, const unsigned long long *__restrict__ tkeys,
            const unsigned long long *__restrict__ tcounts, int32_t *__restrict__ tlabel) {
+    pdl_enter();
     extern __shared__ __align__(16) unsigned char s_rank_raw[];
     UBig *s_num = reinterpret_cast<UBig *>(s_rank_raw);
     UBig *s_den = s_num + kMaxTypes;
@@ -1513,6 +1523,7 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
            int64_t N, int32_t ld, const double *__restrict__ gains, int mode, int64_t B, AllocHeader *hdr,
            int2 *__restrict__ rowstate, const int32_t *__restrict__ rowslot, const int32_t *__restrict__ tlabel,
            long long *bsum_hi, long long *bsum_t, int64_t NB) {
+    pdl_enter();
     __shared__ long long s_warp[kSelThreads / kWarp];
     const bool failed = *(volatile int32_t *)&hdr->status != 0;
     long long hi_sum = 0, t_sum = 0;
@@ -1571,6 +1582,7 @@ select_out(const double *__restrict__ alpha, const double *__restrict__ beta, do
            const int2 *__restrict__ rowstate, const double *__restrict__ objrow, const long long *__restrict__ bpre_hi,
            const long long *__restrict__ bpre_t, double *objpart, int64_t NB, int32_t *__restrict__ delta,
            int32_t *__restrict__ G, int64_t *__restrict__ offsets, int vec, hora_alloc_info *info) {
+    pdl_enter();
     __shared__ long long s_warp[kSelThreads / kWarp];
     __shared__ double s_obj[kSelThreads / kWarp];
     const int32_t status = *(volatile int32_t *)&hdr->status;
@@ -1741,7 +1753,7 @@ static void launch_level0(bool vec2, int grid, cudaStream_t s, const int32_t *ca
     const bool one = ld <= kWarp * E;                     // an item is a whole row
     grid = clamp_grid((N * ((ld + kWarp * E - 1) / (kWarp * E)) + kSelThreads / kWarp - 1) / (kSelThreads / kWarp),
                       level0_per_sm<E>());                // exactly what is resident at once
-    auto go = [&](auto kernel) { kernel<<<grid, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_fine, w.pguess); };
+    auto go = [&](auto kernel) { launch_pdl(kernel, grid, kSelThreads, 0, s, cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_fine, w.pguess); };
     if (vec2) { if (one) go(select_level0<E, true, true>); else go(select_level0<E, true, false>); }
     else { if (one) go(select_level0<E, false, true>); else go(select_level0<E, false, false>); }
 }
@@ -1752,11 +1764,11 @@ static cudaError_t launch_fused(bool vec2, bool estimate, int grid_est, int64_t 
                                 int32_t G0, const int32_t *cap, int32_t cap_scalar, int64_t N, int32_t ld, int64_t B,
                                 const Workspace &w) {
     if (estimate)
-        select_estimate_fused<E><<<grid_est, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N,
-                                                                  ld, every, B, w.hdr, w.hist_est);
+        launch_pdl(select_estimate_fused<E>, grid_est, kSelThreads, 0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar,
+                   N, ld, every, B, w.hdr, w.hist_est);
     auto go = [&](auto kernel) {
-        kernel<<<grid, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, w.gains, B, w.hdr,
-                                            w.hist_fine, w.pguess);
+        launch_pdl(kernel, grid, kSelThreads, 0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, w.gains, B, w.hdr,
+                   w.hist_fine, w.pguess);
     };
     // lanes per row as in hora_gains: short rows share a warp
     if (ld > 128) { if (vec2) go(gains_level0_fused<E, true, kWarp>); else go(gains_level0_fused<E, false, kWarp>); }
@@ -1864,7 +1876,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     const int grid_est = clamp_grid((n_sample + 2 * rows_per_cta - 1) / (2 * rows_per_cta), 2);
     mark_stage(0, s);
     if (B > 0 && !fused)
-        select_estimate<<<grid_est, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, every, gains, B, w.hdr, w.hist_est);
+        launch_pdl(select_estimate, grid_est, kSelThreads, 0, s, cap, cap_scalar, N, ld, every, gains, B, w.hdr, w.hist_est);
     const int grid0 = clamp_grid((N + rows_per_cta - 1) / rows_per_cta, 3);
     const int grid1 = clamp_grid((N + kSelThreads - 1) / kSelThreads, kLevel1PerSm);
     const cudaEvent_t prof_start = g_prof_start, prof_stop = g_prof_stop;
@@ -1881,8 +1893,8 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     } else {                                              // short rows share a warp; ragged ones of up to 256 keys
         auto go = [&](auto kernel, int lg) {
             const int64_t items = (N + kWarp / lg - 1) / (kWarp / lg);
-            kernel<<<clamp_grid((items + rows_per_cta - 1) / rows_per_cta, 3), kSelThreads, 0, s>>>(
-                cap, cap_scalar, N, ld, gains, B, w.hdr, w.hist_fine, w.pguess);
+            launch_pdl(kernel, clamp_grid((items + rows_per_cta - 1) / rows_per_cta, 3), kSelThreads, 0, s, cap, cap_scalar, N,
+                       ld, gains, B, w.hdr, w.hist_fine, w.pguess);
         };
         if (ld > 128) { if (vec2) go(select_level0_short<32, true>, 32); else go(select_level0_short<32, false>, 32); }
         else if (ld > 64) { if (vec2) go(select_level0_short<16, true>, 16); else go(select_level0_short<16, false>, 16); }
@@ -1891,7 +1903,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     }
     if (prof_start != nullptr && prof_stop != nullptr) cudaEventRecord(prof_stop, s);
     if (B > 0)                                            // stands down at once unless the window missed
-        select_level0_full<<<grid0, kSelThreads, 0, s>>>(cap, cap_scalar, N, ld, gains, w.hdr, w.hist_coarse);
+        launch_pdl(select_level0_full, grid0, kSelThreads, 0, s, cap, cap_scalar, N, ld, gains, w.hdr, w.hist_coarse);
     mark_stage(2, s);
     const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
     // utilities of the rows whose Delta is final after level 1 are evaluated there (not in exact mode, where the
@@ -1899,13 +1911,13 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
     double *objrow = (B > 0 && !exact && !(flags & HORA_FLAG_SKIP_OBJECTIVE)) ? w.objrow : nullptr;
     if (B > 0) {
         if (vec2)
-            select_level1<true><<<grid1, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains,
-                                                              w.hdr, w.hist_lv + kBins, w.pguess, w.rowstate,
-                                                              w.active, w.cand_key, w.cand_row, w.bsum_hi, objrow);
+            launch_pdl(select_level1<true>, grid1, kSelThreads, 0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
+                       gains, w.hdr, w.hist_lv + kBins, w.pguess, w.rowstate, w.active, w.cand_key, w.cand_row, w.bsum_hi,
+                       objrow);
         else
-            select_level1<false><<<grid1, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains,
-                                                               w.hdr, w.hist_lv + kBins, w.pguess, w.rowstate,
-                                                               w.active, w.cand_key, w.cand_row, w.bsum_hi, objrow);
+            launch_pdl(select_level1<false>, grid1, kSelThreads, 0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
+                       gains, w.hdr, w.hist_lv + kBins, w.pguess, w.rowstate, w.active, w.cand_key, w.cand_row, w.bsum_hi,
+                       objrow);
         mark_stage(3, s);
         {
             int64_t N_ = N, B_ = B, NB_ = NB;
@@ -1929,26 +1941,25 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         }
         mark_stage(4, s);
         if (exact) {
-            exact_collect<<<grid_rows, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
-                                                            gains, w.hdr, w.rowstate, w.rowslot, w.tkeys, w.tcounts);
+            launch_pdl(exact_collect, grid_rows, kSelThreads, 0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
+                       gains, w.hdr, w.rowstate, w.rowslot, w.tkeys, w.tcounts);
             if (cudaFuncSetAttribute(exact_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kExactRankSmem) !=
                 cudaSuccess)
                 launch_failed = true;
-            exact_rank<<<1, kExactRankThreads, kExactRankSmem, s>>>(B, w.hdr, w.tkeys, w.tcounts, w.tlabel);
-            select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 0, N, ld, gains, 2, B,
-                                                       w.hdr, w.rowstate, w.rowslot, w.tlabel, w.bsum_hi, w.bsum_t, NB);
+            launch_pdl(exact_rank, 1, kExactRankThreads, kExactRankSmem, s, B, w.hdr, w.tkeys, w.tcounts, w.tlabel);
+            launch_pdl(select_sum, (int)NB, kSelThreads, 0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 0, N, ld, gains,
+                       2, B, w.hdr, w.rowstate, w.rowslot, w.tlabel, w.bsum_hi, w.bsum_t, NB);
         }
     } else {
         if (cudaMemsetAsync(w.rowstate, 0, sizeof(int2) * (size_t)N, s) != cudaSuccess) return HORA_ERR_CUDA;
-        select_sum<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 1, N, ld, gains, 0, B,
-                                                   w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi, w.bsum_t, NB);
+        launch_pdl(select_sum, (int)NB, kSelThreads, 0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, 1, N, ld, gains, 0,
+                   B, w.hdr, w.rowstate, nullptr, nullptr, w.bsum_hi, w.bsum_t, NB);
     }
     mark_stage(5, s);
     const int out_vec = ((reinterpret_cast<uintptr_t>(delta) | reinterpret_cast<uintptr_t>(G) |
                           reinterpret_cast<uintptr_t>(group_offsets)) & 15u) == 0;
-    select_out<<<(int)NB, kSelThreads, 0, s>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, flags, w.hdr,
-                                               w.rowstate, objrow, w.bsum_hi, w.bsum_t, w.objpart, NB, delta, G,
-                                               group_offsets, out_vec, info_dev);
+    launch_pdl(select_out, (int)NB, kSelThreads, 0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, B, flags,
+               w.hdr, w.rowstate, objrow, w.bsum_hi, w.bsum_t, w.objpart, NB, delta, G, group_offsets, out_vec, info_dev);
     mark_stage(6, s);
     count_launches(B > 0 ? (exact ? 9 : 6) : 3);
     if (launch_failed) return HORA_ERR_CUDA;

@@ -6,8 +6,9 @@
 // and one CTA solves one segment entirely in shared memory:
 //   1  gain rows of the segment's prompts, computed with the arithmetic of hora_gains (same bits), never
 //      written to global memory;
-//   2  the B_s-th largest key, built bit by bit from the top by one warp: a step is a binary search per sorted
-//      row (inside a range that every step narrows) and one warp sum;
+//   2  the B_s-th largest key, built two bits a step from the top by one warp: a step is a binary search per sorted
+//      row (inside a range that every step narrows) and three warp sums; with at most 32 rows a lane keeps its
+//      row's range in registers and the last keys left in the interval are ranked directly;
 //   3  per row the number of keys above and equal to the threshold (binary search in the sorted row);
 //   4  ties: in prompt order (fp64 equality), or, in exact mode, by exact rational comparison of the at
 //      most one candidate per row that lies within 2^-30 of the threshold (pairwise, cross-multiplied);
@@ -65,8 +66,29 @@ __device__ __forceinline__ BatchedRows carve_rows(unsigned char *base, int rows_
     return r;
 }
 
-template <int E>
-__global__ void __launch_bounds__(kBThreads, 3)
+__host__ __device__ inline size_t batched_row_stride(int32_t ld) { return (size_t)ld | 1u; }
+
+// Three binary searches in lockstep over keys[lo, hi) of one sorted (non-increasing) row: a_k = first position
+// whose key is below t_k, i.e. the number of keys >= t_k given that lo keys are known to be and hi is the most.
+__device__ __forceinline__ void search3(const unsigned long long *rk, int lo, int hi, int32_t ld, unsigned long long t1,
+                                        unsigned long long t2, unsigned long long t3, int &a1, int &a2, int &a3) {
+    int z1 = hi, z2 = hi, z3 = hi;
+    a1 = a2 = a3 = lo;
+    while (a1 < z1 || a2 < z2 || a3 < z3) {
+        const int m1 = (a1 + z1) >> 1, m2 = (a2 + z2) >> 1, m3 = (a3 + z3) >> 1;
+        const unsigned long long k1 = HORA_AT(rk, m1 < hi ? m1 : lo, ld), k2 = HORA_AT(rk, m2 < hi ? m2 : lo, ld),
+                                 k3 = HORA_AT(rk, m3 < hi ? m3 : lo, ld);
+        if (a1 < z1) { if (k1 >= t1) a1 = m1 + 1; else z1 = m1; }
+        if (a2 < z2) { if (k2 >= t2) a2 = m2 + 1; else z2 = m2; }
+        if (a3 < z3) { if (k3 >= t3) a3 = m3 + 1; else z3 = m3; }
+    }
+}
+
+// NT threads per CTA: 256, or 128 when no segment of the call has more than 32 prompts.  The selection is a chain of
+// dependent steps by one warp, so what an SM gets through is set by how many segments it holds at once: shared
+// memory has room for five of the paper's 15-prompt segments, the registers of 256 threads for three CTAs only.
+template <int E, int NT>
+__global__ void __launch_bounds__(NT, NT == 128 ? 5 : 3)
 allocate_batched_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
                         const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
                         int32_t ld, const int64_t *__restrict__ seg_off, const int64_t *__restrict__ budgets, int64_t S,
@@ -77,6 +99,10 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
     const BatchedRows rw = carve_rows(s_raw + sizeof(BatchedSmemFixed), rows_cap);
     unsigned long long *keys =
         reinterpret_cast<unsigned long long *>(s_raw + sizeof(BatchedSmemFixed) + (size_t)rows_cap * kBRowBytes);
+    // Rows sit an odd number of keys apart: the selection has a lane per row probing the same column of many rows
+    // at once, and with an even stride (ld = 360: rows 16 banks apart) those probes met in two banks.
+    const size_t lds = batched_row_stride(ld);
+    constexpr int kWarps = NT / kWarp;
     const int lane = lane_id(), warp = threadIdx.x >> 5;
     const bool exact = (flags & HORA_FLAG_EXACT_INT) != 0;
     for (int64_t s = blockIdx.x; s < S; s += gridDim.x) {
@@ -88,20 +114,20 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         __syncthreads();
         // ---- 1: gain rows into shared memory (a warp per row) ----
         Posterior nxt = warp < n ? load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, r0 + warp) : Posterior{};
-        for (int r = warp; r < n; r += kBWarps) {
+        for (int r = warp; r < n; r += kWarps) {
             const Posterior p = nxt;                          // the next row's inputs are fetched while this row is built
-            if (r + kBWarps < n) nxt = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, r0 + r + kBWarps);
+            if (r + kWarps < n) nxt = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, r0 + r + kWarps);
             if (!p.ok && lane == 0) sm.status = HORA_ERR_INVALID_VALUE;
             const double a = p.ok ? p.a : 1.0, b = p.ok ? p.b : 1.0;
-            if (lane == 0) { rw.a[r] = a; rw.b[r] = b; rw.cap[r] = p.cap; }
+            if (lane == 0) { rw.a[r] = a; rw.b[r] = b; rw.cap[r] = p.cap; rw.lo[r] = 0; rw.hi[r] = p.cap; }
             double carry = 1.0;
-            double *out = reinterpret_cast<double *>(keys + (size_t)r * ld);
+            double *out = reinterpret_cast<double *>(keys + (size_t)r * lds);
             for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E)
                 gains_chunk<E, false, false>(a, b, a + b, p.cap, ld, k0, lane, carry, out, nullptr, nullptr);
         }
         __syncthreads();
         long long sum_cap;
-        block_exclusive_sum(threadIdx.x < n ? rw.cap[threadIdx.x] : 0, &sum_cap, sm.warp_tmp);
+        block_exclusive_sum<NT>(threadIdx.x < n ? rw.cap[threadIdx.x] : 0, &sum_cap, sm.warp_tmp);
         if (threadIdx.x == 0 && sm.status == HORA_OK && B > sum_cap) sm.status = HORA_ERR_INFEASIBLE;
         __syncthreads();
         // ---- 2: the B-th largest key, by warp 0 ----
@@ -110,17 +136,17 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         // largest one that still has B keys at or above it gives the two bits.  A lane owns rows lane, lane + 32,
         // ...; a row is sorted, so a count is one binary search, and it can only move inside [lo, hi], which every
         // step narrows from both sides: after a few steps a search is a probe or two.  The bits that all keys share
-        // (the sign, most of the exponent) are taken from the largest and the smallest key directly.  About thirty
-        // steps of (three searches in flight, three warp sums) replace six histogram sweeps over every key with
-        // block-wide barriers between them.
+        // (the sign, most of the exponent) are taken from the largest and the smallest key directly.
+        // With at most 32 rows a lane owns ONE row and keeps its range in registers, and the steps stop as soon as no
+        // row has more than one key left in the interval the bits describe (some ten steps of thirty): the keys
+        // left, at most one a lane, are ranked directly.
         if (warp == 0 && sm.status == HORA_OK && B > 0) {
+            const bool small = n <= kWarp;
             unsigned long long kmax = 0ull, kmin = ~0ull;
             for (int r = lane; r < n; r += kWarp) {
                 const int cp = rw.cap[r];
-                rw.lo[r] = 0;
-                rw.hi[r] = cp;
                 if (cp > 0) {
-                    const unsigned long long first = keys[(size_t)r * ld], last_k = keys[(size_t)r * ld + cp - 1];
+                    const unsigned long long first = keys[(size_t)r * lds], last_k = keys[(size_t)r * lds + cp - 1];
                     kmax = first > kmax ? first : kmax;
                     kmin = last_k < kmin ? last_k : kmin;
                 }
@@ -135,28 +161,27 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
             int top = 63 - __clzll((long long)((kmax ^ kmin) | 1ull));
             top |= 1;                                          // steps take bits (top, top - 1), ..., (1, 0)
             unsigned long long prefix = top >= 63 ? 0ull : (kmax >> (top + 1)) << (top + 1);
+            const unsigned long long *my_rk = keys + (size_t)(lane < n ? lane : 0) * lds;
+            int my_lo = 0, my_hi = (small && lane < n) ? rw.cap[lane] : 0;
+            bool wide = true;                                  // some row still has more than one key in the interval
 #pragma unroll 1
-            for (int bit = top; bit >= 1; bit -= 2) {
+            for (int bit = top; bit >= 1 && wide; bit -= 2) {
                 const unsigned long long t1 = prefix | (1ull << (bit - 1)), t2 = prefix | (2ull << (bit - 1)),
                                          t3 = prefix | (3ull << (bit - 1));
-                int c1 = 0, c2 = 0, c3 = 0;
+                int c1 = 0, c2 = 0, c3 = 0, m1 = 0, m2 = 0, m3 = 0;
+                if (small) {
+                    search3(my_rk, my_lo, my_hi, ld, t1, t2, t3, m1, m2, m3);
+                    c1 = m1; c2 = m2; c3 = m3;
+                } else {
 #pragma unroll 1
-                for (int r = lane; r < n; r += kWarp) {
-                    const unsigned long long *rk = keys + (size_t)r * ld;
-                    const int lo = rw.lo[r], hi = rw.hi[r];
-                    int a1 = lo, z1 = hi, a2 = lo, z2 = hi, a3 = lo, z3 = hi;   // first position whose key is below t_k
-                    while (a1 < z1 || a2 < z2 || a3 < z3) {
-                        const int m1 = (a1 + z1) >> 1, m2 = (a2 + z2) >> 1, m3 = (a3 + z3) >> 1;
-                        const unsigned long long k1 = HORA_AT(rk, m1 < hi ? m1 : lo, ld), k2 = HORA_AT(rk, m2 < hi ? m2 : lo, ld),
-                                                 k3 = HORA_AT(rk, m3 < hi ? m3 : lo, ld);
-                        if (a1 < z1) { if (k1 >= t1) a1 = m1 + 1; else z1 = m1; }
-                        if (a2 < z2) { if (k2 >= t2) a2 = m2 + 1; else z2 = m2; }
-                        if (a3 < z3) { if (k3 >= t3) a3 = m3 + 1; else z3 = m3; }
+                    for (int r = lane; r < n; r += kWarp) {
+                        int a1, a2, a3;
+                        search3(keys + (size_t)r * lds, rw.lo[r], rw.hi[r], ld, t1, t2, t3, a1, a2, a3);
+                        c1 += a1; c2 += a2; c3 += a3;
+                        rw.band[r] = a1;                       // (scratch until the tie step)
+                        rw.cnt2[r] = a2;
+                        rw.cnt3[r] = a3;
                     }
-                    c1 += a1; c2 += a2; c3 += a3;
-                    rw.band[r] = a1;                           // (scratch until the tie step)
-                    rw.cnt2[r] = a2;
-                    rw.cnt3[r] = a3;
                 }
                 c1 = __reduce_add_sync(kFull, c1);            // at most 22528 keys in a segment
                 c2 = __reduce_add_sync(kFull, c2);
@@ -164,16 +189,42 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                 // counts decrease with the trial value: take the largest trial that still has B keys at or above it
                 const int pick = (long long)c3 >= B ? 3 : ((long long)c2 >= B ? 2 : ((long long)c1 >= B ? 1 : 0));
                 prefix |= (unsigned long long)pick << (bit - 1);
+                // #keys >= threshold lies between the count of the next larger trial and that of the picked one
+                if (small) {
+                    if (pick == 3) my_hi = m3;
+                    else if (pick == 2) { my_lo = m3; my_hi = m2; }
+                    else if (pick == 1) { my_lo = m2; my_hi = m1; }
+                    else my_lo = m1;
+                    wide = __any_sync(kFull, my_hi - my_lo > 1);
+                } else {
 #pragma unroll 1
-                for (int r = lane; r < n; r += kWarp) {
-                    const int a1 = rw.band[r], a2 = rw.cnt2[r], a3 = rw.cnt3[r];
-                    // #keys >= threshold lies between the count of the next larger trial and that of the picked one
-                    if (pick == 3) rw.hi[r] = a3;
-                    else if (pick == 2) { rw.lo[r] = a3; rw.hi[r] = a2; }
-                    else if (pick == 1) { rw.lo[r] = a2; rw.hi[r] = a1; }
-                    else rw.lo[r] = a1;
+                    for (int r = lane; r < n; r += kWarp) {
+                        const int a1 = rw.band[r], a2 = rw.cnt2[r], a3 = rw.cnt3[r];
+                        if (pick == 3) rw.hi[r] = a3;
+                        else if (pick == 2) { rw.lo[r] = a3; rw.hi[r] = a2; }
+                        else if (pick == 1) { rw.lo[r] = a2; rw.hi[r] = a1; }
+                        else rw.lo[r] = a1;
+                    }
                 }
             }
+            if (!wide) {
+                // keys at or above the interval: sum of lo; the threshold is the need-th largest of the keys left
+                const long long need = B - (long long)__reduce_add_sync(kFull, my_lo);
+                const bool has = my_hi > my_lo;
+                const unsigned long long mine = has ? my_rk[my_lo] : 0ull;
+                int gt = 0, ge = 0;
+                for (int j = 0; j < n; ++j) {
+                    const unsigned long long other = __shfl_sync(kFull, mine, j);
+                    const bool other_has = __shfl_sync(kFull, (int)has, j) != 0;
+                    gt += other_has && other > mine;
+                    ge += other_has && other >= mine;
+                }
+                const unsigned hit = __ballot_sync(kFull, has && gt < need && need <= ge);
+                // (B keys exist and fewer than B lie above the interval, so some key qualifies; equal keys agree)
+                prefix = __shfl_sync(kFull, mine, hit ? __ffs(hit) - 1 : 0);
+                if (hit == 0u && lane == 0) sm.status = HORA_ERR_INTERNAL;
+            }
+            if (small && lane < n) { rw.lo[lane] = my_lo; rw.hi[lane] = my_hi; }   // where the count pass starts from
             if (lane == 0) sm.lam_key = prefix;
         }
         __syncthreads();
@@ -181,10 +232,11 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         const unsigned long long lam_key = prefix;
         // ---- 3: per row, keys above and equal to the threshold ----
         int my_hi = 0, my_tied = 0, my_cap = 0;
-        const unsigned long long *row = keys + (size_t)threadIdx.x * ld;
+        const unsigned long long *row = keys + (size_t)threadIdx.x * lds;
         if (threadIdx.x < n && sm.status == HORA_OK && B > 0) {
             my_cap = rw.cap[threadIdx.x];
-            int lo = 0, hi = my_cap;
+            // the selection left the row's range: keys before lo are above the threshold, keys from hi on below it
+            int lo = rw.lo[threadIdx.x], hi = rw.hi[threadIdx.x];
             while (lo < hi) {
                 const int mid = (lo + hi) >> 1;
                 if (HORA_AT(row, mid, ld) > lam_key) lo = mid + 1; else hi = mid;
@@ -198,8 +250,8 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         double lambda = B > 0 ? __longlong_as_double((long long)lam_key) : 0.0;
         if (!exact) {
             long long tot_hi, tot_t;
-            block_exclusive_sum(my_hi, &tot_hi, sm.warp_tmp);
-            const long long pre_t = block_exclusive_sum(my_tied, &tot_t, sm.warp_tmp);
+            block_exclusive_sum<NT>(my_hi, &tot_hi, sm.warp_tmp);
+            const long long pre_t = block_exclusive_sum<NT>(my_tied, &tot_t, sm.warp_tmp);
             const long long R = B - tot_hi;
             long long take = R - pre_t;
             take = take < 0 ? 0 : (take > my_tied ? my_tied : take);
@@ -226,7 +278,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
             }
             if ((int)threadIdx.x < rows_cap) rw.band[threadIdx.x] = (threadIdx.x < n && has && !err) ? q + 1 : 0;
             long long tot_q;
-            block_exclusive_sum(q, &tot_q, sm.warp_tmp);           // has a barrier: band is visible after it
+            block_exclusive_sum<NT>(q, &tot_q, sm.warp_tmp);           // has a barrier: band is visible after it
             const long long Rp = B - tot_q;                        // rollouts to hand out inside the band
             int better = 0, equal = 0;
             if (threadIdx.x < n && rw.band[threadIdx.x] && sm.status == HORA_OK) {
@@ -287,7 +339,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         __syncthreads();
         if (threadIdx.x == 0 && info != nullptr) {
             double tot = 0.0;
-            for (int w = 0; w < kBWarps; ++w) tot += sm.obj_tmp[w];
+            for (int w = 0; w < kWarps; ++w) tot += sm.obj_tmp[w];
             hora_alloc_info o;
             o.status = status;
             o.first_pass_bits = 0;
@@ -518,7 +570,7 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
     }
     const int32_t rows_cap = (int32_t)((max_rows + 3) & ~(int64_t)3);
     const size_t smem = sizeof(BatchedSmemFixed) + (size_t)rows_cap * kBRowBytes +
-                        (size_t)max_rows * (size_t)ld * sizeof(unsigned long long);
+                        (size_t)max_rows * batched_row_stride(ld) * sizeof(unsigned long long);
     // One prior for all prompts: the candidate values are ranked once for all segments (exactly, or as doubles,
     // by the tie mode) and every segment is solved on integer ranks by one warp (no shared-memory keys, no
     // segment size limit).
@@ -556,16 +608,20 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
         launches += tl + 1;
     } else if (S > 0 && N > 0) {
         // 227 KiB of shared memory per SM, 1 KiB of it reserved per resident CTA
-        const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (227 * 1024) / (smem + 1024)));
+        const int threads = max_rows <= kWarp ? 128 : kBThreads;
+        const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(threads == 128 ? 5 : 3, (227 * 1024) / (smem + 1024)));
         const int grid = clamp_grid(S, per_sm);
         auto launch = [&](auto kernel) -> cudaError_t {
             cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
-            kernel<<<grid, kBThreads, smem, st>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, w.seg_off,
-                                                  w.budgets, S, flags, rows_cap, delta, G, info_dev);
+            kernel<<<grid, threads, smem, st>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, w.seg_off,
+                                                w.budgets, S, flags, rows_cap, delta, G, info_dev);
             return cudaGetLastError();
         };
-        if (launch(allocate_batched_kernel<8>) != cudaSuccess) return HORA_ERR_CUDA;   // 8 entries a lane, as hora_gains
+        // 8 entries a lane, as hora_gains
+        if ((threads == 128 ? launch(allocate_batched_kernel<8, 128>) : launch(allocate_batched_kernel<8, kBThreads>)) !=
+            cudaSuccess)
+            return HORA_ERR_CUDA;
         ++launches;
     }
     if (group_offsets != nullptr) {

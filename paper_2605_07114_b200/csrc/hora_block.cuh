@@ -21,7 +21,9 @@ __device__ __forceinline__ bool last_block(unsigned int *ticket) {
     return s_last;
 }
 
-// Block-wide exclusive sum over kSelThreads values (long long), also returns the total.
+// Block-wide exclusive sum over NT values (long long; NT threads per CTA, kSelThreads unless said otherwise), also
+// returns the total.
+template <int NT = kSelThreads>
 __device__ __forceinline__ long long block_exclusive_sum(long long v, long long *total, long long *s_warp) {
     const int lane = lane_id(), warp = threadIdx.x >> 5;
     long long inc = v;
@@ -35,7 +37,7 @@ __device__ __forceinline__ long long block_exclusive_sum(long long v, long long 
     __syncthreads();
     long long base = 0, tot = 0;
 #pragma unroll
-    for (int w = 0; w < kSelThreads / kWarp; ++w) {
+    for (int w = 0; w < NT / kWarp; ++w) {
         const long long x = s_warp[w];
         if (w < warp) base += x;
         tot += x;

@@ -18,6 +18,7 @@ template <bool VEC4>
 __global__ void __launch_bounds__(kBcThreads)
 token_broadcast_kernel(const float *__restrict__ adv, const int64_t *__restrict__ off, int64_t R, int64_t T,
                        int64_t chunk, float *__restrict__ out) {
+    pdl_enter();
     __shared__ int32_t s_rel[kStage + 1];               // offsets relative to the chunk start, clamped to [-1, len]
     __shared__ float s_adv[kStage];
     __shared__ unsigned long long s_bounds[2];
@@ -62,9 +63,9 @@ extern "C" hora_status_t hora_token_broadcast(const float *adv, const int64_t *t
     const bool vec4 = (reinterpret_cast<uintptr_t>(token_adv) & 15u) == 0;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (vec4)
-        token_broadcast_kernel<true><<<(int)grid, kBcThreads, 0, s>>>(adv, token_offsets, R, T, chunk, token_adv);
+        launch_pdl(token_broadcast_kernel<true>, (int)grid, kBcThreads, 0, s, adv, token_offsets, R, T, chunk, token_adv);
     else
-        token_broadcast_kernel<false><<<(int)grid, kBcThreads, 0, s>>>(adv, token_offsets, R, T, chunk, token_adv);
+        launch_pdl(token_broadcast_kernel<false>, (int)grid, kBcThreads, 0, s, adv, token_offsets, R, T, chunk, token_adv);
     count_launches(1);
     return cuda_ok(cudaGetLastError());
 }

@@ -23,6 +23,7 @@ __global__ void __launch_bounds__(kGainsWarps *kWarp, 3)
 gains_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
              const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
              int64_t N, int32_t ld, double *__restrict__ gains, int32_t *status_dev) {
+    pdl_enter();
     NoTap tap;
     gains_rows_cta<E, VEC2, NoTap, LG>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld, gains, status_dev, tap);
 }
@@ -34,11 +35,11 @@ static hora_status_t launch_e(const double *alpha, const double *beta, double al
     const int grid = clamp_grid((N + kCtaRows - 1) / kCtaRows, 3);
     const bool vec2 = (ld % 2 == 0) && ((reinterpret_cast<uintptr_t>(gains) & 15u) == 0);
     if (vec2)
-        gains_kernel<E, true, LG><<<grid, kGainsWarps * kWarp, 0, stream>>>(alpha, beta, alpha0, beta0, c, G0, cap,
-                                                                            cap_scalar, N, ld, gains, status_dev);
+        launch_pdl(gains_kernel<E, true, LG>, grid, kGainsWarps * kWarp, 0, stream, alpha, beta, alpha0, beta0, c, G0, cap,
+                   cap_scalar, N, ld, gains, status_dev);
     else
-        gains_kernel<E, false, LG><<<grid, kGainsWarps * kWarp, 0, stream>>>(alpha, beta, alpha0, beta0, c, G0, cap,
-                                                                             cap_scalar, N, ld, gains, status_dev);
+        launch_pdl(gains_kernel<E, false, LG>, grid, kGainsWarps * kWarp, 0, stream, alpha, beta, alpha0, beta0, c, G0, cap,
+                   cap_scalar, N, ld, gains, status_dev);
     count_launches(1);
     return cuda_ok(cudaGetLastError());
 }

@@ -91,6 +91,7 @@ RankTables rank_tables_carve(void *base, int32_t G0, int32_t ld, bool with_pos) 
 template <int E, bool EXACT>
 __global__ void __launch_bounds__(kSelThreads)
 rank_table_kernel(double alpha0, double beta0, int32_t G0, int32_t ld, RankTables t, int32_t *status) {
+    pdl_enter();
     extern __shared__ __align__(16) unsigned char s_rank_tab[];
     double *s_g = reinterpret_cast<double *>(s_rank_tab);
     const int C = G0 + 1, T = C * ld;
@@ -367,6 +368,7 @@ template <bool HARD>
 __global__ void __launch_bounds__(kSelThreads, 8)
 rank_count_kernel(const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
                   int64_t N, int32_t ld, int64_t B, uint32_t flags, int vec, RankWorkspace w) {
+    pdl_enter();
     extern __shared__ __align__(16) unsigned char s_rank_cnt[];
     unsigned int *s_hist = reinterpret_cast<unsigned int *>(s_rank_cnt);
     __shared__ long long s_warp[kSelThreads / kWarp];
@@ -518,6 +520,7 @@ __device__ __forceinline__ void rank_task_state(const RankQuad (&q)[2], const in
 __global__ void __launch_bounds__(kSelThreads, 4)
 rank_sums_kernel(const int32_t *__restrict__ c, int32_t n_class, int tiers, const int32_t *__restrict__ cap,
                  int32_t cap_scalar, int64_t N, int vec, RankWorkspace w, int64_t NT, int64_t m) {
+    pdl_enter();
     extern __shared__ __align__(16) unsigned char s_rank_cls[];
     int32_t *s_class = reinterpret_cast<int32_t *>(s_rank_cls);
     __shared__ long long s_acc[2][kSelThreads / kWarp];
@@ -561,6 +564,7 @@ rank_out_kernel(const int32_t *__restrict__ c, int32_t G0, int32_t n_class, int 
                 int32_t cap_scalar, int64_t N, int64_t B, int vec, RankWorkspace w, int64_t NT, int64_t m,
                 int32_t *__restrict__ delta,
                 int32_t *__restrict__ G, int64_t *__restrict__ offsets, int vec_out, hora_alloc_info *info) {
+    pdl_enter();
     extern __shared__ __align__(16) unsigned char s_rank_cls[];
     int32_t *s_class = reinterpret_cast<int32_t *>(s_rank_cls);
     __shared__ long long s_warp[kSelThreads / kWarp];
@@ -684,7 +688,7 @@ static hora_status_t launch_rank_passes(const RankWorkspace &w, const int32_t *c
     const int vec = ((reinterpret_cast<uintptr_t>(c) | reinterpret_cast<uintptr_t>(cap)) & 15u) == 0;
     const int per_sm = (int)std::fmax(1.0, std::fmin(8.0, std::floor(200.0 * 1024.0 / (double)(smem_h + 1024))));
     const int grid = clamp_grid((N + 8 * kSelThreads - 1) / (8 * kSelThreads), per_sm);
-    rank_count_kernel<HARD><<<grid, kSelThreads, smem_h, s>>>(c, G0, cap, cap_scalar, N, ld, B, flags, vec, w);
+    launch_pdl(rank_count_kernel<HARD>, grid, kSelThreads, smem_h, s, c, G0, cap, cap_scalar, N, ld, B, flags, vec, w);
     if (mark) { mark(2, s); mark(3, s); }
     const size_t smem_c = sizeof(int32_t) * (size_t)C;
     const int warps = kSelThreads / kWarp;
@@ -692,12 +696,12 @@ static hora_status_t launch_rank_passes(const RankWorkspace &w, const int32_t *c
     int grid_b = clamp_grid((NT + warps - 1) / warps, 3);       // what the output pass keeps resident
     if (grid_b > kRankMaxCtas) grid_b = kRankMaxCtas;
     const int64_t m = (NT + grid_b - 1) / grid_b;            // tasks per CTA, a contiguous run
-    rank_sums_kernel<<<grid_b, kSelThreads, smem_c, s>>>(c, C, HARD ? 1 : 0, cap, cap_scalar, N, vec, w, NT, m);
+    launch_pdl(rank_sums_kernel, grid_b, kSelThreads, smem_c, s, c, C, HARD ? 1 : 0, cap, cap_scalar, N, vec, w, NT, m);
     if (mark) { mark(4, s); mark(5, s); }
     const int out_vec = ((reinterpret_cast<uintptr_t>(delta) | reinterpret_cast<uintptr_t>(G) |
                           reinterpret_cast<uintptr_t>(group_offsets)) & 15u) == 0;
-    rank_out_kernel<<<grid_b, kSelThreads, smem_c, s>>>(c, G0, C, HARD ? 1 : 0, cap, cap_scalar, N, B, vec, w, NT, m, delta,
-                                                        G, group_offsets, out_vec, info_dev);
+    launch_pdl(rank_out_kernel, grid_b, kSelThreads, smem_c, s, c, G0, C, HARD ? 1 : 0, cap, cap_scalar, N, B, vec, w, NT, m,
+               delta, G, group_offsets, out_vec, info_dev);
     if (mark) mark(6, s);
     return cuda_ok(cudaGetLastError());
 }
