@@ -27,7 +27,8 @@
 //     digits  more than that (a missed window, or heavy ties): level 1 histogrammed the next 13 bits and
 //             listed the rows whose segment is not empty; all CTAs narrow the listed rows' segments digit by
 //             digit (13 bits at a time, a grid-wide barrier between levels), close them with the finished
-//             threshold, form the block sums and scan them.
+//             threshold, form the block sums and scan them.  If level 1 found every key of the threshold's bin
+//             to be one value (a mass tie), that value is the threshold and the digit levels are skipped.
 //   out       p_hi = #keys > lambda, tied = #keys == lambda per row (segments left open by the list route are
 //             closed here); Delta_i = p_hi + (tied candidates of row i that fall within the first
 //             R = B - n_above tied candidates in prompt order); G_i, CSR offsets, objective.
@@ -104,6 +105,9 @@ struct AllocHeader {
     long long bin_count;               // keys that carry the prefix resolved so far
     int32_t list_mode;                 // 1: the keys of level 1's segments go to the candidate list
     int32_t pad1;
+    unsigned long long seg_ref;        // digit route: the first segment key any thread of level 1 registered
+    int32_t seg_differs;               // digit route: 1 if some segment key differs from seg_ref
+    int32_t pad2;
 };
 
 struct Workspace {
@@ -904,12 +908,15 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
     pdl_enter();
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
+    __shared__ unsigned long long s_ref;                         // digit route: the CTA's reference key, once it has one
     if (*(volatile int32_t *)&hdr->status != 0) return;
     const bool list = hdr->list_mode != 0;
     if (!list) {
         for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
+        if (threadIdx.x == 0) s_ref = 0ull;
         __syncthreads();
     }
+    bool differs = false;
     const int lane = lane_id();
     const int r = hdr->resolved;                                 // 13 or 23: the prefix lies in the key's high word
     const unsigned P = (unsigned)(hdr->prefix_key >> 32) >> (32 - r);
@@ -1026,9 +1033,27 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
                                  : 0.0;
                 objrow[row] = u;
             }
-            if (!list)                                           // digit route: the segment's keys on the next digit
-                for (int32_t j = 0; j < n_eq; ++j)
-                    atomicAdd(&HORA_AT(s_hist, (__ldg(&HORA_AT(keys, p_hi + j, ld)) >> shift) & digit_mask, kBins), 1u);
+            if (!list) {
+                // digit route: the segment's keys on the next digit.  This route means many keys in one bin — in the
+                // extreme one value tied a million times — so every key is held against a reference key (the CTA's first
+                // key, itself held against the first that any CTA put into the header; 0 stands for "none yet"): if
+                // none differs, the threshold is known.  (Letting the lanes that meet in a bin send one update
+                // between them made the pass slower.)
+                for (int32_t j = 0; j < n_eq; ++j) {
+                    const unsigned long long key = __ldg(&HORA_AT(keys, p_hi + j, ld));
+                    unsigned long long ref = *(volatile unsigned long long *)&s_ref;
+                    if (ref == 0ull) {                           // the CTA's first key becomes its reference ...
+                        ref = atomicCAS(&s_ref, 0ull, key);
+                        if (ref == 0ull) {                       // ... and is held against the header's, once per CTA
+                            const unsigned long long g = atomicCAS(&hdr->seg_ref, 0ull, key);
+                            differs |= g != 0ull && g != key;
+                            ref = key;
+                        }
+                    }
+                    differs |= key != ref || key == 0ull;      // (a caller's matrix may hold zeros: no shortcut then)
+                    atomicAdd(&HORA_AT(s_hist, (key >> shift) & digit_mask, kBins), 1u);
+                }
+            }
         }
         if (list) {
             // per warp: one addition to the block sum of p_hi, one slot reservation for the warp's keys (the
@@ -1071,6 +1096,7 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
     }
     if (bad) raise_status(&hdr->status, HORA_ERR_INVALID_VALUE);
     if (list) return;
+    if (differs) *(volatile int32_t *)&hdr->seg_differs = 1;
     __syncthreads();
     flush_hist(s_hist, hist1, 1 << bits);
     if (last_block(&hdr->ticket[1])) find_digit(hdr, hist1, 1 << bits, bits, shift, 1, false, s_warp);
@@ -1271,7 +1297,20 @@ __device__ void tail_digits(int64_t N, int32_t ld, const double *__restrict__ ga
     cooperative_groups::grid_group grid = cooperative_groups::this_grid();
     const unsigned int n_active = hdr->n_active;
     const unsigned int stride = gridDim.x * kSelThreads;
-    for (int level = 2; level < kLevels; ++level) {
+    // Every key that carries level 0's prefix has the same value (a mass tie: one candidate type shared by a million
+    // prompts): that value is the threshold, and the digit levels, a pass over the active rows each, are skipped.
+    // (The rank `need` lies within those keys, so it stays as it is.)
+    const unsigned long long seg_ref = hdr->seg_ref;
+    const bool all_equal = seg_ref != 0ull && hdr->seg_differs == 0;
+    if (all_equal) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            hdr->prefix_key = seg_ref;
+            hdr->resolved = 64;
+            __threadfence();
+        }
+        grid.sync();
+    }
+    for (int level = 2; level < kLevels && !all_equal; ++level) {
         int bits = 0, shift = 0;
         next_digit(*(volatile int32_t *)&hdr->resolved, &bits, &shift);
         const int bins = 1 << bits;
@@ -1379,7 +1418,14 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
               int32_t *__restrict__ rowslot, unsigned long long *tkeys, unsigned long long *tcounts) {
     pdl_enter();
     __shared__ long long s_warp[kSelThreads / kWarp];
-    if (*(volatile int32_t *)&hdr->status != 0) return;
+    // instances per table slot, added up in the CTA first: with one type tied a million times every warp of the
+    // grid would otherwise update the same global counter
+    __shared__ unsigned int s_cnt[kTypeSlots];
+    __shared__ int s_stop;                                       // one reading of the status for the whole CTA
+    if (threadIdx.x == 0) s_stop = *(volatile int32_t *)&hdr->status != 0;
+    for (int h = threadIdx.x; h < kTypeSlots; h += kSelThreads) s_cnt[h] = 0u;
+    __syncthreads();
+    if (s_stop) return;
     const unsigned long long lam_key = hdr->prefix_key;
     const bool list = hdr->list_mode != 0;
     const double lam = __longlong_as_double((long long)lam_key);
@@ -1422,7 +1468,9 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
             if (lane == leader) {
                 unsigned int h = (unsigned int)((tkey * 0x9E3779B97F4A7C15ull) >> 52) & (kTypeSlots - 1);
                 for (int probe = 0; probe < kTypeSlots; ++probe) {
-                    const unsigned long long old = atomicCAS(&HORA_AT(tkeys, h, kTypeSlots), 0ull, tkey);
+                    // a slot once taken never changes: look before trying to take it
+                    unsigned long long old = *(volatile unsigned long long *)&HORA_AT(tkeys, h, kTypeSlots);
+                    if (old == 0ull) old = atomicCAS(&HORA_AT(tkeys, h, kTypeSlots), 0ull, tkey);
                     if (old == 0ull || old == tkey) {
                         if (old == 0ull) atomicAdd(&hdr->n_types, 1u);
                         slot = (int32_t)h;
@@ -1430,7 +1478,7 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
                     }
                     h = (h + 1) & (kTypeSlots - 1);
                 }
-                if (slot >= 0) atomicAdd(&HORA_AT(tcounts, slot, kTypeSlots), (unsigned long long)__popc(peers));
+                if (slot >= 0) atomicAdd(&HORA_AT(s_cnt, slot, kTypeSlots), (unsigned int)__popc(peers));
                 else err = err ? err : HORA_ERR_EXACT_RANGE;
             }
             slot = __shfl_sync(peers, slot, leader);
@@ -1442,8 +1490,12 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
     }
     if (err) raise_status(&hdr->status, err);
     long long tot;
-    block_exclusive_sum(above, &tot, s_warp);
+    block_exclusive_sum(above, &tot, s_warp);                   // (its barriers also put the CTA's counts in place)
     if (threadIdx.x == 0 && tot) atomicAdd(&hdr->band_above, (unsigned long long)tot);
+    for (int h = threadIdx.x; h < kTypeSlots; h += kSelThreads) {
+        const unsigned int v = s_cnt[h];
+        if (v) atomicAdd(&HORA_AT(tcounts, h, kTypeSlots), (unsigned long long)v);
+    }
 }
 
 // Exact mode, step 2 (one CTA): rank the collected types exactly and label them.

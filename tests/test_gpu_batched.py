@@ -69,12 +69,16 @@ def random_problem(rng, S, G0, ld, real, max_rows=40, int_priors=False):
 
 @pytest.mark.parametrize("G0,ld", [(2, 24), (4, 60), (8, 130), (8, 256)])
 @pytest.mark.parametrize("prior", ["shared", "integer", "real"])
-def test_batched_matches_oracle_per_segment(G0, ld, prior):
+@pytest.mark.parametrize("max_rows", [40, 15])
+def test_batched_matches_oracle_per_segment(G0, ld, prior, max_rows):
     """shared: one Beta(1,1) prior, exact ties (solved on exact ranks, a warp per segment); integer: per-prompt
-    integer priors, exact ties (a CTA per segment, keys in shared memory); real: per-prompt real priors."""
+    integer priors, exact ties (a CTA per segment, keys in shared memory); real: per-prompt real priors.
+    max_rows: segments of up to 40 prompts run 256 threads a CTA (a lane owns several rows in the selection where a
+    segment has more than 32), calls whose segments all have at most 32 prompts run 128 threads a CTA."""
     real = prior == "real"
-    rng = np.random.default_rng(G0 * 1000 + ld + real)
-    alpha, beta, c, cap, seg, budgets = random_problem(rng, 300, G0, ld, real, int_priors=prior == "integer")
+    rng = np.random.default_rng(G0 * 1000 + ld + real + 7 * (max_rows != 40))
+    alpha, beta, c, cap, seg, budgets = random_problem(rng, 300, G0, ld, real, max_rows=max_rows,
+                                                       int_priors=prior == "integer")
     d, G, off, infos = run_batched(alpha, beta, 1.0, 1.0, c, G0, cap, ld, seg, budgets, exact=not real)
     d_o, lam_o, obj_o = oracle_segments(alpha, beta, 1.0, 1.0, c, G0, cap, seg, budgets, exact=not real)
     np.testing.assert_array_equal(d, d_o)
@@ -114,6 +118,36 @@ def test_paper_shard_shape_and_agreement_with_single_problem_call():
         assert infos[s].n_above == info1.n_above and infos[s].n_tied == info1.n_tied
         assert abs(infos[s].objective - info1.objective) <= 1e-13 * info1.objective
     assert d[c == 0].mean() > d[c == G0].mean()          # hopeless prompts get more than saturated ones
+
+
+@pytest.mark.parametrize("exact", [False, True])
+def test_paper_shard_shape_with_per_prompt_priors(exact):
+    """The shape the benchmark times through the CTA-per-segment kernel: shards of 15 prompts, ld = 360, budget 360,
+    G0 = 8, per-prompt priors (real with fp64 ties, integer with exact ties)."""
+    rng = np.random.default_rng(61 + exact)
+    G0, shard, B, ld, S = 8, 15, 360, 360, 96
+    N = S * shard
+    c = rng.choice(G0 + 1, size=N, p=[0.15] + [0.34 / 7] * 7 + [0.51]).astype(np.int32)
+    cap = np.full(N, ld, np.int32)
+    if exact:
+        alpha = rng.integers(1, 4, N).astype(np.float64)
+        beta = rng.integers(1, 4, N).astype(np.float64)
+    else:
+        alpha = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
+        beta = np.exp(rng.uniform(np.log(0.05), np.log(20), N))
+    seg = np.arange(0, N + 1, shard, dtype=np.int64)
+    budgets = np.full(S, B, np.int64)
+    budgets[:8] = [0, 1, 2, 15, 359, 361, 15 * 360, 15 * 360 - 1]      # the ends of the range too
+    d, G, off, infos = run_batched(alpha, beta, 1.0, 1.0, c, G0, cap, ld, seg, budgets, exact=exact)
+    d_o, lam_o, obj_o = oracle_segments(alpha, beta, 1.0, 1.0, c, G0, cap, seg, budgets, exact=exact)
+    np.testing.assert_array_equal(d, d_o)
+    np.testing.assert_array_equal(G, G0 + d_o)
+    for s, inf in enumerate(infos):
+        assert inf.status == 0
+        if budgets[s] > 0:
+            assert abs(inf.objective - obj_o[s]) <= 1e-12 * abs(obj_o[s])
+            assert abs(inf.lambda_ - lam_o[s]) <= 1e-12 * lam_o[s]
+            assert inf.n_above + inf.n_tied_taken == budgets[s] and 1 <= inf.n_tied_taken <= inf.n_tied
 
 
 def test_a_failing_segment_leaves_the_others_alone():

@@ -97,8 +97,8 @@ def test_batched_and_advantages(checked):
     import gpu_util as gu
     import test_gpu_batched as tb
     rng = np.random.default_rng(77)
-    for prior in ("shared", "integer", "real"):
-        alpha, beta, c, cap, seg, budgets = tb.random_problem(rng, 120, 8, 131, prior == "real", max_rows=37,
+    for prior, max_rows in (("shared", 37), ("integer", 37), ("real", 37), ("integer", 15), ("real", 15)):
+        alpha, beta, c, cap, seg, budgets = tb.random_problem(rng, 120, 8, 131, prior == "real", max_rows=max_rows,
                                                               int_priors=prior == "integer")
         d, G, off, infos = tb.run_batched(alpha, beta, 1.0, 1.0, c, 8, cap, 131, seg, budgets, exact=prior != "real")
         d_o, _, _ = tb.oracle_segments(alpha, beta, 1.0, 1.0, c, 8, cap, seg, budgets, exact=prior != "real")

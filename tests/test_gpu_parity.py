@@ -333,6 +333,35 @@ def test_heavy_ties_take_the_digit_route_at_moderate_size(exact, materialise):
     assert abs(info.objective - obj) <= 1e-12 * obj
 
 
+@pytest.mark.parametrize("case", ["two_values", "zeros"])
+def test_mass_ties_in_a_given_matrix_that_are_not_one_value(case):
+    """The digit route has a shortcut for the case that every key carrying the resolved prefix is one value.  Here
+    it must not fire: (two_values) 2^17 keys share 23 bits but are two values 2^-40 apart, the threshold being the
+    larger; (zeros) the budget reaches into 2^18 zero gains, two a row.  Expected: the B largest candidates under
+    (gain descending, prompt ascending, column ascending), by a global sort of the matrix."""
+    from paper_2605_07114_b200 import hora
+    N, G0, ld = 1 << 17, 2, 4
+    rng = np.random.default_rng(17)
+    k1 = 0.5
+    k2 = float(np.float64(0.5) * (1.0 + 2.0 ** -40))
+    second = np.where(rng.random(N) < 0.5, k1, k2)
+    g = np.stack([np.full(N, 0.9), second, np.zeros(N), np.zeros(N)], axis=1)
+    B = N + N // 4 if case == "two_values" else 2 * N + N // 2
+    order = np.lexsort((np.tile(np.arange(ld), N), np.repeat(np.arange(N), ld), -g.ravel()))
+    d_o = np.bincount(order[:B] // ld, minlength=N).astype(np.int32)
+    al = hora.Allocator(N, ld, G0, exact_int=False)
+    al.gains.copy_(torch.from_numpy(g).cuda())
+    ones = gu_dev(np.ones(N))
+    hora.hora_allocate(ones, ones, 1.0, 1.0, gu_dev(np.zeros(N, np.int32)), G0, None, ld, N, ld, al.gains, B, al.flags,
+                       al.delta, al.G, al.group_offsets, al.info, al.workspace)
+    torch.cuda.synchronize()
+    info = al.read_info()
+    assert info.status == 0
+    assert info.n_tied == (int((second == k2).sum()) if case == "two_values" else 2 * N)
+    assert info.lambda_ == (k2 if case == "two_values" else 0.0)
+    np.testing.assert_array_equal(al.delta.cpu().numpy(), d_o)
+
+
 def test_allocation_with_long_rows():
     """ld > 256: several items per row in the full-read pass, whose counts above the guess add up per row."""
     gu = _util()
