@@ -608,8 +608,8 @@ def bench_batched(torch, hora, wl, dev, hbm_peak, fp64_peak, shards=65536, shard
     ach = flops / (ms2 * 1e-3) / 1e12
     out["real_priors"] = {"shards": s2, "ms": round(ms2, 4), "shards_per_s": s2 / (ms2 * 1e-3),
                           "prompts_per_s": n2 / (ms2 * 1e-3),
-                          "roofline": {"bound": "alu", "kernel": "allocate_batched_kernel (rows built in shared memory, "
-                                       "selection by digit sweeps)", "achieved": round(ach, 3), "peak": fp64_peak,
+                          "roofline": {"bound": "alu", "kernel": "allocate_batched_kernel (a CTA of 128 threads per shard: rows built in "
+                                       "shared memory, the threshold built two bits a step by one warp)", "achieved": round(ach, 3), "peak": fp64_peak,
                                        "unit": "TFLOP/s", "frac": round(ach / fp64_peak, 4), "traffic": None,
                                        "algorithmic_flops_per_launch": int(flops),
                                        "flops_per_candidate": FP64_OPS_PER_CANDIDATE}}

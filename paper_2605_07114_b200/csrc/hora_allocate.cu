@@ -558,6 +558,8 @@ select_level0(const int32_t *__restrict__ cap, int32_t cap_scalar, int64_t N, in
     long long capsum = 0, sum_pg = 0;
     bool bad = false;
     // two items in flight, in two fixed register sets (no copies): A is processed while B's loads land
+    // (reading the matrix from its end, so that what the L2 still holds of the rows hora_gains wrote last is read
+    // first, was tried: no difference in the step)
     Level0Item<E> A, Bq;
     level0_fetch<E, VEC2, ONE>(A, cap, cap_scalar, n_items, items_per_row, ld, gains, item0, lane, &bad);
     for (int64_t item = item0; item < n_items; item += 2 * stride) {
@@ -1393,7 +1395,7 @@ select_tail(int64_t N, int32_t ld, const double *__restrict__ gains, int64_t B, 
     pdl_enter();
     __shared__ unsigned int s_hist[kBins];
     __shared__ unsigned long long s_keys[kListSmall];
-    __shared__ long long s_warp[kSelThreads / kWarp];
+    __shared__ long long s_warp[2 * (kSelThreads / kWarp)];
     if (*(volatile int32_t *)&hdr->status != 0) return;         // the same answer in every CTA: nobody waits at a barrier
     if (hdr->list_mode != 0) {
         if (blockIdx.x == 0) tail_list(B, hdr, hist_all + kBins, cand_key, cand_row, bsum_hi, bsum_t, NB, s_hist, s_keys, s_warp);
@@ -1576,7 +1578,7 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
            int2 *__restrict__ rowstate, const int32_t *__restrict__ rowslot, const int32_t *__restrict__ tlabel,
            long long *bsum_hi, long long *bsum_t, int64_t NB) {
     pdl_enter();
-    __shared__ long long s_warp[kSelThreads / kWarp];
+    __shared__ long long s_warp[2 * (kSelThreads / kWarp)];
     const bool failed = *(volatile int32_t *)&hdr->status != 0;
     long long hi_sum = 0, t_sum = 0;
     if (!failed) {
@@ -1608,9 +1610,8 @@ select_sum(const double *__restrict__ alpha, const double *__restrict__ beta, do
             }
         }
     }
-    long long tot_hi, tot_t;
-    block_exclusive_sum(hi_sum, &tot_hi, s_warp);
-    block_exclusive_sum(t_sum, &tot_t, s_warp);
+    long long tot_hi, tot_t, e_hi, e_t;
+    block_exclusive_sum2(hi_sum, t_sum, e_hi, e_t, tot_hi, tot_t, s_warp);
     if (threadIdx.x == 0) { bsum_hi[blockIdx.x] = tot_hi; bsum_t[blockIdx.x] = tot_t; }
     if (last_block(&hdr->ticket[8 + mode])) {
         long long run_hi = 0, run_t = 0;
@@ -1635,19 +1636,21 @@ select_out(const double *__restrict__ alpha, const double *__restrict__ beta, do
            const long long *__restrict__ bpre_t, double *objpart, int64_t NB, int32_t *__restrict__ delta,
            int32_t *__restrict__ G, int64_t *__restrict__ offsets, int vec, hora_alloc_info *info) {
     pdl_enter();
-    __shared__ long long s_warp[kSelThreads / kWarp];
+    __shared__ long long s_warp[2 * (kSelThreads / kWarp)];
     __shared__ double s_obj[kSelThreads / kWarp];
-    const int32_t status = *(volatile int32_t *)&hdr->status;
-    const bool failed = status != 0;
     constexpr int kPer = kRowsPerBlock / kSelThreads;
     static_assert(kPer == 4, "a thread owns four consecutive prompts");
     const int64_t row0 = (int64_t)blockIdx.x * kRowsPerBlock + (int64_t)threadIdx.x * kPer;
     const bool whole = row0 + kPer <= N;                      // all four prompts exist
-    // the list route of the tail leaves the segments as level 1 found them (exact mode has closed them since)
-    const bool open = !failed && hdr->list_mode != 0 && !(flags & HORA_FLAG_EXACT_INT);
+    // Every load that does not depend on another is issued here, before the first is used: the header's fields,
+    // the block prefixes, the rows' states and utilities (the arrays are read whether or not the call has failed;
+    // they lie inside the workspace either way).
+    const int32_t status = hdr->status;                       // (raised by earlier kernels only)
+    const int32_t list_mode = hdr->list_mode;
     const unsigned long long lam_key = hdr->prefix_key;
-    const bool want_obj = !failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE);
-    // every load that does not depend on another is issued here
+    const long long R_hdr = hdr->R;
+    const long long blk_hi_raw = bpre_hi[blockIdx.x], blk_t_raw = bpre_t[blockIdx.x];
+    const bool use_objrow = objrow != nullptr && !(flags & HORA_FLAG_SKIP_OBJECTIVE);
     int2 st[kPer];
     double o[kPer];
     if (whole) {
@@ -1660,7 +1663,7 @@ select_out(const double *__restrict__ alpha, const double *__restrict__ beta, do
     }
 #pragma unroll
     for (int q = 0; q < kPer; ++q) o[q] = -1.0;
-    if (want_obj && objrow != nullptr) {
+    if (use_objrow) {
         if (whole) {
             const double2 o01 = *reinterpret_cast<const double2 *>(objrow + row0), o23 = *reinterpret_cast<const double2 *>(objrow + row0 + 2);
             o[0] = o01.x; o[1] = o01.y; o[2] = o23.x; o[3] = o23.y;
@@ -1669,8 +1672,12 @@ select_out(const double *__restrict__ alpha, const double *__restrict__ beta, do
             for (int q = 0; q < kPer; ++q) if (row0 + q < N) o[q] = objrow[row0 + q];
         }
     }
-    const long long blk_hi = failed ? 0 : bpre_hi[blockIdx.x], blk_t = failed ? 0 : bpre_t[blockIdx.x];
-    const long long R = failed ? 0 : hdr->R;
+    const bool failed = status != 0;
+    // the list route of the tail leaves the segments as level 1 found them (exact mode has closed them since)
+    const bool open = !failed && list_mode != 0 && !(flags & HORA_FLAG_EXACT_INT);
+    const bool want_obj = !failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE);
+    const long long blk_hi = failed ? 0 : blk_hi_raw, blk_t = failed ? 0 : blk_t_raw;
+    const long long R = failed ? 0 : R_hdr;
     int32_t hi[kPer], tied[kPer];
     long long hi_sum = 0, t_sum = 0;
 #pragma unroll
@@ -1683,9 +1690,10 @@ select_out(const double *__restrict__ alpha, const double *__restrict__ beta, do
         hi_sum += hi[q];
         t_sum += tied[q];
     }
-    long long th, tt;
-    long long pre_hi = blk_hi + block_exclusive_sum(hi_sum, &th, s_warp);
-    long long pre_t = blk_t + block_exclusive_sum(t_sum, &tt, s_warp);
+    long long th, tt, pre_hi, pre_t;
+    block_exclusive_sum2(hi_sum, t_sum, pre_hi, pre_t, th, tt, s_warp);
+    pre_hi += blk_hi;
+    pre_t += blk_t;
     int32_t d[kPer];
     int64_t of[kPer];
 #pragma unroll

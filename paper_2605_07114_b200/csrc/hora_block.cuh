@@ -46,6 +46,35 @@ __device__ __forceinline__ long long block_exclusive_sum(long long v, long long 
     return base + inc - v;
 }
 
+// Two block-wide exclusive sums at once (one pair of barriers instead of two): v0, v1 in, their exclusive
+// prefixes in e0, e1, the totals in t0, t1.  s_warp2 holds 2 * (NT / 32) values.
+template <int NT = kSelThreads>
+__device__ __forceinline__ void block_exclusive_sum2(long long v0, long long v1, long long &e0, long long &e1,
+                                                     long long &t0, long long &t1, long long *s_warp2) {
+    constexpr int kW = NT / kWarp;
+    const int lane = lane_id(), warp = threadIdx.x >> 5;
+    long long i0 = v0, i1 = v1;
+#pragma unroll
+    for (int d = 1; d < kWarp; d <<= 1) {
+        const long long a = __shfl_up_sync(kFull, i0, d), b = __shfl_up_sync(kFull, i1, d);
+        if (lane >= d) { i0 += a; i1 += b; }
+    }
+    __syncthreads();
+    if (lane == kWarp - 1) { s_warp2[warp] = i0; s_warp2[kW + warp] = i1; }
+    __syncthreads();
+    long long b0 = 0, b1 = 0;
+    t0 = t1 = 0;
+#pragma unroll
+    for (int w = 0; w < kW; ++w) {
+        const long long x = s_warp2[w], y = s_warp2[kW + w];
+        if (w < warp) { b0 += x; b1 += y; }
+        t0 += x;
+        t1 += y;
+    }
+    e0 = b0 + i0 - v0;
+    e1 = b1 + i1 - v1;
+}
+
 // Run by ONE CTA.  Scanning from the top bin down, find the bin where the running count reaches `need`:
 //   count(bins above d) < need <= count(bins above d) + count(d).
 // Returns d (or -1 if need is out of range) to every thread, with the count above d in *above_out and the
@@ -141,7 +170,8 @@ __device__ __forceinline__ void locate_rank_shared(const unsigned int *s_hist, i
 }
 
 // Exclusive scan of the block sums (plus, in list mode, the corrections held in shared memory for blocks
-// [b0, b0 + n_here)), kSelThreads * 4 entries per step, in index order; run by one CTA.
+// [b0, b0 + n_here)), kSelThreads * 4 entries per step, in index order; run by one CTA.  s_warp holds
+// 2 * (kSelThreads / 32) values.
 __device__ inline void scan_block_sums(long long *bsum_hi, long long *bsum_t, int64_t b0, int64_t n_here,
                                 const unsigned int *s_fix_hi, const unsigned int *s_fix_t, long long &run_hi,
                                 long long &run_t, long long *s_warp) {
@@ -157,9 +187,10 @@ __device__ inline void scan_block_sums(long long *bsum_hi, long long *bsum_t, in
         }
 #pragma unroll
         for (int u = 0; u < kRun; ++u) { sh += vh[u]; st += vt[u]; }
-        long long th, tt;
-        long long eh = run_hi + block_exclusive_sum(sh, &th, s_warp);
-        long long et = run_t + block_exclusive_sum(st, &tt, s_warp);
+        long long th, tt, eh, et;
+        block_exclusive_sum2(sh, st, eh, et, th, tt, s_warp);
+        eh += run_hi;
+        et += run_t;
 #pragma unroll
         for (int u = 0; u < kRun; ++u) {
             if (c + u < n_here) { bsum_hi[b0 + c + u] = eh; bsum_t[b0 + c + u] = et; }
