@@ -168,6 +168,17 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     hora.load()
 
+    if args.only is not None:
+        # one of the secondary measurements alone (a small process to profile): its object, as one JSON line
+        peak = measured_peak()[0]
+        fp64 = measure_fp64_peak(torch, hora, dev)
+        if args.only == "batched":
+            res = bench_batched(torch, hora, wl, dev, peak, fp64["value"], shards=args.shards)
+        else:
+            res = bench_configs(torch, hora, wl, dev, peak)
+        print(json.dumps({args.only: res}))
+        return
+
     w = wl.make(WORKLOAD, args.prompts, seed=shard_seed(rank))
     N, ld, G0, B = w.N, w.ld, w.G0, w.B
     h_alpha = torch.from_numpy(w.alpha).pin_memory()
@@ -888,6 +899,9 @@ def main():
     ap.add_argument("--prompts", type=int, default=None, help="override N (default: the workload's 2^20)")
     ap.add_argument("--cpu-sample", type=int, default=1 << 20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default=None, choices=["batched", "configs"],
+                    help="run one secondary measurement alone and print its object (not the benchmark line)")
+    ap.add_argument("--shards", type=int, default=65536, help="shards of the batched measurement")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -13,6 +13,8 @@
 //   4  ties: in prompt order (fp64 equality), or, in exact mode, by exact rational comparison of the at
 //      most one candidate per row that lies within 2^-30 of the threshold (pairwise, cross-multiplied);
 //   5  Delta, G, the segment's summary.
+// Rows longer than 256 candidates are first cut to 256 (a narrow pass; exact unless a row takes them all), and
+// only the segments that this does not settle are solved at full width.
 // Group offsets over all prompts are an exclusive scan of G by two small kernels afterwards.
 #include <algorithm>
 
@@ -33,14 +35,16 @@ constexpr int kBWarps = kBThreads / kWarp;
 constexpr int kBMaxRows = 256;                 // prompts per segment (one thread per prompt in the row phases)
 constexpr size_t kBMaxSmem = 200 * 1024;       // keys + bookkeeping must fit this
 constexpr int kScanRows = 1024;                // rows per CTA in the offsets scan
+constexpr int32_t kBNarrow = 256;              // candidates per row the narrow pass builds (one pass of 32 lanes x 8)
 
 struct BatchedSmemFixed {
     unsigned long long lam_key;
-    long long warp_tmp[kBWarps];
+    long long warp_tmp[2 * kBWarps];
     double obj_tmp[kBWarps];
     long long found[3];
     double lam_exact;
     int status;
+    int redo;                      // narrow pass: this segment has to go through the full-width pass
 };
 
 // Per-prompt arrays of a segment, carved behind the fixed part for the longest segment of the call (so that
@@ -50,8 +54,9 @@ struct BatchedRows {
     int32_t *cap, *band;           // band: Delta of the row's near-threshold candidate (exact mode), 0 if it has none
     int32_t *lo, *hi;              // selection: the row's count of keys >= the threshold lies in [lo, hi]
     int32_t *cnt2, *cnt3;          // selection: the row's counts for the second and third trial value of a step
+    int32_t *capt;                 // the prompt's own cap (cap: what the pass works with, at most its row width)
 };
-constexpr size_t kBRowBytes = 2 * sizeof(double) + 6 * sizeof(int32_t);   // 40 bytes per prompt
+constexpr size_t kBRowBytes = 2 * sizeof(double) + 7 * sizeof(int32_t);   // 44 bytes per prompt
 
 __device__ __forceinline__ BatchedRows carve_rows(unsigned char *base, int rows_cap) {
     BatchedRows r;
@@ -63,8 +68,11 @@ __device__ __forceinline__ BatchedRows carve_rows(unsigned char *base, int rows_
     r.hi = r.lo + rows_cap;
     r.cnt2 = r.hi + rows_cap;
     r.cnt3 = r.cnt2 + rows_cap;
+    r.capt = r.cnt3 + rows_cap;
     return r;
 }
+
+struct ScanHeader { unsigned int ticket; unsigned int n_redo; };   // n_redo: segments the narrow pass handed on
 
 __host__ __device__ inline size_t batched_row_stride(int32_t ld) { return (size_t)ld | 1u; }
 
@@ -87,13 +95,21 @@ __device__ __forceinline__ void search3(const unsigned long long *rk, int lo, in
 // NT threads per CTA: 256, or 128 when no segment of the call has more than 32 prompts.  The selection is a chain of
 // dependent steps by one warp, so what an SM gets through is set by how many segments it holds at once: shared
 // memory has room for five of the paper's 15-prompt segments, the registers of 256 threads for three CTAs only.
-template <int E, int NT>
-__global__ void __launch_bounds__(NT, NT == 128 ? 5 : 3)
+//
+// Two passes when rows are longer than 256 candidates.  The NARROW pass (W = 256 < ld, todo == nullptr) builds and
+// searches only the first W candidates of every row: half the row passes at ld = 360, and a segment's keys take a
+// third less shared memory.  Its answer is the full problem's answer unless some row takes all W of its candidates
+// while it has more (its next candidate might belong to the B largest), or the budget exceeds what the narrow rows
+// hold; such a segment writes nothing and puts its index on the redo list.  The FULL pass (W = ld) then runs over
+// that list (todo, *n_todo) — as a rule it is empty — or, where ld <= 256, over every segment (todo == nullptr).
+template <int E, int NT, int PER_SM>
+__global__ void __launch_bounds__(NT, PER_SM)
 allocate_batched_kernel(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
                         const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
-                        int32_t ld, const int64_t *__restrict__ seg_off, const int64_t *__restrict__ budgets, int64_t S,
-                        uint32_t flags, int32_t rows_cap, int32_t *__restrict__ delta, int32_t *__restrict__ G,
-                        hora_alloc_info *__restrict__ info) {
+                        int32_t ld, int32_t W, const int64_t *__restrict__ seg_off, const int64_t *__restrict__ budgets,
+                        int64_t S, const int32_t *__restrict__ todo, const unsigned int *__restrict__ n_todo,
+                        int32_t *__restrict__ redo, unsigned int *n_redo, uint32_t flags, int32_t rows_cap,
+                        int32_t *__restrict__ delta, int32_t *__restrict__ G, hora_alloc_info *__restrict__ info) {
     extern __shared__ __align__(16) unsigned char s_raw[];
     BatchedSmemFixed &sm = *reinterpret_cast<BatchedSmemFixed *>(s_raw);
     const BatchedRows rw = carve_rows(s_raw + sizeof(BatchedSmemFixed), rows_cap);
@@ -101,16 +117,19 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         reinterpret_cast<unsigned long long *>(s_raw + sizeof(BatchedSmemFixed) + (size_t)rows_cap * kBRowBytes);
     // Rows sit an odd number of keys apart: the selection has a lane per row probing the same column of many rows
     // at once, and with an even stride (ld = 360: rows 16 banks apart) those probes met in two banks.
-    const size_t lds = batched_row_stride(ld);
+    const size_t lds = batched_row_stride(W);
     constexpr int kWarps = NT / kWarp;
     const int lane = lane_id(), warp = threadIdx.x >> 5;
     const bool exact = (flags & HORA_FLAG_EXACT_INT) != 0;
-    for (int64_t s = blockIdx.x; s < S; s += gridDim.x) {
+    const bool narrow = W < ld;
+    const int64_t n_seg = todo != nullptr ? (int64_t)*n_todo : S;
+    for (int64_t idx = blockIdx.x; idx < n_seg; idx += gridDim.x) {
+        const int64_t s = todo != nullptr ? (int64_t)todo[idx] : idx;
         const int64_t r0 = seg_off[s];
         const int n = (int)(seg_off[s + 1] - r0);
         const long long B = budgets[s];
         __syncthreads();
-        if (threadIdx.x == 0) sm.status = (B < 0) ? HORA_ERR_INVALID_VALUE : HORA_OK;
+        if (threadIdx.x == 0) { sm.status = (B < 0) ? HORA_ERR_INVALID_VALUE : HORA_OK; sm.redo = 0; }
         __syncthreads();
         // ---- 1: gain rows into shared memory (a warp per row) ----
         Posterior nxt = warp < n ? load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, r0 + warp) : Posterior{};
@@ -119,17 +138,26 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
             if (r + kWarps < n) nxt = load_posterior(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, r0 + r + kWarps);
             if (!p.ok && lane == 0) sm.status = HORA_ERR_INVALID_VALUE;
             const double a = p.ok ? p.a : 1.0, b = p.ok ? p.b : 1.0;
-            if (lane == 0) { rw.a[r] = a; rw.b[r] = b; rw.cap[r] = p.cap; rw.lo[r] = 0; rw.hi[r] = p.cap; }
+            const int32_t ce = p.cap < W ? p.cap : W;          // what this pass builds of the row
+            if (lane == 0) { rw.a[r] = a; rw.b[r] = b; rw.cap[r] = ce; rw.capt[r] = p.cap; rw.lo[r] = 0; rw.hi[r] = ce; }
             double carry = 1.0;
             double *out = reinterpret_cast<double *>(keys + (size_t)r * lds);
-            for (int32_t k0 = 0; k0 < ld; k0 += kWarp * E)
-                gains_chunk<E, false, false>(a, b, a + b, p.cap, ld, k0, lane, carry, out, nullptr, nullptr);
+            for (int32_t k0 = 0; k0 < W; k0 += kWarp * E)
+                gains_chunk<E, false, false>(a, b, a + b, ce, W, k0, lane, carry, out, nullptr, nullptr);
         }
         __syncthreads();
-        long long sum_cap;
-        block_exclusive_sum<NT>(threadIdx.x < n ? rw.cap[threadIdx.x] : 0, &sum_cap, sm.warp_tmp);
-        if (threadIdx.x == 0 && sm.status == HORA_OK && B > sum_cap) sm.status = HORA_ERR_INFEASIBLE;
+        long long sum_cap, sum_built;
+        {
+            long long e0, e1;
+            block_exclusive_sum2<NT>(threadIdx.x < n ? rw.capt[threadIdx.x] : 0, threadIdx.x < n ? rw.cap[threadIdx.x] : 0, e0, e1,
+                                     sum_cap, sum_built, sm.warp_tmp);
+        }
+        if (threadIdx.x == 0 && sm.status == HORA_OK) {
+            if (B > sum_cap) sm.status = HORA_ERR_INFEASIBLE;
+            else if (B > sum_built) sm.redo = 1;               // (narrow pass only: the budget reaches past its rows)
+        }
         __syncthreads();
+        const bool run = sm.status == HORA_OK && sm.redo == 0 && B > 0;   // the same in every thread
         // ---- 2: the B-th largest key, by warp 0 ----
         // The key is built from its top bits down, two bits a step: with p the bits so far, the three trial values
         // p | 1, p | 2, p | 3 (at the step's position) are counted at once — how many keys are >= each — and the
@@ -140,7 +168,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         // With at most 32 rows a lane owns ONE row and keeps its range in registers, and the steps stop as soon as no
         // row has more than one key left in the interval the bits describe (some ten steps of thirty): the keys
         // left, at most one a lane, are ranked directly.
-        if (warp == 0 && sm.status == HORA_OK && B > 0) {
+        if (warp == 0 && run) {
             const bool small = n <= kWarp;
             unsigned long long kmax = 0ull, kmin = ~0ull;
             for (int r = lane; r < n; r += kWarp) {
@@ -170,13 +198,13 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
                                          t3 = prefix | (3ull << (bit - 1));
                 int c1 = 0, c2 = 0, c3 = 0, m1 = 0, m2 = 0, m3 = 0;
                 if (small) {
-                    search3(my_rk, my_lo, my_hi, ld, t1, t2, t3, m1, m2, m3);
+                    search3(my_rk, my_lo, my_hi, W, t1, t2, t3, m1, m2, m3);
                     c1 = m1; c2 = m2; c3 = m3;
                 } else {
 #pragma unroll 1
                     for (int r = lane; r < n; r += kWarp) {
                         int a1, a2, a3;
-                        search3(keys + (size_t)r * lds, rw.lo[r], rw.hi[r], ld, t1, t2, t3, a1, a2, a3);
+                        search3(keys + (size_t)r * lds, rw.lo[r], rw.hi[r], W, t1, t2, t3, a1, a2, a3);
                         c1 += a1; c2 += a2; c3 += a3;
                         rw.band[r] = a1;                       // (scratch until the tie step)
                         rw.cnt2[r] = a2;
@@ -233,16 +261,18 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         // ---- 3: per row, keys above and equal to the threshold ----
         int my_hi = 0, my_tied = 0, my_cap = 0;
         const unsigned long long *row = keys + (size_t)threadIdx.x * lds;
-        if (threadIdx.x < n && sm.status == HORA_OK && B > 0) {
+        if (threadIdx.x < n && run) {
             my_cap = rw.cap[threadIdx.x];
             // the selection left the row's range: keys before lo are above the threshold, keys from hi on below it
             int lo = rw.lo[threadIdx.x], hi = rw.hi[threadIdx.x];
             while (lo < hi) {
                 const int mid = (lo + hi) >> 1;
-                if (HORA_AT(row, mid, ld) > lam_key) lo = mid + 1; else hi = mid;
+                if (HORA_AT(row, mid, W) > lam_key) lo = mid + 1; else hi = mid;
             }
             my_hi = lo;
-            while (my_hi + my_tied < my_cap && HORA_AT(row, my_hi + my_tied, ld) == lam_key) ++my_tied;
+            while (my_hi + my_tied < my_cap && HORA_AT(row, my_hi + my_tied, W) == lam_key) ++my_tied;
+            // narrow pass: the row takes every candidate this pass built and has more: the full pass decides
+            if (narrow && my_hi + my_tied >= W && rw.capt[threadIdx.x] > W) sm.redo = 1;
         }
         // ---- 4: ties ----
         int my_delta = 0;
@@ -263,17 +293,17 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
             const unsigned long long k_hi = (unsigned long long)__double_as_longlong(lam * (1.0 + 9.313225746154785e-10));
             const unsigned long long k_lo = (unsigned long long)__double_as_longlong(lam * (1.0 - 9.313225746154785e-10));
             int q = my_hi, has = 0, err = 0;
-            if (threadIdx.x < n && sm.status == HORA_OK && B > 0) {
+            if (threadIdx.x < n && run) {
                 const double al = alpha ? __ldg(alpha + r0 + threadIdx.x) : alpha0;
                 const double be = beta ? __ldg(beta + r0 + threadIdx.x) : beta0;
                 if (!(al >= 1.0 && be >= 1.0 && al == floor(al) && be == floor(be))) err = HORA_ERR_NOT_INTEGER;
                 else if (al + be + (double)G0 + (double)ld >= 1048576.0) err = HORA_ERR_EXACT_RANGE;
-                if (q > 0 && HORA_AT(row, q - 1, ld) <= k_hi) {
+                if (q > 0 && HORA_AT(row, q - 1, W) <= k_hi) {
                     --q;
-                    if (q > 0 && HORA_AT(row, q - 1, ld) <= k_hi) err = err ? err : HORA_ERR_EXACT_RANGE;
+                    if (q > 0 && HORA_AT(row, q - 1, W) <= k_hi) err = err ? err : HORA_ERR_EXACT_RANGE;
                 }
-                has = (q < my_cap) && (HORA_AT(row, q, ld) >= k_lo);
-                if (has && q + 1 < my_cap && HORA_AT(row, q + 1, ld) >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
+                has = (q < my_cap) && (HORA_AT(row, q, W) >= k_lo);
+                if (has && q + 1 < my_cap && HORA_AT(row, q + 1, W) >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
                 if (err) atomicCAS(&sm.status, 0, err);
             }
             if ((int)threadIdx.x < rows_cap) rw.band[threadIdx.x] = (threadIdx.x < n && has && !err) ? q + 1 : 0;
@@ -319,6 +349,10 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
             __syncthreads();
         }
         // ---- 5: outputs and summary ----
+        if (sm.redo) {                                         // (set before the barriers of step 4: the same in every thread)
+            if (threadIdx.x == 0) redo[atomicAdd(n_redo, 1u)] = (int32_t)s;
+            continue;
+        }
         const int status = sm.status;
         const bool failed = status != HORA_OK;
         if (threadIdx.x < n) {
@@ -330,7 +364,7 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
         // is g_i(Delta) (b + Delta - 1) / a  (Eq. marginal); the product loop itself took up to Delta iterations of
         // the slowest lane
         if (!failed && !(flags & HORA_FLAG_SKIP_OBJECTIVE) && threadIdx.x < n && my_delta > 0)
-            obj = 1.0 - __longlong_as_double((long long)HORA_AT(row, my_delta - 1, ld)) *
+            obj = 1.0 - __longlong_as_double((long long)HORA_AT(row, my_delta - 1, W)) *
                             (rw.b[threadIdx.x] + (double)(my_delta - 1)) / rw.a[threadIdx.x];
 #pragma unroll
         for (int d = 16; d >= 1; d >>= 1) obj += __shfl_xor_sync(kFull, obj, d);
@@ -356,7 +390,6 @@ allocate_batched_kernel(const double *__restrict__ alpha, const double *__restri
 }
 
 // ---- group offsets: exclusive scan of G over all prompts ----
-struct ScanHeader { unsigned int ticket; unsigned int pad; };
 
 __global__ void __launch_bounds__(kBThreads)
 scan_block_sums(const int32_t *__restrict__ G, int64_t N, long long *bsum, int64_t NB, ScanHeader *hdr) {
@@ -516,6 +549,7 @@ hard_first_batched_kernel(const int32_t *__restrict__ c, int32_t G0, const int32
 struct BatchedWorkspace {
     int64_t *seg_off, *budgets;
     long long *bsum;
+    int32_t *redo;                 // [S] segments the narrow pass hands to the full pass
     ScanHeader *hdr;
     int32_t *table_status;
     void *tables;
@@ -532,6 +566,7 @@ static BatchedWorkspace carve_batched(void *base, int64_t N, int64_t S) {
     w.seg_off = reinterpret_cast<int64_t *>(take(sizeof(int64_t) * (size_t)(S + 1)));
     w.budgets = reinterpret_cast<int64_t *>(take(sizeof(int64_t) * (size_t)(S > 0 ? S : 1)));
     w.bsum = reinterpret_cast<long long *>(take(sizeof(long long) * (size_t)(NB > 0 ? NB : 1)));
+    w.redo = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (size_t)(S > 0 ? S : 1)));
     w.table_status = reinterpret_cast<int32_t *>(take(sizeof(int32_t)));
     w.tables = take(kBRankReserve);
     w.bytes = o;
@@ -553,6 +588,7 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
                                                void *workspace, size_t workspace_bytes, void *stream) {
     using namespace hora;
     if (N < 0 || S < 0 || ld < 1 || G0 < 0) return HORA_ERR_INVALID_ARG;
+    if (S > 0x7FFFFFFFll) return HORA_ERR_INVALID_ARG;      // segment indices are kept in 32 bits
     if ((alpha == nullptr) != (beta == nullptr)) return HORA_ERR_INVALID_ARG;
     if (alpha == nullptr && !(alpha0 > 0.0 && beta0 > 0.0 && alpha0 < 1.0e300 && beta0 < 1.0e300))
         return HORA_ERR_INVALID_ARG;
@@ -607,21 +643,35 @@ extern "C" hora_status_t hora_allocate_batched(const double *alpha, const double
             return HORA_ERR_CUDA;
         launches += tl + 1;
     } else if (S > 0 && N > 0) {
-        // 227 KiB of shared memory per SM, 1 KiB of it reserved per resident CTA
+        // Rows longer than 256 candidates: a narrow pass over every segment, then the full pass over the segments it
+        // handed on (see the kernel).  227 KiB of shared memory per SM, 1 KiB of it reserved per resident CTA.
         const int threads = max_rows <= kWarp ? 128 : kBThreads;
-        const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(threads == 128 ? 5 : 3, (227 * 1024) / (smem + 1024)));
-        const int grid = clamp_grid(S, per_sm);
-        auto launch = [&](auto kernel) -> cudaError_t {
+        auto launch = [&](auto kernel, int cap_per_sm, int32_t W, const int32_t *todo, const unsigned int *n_todo) -> cudaError_t {
+            const size_t sm_bytes = sizeof(BatchedSmemFixed) + (size_t)rows_cap * kBRowBytes +
+                                    (size_t)max_rows * batched_row_stride(W) * sizeof(unsigned long long);
+            const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(cap_per_sm, (227 * 1024) / (sm_bytes + 1024)));
             cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
-            kernel<<<grid, threads, smem, st>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, w.seg_off,
-                                                w.budgets, S, flags, rows_cap, delta, G, info_dev);
+            kernel<<<clamp_grid(S, per_sm), threads, sm_bytes, st>>>(alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, ld, W,
+                                                                     w.seg_off, w.budgets, S, todo, n_todo, w.redo,
+                                                                     &w.hdr->n_redo, flags, rows_cap, delta, G, info_dev);
             return cudaGetLastError();
         };
-        // 8 entries a lane, as hora_gains
-        if ((threads == 128 ? launch(allocate_batched_kernel<8, 128>) : launch(allocate_batched_kernel<8, kBThreads>)) !=
-            cudaSuccess)
-            return HORA_ERR_CUDA;
+        // 8 entries a lane, as hora_gains; the narrow pass of small segments is compiled for six CTAs per SM (its
+        // 31 KB of keys leave room for them), the others for five (128 threads) or three (256)
+        cudaError_t e;
+        if (ld > kBNarrow) {
+            e = threads == 128 ? launch(allocate_batched_kernel<8, 128, 6>, 6, kBNarrow, nullptr, nullptr)
+                               : launch(allocate_batched_kernel<8, kBThreads, 3>, 3, kBNarrow, nullptr, nullptr);
+            if (e != cudaSuccess) return HORA_ERR_CUDA;
+            ++launches;
+            e = threads == 128 ? launch(allocate_batched_kernel<8, 128, 5>, 5, ld, w.redo, &w.hdr->n_redo)
+                               : launch(allocate_batched_kernel<8, kBThreads, 3>, 3, ld, w.redo, &w.hdr->n_redo);
+        } else {
+            e = threads == 128 ? launch(allocate_batched_kernel<8, 128, 5>, 5, ld, nullptr, nullptr)
+                               : launch(allocate_batched_kernel<8, kBThreads, 3>, 3, ld, nullptr, nullptr);
+        }
+        if (e != cudaSuccess) return HORA_ERR_CUDA;
         ++launches;
     }
     if (group_offsets != nullptr) {

@@ -138,7 +138,18 @@ def test_paper_shard_shape_with_per_prompt_priors(exact):
     seg = np.arange(0, N + 1, shard, dtype=np.int64)
     budgets = np.full(S, B, np.int64)
     budgets[:8] = [0, 1, 2, 15, 359, 361, 15 * 360, 15 * 360 - 1]      # the ends of the range too
+    # Rows of 360 candidates are first solved on their first 256; segments 8..15 hold one hopeless prompt among
+    # saturated ones, which takes (nearly) the whole budget — more than 256 — so these must be solved again in full;
+    # so must the two budgets above that exceed 15 * 256.
+    for s in range(8, 16):
+        sl = slice(s * shard, (s + 1) * shard)
+        c[sl] = G0
+        c[s * shard + s % shard] = 0
+        alpha[sl], beta[sl] = (3.0, 1.0) if exact else (20.0, 0.05)
+        alpha[s * shard + s % shard], beta[s * shard + s % shard] = (1.0, 3.0) if exact else (0.05, 20.0)
+        budgets[s] = 250 + 12 * (s - 8)                            # 250 .. 334: on both sides of 256
     d, G, off, infos = run_batched(alpha, beta, 1.0, 1.0, c, G0, cap, ld, seg, budgets, exact=exact)
+    assert d[8 * shard:16 * shard].max() > 256                  # (some row did take more than the narrow pass holds)
     d_o, lam_o, obj_o = oracle_segments(alpha, beta, 1.0, 1.0, c, G0, cap, seg, budgets, exact=exact)
     np.testing.assert_array_equal(d, d_o)
     np.testing.assert_array_equal(G, G0 + d_o)
