@@ -45,7 +45,7 @@ FP64_OPS_PER_CANDIDATE = 4
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
 # under profiles/ (taken at N = 131072 and scaled by the row count: the traffic is proportional to it);
 # None = no usable capture (for gains_kernel the small case leaves a large share of its output in L2).
-TRAFFIC_BYTES = {"select_level0": 2189188352, "gains_kernel": None}
+TRAFFIC_BYTES = {"select_level0": 2185488128, "gains_kernel": None}
 
 
 def measured_peak():
