@@ -911,13 +911,16 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
     __shared__ unsigned int s_hist[kBins];
     __shared__ long long s_warp[kSelThreads / kWarp];
     __shared__ unsigned long long s_ref;                         // digit route: the CTA's reference key, once it has one
-    if (*(volatile int32_t *)&hdr->status != 0) return;
+    __shared__ int s_stop;
+    // one reading of the status for the whole CTA: this kernel's own CTAs raise it when they finish, and the
+    // threads of a CTA that read it one by one could disagree on whether to stay for the barriers below
+    if (threadIdx.x == 0) s_stop = *(volatile int32_t *)&hdr->status != 0;
     const bool list = hdr->list_mode != 0;
     if (!list) {
         for (int b = threadIdx.x; b < kBins; b += kSelThreads) s_hist[b] = 0;
         if (threadIdx.x == 0) s_ref = 0ull;
-        __syncthreads();
     }
+
     bool differs = false;
     const int lane = lane_id();
     const int r = hdr->resolved;                                 // 13 or 23: the prefix lies in the key's high word
@@ -941,7 +944,9 @@ select_level1(const double *__restrict__ alpha, const double *__restrict__ beta,
         }
         return in;
     };
-    RowInputs nxt = fetch_inputs((int64_t)blockIdx.x * kSelThreads + threadIdx.x);
+    RowInputs nxt = fetch_inputs((int64_t)blockIdx.x * kSelThreads + threadIdx.x);   // (in flight across the barrier)
+    __syncthreads();
+    if (s_stop) return;
     for (int64_t base = (int64_t)blockIdx.x * kSelThreads; base < N; base += stride) {
         const int64_t row = base + threadIdx.x;
         int32_t p_hi = 0, n_eq = 0;
