@@ -67,14 +67,16 @@ def random_problem(rng, S, G0, ld, real, max_rows=40, int_priors=False):
     return alpha, beta, c, cap, seg, budgets
 
 
-@pytest.mark.parametrize("G0,ld", [(2, 24), (4, 60), (8, 130), (8, 256)])
+@pytest.mark.parametrize("G0,ld", [(2, 24), (4, 60), (8, 130), (8, 256), (8, 300)])
 @pytest.mark.parametrize("prior", ["shared", "integer", "real"])
 @pytest.mark.parametrize("max_rows", [40, 15])
 def test_batched_matches_oracle_per_segment(G0, ld, prior, max_rows):
     """shared: one Beta(1,1) prior, exact ties (solved on exact ranks, a warp per segment); integer: per-prompt
     integer priors, exact ties (a CTA per segment, keys in shared memory); real: per-prompt real priors.
     max_rows: segments of up to 40 prompts run 256 threads a CTA (a lane owns several rows in the selection where a
-    segment has more than 32), calls whose segments all have at most 32 prompts run 128 threads a CTA."""
+    segment has more than 32), calls whose segments all have at most 32 prompts run 128 threads a CTA.
+    ld = 300: rows longer than 256 candidates are solved on their first 256 first; with random caps and budgets many
+    segments are not settled by that and go through the full-width pass."""
     real = prior == "real"
     rng = np.random.default_rng(G0 * 1000 + ld + real + 7 * (max_rows != 40))
     alpha, beta, c, cap, seg, budgets = random_problem(rng, 300, G0, ld, real, max_rows=max_rows,
