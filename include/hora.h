@@ -29,6 +29,10 @@
  *   - Results are deterministic: the same inputs give bitwise identical outputs on every run.
  *   - Calls on different streams may run concurrently as long as they do not share output
  *     buffers or workspaces.
+ *   - The kernels of hora_gains, hora_allocate, hora_group_advantage, hora_token_broadcast and
+ *     hora_group_advantage_tokens are launched with the programmatic-dependent-launch attribute and wait
+ *     (griddepcontrol.wait) for the work before them in the stream before they touch memory, so stream order
+ *     holds as usual; a kernel of the caller's that follows them with the same attribute must do its own wait.
  */
 #ifndef HORA_H
 #define HORA_H
@@ -249,6 +253,8 @@ hora_status_t hora_allocate_hard_first(const int32_t *c, int32_t G0, const int32
  *                          data-dependent failures are per segment: that segment's status is set and its
  *                          delta / G are zero, other segments are unaffected
  *   workspace              device scratch, 256-byte aligned, hora_allocate_batched_workspace_bytes(N, S)
+ * Rows longer than 256 candidates are first solved on their first 256 (exact unless a prompt takes them all, or
+ * the budget exceeds them); only the segments this does not settle are solved at full width, inside the same call.
  * Limits: a segment may hold at most 256 prompts and 176 KiB of keys (prompts * ld * 8 bytes); beyond that the
  * call returns HORA_ERR_WORKSPACE and hora_allocate should be used for that problem.  With ONE prior for all
  * prompts (alpha == beta == NULL) and (G0 + 1) * ld <= 8192 neither limit applies: the candidate values are ranked
