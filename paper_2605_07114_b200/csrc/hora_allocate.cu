@@ -1422,7 +1422,8 @@ __global__ void __launch_bounds__(kSelThreads)
 exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta, double alpha0, double beta0,
               const int32_t *__restrict__ c, int32_t G0, const int32_t *__restrict__ cap, int32_t cap_scalar,
               int64_t N, int32_t ld, const double *__restrict__ gains, AllocHeader *hdr, int2 *__restrict__ rowstate,
-              int32_t *__restrict__ rowslot, unsigned long long *tkeys, unsigned long long *tcounts) {
+              int32_t *__restrict__ rowslot, unsigned long long *tkeys, unsigned long long *tcounts,
+              double *__restrict__ objrow) {
     pdl_enter();
     __shared__ long long s_warp[kSelThreads / kWarp];
     // instances per table slot, added up in the CTA first: with one type tied a million times every warp of the
@@ -1455,6 +1456,8 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
             else if (al + be + (double)G0 + (double)ld >= 1048576.0) err = err ? err : HORA_ERR_EXACT_RANGE;
             const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(gains) + row * (int64_t)ld;
             int2 st = rowstate[row];
+            const bool had_segment = st.y > st.x;             // (level 1 evaluated the row's utility only if not)
+            const int32_t p_level1 = st.x;
             if (list && st.y > st.x) st = close_segment(keys, st, lam_key, ld);   // the list route leaves segments open
             q = st.x;                                         // #keys > lambda
             if (q > 0 && __ldg(&HORA_AT(keys, q - 1, ld)) <= k_hi) {
@@ -1465,6 +1468,9 @@ exact_collect(const double *__restrict__ alpha, const double *__restrict__ beta,
             if (has && q + 1 < capi && __ldg(&HORA_AT(keys, q + 1, ld)) >= k_lo) err = err ? err : HORA_ERR_EXACT_RANGE;
             if (has && !err)
                 tkey = pack_type((unsigned long long)al + ci, (unsigned long long)be + (G0 - ci), (unsigned long long)q + 1);
+            // Level 1 left U_i(p_hi) for the rows without a key in the threshold's bin.  It stands unless the exact
+            // ranking can still move the row's Delta: a candidate inside the band, or a count that the band changed.
+            if (objrow != nullptr && !had_segment && (has || q != p_level1)) objrow[row] = -1.0;
             above += q;
         }
         // one table update per distinct type per warp
@@ -1971,9 +1977,9 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         launch_pdl(select_level0_full, grid0, kSelThreads, 0, s, cap, cap_scalar, N, ld, gains, w.hdr, w.hist_coarse);
     mark_stage(2, s);
     const int grid_rows = clamp_grid((N + kSelThreads - 1) / kSelThreads, 6);
-    // utilities of the rows whose Delta is final after level 1 are evaluated there (not in exact mode, where the
-    // tie ranking may still move a row's Delta)
-    double *objrow = (B > 0 && !exact && !(flags & HORA_FLAG_SKIP_OBJECTIVE)) ? w.objrow : nullptr;
+    // utilities of the rows without a key in the threshold's bin are evaluated by level 1, which has the row's
+    // entry at hand (in exact mode exact_collect withdraws those that the tie ranking can still move)
+    double *objrow = (B > 0 && !(flags & HORA_FLAG_SKIP_OBJECTIVE)) ? w.objrow : nullptr;
     if (B > 0) {
         if (vec2)
             launch_pdl(select_level1<true>, grid1, kSelThreads, 0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
@@ -2007,7 +2013,7 @@ extern "C" hora_status_t hora_allocate(const double *alpha, const double *beta, 
         mark_stage(4, s);
         if (exact) {
             launch_pdl(exact_collect, grid_rows, kSelThreads, 0, s, alpha, beta, alpha0, beta0, c, G0, cap, cap_scalar, N, ld,
-                       gains, w.hdr, w.rowstate, w.rowslot, w.tkeys, w.tcounts);
+                       gains, w.hdr, w.rowstate, w.rowslot, w.tkeys, w.tcounts, objrow);
             if (cudaFuncSetAttribute(exact_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kExactRankSmem) !=
                 cudaSuccess)
                 launch_failed = true;
